@@ -1,0 +1,191 @@
+/*
+ * sqn.h -- C ABI of the forward-CNN library (SqueezeNet v1.0 hot path, sm_100a).
+ *
+ * Conventions that hold for every entry point unless its comment says otherwise
+ * ---------------------------------------------------------------------------
+ *  - Pointers named in/out/weights/bias/workspace/scratch/logits/probs are DEVICE
+ *    pointers owned by the caller.  The library never allocates or frees device
+ *    memory on the caller's behalf and never keeps a pointer past the call,
+ *    except the weight/bias pointers stored inside an sqn_net the caller created.
+ *  - Activations are NHWC: [batch][row][col][layer], layers contiguous.
+ *    Kernels are OHWI: [outLayer][K][K][inLayer].  Bias is fp32 [outLayer].
+ *    (The paper, Section III-B/C, reorders data so that values of consecutive
+ *    layers at one pixel are adjacent and has every layer write its output in
+ *    that order; NHWC/OHWI is the same idea carried to all layers of a pixel.)
+ *  - dtype SQN_F32: activations and kernels fp32, fp32 FFMA accumulation.
+ *    dtype SQN_BF16: activations and kernels bf16, fp32 accumulation on the
+ *    tensor cores, bias/ReLU/pooling arithmetic in fp32, outputs rounded to
+ *    bf16 (round to nearest even).  Logits and probabilities are always fp32.
+ *  - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is
+ *    the legacy default stream).  No entry point synchronises except sqn_check.
+ *  - Every argument is validated on the host before anything is launched.  On
+ *    error nothing is launched and a negative sqn_status is returned.  There is
+ *    no CPU fallback and no silent slow path: a shape the selected dtype path
+ *    cannot run returns SQN_ERR_UNSUPPORTED.
+ *  - in and out must not overlap.  All base pointers must be 16-byte aligned.
+ */
+#ifndef SQN_H
+#define SQN_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SQN_OK = 0,
+    SQN_ERR_BADARG = -1,       /* null pointer, non-positive size, window larger than padded input */
+    SQN_ERR_UNSUPPORTED = -2,  /* valid request the selected dtype path does not implement */
+    SQN_ERR_ALIGN = -3,        /* pointer or layer count breaks an alignment rule */
+    SQN_ERR_CUDA = -4,         /* a CUDA runtime/driver call failed */
+    SQN_ERR_TIMEOUT = -5,      /* a bounded device-side wait ran out (reported by sqn_check) */
+    SQN_ERR_WORKSPACE = -6     /* workspace missing or too small */
+} sqn_status;
+
+typedef enum { SQN_F32 = 0, SQN_BF16 = 1 } sqn_dtype;
+
+/*
+ * Convolution layer (paper Section II; Section III Fig. 2 prose; Eq. 1):
+ *   out[n][h][w][m] = max(0, bias[m] + sum_{i,j<K, c<numInputLayers}
+ *                              in[n][h*S+i-pad][w*S+j-pad][c] * weights[m][i][j][c])
+ * with zero padding, output extent (H + 2*pad - K)/S + 1 in each direction
+ * (integer division).  fp32, ReLU on, dense output (all numOutputLayers layers),
+ * legacy default stream.
+ *   in       [batch][H][W][numInputLayers]
+ *   weights  [numOutputLayers][K][K][numInputLayers]
+ *   bias     [numOutputLayers] fp32
+ *   out      [batch][outH][outW][numOutputLayers]
+ * Any K>=1, S>=1, pad>=0 and any layer counts are accepted.
+ */
+int conv_forward(const void* in, const void* weights, const void* bias, void* out,
+                 int numInputLayers, int numOutputLayers, int H, int W, int K, int S, int pad, int batch);
+
+/*
+ * Options for conv_forward_ex.
+ *   dtype          SQN_F32 or SQN_BF16
+ *   relu           non-zero: max(0, .) after the bias; zero: identity
+ *   out_c_offset,
+ *   out_c_total    the layer writes layers [out_c_offset, out_c_offset+numOutputLayers) of an
+ *                  output tensor that has out_c_total layers per pixel (a fire layer's two
+ *                  expands write their halves of one tensor this way).  out_c_total = 0 means
+ *                  dense: offset 0, total numOutputLayers.
+ *   stream         cudaStream_t
+ *   workspace,
+ *   workspace_bytes  device scratch, needed only when conv_workspace_bytes reports > 0
+ */
+typedef struct {
+    int dtype;
+    int relu;
+    int out_c_offset;
+    int out_c_total;
+    void* stream;
+    void* workspace;
+    size_t workspace_bytes;
+} sqn_conv_opts;
+
+/*
+ * Same operation as conv_forward with every choice exposed.  opts may be NULL
+ * (fp32, ReLU, dense, default stream).
+ * SQN_BF16 restrictions (else SQN_ERR_UNSUPPORTED / SQN_ERR_ALIGN):
+ *   - S == 1, 2*pad == K-1 or pad == 0, numInputLayers a multiple of 16,
+ *     numOutputLayers a multiple of 8 (16 when <= 256 is not met see below),
+ *     out_c_offset and out_c_total multiples of 8; or
+ *   - the stem shape K=7, S=2, pad=0, numInputLayers=3, which needs a workspace
+ *     (conv_workspace_bytes) for its repacked input and kernels.
+ */
+int conv_forward_ex(const void* in, const void* weights, const void* bias, void* out,
+                    int numInputLayers, int numOutputLayers, int H, int W, int K, int S, int pad, int batch,
+                    const sqn_conv_opts* opts);
+
+/* Bytes of workspace conv_forward_ex needs for this shape and dtype (0 for most). */
+int conv_workspace_bytes(int numInputLayers, int numOutputLayers, int H, int W, int K, int S, int pad, int batch,
+                         int dtype, size_t* bytes);
+
+/*
+ * Fire layer (paper Section II: one squeeze layer feeding two expand layers):
+ *   sq  = relu(conv1x1(in,  w_sq, b_sq))            [batch][H][W][s]     -> squeeze_scratch
+ *   out[..., 0:e1]      = relu(conv1x1(sq, w_e1, b_e1))
+ *   out[..., e1:e1+e3]  = relu(conv3x3 pad 1 (sq, w_e3, b_e3))
+ * Both expands store straight into their slice of out [batch][H][W][e1+e3];
+ * there is no concatenation pass.  squeeze_scratch must hold batch*H*W*s
+ * elements of the chosen dtype and must not overlap in or out.
+ * SQN_BF16: Cin, s multiples of 16; e1, e3 multiples of 16.
+ */
+int fire_forward(const void* in, const void* w_sq, const void* b_sq, const void* w_e1, const void* b_e1,
+                 const void* w_e3, const void* b_e3, void* squeeze_scratch, void* out,
+                 int Cin, int s, int e1, int e3, int H, int W, int batch, int dtype, void* stream);
+
+/*
+ * Max pooling 3x3, stride 2, no padding (paper Section III-E):
+ *   out[n][h][w][c] = max_{i,j<3} in[n][2h+i][2w+j][c],  out extent (H-3)/2+1.
+ */
+int maxpool3x3s2_forward(const void* in, void* out, int C, int H, int W, int batch, int dtype, void* stream);
+
+/*
+ * Global average pooling followed by softmax (paper Section III-E):
+ *   logits[n][c] = mean over H*W of in[n][.][.][c]        (fp32)
+ *   probs[n][c]  = exp(logits[n][c] - max_c) / sum_c exp(logits[n][c] - max_c)
+ * in has dtype `dtype`; logits and probs are fp32 [batch][C]; probs may be NULL.
+ * C <= 8192.
+ */
+int avgpool_softmax_forward(const void* in, void* logits_f32, void* probs_f32, int C, int H, int W, int batch,
+                            int dtype, void* stream);
+
+/*
+ * SqueezeNet v1.0 forward (paper Section II: two convolutional layers, eight
+ * fire layers, pooling, softmax, 1000 classes) on 227x227x3 images:
+ *   conv1 96x7x7/2 -> maxpool -> fire2,3 (16,64,64) -> fire4 (32,128,128) -> maxpool
+ *   -> fire5 (32,128,128) -> fire6,7 (48,192,192) -> fire8 (64,256,256) -> maxpool
+ *   -> fire9 (64,256,256) -> conv10 1000x1x1 -> global average -> softmax,
+ * ReLU after every convolution (conv10 included).
+ *
+ * squeezenet_create: weights26/bias26 are host arrays of 26 device pointers in
+ *   network order (conv1; fireN squeeze, expand1x1, expand3x3 for N=2..9; conv10),
+ *   kernels OHWI in `dtype`, bias fp32.  The net stores the pointers (the caller
+ *   keeps the memory alive) and host-side launch plans; it holds no device memory.
+ * squeezenet_workspace_bytes: device scratch one forward of `batch` images needs.
+ * squeezenet_forward: in_nhwc [batch][227][227][3] in the net's dtype;
+ *   logits_f32, probs_f32 fp32 [batch][1000] (probs may be NULL);
+ *   batch <= max_batch.  Returns after enqueuing all launches on `stream`.
+ * squeezenet_layer_output: after a forward with the same workspace and batch,
+ *   gives the device address, layer count and extent of a named intermediate
+ *   ("conv1", "pool1", "fire2_sq", "fire2", ..., "pool8", "fire9", "conv10");
+ *   the data is in the net's dtype, NHWC, valid until the next forward.
+ */
+typedef struct sqn_net sqn_net;
+int squeezenet_create(sqn_net** net, const void* const* weights26, const void* const* bias26, int dtype,
+                      int max_batch);
+int squeezenet_workspace_bytes(const sqn_net* net, int batch, size_t* bytes);
+int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logits_f32, void* probs_f32, void* workspace,
+                       int batch, void* stream);
+int squeezenet_layer_output(const sqn_net* net, const char* name, void* workspace, int batch, void** ptr, int* C,
+                            int* H, int* W);
+int squeezenet_destroy(sqn_net* net);
+
+/*
+ * Host-side layout helpers (the paper's offline reordering of the model file,
+ * Section III-C).  src and dst are HOST pointers.  dtype selects the element
+ * type of the reordered side (fp32, or bf16 rounded to nearest even).
+ */
+int sqn_pack_weights_oihw_to_ohwi(const float* src, void* dst, int O, int I, int K, int dtype);
+int sqn_pack_nchw_to_nhwc(const float* src, void* dst, int N, int C, int H, int W, int dtype);
+int sqn_unpack_nhwc_to_nchw(const void* src, float* dst, int N, int C, int H, int W, int dtype);
+
+/*
+ * Synchronises `stream` and returns SQN_OK, SQN_ERR_CUDA, or the error a kernel
+ * recorded (SQN_ERR_TIMEOUT when a bounded device-side wait ran out).  The
+ * recorded error is cleared by the call.
+ */
+int sqn_check(void* stream);
+
+/* Static, human-readable name of a status code. */
+const char* sqn_status_string(int status);
+
+/* Number of kernel launches the library has enqueued since it was loaded (host counter). */
+unsigned long long sqn_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SQN_H */

@@ -1,0 +1,403 @@
+// C-ABI entry points: argument validation, dispatch, the fire layer and the SqueezeNet v1.0
+// forward composition, host-side layout helpers.  No device memory is allocated here.
+#include <atomic>
+#include <cmath>
+#include <cstring>
+#include <mutex>
+#include <string>
+#include <vector>
+
+#include "sqn_internal.h"
+
+namespace sqn {
+
+static std::atomic<unsigned long long> g_launches{0};
+void note_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+
+__device__ int g_device_status;   // written by kernels whose bounded waits run out
+
+int* device_status_word()
+{
+    static std::mutex mu;
+    static int* ptrs[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!ptrs[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_device_status) != cudaSuccess) return nullptr;
+        ptrs[dev] = static_cast<int*>(p);
+    }
+    return ptrs[dev];
+}
+
+namespace {
+
+inline size_t esize(int dtype) { return dtype == SQN_BF16 ? 2 : 4; }
+inline int out_extent(int H, int K, int S, int pad) { return (H + 2 * pad - K) / S + 1; }
+
+inline uint16_t f32_to_bf16_rne(float f)
+{
+    uint32_t u;
+    std::memcpy(&u, &f, 4);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x0040u);   // NaN stays NaN
+    u += 0x7fffu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+inline float bf16_to_f32(uint16_t h)
+{
+    uint32_t u = (uint32_t)h << 16;
+    float f;
+    std::memcpy(&f, &u, 4);
+    return f;
+}
+
+// Validates one convolution request and fills the descriptor.
+int make_conv_desc(const void* in, const void* w, const void* bias, void* out, int Cin, int Cout, int H, int W, int K,
+                   int S, int pad, int batch, int relu, int c_off, int c_total, ConvDesc* d)
+{
+    if (!in || !w || !bias || !out) return SQN_ERR_BADARG;
+    if (Cin <= 0 || Cout <= 0 || H <= 0 || W <= 0 || K <= 0 || S <= 0 || pad < 0 || batch <= 0) return SQN_ERR_BADARG;
+    if (H + 2 * pad < K || W + 2 * pad < K) return SQN_ERR_BADARG;
+    if (c_total == 0) { c_total = Cout; if (c_off != 0) return SQN_ERR_BADARG; }
+    if (c_off < 0 || c_off + Cout > c_total) return SQN_ERR_BADARG;
+    if (!aligned16(in) || !aligned16(w) || !aligned16(out) || (reinterpret_cast<uintptr_t>(bias) & 3u))
+        return SQN_ERR_ALIGN;
+    d->in = in; d->w = w; d->bias = static_cast<const float*>(bias); d->out = out;
+    d->N = batch; d->Cin = Cin; d->H = H; d->W = W; d->Cout = Cout; d->K = K; d->S = S; d->pad = pad;
+    d->OH = out_extent(H, K, S, pad); d->OW = out_extent(W, K, S, pad);
+    d->out_c_offset = c_off; d->out_c_total = c_total; d->relu = relu ? 1 : 0;
+    return SQN_OK;
+}
+
+inline bool is_stem_shape(const ConvDesc& d) { return d.K == 7 && d.S == 2 && d.pad == 0 && d.Cin == 3; }
+
+int run_conv(const ConvDesc& d, int dtype, void* ws, size_t ws_bytes, cudaStream_t stream)
+{
+    if (dtype == SQN_F32) return launch_conv_f32(d, stream);
+    if (dtype != SQN_BF16) return SQN_ERR_BADARG;
+    if (is_stem_shape(d)) return launch_stem_bf16(d, ws, ws_bytes, stream);
+    const int rc = conv_bf16_supported(d);
+    if (rc != SQN_OK) return rc;
+    return launch_conv_bf16(d, stream);
+}
+
+}  // namespace
+}  // namespace sqn
+
+using namespace sqn;
+
+// ------------------------------------------------------------------------- convolution
+extern "C" int conv_forward_ex(const void* in, const void* weights, const void* bias, void* out, int numInputLayers,
+                               int numOutputLayers, int H, int W, int K, int S, int pad, int batch,
+                               const sqn_conv_opts* opts)
+{
+    sqn_conv_opts o;
+    if (opts) o = *opts;
+    else { std::memset(&o, 0, sizeof(o)); o.dtype = SQN_F32; o.relu = 1; }
+    if (o.dtype != SQN_F32 && o.dtype != SQN_BF16) return SQN_ERR_BADARG;
+    ConvDesc d;
+    const int rc = make_conv_desc(in, weights, bias, out, numInputLayers, numOutputLayers, H, W, K, S, pad, batch,
+                                  o.relu, o.out_c_offset, o.out_c_total, &d);
+    if (rc != SQN_OK) return rc;
+    return run_conv(d, o.dtype, o.workspace, o.workspace_bytes, static_cast<cudaStream_t>(o.stream));
+}
+
+extern "C" int conv_forward(const void* in, const void* weights, const void* bias, void* out, int numInputLayers,
+                            int numOutputLayers, int H, int W, int K, int S, int pad, int batch)
+{
+    return conv_forward_ex(in, weights, bias, out, numInputLayers, numOutputLayers, H, W, K, S, pad, batch, nullptr);
+}
+
+extern "C" int conv_workspace_bytes(int Cin, int Cout, int H, int W, int K, int S, int pad, int batch, int dtype,
+                                    size_t* bytes)
+{
+    if (!bytes || Cin <= 0 || Cout <= 0 || H <= 0 || W <= 0 || K <= 0 || S <= 0 || pad < 0 || batch <= 0)
+        return SQN_ERR_BADARG;
+    if (dtype != SQN_F32 && dtype != SQN_BF16) return SQN_ERR_BADARG;
+    *bytes = 0;
+    if (dtype == SQN_BF16 && K == 7 && S == 2 && pad == 0 && Cin == 3) *bytes = stem_bf16_workspace_bytes(batch, H, W, Cout);
+    return SQN_OK;
+}
+
+// ------------------------------------------------------------------------------- fire
+extern "C" int fire_forward(const void* in, const void* w_sq, const void* b_sq, const void* w_e1, const void* b_e1,
+                            const void* w_e3, const void* b_e3, void* squeeze_scratch, void* out, int Cin, int s,
+                            int e1, int e3, int H, int W, int batch, int dtype, void* stream)
+{
+    if (dtype != SQN_F32 && dtype != SQN_BF16) return SQN_ERR_BADARG;
+    if (!squeeze_scratch) return SQN_ERR_BADARG;
+    if (e1 <= 0 || e3 <= 0) return SQN_ERR_BADARG;
+    ConvDesc dsq, d1, d3;
+    int rc = make_conv_desc(in, w_sq, b_sq, squeeze_scratch, Cin, s, H, W, 1, 1, 0, batch, 1, 0, 0, &dsq);
+    if (rc != SQN_OK) return rc;
+    rc = make_conv_desc(squeeze_scratch, w_e1, b_e1, out, s, e1, H, W, 1, 1, 0, batch, 1, 0, e1 + e3, &d1);
+    if (rc != SQN_OK) return rc;
+    rc = make_conv_desc(squeeze_scratch, w_e3, b_e3, out, s, e3, H, W, 3, 1, 1, batch, 1, e1, e1 + e3, &d3);
+    if (rc != SQN_OK) return rc;
+    if (dtype == SQN_BF16) {
+        if ((rc = conv_bf16_supported(dsq)) != SQN_OK) return rc;
+        if ((rc = conv_bf16_supported(d1)) != SQN_OK) return rc;
+        if ((rc = conv_bf16_supported(d3)) != SQN_OK) return rc;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if ((rc = run_conv(dsq, dtype, nullptr, 0, st)) != SQN_OK) return rc;
+    if ((rc = run_conv(d1, dtype, nullptr, 0, st)) != SQN_OK) return rc;
+    return run_conv(d3, dtype, nullptr, 0, st);
+}
+
+// ---------------------------------------------------------------------------- pooling
+extern "C" int maxpool3x3s2_forward(const void* in, void* out, int C, int H, int W, int batch, int dtype, void* stream)
+{
+    if (!in || !out || C <= 0 || H < 3 || W < 3 || batch <= 0) return SQN_ERR_BADARG;
+    if (dtype != SQN_F32 && dtype != SQN_BF16) return SQN_ERR_BADARG;
+    if (!aligned16(in) || !aligned16(out)) return SQN_ERR_ALIGN;
+    return launch_maxpool3x3s2(in, out, C, H, W, batch, dtype, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int avgpool_softmax_forward(const void* in, void* logits_f32, void* probs_f32, int C, int H, int W,
+                                       int batch, int dtype, void* stream)
+{
+    if (!in || !logits_f32 || C <= 0 || H <= 0 || W <= 0 || batch <= 0) return SQN_ERR_BADARG;
+    if (dtype != SQN_F32 && dtype != SQN_BF16) return SQN_ERR_BADARG;
+    if (C > 8192) return SQN_ERR_UNSUPPORTED;
+    return launch_avgpool_softmax(in, static_cast<float*>(logits_f32), static_cast<float*>(probs_f32), C, H, W, batch,
+                                  dtype, static_cast<cudaStream_t>(stream));
+}
+
+// ------------------------------------------------------------------ SqueezeNet v1.0
+namespace {
+
+struct FireSpec { const char* name; int cin, s, e, hw; bool pool_after; };
+const FireSpec kFire[8] = {
+    {"fire2", 96, 16, 64, 55, false},  {"fire3", 128, 16, 64, 55, false}, {"fire4", 128, 32, 128, 55, true},
+    {"fire5", 256, 32, 128, 27, false}, {"fire6", 256, 48, 192, 27, false}, {"fire7", 384, 48, 192, 27, false},
+    {"fire8", 384, 64, 256, 27, true},  {"fire9", 512, 64, 256, 13, false}};
+
+struct Slot { std::string name; int C, H, W; size_t offset; };   // offset in bytes for batch 1 element counts below
+
+}  // namespace
+
+struct sqn_net {
+    const void* w[26];
+    const float* b[26];
+    int dtype;
+    int max_batch;
+    std::vector<Slot> slots;   // per-image element counts; byte offsets are computed per batch
+};
+
+namespace {
+
+constexpr int IMG = 227;
+
+void build_slots(sqn_net* net)
+{
+    auto add = [&](const std::string& n, int C, int H, int W) { net->slots.push_back({n, C, H, W, 0}); };
+    add("conv1", 96, 111, 111);
+    add("pool1", 96, 55, 55);
+    for (const FireSpec& f : kFire) {
+        add(std::string(f.name) + "_sq", f.s, f.hw, f.hw);
+        add(f.name, 2 * f.e, f.hw, f.hw);
+        if (f.pool_after) add(std::string("pool") + (f.name + 4), 2 * f.e, (f.hw - 3) / 2 + 1, (f.hw - 3) / 2 + 1);
+    }
+    add("conv10", 1000, 13, 13);
+}
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Byte offset of every slot inside the workspace for a given batch; returns total bytes.
+size_t layout(const sqn_net* net, int batch, std::vector<size_t>* offs, size_t* stem_off)
+{
+    size_t cur = 0;
+    const size_t es = esize(net->dtype);
+    if (offs) offs->clear();
+    for (const Slot& s : net->slots) {
+        if (offs) offs->push_back(cur);
+        cur = align_up(cur + (size_t)batch * s.C * s.H * s.W * es, 1024);
+    }
+    if (stem_off) *stem_off = cur;
+    if (net->dtype == SQN_BF16) cur = align_up(cur + stem_bf16_workspace_bytes(batch, IMG, IMG, 96), 1024);
+    return cur;
+}
+
+int find_slot(const sqn_net* net, const char* name)
+{
+    for (size_t i = 0; i < net->slots.size(); ++i)
+        if (net->slots[i].name == name) return (int)i;
+    return -1;
+}
+
+}  // namespace
+
+extern "C" int squeezenet_create(sqn_net** net, const void* const* weights26, const void* const* bias26, int dtype,
+                                 int max_batch)
+{
+    if (!net || !weights26 || !bias26 || max_batch <= 0) return SQN_ERR_BADARG;
+    if (dtype != SQN_F32 && dtype != SQN_BF16) return SQN_ERR_BADARG;
+    for (int i = 0; i < 26; ++i) {
+        if (!weights26[i] || !bias26[i]) return SQN_ERR_BADARG;
+        if (!aligned16(weights26[i]) || (reinterpret_cast<uintptr_t>(bias26[i]) & 3u)) return SQN_ERR_ALIGN;
+    }
+    sqn_net* n = new (std::nothrow) sqn_net();
+    if (!n) return SQN_ERR_BADARG;
+    for (int i = 0; i < 26; ++i) { n->w[i] = weights26[i]; n->b[i] = static_cast<const float*>(bias26[i]); }
+    n->dtype = dtype;
+    n->max_batch = max_batch;
+    build_slots(n);
+    *net = n;
+    return SQN_OK;
+}
+
+extern "C" int squeezenet_destroy(sqn_net* net)
+{
+    delete net;
+    return SQN_OK;
+}
+
+extern "C" int squeezenet_workspace_bytes(const sqn_net* net, int batch, size_t* bytes)
+{
+    if (!net || !bytes || batch <= 0 || batch > net->max_batch) return SQN_ERR_BADARG;
+    *bytes = layout(net, batch, nullptr, nullptr);
+    return SQN_OK;
+}
+
+extern "C" int squeezenet_layer_output(const sqn_net* net, const char* name, void* workspace, int batch, void** ptr,
+                                       int* C, int* H, int* W)
+{
+    if (!net || !name || !workspace || !ptr || batch <= 0 || batch > net->max_batch) return SQN_ERR_BADARG;
+    const int i = find_slot(net, name);
+    if (i < 0) return SQN_ERR_BADARG;
+    std::vector<size_t> offs;
+    layout(net, batch, &offs, nullptr);
+    *ptr = static_cast<char*>(workspace) + offs[i];
+    if (C) *C = net->slots[i].C;
+    if (H) *H = net->slots[i].H;
+    if (W) *W = net->slots[i].W;
+    return SQN_OK;
+}
+
+extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logits_f32, void* probs_f32,
+                                  void* workspace, int batch, void* stream)
+{
+    if (!net || !in_nhwc || !logits_f32 || batch <= 0 || batch > net->max_batch) return SQN_ERR_BADARG;
+    if (!workspace) return SQN_ERR_WORKSPACE;
+    if (!aligned16(in_nhwc) || !aligned16(workspace)) return SQN_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int dt = net->dtype;
+    std::vector<size_t> offs;
+    size_t stem_off = 0;
+    const size_t total = layout(net, batch, &offs, &stem_off);
+    char* ws = static_cast<char*>(workspace);
+    auto buf = [&](const std::string& name) -> void* { return ws + offs[find_slot(net, name.c_str())]; };
+
+    int rc;
+    ConvDesc d;
+    // conv1 7x7/2 + ReLU, then max-pool
+    rc = make_conv_desc(in_nhwc, net->w[0], net->b[0], buf("conv1"), 3, 96, IMG, IMG, 7, 2, 0, batch, 1, 0, 0, &d);
+    if (rc != SQN_OK) return rc;
+    if ((rc = run_conv(d, dt, ws + stem_off, total - stem_off, st)) != SQN_OK) return rc;
+    if ((rc = launch_maxpool3x3s2(buf("conv1"), buf("pool1"), 96, 111, 111, batch, dt, st)) != SQN_OK) return rc;
+
+    const void* cur = buf("pool1");
+    for (int i = 0; i < 8; ++i) {
+        const FireSpec& f = kFire[i];
+        void* sq = buf(std::string(f.name) + "_sq");
+        void* out = buf(f.name);
+        rc = fire_forward(cur, net->w[1 + 3 * i], net->b[1 + 3 * i], net->w[2 + 3 * i], net->b[2 + 3 * i],
+                          net->w[3 + 3 * i], net->b[3 + 3 * i], sq, out, f.cin, f.s, f.e, f.e, f.hw, f.hw, batch, dt,
+                          stream);
+        if (rc != SQN_OK) return rc;
+        cur = out;
+        if (f.pool_after) {
+            void* po = buf(std::string("pool") + (f.name + 4));
+            if ((rc = launch_maxpool3x3s2(cur, po, 2 * f.e, f.hw, f.hw, batch, dt, st)) != SQN_OK) return rc;
+            cur = po;
+        }
+    }
+    // conv10 1x1 + ReLU, global average, softmax
+    rc = make_conv_desc(cur, net->w[25], net->b[25], buf("conv10"), 512, 1000, 13, 13, 1, 1, 0, batch, 1, 0, 0, &d);
+    if (rc != SQN_OK) return rc;
+    if ((rc = run_conv(d, dt, nullptr, 0, st)) != SQN_OK) return rc;
+    return launch_avgpool_softmax(buf("conv10"), static_cast<float*>(logits_f32), static_cast<float*>(probs_f32), 1000,
+                                  13, 13, batch, dt, st);
+}
+
+// ---------------------------------------------------------------- host layout helpers
+extern "C" int sqn_pack_weights_oihw_to_ohwi(const float* src, void* dst, int O, int I, int K, int dtype)
+{
+    if (!src || !dst || O <= 0 || I <= 0 || K <= 0) return SQN_ERR_BADARG;
+    if (dtype != SQN_F32 && dtype != SQN_BF16) return SQN_ERR_BADARG;
+    for (int o = 0; o < O; ++o)
+        for (int i = 0; i < I; ++i)
+            for (int kh = 0; kh < K; ++kh)
+                for (int kw = 0; kw < K; ++kw) {
+                    const float v = src[(((size_t)o * I + i) * K + kh) * K + kw];
+                    const size_t di = (((size_t)o * K + kh) * K + kw) * I + i;
+                    if (dtype == SQN_F32) static_cast<float*>(dst)[di] = v;
+                    else static_cast<uint16_t*>(dst)[di] = f32_to_bf16_rne(v);
+                }
+    return SQN_OK;
+}
+
+extern "C" int sqn_pack_nchw_to_nhwc(const float* src, void* dst, int N, int C, int H, int W, int dtype)
+{
+    if (!src || !dst || N <= 0 || C <= 0 || H <= 0 || W <= 0) return SQN_ERR_BADARG;
+    if (dtype != SQN_F32 && dtype != SQN_BF16) return SQN_ERR_BADARG;
+    for (int n = 0; n < N; ++n)
+        for (int c = 0; c < C; ++c)
+            for (int h = 0; h < H; ++h)
+                for (int w = 0; w < W; ++w) {
+                    const float v = src[(((size_t)n * C + c) * H + h) * W + w];
+                    const size_t di = (((size_t)n * H + h) * W + w) * C + c;
+                    if (dtype == SQN_F32) static_cast<float*>(dst)[di] = v;
+                    else static_cast<uint16_t*>(dst)[di] = f32_to_bf16_rne(v);
+                }
+    return SQN_OK;
+}
+
+extern "C" int sqn_unpack_nhwc_to_nchw(const void* src, float* dst, int N, int C, int H, int W, int dtype)
+{
+    if (!src || !dst || N <= 0 || C <= 0 || H <= 0 || W <= 0) return SQN_ERR_BADARG;
+    if (dtype != SQN_F32 && dtype != SQN_BF16) return SQN_ERR_BADARG;
+    for (int n = 0; n < N; ++n)
+        for (int h = 0; h < H; ++h)
+            for (int w = 0; w < W; ++w)
+                for (int c = 0; c < C; ++c) {
+                    const size_t si = (((size_t)n * H + h) * W + w) * C + c;
+                    const float v = dtype == SQN_F32 ? static_cast<const float*>(src)[si]
+                                                     : bf16_to_f32(static_cast<const uint16_t*>(src)[si]);
+                    dst[(((size_t)n * C + c) * H + h) * W + w] = v;
+                }
+    return SQN_OK;
+}
+
+// ------------------------------------------------------------------------------ misc
+extern "C" int sqn_check(void* stream)
+{
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return SQN_ERR_CUDA;
+    int* word = device_status_word();
+    if (!word) return SQN_ERR_CUDA;
+    int v = 0;
+    if (cudaMemcpy(&v, word, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return SQN_ERR_CUDA;
+    if (v != 0) {
+        const int zero = 0;
+        if (cudaMemcpy(word, &zero, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) return SQN_ERR_CUDA;
+    }
+    return v;
+}
+
+extern "C" const char* sqn_status_string(int status)
+{
+    switch (status) {
+        case SQN_OK: return "ok";
+        case SQN_ERR_BADARG: return "bad argument";
+        case SQN_ERR_UNSUPPORTED: return "unsupported shape for this dtype path";
+        case SQN_ERR_ALIGN: return "alignment rule violated";
+        case SQN_ERR_CUDA: return "CUDA call failed";
+        case SQN_ERR_TIMEOUT: return "device-side wait timed out";
+        case SQN_ERR_WORKSPACE: return "workspace missing or too small";
+        default: return "unknown status";
+    }
+}
+
+extern "C" unsigned long long sqn_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

@@ -1,0 +1,196 @@
+// Pooling layers and the classifier head (paper Section III-E), NHWC.
+//   max pooling 3x3 / stride 2, no padding: one thread per output pixel and group of layers,
+//   128-bit loads and stores along the layer dimension (memory bound: one read, one write);
+//   global average pooling + softmax: one block per image.
+#include <cuda_bf16.h>
+
+#include "sqn_internal.h"
+
+namespace sqn {
+namespace {
+
+__device__ __forceinline__ float4 max4(float4 a, float4 b)
+{
+    return make_float4(fmaxf(a.x, b.x), fmaxf(a.y, b.y), fmaxf(a.z, b.z), fmaxf(a.w, b.w));
+}
+
+// fp32, C % 4 == 0: each thread produces 4 layers of one output pixel.
+__global__ void maxpool_f32_v4(const float* __restrict__ in, float* __restrict__ out, int C4, int H, int W, int OH,
+                               int OW, long long total)
+{
+    const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if (idx >= total) return;
+    const int c4 = (int)(idx % C4);
+    long long r = idx / C4;
+    const int ow = (int)(r % OW); r /= OW;
+    const int oh = (int)(r % OH);
+    const long long n = r / OH;
+    const float4* src = reinterpret_cast<const float4*>(in) + ((n * H + 2 * oh) * W + 2 * ow) * C4 + c4;
+    float4 m = __ldg(src);
+#pragma unroll
+    for (int i = 0; i < 3; ++i)
+#pragma unroll
+        for (int j = 0; j < 3; ++j) m = max4(m, __ldg(src + ((long long)i * W + j) * C4));
+    reinterpret_cast<float4*>(out)[idx] = m;
+}
+
+// fp32, any C: one thread per output element.
+__global__ void maxpool_f32_s(const float* __restrict__ in, float* __restrict__ out, int C, int H, int W, int OH,
+                              int OW, long long total)
+{
+    const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if (idx >= total) return;
+    const int c = (int)(idx % C);
+    long long r = idx / C;
+    const int ow = (int)(r % OW); r /= OW;
+    const int oh = (int)(r % OH);
+    const long long n = r / OH;
+    const float* src = in + ((n * H + 2 * oh) * W + 2 * ow) * C + c;
+    float m = __ldg(src);
+    for (int i = 0; i < 3; ++i)
+        for (int j = 0; j < 3; ++j) m = fmaxf(m, __ldg(src + ((long long)i * W + j) * C));
+    out[idx] = m;
+}
+
+__device__ __forceinline__ uint32_t bmax2(uint32_t a, uint32_t b)
+{
+    __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162*>(&a);
+    __nv_bfloat162 y = *reinterpret_cast<__nv_bfloat162*>(&b);
+    __nv_bfloat162 m = __hmax2(x, y);
+    return *reinterpret_cast<uint32_t*>(&m);
+}
+
+// bf16, C % 8 == 0: each thread produces 8 layers (16 bytes) of one output pixel.
+__global__ void maxpool_bf16_v8(const uint4* __restrict__ in, uint4* __restrict__ out, int C8, int H, int W, int OH,
+                                int OW, long long total)
+{
+    const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if (idx >= total) return;
+    const int c8 = (int)(idx % C8);
+    long long r = idx / C8;
+    const int ow = (int)(r % OW); r /= OW;
+    const int oh = (int)(r % OH);
+    const long long n = r / OH;
+    const uint4* src = in + ((n * H + 2 * oh) * W + 2 * ow) * C8 + c8;
+    uint4 m = __ldg(src);
+#pragma unroll
+    for (int i = 0; i < 3; ++i)
+#pragma unroll
+        for (int j = 0; j < 3; ++j) {
+            const uint4 v = __ldg(src + ((long long)i * W + j) * C8);
+            m.x = bmax2(m.x, v.x); m.y = bmax2(m.y, v.y); m.z = bmax2(m.z, v.z); m.w = bmax2(m.w, v.w);
+        }
+    out[idx] = m;
+}
+
+__global__ void maxpool_bf16_s(const __nv_bfloat16* __restrict__ in, __nv_bfloat16* __restrict__ out, int C, int H,
+                               int W, int OH, int OW, long long total)
+{
+    const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if (idx >= total) return;
+    const int c = (int)(idx % C);
+    long long r = idx / C;
+    const int ow = (int)(r % OW); r /= OW;
+    const int oh = (int)(r % OH);
+    const long long n = r / OH;
+    const __nv_bfloat16* src = in + ((n * H + 2 * oh) * W + 2 * ow) * C + c;
+    float m = __bfloat162float(src[0]);
+    for (int i = 0; i < 3; ++i)
+        for (int j = 0; j < 3; ++j) m = fmaxf(m, __bfloat162float(src[((long long)i * W + j) * C]));
+    out[idx] = __float2bfloat16(m);
+}
+
+// Global average + softmax.  One block per image; logits kept in shared memory.
+template <bool BF16>
+__global__ void __launch_bounds__(256) avgpool_softmax_kernel(const void* __restrict__ in_, float* __restrict__ logits,
+                                                               float* __restrict__ probs, int C, int HW)
+{
+    extern __shared__ float z[];          // [C]
+    __shared__ float red[32];
+    const int n = blockIdx.x;
+    const float inv = 1.0f / (float)HW;
+    for (int c = threadIdx.x; c < C; c += blockDim.x) {
+        float s = 0.f;
+        if (BF16) {
+            const __nv_bfloat16* src = static_cast<const __nv_bfloat16*>(in_) + (size_t)n * HW * C + c;
+            for (int p = 0; p < HW; ++p) s += __bfloat162float(src[(size_t)p * C]);
+        } else {
+            const float* src = static_cast<const float*>(in_) + (size_t)n * HW * C + c;
+            for (int p = 0; p < HW; ++p) s += __ldg(src + (size_t)p * C);
+        }
+        s *= inv;
+        z[c] = s;
+        logits[(size_t)n * C + c] = s;
+    }
+    __syncthreads();
+    if (probs == nullptr) return;
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    float m = -INFINITY;
+    for (int c = threadIdx.x; c < C; c += blockDim.x) m = fmaxf(m, z[c]);
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0) red[warp] = m;
+    __syncthreads();
+    m = red[0];
+    for (int i = 1; i < nwarps; ++i) m = fmaxf(m, red[i]);
+    __syncthreads();
+
+    float s = 0.f;
+    for (int c = threadIdx.x; c < C; c += blockDim.x) {
+        const float e = expf(z[c] - m);
+        z[c] = e;
+        s += e;
+    }
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) red[warp] = s;
+    __syncthreads();
+    s = 0.f;
+    for (int i = 0; i < nwarps; ++i) s += red[i];
+    const float r = 1.0f / s;
+    for (int c = threadIdx.x; c < C; c += blockDim.x) probs[(size_t)n * C + c] = z[c] * r;
+}
+
+}  // namespace
+
+int launch_maxpool3x3s2(const void* in, void* out, int C, int H, int W, int N, int dtype, cudaStream_t stream)
+{
+    const int OH = (H - 3) / 2 + 1, OW = (W - 3) / 2 + 1;
+    const int threads = 256;
+    if (dtype == SQN_F32) {
+        if (C % 4 == 0) {
+            const long long total = (long long)N * OH * OW * (C / 4);
+            maxpool_f32_v4<<<(unsigned)((total + threads - 1) / threads), threads, 0, stream>>>(
+                static_cast<const float*>(in), static_cast<float*>(out), C / 4, H, W, OH, OW, total);
+        } else {
+            const long long total = (long long)N * OH * OW * C;
+            maxpool_f32_s<<<(unsigned)((total + threads - 1) / threads), threads, 0, stream>>>(
+                static_cast<const float*>(in), static_cast<float*>(out), C, H, W, OH, OW, total);
+        }
+    } else {
+        if (C % 8 == 0) {
+            const long long total = (long long)N * OH * OW * (C / 8);
+            maxpool_bf16_v8<<<(unsigned)((total + threads - 1) / threads), threads, 0, stream>>>(
+                static_cast<const uint4*>(in), static_cast<uint4*>(out), C / 8, H, W, OH, OW, total);
+        } else {
+            const long long total = (long long)N * OH * OW * C;
+            maxpool_bf16_s<<<(unsigned)((total + threads - 1) / threads), threads, 0, stream>>>(
+                static_cast<const __nv_bfloat16*>(in), static_cast<__nv_bfloat16*>(out), C, H, W, OH, OW, total);
+        }
+    }
+    note_launch();
+    return cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
+}
+
+int launch_avgpool_softmax(const void* in, float* logits, float* probs, int C, int H, int W, int N, int dtype,
+                           cudaStream_t stream)
+{
+    const size_t smem = (size_t)C * sizeof(float);
+    if (dtype == SQN_F32)
+        avgpool_softmax_kernel<false><<<N, 256, smem, stream>>>(in, logits, probs, C, H * W);
+    else
+        avgpool_softmax_kernel<true><<<N, 256, smem, stream>>>(in, logits, probs, C, H * W);
+    note_launch();
+    return cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
+}
+
+}  // namespace sqn

@@ -1,0 +1,46 @@
+// Internal declarations shared by the library's translation units.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "sqn.h"
+
+namespace sqn {
+
+// One convolution layer as the kernels see it (validated by the caller).
+struct ConvDesc {
+    const void* in;       // [N][H][W][Cin]
+    const void* w;        // [Cout][K][K][Cin]
+    const float* bias;    // [Cout]
+    void* out;            // [N][OH][OW][out_c_total], written at out_c_offset
+    int N, Cin, H, W, Cout, K, S, pad, OH, OW;
+    int out_c_offset, out_c_total, relu;
+};
+
+// Launch counter (host side): every kernel launch goes through note_launch().
+void note_launch(int n = 1);
+
+// Device status word shared by all kernels (0 = fine, else an sqn_status).
+int* device_status_word();
+
+// fp32 path: register-tiled FFMA implicit GEMM, any (K, S, pad, Cin, Cout).
+int launch_conv_f32(const ConvDesc& d, cudaStream_t stream);
+
+// bf16 path: tcgen05/TMEM implicit GEMM fed by TMA.
+// Returns SQN_ERR_UNSUPPORTED for shapes outside its family.
+int conv_bf16_supported(const ConvDesc& d);
+int launch_conv_bf16(const ConvDesc& d, cudaStream_t stream);
+// Stem (7x7/2 on 3 layers): needs scratch for the repacked input and kernels.
+size_t stem_bf16_workspace_bytes(int N, int H, int W, int Cout);
+int launch_stem_bf16(const ConvDesc& d, void* workspace, size_t workspace_bytes, cudaStream_t stream);
+
+// Pooling / head.
+int launch_maxpool3x3s2(const void* in, void* out, int C, int H, int W, int N, int dtype, cudaStream_t stream);
+int launch_avgpool_softmax(const void* in, float* logits, float* probs, int C, int H, int W, int N, int dtype,
+                           cudaStream_t stream);
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace sqn

@@ -1,0 +1,107 @@
+"""CPU-side checks of the boundary: the library loads, exports what include/sqn.h declares,
+validates arguments before touching the GPU, and its host layout helpers are exact."""
+import os
+import re
+
+import numpy as np
+import pytest
+import torch
+
+from paper_1611_07151_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "sqn.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b([a-z_0-9]+)\s*\(", text)) - {"defined"})
+
+
+def test_library_exports_every_declared_symbol():
+    names = declared_functions()
+    assert "conv_forward" in names and "fire_forward" in names and "squeezenet_forward" in names
+    l = B.lib()
+    for n in names:
+        assert hasattr(l, n), "libsqn.so does not export " + n
+    assert sorted(B.SIGNATURES) == names, "binding and header disagree on the entry points"
+
+
+def test_status_strings():
+    assert B.sqn_status_string(0) == "ok"
+    for s in range(-6, 0):
+        assert B.sqn_status_string(s) not in ("ok", "unknown status")
+    assert B.sqn_status_string(-99) == "unknown status"
+
+
+def test_bad_arguments_are_rejected_before_any_launch():
+    l = B.lib()
+    n0 = B.sqn_launch_count()
+    p = 0x1000      # never dereferenced: validation fails first
+    assert l.conv_forward(None, p, p, p, 3, 4, 8, 8, 3, 1, 1, 1) == B.SQN_ERR_BADARG
+    assert l.conv_forward(p, p, p, p, 0, 4, 8, 8, 3, 1, 1, 1) == B.SQN_ERR_BADARG
+    assert l.conv_forward(p, p, p, p, 3, 4, 8, 8, 0, 1, 1, 1) == B.SQN_ERR_BADARG
+    assert l.conv_forward(p, p, p, p, 3, 4, 8, 8, 3, 0, 1, 1) == B.SQN_ERR_BADARG
+    assert l.conv_forward(p, p, p, p, 3, 4, 8, 8, 3, 1, -1, 1) == B.SQN_ERR_BADARG
+    assert l.conv_forward(p, p, p, p, 3, 4, 2, 2, 5, 1, 1, 1) == B.SQN_ERR_BADARG      # window > padded input
+    assert l.conv_forward(p + 4, p, p, p, 3, 4, 8, 8, 3, 1, 1, 1) == B.SQN_ERR_ALIGN
+    opts = B.sqn_conv_opts(7, 1, 0, 0, None, None, 0)
+    assert l.conv_forward_ex(p, p, p, p, 3, 4, 8, 8, 3, 1, 1, 1, opts) == B.SQN_ERR_BADARG   # unknown dtype
+    opts = B.sqn_conv_opts(B.SQN_F32, 1, 4, 6, None, None, 0)
+    assert l.conv_forward_ex(p, p, p, p, 3, 4, 8, 8, 3, 1, 1, 1, opts) == B.SQN_ERR_BADARG   # slice overruns
+    assert l.maxpool3x3s2_forward(p, p, 8, 2, 8, 1, 0, None) == B.SQN_ERR_BADARG
+    assert l.avgpool_softmax_forward(p, p, p, 10000, 2, 2, 1, 0, None) == B.SQN_ERR_UNSUPPORTED
+    assert l.fire_forward(p, p, p, p, p, p, p, None, p, 8, 4, 8, 8, 5, 5, 1, 0, None) == B.SQN_ERR_BADARG
+    assert B.sqn_launch_count() == n0
+
+
+def test_bf16_path_refuses_shapes_outside_its_family():
+    l = B.lib()
+    p = 0x1000
+    n0 = B.sqn_launch_count()
+    for (cin, cout, k, s, pad) in [(12, 16, 1, 1, 0), (16, 20, 1, 1, 0), (16, 16, 3, 2, 1), (16, 16, 5, 1, 1)]:
+        opts = B.sqn_conv_opts(B.SQN_BF16, 1, 0, 0, None, None, 0)
+        rc = l.conv_forward_ex(p, p, p, p, cin, cout, 9, 9, k, s, pad, 1, opts)
+        assert rc in (B.SQN_ERR_UNSUPPORTED, B.SQN_ERR_ALIGN), (cin, cout, k, s, pad, rc)
+    assert B.sqn_launch_count() == n0
+
+
+def test_pack_helpers_are_exact_transposes():
+    rng = np.random.default_rng(0)
+    w = rng.standard_normal((5, 3, 7, 7)).astype(np.float32)
+    np.testing.assert_array_equal(B.sqn_pack_weights_oihw_to_ohwi(w), w.transpose(0, 2, 3, 1))
+    x = rng.standard_normal((2, 6, 4, 5)).astype(np.float32)
+    nhwc = B.sqn_pack_nchw_to_nhwc(x)
+    np.testing.assert_array_equal(nhwc, x.transpose(0, 2, 3, 1))
+    np.testing.assert_array_equal(B.sqn_unpack_nhwc_to_nchw(nhwc), x)
+
+
+def test_bf16_rounding_is_nearest_even():
+    rng = np.random.default_rng(1)
+    x = np.concatenate([rng.standard_normal(4096).astype(np.float32) * 10,
+                        np.array([0.0, -0.0, 1.0, 1.00390625, 1.01171875, 3.3895314e38, 1e-40, np.inf], np.float32)])
+    x = x.reshape(1, -1, 1, 1)
+    got = B.sqn_pack_nchw_to_nhwc(x, B.SQN_BF16).ravel()
+    exp = torch.from_numpy(x.ravel()).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    np.testing.assert_array_equal(got, exp)
+    back = B.sqn_unpack_nhwc_to_nchw(got.reshape(1, 1, 1, -1), B.SQN_BF16).ravel()
+    np.testing.assert_array_equal(back, torch.from_numpy(x.ravel()).to(torch.bfloat16).float().numpy())
+
+
+def test_squeezenet_handle_and_workspace_without_gpu():
+    l = B.lib()
+    p = 0x1000
+    h = B.squeezenet_create([p] * 26, [p] * 26, B.SQN_F32, 4)
+    b1 = B.squeezenet_workspace_bytes(h, 1)
+    b4 = B.squeezenet_workspace_bytes(h, 4)
+    per_image = 4 * (1182816 + 290400 + 2 * (48400 + 387200) + 96800 + 774400 + 186624 + 23328 + 186624
+                     + 2 * (34992 + 279936) + 46656 + 373248 + 86528 + 10816 + 86528 + 169000)
+    assert per_image <= b1 <= per_image + 32 * 1024
+    assert 4 * per_image <= b4 <= 4 * per_image + 32 * 1024
+    with pytest.raises(B.SqnError):
+        B.squeezenet_workspace_bytes(h, 5)            # beyond max_batch
+    ptr, C, H, W = B.squeezenet_layer_output(h, "fire4", 0x100000, 1)
+    assert (C, H, W) == (256, 55, 55) and ptr > 0x100000
+    with pytest.raises(B.SqnError):
+        B.squeezenet_layer_output(h, "fire99", 0x100000, 1)
+    B.squeezenet_destroy(h)
