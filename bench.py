@@ -1,0 +1,337 @@
+"""Benchmark: SqueezeNet v1.0 forward, images/s.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+  python -m torch.distributed.run --nnodes=1 --nproc-per-node N ... bench.py --gpus N ...
+
+A step is one forward of the whole network over one batch of synthetic images
+(default: batch 256 per GPU, bf16 activations/kernels with fp32 accumulation on the
+tensor cores).  Images are independent, so N GPUs run N replicas on their own batches
+(weak scaling, no collective on the data path); the job's value is all images / the
+slowest rank's device time.  Rank 0 prints one JSON line.
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_1611_07151_b200 import dist as D
+from paper_1611_07151_b200 import synth
+
+IMG = 227
+METRIC = "squeezenet_v1.0_forward_images_per_s"
+UNIT = "images/s"
+
+
+# --------------------------------------------------------------------------- peaks
+def measured_peaks():
+    """Roofline denominators measured on this machine (written by the driver), else the fallback figures."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def fp32_ffma_peak_tflops(sm_count, sm_mhz):
+    """FP32 pipe peak: SMs x 128 lanes x 2 flop x clock."""
+    return sm_count * 128 * 2 * sm_mhz * 1e6 / 1e12
+
+
+# ---------------------------------------------------------- algorithmic work per launch
+def launch_work(batch, es):
+    """name -> dict(flops, bytes) per forward, counting every tensor a launch must read or write once."""
+    work = {}
+    hw_out = {"conv1": 111}
+    for name, cin, cout, k, s, pad, hw in synth.SQUEEZENET_CONVS:
+        oh = (hw + 2 * pad - k) // s + 1
+        flops = 2.0 * batch * oh * oh * cout * cin * k * k
+        byts = es * batch * (hw * hw * cin + oh * oh * cout) + es * cout * cin * k * k + 4 * cout
+        work[name] = {"flops": flops, "bytes": float(byts)}
+    for name, c, h in (("pool1", 96, 111), ("pool4", 256, 55), ("pool8", 512, 27)):
+        o = (h - 3) // 2 + 1
+        work[name] = {"flops": 0.0, "bytes": float(es * batch * c * (h * h + o * o))}
+    work["head"] = {"flops": 0.0, "bytes": float(batch * (es * 1000 * 169 + 8 * 1000))}
+    # repack of the stem's input (3 -> 4 layers, padded rows): an extra pass, counted at its real traffic
+    work["conv1_pack"] = {"flops": 0.0, "bytes": float(batch * (IMG * IMG * 3 * 2 + 228 * 228 * 8))}
+    return work
+
+
+# ------------------------------------------------------------------- clock sampling
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs (read only)."""
+
+    def __init__(self, index, period=0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {"hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+                 "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4)}
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        med = int(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_rank):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# ------------------------------------------------------------------ oracle timings
+def oracle_images_per_s(n_images, seed, repeats=1):
+    """Times the CPU oracle, as it stands, on n_images of the workload.  Returns (images/s, threads)."""
+    from oracle import ref
+    x, params = synth.squeezenet_case(seed, n_images)
+    t0 = time.perf_counter()
+    for _ in range(repeats):
+        ref.squeezenet(x, params)
+    dt = time.perf_counter() - t0
+    return n_images * repeats / dt, ref.max_threads()
+
+
+def run_reference(args):
+    """--impl reference: the oracle on the host cores, same metric/config, bounded sample per step."""
+    rank, _local, world = D.env_world()
+    if rank != 0:
+        return
+    from oracle import ref
+    x1, params = synth.squeezenet_case(3, 1)
+    t0 = time.perf_counter()
+    ref.squeezenet(x1, params)
+    t_img = time.perf_counter() - t0
+    budget = 150.0 / max(1, args.steps + args.warmup)
+    n_img = int(max(1, min(args.batch, budget // max(t_img, 1e-6))))
+    x, _ = synth.squeezenet_case(3, n_img)
+    for _ in range(args.warmup):
+        ref.squeezenet(x, params)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        ref.squeezenet(x, params)
+    dt = time.perf_counter() - t0
+    value = n_img * args.steps / dt
+    cores = ref.max_threads()
+    sample = "%d of the %d images of the batch per step, full network, all host threads" % (n_img, args.batch)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64 accumulate, f32 storage",
+            "data": "synthetic",
+            "config": {"workload": workload_name(args), "batch_per_gpu": args.batch, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def workload_name(args):
+    return "squeezenet_v1.0_forward_b%d_%s" % (args.batch, args.dtype)
+
+
+# --------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=256, help="images per GPU per step")
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"])
+    ap.add_argument("--e2e-steps", type=int, default=0, help="steps of the host-buffer loop (0: min(steps, 50))")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    from paper_1611_07151_b200 import binding as B
+
+    rank, local_rank, world = D.env_world()
+    torch.cuda.set_device(local_rank)
+    dev = "cuda:%d" % local_rank
+    D.init("nccl")
+    B.lib()                                     # raises if the CUDA library is missing: no other path exists
+
+    dtype = B.SQN_BF16 if args.dtype == "bf16" else B.SQN_F32
+    es = 2 if dtype == B.SQN_BF16 else 4
+    batch = args.batch
+
+    # ---- synthetic workload: U[0,1) images, He-normal kernels, N(0,.01) bias (seed 3 + rank)
+    x, params = synth.squeezenet_case(3 + rank, batch)
+    names = [n for n, *_ in synth.SQUEEZENET_CONVS]
+    ws = [B.to_device(B.sqn_pack_weights_oihw_to_ohwi(params[n][0], dtype), dtype) for n in names]
+    bs = [B.to_device(np.ascontiguousarray(params[n][1], dtype=np.float32)) for n in names]
+    x_host = B.sqn_pack_nchw_to_nhwc(x, dtype)
+    del x
+    host_t = torch.from_numpy(x_host)
+    if dtype == B.SQN_BF16:
+        host_t = host_t.view(torch.int16).view(torch.bfloat16)
+    x_pinned = host_t.pin_memory()
+    inputs = [x_pinned.to(dev), torch.flip(x_pinned, dims=[0]).contiguous().to(dev)]   # rotated between steps
+
+    net = B.squeezenet_create(ws, bs, dtype, batch)
+    work_bytes = B.squeezenet_host_workspace_bytes(net, batch)
+    workspace = torch.empty(work_bytes, dtype=torch.uint8, device=dev)
+    logits = torch.empty((batch, 1000), dtype=torch.float32, device=dev)
+    probs = torch.empty((batch, 1000), dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        B.squeezenet_forward(net, inputs[i & 1], logits, probs, workspace, batch)
+
+    # ---- warm-up, then the timed region (device-resident inputs)
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    assert B.sqn_check() == B.SQN_OK
+    B.squeezenet_profile(net, min(args.steps, 256))
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    D.barrier()
+    torch.cuda.synchronize()
+    launches0 = B.sqn_launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.start()
+    ev0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    D.barrier()
+    clocks = sampler.stop()
+    gpu_launches = B.sqn_launch_count() - launches0
+    ms_local = ev0.elapsed_time(ev1)
+    status = B.sqn_check()
+    assert status == B.SQN_OK, B.sqn_status_string(status)
+    value, ms_total = D.job_throughput(batch * args.steps, ms_local, dev)
+
+    # ---- per-launch times recorded inside the timed region -> per-layer roofline
+    lnames, lms, nfwd = B.squeezenet_profile_read(net)
+    B.squeezenet_profile(net, 0)
+    peaks = measured_peaks()
+    props = torch.cuda.get_device_properties(local_rank)
+    sm_mhz = clocks["sm_mhz"] or clocks["sm_max_mhz"] or 1965
+    pipe_tf = peaks["bf16_tflops_sustained"] if dtype == B.SQN_BF16 else fp32_ffma_peak_tflops(
+        props.multi_processor_count, sm_mhz)
+    work = launch_work(batch, es)
+    layers = []
+    total_ms = sum(lms) / max(nfwd, 1)
+    for n, ms_sum in zip(lnames, lms):
+        ms = ms_sum / max(nfwd, 1)
+        w = work.get(n, {"flops": 0.0, "bytes": 0.0})
+        t_hbm = w["bytes"] / (peaks["hbm_gbs"] * 1e9)
+        t_pipe = w["flops"] / (pipe_tf * 1e12)
+        bound = "hbm" if t_hbm >= t_pipe else ("tensor" if dtype == B.SQN_BF16 else "alu")
+        layers.append({"name": n, "ms": ms, "share": ms / total_ms if total_ms else 0.0, "bound": bound,
+                       "gbs": w["bytes"] / (ms * 1e-3) / 1e9 if ms > 0 else 0.0,
+                       "tflops": w["flops"] / (ms * 1e-3) / 1e12 if ms > 0 else 0.0,
+                       "frac": max(t_hbm, t_pipe) / (ms * 1e-3) if ms > 0 else 0.0,
+                       "bytes": w["bytes"], "flops": w["flops"]})
+    top = max(layers, key=lambda l: l["ms"])
+    if top["bound"] == "hbm":
+        roof = {"bound": "hbm", "achieved": top["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    else:
+        roof = {"bound": top["bound"], "achieved": top["tflops"], "peak": pipe_tf, "unit": "TFLOP/s"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = None
+    roof["kernel"] = ("conv_tc_kernel" if dtype == B.SQN_BF16 else "conv_f32_kernel") + "[%s]" % top["name"]
+    roof["peak_source"] = "of " + peaks["source"]
+    roof["launch_ms"] = top["ms"]
+    roof["share_of_step"] = top["share"]
+    sum_bound_ms = sum(l["frac"] * l["ms"] for l in layers)
+    roof["whole_step_frac_of_layer_bounds"] = sum_bound_ms / total_ms if total_ms else None
+
+    # ---- end to end: host buffers in, host buffers out, through the C ABI (copies inside the timed region)
+    e2e_steps = args.e2e_steps or min(args.steps, 50)
+    out_host = torch.empty((2, batch, 1000), dtype=torch.float32).pin_memory()
+    for i in range(3):
+        B.squeezenet_forward_host(net, x_pinned, out_host[0], out_host[1], workspace, batch)
+    torch.cuda.synchronize()
+    D.barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(e2e_steps):
+        B.squeezenet_forward_host(net, x_pinned, out_host[0], out_host[1], workspace, batch)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    D.barrier()
+    e2e_value, _ = D.job_throughput(batch * e2e_steps, e0.elapsed_time(e1), dev)
+    h2d = batch * IMG * IMG * 3 * es
+    d2h = 2 * batch * 1000 * 4
+    assert abs(float(out_host[1].sum()) - batch) < 1e-2 * batch     # probabilities came back
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v1, cores = oracle_images_per_s(1, 3)
+        n = int(min(64, max(2, 15.0 * v1)))
+        v, cores = oracle_images_per_s(n, 3)
+        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": "%d of the %d images of one batch, full network, double accumulation" % (n, batch)}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": args.dtype, "data": "synthetic",
+                "config": {"workload": workload_name(args), "batch_per_gpu": batch, "global_batch": batch * world,
+                           "image": "227x227x3", "parallelism": "replicas, batch sharded by image, no collective",
+                           "l2": "per-step activations (%.1f GB) exceed the 126 MB L2; two input batches alternate"
+                                 % (B.squeezenet_workspace_bytes(net, batch) / 1e9)},
+                "clocks": clocks,
+                "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                        "steps": e2e_steps},
+                "gpu_launches": int(gpu_launches),
+                "roofline": roof,
+                "cpu_baseline": cpu,
+                "layers": [{k: (round(v, 6) if isinstance(v, float) else v) for k, v in l.items()} for l in layers]}
+        print(json.dumps(line), flush=True)
+    B.squeezenet_destroy(net)
+
+
+if __name__ == "__main__":
+    main()

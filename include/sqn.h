@@ -87,12 +87,12 @@ typedef struct {
 /*
  * Same operation as conv_forward with every choice exposed.  opts may be NULL
  * (fp32, ReLU, dense, default stream).
- * SQN_BF16 restrictions (else SQN_ERR_UNSUPPORTED / SQN_ERR_ALIGN):
- *   - S == 1, 2*pad == K-1 or pad == 0, numInputLayers a multiple of 16,
- *     numOutputLayers a multiple of 8 (16 when <= 256 is not met see below),
- *     out_c_offset and out_c_total multiples of 8; or
- *   - the stem shape K=7, S=2, pad=0, numInputLayers=3, which needs a workspace
- *     (conv_workspace_bytes) for its repacked input and kernels.
+ * SQN_BF16 accepts (else SQN_ERR_UNSUPPORTED / SQN_ERR_ALIGN):
+ *   - S == 1, K <= 7 (pad == 0 when K == 1), numInputLayers a multiple of 16,
+ *     numOutputLayers a multiple of 16 (of 8 when above 256), out_c_offset and out_c_total
+ *     multiples of 8; or
+ *   - the stem shape K=7, S=2, pad=0, numInputLayers=3 with numOutputLayers a multiple of 16
+ *     up to 256, which needs a workspace (conv_workspace_bytes) for its repacked input and kernels.
  */
 int conv_forward_ex(const void* in, const void* weights, const void* bias, void* out,
                     int numInputLayers, int numOutputLayers, int H, int W, int K, int S, int pad, int batch,
@@ -162,6 +162,34 @@ int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logits_f32, void
 int squeezenet_layer_output(const sqn_net* net, const char* name, void* workspace, int batch, void** ptr, int* C,
                             int* H, int* W);
 int squeezenet_destroy(sqn_net* net);
+
+/*
+ * The same forward with HOST input and output buffers (the call a user with data in host
+ * memory makes).  Enqueues on `stream`: copy of in_host [batch][227][227][3] (net dtype) to the
+ * device, the forward, copies of logits (and probs, unless NULL) [batch][1000] fp32 back to
+ * the host.  The copies are asynchronous when the host buffers are pinned.  workspace is
+ * DEVICE memory of squeezenet_host_workspace_bytes(net, batch) bytes (the forward's scratch
+ * plus staging for the input and the two outputs).  The host buffers must stay valid until
+ * the stream has passed the call.
+ */
+int squeezenet_host_workspace_bytes(const sqn_net* net, int batch, size_t* bytes);
+int squeezenet_forward_host(sqn_net* net, const void* in_host, void* logits_host, void* probs_host,
+                            void* workspace, int batch, void* stream);
+
+/*
+ * Per-launch timing of squeezenet_forward with CUDA events on the caller's stream (the
+ * paper reports per-layer times, Section IV, Table 4).
+ * squeezenet_profile(net, slots): slots > 0 records an event after every launch of each
+ *   following forward, keeping the most recent `slots` forwards; 0 turns it off.
+ * squeezenet_profile_read: waits for the recorded forwards, then writes into ms_sum[i] the
+ *   time of launch group i summed over *forwards recorded forwards; *launches = number of
+ *   groups per forward.  ms_sum may be NULL to query the counts only.
+ * squeezenet_profile_name(net, i): name of group i ("conv1_pack", "conv1", "pool1",
+ *   "fire2_sq", "fire2_e1", "fire2_e3", ..., "conv10", "head"); "" if out of range.
+ */
+int squeezenet_profile(sqn_net* net, int slots);
+int squeezenet_profile_read(sqn_net* net, float* ms_sum, int capacity, int* launches, int* forwards);
+const char* squeezenet_profile_name(const sqn_net* net, int i);
 
 /*
  * Host-side layout helpers (the paper's offline reordering of the model file,

@@ -47,6 +47,12 @@ SIGNATURES = {
     "squeezenet_layer_output": (_c_int, [_c_vp, ctypes.c_char_p, _c_vp, _c_int, ctypes.POINTER(_c_vp),
                                          ctypes.POINTER(_c_int), ctypes.POINTER(_c_int), ctypes.POINTER(_c_int)]),
     "squeezenet_destroy": (_c_int, [_c_vp]),
+    "squeezenet_host_workspace_bytes": (_c_int, [_c_vp, _c_int, ctypes.POINTER(_c_sz)]),
+    "squeezenet_forward_host": (_c_int, [_c_vp] * 5 + [_c_int, _c_vp]),
+    "squeezenet_profile": (_c_int, [_c_vp, _c_int]),
+    "squeezenet_profile_read": (_c_int, [_c_vp, ctypes.POINTER(ctypes.c_float), _c_int, ctypes.POINTER(_c_int),
+                                         ctypes.POINTER(_c_int)]),
+    "squeezenet_profile_name": (ctypes.c_char_p, [_c_vp, _c_int]),
     "sqn_pack_weights_oihw_to_ohwi": (_c_int, [_c_vp, _c_vp, _c_int, _c_int, _c_int, _c_int]),
     "sqn_pack_nchw_to_nhwc": (_c_int, [_c_vp, _c_vp] + [_c_int] * 5),
     "sqn_unpack_nhwc_to_nchw": (_c_int, [_c_vp, _c_vp] + [_c_int] * 5),
@@ -174,6 +180,32 @@ def squeezenet_layer_output(net, name, workspace, batch):
 
 def squeezenet_destroy(net):
     _check(lib().squeezenet_destroy(net), "squeezenet_destroy")
+
+
+def squeezenet_host_workspace_bytes(net, batch):
+    n = _c_sz(0)
+    _check(lib().squeezenet_host_workspace_bytes(net, batch, ctypes.byref(n)), "squeezenet_host_workspace_bytes")
+    return n.value
+
+
+def squeezenet_forward_host(net, in_host, logits_host, probs_host, workspace, batch, stream=None):
+    """in_host / logits_host / probs_host: host tensors or arrays (pinned for asynchronous copies)."""
+    _check(lib().squeezenet_forward_host(net, _p(in_host), _p(logits_host), _p(probs_host), _p(workspace), batch,
+                                         current_stream() if stream is None else stream), "squeezenet_forward_host")
+
+
+def squeezenet_profile(net, slots):
+    _check(lib().squeezenet_profile(net, slots), "squeezenet_profile")
+
+
+def squeezenet_profile_read(net):
+    """-> (names, ms summed over the recorded forwards, number of forwards recorded)."""
+    n, f = _c_int(0), _c_int(0)
+    _check(lib().squeezenet_profile_read(net, None, 0, ctypes.byref(n), ctypes.byref(f)), "squeezenet_profile_read")
+    ms = (ctypes.c_float * max(n.value, 1))()
+    _check(lib().squeezenet_profile_read(net, ms, n.value, ctypes.byref(n), ctypes.byref(f)), "squeezenet_profile_read")
+    names = [lib().squeezenet_profile_name(net, i).decode() for i in range(n.value)]
+    return names, [float(ms[i]) for i in range(n.value)], f.value
 
 
 def sqn_check(stream=None):

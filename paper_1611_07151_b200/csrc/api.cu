@@ -76,7 +76,10 @@ int run_conv(const ConvDesc& d, int dtype, void* ws, size_t ws_bytes, cudaStream
 {
     if (dtype == SQN_F32) return launch_conv_f32(d, stream);
     if (dtype != SQN_BF16) return SQN_ERR_BADARG;
-    if (is_stem_shape(d)) return launch_stem_bf16(d, ws, ws_bytes, stream);
+    if (is_stem_shape(d)) {
+        const int rc = launch_stem_pack_bf16(d, ws, ws_bytes, stream);
+        return rc != SQN_OK ? rc : launch_stem_conv_bf16(d, ws, ws_bytes, stream);
+    }
     const int rc = conv_bf16_supported(d);
     if (rc != SQN_OK) return rc;
     return launch_conv_bf16(d, stream);
@@ -184,6 +187,11 @@ struct sqn_net {
     int dtype;
     int max_batch;
     std::vector<Slot> slots;   // per-image element counts; byte offsets are computed per batch
+    // optional per-launch timing: a ring of event rows, one row per forward
+    int prof_slots = 0;
+    long long prof_forwards = 0;
+    std::vector<std::string> prof_names;
+    std::vector<std::vector<cudaEvent_t>> prof_events;
 };
 
 namespace {
@@ -229,6 +237,8 @@ int find_slot(const sqn_net* net, const char* name)
 
 }  // namespace
 
+namespace { void free_profile(sqn_net* net); }
+
 extern "C" int squeezenet_create(sqn_net** net, const void* const* weights26, const void* const* bias26, int dtype,
                                  int max_batch)
 {
@@ -250,6 +260,7 @@ extern "C" int squeezenet_create(sqn_net** net, const void* const* weights26, co
 
 extern "C" int squeezenet_destroy(sqn_net* net)
 {
+    if (net) free_profile(net);
     delete net;
     return SQN_OK;
 }
@@ -276,6 +287,20 @@ extern "C" int squeezenet_layer_output(const sqn_net* net, const char* name, voi
     return SQN_OK;
 }
 
+namespace {
+
+void free_profile(sqn_net* net)
+{
+    for (auto& row : net->prof_events)
+        for (cudaEvent_t e : row) cudaEventDestroy(e);
+    net->prof_events.clear();
+    net->prof_names.clear();
+    net->prof_slots = 0;
+    net->prof_forwards = 0;
+}
+
+}  // namespace
+
 extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logits_f32, void* probs_f32,
                                   void* workspace, int batch, void* stream)
 {
@@ -290,27 +315,67 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
     char* ws = static_cast<char*>(workspace);
     auto buf = [&](const std::string& name) -> void* { return ws + offs[find_slot(net, name.c_str())]; };
 
+    // per-launch timing (off unless squeezenet_profile enabled it)
+    const bool prof = net->prof_slots > 0;
+    std::vector<cudaEvent_t>* row = prof ? &net->prof_events[net->prof_forwards % net->prof_slots] : nullptr;
+    const bool first = prof && net->prof_names.empty();
+    size_t mark_i = 0;
+    auto mark = [&](const char* name) {
+        if (!prof) return;
+        if (first) net->prof_names.push_back(name);
+        if (row->size() <= mark_i) {
+            cudaEvent_t e;
+            cudaEventCreate(&e);
+            row->push_back(e);
+        }
+        cudaEventRecord((*row)[mark_i++], st);
+    };
+    mark("start");
+
     int rc;
     ConvDesc d;
     // conv1 7x7/2 + ReLU, then max-pool
     rc = make_conv_desc(in_nhwc, net->w[0], net->b[0], buf("conv1"), 3, 96, IMG, IMG, 7, 2, 0, batch, 1, 0, 0, &d);
     if (rc != SQN_OK) return rc;
-    if ((rc = run_conv(d, dt, ws + stem_off, total - stem_off, st)) != SQN_OK) return rc;
+    if (dt == SQN_BF16) {
+        if ((rc = launch_stem_pack_bf16(d, ws + stem_off, total - stem_off, st)) != SQN_OK) return rc;
+        mark("conv1_pack");
+        if ((rc = launch_stem_conv_bf16(d, ws + stem_off, total - stem_off, st)) != SQN_OK) return rc;
+    } else {
+        if ((rc = launch_conv_f32(d, st)) != SQN_OK) return rc;
+    }
+    mark("conv1");
     if ((rc = launch_maxpool3x3s2(buf("conv1"), buf("pool1"), 96, 111, 111, batch, dt, st)) != SQN_OK) return rc;
+    mark("pool1");
 
     const void* cur = buf("pool1");
     for (int i = 0; i < 8; ++i) {
         const FireSpec& f = kFire[i];
         void* sq = buf(std::string(f.name) + "_sq");
         void* out = buf(f.name);
-        rc = fire_forward(cur, net->w[1 + 3 * i], net->b[1 + 3 * i], net->w[2 + 3 * i], net->b[2 + 3 * i],
-                          net->w[3 + 3 * i], net->b[3 + 3 * i], sq, out, f.cin, f.s, f.e, f.e, f.hw, f.hw, batch, dt,
-                          stream);
+        ConvDesc dsq, d1, d3;
+        rc = make_conv_desc(cur, net->w[1 + 3 * i], net->b[1 + 3 * i], sq, f.cin, f.s, f.hw, f.hw, 1, 1, 0, batch, 1, 0,
+                            0, &dsq);
         if (rc != SQN_OK) return rc;
+        rc = make_conv_desc(sq, net->w[2 + 3 * i], net->b[2 + 3 * i], out, f.s, f.e, f.hw, f.hw, 1, 1, 0, batch, 1, 0,
+                            2 * f.e, &d1);
+        if (rc != SQN_OK) return rc;
+        rc = make_conv_desc(sq, net->w[3 + 3 * i], net->b[3 + 3 * i], out, f.s, f.e, f.hw, f.hw, 3, 1, 1, batch, 1, f.e,
+                            2 * f.e, &d3);
+        if (rc != SQN_OK) return rc;
+        const std::string nm(f.name);
+        if ((rc = run_conv(dsq, dt, nullptr, 0, st)) != SQN_OK) return rc;
+        mark((nm + "_sq").c_str());
+        if ((rc = run_conv(d1, dt, nullptr, 0, st)) != SQN_OK) return rc;
+        mark((nm + "_e1").c_str());
+        if ((rc = run_conv(d3, dt, nullptr, 0, st)) != SQN_OK) return rc;
+        mark((nm + "_e3").c_str());
         cur = out;
         if (f.pool_after) {
-            void* po = buf(std::string("pool") + (f.name + 4));
+            const std::string pn = std::string("pool") + (f.name + 4);
+            void* po = buf(pn);
             if ((rc = launch_maxpool3x3s2(cur, po, 2 * f.e, f.hw, f.hw, batch, dt, st)) != SQN_OK) return rc;
+            mark(pn.c_str());
             cur = po;
         }
     }
@@ -318,8 +383,83 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
     rc = make_conv_desc(cur, net->w[25], net->b[25], buf("conv10"), 512, 1000, 13, 13, 1, 1, 0, batch, 1, 0, 0, &d);
     if (rc != SQN_OK) return rc;
     if ((rc = run_conv(d, dt, nullptr, 0, st)) != SQN_OK) return rc;
-    return launch_avgpool_softmax(buf("conv10"), static_cast<float*>(logits_f32), static_cast<float*>(probs_f32), 1000,
-                                  13, 13, batch, dt, st);
+    mark("conv10");
+    rc = launch_avgpool_softmax(buf("conv10"), static_cast<float*>(logits_f32), static_cast<float*>(probs_f32), 1000,
+                                13, 13, batch, dt, st);
+    if (rc != SQN_OK) return rc;
+    mark("head");
+    if (prof) net->prof_forwards++;
+    return SQN_OK;
+}
+
+extern "C" int squeezenet_host_workspace_bytes(const sqn_net* net, int batch, size_t* bytes)
+{
+    if (!net || !bytes || batch <= 0 || batch > net->max_batch) return SQN_ERR_BADARG;
+    const size_t in_bytes = align_up((size_t)batch * IMG * IMG * 3 * esize(net->dtype), 1024);
+    const size_t out_bytes = align_up((size_t)batch * 1000 * sizeof(float), 1024);
+    *bytes = layout(net, batch, nullptr, nullptr) + in_bytes + 2 * out_bytes;
+    return SQN_OK;
+}
+
+extern "C" int squeezenet_forward_host(sqn_net* net, const void* in_host, void* logits_host, void* probs_host,
+                                       void* workspace, int batch, void* stream)
+{
+    if (!net || !in_host || !logits_host || batch <= 0 || batch > net->max_batch) return SQN_ERR_BADARG;
+    if (!workspace) return SQN_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return SQN_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t fwd_bytes = layout(net, batch, nullptr, nullptr);
+    const size_t in_bytes = (size_t)batch * IMG * IMG * 3 * esize(net->dtype);
+    const size_t out_bytes = (size_t)batch * 1000 * sizeof(float);
+    char* ws = static_cast<char*>(workspace);
+    char* d_in = ws + fwd_bytes;
+    char* d_logits = d_in + align_up(in_bytes, 1024);
+    char* d_probs = d_logits + align_up(out_bytes, 1024);
+    if (cudaMemcpyAsync(d_in, in_host, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SQN_ERR_CUDA;
+    const int rc = squeezenet_forward(net, d_in, d_logits, probs_host ? d_probs : nullptr, workspace, batch, stream);
+    if (rc != SQN_OK) return rc;
+    if (cudaMemcpyAsync(logits_host, d_logits, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SQN_ERR_CUDA;
+    if (probs_host && cudaMemcpyAsync(probs_host, d_probs, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return SQN_ERR_CUDA;
+    return SQN_OK;
+}
+
+extern "C" int squeezenet_profile(sqn_net* net, int slots)
+{
+    if (!net || slots < 0 || slots > 4096) return SQN_ERR_BADARG;
+    free_profile(net);
+    net->prof_slots = slots;
+    net->prof_events.resize((size_t)slots);
+    return SQN_OK;
+}
+
+extern "C" int squeezenet_profile_read(sqn_net* net, float* ms_sum, int capacity, int* launches, int* forwards)
+{
+    if (!net || !launches || !forwards) return SQN_ERR_BADARG;
+    const int n = net->prof_names.empty() ? 0 : (int)net->prof_names.size() - 1;
+    *launches = n;
+    const long long have = net->prof_forwards < net->prof_slots ? net->prof_forwards : net->prof_slots;
+    *forwards = (int)have;
+    if (!ms_sum) return SQN_OK;
+    if (capacity < n) return SQN_ERR_BADARG;
+    for (int i = 0; i < n; ++i) ms_sum[i] = 0.f;
+    for (long long r = 0; r < have; ++r) {
+        std::vector<cudaEvent_t>& row = net->prof_events[(size_t)r];
+        if ((int)row.size() < n + 1) return SQN_ERR_CUDA;
+        if (cudaEventSynchronize(row[n]) != cudaSuccess) return SQN_ERR_CUDA;
+        for (int i = 0; i < n; ++i) {
+            float ms = 0.f;
+            if (cudaEventElapsedTime(&ms, row[i], row[i + 1]) != cudaSuccess) return SQN_ERR_CUDA;
+            ms_sum[i] += ms;
+        }
+    }
+    return SQN_OK;
+}
+
+extern "C" const char* squeezenet_profile_name(const sqn_net* net, int i)
+{
+    if (!net || i < 0 || i + 1 >= (int)net->prof_names.size()) return "";
+    return net->prof_names[(size_t)i + 1].c_str();
 }
 
 // ---------------------------------------------------------------- host layout helpers

@@ -599,27 +599,44 @@ size_t stem_bf16_workspace_bytes(int N, int H, int W, int Cout)
     return align_up((size_t)N * Hp * Wp * 8, 1024) + align_up((size_t)Cout * 224 * 2, 1024);
 }
 
-int launch_stem_bf16(const ConvDesc& d, void* workspace, size_t workspace_bytes, cudaStream_t stream)
+namespace {
+int stem_check(const ConvDesc& d, void* workspace, size_t workspace_bytes)
 {
     if (d.Cout % 16 != 0 || d.Cout > 256) return SQN_ERR_UNSUPPORTED;
     if (d.out_c_offset % 8 != 0 || d.out_c_total % 8 != 0) return SQN_ERR_ALIGN;
     if (!workspace || workspace_bytes < stem_bf16_workspace_bytes(d.N, d.H, d.W, d.Cout)) return SQN_ERR_WORKSPACE;
     if (!aligned16(workspace)) return SQN_ERR_ALIGN;
+    return SQN_OK;
+}
+}  // namespace
+
+// Repack of the stem's input and kernels into the workspace (two small launches).
+int launch_stem_pack_bf16(const ConvDesc& d, void* workspace, size_t workspace_bytes, cudaStream_t stream)
+{
+    const int rc = stem_check(d, workspace, workspace_bytes);
+    if (rc != SQN_OK) return rc;
     const int Hp = (d.H + 1) / 2 * 2, Wp = (d.W + 2) / 2 * 2;
     unsigned char* ws = static_cast<unsigned char*>(workspace);
     uint2* pin = reinterpret_cast<uint2*>(ws);
     unsigned short* pw = reinterpret_cast<unsigned short*>(ws + align_up((size_t)d.N * Hp * Wp * 8, 1024));
-
     const long long total = (long long)d.N * Hp * Wp;
     stem_pack_input<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(d.in), pin,
                                                                         d.N, d.H, d.W, Hp, Wp);
     stem_pack_weights<<<(d.Cout * 224 + 255) / 256, 256, 0, stream>>>(static_cast<const unsigned short*>(d.w), pw,
                                                                        d.Cout);
     note_launch(2);
-    if (cudaGetLastError() != cudaSuccess) return SQN_ERR_CUDA;
+    return cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
+}
 
+// The stem convolution itself, on the repacked tensors left in the workspace by the call above.
+int launch_stem_conv_bf16(const ConvDesc& d, void* workspace, size_t workspace_bytes, cudaStream_t stream)
+{
+    int rc = stem_check(d, workspace, workspace_bytes);
+    if (rc != SQN_OK) return rc;
+    const int Hp = (d.H + 1) / 2 * 2, Wp = (d.W + 2) / 2 * 2;
+    unsigned char* ws = static_cast<unsigned char*>(workspace);
     Plan plan;
-    const int rc = cached_plan(d, true, pin, pw, Hp, Wp, workspace, &plan);
+    rc = cached_plan(d, true, ws, ws + align_up((size_t)d.N * Hp * Wp * 8, 1024), Hp, Wp, workspace, &plan);
     if (rc != SQN_OK) return rc;
     return launch_plan(plan, stream);
 }

@@ -34,7 +34,8 @@ int conv_bf16_supported(const ConvDesc& d);
 int launch_conv_bf16(const ConvDesc& d, cudaStream_t stream);
 // Stem (7x7/2 on 3 layers): needs scratch for the repacked input and kernels.
 size_t stem_bf16_workspace_bytes(int N, int H, int W, int Cout);
-int launch_stem_bf16(const ConvDesc& d, void* workspace, size_t workspace_bytes, cudaStream_t stream);
+int launch_stem_pack_bf16(const ConvDesc& d, void* workspace, size_t workspace_bytes, cudaStream_t stream);
+int launch_stem_conv_bf16(const ConvDesc& d, void* workspace, size_t workspace_bytes, cudaStream_t stream);
 
 // Pooling / head.
 int launch_maxpool3x3s2(const void* in, void* out, int C, int H, int W, int N, int dtype, cudaStream_t stream);

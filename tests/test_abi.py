@@ -59,7 +59,7 @@ def test_bf16_path_refuses_shapes_outside_its_family():
     l = B.lib()
     p = 0x1000
     n0 = B.sqn_launch_count()
-    for (cin, cout, k, s, pad) in [(12, 16, 1, 1, 0), (16, 20, 1, 1, 0), (16, 16, 3, 2, 1), (16, 16, 5, 1, 1)]:
+    for (cin, cout, k, s, pad) in [(12, 16, 1, 1, 0), (16, 20, 1, 1, 0), (16, 16, 3, 2, 1), (16, 16, 9, 1, 4), (16, 16, 1, 1, 1)]:
         opts = B.sqn_conv_opts(B.SQN_BF16, 1, 0, 0, None, None, 0)
         rc = l.conv_forward_ex(p, p, p, p, cin, cout, 9, 9, k, s, pad, 1, opts)
         assert rc in (B.SQN_ERR_UNSUPPORTED, B.SQN_ERR_ALIGN), (cin, cout, k, s, pad, rc)
