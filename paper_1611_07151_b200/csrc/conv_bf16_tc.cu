@@ -37,8 +37,9 @@ namespace {
 using namespace ptx;
 
 constexpr int TILE_M = 128;            // MMA M: TMEM lanes
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 224;       // producer, MMA, 4 epilogue warps, store issuer
 constexpr int MAX_STAGES = 8;
+constexpr int MAX_STG = 4;             // staging ring slots
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // about two seconds
 constexpr size_t SMEM_LIMIT = 227 * 1024;
 
@@ -46,6 +47,8 @@ struct TcParams {
     int tiles_w, tiles_h, tiles_i;   // output-pixel tiles: columns, rows, images
     int BW, BH, BI;                  // box extents, BW*BH*BI <= 128
     int n_tiles, BN;                 // output-layer tiles and their width (multiple of 16, <= 256)
+    int total_tiles;
+    int g_nt, g_tw, g_th, g_ti;      // gridDim.x written in the mixed radix (n_tiles, tiles_w, tiles_h, tiles_i)
     int Cout;
     int taps, taps_w, pad;           // kernel taps, taps per kernel row, zero padding
     int chunks, BKc;                 // reduction chunks per tap, elements per chunk (16/32/64)
@@ -53,21 +56,27 @@ struct TcParams {
     int stem;                        // 1: 7x7 stride-2 stem on the repacked input (tap = kernel row)
     int c_off;                       // first output layer inside the destination tensor
     int relu;
-    int stages;
+    int stages;                      // A (or A+B) ring slots
+    int b_resident;                  // 1: all kernel tiles are loaded once and stay in shared memory
     int CW;                          // layers per TMA store (16/32/64)
+    int nstg;                        // staging ring slots (2 or 4)
     int bn_pad;                      // TMEM column stride between the two accumulators
     unsigned tmem_cols;
-    unsigned a_bytes, b_bytes;       // bytes one stage's two boxes deliver
-    unsigned a_tile, b_tile;         // shared-memory bytes reserved per stage for A and B
+    unsigned a_bytes, b_bytes;       // bytes one item's A box / B box delivers
+    unsigned a_tile, b_tile;         // shared-memory bytes reserved per A / B tile
+    unsigned off_b, off_stg, off_bias, off_ctl;   // byte offsets from the 1024-aligned base
     const float* bias;
     int* status;
 };
 
-struct Shared {                       // small control block placed after the tiles
+struct Shared {                       // control block placed after the tiles
     unsigned long long full[MAX_STAGES];
     unsigned long long empty[MAX_STAGES];
+    unsigned long long b_full;
     unsigned long long tmem_full[2];
     unsigned long long tmem_empty[2];
+    unsigned long long stg_full[MAX_STG];
+    unsigned long long stg_free[MAX_STG];
     unsigned tmem_base;
     volatile int abort_flag;
 };
@@ -90,25 +99,36 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     }
 }
 
-// AND-reduction of a predicate over the 128 epilogue threads (named barrier 2).
-__device__ __forceinline__ bool epilogue_vote(bool ok)
-{
-    uint32_t all;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.u32 q, %1, 0;\n\t"
-        "bar.red.and.pred p, 2, 128, q;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(all)
-        : "r"((uint32_t)ok)
-        : "memory");
-    return all != 0;
-}
-
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Position of a tile in (output-layer tile, column tile, row tile, image tile) digits.  A CTA
+// walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...; the step is added digit by digit, so the
+// loops below contain no integer division.
+struct TileCoord { int nt, tw, th, ti; };
+
+__device__ __forceinline__ void tile_first(const TcParams& p, int t, TileCoord& c)
+{
+    c.nt = t % p.n_tiles;
+    const int mt = t / p.n_tiles;
+    c.tw = mt % p.tiles_w;
+    const int r = mt / p.tiles_w;
+    c.th = r % p.tiles_h;
+    c.ti = r / p.tiles_h;
+}
+__device__ __forceinline__ void tile_next(const TcParams& p, TileCoord& c)
+{
+    int carry = 0;
+    c.nt += p.g_nt;
+    if (c.nt >= p.n_tiles) { c.nt -= p.n_tiles; carry = 1; }
+    c.tw += p.g_tw + carry; carry = 0;
+    if (c.tw >= p.tiles_w) { c.tw -= p.tiles_w; carry = 1; }
+    c.th += p.g_th + carry; carry = 0;
+    if (c.th >= p.tiles_h) { c.th -= p.tiles_h; carry = 1; }
+    c.ti += p.g_ti + carry;
 }
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
@@ -121,27 +141,30 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     unsigned char* base_ptr = smem_raw + (base - raw);
 
     const uint32_t smA = base;
-    const uint32_t smB = smA + (uint32_t)p.stages * p.a_tile;
-    const uint32_t smStage = smB + (uint32_t)p.stages * p.b_tile;          // epilogue staging, 128 x BN bf16
-    const uint32_t stage_bytes = (uint32_t)TILE_M * p.BN * 2u;
-    float* bias_s = reinterpret_cast<float*>(base_ptr + (smStage - base) + stage_bytes);
-    Shared* sh = reinterpret_cast<Shared*>(reinterpret_cast<unsigned char*>(bias_s) + 256 * sizeof(float));
+    const uint32_t smB = base + p.off_b;
+    const uint32_t smStg = base + p.off_stg;
+    float* bias_s = reinterpret_cast<float*>(base_ptr + p.off_bias);
+    Shared* sh = reinterpret_cast<Shared*>(base_ptr + p.off_ctl);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const uint32_t row_bytes = (uint32_t)p.BKc * 2u;
     const int items = p.taps * p.chunks;
-    const int m_tiles = p.tiles_w * p.tiles_h * p.tiles_i;
-    const int total_tiles = m_tiles * p.n_tiles;
+    const int nchunks = p.BN / p.CW;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(smem_u32(&sh->full[s]), 1);
             mbar_init(smem_u32(&sh->empty[s]), 1);
         }
+        mbar_init(smem_u32(&sh->b_full), 1);
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&sh->tmem_full[a]), 1);
             mbar_init(smem_u32(&sh->tmem_empty[a]), 4);
+        }
+        for (int b = 0; b < p.nstg; ++b) {
+            mbar_init(smem_u32(&sh->stg_full[b]), 4);
+            mbar_init(smem_u32(&sh->stg_free[b]), 1);
         }
         sh->abort_flag = 0;
         fence_mbar_init();
@@ -153,6 +176,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tmem_alloc(smem_u32(&sh->tmem_base), p.tmem_cols);
         tmem_relinquish();
     }
+    // bias of every output layer, once per CTA
+    for (int c = threadIdx.x; c < p.n_tiles * p.BN; c += NUM_THREADS) bias_s[c] = c < p.Cout ? __ldg(p.bias + c) : 0.f;
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -162,41 +187,52 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
-            int it = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                const int nt = t % p.n_tiles;
-                const int mt = t / p.n_tiles;
-                const int w0 = (mt % p.tiles_w) * p.BW;
-                const int h0 = ((mt / p.tiles_w) % p.tiles_h) * p.BH;
-                const int i0 = (mt / (p.tiles_w * p.tiles_h)) * p.BI;
-                const int n0 = nt * p.BN;
-                for (int i = 0; i < items; ++i, ++it) {
-                    const int s = it % p.stages;
-                    const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
+            if (p.b_resident) {
+                // every kernel tile, once: they stay in shared memory for all tiles of this CTA
+                const uint32_t bf = smem_u32(&sh->b_full);
+                mbar_arrive_expect_tx(bf, (uint32_t)items * p.b_bytes);
+                int tap = 0, ch = 0;
+                for (int i = 0; i < items; ++i) {
+                    tma_load_2d(smB + (uint32_t)i * p.b_tile, &tmB, bf, tap * p.k_per_tap + ch * p.BKc, 0);
+                    if (++ch == p.chunks) { ch = 0; ++tap; }
+                }
+            }
+            const uint32_t tx = p.b_resident ? p.a_bytes : p.a_bytes + p.b_bytes;
+            int s = 0, issued = 0;
+            uint32_t ph = 0;
+            TileCoord tc;
+            tile_first(p, blockIdx.x, tc);
+            for (int t = blockIdx.x; t < p.total_tiles && ok; t += gridDim.x, tile_next(p, tc)) {
+                const int w0 = tc.tw * p.BW, h0 = tc.th * p.BH, i0 = tc.ti * p.BI, n0 = tc.nt * p.BN;
+                int tap = 0, kh = 0, kw = 0, ch = 0;
+                for (int i = 0; i < items; ++i) {
                     if (!wait_bar(smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-                    const int tap = i / p.chunks;
-                    const int x = (i - tap * p.chunks) * p.BKc;
                     const uint32_t full = smem_u32(&sh->full[s]);
-                    mbar_arrive_expect_tx(full, p.a_bytes + p.b_bytes);
-                    if (p.stem) {
-                        // tap = kernel row kh = 2a + b: input rows are split into (pair, parity)
-                        tma_load_5d(smA + s * p.a_tile, &tmA, full, 0, w0, h0 + (tap >> 1), tap & 1, i0);
-                    } else {
-                        const int kh = tap / p.taps_w;
-                        const int kw = tap - kh * p.taps_w;
-                        tma_load_5d(smA + s * p.a_tile, &tmA, full, x, w0 + kw - p.pad, h0 + kh - p.pad, i0, 0);
+                    const int x = ch * p.BKc;
+                    mbar_arrive_expect_tx(full, tx);
+                    if (p.stem)   // tap = kernel row kh = 2a + b: input rows are split into (pair, parity)
+                        tma_load_5d(smA + (uint32_t)s * p.a_tile, &tmA, full, 0, w0, h0 + (tap >> 1), tap & 1, i0);
+                    else
+                        tma_load_5d(smA + (uint32_t)s * p.a_tile, &tmA, full, x, w0 + kw - p.pad, h0 + kh - p.pad, i0, 0);
+                    if (!p.b_resident)
+                        tma_load_2d(smB + (uint32_t)s * p.b_tile, &tmB, full, tap * p.k_per_tap + x, n0);
+                    ++issued;
+                    if (++ch == p.chunks) {
+                        ch = 0; ++tap;
+                        if (++kw == p.taps_w) { kw = 0; ++kh; }
                     }
-                    tma_load_2d(smB + s * p.b_tile, &tmB, full, tap * p.k_per_tap + x, n0);
+                    if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
             }
             if (!ok) {
                 // give the copies already issued a bounded chance to land before the CTA exits
-                const int pending = it < p.stages ? it : p.stages;
-                for (int j = 1; j <= pending; ++j) {
-                    const int q = it - j;
+                int pending = issued < p.stages ? issued : p.stages;
+                while (pending-- > 0) {
+                    if (s == 0) { s = p.stages; ph ^= 1u; }
+                    --s;
                     const long long t0 = clock64();
-                    while (!mbar_try_wait(smem_u32(&sh->full[q % p.stages]), (uint32_t)(q / p.stages) & 1u)) {
+                    while (!mbar_try_wait(smem_u32(&sh->full[s]), ph)) {
                         if (clock64() - t0 > WAIT_LIMIT_CYCLES / 8) break;
                         __nanosleep(100);
                     }
@@ -208,101 +244,128 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (lane == 0) {
             const uint32_t idesc = make_idesc_bf16(TILE_M, (uint32_t)p.BN);
             const int ksteps = p.BKc / 16;
-            int it = 0, ti = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++ti) {
-                const int as = ti & 1;
-                const uint32_t aph = (uint32_t)(ti >> 1) & 1u;
+            if (p.b_resident) ok = wait_bar(smem_u32(&sh->b_full), 0u, abort_flag, p.status);
+            int s = 0, as = 0;
+            uint32_t ph = 0, aph = 0;
+            for (int t = blockIdx.x; t < p.total_tiles && ok; t += gridDim.x) {
                 if (!wait_bar(smem_u32(&sh->tmem_empty[as]), aph ^ 1u, abort_flag, p.status)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(as * p.bn_pad);
-                for (int i = 0; i < items; ++i, ++it) {
-                    const int s = it % p.stages;
-                    const uint32_t ph = (uint32_t)(it / p.stages) & 1u;
+                for (int i = 0; i < items; ++i) {
                     if (!wait_bar(smem_u32(&sh->full[s]), ph, abort_flag, p.status)) { ok = false; break; }
                     tc_fence_after();
-                    const uint64_t adesc = make_kmajor_desc(smA + s * p.a_tile, row_bytes);
-                    const uint64_t bdesc = make_kmajor_desc(smB + s * p.b_tile, row_bytes);
+                    const uint64_t adesc = make_kmajor_desc(smA + (uint32_t)s * p.a_tile, row_bytes);
+                    const uint64_t bdesc = make_kmajor_desc(smB + (uint32_t)(p.b_resident ? i : s) * p.b_tile, row_bytes);
                     for (int k = 0; k < ksteps; ++k) {
                         // 16 bf16 = 32 bytes further along the row: +2 in the (>>4) address field
                         mma_bf16_ss(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
                                     (i > 0 || k > 0) ? 1u : 0u);
                     }
                     mma_commit(smem_u32(&sh->empty[s]));        // slot free once these MMAs have read it
+                    if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
                 if (ok) mma_commit(smem_u32(&sh->tmem_full[as]));   // accumulator complete
+                if (++as == 2) { as = 0; aph ^= 1u; }
             }
         }
-    } else {
+    } else if (warp < 6) {
         // -------------------------------------------------------------------- epilogue
+        // One output pixel (TMEM lane) per thread.  Per chunk of CW layers: TMEM -> registers,
+        // + bias, ReLU, -> bf16, into a slot of the staging ring (TMA-swizzled rows); the store
+        // warp sends the slot to global memory while the next chunk is converted.
         const int q = warp & 3;                        // TMEM lane quadrant this warp may read
-        const int row = q * 32 + lane;                 // output pixel within the tile
-        const int et = threadIdx.x - 64;               // 0..127
-        const bool store_thread = (et == 0);
-        const uint32_t cw_bytes = (uint32_t)p.CW * 2u;             // bytes per staging row
-        const uint32_t chunk_bytes = (uint32_t)TILE_M * cw_bytes;  // one store chunk
-        // TMA swizzle of width cw_bytes: 16-byte unit index XOR (row-derived bits)
+        const int row = q * 32 + lane;
+        const uint32_t cw_bytes = (uint32_t)p.CW * 2u;
+        const uint32_t slot_bytes = (uint32_t)TILE_M * cw_bytes;
         const uint32_t sw = cw_bytes == 128 ? (uint32_t)(row & 7)
                           : cw_bytes == 64 ? (uint32_t)((row >> 1) & 3) : (uint32_t)((row >> 2) & 1);
-        int ti = 0;
+        const int nld = p.CW / 16;
         bool ok = true;
-        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++ti) {
-            const int nt = t % p.n_tiles;
-            const int mt = t / p.n_tiles;
-            const int w0 = (mt % p.tiles_w) * p.BW;
-            const int h0 = ((mt / p.tiles_w) % p.tiles_h) * p.BH;
-            const int i0 = (mt / (p.tiles_w * p.tiles_h)) * p.BI;
-            const int n0 = nt * p.BN;
-            const int as = ti & 1;
-            const uint32_t aph = (uint32_t)(ti >> 1) & 1u;
-
-            // staging and bias buffers are free once the previous tile's stores have read them
-            if (store_thread) tma_store_wait_read();
-            for (int c = et; c < p.BN; c += 128) bias_s[c] = (n0 + c < p.Cout) ? __ldg(p.bias + n0 + c) : 0.f;
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-
-            // all 128 epilogue threads take the same decision, so nobody is left alone at a barrier
-            if (!epilogue_vote(wait_bar(smem_u32(&sh->tmem_full[as]), aph, abort_flag, p.status))) { ok = false; break; }
+        int as = 0, sb = 0;
+        uint32_t aph = 0, sph = 0;
+        TileCoord tc;
+        tile_first(p, blockIdx.x, tc);
+        for (int t = blockIdx.x; t < p.total_tiles && ok; t += gridDim.x, tile_next(p, tc)) {
+            const int n0 = tc.nt * p.BN;
+            ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_full[as]), aph, abort_flag, p.status));
+            if (!ok) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * p.bn_pad);
-            for (int c = 0; c < p.BN; c += 16) {
-                uint32_t v[16];
-                tmem_ld_x16(taddr + (uint32_t)c, v);
-                tmem_ld_wait();
-                uint32_t o[8];
+            for (int chunk = 0; chunk < nchunks; ++chunk) {
+                const int c0 = chunk * p.CW;
+                if (n0 + c0 >= p.Cout) break;
+                uint32_t v[64];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    float a = __uint_as_float(v[2 * j]) + bias_s[c + 2 * j];
-                    float b = __uint_as_float(v[2 * j + 1]) + bias_s[c + 2 * j + 1];
-                    if (p.relu) { a = fmaxf(a, 0.f); b = fmaxf(b, 0.f); }
-                    o[j] = pack_bf16x2(a, b);
+                for (int j = 0; j < 4; ++j)
+                    if (j < nld) tmem_ld_x16(taddr + (uint32_t)(c0 + 16 * j), *reinterpret_cast<uint32_t(*)[16]>(&v[16 * j]));
+                ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->stg_free[sb]), sph ^ 1u, abort_flag, p.status));
+                tmem_ld_wait();
+                if (!ok) break;
+                const uint32_t rbase = smStg + (uint32_t)sb * slot_bytes + (uint32_t)row * cw_bytes;
+                const float* bch = bias_s + n0 + c0;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (j < nld) {
+                        uint32_t o[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            float a = __uint_as_float(v[16 * j + 2 * e]) + bch[16 * j + 2 * e];
+                            float b = __uint_as_float(v[16 * j + 2 * e + 1]) + bch[16 * j + 2 * e + 1];
+                            if (p.relu) { a = fmaxf(a, 0.f); b = fmaxf(b, 0.f); }
+                            o[e] = pack_bf16x2(a, b);
+                        }
+                        const uint32_t a0 = rbase + ((((uint32_t)(2 * j)) ^ sw) << 4);
+                        const uint32_t a1 = rbase + ((((uint32_t)(2 * j + 1)) ^ sw) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a0), "r"(o[0]), "r"(o[1]),
+                                     "r"(o[2]), "r"(o[3]) : "memory");
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a1), "r"(o[4]), "r"(o[5]),
+                                     "r"(o[6]), "r"(o[7]) : "memory");
+                    }
                 }
-                const int chunk = c / p.CW;
-                const int u0 = (c - chunk * p.CW) / 8;           // first of two 16-byte units
-                const uint32_t rbase = smStage + (uint32_t)chunk * chunk_bytes + (uint32_t)row * cw_bytes;
-                const uint32_t a0 = rbase + ((((uint32_t)u0) ^ sw) << 4);
-                const uint32_t a1 = rbase + ((((uint32_t)u0 + 1u) ^ sw) << 4);
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a0), "r"(o[0]), "r"(o[1]), "r"(o[2]),
-                             "r"(o[3]) : "memory");
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a1), "r"(o[4]), "r"(o[5]), "r"(o[6]),
-                             "r"(o[7]) : "memory");
+                fence_proxy_async_smem();             // staging rows visible to the TMA unit
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sh->stg_full[sb]));
+                if (++sb == p.nstg) { sb = 0; sph ^= 1u; }
             }
+            if (!ok) break;
             // accumulator drained: hand it back to the MMA issuer
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[as]));
-            // staging tile complete and visible to the TMA unit
-            fence_proxy_async_smem();
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (store_thread) {
-                for (int chunk = 0; chunk * p.CW < p.BN; ++chunk) {
-                    if (n0 + chunk * p.CW >= p.Cout) break;
-                    tma_store_4d(&tmO, smStage + (uint32_t)chunk * chunk_bytes, p.c_off + n0 + chunk * p.CW, w0, h0, i0);
-                }
-                tma_store_commit();
-            }
+            if (++as == 2) { as = 0; aph ^= 1u; }
         }
-        if (store_thread) tma_store_wait_all();
+    } else {
+        // ----------------------------------------------------------------- store issuer
+        if (lane == 0) {
+            const uint32_t slot_bytes = (uint32_t)TILE_M * (uint32_t)p.CW * 2u;
+            bool ok = true;
+            int sb = 0, pend = 0, fb = 0;       // next slot, stores whose slot is not yet released, next slot to release
+            uint32_t sph = 0;
+            TileCoord tc;
+            tile_first(p, blockIdx.x, tc);
+            for (int t = blockIdx.x; t < p.total_tiles && ok; t += gridDim.x, tile_next(p, tc)) {
+                const int w0 = tc.tw * p.BW, h0 = tc.th * p.BH, i0 = tc.ti * p.BI, n0 = tc.nt * p.BN;
+                for (int chunk = 0; chunk < nchunks; ++chunk) {
+                    const int c0 = chunk * p.CW;
+                    if (n0 + c0 >= p.Cout) break;
+                    if (!wait_bar(smem_u32(&sh->stg_full[sb]), sph, abort_flag, p.status)) { ok = false; break; }
+                    tma_store_4d(&tmO, smStg + (uint32_t)sb * slot_bytes, p.c_off + n0 + c0, w0, h0, i0);
+                    tma_store_commit();
+                    if (++sb == p.nstg) { sb = 0; sph ^= 1u; }
+                    // a slot is free again once its store has finished reading shared memory:
+                    // keep nstg-1 stores in flight, release the oldest
+                    if (++pend == p.nstg) {
+                        if (p.nstg == 4) asm volatile("cp.async.bulk.wait_group.read 3;" ::: "memory");
+                        else asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                        mbar_arrive(smem_u32(&sh->stg_free[fb]));
+                        if (++fb == p.nstg) fb = 0;
+                        --pend;
+                    }
+                }
+            }
+            tma_store_wait_all();
+        }
     }
 
     tc_fence_before();
@@ -466,16 +529,47 @@ int build_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_pt
     p.b_tile = ((unsigned)p.BN * row_bytes + 1023u) / 1024u * 1024u;
     p.a_bytes = (unsigned)rows * row_bytes;
     p.b_bytes = (unsigned)p.BN * row_bytes;
-    const size_t fixed = 1024 /*alignment slack*/ + (size_t)TILE_M * p.BN * 2 + 256 * sizeof(float) + sizeof(Shared) + 64;
-    int stages = (int)((SMEM_LIMIT - fixed) / (p.a_tile + p.b_tile));
+
+    // shared-memory budget: [A ring | B ring or resident kernels | staging ring | bias | control]
+    const int items = p.taps * p.chunks;
+    const size_t slot = (size_t)TILE_M * p.CW * 2;
+    const size_t bias_bytes = ((size_t)p.n_tiles * p.BN * sizeof(float) + 1023) / 1024 * 1024;
+    const size_t ctl_bytes = 1024;
+    static_assert(sizeof(Shared) <= 1024, "control block");
+    const size_t avail = SMEM_LIMIT - 1024 /*alignment slack*/ - bias_bytes - ctl_bytes;
+    p.nstg = slot <= 8192 ? 4 : 2;
+    const size_t stg_bytes = (size_t)p.nstg * slot;
+    const size_t b_all = (size_t)items * p.b_tile;
+    int stages = 0;
+    p.b_resident = 0;
+    if (p.n_tiles == 1 && b_all + stg_bytes + 3 * (size_t)p.a_tile <= avail) {
+        p.b_resident = 1;
+        stages = (int)((avail - b_all - stg_bytes) / p.a_tile);
+    } else {
+        if (stg_bytes + 2 * (size_t)(p.a_tile + p.b_tile) > avail) return SQN_ERR_UNSUPPORTED;
+        stages = (int)((avail - stg_bytes) / (p.a_tile + p.b_tile));
+    }
     if (stages > MAX_STAGES) stages = MAX_STAGES;
-    if (stages < 2) return SQN_ERR_UNSUPPORTED;
     p.stages = stages;
-    plan->smem = fixed + (size_t)stages * (p.a_tile + p.b_tile);
+    const size_t b_region = p.b_resident ? b_all : (size_t)stages * p.b_tile;
+    p.off_b = (unsigned)((size_t)stages * p.a_tile);
+    p.off_stg = p.off_b + (unsigned)b_region;
+    p.off_bias = p.off_stg + (unsigned)stg_bytes;
+    p.off_ctl = p.off_bias + (unsigned)bias_bytes;
+    plan->smem = 1024 + (size_t)p.off_ctl + ctl_bytes;
+    if (plan->smem > SMEM_LIMIT) return SQN_ERR_UNSUPPORTED;
 
     const long long total = (long long)p.tiles_w * p.tiles_h * p.tiles_i * p.n_tiles;
     if (total > 0x7fffffffLL) return SQN_ERR_UNSUPPORTED;
+    p.total_tiles = (int)total;
     plan->grid = (int)(total < num_sms() ? total : num_sms());
+    {
+        int g = plan->grid;
+        p.g_nt = g % p.n_tiles; g /= p.n_tiles;
+        p.g_tw = g % p.tiles_w; g /= p.tiles_w;
+        p.g_th = g % p.tiles_h; g /= p.tiles_h;
+        p.g_ti = g;
+    }
 
     // ---- tensor maps
     if (stem) {
