@@ -53,7 +53,12 @@ struct TcParams {
     int taps, taps_w, pad;           // kernel taps, taps per kernel row, zero padding
     int chunks, BKc;                 // reduction chunks per tap, elements per chunk (16/32/64)
     int k_per_tap;                   // reduction elements per tap in the kernel matrix
-    int stem;                        // 1: 7x7 stride-2 stem on the repacked input (tap = kernel row)
+    int patch;                       // 1: one input patch per tile serves every tap (see below)
+    int taps_h;                      // kernel rows
+    int tap_h_rows, tap_w_rows;      // patch rows to skip per kernel row / kernel column
+    int h_mul;                       // input rows per output row (2 for the stride-2 stem)
+    unsigned sbo_bytes;              // patch bytes between consecutive groups of 8 output pixels
+    unsigned patch_tile;             // shared-memory bytes reserved per reduction chunk of a patch
     int c_off;                       // first output layer inside the destination tensor
     int relu;
     int stages;                      // A (or A+B) ring slots
@@ -205,16 +210,25 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             tile_first(p, blockIdx.x, tc);
             for (int t = blockIdx.x; t < p.total_tiles && ok; t += gridDim.x, tile_next(p, tc)) {
                 const int w0 = tc.tw * p.BW, h0 = tc.th * p.BH, i0 = tc.ti * p.BI, n0 = tc.nt * p.BN;
+                if (p.patch) {
+                    // one box per reduction chunk covers the tile plus its halo; every tap reads from it
+                    if (!wait_bar(smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                    const uint32_t full = smem_u32(&sh->full[s]);
+                    mbar_arrive_expect_tx(full, p.a_bytes);
+                    for (int ch = 0; ch < p.chunks; ++ch)
+                        tma_load_5d(smA + (uint32_t)s * p.a_tile + (uint32_t)ch * p.patch_tile, &tmA, full, ch * p.BKc,
+                                    w0 - p.pad, h0 * p.h_mul - p.pad, i0, 0);
+                    ++issued;
+                    if (++s == p.stages) { s = 0; ph ^= 1u; }
+                    continue;
+                }
                 int tap = 0, kh = 0, kw = 0, ch = 0;
                 for (int i = 0; i < items; ++i) {
                     if (!wait_bar(smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
                     const uint32_t full = smem_u32(&sh->full[s]);
                     const int x = ch * p.BKc;
                     mbar_arrive_expect_tx(full, tx);
-                    if (p.stem)   // tap = kernel row kh = 2a + b: input rows are split into (pair, parity)
-                        tma_load_5d(smA + (uint32_t)s * p.a_tile, &tmA, full, 0, w0, h0 + (tap >> 1), tap & 1, i0);
-                    else
-                        tma_load_5d(smA + (uint32_t)s * p.a_tile, &tmA, full, x, w0 + kw - p.pad, h0 + kh - p.pad, i0, 0);
+                    tma_load_5d(smA + (uint32_t)s * p.a_tile, &tmA, full, x, w0 + kw - p.pad, h0 + kh - p.pad, i0, 0);
                     if (!p.b_resident)
                         tma_load_2d(smB + (uint32_t)s * p.b_tile, &tmB, full, tap * p.k_per_tap + x, n0);
                     ++issued;
@@ -252,11 +266,37 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (!wait_bar(smem_u32(&sh->tmem_empty[as]), aph ^ 1u, abort_flag, p.status)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(as * p.bn_pad);
+                if (p.patch) {
+                    if (!wait_bar(smem_u32(&sh->full[s]), ph, abort_flag, p.status)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t pbase = smA + (uint32_t)s * p.a_tile;
+                    int i = 0;
+                    for (int kh = 0; kh < p.taps_h; ++kh) {
+                        for (int kw = 0; kw < p.taps_w; ++kw) {
+                            // output pixel (g, j) of the tile reads patch row g*(rows per line) + j + this offset
+                            const uint32_t off = (uint32_t)(kh * p.tap_h_rows + kw * p.tap_w_rows) * row_bytes;
+                            for (int ch = 0; ch < p.chunks; ++ch, ++i) {
+                                const uint64_t adesc = make_kmajor_desc(pbase + (uint32_t)ch * p.patch_tile + off,
+                                                                        row_bytes, p.sbo_bytes);
+                                const uint64_t bdesc = make_kmajor_desc(smB + (uint32_t)i * p.b_tile, row_bytes,
+                                                                        8u * row_bytes);
+                                for (int k = 0; k < ksteps; ++k)
+                                    mma_bf16_ss(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
+                                                (i > 0 || k > 0) ? 1u : 0u);
+                            }
+                        }
+                    }
+                    mma_commit(smem_u32(&sh->empty[s]));
+                    if (++s == p.stages) { s = 0; ph ^= 1u; }
+                    mma_commit(smem_u32(&sh->tmem_full[as]));
+                    if (++as == 2) { as = 0; aph ^= 1u; }
+                    continue;
+                }
                 for (int i = 0; i < items; ++i) {
                     if (!wait_bar(smem_u32(&sh->full[s]), ph, abort_flag, p.status)) { ok = false; break; }
                     tc_fence_after();
-                    const uint64_t adesc = make_kmajor_desc(smA + (uint32_t)s * p.a_tile, row_bytes);
-                    const uint64_t bdesc = make_kmajor_desc(smB + (uint32_t)(p.b_resident ? i : s) * p.b_tile, row_bytes);
+                    const uint64_t adesc = make_kmajor_desc(smA + (uint32_t)s * p.a_tile, row_bytes, 8u * row_bytes);
+                    const uint64_t bdesc = make_kmajor_desc(smB + (uint32_t)(p.b_resident ? i : s) * p.b_tile, row_bytes, 8u * row_bytes);
                     for (int k = 0; k < ksteps; ++k) {
                         // 16 bf16 = 32 bytes further along the row: +2 in the (>>4) address field
                         mma_bf16_ss(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
@@ -484,38 +524,77 @@ int num_sms()
 
 // Builds tensor maps and kernel parameters.  For the stem, a_ptr / w_ptr are the repacked
 // tensors ([N][Hp][Wp][4] and [Cout][7][8][4]).
+// Shared-memory layout for one candidate (store chunk width, staging slots); returns the number
+// of A stages that fit (0 if the candidate does not fit at all).
+int fit_stages(TcParams& p, size_t a_tile, bool want_resident, int cw, int nstg, size_t* smem_bytes)
+{
+    const int items = p.taps * p.chunks;
+    const size_t slot = (size_t)TILE_M * cw * 2;
+    const size_t bias_bytes = ((size_t)p.n_tiles * p.BN * sizeof(float) + 1023) / 1024 * 1024;
+    const size_t ctl_bytes = 1024;
+    static_assert(sizeof(Shared) <= 1024, "control block");
+    if (SMEM_LIMIT < 1024 + bias_bytes + ctl_bytes) return 0;
+    const size_t avail = SMEM_LIMIT - 1024 /*alignment slack*/ - bias_bytes - ctl_bytes;
+    const size_t stg_bytes = (size_t)nstg * slot;
+    const size_t b_all = (size_t)items * p.b_tile;
+    int stages;
+    size_t b_region;
+    if (want_resident) {
+        if (p.n_tiles != 1 || b_all + stg_bytes + 2 * a_tile > avail) return 0;
+        stages = (int)((avail - b_all - stg_bytes) / a_tile);
+        if (stages > MAX_STAGES) stages = MAX_STAGES;
+        b_region = b_all;
+    } else {
+        if (stg_bytes + 2 * (a_tile + p.b_tile) > avail) return 0;
+        stages = (int)((avail - stg_bytes) / (a_tile + p.b_tile));
+        if (stages > MAX_STAGES) stages = MAX_STAGES;
+        b_region = (size_t)stages * p.b_tile;
+    }
+    p.b_resident = want_resident ? 1 : 0;
+    p.stages = stages;
+    p.CW = cw;
+    p.nstg = nstg;
+    p.a_tile = (unsigned)a_tile;
+    p.off_b = (unsigned)((size_t)stages * a_tile);
+    p.off_stg = p.off_b + (unsigned)b_region;
+    p.off_bias = p.off_stg + (unsigned)stg_bytes;
+    p.off_ctl = p.off_bias + (unsigned)bias_bytes;
+    *smem_bytes = 1024 + (size_t)p.off_ctl + ctl_bytes;
+    return stages;
+}
+
+// Tries the staging candidates in order of preference; true when one gives at least min_stages.
+bool choose_layout(TcParams& p, size_t a_tile, bool want_resident, int min_stages, size_t* smem_bytes)
+{
+    static const int cand[][2] = {{64, 2}, {32, 4}, {32, 2}, {16, 4}, {16, 2}};
+    for (const auto& c : cand) {
+        if (p.BN % c[0] != 0) continue;
+        if (fit_stages(p, a_tile, want_resident, c[0], c[1], smem_bytes) >= min_stages) return true;
+    }
+    return false;
+}
+
+// Builds tensor maps and kernel parameters.  For the stem, a_ptr / w_ptr are the repacked
+// tensors ([N][Hp][Wp][4] and [Cout][7][8][4]).
 int build_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_ptr, int Hp, int Wp, Plan* plan)
 {
     TcParams& p = plan->p;
     std::memset(&p, 0, sizeof(p));
-    p.stem = stem ? 1 : 0;
     p.Cout = d.Cout;
     p.c_off = d.out_c_offset;
     p.relu = d.relu;
     p.bias = d.bias;
     p.status = device_status_word();
+    p.h_mul = 1;
     if (stem) {
-        p.taps = 7; p.taps_w = 1; p.pad = 0; p.BKc = 32; p.chunks = 1; p.k_per_tap = 32;
+        p.taps = 7; p.taps_h = 7; p.taps_w = 1; p.pad = 0; p.BKc = 32; p.chunks = 1; p.k_per_tap = 32;
     } else {
-        p.taps = d.K * d.K; p.taps_w = d.K; p.pad = d.pad;
+        p.taps = d.K * d.K; p.taps_h = d.K; p.taps_w = d.K; p.pad = d.pad;
         p.BKc = d.Cin % 64 == 0 ? 64 : (d.Cin % 32 == 0 ? 32 : 16);
         p.chunks = d.Cin / p.BKc;
         p.k_per_tap = d.Cin;
     }
     const unsigned row_bytes = (unsigned)p.BKc * 2u;
-
-    // output-pixel tiling; a 1x1 layer is tiled over the flattened pixel index
-    const bool flat = !stem && d.K == 1 && d.pad == 0;
-    long long OWl = d.OW, OHl = d.OH, NIl = d.N;
-    if (flat) { OWl = (long long)d.N * d.OH * d.OW; OHl = 1; NIl = 1; }
-    if (OWl > 0x7fffffffLL) return SQN_ERR_UNSUPPORTED;
-    const int OW = (int)OWl, OH = (int)OHl, NI = (int)NIl;
-    if (flat) { p.BW = OW < TILE_M ? OW : TILE_M; p.BH = 1; p.BI = 1; }
-    else choose_box(OW, OH, NI, &p.BW, &p.BH, &p.BI);
-    p.tiles_w = (OW + p.BW - 1) / p.BW;
-    p.tiles_h = (OH + p.BH - 1) / p.BH;
-    p.tiles_i = (NI + p.BI - 1) / p.BI;
-    const int rows = p.BW * p.BH * p.BI;
 
     p.BN = d.Cout <= 256 ? d.Cout : 256;
     p.n_tiles = (d.Cout + p.BN - 1) / p.BN;
@@ -523,41 +602,60 @@ int build_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_pt
     unsigned cols = 32;
     while (cols < 2u * (unsigned)p.bn_pad) cols *= 2;
     p.tmem_cols = cols;
-    p.CW = p.BN % 64 == 0 ? 64 : (p.BN % 32 == 0 ? 32 : 16);
-
-    p.a_tile = (unsigned)TILE_M * row_bytes;
     p.b_tile = ((unsigned)p.BN * row_bytes + 1023u) / 1024u * 1024u;
-    p.a_bytes = (unsigned)rows * row_bytes;
     p.b_bytes = (unsigned)p.BN * row_bytes;
 
-    // shared-memory budget: [A ring | B ring or resident kernels | staging ring | bias | control]
-    const int items = p.taps * p.chunks;
-    const size_t slot = (size_t)TILE_M * p.CW * 2;
-    const size_t bias_bytes = ((size_t)p.n_tiles * p.BN * sizeof(float) + 1023) / 1024 * 1024;
-    const size_t ctl_bytes = 1024;
-    static_assert(sizeof(Shared) <= 1024, "control block");
-    const size_t avail = SMEM_LIMIT - 1024 /*alignment slack*/ - bias_bytes - ctl_bytes;
-    p.nstg = slot <= 8192 ? 4 : 2;
-    const size_t stg_bytes = (size_t)p.nstg * slot;
-    const size_t b_all = (size_t)items * p.b_tile;
-    int stages = 0;
-    p.b_resident = 0;
-    if (p.n_tiles == 1 && b_all + stg_bytes + 3 * (size_t)p.a_tile <= avail) {
-        p.b_resident = 1;
-        stages = (int)((avail - b_all - stg_bytes) / p.a_tile);
-    } else {
-        if (stg_bytes + 2 * (size_t)(p.a_tile + p.b_tile) > avail) return SQN_ERR_UNSUPPORTED;
-        stages = (int)((avail - stg_bytes) / (p.a_tile + p.b_tile));
+    // output-pixel tiling; a 1x1 layer is tiled over the flattened pixel index
+    const bool flat = !stem && d.K == 1 && d.pad == 0;
+    long long OWl = d.OW, OHl = d.OH, NIl = d.N;
+    if (flat) { OWl = (long long)d.N * d.OH * d.OW; OHl = 1; NIl = 1; }
+    if (OWl > 0x7fffffffLL) return SQN_ERR_UNSUPPORTED;
+    const int OW = (int)OWl, OH = (int)OHl, NI = (int)NIl;
+
+    // Patch mode (stem and KxK stride-1 layers whose kernels fit in shared memory): the tile is
+    // 8 output columns x BH <= 16 output rows of one image, so that each group of 8 MMA rows is a
+    // run of 8 consecutive patch rows and consecutive groups are a constant number of bytes apart.
+    int patch_w = 0, patch_h = 0;     // TMA box extents of the patch (lines of patch_w rows)
+    bool patch_ok = false;
+    if (!flat && p.n_tiles == 1) {
+        const int th = (OH + 15) / 16;
+        const int bh = (OH + th - 1) / th;
+        int max_rows;
+        if (stem) {
+            patch_w = 8; patch_h = 2 * bh + 5;
+            p.tap_h_rows = 8; p.tap_w_rows = 0; p.sbo_bytes = 16u * row_bytes; p.h_mul = 2;
+            max_rows = 15 * 16 + 8 + 6 * 8;
+        } else {
+            patch_w = 8 + d.K - 1; patch_h = bh + d.K - 1;
+            p.tap_h_rows = patch_w; p.tap_w_rows = 1; p.sbo_bytes = (unsigned)patch_w * row_bytes;
+            max_rows = 15 * patch_w + 8 + (d.K - 1) * patch_w + (d.K - 1);
+        }
+        if (max_rows < patch_w * patch_h) max_rows = patch_w * patch_h;
+        p.patch_tile = ((unsigned)max_rows * row_bytes + 1023u) / 1024u * 1024u;
+        if (patch_h <= 256 && p.sbo_bytes < (1u << 18) &&
+            choose_layout(p, (size_t)p.chunks * p.patch_tile, true, 2, &plan->smem)) {
+            patch_ok = true;
+            p.patch = 1;
+            p.BW = 8; p.BH = bh; p.BI = 1;
+            p.a_bytes = (unsigned)p.chunks * (unsigned)(patch_w * patch_h) * row_bytes;
+        }
     }
-    if (stages > MAX_STAGES) stages = MAX_STAGES;
-    p.stages = stages;
-    const size_t b_region = p.b_resident ? b_all : (size_t)stages * p.b_tile;
-    p.off_b = (unsigned)((size_t)stages * p.a_tile);
-    p.off_stg = p.off_b + (unsigned)b_region;
-    p.off_bias = p.off_stg + (unsigned)stg_bytes;
-    p.off_ctl = p.off_bias + (unsigned)bias_bytes;
-    plan->smem = 1024 + (size_t)p.off_ctl + ctl_bytes;
+    if (!patch_ok) {
+        if (stem) return SQN_ERR_UNSUPPORTED;
+        p.patch = 0;
+        p.h_mul = 1;
+        if (flat) { p.BW = OW < TILE_M ? OW : TILE_M; p.BH = 1; p.BI = 1; }
+        else choose_box(OW, OH, NI, &p.BW, &p.BH, &p.BI);
+        p.a_bytes = (unsigned)(p.BW * p.BH * p.BI) * row_bytes;
+        const size_t a_tile = (size_t)TILE_M * row_bytes;
+        if (!choose_layout(p, a_tile, true, 3, &plan->smem) && !choose_layout(p, a_tile, false, 3, &plan->smem) &&
+            !choose_layout(p, a_tile, false, 2, &plan->smem))
+            return SQN_ERR_UNSUPPORTED;
+    }
     if (plan->smem > SMEM_LIMIT) return SQN_ERR_UNSUPPORTED;
+    p.tiles_w = (OW + p.BW - 1) / p.BW;
+    p.tiles_h = (OH + p.BH - 1) / p.BH;
+    p.tiles_i = (NI + p.BI - 1) / p.BI;
 
     const long long total = (long long)p.tiles_w * p.tiles_h * p.tiles_i * p.n_tiles;
     if (total > 0x7fffffffLL) return SQN_ERR_UNSUPPORTED;
@@ -573,11 +671,12 @@ int build_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_pt
 
     // ---- tensor maps
     if (stem) {
-        // [32 window elements][OW windows, 16 B apart][row pairs][row parity][image]
+        // [32 window elements][OW windows, 16 B apart][input rows][image]: window ow of row y starts at
+        // pixel 2*ow, so consecutive windows overlap; the patch box is 8 windows x (2*BH+5) rows
         const cuuint64_t row_pitch = (cuuint64_t)Wp * 8;
-        cuuint64_t dims[5] = {32, (cuuint64_t)d.OW, (cuuint64_t)(Hp / 2), 2, (cuuint64_t)d.N};
-        cuuint64_t str[4] = {16, 2 * row_pitch, row_pitch, (cuuint64_t)Hp * row_pitch};
-        cuuint32_t box[5] = {32, (cuuint32_t)p.BW, (cuuint32_t)p.BH, 1, (cuuint32_t)p.BI};
+        cuuint64_t dims[5] = {32, (cuuint64_t)d.OW, (cuuint64_t)Hp, (cuuint64_t)d.N, 1};
+        cuuint64_t str[4] = {16, row_pitch, (cuuint64_t)Hp * row_pitch, (cuuint64_t)Hp * row_pitch * d.N};
+        cuuint32_t box[5] = {32, (cuuint32_t)patch_w, (cuuint32_t)patch_h, 1, 1};
         if (!encode(&plan->a, 5, a_ptr, dims, str, box, row_bytes)) return SQN_ERR_CUDA;
     } else if (flat) {
         cuuint64_t dims[5] = {(cuuint64_t)d.Cin, (cuuint64_t)OW, 1, 1, 1};
@@ -589,7 +688,8 @@ int build_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_pt
         cuuint64_t dims[5] = {(cuuint64_t)d.Cin, (cuuint64_t)d.W, (cuuint64_t)d.H, (cuuint64_t)d.N, 1};
         const cuuint64_t s1 = (cuuint64_t)d.Cin * 2;
         cuuint64_t str[4] = {s1, s1 * d.W, s1 * d.W * d.H, s1 * d.W * d.H * d.N};
-        cuuint32_t box[5] = {(cuuint32_t)p.BKc, (cuuint32_t)p.BW, (cuuint32_t)p.BH, (cuuint32_t)p.BI, 1};
+        cuuint32_t box[5] = {(cuuint32_t)p.BKc, (cuuint32_t)(p.patch ? patch_w : p.BW),
+                             (cuuint32_t)(p.patch ? patch_h : p.BH), (cuuint32_t)p.BI, 1};
         if (!encode(&plan->a, 5, a_ptr, dims, str, box, row_bytes)) return SQN_ERR_CUDA;
     }
     {

@@ -124,17 +124,20 @@ __device__ __forceinline__ void tmem_ld_x16(uint32_t taddr, uint32_t (&v)[16])
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor, K-major operand, rows of `row_bytes` (32, 64 or 128) bytes
-// stored with the TMA swizzle of the same width; groups of 8 rows are contiguous.
+// stored with the TMA swizzle of the same width.  Rows 0..7 of a group are consecutive;
+// group g starts `sbo_bytes` after group g-1 (8*row_bytes when the tile is dense).
 //   bits  0..13  start address >> 4        bits 32..45  stride between 8-row groups >> 4
 //   bits 16..29  leading offset (unused for swizzled K-major, set to 1)
 //   bits 46..47  descriptor version 1      bits 61..63  swizzle: 2 = 128B, 4 = 64B, 6 = 32B
-__device__ __forceinline__ uint64_t make_kmajor_desc(uint32_t smem_addr, uint32_t row_bytes)
+// The swizzle is a function of the absolute shared-memory address, so the start address may
+// be any whole number of rows into a TMA-written tile (base-offset field left at zero).
+__device__ __forceinline__ uint64_t make_kmajor_desc(uint32_t smem_addr, uint32_t row_bytes, uint32_t sbo_bytes)
 {
     const uint64_t layout = row_bytes == 128 ? 2ull : (row_bytes == 64 ? 4ull : 6ull);
     uint64_t d = 0;
     d |= (uint64_t)((smem_addr & 0x3ffffu) >> 4);
     d |= (uint64_t)1 << 16;
-    d |= (uint64_t)((8u * row_bytes) >> 4) << 32;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
     d |= (uint64_t)1 << 46;
     d |= layout << 61;
     return d;
