@@ -37,9 +37,12 @@ namespace {
 using namespace ptx;
 
 constexpr int TILE_M = 128;            // MMA M: TMEM lanes
-constexpr int NUM_THREADS = 224;       // producer, MMA, 4 epilogue warps, store issuer
+constexpr int NUM_THREADS = 352;       // producer, MMA, 8 epilogue warps, store issuer
+constexpr int EPI_WARPS = 8;
 constexpr int MAX_STAGES = 8;
 constexpr int MAX_STG = 4;             // staging ring slots
+constexpr int MAX_TAB = 448;           // MMAs per tile in patch mode
+constexpr size_t CTL_BYTES = 4096;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // about two seconds
 constexpr size_t SMEM_LIMIT = 227 * 1024;
 
@@ -84,23 +87,27 @@ struct Shared {                       // control block placed after the tiles
     unsigned long long stg_free[MAX_STG];
     unsigned tmem_base;
     volatile int abort_flag;
+    uint2 mma_tab[MAX_TAB];           // patch mode: per MMA, {A offset from the stage base, B address} in 16-byte units
 };
 
+// Bounded mbarrier wait.  Polls back to back at first (hand-offs between the roles take a few
+// hundred cycles), backs off with nanosleep on long waits, and gives up after WAIT_LIMIT_CYCLES:
+// the CTA then records SQN_ERR_TIMEOUT and every role leaves its loop.
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (uint32_t i = 1;; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 31u) == 0u) {
+        if ((i & 255u) == 0u) {
             if (*abort_flag) return false;
             if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
                 *abort_flag = 1;
                 if (status) atomicExch(status, (int)SQN_ERR_TIMEOUT);
                 return false;
             }
-            __nanosleep(40);
         }
+        if (i > 4096u) __nanosleep(128);
     }
 }
 
@@ -165,10 +172,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         mbar_init(smem_u32(&sh->b_full), 1);
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&sh->tmem_full[a]), 1);
-            mbar_init(smem_u32(&sh->tmem_empty[a]), 4);
+            mbar_init(smem_u32(&sh->tmem_empty[a]), EPI_WARPS);
         }
         for (int b = 0; b < p.nstg; ++b) {
-            mbar_init(smem_u32(&sh->stg_full[b]), 4);
+            mbar_init(smem_u32(&sh->stg_full[b]), EPI_WARPS);
             mbar_init(smem_u32(&sh->stg_free[b]), 1);
         }
         sh->abort_flag = 0;
@@ -183,6 +190,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     // bias of every output layer, once per CTA
     for (int c = threadIdx.x; c < p.n_tiles * p.BN; c += NUM_THREADS) bias_s[c] = c < p.Cout ? __ldg(p.bias + c) : 0.f;
+    if (p.patch) {
+        // operand addresses of every MMA of a tile, in issue order (tap-major, then chunk, then k-step)
+        const int ksteps = p.BKc / 16;
+        for (int e = threadIdx.x; e < items * ksteps; e += NUM_THREADS) {
+            const int k = e % ksteps, it = e / ksteps;
+            const int ch = it % p.chunks, tap = it / p.chunks;
+            const int kw = tap % p.taps_w, kh = tap / p.taps_w;
+            const uint32_t a_off = (uint32_t)ch * p.patch_tile + (uint32_t)(kh * p.tap_h_rows + kw * p.tap_w_rows) * row_bytes;
+            sh->mma_tab[e] = make_uint2((a_off >> 4) + 2u * k, ((smB + (uint32_t)it * p.b_tile) >> 4) + 2u * k);
+        }
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -255,9 +273,27 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
+        // One thread issues every MMA, so its loop is kept to a few adds per instruction: the
+        // descriptors' constant halves are built once and only the 14-bit address field (in
+        // 16-byte units) is advanced.
         if (lane == 0) {
             const uint32_t idesc = make_idesc_bf16(TILE_M, (uint32_t)p.BN);
             const int ksteps = p.BKc / 16;
+            const uint32_t hiA = (uint32_t)(make_kmajor_desc(0, row_bytes, p.patch ? p.sbo_bytes : 8u * row_bytes) >> 32);
+            const uint32_t hiB = (uint32_t)(make_kmajor_desc(0, row_bytes, 8u * row_bytes) >> 32);
+            const uint32_t a_tile16 = p.a_tile >> 4, b_tile16 = p.b_tile >> 4;
+            const uint32_t smA16 = smA >> 4, smB16 = smB >> 4;
+            auto issue = [&](uint32_t d_tmem, uint32_t a16, uint32_t b16, uint32_t acc) {
+                // ksteps MMAs of K = 16 (32 bytes = 2 address units along the row)
+                const uint64_t da = ((uint64_t)hiA << 32) | (uint64_t)(a16 | 0x10000u);
+                const uint64_t db = ((uint64_t)hiB << 32) | (uint64_t)(b16 | 0x10000u);
+                mma_bf16_ss(d_tmem, da, db, idesc, acc);
+                if (ksteps >= 2) mma_bf16_ss(d_tmem, da + 2, db + 2, idesc, 1u);
+                if (ksteps == 4) {
+                    mma_bf16_ss(d_tmem, da + 4, db + 4, idesc, 1u);
+                    mma_bf16_ss(d_tmem, da + 6, db + 6, idesc, 1u);
+                }
+            };
             bool ok = true;
             if (p.b_resident) ok = wait_bar(smem_u32(&sh->b_full), 0u, abort_flag, p.status);
             int s = 0, as = 0;
@@ -269,58 +305,54 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (p.patch) {
                     if (!wait_bar(smem_u32(&sh->full[s]), ph, abort_flag, p.status)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t pbase = smA + (uint32_t)s * p.a_tile;
-                    int i = 0;
-                    for (int kh = 0; kh < p.taps_h; ++kh) {
-                        for (int kw = 0; kw < p.taps_w; ++kw) {
-                            // output pixel (g, j) of the tile reads patch row g*(rows per line) + j + this offset
-                            const uint32_t off = (uint32_t)(kh * p.tap_h_rows + kw * p.tap_w_rows) * row_bytes;
-                            for (int ch = 0; ch < p.chunks; ++ch, ++i) {
-                                const uint64_t adesc = make_kmajor_desc(pbase + (uint32_t)ch * p.patch_tile + off,
-                                                                        row_bytes, p.sbo_bytes);
-                                const uint64_t bdesc = make_kmajor_desc(smB + (uint32_t)i * p.b_tile, row_bytes,
-                                                                        8u * row_bytes);
-                                for (int k = 0; k < ksteps; ++k)
-                                    mma_bf16_ss(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
-                                                (i > 0 || k > 0) ? 1u : 0u);
-                            }
-                        }
+                    // output pixel (g, j) of the tile reads patch row g*(rows per line) + j + tap offset;
+                    // the offsets were tabulated once, so each MMA costs a load, an add and the issue
+                    const uint32_t a_base = smA16 + (uint32_t)s * a_tile16;
+                    const int nmma = items * ksteps;
+                    {
+                        const uint2 o = sh->mma_tab[0];
+                        mma_bf16_ss(d_tmem, ((uint64_t)hiA << 32) | (uint64_t)((a_base + o.x) | 0x10000u),
+                                    ((uint64_t)hiB << 32) | (uint64_t)(o.y | 0x10000u), idesc, 0u);
+                    }
+#pragma unroll 4
+                    for (int e = 1; e < nmma; ++e) {
+                        const uint2 o = sh->mma_tab[e];
+                        mma_bf16_ss(d_tmem, ((uint64_t)hiA << 32) | (uint64_t)((a_base + o.x) | 0x10000u),
+                                    ((uint64_t)hiB << 32) | (uint64_t)(o.y | 0x10000u), idesc, 1u);
                     }
                     mma_commit(smem_u32(&sh->empty[s]));
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
-                    mma_commit(smem_u32(&sh->tmem_full[as]));
-                    if (++as == 2) { as = 0; aph ^= 1u; }
-                    continue;
-                }
-                for (int i = 0; i < items; ++i) {
-                    if (!wait_bar(smem_u32(&sh->full[s]), ph, abort_flag, p.status)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint64_t adesc = make_kmajor_desc(smA + (uint32_t)s * p.a_tile, row_bytes, 8u * row_bytes);
-                    const uint64_t bdesc = make_kmajor_desc(smB + (uint32_t)(p.b_resident ? i : s) * p.b_tile, row_bytes, 8u * row_bytes);
-                    for (int k = 0; k < ksteps; ++k) {
-                        // 16 bf16 = 32 bytes further along the row: +2 in the (>>4) address field
-                        mma_bf16_ss(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
-                                    (i > 0 || k > 0) ? 1u : 0u);
+                } else {
+                    uint32_t bres16 = smB16;
+                    for (int i = 0; i < items; ++i, bres16 += b_tile16) {
+                        if (!wait_bar(smem_u32(&sh->full[s]), ph, abort_flag, p.status)) { ok = false; break; }
+                        tc_fence_after();
+                        issue(d_tmem, smA16 + (uint32_t)s * a_tile16, p.b_resident ? bres16 : smB16 + (uint32_t)s * b_tile16,
+                              i > 0 ? 1u : 0u);
+                        mma_commit(smem_u32(&sh->empty[s]));        // slot free once these MMAs have read it
+                        if (++s == p.stages) { s = 0; ph ^= 1u; }
                     }
-                    mma_commit(smem_u32(&sh->empty[s]));        // slot free once these MMAs have read it
-                    if (++s == p.stages) { s = 0; ph ^= 1u; }
+                    if (!ok) break;
                 }
-                if (ok) mma_commit(smem_u32(&sh->tmem_full[as]));   // accumulator complete
+                mma_commit(smem_u32(&sh->tmem_full[as]));           // accumulator complete
                 if (++as == 2) { as = 0; aph ^= 1u; }
             }
         }
-    } else if (warp < 6) {
+    } else if (warp < 2 + EPI_WARPS) {
         // -------------------------------------------------------------------- epilogue
-        // One output pixel (TMEM lane) per thread.  Per chunk of CW layers: TMEM -> registers,
-        // + bias, ReLU, -> bf16, into a slot of the staging ring (TMA-swizzled rows); the store
-        // warp sends the slot to global memory while the next chunk is converted.
-        const int q = warp & 3;                        // TMEM lane quadrant this warp may read
+        // Eight warps: warp w reads TMEM lane quadrant w % 4 (one output pixel per thread) and, of
+        // every chunk of CW layers, the half (w - 2) / 4.  TMEM -> registers, + bias, ReLU, -> bf16,
+        // into a slot of the staging ring (TMA-swizzled rows); the store warp sends the slot to
+        // global memory while the next chunk is converted.
+        const int q = warp & 3;
+        const int half = (warp - 2) >> 2;
         const int row = q * 32 + lane;
         const uint32_t cw_bytes = (uint32_t)p.CW * 2u;
         const uint32_t slot_bytes = (uint32_t)TILE_M * cw_bytes;
         const uint32_t sw = cw_bytes == 128 ? (uint32_t)(row & 7)
                           : cw_bytes == 64 ? (uint32_t)((row >> 1) & 3) : (uint32_t)((row >> 2) & 1);
-        const int nld = p.CW / 16;
+        const int hc = p.CW / 2;                       // layers per thread per chunk: 8, 16 or 32
+        const int col_h = half * hc;
         bool ok = true;
         int as = 0, sb = 0;
         uint32_t aph = 0, sph = 0;
@@ -331,36 +363,47 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_full[as]), aph, abort_flag, p.status));
             if (!ok) break;
             tc_fence_after();
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * p.bn_pad);
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * p.bn_pad + col_h);
             for (int chunk = 0; chunk < nchunks; ++chunk) {
                 const int c0 = chunk * p.CW;
                 if (n0 + c0 >= p.Cout) break;
-                uint32_t v[64];
-#pragma unroll
-                for (int j = 0; j < 4; ++j)
-                    if (j < nld) tmem_ld_x16(taddr + (uint32_t)(c0 + 16 * j), *reinterpret_cast<uint32_t(*)[16]>(&v[16 * j]));
+                uint32_t v[32];
+                if (hc == 32) {
+                    tmem_ld_x16(taddr + (uint32_t)c0, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
+                    tmem_ld_x16(taddr + (uint32_t)(c0 + 16), *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
+                } else if (hc == 16) {
+                    tmem_ld_x16(taddr + (uint32_t)c0, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
+                } else {
+                    tmem_ld_x8(taddr + (uint32_t)c0, *reinterpret_cast<uint32_t(*)[8]>(&v[0]));
+                }
                 ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->stg_free[sb]), sph ^ 1u, abort_flag, p.status));
                 tmem_ld_wait();
                 if (!ok) break;
                 const uint32_t rbase = smStg + (uint32_t)sb * slot_bytes + (uint32_t)row * cw_bytes;
-                const float* bch = bias_s + n0 + c0;
+                const float4* bch = reinterpret_cast<const float4*>(bias_s + n0 + c0 + col_h);
+                const uint32_t u_h = (uint32_t)(col_h >> 3);           // first 16-byte unit of this half
+                // all bias loads first, then the arithmetic, then the stores: three independent batches
+                float4 bv[8];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    if (j < nld) {
-                        uint32_t o[8];
+                for (int j = 0; j < 8; ++j)
+                    if (4 * j < hc) bv[j] = bch[j];
+                uint32_t o[16];
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            float a = __uint_as_float(v[16 * j + 2 * e]) + bch[16 * j + 2 * e];
-                            float b = __uint_as_float(v[16 * j + 2 * e + 1]) + bch[16 * j + 2 * e + 1];
-                            if (p.relu) { a = fmaxf(a, 0.f); b = fmaxf(b, 0.f); }
-                            o[e] = pack_bf16x2(a, b);
-                        }
-                        const uint32_t a0 = rbase + ((((uint32_t)(2 * j)) ^ sw) << 4);
-                        const uint32_t a1 = rbase + ((((uint32_t)(2 * j + 1)) ^ sw) << 4);
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a0), "r"(o[0]), "r"(o[1]),
-                                     "r"(o[2]), "r"(o[3]) : "memory");
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a1), "r"(o[4]), "r"(o[5]),
-                                     "r"(o[6]), "r"(o[7]) : "memory");
+                for (int j = 0; j < 8; ++j) {
+                    if (4 * j < hc) {
+                        float f0 = __uint_as_float(v[4 * j + 0]) + bv[j].x, f1 = __uint_as_float(v[4 * j + 1]) + bv[j].y;
+                        float f2 = __uint_as_float(v[4 * j + 2]) + bv[j].z, f3 = __uint_as_float(v[4 * j + 3]) + bv[j].w;
+                        if (p.relu) { f0 = fmaxf(f0, 0.f); f1 = fmaxf(f1, 0.f); f2 = fmaxf(f2, 0.f); f3 = fmaxf(f3, 0.f); }
+                        o[2 * j] = pack_bf16x2(f0, f1);
+                        o[2 * j + 1] = pack_bf16x2(f2, f3);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {                           // 8 layers = one 16-byte unit
+                    if (8 * u < hc) {
+                        const uint32_t addr = rbase + (((u_h + (uint32_t)u) ^ sw) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(o[4 * u]), "r"(o[4 * u + 1]),
+                                     "r"(o[4 * u + 2]), "r"(o[4 * u + 3]));
                     }
                 }
                 fence_proxy_async_smem();             // staging rows visible to the TMA unit
@@ -397,6 +440,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     // keep nstg-1 stores in flight, release the oldest
                     if (++pend == p.nstg) {
                         if (p.nstg == 4) asm volatile("cp.async.bulk.wait_group.read 3;" ::: "memory");
+                        else if (p.nstg == 3) asm volatile("cp.async.bulk.wait_group.read 2;" ::: "memory");
                         else asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                         mbar_arrive(smem_u32(&sh->stg_free[fb]));
                         if (++fb == p.nstg) fb = 0;
@@ -531,8 +575,8 @@ int fit_stages(TcParams& p, size_t a_tile, bool want_resident, int cw, int nstg,
     const int items = p.taps * p.chunks;
     const size_t slot = (size_t)TILE_M * cw * 2;
     const size_t bias_bytes = ((size_t)p.n_tiles * p.BN * sizeof(float) + 1023) / 1024 * 1024;
-    const size_t ctl_bytes = 1024;
-    static_assert(sizeof(Shared) <= 1024, "control block");
+    const size_t ctl_bytes = CTL_BYTES;
+    static_assert(sizeof(Shared) <= CTL_BYTES, "control block");
     if (SMEM_LIMIT < 1024 + bias_bytes + ctl_bytes) return 0;
     const size_t avail = SMEM_LIMIT - 1024 /*alignment slack*/ - bias_bytes - ctl_bytes;
     const size_t stg_bytes = (size_t)nstg * slot;
@@ -566,7 +610,7 @@ int fit_stages(TcParams& p, size_t a_tile, bool want_resident, int cw, int nstg,
 // Tries the staging candidates in order of preference; true when one gives at least min_stages.
 bool choose_layout(TcParams& p, size_t a_tile, bool want_resident, int min_stages, size_t* smem_bytes)
 {
-    static const int cand[][2] = {{64, 2}, {32, 4}, {32, 2}, {16, 4}, {16, 2}};
+    static const int cand[][2] = {{64, 4}, {64, 3}, {32, 4}, {64, 2}, {32, 3}, {32, 2}, {16, 4}, {16, 2}};
     for (const auto& c : cand) {
         if (p.BN % c[0] != 0) continue;
         if (fit_stages(p, a_tile, want_resident, c[0], c[1], smem_bytes) >= min_stages) return true;
@@ -632,7 +676,7 @@ int build_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_pt
         }
         if (max_rows < patch_w * patch_h) max_rows = patch_w * patch_h;
         p.patch_tile = ((unsigned)max_rows * row_bytes + 1023u) / 1024u * 1024u;
-        if (patch_h <= 256 && p.sbo_bytes < (1u << 18) &&
+        if (patch_h <= 256 && p.sbo_bytes < (1u << 18) && p.taps * p.chunks * (p.BKc / 16) <= MAX_TAB &&
             choose_layout(p, (size_t)p.chunks * p.patch_tile, true, 2, &plan->smem)) {
             patch_ok = true;
             p.patch = 1;
