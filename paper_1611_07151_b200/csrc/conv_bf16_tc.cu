@@ -87,7 +87,7 @@ struct Shared {                       // control block placed after the tiles
     unsigned long long stg_free[MAX_STG];
     unsigned tmem_base;
     volatile int abort_flag;
-    uint2 mma_tab[MAX_TAB];           // patch mode: per MMA, {A offset from the stage base, B address} in 16-byte units
+    uint2 mma_tab[MAX_TAB + 1];           // patch mode: per MMA, {A offset from the stage base, B address} in 16-byte units
 };
 
 // Bounded mbarrier wait.  Polls back to back at first (hand-offs between the roles take a few
@@ -309,16 +309,15 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     // the offsets were tabulated once, so each MMA costs a load, an add and the issue
                     const uint32_t a_base = smA16 + (uint32_t)s * a_tile16;
                     const int nmma = items * ksteps;
-                    {
-                        const uint2 o = sh->mma_tab[0];
+                    uint2 o = sh->mma_tab[0];
+                    uint32_t acc = 0u;
+#pragma unroll 2
+                    for (int e = 1; e <= nmma; ++e) {
+                        const uint2 nxt = sh->mma_tab[e];            // one entry ahead (the table has a spare slot)
                         mma_bf16_ss(d_tmem, ((uint64_t)hiA << 32) | (uint64_t)((a_base + o.x) | 0x10000u),
-                                    ((uint64_t)hiB << 32) | (uint64_t)(o.y | 0x10000u), idesc, 0u);
-                    }
-#pragma unroll 4
-                    for (int e = 1; e < nmma; ++e) {
-                        const uint2 o = sh->mma_tab[e];
-                        mma_bf16_ss(d_tmem, ((uint64_t)hiA << 32) | (uint64_t)((a_base + o.x) | 0x10000u),
-                                    ((uint64_t)hiB << 32) | (uint64_t)(o.y | 0x10000u), idesc, 1u);
+                                    ((uint64_t)hiB << 32) | (uint64_t)(o.y | 0x10000u), idesc, acc);
+                        acc = 1u;
+                        o = nxt;
                     }
                     mma_commit(smem_u32(&sh->empty[s]));
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
