@@ -117,6 +117,36 @@ int fire_forward(const void* in, const void* w_sq, const void* b_sq, const void*
                  int Cin, int s, int e1, int e3, int H, int W, int batch, int dtype, void* stream);
 
 /*
+ * fire_forward for callers that must not allocate.  (The paper has no counterpart: this is a
+ * convenience of this library, not a step of the method.)
+ *
+ * Who needs it: code that runs where device memory can no longer be obtained -- a worker inside a
+ * serving process whose memory was handed out once at start-up and is owned by someone else, a
+ * plug-in or callback that is forbidden to call cudaMalloc because that call may synchronise the
+ * whole device under the host application's feet, or a process running under a fixed memory
+ * budget that is already spent.  Such a caller has its input, its kernels and its output, but
+ * nowhere to put the squeeze map that fire_forward wants in `squeeze_scratch`.
+ *
+ * This entry point computes exactly what fire_forward computes, with the squeeze map kept in a
+ * buffer built into the library image.  It calls no cudaMalloc/cudaFree and no allocating library
+ * routine, on the device or on the host (the bf16 path encodes its tensor maps on the stack on
+ * every call instead of caching them).
+ *
+ *   - Limit: batch*H*W*s elements of `dtype` must fit in 8 MiB (8388608 bytes), e.g. fire4 in fp32
+ *     up to batch 21.  Larger requests return SQN_ERR_WORKSPACE and launch nothing.
+ *   - Every GPU that loads the library carries those 8 MiB until the process exits.
+ *   - The first call on a device looks up the buffer's device address (cudaGetSymbolAddress, with
+ *     that device current) and keeps it; make that first call before any stream capture begins.
+ *   - All calls on a device share the one buffer, whatever their stream: two calls that overlap on
+ *     the GPU race on it.  Order them (same stream, or events).  Nothing needs clearing between
+ *     calls: every element the expands read is written by the squeeze of the same call.
+ * Arguments, layouts and dtype rules are those of fire_forward minus `squeeze_scratch`.
+ */
+int fire_forward_static(const void* in, const void* w_sq, const void* b_sq, const void* w_e1, const void* b_e1,
+                        const void* w_e3, const void* b_e3, void* out,
+                        int Cin, int s, int e1, int e3, int H, int W, int batch, int dtype, void* stream);
+
+/*
  * Max pooling 3x3, stride 2, no padding (paper Section III-E):
  *   out[n][h][w][c] = max_{i,j<3} in[n][2h+i][2w+j][c],  out extent (H-3)/2+1.
  */

@@ -39,6 +39,7 @@ SIGNATURES = {
     "conv_forward_ex": (_c_int, [_c_vp] * 4 + [_c_int] * 8 + [ctypes.POINTER(sqn_conv_opts)]),
     "conv_workspace_bytes": (_c_int, [_c_int] * 9 + [ctypes.POINTER(_c_sz)]),
     "fire_forward": (_c_int, [_c_vp] * 9 + [_c_int] * 8 + [_c_vp]),
+    "fire_forward_static": (_c_int, [_c_vp] * 8 + [_c_int] * 8 + [_c_vp]),
     "maxpool3x3s2_forward": (_c_int, [_c_vp, _c_vp] + [_c_int] * 5 + [_c_vp]),
     "avgpool_softmax_forward": (_c_int, [_c_vp] * 3 + [_c_int] * 5 + [_c_vp]),
     "squeezenet_create": (_c_int, [ctypes.POINTER(_c_vp), ctypes.POINTER(_c_vp), ctypes.POINTER(_c_vp), _c_int, _c_int]),
@@ -136,6 +137,14 @@ def fire_forward(inp, w_sq, b_sq, w_e1, b_e1, w_e3, b_e3, squeeze_scratch, out, 
     _check(lib().fire_forward(_p(inp), _p(w_sq), _p(b_sq), _p(w_e1), _p(b_e1), _p(w_e3), _p(b_e3),
                               _p(squeeze_scratch), _p(out), Cin, s, e1, e3, H, W, batch, dtype,
                               current_stream() if stream is None else stream), "fire_forward")
+
+
+def fire_forward_static(inp, w_sq, b_sq, w_e1, b_e1, w_e3, b_e3, out, Cin, s, e1, e3, H, W, batch, dtype, stream=None):
+    """fire_forward without a scratch argument: the squeeze map lives in an 8 MiB buffer inside the
+    library, so nothing is allocated.  For callers that cannot obtain device memory (see include/sqn.h)."""
+    _check(lib().fire_forward_static(_p(inp), _p(w_sq), _p(b_sq), _p(w_e1), _p(b_e1), _p(w_e3), _p(b_e3), _p(out),
+                                     Cin, s, e1, e3, H, W, batch, dtype,
+                                     current_stream() if stream is None else stream), "fire_forward_static")
 
 
 def maxpool3x3s2_forward(inp, out, C, H, W, batch, dtype, stream=None):

@@ -149,6 +149,59 @@ extern "C" int fire_forward(const void* in, const void* w_sq, const void* b_sq, 
     return run_conv(d3, dtype, nullptr, 0, st);
 }
 
+// ------------------------------------------------- fire layer without any allocation
+// Scratch for fire_forward_static: lives in the library image, one copy per GPU that loads it.
+constexpr size_t kStaticFireScratchBytes = (size_t)8 << 20;
+static __device__ __align__(256) unsigned char g_fire_static_scratch[kStaticFireScratchBytes];
+
+// Device address of the array above on the current device.  In host code the array's name is only a
+// handle for the runtime, not an address a kernel may use, so the address is looked up once per
+// device (with that device current) and remembered.
+static void* fire_static_scratch_ptr()
+{
+    static std::mutex mu;
+    static void* ptrs[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!ptrs[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_fire_static_scratch) != cudaSuccess) return nullptr;
+        ptrs[dev] = p;
+    }
+    return ptrs[dev];
+}
+
+extern "C" int fire_forward_static(const void* in, const void* w_sq, const void* b_sq, const void* w_e1,
+                                   const void* b_e1, const void* w_e3, const void* b_e3, void* out, int Cin, int s,
+                                   int e1, int e3, int H, int W, int batch, int dtype, void* stream)
+{
+    if (dtype != SQN_F32 && dtype != SQN_BF16) return SQN_ERR_BADARG;
+    if (e1 <= 0 || e3 <= 0 || s <= 0 || H <= 0 || W <= 0 || batch <= 0) return SQN_ERR_BADARG;
+    // the squeeze map must fit the built-in scratch
+    const unsigned long long need = (unsigned long long)batch * H * W * s * esize(dtype);
+    if (need > kStaticFireScratchBytes) return SQN_ERR_WORKSPACE;
+    void* scratch = fire_static_scratch_ptr();
+    if (!scratch) return SQN_ERR_CUDA;
+    ConvDesc dsq, d1, d3;
+    int rc = make_conv_desc(in, w_sq, b_sq, scratch, Cin, s, H, W, 1, 1, 0, batch, 1, 0, 0, &dsq);
+    if (rc != SQN_OK) return rc;
+    rc = make_conv_desc(scratch, w_e1, b_e1, out, s, e1, H, W, 1, 1, 0, batch, 1, 0, e1 + e3, &d1);
+    if (rc != SQN_OK) return rc;
+    rc = make_conv_desc(scratch, w_e3, b_e3, out, s, e3, H, W, 3, 1, 1, batch, 1, e1, e1 + e3, &d3);
+    if (rc != SQN_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const ConvDesc* seq[3] = {&dsq, &d1, &d3};
+    if (dtype == SQN_BF16)
+        for (const ConvDesc* d : seq)
+            if ((rc = conv_bf16_supported(*d)) != SQN_OK) return rc;
+    for (const ConvDesc* d : seq) {
+        rc = dtype == SQN_F32 ? launch_conv_f32(*d, st) : launch_conv_bf16_uncached(*d, st);
+        if (rc != SQN_OK) return rc;
+    }
+    return SQN_OK;
+}
+
 // ---------------------------------------------------------------------------- pooling
 extern "C" int maxpool3x3s2_forward(const void* in, void* out, int C, int H, int W, int batch, int dtype, void* stream)
 {

@@ -830,6 +830,16 @@ int launch_conv_bf16(const ConvDesc& d, cudaStream_t stream)
     return launch_plan(plan, stream);
 }
 
+// Same launch without touching the plan cache: the tensor maps are encoded into a stack object on
+// every call, so nothing is allocated on the host or on the device.
+int launch_conv_bf16_uncached(const ConvDesc& d, cudaStream_t stream)
+{
+    Plan plan;
+    const int rc = build_plan(d, false, d.in, d.w, 0, 0, &plan);
+    if (rc != SQN_OK) return rc;
+    return launch_plan(plan, stream);
+}
+
 size_t stem_bf16_workspace_bytes(int N, int H, int W, int Cout)
 {
     const int Hp = (H + 1) / 2 * 2, Wp = (W + 2) / 2 * 2;

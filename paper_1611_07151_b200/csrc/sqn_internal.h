@@ -32,6 +32,7 @@ int launch_conv_f32(const ConvDesc& d, cudaStream_t stream);
 // Returns SQN_ERR_UNSUPPORTED for shapes outside its family.
 int conv_bf16_supported(const ConvDesc& d);
 int launch_conv_bf16(const ConvDesc& d, cudaStream_t stream);
+int launch_conv_bf16_uncached(const ConvDesc& d, cudaStream_t stream);   // no plan cache, no allocation
 // Stem (7x7/2 on 3 layers): needs scratch for the repacked input and kernels.
 size_t stem_bf16_workspace_bytes(int N, int H, int W, int Cout);
 int launch_stem_pack_bf16(const ConvDesc& d, void* workspace, size_t workspace_bytes, cudaStream_t stream);
