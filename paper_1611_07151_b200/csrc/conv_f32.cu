@@ -34,7 +34,7 @@ __host__ __device__ constexpr int ld_for(int bn) { return bn <= 32 ? 32 : (bn <=
 __device__ __forceinline__ int swz(int k) { return ((k >> 2) & 3) << 3; }
 
 template <int BM, int BN, int VN, int QN, bool VEC>
-__global__ void __launch_bounds__(NTHREADS) conv_f32_kernel(const F32Params p)
+__global__ void __launch_bounds__(NTHREADS, 2) conv_f32_kernel(const F32Params p)
 {
     constexpr int TN = VN * QN;
     constexpr int TX = BN / TN;
