@@ -116,6 +116,13 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
+// max(.,0) and round-to-nearest-even conversion of two values in one instruction
+__device__ __forceinline__ uint32_t pack_relu_bf16x2(float lo, float hi)
+{
+    uint32_t d;
+    asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
 
 // Position of a tile in (output-layer tile, column tile, row tile, image tile) digits.  A CTA
 // walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...; the step is added digit by digit, so the
@@ -392,9 +399,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if (4 * j < hc) {
                         float f0 = __uint_as_float(v[4 * j + 0]) + bv[j].x, f1 = __uint_as_float(v[4 * j + 1]) + bv[j].y;
                         float f2 = __uint_as_float(v[4 * j + 2]) + bv[j].z, f3 = __uint_as_float(v[4 * j + 3]) + bv[j].w;
-                        if (p.relu) { f0 = fmaxf(f0, 0.f); f1 = fmaxf(f1, 0.f); f2 = fmaxf(f2, 0.f); f3 = fmaxf(f3, 0.f); }
-                        o[2 * j] = pack_bf16x2(f0, f1);
-                        o[2 * j + 1] = pack_bf16x2(f2, f3);
+                        if (p.relu) {
+                            o[2 * j] = pack_relu_bf16x2(f0, f1);
+                            o[2 * j + 1] = pack_relu_bf16x2(f2, f3);
+                        } else {
+                            o[2 * j] = pack_bf16x2(f0, f1);
+                            o[2 * j + 1] = pack_bf16x2(f2, f3);
+                        }
                     }
                 }
 #pragma unroll
@@ -463,22 +474,26 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 // ---------------------------------------------------------------------------- stem repack
 // Input [N][H][W][3] bf16 -> [N][Hp][Wp][4] bf16, zero in the fourth layer and in the padding
 // column/row, so that every pixel is 8 bytes and two pixels are one 16-byte TMA stride.
+// Each thread converts four consecutive pixels of a row (Wp is a multiple of 4 or handled by the tail test).
 __global__ void stem_pack_input(const __nv_bfloat16* __restrict__ in, uint2* __restrict__ out, int N, int H, int W,
                                 int Hp, int Wp)
 {
+    const int Wq = (Wp + 3) / 4;
     const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
-    const long long total = (long long)N * Hp * Wp;
+    const long long total = (long long)N * Hp * Wq;
     if (idx >= total) return;
-    const int x = (int)(idx % Wp);
-    const int y = (int)((idx / Wp) % Hp);
-    const long long n = idx / ((long long)Wp * Hp);
-    uint2 v = make_uint2(0u, 0u);
-    if (x < W && y < H) {
-        const unsigned short* src = reinterpret_cast<const unsigned short*>(in) + ((n * H + y) * W + x) * 3;
-        v.x = (unsigned)src[0] | ((unsigned)src[1] << 16);
-        v.y = (unsigned)src[2];
-    }
-    out[idx] = v;
+    const int x0 = (int)(idx % Wq) * 4;
+    const int y = (int)((idx / Wq) % Hp);
+    const long long n = idx / ((long long)Wq * Hp);
+    const unsigned short* src = reinterpret_cast<const unsigned short*>(in) + ((n * H + y) * W + x0) * 3;
+    unsigned short e[12];
+#pragma unroll
+    for (int j = 0; j < 12; ++j) e[j] = (y < H && x0 + j / 3 < W) ? __ldg(src + j) : (unsigned short)0;
+    uint2* dst = out + (n * Hp + y) * Wp + x0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+        if (x0 + q < Wp)
+            dst[q] = make_uint2((unsigned)e[3 * q] | ((unsigned)e[3 * q + 1] << 16), (unsigned)e[3 * q + 2]);
 }
 
 // Kernels [Cout][7][7][3] bf16 -> [Cout][7][8][4] bf16 (zero for the eighth column and fourth layer).
@@ -866,7 +881,7 @@ int launch_stem_pack_bf16(const ConvDesc& d, void* workspace, size_t workspace_b
     unsigned char* ws = static_cast<unsigned char*>(workspace);
     uint2* pin = reinterpret_cast<uint2*>(ws);
     unsigned short* pw = reinterpret_cast<unsigned short*>(ws + align_up((size_t)d.N * Hp * Wp * 8, 1024));
-    const long long total = (long long)d.N * Hp * Wp;
+    const long long total = (long long)d.N * Hp * ((Wp + 3) / 4);
     stem_pack_input<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(d.in), pin,
                                                                         d.N, d.H, d.W, Hp, Wp);
     stem_pack_weights<<<(d.Cout * 224 + 255) / 256, 256, 0, stream>>>(static_cast<const unsigned short*>(d.w), pw,
