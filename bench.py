@@ -167,6 +167,111 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def run_batch1(B, ws, bs, x_pinned, dtype, dev, iters=300):
+    """The paper's own regime: one image at a time.  Launch-latency bound (all tensors sit in L2); timed
+    as back-to-back launches and as replays of a CUDA graph captured around the same call."""
+    import torch
+    net1 = B.squeezenet_create(ws, bs, dtype, 1)
+    work = torch.empty(B.squeezenet_workspace_bytes(net1, 1), dtype=torch.uint8, device=dev)
+    x1 = x_pinned[:1].to(dev)
+    logits = torch.empty((1, 1000), dtype=torch.float32, device=dev)
+    probs = torch.empty((1, 1000), dtype=torch.float32, device=dev)
+    out = {"note": "batch 1, inputs and activations resident in L2 (hot)"}
+    for _ in range(5):
+        B.squeezenet_forward(net1, x1, logits, probs, work, 1)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        B.squeezenet_forward(net1, x1, logits, probs, work, 1)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    out["eager"] = {"images_per_s": 1e3 / ms, "latency_us": ms * 1e3}
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            B.squeezenet_forward(net1, x1, logits, probs, work, 1)
+            with torch.cuda.graph(g, stream=side):
+                B.squeezenet_forward(net1, x1, logits, probs, work, 1)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        for _ in range(5):
+            g.replay()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(iters):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / iters
+        out["cuda_graph"] = {"images_per_s": 1e3 / ms, "latency_us": ms * 1e3}
+    except Exception as exc:                      # graph capture is optional plumbing, not the product
+        out["cuda_graph"] = {"error": str(exc)[:200]}
+    assert B.sqn_check() == B.SQN_OK
+    B.squeezenet_destroy(net1)
+    return out
+
+
+def run_sweep(B):
+    """Every distinct SqueezeNet conv shape at batch 1, 16, 64, 256 in fp32 and bf16 (seed 4 recipe, values
+    drawn on the device): time per launch with CUDA events, L2 flushed before each timed launch."""
+    import torch
+    peaks = measured_peaks()
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    props = torch.cuda.get_device_properties(0)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(4)
+    seen, rows = set(), []
+    for name, cin, cout, k, s, pad, hw in synth.SQUEEZENET_CONVS:
+        key = (cin, cout, k, s, pad, hw)
+        if key in seen:
+            continue
+        seen.add(key)
+        oh = (hw + 2 * pad - k) // s + 1
+        for dtype, tag, es in ((B.SQN_F32, "f32", 4), (B.SQN_BF16, "bf16", 2)):
+            tdt = torch.float32 if dtype == B.SQN_F32 else torch.bfloat16
+            pipe_tf = peaks["bf16_tflops"] if dtype == B.SQN_BF16 else fp32_ffma_peak_tflops(
+                props.multi_processor_count, 1965.0)
+            for batch in (1, 16, 64, 256):
+                x = torch.rand((batch, hw, hw, cin), device=dev, generator=gen).to(tdt)
+                w = (torch.randn((cout, k, k, cin), device=dev, generator=gen) * (2.0 / (cin * k * k)) ** 0.5).to(tdt)
+                b = torch.randn((cout,), device=dev, generator=gen) * 0.01
+                out = torch.empty((batch, oh, oh, cout), device=dev, dtype=tdt)
+                nb = B.conv_workspace_bytes(cin, cout, hw, hw, k, s, pad, batch, dtype)
+                wsb = torch.empty(max(nb, 16), dtype=torch.uint8, device=dev)
+
+                def call():
+                    B.conv_forward_ex(x, w, b, out, cin, cout, hw, hw, k, s, pad, batch, dtype=dtype, workspace=wsb,
+                                      workspace_bytes=nb)
+                for _ in range(3):
+                    call()
+                times = []
+                for _ in range(10):
+                    flush.zero_()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    call()
+                    e1.record()
+                    torch.cuda.synchronize()
+                    times.append(e0.elapsed_time(e1))
+                ms = float(np.median(times))
+                flops = 2.0 * batch * oh * oh * cout * cin * k * k
+                byts = es * batch * (hw * hw * cin + oh * oh * cout) + es * cout * cin * k * k + 4 * cout
+                t_hbm, t_pipe = byts / (peaks["hbm_gbs"] * 1e9), flops / (pipe_tf * 1e12)
+                rows.append({"layer": name, "dtype": tag, "batch": batch, "ms": ms, "tflops": flops / ms / 1e9,
+                             "gbs": byts / ms / 1e6, "bound": "hbm" if t_hbm >= t_pipe else ("tensor" if tag == "bf16" else "alu"),
+                             "frac": max(t_hbm, t_pipe) / (ms * 1e-3)})
+                del x, w, out
+    assert B.sqn_check() == B.SQN_OK
+    print(json.dumps({"sweep": rows, "peaks": peaks,
+                      "note": "bf16 stem time includes its repack launches; one launch, L2 flushed, median of 10"}))
+
+
 def workload_name(args):
     return "squeezenet_v1.0_forward_b%d_%s" % (args.batch, args.dtype)
 
@@ -182,6 +287,8 @@ def main():
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"])
     ap.add_argument("--e2e-steps", type=int, default=0, help="steps of the host-buffer loop (0: min(steps, 50))")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-batch1", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="per-layer sweep of every conv shape instead of the network")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -192,6 +299,10 @@ def main():
 
     import torch
     from paper_1611_07151_b200 import binding as B
+
+    if args.sweep:
+        run_sweep(B)
+        return
 
     rank, local_rank, world = D.env_world()
     torch.cuda.set_device(local_rank)
@@ -306,6 +417,10 @@ def main():
     d2h = 2 * batch * 1000 * 4
     assert abs(float(out_host[1].sum()) - batch) < 1e-2 * batch     # probabilities came back
 
+    batch1 = None
+    if rank == 0 and world == 1 and not args.no_batch1:
+        batch1 = run_batch1(B, ws, bs, x_pinned, dtype, dev)
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v1, cores = oracle_images_per_s(1, 3)
@@ -328,6 +443,7 @@ def main():
                 "gpu_launches": int(gpu_launches),
                 "roofline": roof,
                 "cpu_baseline": cpu,
+                "batch1": batch1,
                 "layers": [{k: (round(v, 6) if isinstance(v, float) else v) for k, v in l.items()} for l in layers]}
         print(json.dumps(line), flush=True)
     B.squeezenet_destroy(net)
