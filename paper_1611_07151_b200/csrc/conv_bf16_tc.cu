@@ -37,14 +37,17 @@ namespace {
 using namespace ptx;
 
 constexpr int TILE_M = 128;            // MMA M: TMEM lanes
-constexpr int NUM_THREADS = 352;       // producer, MMA, 8 epilogue warps, store issuer
-constexpr int EPI_WARPS = 8;
+// Threads per CTA: producer warp, MMA warp, 4*HALVES epilogue warps, store warp.  HALVES = 2: one CTA per SM
+// (large tiles, kernels resident in up to 227 KB); HALVES = 1: two lighter CTAs per SM, i.e. two MMA issuers,
+// two producers and two store threads per SM, for the layers whose tiles are small.
+__host__ __device__ constexpr int threads_for(int halves) { return 96 + 128 * halves; }
 constexpr int MAX_STAGES = 8;
 constexpr int MAX_STG = 4;             // staging ring slots
 constexpr int MAX_TAB = 448;           // MMAs per tile in patch mode
 constexpr size_t CTL_BYTES = 4096;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // about two seconds
 constexpr size_t SMEM_LIMIT = 227 * 1024;
+constexpr size_t SMEM_LIMIT_2CTA = 113 * 1024;     // two CTAs share an SM's 228 KB (1 KB reserved each)
 
 struct TcParams {
     int tiles_w, tiles_h, tiles_i;   // output-pixel tiles: columns, rows, images
@@ -150,10 +153,13 @@ __device__ __forceinline__ void tile_next(const TcParams& p, TileCoord& c)
     c.ti += p.g_ti + carry;
 }
 
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+template <int HALVES>
+__global__ void __launch_bounds__(threads_for(HALVES), 3 - HALVES)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmO, const TcParams p)
 {
+    constexpr int NUM_THREADS = threads_for(HALVES);
+    constexpr int EPI_WARPS = 4 * HALVES;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -351,14 +357,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // into a slot of the staging ring (TMA-swizzled rows); the store warp sends the slot to
         // global memory while the next chunk is converted.
         const int q = warp & 3;
-        const int half = (warp - 2) >> 2;
+        constexpr int NH = 2 / HALVES;                 // half-chunks each thread converts per chunk
+        const int half0 = ((warp - 2) >> 2) * NH;      // first half-chunk of this warp (0 when HALVES == 1)
         const int row = q * 32 + lane;
         const uint32_t cw_bytes = (uint32_t)p.CW * 2u;
         const uint32_t slot_bytes = (uint32_t)TILE_M * cw_bytes;
         const uint32_t sw = cw_bytes == 128 ? (uint32_t)(row & 7)
                           : cw_bytes == 64 ? (uint32_t)((row >> 1) & 3) : (uint32_t)((row >> 2) & 1);
-        const int hc = p.CW / 2;                       // layers per thread per chunk: 8, 16 or 32
-        const int col_h = half * hc;
+        const int hc = p.CW / 2;                       // layers per half-chunk: 8, 16 or 32
         bool ok = true;
         int as = 0, sb = 0;
         uint32_t aph = 0, sph = 0;
@@ -369,51 +375,59 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_full[as]), aph, abort_flag, p.status));
             if (!ok) break;
             tc_fence_after();
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * p.bn_pad + col_h);
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * p.bn_pad);
             for (int chunk = 0; chunk < nchunks; ++chunk) {
                 const int c0 = chunk * p.CW;
                 if (n0 + c0 >= p.Cout) break;
-                uint32_t v[32];
-                if (hc == 32) {
-                    tmem_ld_x16(taddr + (uint32_t)c0, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
-                    tmem_ld_x16(taddr + (uint32_t)(c0 + 16), *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
-                } else if (hc == 16) {
-                    tmem_ld_x16(taddr + (uint32_t)c0, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
-                } else {
-                    tmem_ld_x8(taddr + (uint32_t)c0, *reinterpret_cast<uint32_t(*)[8]>(&v[0]));
+                uint32_t v[NH][32];
+#pragma unroll
+                for (int h = 0; h < NH; ++h) {
+                    const uint32_t ta = taddr + (uint32_t)(c0 + (half0 + h) * hc);
+                    if (hc == 32) {
+                        tmem_ld_x16(ta, *reinterpret_cast<uint32_t(*)[16]>(&v[h][0]));
+                        tmem_ld_x16(ta + 16u, *reinterpret_cast<uint32_t(*)[16]>(&v[h][16]));
+                    } else if (hc == 16) {
+                        tmem_ld_x16(ta, *reinterpret_cast<uint32_t(*)[16]>(&v[h][0]));
+                    } else {
+                        tmem_ld_x8(ta, *reinterpret_cast<uint32_t(*)[8]>(&v[h][0]));
+                    }
                 }
                 ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->stg_free[sb]), sph ^ 1u, abort_flag, p.status));
                 tmem_ld_wait();
                 if (!ok) break;
                 const uint32_t rbase = smStg + (uint32_t)sb * slot_bytes + (uint32_t)row * cw_bytes;
-                const float4* bch = reinterpret_cast<const float4*>(bias_s + n0 + c0 + col_h);
-                const uint32_t u_h = (uint32_t)(col_h >> 3);           // first 16-byte unit of this half
-                // all bias loads first, then the arithmetic, then the stores: three independent batches
-                float4 bv[8];
 #pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    if (4 * j < hc) bv[j] = bch[j];
-                uint32_t o[16];
+                for (int h = 0; h < NH; ++h) {
+                    const int col_h = (half0 + h) * hc;
+                    const float4* bch = reinterpret_cast<const float4*>(bias_s + n0 + c0 + col_h);
+                    const uint32_t u_h = (uint32_t)(col_h >> 3);       // first 16-byte unit of this half-chunk
+                    // all bias loads first, then the arithmetic, then the stores: three independent batches
+                    float4 bv[8];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    if (4 * j < hc) {
-                        float f0 = __uint_as_float(v[4 * j + 0]) + bv[j].x, f1 = __uint_as_float(v[4 * j + 1]) + bv[j].y;
-                        float f2 = __uint_as_float(v[4 * j + 2]) + bv[j].z, f3 = __uint_as_float(v[4 * j + 3]) + bv[j].w;
-                        if (p.relu) {
-                            o[2 * j] = pack_relu_bf16x2(f0, f1);
-                            o[2 * j + 1] = pack_relu_bf16x2(f2, f3);
-                        } else {
-                            o[2 * j] = pack_bf16x2(f0, f1);
-                            o[2 * j + 1] = pack_bf16x2(f2, f3);
+                    for (int j = 0; j < 8; ++j)
+                        if (4 * j < hc) bv[j] = bch[j];
+                    uint32_t o[16];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        if (4 * j < hc) {
+                            float f0 = __uint_as_float(v[h][4 * j + 0]) + bv[j].x, f1 = __uint_as_float(v[h][4 * j + 1]) + bv[j].y;
+                            float f2 = __uint_as_float(v[h][4 * j + 2]) + bv[j].z, f3 = __uint_as_float(v[h][4 * j + 3]) + bv[j].w;
+                            if (p.relu) {
+                                o[2 * j] = pack_relu_bf16x2(f0, f1);
+                                o[2 * j + 1] = pack_relu_bf16x2(f2, f3);
+                            } else {
+                                o[2 * j] = pack_bf16x2(f0, f1);
+                                o[2 * j + 1] = pack_bf16x2(f2, f3);
+                            }
                         }
                     }
-                }
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {                           // 8 layers = one 16-byte unit
-                    if (8 * u < hc) {
-                        const uint32_t addr = rbase + (((u_h + (uint32_t)u) ^ sw) << 4);
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(o[4 * u]), "r"(o[4 * u + 1]),
-                                     "r"(o[4 * u + 2]), "r"(o[4 * u + 3]));
+                    for (int u = 0; u < 4; ++u) {                       // 8 layers = one 16-byte unit
+                        if (8 * u < hc) {
+                            const uint32_t addr = rbase + (((u_h + (uint32_t)u) ^ sw) << 4);
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(o[4 * u]),
+                                         "r"(o[4 * u + 1]), "r"(o[4 * u + 2]), "r"(o[4 * u + 3]));
+                        }
                     }
                 }
                 fence_proxy_async_smem();             // staging rows visible to the TMA unit
@@ -565,6 +579,7 @@ struct Plan {
     CUtensorMap a, b, o;
     TcParams p;
     int grid;
+    int halves;      // kernel variant: 1 = two light CTAs per SM, 2 = one CTA per SM
     size_t smem;
 };
 
@@ -584,8 +599,11 @@ int num_sms()
 // tensors ([N][Hp][Wp][4] and [Cout][7][8][4]).
 // Shared-memory layout for one candidate (store chunk width, staging slots); returns the number
 // of A stages that fit (0 if the candidate does not fit at all).
+thread_local size_t t_smem_limit = SMEM_LIMIT;   // budget the layout search below works against
+
 int fit_stages(TcParams& p, size_t a_tile, bool want_resident, int cw, int nstg, size_t* smem_bytes)
 {
+    const size_t SMEM_LIMIT = t_smem_limit;
     const int items = p.taps * p.chunks;
     const size_t slot = (size_t)TILE_M * cw * 2;
     const size_t bias_bytes = ((size_t)p.n_tiles * p.BN * sizeof(float) + 1023) / 1024 * 1024;
@@ -634,10 +652,13 @@ bool choose_layout(TcParams& p, size_t a_tile, bool want_resident, int min_stage
 
 // Builds tensor maps and kernel parameters.  For the stem, a_ptr / w_ptr are the repacked
 // tensors ([N][Hp][Wp][4] and [Cout][7][8][4]).
-int build_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_ptr, int Hp, int Wp, Plan* plan)
+int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_ptr, int Hp, int Wp, int halves,
+                   Plan* plan)
 {
     TcParams& p = plan->p;
     std::memset(&p, 0, sizeof(p));
+    plan->halves = halves;
+    t_smem_limit = halves == 1 ? SMEM_LIMIT_2CTA : SMEM_LIMIT;
     p.Cout = d.Cout;
     p.c_off = d.out_c_offset;
     p.relu = d.relu;
@@ -660,6 +681,7 @@ int build_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_pt
     unsigned cols = 32;
     while (cols < 2u * (unsigned)p.bn_pad) cols *= 2;
     p.tmem_cols = cols;
+    if (halves == 1 && cols > 256) return SQN_ERR_UNSUPPORTED;     // two CTAs share the SM's 512 TMEM columns
     p.b_tile = ((unsigned)p.BN * row_bytes + 1023u) / 1024u * 1024u;
     p.b_bytes = (unsigned)p.BN * row_bytes;
 
@@ -710,7 +732,7 @@ int build_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_pt
             !choose_layout(p, a_tile, false, 2, &plan->smem))
             return SQN_ERR_UNSUPPORTED;
     }
-    if (plan->smem > SMEM_LIMIT) return SQN_ERR_UNSUPPORTED;
+    if (plan->smem > t_smem_limit) return SQN_ERR_UNSUPPORTED;
     p.tiles_w = (OW + p.BW - 1) / p.BW;
     p.tiles_h = (OH + p.BH - 1) / p.BH;
     p.tiles_i = (NI + p.BI - 1) / p.BI;
@@ -718,7 +740,8 @@ int build_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_pt
     const long long total = (long long)p.tiles_w * p.tiles_h * p.tiles_i * p.n_tiles;
     if (total > 0x7fffffffLL) return SQN_ERR_UNSUPPORTED;
     p.total_tiles = (int)total;
-    plan->grid = (int)(total < num_sms() ? total : num_sms());
+    const long long ctas = (long long)num_sms() * (halves == 1 ? 2 : 1);
+    plan->grid = (int)(total < ctas ? total : ctas);
     {
         int g = plan->grid;
         p.g_nt = g % p.n_tiles; g /= p.n_tiles;
@@ -769,15 +792,35 @@ int build_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_pt
     return SQN_OK;
 }
 
+// Two light CTAs per SM when the layer's tiles, kernels and accumulators fit twice; else one CTA per SM.
+int build_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_ptr, int Hp, int Wp, Plan* plan)
+{
+    // Measured on B200 over the SqueezeNet shapes: the light variant wins where one MMA thread per SM is the
+    // limit (many small MMAs per tile, short epilogue): patch-mode layers up to 64 output layers and 1x1
+    // layers up to 32 output layers with at least three MMAs per tile.  Elsewhere the deeper rings win.
+    if (build_plan_cfg(d, stem, a_ptr, w_ptr, Hp, Wp, 1, plan) == SQN_OK) {
+        const TcParams& p = plan->p;
+        const int nmma = p.taps * p.chunks * (p.BKc / 16);
+        if ((p.patch && p.BN <= 64) || (!p.patch && p.BN <= 32 && nmma >= 3)) return SQN_OK;
+    }
+    return build_plan_cfg(d, stem, a_ptr, w_ptr, Hp, Wp, 2, plan);
+}
+
 int launch_plan(const Plan& plan, cudaStream_t stream)
 {
     static std::once_flag once;
     static cudaError_t attr_rc = cudaSuccess;
     std::call_once(once, [] {
-        attr_rc = cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
+        attr_rc = cudaFuncSetAttribute(conv_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
+        if (attr_rc == cudaSuccess)
+            attr_rc = cudaFuncSetAttribute(conv_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)SMEM_LIMIT_2CTA);
     });
     if (attr_rc != cudaSuccess) return SQN_ERR_CUDA;
-    conv_tc_kernel<<<plan.grid, NUM_THREADS, plan.smem, stream>>>(plan.a, plan.b, plan.o, plan.p);
+    if (plan.halves == 1)
+        conv_tc_kernel<1><<<plan.grid, threads_for(1), plan.smem, stream>>>(plan.a, plan.b, plan.o, plan.p);
+    else
+        conv_tc_kernel<2><<<plan.grid, threads_for(2), plan.smem, stream>>>(plan.a, plan.b, plan.o, plan.p);
     note_launch();
     return cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
 }
