@@ -63,6 +63,9 @@ def launch_work(batch, es):
     work["head"] = {"flops": 0.0, "bytes": float(batch * (es * 1000 * 169 + 8 * 1000))}
     # repack of the stem's input (3 -> 4 layers, padded rows): an extra pass, counted at its real traffic
     work["conv1_pack"] = {"flops": 0.0, "bytes": float(batch * (IMG * IMG * 3 * 2 + 228 * 228 * 8))}
+    # stem with its max-pool fused: the 96x111x111 map is never stored, only the pooled 96x55x55 one
+    work["conv1+pool1"] = {"flops": work["conv1"]["flops"],
+                           "bytes": float(es * batch * (IMG * IMG * 3 + 55 * 55 * 96) + es * 96 * 147 + 4 * 96)}
     return work
 
 

@@ -73,6 +73,10 @@ int conv_forward(const void* in, const void* weights, const void* bias, void* ou
  *   stream         cudaStream_t
  *   workspace,
  *   workspace_bytes  device scratch, needed only when conv_workspace_bytes reports > 0
+ *   fuse_maxpool   the 3x3 / stride 2 max-pool that follows the layer (paper Section III-E) is applied inside the
+ *                  kernel and only the pooled map is written: out is [batch][(outH-3)/2+1][(outW-3)/2+1][out_c_total].
+ *                  SQN_BF16 only, K >= 2 (or the stem shape), numOutputLayers a multiple of 32 up to 256, kernels
+ *                  small enough to stay in shared memory; otherwise SQN_ERR_UNSUPPORTED.
  */
 typedef struct {
     int dtype;
@@ -82,6 +86,7 @@ typedef struct {
     void* stream;
     void* workspace;
     size_t workspace_bytes;
+    int fuse_maxpool;   /* non-zero: out receives maxpool3x3/stride2 of the layer's output, extent ((outH-3)/2+1) */
 } sqn_conv_opts;
 
 /*
@@ -181,7 +186,8 @@ int avgpool_softmax_forward(const void* in, void* logits_f32, void* probs_f32, i
  * squeezenet_layer_output: after a forward with the same workspace and batch,
  *   gives the device address, layer count and extent of a named intermediate
  *   ("conv1", "pool1", "fire2_sq", "fire2", ..., "pool8", "fire9", "conv10");
- *   the data is in the net's dtype, NHWC, valid until the next forward.
+ *   the data is in the net's dtype, NHWC, valid until the next forward.  A bf16 net computes conv1 and
+ *   pool1 in one kernel and never stores conv1's map: asking for "conv1" returns SQN_ERR_UNSUPPORTED.
  */
 typedef struct sqn_net sqn_net;
 int squeezenet_create(sqn_net** net, const void* const* weights26, const void* const* bias26, int dtype,

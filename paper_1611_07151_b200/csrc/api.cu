@@ -67,6 +67,7 @@ int make_conv_desc(const void* in, const void* w, const void* bias, void* out, i
     d->N = batch; d->Cin = Cin; d->H = H; d->W = W; d->Cout = Cout; d->K = K; d->S = S; d->pad = pad;
     d->OH = out_extent(H, K, S, pad); d->OW = out_extent(W, K, S, pad);
     d->out_c_offset = c_off; d->out_c_total = c_total; d->relu = relu ? 1 : 0;
+    d->pool = 0;
     return SQN_OK;
 }
 
@@ -74,7 +75,7 @@ inline bool is_stem_shape(const ConvDesc& d) { return d.K == 7 && d.S == 2 && d.
 
 int run_conv(const ConvDesc& d, int dtype, void* ws, size_t ws_bytes, cudaStream_t stream)
 {
-    if (dtype == SQN_F32) return launch_conv_f32(d, stream);
+    if (dtype == SQN_F32) return d.pool ? SQN_ERR_UNSUPPORTED : launch_conv_f32(d, stream);
     if (dtype != SQN_BF16) return SQN_ERR_BADARG;
     if (is_stem_shape(d)) {
         const int rc = launch_stem_pack_bf16(d, ws, ws_bytes, stream);
@@ -103,6 +104,10 @@ extern "C" int conv_forward_ex(const void* in, const void* weights, const void* 
     const int rc = make_conv_desc(in, weights, bias, out, numInputLayers, numOutputLayers, H, W, K, S, pad, batch,
                                   o.relu, o.out_c_offset, o.out_c_total, &d);
     if (rc != SQN_OK) return rc;
+    if (o.fuse_maxpool) {
+        if (d.OH < 3 || d.OW < 3) return SQN_ERR_BADARG;
+        d.pool = 1;
+    }
     return run_conv(d, o.dtype, o.workspace, o.workspace_bytes, static_cast<cudaStream_t>(o.stream));
 }
 
@@ -331,6 +336,7 @@ extern "C" int squeezenet_layer_output(const sqn_net* net, const char* name, voi
     if (!net || !name || !workspace || !ptr || batch <= 0 || batch > net->max_batch) return SQN_ERR_BADARG;
     const int i = find_slot(net, name);
     if (i < 0) return SQN_ERR_BADARG;
+    if (net->dtype == SQN_BF16 && std::strcmp(name, "conv1") == 0) return SQN_ERR_UNSUPPORTED;   // fused with pool1
     std::vector<size_t> offs;
     layout(net, batch, &offs, nullptr);
     *ptr = static_cast<char*>(workspace) + offs[i];
@@ -388,18 +394,23 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
     int rc;
     ConvDesc d;
     // conv1 7x7/2 + ReLU, then max-pool
-    rc = make_conv_desc(in_nhwc, net->w[0], net->b[0], buf("conv1"), 3, 96, IMG, IMG, 7, 2, 0, batch, 1, 0, 0, &d);
-    if (rc != SQN_OK) return rc;
     if (dt == SQN_BF16) {
+        // stem and its max-pool in one kernel: the 96x111x111 map never goes to memory
+        rc = make_conv_desc(in_nhwc, net->w[0], net->b[0], buf("pool1"), 3, 96, IMG, IMG, 7, 2, 0, batch, 1, 0, 0, &d);
+        if (rc != SQN_OK) return rc;
+        d.pool = 1;
         if ((rc = launch_stem_pack_bf16(d, ws + stem_off, total - stem_off, st)) != SQN_OK) return rc;
         mark("conv1_pack");
         if ((rc = launch_stem_conv_bf16(d, ws + stem_off, total - stem_off, st)) != SQN_OK) return rc;
+        mark("conv1+pool1");
     } else {
+        rc = make_conv_desc(in_nhwc, net->w[0], net->b[0], buf("conv1"), 3, 96, IMG, IMG, 7, 2, 0, batch, 1, 0, 0, &d);
+        if (rc != SQN_OK) return rc;
         if ((rc = launch_conv_f32(d, st)) != SQN_OK) return rc;
+        mark("conv1");
+        if ((rc = launch_maxpool3x3s2(buf("conv1"), buf("pool1"), 96, 111, 111, batch, dt, st)) != SQN_OK) return rc;
+        mark("pool1");
     }
-    mark("conv1");
-    if ((rc = launch_maxpool3x3s2(buf("conv1"), buf("pool1"), 96, 111, 111, batch, dt, st)) != SQN_OK) return rc;
-    mark("pool1");
 
     const void* cur = buf("pool1");
     for (int i = 0; i < 8; ++i) {

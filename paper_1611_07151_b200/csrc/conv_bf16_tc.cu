@@ -76,6 +76,14 @@ struct TcParams {
     unsigned a_bytes, b_bytes;       // bytes one item's A box / B box delivers
     unsigned a_tile, b_tile;         // shared-memory bytes reserved per A / B tile
     unsigned off_b, off_stg, off_bias, off_ctl;   // byte offsets from the 1024-aligned base
+    // fused 3x3/stride-2 max-pool (patch mode only): a CTA walks the tiles of a strip of output rows from
+    // left to right, keeps the last columns in shared memory and emits pooled pixels directly
+    int pool;                        // 1: write max-pooled output instead of the convolution's own
+    int h_step;                      // output rows between consecutive tile rows (BH, or 14 when pooling)
+    int PW_out, PH_out;              // pooled extents
+    int pool_ctot;                   // layers per pixel of the pooled tensor
+    unsigned off_pool;               // shared-memory offset of the column ring [16 rows][16 cols][BN]
+    __nv_bfloat16* pool_out;
     const float* bias;
     int* status;
 };
@@ -134,6 +142,12 @@ struct TileCoord { int nt, tw, th, ti; };
 
 __device__ __forceinline__ void tile_first(const TcParams& p, int t, TileCoord& c)
 {
+    if (p.pool) {                 // t is a strip: (row tile, image)
+        c.nt = 0; c.tw = 0;
+        c.th = t % p.tiles_h;
+        c.ti = t / p.tiles_h;
+        return;
+    }
     c.nt = t % p.n_tiles;
     const int mt = t / p.n_tiles;
     c.tw = mt % p.tiles_w;
@@ -144,6 +158,14 @@ __device__ __forceinline__ void tile_first(const TcParams& p, int t, TileCoord& 
 __device__ __forceinline__ void tile_next(const TcParams& p, TileCoord& c)
 {
     int carry = 0;
+    if (p.pool) {                 // left to right inside the strip, then this CTA's next strip
+        if (++c.tw < p.tiles_w) return;
+        c.tw = 0;
+        c.th += p.g_th;
+        if (c.th >= p.tiles_h) { c.th -= p.tiles_h; carry = 1; }
+        c.ti += p.g_ti + carry;
+        return;
+    }
     c.nt += p.g_nt;
     if (c.nt >= p.n_tiles) { c.nt -= p.n_tiles; carry = 1; }
     c.tw += p.g_tw + carry; carry = 0;
@@ -152,8 +174,43 @@ __device__ __forceinline__ void tile_next(const TcParams& p, TileCoord& c)
     if (c.th >= p.tiles_h) { c.th -= p.tiles_h; carry = 1; }
     c.ti += p.g_ti + carry;
 }
+// Number of tiles this CTA processes (it takes tiles, or strips of tiles_w tiles, blockIdx.x + k*gridDim.x).
+__device__ __forceinline__ int tiles_of_cta(const TcParams& p)
+{
+    const int units = p.pool ? p.tiles_h * p.tiles_i : p.total_tiles;
+    if ((int)blockIdx.x >= units) return 0;
+    const int mine = (units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    return p.pool ? mine * p.tiles_w : mine;
+}
 
-template <int HALVES>
+// AND of a predicate over the 4*HALVES epilogue warps (named barrier 2); used where those warps meet at
+// barriers afterwards, so that all of them take the same way out when a bounded wait has run out.
+__device__ __forceinline__ bool epilogue_vote(bool ok, int nthreads)
+{
+    uint32_t all;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.and.pred p, 2, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(all)
+        : "r"((uint32_t)ok), "r"(nthreads)
+        : "memory");
+    return all != 0;
+}
+
+__device__ __forceinline__ uint4 bmax8(uint4 a, uint4 b)
+{
+    uint4 r;
+    __nv_bfloat162 x, y, m;
+    x = *reinterpret_cast<__nv_bfloat162*>(&a.x); y = *reinterpret_cast<__nv_bfloat162*>(&b.x); m = __hmax2(x, y); r.x = *reinterpret_cast<uint32_t*>(&m);
+    x = *reinterpret_cast<__nv_bfloat162*>(&a.y); y = *reinterpret_cast<__nv_bfloat162*>(&b.y); m = __hmax2(x, y); r.y = *reinterpret_cast<uint32_t*>(&m);
+    x = *reinterpret_cast<__nv_bfloat162*>(&a.z); y = *reinterpret_cast<__nv_bfloat162*>(&b.z); m = __hmax2(x, y); r.z = *reinterpret_cast<uint32_t*>(&m);
+    x = *reinterpret_cast<__nv_bfloat162*>(&a.w); y = *reinterpret_cast<__nv_bfloat162*>(&b.w); m = __hmax2(x, y); r.w = *reinterpret_cast<uint32_t*>(&m);
+    return r;
+}
+
+template <int HALVES, bool POOL>
 __global__ void __launch_bounds__(threads_for(HALVES), 3 - HALVES)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmO, const TcParams p)
@@ -176,6 +233,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t row_bytes = (uint32_t)p.BKc * 2u;
     const int items = p.taps * p.chunks;
     const int nchunks = p.BN / p.CW;
+    const int my_tiles = tiles_of_cta(p);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -239,8 +297,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             uint32_t ph = 0;
             TileCoord tc;
             tile_first(p, blockIdx.x, tc);
-            for (int t = blockIdx.x; t < p.total_tiles && ok; t += gridDim.x, tile_next(p, tc)) {
-                const int w0 = tc.tw * p.BW, h0 = tc.th * p.BH, i0 = tc.ti * p.BI, n0 = tc.nt * p.BN;
+            for (int it = 0; it < my_tiles && ok; ++it, tile_next(p, tc)) {
+                const int w0 = tc.tw * p.BW, h0 = tc.th * p.h_step, i0 = tc.ti * p.BI, n0 = tc.nt * p.BN;
                 if (p.patch) {
                     // one box per reduction chunk covers the tile plus its halo; every tap reads from it
                     if (!wait_bar(smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
@@ -311,7 +369,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (p.b_resident) ok = wait_bar(smem_u32(&sh->b_full), 0u, abort_flag, p.status);
             int s = 0, as = 0;
             uint32_t ph = 0, aph = 0;
-            for (int t = blockIdx.x; t < p.total_tiles && ok; t += gridDim.x) {
+            for (int it = 0; it < my_tiles && ok; ++it) {
                 if (!wait_bar(smem_u32(&sh->tmem_empty[as]), aph ^ 1u, abort_flag, p.status)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(as * p.bn_pad);
@@ -370,12 +428,81 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         uint32_t aph = 0, sph = 0;
         TileCoord tc;
         tile_first(p, blockIdx.x, tc);
-        for (int t = blockIdx.x; t < p.total_tiles && ok; t += gridDim.x, tile_next(p, tc)) {
+        for (int it = 0; it < my_tiles && ok; ++it, tile_next(p, tc)) {
             const int n0 = tc.nt * p.BN;
             ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_full[as]), aph, abort_flag, p.status));
+            if (POOL) ok = epilogue_vote(ok, EPI_WARPS * 32);        // the pooled path meets at barriers below
             if (!ok) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * p.bn_pad);
+            if (POOL) {
+                // ---- fused max-pool.  Column ring X[16 rows][16 columns][BN] (bf16): output column x of the
+                // strip lives at ring column (x + 2) & 15, so the two columns a window may need from the
+                // previous tile are still there.  Tile k adds columns 8k..8k+7 and emits the pooled columns
+                // 4k-1..4k+2 (windows 2pw..2pw+2) for the seven pooled rows that lie inside its 16 rows.
+                const uint32_t smX = base + p.off_pool;
+                const int et = threadIdx.x - 64;                       // 0 .. 128*HALVES-1
+                const int r = row >> 3, j = row & 7;
+                const int half = (warp - 2) >> 2;
+                const int cper = p.BN / HALVES;                        // layers this thread converts
+                const int cb = (8 * tc.tw + 2 + j) & 15;
+                const uint32_t xrow = smX + (uint32_t)(((r * 16 + cb) * p.BN + half * cper) * 2);
+                for (int c16 = 0; c16 < cper; c16 += 16) {
+                    uint32_t v[16];
+                    tmem_ld_x16(taddr + (uint32_t)(half * cper + c16), v);
+                    tmem_ld_wait();
+                    const float4* bch = reinterpret_cast<const float4*>(bias_s + half * cper + c16);
+                    const float4 b0 = bch[0], b1 = bch[1], b2 = bch[2], b3 = bch[3];
+                    float f[16];
+                    f[0] = __uint_as_float(v[0]) + b0.x;   f[1] = __uint_as_float(v[1]) + b0.y;
+                    f[2] = __uint_as_float(v[2]) + b0.z;   f[3] = __uint_as_float(v[3]) + b0.w;
+                    f[4] = __uint_as_float(v[4]) + b1.x;   f[5] = __uint_as_float(v[5]) + b1.y;
+                    f[6] = __uint_as_float(v[6]) + b1.z;   f[7] = __uint_as_float(v[7]) + b1.w;
+                    f[8] = __uint_as_float(v[8]) + b2.x;   f[9] = __uint_as_float(v[9]) + b2.y;
+                    f[10] = __uint_as_float(v[10]) + b2.z; f[11] = __uint_as_float(v[11]) + b2.w;
+                    f[12] = __uint_as_float(v[12]) + b3.x; f[13] = __uint_as_float(v[13]) + b3.y;
+                    f[14] = __uint_as_float(v[14]) + b3.z; f[15] = __uint_as_float(v[15]) + b3.w;
+                    uint32_t o[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        o[e] = p.relu ? pack_relu_bf16x2(f[2 * e], f[2 * e + 1]) : pack_bf16x2(f[2 * e], f[2 * e + 1]);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(xrow + (uint32_t)(c16 * 2)), "r"(o[0]),
+                                 "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(xrow + (uint32_t)(c16 * 2 + 16)), "r"(o[4]),
+                                 "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+                }
+                // accumulator drained: hand it back to the MMA issuer
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[as]));
+                if (++as == 2) { as = 0; aph ^= 1u; }
+                asm volatile("bar.sync 1, %0;" ::"r"(EPI_WARPS * 32) : "memory");      // tile is in the ring
+                const int vecs = p.BN >> 3;                              // 16-byte vectors per pixel
+                const int nwork = 28 * vecs;                             // 7 pooled rows x 4 pooled columns
+                const int ph0 = tc.th * 7, pw0 = tc.tw * 4 - 1, img = tc.ti;
+                for (int wk = et; wk < nwork; wk += EPI_WARPS * 32) {
+                    const int vec = wk % vecs;
+                    const int px = wk / vecs;
+                    const int pi = px & 3, pr = px >> 2;
+                    const int pw = pw0 + pi, ph = ph0 + pr;
+                    if (pw < 0 || pw >= p.PW_out || ph >= p.PH_out) continue;
+                    uint4 m = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                    for (int dy = 0; dy < 3; ++dy)
+#pragma unroll
+                        for (int dx = 0; dx < 3; ++dx) {
+                            const int xr = 2 * pr + dy, xc = (8 * tc.tw + 2 * pi + dx) & 15;
+                            uint4 w;
+                            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w)
+                                         : "r"(smX + (uint32_t)(((xr * 16 + xc) * p.BN + vec * 8) * 2)) : "memory");
+                            m = (dy == 0 && dx == 0) ? w : bmax8(m, w);
+                        }
+                    __nv_bfloat16* dst = p.pool_out + (((size_t)img * p.PH_out + ph) * p.PW_out + pw) * p.pool_ctot + p.c_off + vec * 8;
+                    *reinterpret_cast<uint4*>(dst) = m;
+                }
+                asm volatile("bar.sync 1, %0;" ::"r"(EPI_WARPS * 32) : "memory");      // ring columns may be overwritten
+                continue;
+            }
             for (int chunk = 0; chunk < nchunks; ++chunk) {
                 const int c0 = chunk * p.CW;
                 if (n0 + c0 >= p.Cout) break;
@@ -451,8 +578,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             uint32_t sph = 0;
             TileCoord tc;
             tile_first(p, blockIdx.x, tc);
-            for (int t = blockIdx.x; t < p.total_tiles && ok; t += gridDim.x, tile_next(p, tc)) {
-                const int w0 = tc.tw * p.BW, h0 = tc.th * p.BH, i0 = tc.ti * p.BI, n0 = tc.nt * p.BN;
+            for (int it = 0; it < (p.pool ? 0 : my_tiles) && ok; ++it, tile_next(p, tc)) {
+                const int w0 = tc.tw * p.BW, h0 = tc.th * p.h_step, i0 = tc.ti * p.BI, n0 = tc.nt * p.BN;
                 for (int chunk = 0; chunk < nchunks; ++chunk) {
                     const int c0 = chunk * p.CW;
                     if (n0 + c0 >= p.Cout) break;
@@ -611,7 +738,7 @@ int fit_stages(TcParams& p, size_t a_tile, bool want_resident, int cw, int nstg,
     static_assert(sizeof(Shared) <= CTL_BYTES, "control block");
     if (SMEM_LIMIT < 1024 + bias_bytes + ctl_bytes) return 0;
     const size_t avail = SMEM_LIMIT - 1024 /*alignment slack*/ - bias_bytes - ctl_bytes;
-    const size_t stg_bytes = (size_t)nstg * slot;
+    const size_t stg_bytes = p.pool ? (size_t)16 * 16 * p.BN * 2 : (size_t)nstg * slot;   // column ring when pooling
     const size_t b_all = (size_t)items * p.b_tile;
     int stages;
     size_t b_region;
@@ -633,6 +760,7 @@ int fit_stages(TcParams& p, size_t a_tile, bool want_resident, int cw, int nstg,
     p.a_tile = (unsigned)a_tile;
     p.off_b = (unsigned)((size_t)stages * a_tile);
     p.off_stg = p.off_b + (unsigned)b_region;
+    p.off_pool = p.off_stg;
     p.off_bias = p.off_stg + (unsigned)stg_bytes;
     p.off_ctl = p.off_bias + (unsigned)bias_bytes;
     *smem_bytes = 1024 + (size_t)p.off_ctl + ctl_bytes;
@@ -665,6 +793,8 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     p.bias = d.bias;
     p.status = device_status_word();
     p.h_mul = 1;
+    p.pool = d.pool ? 1 : 0;
+    if (p.pool && (d.OH < 3 || d.OW < 3 || d.Cout % 32 != 0 || d.Cout > 256)) return SQN_ERR_UNSUPPORTED;
     if (stem) {
         p.taps = 7; p.taps_h = 7; p.taps_w = 1; p.pad = 0; p.BKc = 32; p.chunks = 1; p.k_per_tap = 32;
     } else {
@@ -681,7 +811,7 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     unsigned cols = 32;
     while (cols < 2u * (unsigned)p.bn_pad) cols *= 2;
     p.tmem_cols = cols;
-    if (halves == 1 && cols > 256) return SQN_ERR_UNSUPPORTED;     // two CTAs share the SM's 512 TMEM columns
+    if (halves == 1 && (cols > 256 || d.pool)) return SQN_ERR_UNSUPPORTED;   // two CTAs share the SM's 512 TMEM columns
     p.b_tile = ((unsigned)p.BN * row_bytes + 1023u) / 1024u * 1024u;
     p.b_bytes = (unsigned)p.BN * row_bytes;
 
@@ -699,7 +829,7 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     bool patch_ok = false;
     if (!flat && p.n_tiles == 1) {
         const int th = (OH + 15) / 16;
-        const int bh = (OH + th - 1) / th;
+        const int bh = p.pool ? 16 : (OH + th - 1) / th;     // pooling: 16 rows give 7 pooled rows, strips 14 rows apart
         int max_rows;
         if (stem) {
             patch_w = 8; patch_h = 2 * bh + 5;
@@ -721,7 +851,7 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
         }
     }
     if (!patch_ok) {
-        if (stem) return SQN_ERR_UNSUPPORTED;
+        if (stem || p.pool) return SQN_ERR_UNSUPPORTED;
         p.patch = 0;
         p.h_mul = 1;
         if (flat) { p.BW = OW < TILE_M ? OW : TILE_M; p.BH = 1; p.BI = 1; }
@@ -736,13 +866,29 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     p.tiles_w = (OW + p.BW - 1) / p.BW;
     p.tiles_h = (OH + p.BH - 1) / p.BH;
     p.tiles_i = (NI + p.BI - 1) / p.BI;
+    p.h_step = p.BH;
+    if (p.pool) {
+        p.PW_out = (d.OW - 3) / 2 + 1;
+        p.PH_out = (d.OH - 3) / 2 + 1;
+        p.h_step = 14;
+        p.tiles_h = (p.PH_out + 6) / 7;                       // seven pooled rows per strip
+        const int tw_pool = (p.PW_out + 1 + 3) / 4;            // tile k emits pooled columns 4k-1 .. 4k+2
+        if (tw_pool > p.tiles_w) p.tiles_w = tw_pool;
+        p.pool_out = static_cast<__nv_bfloat16*>(d.out);
+        p.pool_ctot = d.out_c_total;
+    }
 
     const long long total = (long long)p.tiles_w * p.tiles_h * p.tiles_i * p.n_tiles;
     if (total > 0x7fffffffLL) return SQN_ERR_UNSUPPORTED;
     p.total_tiles = (int)total;
     const long long ctas = (long long)num_sms() * (halves == 1 ? 2 : 1);
-    plan->grid = (int)(total < ctas ? total : ctas);
-    {
+    const long long units = p.pool ? (long long)p.tiles_h * p.tiles_i : total;
+    plan->grid = (int)(units < ctas ? units : ctas);
+    if (p.pool) {
+        p.g_nt = 0; p.g_tw = 0;
+        p.g_th = plan->grid % p.tiles_h;
+        p.g_ti = plan->grid / p.tiles_h;
+    } else {
         int g = plan->grid;
         p.g_nt = g % p.n_tiles; g /= p.n_tiles;
         p.g_tw = g % p.tiles_w; g /= p.tiles_w;
@@ -784,9 +930,11 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
         // extent of the layer dimension stops at the end of this layer's slice so that a
         // partial last tile is clipped instead of spilling into the neighbouring slice
         const cuuint64_t s1 = (cuuint64_t)d.out_c_total * 2;
-        cuuint64_t dims[4] = {(cuuint64_t)(d.out_c_offset + d.Cout), (cuuint64_t)OW, (cuuint64_t)OH, (cuuint64_t)NI};
-        cuuint64_t str[3] = {s1, s1 * OW, s1 * OW * OH};
-        cuuint32_t box[4] = {(cuuint32_t)p.CW, (cuuint32_t)p.BW, (cuuint32_t)p.BH, (cuuint32_t)p.BI};
+        // (when the max-pool is fused the kernel stores pooled pixels itself; the map then only has to be valid)
+        const cuuint64_t ow = p.pool ? (cuuint64_t)p.PW_out : (cuuint64_t)OW, oh = p.pool ? (cuuint64_t)p.PH_out : (cuuint64_t)OH;
+        cuuint64_t dims[4] = {(cuuint64_t)(d.out_c_offset + d.Cout), ow, oh, (cuuint64_t)NI};
+        cuuint64_t str[3] = {s1, s1 * ow, s1 * ow * oh};
+        cuuint32_t box[4] = {(cuuint32_t)p.CW, (cuuint32_t)(p.pool ? 1 : p.BW), (cuuint32_t)(p.pool ? 1 : p.BH), (cuuint32_t)p.BI};
         if (!encode(&plan->o, 4, d.out, dims, str, box, (unsigned)p.CW * 2u)) return SQN_ERR_CUDA;
     }
     return SQN_OK;
@@ -811,16 +959,20 @@ int launch_plan(const Plan& plan, cudaStream_t stream)
     static std::once_flag once;
     static cudaError_t attr_rc = cudaSuccess;
     std::call_once(once, [] {
-        attr_rc = cudaFuncSetAttribute(conv_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
+        attr_rc = cudaFuncSetAttribute(conv_tc_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
         if (attr_rc == cudaSuccess)
-            attr_rc = cudaFuncSetAttribute(conv_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            attr_rc = cudaFuncSetAttribute(conv_tc_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
+        if (attr_rc == cudaSuccess)
+            attr_rc = cudaFuncSetAttribute(conv_tc_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)SMEM_LIMIT_2CTA);
     });
     if (attr_rc != cudaSuccess) return SQN_ERR_CUDA;
-    if (plan.halves == 1)
-        conv_tc_kernel<1><<<plan.grid, threads_for(1), plan.smem, stream>>>(plan.a, plan.b, plan.o, plan.p);
+    if (plan.p.pool)
+        conv_tc_kernel<2, true><<<plan.grid, threads_for(2), plan.smem, stream>>>(plan.a, plan.b, plan.o, plan.p);
+    else if (plan.halves == 1)
+        conv_tc_kernel<1, false><<<plan.grid, threads_for(1), plan.smem, stream>>>(plan.a, plan.b, plan.o, plan.p);
     else
-        conv_tc_kernel<2><<<plan.grid, threads_for(2), plan.smem, stream>>>(plan.a, plan.b, plan.o, plan.p);
+        conv_tc_kernel<2, false><<<plan.grid, threads_for(2), plan.smem, stream>>>(plan.a, plan.b, plan.o, plan.p);
     note_launch();
     return cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
 }
@@ -841,7 +993,7 @@ int cached_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_p
     PlanKey k;
     std::memset(&k, 0, sizeof(k));
     k.in = d.in; k.w = d.w; k.bias = d.bias; k.out = d.out; k.ws = ws;
-    const int v[14] = {d.N, d.Cin, d.H, d.W, d.Cout, d.K, d.S, d.pad, d.out_c_offset, d.out_c_total, d.relu,
+    const int v[14] = {d.N, d.Cin, d.H, d.W, d.Cout, d.K, d.S, d.pad, d.out_c_offset, d.out_c_total, d.relu | (d.pool << 1),
                        stem ? 1 : 0, Hp, Wp};
     std::memcpy(k.v, v, sizeof(v));
     int dev = 0;
@@ -877,6 +1029,7 @@ int conv_bf16_supported(const ConvDesc& d)
     if (d.Cout <= 256 ? (d.Cout % 16 != 0) : (d.Cout % 8 != 0)) return SQN_ERR_UNSUPPORTED;
     if (d.out_c_offset % 8 != 0 || d.out_c_total % 8 != 0) return SQN_ERR_ALIGN;
     if (d.K == 1 && d.pad != 0) return SQN_ERR_UNSUPPORTED;
+    if (d.pool && d.K < 2) return SQN_ERR_UNSUPPORTED;      // the fused max-pool lives in the patch-mode kernel
     return SQN_OK;
 }
 

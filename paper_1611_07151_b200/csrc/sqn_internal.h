@@ -17,6 +17,7 @@ struct ConvDesc {
     void* out;            // [N][OH][OW][out_c_total], written at out_c_offset
     int N, Cin, H, W, Cout, K, S, pad, OH, OW;
     int out_c_offset, out_c_total, relu;
+    int pool;             // 1: out receives the 3x3/stride-2 max-pool of the layer's output (bf16 path only)
 };
 
 // Launch counter (host side): every kernel launch goes through note_launch().

@@ -33,12 +33,14 @@ def out_extent(H, K, S, pad):
     return (H + 2 * pad - K) // S + 1
 
 
-def gpu_conv(x, w, b, S, pad, relu=True, dtype=B.SQN_F32, c_offset=0, c_total=0, fill=None):
+def gpu_conv(x, w, b, S, pad, relu=True, dtype=B.SQN_F32, c_offset=0, c_total=0, fill=None, fuse_maxpool=False):
     """Run one convolution through conv_forward_ex; returns the full output tensor as NCHW."""
     import torch
     N, C, H, W = x.shape
     M, _, K, _ = w.shape
     oh, ow = out_extent(H, K, S, pad), out_extent(W, K, S, pad)
+    if fuse_maxpool:
+        oh, ow = (oh - 3) // 2 + 1, (ow - 3) // 2 + 1
     ct = c_total if c_total else M
     out = B.empty_device((N, oh, ow, ct), dtype)
     out.fill_(float("nan") if fill is None else fill)
@@ -46,6 +48,6 @@ def gpu_conv(x, w, b, S, pad, relu=True, dtype=B.SQN_F32, c_offset=0, c_total=0,
     ws = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device="cuda")
     xd, wd, bd = dev_act(x, dtype), dev_w(w, dtype), dev_b(b)
     B.conv_forward_ex(xd, wd, bd, out, C, M, H, W, K, S, pad, N, dtype=dtype, relu=relu, out_c_offset=c_offset,
-                      out_c_total=c_total, workspace=ws, workspace_bytes=ws_bytes)
+                      out_c_total=c_total, workspace=ws, workspace_bytes=ws_bytes, fuse_maxpool=fuse_maxpool)
     assert B.sqn_check() == B.SQN_OK
     return host_act(out, dtype)

@@ -79,6 +79,42 @@ def test_stem_7x7_stride2(hw, batch, cout):
     assert G.rel_err(got, exp) <= TOL
 
 
+# (N, Cin, Cout, H, W, K, S, pad): convolution with the following 3x3/2 max-pool fused into its epilogue
+POOLED = [
+    (2, 3, 96, 227, 227, 7, 2, 0),     # conv1 + pool1 of the network
+    (3, 3, 32, 37, 41, 7, 2, 0),       # stem shape on a small, non-square map (ragged strips and columns)
+    (2, 32, 64, 27, 27, 3, 1, 1),      # 3x3 layer, one and a bit strips
+    (1, 16, 128, 55, 55, 3, 1, 1),
+    (2, 64, 32, 9, 12, 3, 1, 0),
+]
+
+
+@pytest.mark.parametrize("shape", POOLED, ids=lambda s: "x".join(map(str, s)))
+def test_conv_with_fused_maxpool(shape):
+    N, C, M, H, W, K, S, pad = shape
+    rng = np.random.default_rng(sum(shape))
+    x = synth.draw_input(rng, (N, C, H, W))
+    w, b = synth.draw_conv_params(rng, C, M, K)
+    b = b + np.float32(0.2) * rng.standard_normal(M).astype(np.float32)      # make some layers mostly negative
+    exp = ref.maxpool(ref.conv2d(x, w, b, S=S, pad=pad, relu=True), 3, 2)
+    got = G.gpu_conv(x, w, b, S, pad, True, BF16, fuse_maxpool=True, c_offset=32, c_total=M + 64, fill=-7.0)
+    assert got.shape == (N, M + 64) + exp.shape[2:]
+    assert G.rel_err(got[:, 32:32 + M], exp) <= TOL
+    assert (got[:, :32] == -7.0).all() and (got[:, 32 + M:] == -7.0).all()
+    # the unfused pair of calls gives the very same bf16 values
+    full = G.gpu_conv(x, w, b, S, pad, True, BF16)
+    np.testing.assert_array_equal(got[:, 32:32 + M], ref.maxpool(full, 3, 2))
+
+
+def test_fused_maxpool_is_refused_where_it_cannot_run():
+    import torch
+    p = torch.empty(64, device="cuda")
+    for dtype, cin, cout, k in [(B.SQN_F32, 16, 64, 3), (BF16, 16, 64, 1), (BF16, 16, 48, 3), (BF16, 64, 256, 3)]:
+        with pytest.raises(B.SqnError) as e:
+            B.conv_forward_ex(p, p, p, p, cin, cout, 13, 13, k, 1, k // 2, 1, dtype=dtype, fuse_maxpool=True)
+        assert e.value.status == B.SQN_ERR_UNSUPPORTED
+
+
 def test_per_layer_sweep():
     """Every distinct SqueezeNet conv shape, isolated, batch 1 and 3, seed 4."""
     seen = set()
