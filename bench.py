@@ -66,6 +66,10 @@ def launch_work(batch, es):
     # stem with its max-pool fused: the 96x111x111 map is never stored, only the pooled 96x55x55 one
     work["conv1+pool1"] = {"flops": work["conv1"]["flops"],
                            "bytes": float(es * batch * (IMG * IMG * 3 + 55 * 55 * 96) + es * 96 * 147 + 4 * 96)}
+    # fire4's expands with pool4 fused: squeeze map in, pooled half (128 x 27 x 27) out
+    for nm, k in (("fire4_e1", 1), ("fire4_e3", 3)):
+        work[nm + "+pool"] = {"flops": work[nm]["flops"],
+                              "bytes": float(es * batch * (55 * 55 * 32 + 27 * 27 * 128) + es * 128 * 32 * k * k + 4 * 128)}
     return work
 
 

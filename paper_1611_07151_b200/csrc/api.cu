@@ -336,7 +336,8 @@ extern "C" int squeezenet_layer_output(const sqn_net* net, const char* name, voi
     if (!net || !name || !workspace || !ptr || batch <= 0 || batch > net->max_batch) return SQN_ERR_BADARG;
     const int i = find_slot(net, name);
     if (i < 0) return SQN_ERR_BADARG;
-    if (net->dtype == SQN_BF16 && std::strcmp(name, "conv1") == 0) return SQN_ERR_UNSUPPORTED;   // fused with pool1
+    if (net->dtype == SQN_BF16 && (std::strcmp(name, "conv1") == 0 || std::strcmp(name, "fire4") == 0))
+        return SQN_ERR_UNSUPPORTED;   // computed inside the kernels that write pool1 / pool4, never stored
     std::vector<size_t> offs;
     layout(net, batch, &offs, nullptr);
     *ptr = static_cast<char*>(workspace) + offs[i];
@@ -430,17 +431,36 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
         const std::string nm(f.name);
         if ((rc = run_conv(dsq, dt, nullptr, 0, st)) != SQN_OK) return rc;
         mark((nm + "_sq").c_str());
-        if ((rc = run_conv(d1, dt, nullptr, 0, st)) != SQN_OK) return rc;
-        mark((nm + "_e1").c_str());
-        if ((rc = run_conv(d3, dt, nullptr, 0, st)) != SQN_OK) return rc;
-        mark((nm + "_e3").c_str());
-        cur = out;
-        if (f.pool_after) {
+        // bf16: where a max-pool follows and the expands' kernels fit in shared memory, both expands pool
+        // in their epilogues and write their halves of the pooled map; the unpooled map is never stored
+        bool fused_pool = false;
+        if (f.pool_after && dt == SQN_BF16) {
             const std::string pn = std::string("pool") + (f.name + 4);
-            void* po = buf(pn);
-            if ((rc = launch_maxpool3x3s2(cur, po, 2 * f.e, f.hw, f.hw, batch, dt, st)) != SQN_OK) return rc;
-            mark(pn.c_str());
-            cur = po;
+            ConvDesc p1 = d1, p3 = d3;
+            p1.out = p3.out = buf(pn);
+            p1.pool = p3.pool = 1;
+            if (conv_bf16_pool_fits(p1) && conv_bf16_pool_fits(p3)) {
+                if ((rc = run_conv(p1, dt, nullptr, 0, st)) != SQN_OK) return rc;
+                mark((nm + "_e1+pool").c_str());
+                if ((rc = run_conv(p3, dt, nullptr, 0, st)) != SQN_OK) return rc;
+                mark((nm + "_e3+pool").c_str());
+                cur = buf(pn);
+                fused_pool = true;
+            }
+        }
+        if (!fused_pool) {
+            if ((rc = run_conv(d1, dt, nullptr, 0, st)) != SQN_OK) return rc;
+            mark((nm + "_e1").c_str());
+            if ((rc = run_conv(d3, dt, nullptr, 0, st)) != SQN_OK) return rc;
+            mark((nm + "_e3").c_str());
+            cur = out;
+            if (f.pool_after) {
+                const std::string pn = std::string("pool") + (f.name + 4);
+                void* po = buf(pn);
+                if ((rc = launch_maxpool3x3s2(cur, po, 2 * f.e, f.hw, f.hw, batch, dt, st)) != SQN_OK) return rc;
+                mark(pn.c_str());
+                cur = po;
+            }
         }
     }
     // conv10 1x1 + ReLU, global average, softmax

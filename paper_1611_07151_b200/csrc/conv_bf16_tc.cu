@@ -446,7 +446,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const int half = (warp - 2) >> 2;
                 const int cper = p.BN / HALVES;                        // layers this thread converts
                 const int cb = (8 * tc.tw + 2 + j) & 15;
-                const uint32_t xrow = smX + (uint32_t)(((r * 16 + cb) * p.BN + half * cper) * 2);
+                const uint32_t xpix = (uint32_t)p.BN * 2u + 16u;          // pixel pitch: 16 bytes of padding keep the 8
+                                                                            // pixels a quarter-warp writes in different banks
+                const uint32_t xrow = smX + (uint32_t)(r * 16 + cb) * xpix + (uint32_t)(half * cper * 2);
                 for (int c16 = 0; c16 < cper; c16 += 16) {
                     uint32_t v[16];
                     tmem_ld_x16(taddr + (uint32_t)(half * cper + c16), v);
@@ -494,7 +496,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             const int xr = 2 * pr + dy, xc = (8 * tc.tw + 2 * pi + dx) & 15;
                             uint4 w;
                             asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w)
-                                         : "r"(smX + (uint32_t)(((xr * 16 + xc) * p.BN + vec * 8) * 2)) : "memory");
+                                         : "r"(smX + (uint32_t)(xr * 16 + xc) * xpix + (uint32_t)(vec * 16)) : "memory");
                             m = (dy == 0 && dx == 0) ? w : bmax8(m, w);
                         }
                     __nv_bfloat16* dst = p.pool_out + (((size_t)img * p.PH_out + ph) * p.PW_out + pw) * p.pool_ctot + p.c_off + vec * 8;
@@ -738,7 +740,8 @@ int fit_stages(TcParams& p, size_t a_tile, bool want_resident, int cw, int nstg,
     static_assert(sizeof(Shared) <= CTL_BYTES, "control block");
     if (SMEM_LIMIT < 1024 + bias_bytes + ctl_bytes) return 0;
     const size_t avail = SMEM_LIMIT - 1024 /*alignment slack*/ - bias_bytes - ctl_bytes;
-    const size_t stg_bytes = p.pool ? (size_t)16 * 16 * p.BN * 2 : (size_t)nstg * slot;   // column ring when pooling
+    const size_t stg_bytes = p.pool ? ((size_t)16 * 16 * (p.BN * 2 + 16) + 1023) / 1024 * 1024   // column ring when pooling
+                                    : (size_t)nstg * slot;
     const size_t b_all = (size_t)items * p.b_tile;
     int stages;
     size_t b_region;
@@ -816,7 +819,7 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     p.b_bytes = (unsigned)p.BN * row_bytes;
 
     // output-pixel tiling; a 1x1 layer is tiled over the flattened pixel index
-    const bool flat = !stem && d.K == 1 && d.pad == 0;
+    const bool flat = !stem && d.K == 1 && d.pad == 0 && !d.pool;      // (a pooled 1x1 layer needs the 8x16 spatial tiles)
     long long OWl = d.OW, OHl = d.OH, NIl = d.N;
     if (flat) { OWl = (long long)d.N * d.OH * d.OW; OHl = 1; NIl = 1; }
     if (OWl > 0x7fffffffLL) return SQN_ERR_UNSUPPORTED;
@@ -1029,7 +1032,6 @@ int conv_bf16_supported(const ConvDesc& d)
     if (d.Cout <= 256 ? (d.Cout % 16 != 0) : (d.Cout % 8 != 0)) return SQN_ERR_UNSUPPORTED;
     if (d.out_c_offset % 8 != 0 || d.out_c_total % 8 != 0) return SQN_ERR_ALIGN;
     if (d.K == 1 && d.pad != 0) return SQN_ERR_UNSUPPORTED;
-    if (d.pool && d.K < 2) return SQN_ERR_UNSUPPORTED;      // the fused max-pool lives in the patch-mode kernel
     return SQN_OK;
 }
 
@@ -1039,6 +1041,14 @@ int launch_conv_bf16(const ConvDesc& d, cudaStream_t stream)
     const int rc = cached_plan(d, false, d.in, d.w, 0, 0, nullptr, &plan);
     if (rc != SQN_OK) return rc;
     return launch_plan(plan, stream);
+}
+
+// Host-only feasibility test of the fused max-pool for a layer (shared-memory budget, shape rules).
+bool conv_bf16_pool_fits(const ConvDesc& d)
+{
+    if (!d.pool || conv_bf16_supported(d) != SQN_OK) return false;
+    Plan plan;
+    return cached_plan(d, false, d.in, d.w, 0, 0, nullptr, &plan) == SQN_OK;
 }
 
 // Same launch without touching the plan cache: the tensor maps are encoded into a stack object on
