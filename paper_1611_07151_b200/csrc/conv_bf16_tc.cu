@@ -426,6 +426,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         bool ok = true;
         int as = 0, sb = 0;
         uint32_t aph = 0, sph = 0;
+        // fused max-pool: the (pooled pixel, 16-byte vector) items of this thread are the same for every
+        // tile, so they are worked out once (28 pooled pixels x BN/8 vectors over the epilogue threads)
+        int pool_item[4] = {-1, -1, -1, -1};
+        if (POOL) {
+            const int vecs = p.BN >> 3, nwork = 28 * vecs;
+            for (int k = 0, wk = threadIdx.x - 64; k < 4 && wk < nwork; ++k, wk += EPI_WARPS * 32)
+                pool_item[k] = ((wk / vecs) << 16) | (wk % vecs);
+        }
         TileCoord tc;
         tile_first(p, blockIdx.x, tc);
         for (int it = 0; it < my_tiles && ok; ++it, tile_next(p, tc)) {
@@ -479,12 +487,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[as]));
                 if (++as == 2) { as = 0; aph ^= 1u; }
                 asm volatile("bar.sync 1, %0;" ::"r"(EPI_WARPS * 32) : "memory");      // tile is in the ring
-                const int vecs = p.BN >> 3;                              // 16-byte vectors per pixel
-                const int nwork = 28 * vecs;                             // 7 pooled rows x 4 pooled columns
                 const int ph0 = tc.th * 7, pw0 = tc.tw * 4 - 1, img = tc.ti;
-                for (int wk = et; wk < nwork; wk += EPI_WARPS * 32) {
-                    const int vec = wk % vecs;
-                    const int px = wk / vecs;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {                            // this thread's (pooled pixel, vector) items
+                    if (pool_item[k] < 0) continue;
+                    const int vec = pool_item[k] & 0xffff;
+                    const int px = pool_item[k] >> 16;
                     const int pi = px & 3, pr = px >> 2;
                     const int pw = pw0 + pi, ph = ph0 + pr;
                     if (pw < 0 || pw >= p.PW_out || ph >= p.PH_out) continue;
