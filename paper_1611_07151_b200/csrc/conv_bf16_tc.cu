@@ -44,6 +44,7 @@ __host__ __device__ constexpr int threads_for(int halves) { return 96 + 128 * ha
 constexpr int MAX_STAGES = 8;
 constexpr int MAX_STG = 4;             // staging ring slots
 constexpr int MAX_TAB = 448;           // MMAs per tile in patch mode
+constexpr int PARAM_TAB = 160;         // ... of which this many can be tabulated in the kernel parameters
 constexpr size_t CTL_BYTES = 4096;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // about two seconds
 constexpr size_t SMEM_LIMIT = 227 * 1024;
@@ -86,6 +87,10 @@ struct TcParams {
     __nv_bfloat16* pool_out;
     const float* bias;
     int* status;
+    // patch mode, at most PARAM_TAB MMAs per tile: per MMA {A offset from the stage base, B offset from the
+    // kernel region} in 16-byte units.  Read from the constant bank, i.e. with warp-uniform loads.
+    int use_ptab;
+    uint2 ptab[PARAM_TAB];
 };
 
 struct Shared {                       // control block placed after the tiles
@@ -344,69 +349,87 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        // One thread issues every MMA, so its loop is kept to a few adds per instruction: the
-        // descriptors' constant halves are built once and only the 14-bit address field (in
-        // 16-byte units) is advanced.
-        if (lane == 0) {
-            const uint32_t idesc = make_idesc_bf16(TILE_M, (uint32_t)p.BN);
-            const int ksteps = p.BKc / 16;
-            const uint32_t hiA = (uint32_t)(make_kmajor_desc(0, row_bytes, p.patch ? p.sbo_bytes : 8u * row_bytes) >> 32);
-            const uint32_t hiB = (uint32_t)(make_kmajor_desc(0, row_bytes, 8u * row_bytes) >> 32);
-            const uint32_t a_tile16 = p.a_tile >> 4, b_tile16 = p.b_tile >> 4;
-            const uint32_t smA16 = smA >> 4, smB16 = smB >> 4;
-            auto issue = [&](uint32_t d_tmem, uint32_t a16, uint32_t b16, uint32_t acc) {
-                // ksteps MMAs of K = 16 (32 bytes = 2 address units along the row)
-                const uint64_t da = ((uint64_t)hiA << 32) | (uint64_t)(a16 | 0x10000u);
-                const uint64_t db = ((uint64_t)hiB << 32) | (uint64_t)(b16 | 0x10000u);
-                mma_bf16_ss(d_tmem, da, db, idesc, acc);
-                if (ksteps >= 2) mma_bf16_ss(d_tmem, da + 2, db + 2, idesc, 1u);
-                if (ksteps == 4) {
-                    mma_bf16_ss(d_tmem, da + 4, db + 4, idesc, 1u);
-                    mma_bf16_ss(d_tmem, da + 6, db + 6, idesc, 1u);
-                }
-            };
-            bool ok = true;
-            if (p.b_resident) ok = wait_bar(smem_u32(&sh->b_full), 0u, abort_flag, p.status);
-            int s = 0, as = 0;
-            uint32_t ph = 0, aph = 0;
-            for (int it = 0; it < my_tiles && ok; ++it) {
-                if (!wait_bar(smem_u32(&sh->tmem_empty[as]), aph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        // The whole warp walks the loop converged (all lanes wait on the barriers) and one elected
+        // lane issues the MMAs and their commits.  With the operand offsets read from the kernel
+        // parameters everything the issuing instruction needs is warp-uniform, which is what lets the
+        // MMAs go out back to back (about 55 clocks each for N <= 128, the tensor pipe's own rate; a
+        // single diverged thread reading a shared-memory table needs about 100).
+        const uint32_t idesc = make_idesc_bf16(TILE_M, (uint32_t)p.BN);
+        const int ksteps = p.BKc / 16;
+        const uint32_t hiA = (uint32_t)(make_kmajor_desc(0, row_bytes, p.patch ? p.sbo_bytes : 8u * row_bytes) >> 32);
+        const uint32_t hiB = (uint32_t)(make_kmajor_desc(0, row_bytes, 8u * row_bytes) >> 32);
+        const uint32_t a_tile16 = p.a_tile >> 4, b_tile16 = p.b_tile >> 4;
+        const uint32_t smA16 = smA >> 4, smB16 = smB >> 4;
+        const int nmma = items * ksteps;
+        bool ok = true;
+        if (p.b_resident) ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->b_full), 0u, abort_flag, p.status));
+        int s = 0, as = 0;
+        uint32_t ph = 0, aph = 0;
+        for (int it = 0; it < my_tiles && ok; ++it) {
+            ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_empty[as]), aph ^ 1u, abort_flag, p.status));
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(as * p.bn_pad);
+            if (p.patch) {
+                ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->full[s]), ph, abort_flag, p.status));
+                if (!ok) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(as * p.bn_pad);
-                if (p.patch) {
-                    if (!wait_bar(smem_u32(&sh->full[s]), ph, abort_flag, p.status)) { ok = false; break; }
-                    tc_fence_after();
-                    // output pixel (g, j) of the tile reads patch row g*(rows per line) + j + tap offset;
-                    // the offsets were tabulated once, so each MMA costs a load, an add and the issue
-                    const uint32_t a_base = smA16 + (uint32_t)s * a_tile16;
-                    const int nmma = items * ksteps;
-                    uint2 o = sh->mma_tab[0];
-                    uint32_t acc = 0u;
+                // output pixel (g, j) of the tile reads patch row g*(rows per line) + j + tap offset
+                const uint32_t a_base = smA16 + (uint32_t)s * a_tile16;
+                if (elect_one()) {
+                    if (p.use_ptab) {
+                        uint32_t acc = 0u;
 #pragma unroll 2
-                    for (int e = 1; e <= nmma; ++e) {
-                        const uint2 nxt = sh->mma_tab[e];            // one entry ahead (the table has a spare slot)
-                        mma_bf16_ss(d_tmem, ((uint64_t)hiA << 32) | (uint64_t)((a_base + o.x) | 0x10000u),
-                                    ((uint64_t)hiB << 32) | (uint64_t)(o.y | 0x10000u), idesc, acc);
-                        acc = 1u;
-                        o = nxt;
+                        for (int e = 0; e < nmma; ++e) {
+                            const uint2 o = p.ptab[e];
+                            mma_bf16_ss(d_tmem, ((uint64_t)hiA << 32) | (uint64_t)((a_base + o.x) | 0x10000u),
+                                        ((uint64_t)hiB << 32) | (uint64_t)((smB16 + o.y) | 0x10000u), idesc, acc);
+                            acc = 1u;
+                        }
+                    } else {
+                        uint2 o = sh->mma_tab[0];
+                        uint32_t acc = 0u;
+#pragma unroll 2
+                        for (int e = 1; e <= nmma; ++e) {
+                            const uint2 nxt = sh->mma_tab[e];        // one entry ahead (the table has a spare slot)
+                            mma_bf16_ss(d_tmem, ((uint64_t)hiA << 32) | (uint64_t)((a_base + o.x) | 0x10000u),
+                                        ((uint64_t)hiB << 32) | (uint64_t)(o.y | 0x10000u), idesc, acc);
+                            acc = 1u;
+                            o = nxt;
+                        }
                     }
-                    mma_commit(smem_u32(&sh->empty[s]));
-                    if (++s == p.stages) { s = 0; ph ^= 1u; }
-                } else {
-                    uint32_t bres16 = smB16;
-                    for (int i = 0; i < items; ++i, bres16 += b_tile16) {
-                        if (!wait_bar(smem_u32(&sh->full[s]), ph, abort_flag, p.status)) { ok = false; break; }
-                        tc_fence_after();
-                        issue(d_tmem, smA16 + (uint32_t)s * a_tile16, p.b_resident ? bres16 : smB16 + (uint32_t)s * b_tile16,
-                              i > 0 ? 1u : 0u);
-                        mma_commit(smem_u32(&sh->empty[s]));        // slot free once these MMAs have read it
-                        if (++s == p.stages) { s = 0; ph ^= 1u; }
-                    }
-                    if (!ok) break;
+                    mma_commit(smem_u32(&sh->empty[s]));            // patch slot free once these MMAs have read it
+                    mma_commit(smem_u32(&sh->tmem_full[as]));       // accumulator complete
                 }
-                mma_commit(smem_u32(&sh->tmem_full[as]));           // accumulator complete
-                if (++as == 2) { as = 0; aph ^= 1u; }
+                __syncwarp();
+                if (++s == p.stages) { s = 0; ph ^= 1u; }
+            } else {
+                uint32_t bres16 = smB16;
+                for (int i = 0; i < items; ++i, bres16 += b_tile16) {
+                    ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->full[s]), ph, abort_flag, p.status));
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a16 = smA16 + (uint32_t)s * a_tile16;
+                    const uint32_t b16 = p.b_resident ? bres16 : smB16 + (uint32_t)s * b_tile16;
+                    if (elect_one()) {
+                        // ksteps MMAs of K = 16 (32 bytes = 2 address units along the row)
+                        const uint64_t da = ((uint64_t)hiA << 32) | (uint64_t)(a16 | 0x10000u);
+                        const uint64_t db = ((uint64_t)hiB << 32) | (uint64_t)(b16 | 0x10000u);
+                        mma_bf16_ss(d_tmem, da, db, idesc, i > 0 ? 1u : 0u);
+                        if (ksteps >= 2) mma_bf16_ss(d_tmem, da + 2, db + 2, idesc, 1u);
+                        if (ksteps == 4) {
+                            mma_bf16_ss(d_tmem, da + 4, db + 4, idesc, 1u);
+                            mma_bf16_ss(d_tmem, da + 6, db + 6, idesc, 1u);
+                        }
+                        mma_commit(smem_u32(&sh->empty[s]));        // slot free once these MMAs have read it
+                        if (i == items - 1) mma_commit(smem_u32(&sh->tmem_full[as]));   // accumulator complete
+                    }
+                    __syncwarp();
+                    if (++s == p.stages) { s = 0; ph ^= 1u; }
+                }
+                if (!ok) break;
             }
+            if (++as == 2) { as = 0; aph ^= 1u; }
         }
     } else if (warp < 2 + EPI_WARPS) {
         // -------------------------------------------------------------------- epilogue
@@ -872,6 +895,23 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
         if (!choose_layout(p, a_tile, true, 3, &plan->smem) && !choose_layout(p, a_tile, false, 3, &plan->smem) &&
             !choose_layout(p, a_tile, false, 2, &plan->smem))
             return SQN_ERR_UNSUPPORTED;
+    }
+    p.use_ptab = 0;
+    if (p.patch && p.taps * p.chunks * (p.BKc / 16) <= PARAM_TAB) {
+        // operand offsets of every MMA of a tile, in issue order (tap-major, then chunk, then k-step)
+        p.use_ptab = 1;
+        const int ksteps = p.BKc / 16;
+        int e = 0;
+        for (int kh = 0; kh < p.taps_h; ++kh)
+            for (int kw = 0; kw < p.taps_w; ++kw)
+                for (int ch = 0; ch < p.chunks; ++ch)
+                    for (int k = 0; k < ksteps; ++k, ++e) {
+                        const unsigned it = (unsigned)((kh * p.taps_w + kw) * p.chunks + ch);
+                        const unsigned a_off = (unsigned)ch * p.patch_tile +
+                                               (unsigned)(kh * p.tap_h_rows + kw * p.tap_w_rows) * row_bytes;
+                        p.ptab[e].x = (a_off >> 4) + 2u * k;
+                        p.ptab[e].y = ((it * p.b_tile) >> 4) + 2u * k;
+                    }
     }
     if (plan->smem > t_smem_limit) return SQN_ERR_UNSUPPORTED;
     p.tiles_w = (OW + p.BW - 1) / p.BW;
