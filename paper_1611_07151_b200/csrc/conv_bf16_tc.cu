@@ -37,10 +37,10 @@ namespace {
 using namespace ptx;
 
 constexpr int TILE_M = 128;            // MMA M: TMEM lanes
-// Threads per CTA: producer warp, MMA warp, 4*HALVES epilogue warps, store warp.  HALVES = 2: one CTA per SM
-// (large tiles, kernels resident in up to 227 KB); HALVES = 1: two lighter CTAs per SM, i.e. two MMA issuers,
+// Threads per CTA: producer warp, MMA warp, 4*SPLIT epilogue warps, store warp.  SPLIT = 2 or 4: one CTA per SM
+// (large tiles, kernels resident in up to 227 KB); SPLIT = 1: two lighter CTAs per SM, i.e. two MMA issuers,
 // two producers and two store threads per SM, for the layers whose tiles are small.
-__host__ __device__ constexpr int threads_for(int halves) { return 96 + 128 * halves; }
+__host__ __device__ constexpr int threads_for(int split) { return 96 + 128 * split; }
 constexpr int MAX_STAGES = 8;
 constexpr int MAX_STG = 4;             // staging ring slots
 constexpr int MAX_TAB = 448;           // MMAs per tile in patch mode
@@ -188,7 +188,7 @@ __device__ __forceinline__ int tiles_of_cta(const TcParams& p)
     return p.pool ? mine * p.tiles_w : mine;
 }
 
-// AND of a predicate over the 4*HALVES epilogue warps (named barrier 2); used where those warps meet at
+// AND of a predicate over the 4*SPLIT epilogue warps (named barrier 2); used where those warps meet at
 // barriers afterwards, so that all of them take the same way out when a bounded wait has run out.
 __device__ __forceinline__ bool epilogue_vote(bool ok, int nthreads)
 {
@@ -215,13 +215,13 @@ __device__ __forceinline__ uint4 bmax8(uint4 a, uint4 b)
     return r;
 }
 
-template <int HALVES, bool POOL>
-__global__ void __launch_bounds__(threads_for(HALVES), 3 - HALVES)
+template <int SPLIT, bool POOL>
+__global__ void __launch_bounds__(threads_for(SPLIT), SPLIT == 1 ? 2 : 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmO, const TcParams p)
 {
-    constexpr int NUM_THREADS = threads_for(HALVES);
-    constexpr int EPI_WARPS = 4 * HALVES;
+    constexpr int NUM_THREADS = threads_for(SPLIT);
+    constexpr int EPI_WARPS = 4 * SPLIT;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -433,19 +433,20 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
     } else if (warp < 2 + EPI_WARPS) {
         // -------------------------------------------------------------------- epilogue
-        // Eight warps: warp w reads TMEM lane quadrant w % 4 (one output pixel per thread) and, of
-        // every chunk of CW layers, the half (w - 2) / 4.  TMEM -> registers, + bias, ReLU, -> bf16,
+        // 4*SPLIT warps: warp w reads TMEM lane quadrant w % 4 (one output pixel per thread) and, of
+        // every chunk of CW layers, the piece(s) given by (w - 2) / 4.  TMEM -> registers, + bias, ReLU, -> bf16,
         // into a slot of the staging ring (TMA-swizzled rows); the store warp sends the slot to
         // global memory while the next chunk is converted.
         const int q = warp & 3;
-        constexpr int NH = 2 / HALVES;                 // half-chunks each thread converts per chunk
-        const int half0 = ((warp - 2) >> 2) * NH;      // first half-chunk of this warp (0 when HALVES == 1)
+        constexpr int PIECES = SPLIT < 2 ? 2 : SPLIT;  // a chunk is converted in this many pieces
+        constexpr int NH = PIECES / SPLIT;             // pieces each thread converts per chunk (2 when SPLIT == 1)
+        const int half0 = ((warp - 2) >> 2) * NH;      // first piece of this warp
         const int row = q * 32 + lane;
         const uint32_t cw_bytes = (uint32_t)p.CW * 2u;
         const uint32_t slot_bytes = (uint32_t)TILE_M * cw_bytes;
         const uint32_t sw = cw_bytes == 128 ? (uint32_t)(row & 7)
                           : cw_bytes == 64 ? (uint32_t)((row >> 1) & 3) : (uint32_t)((row >> 2) & 1);
-        const int hc = p.CW / 2;                       // layers per half-chunk: 8, 16 or 32
+        const int hc = p.CW / PIECES;                  // layers per piece: 8, 16 or 32
         bool ok = true;
         int as = 0, sb = 0;
         uint32_t aph = 0, sph = 0;
@@ -472,10 +473,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 // previous tile are still there.  Tile k adds columns 8k..8k+7 and emits the pooled columns
                 // 4k-1..4k+2 (windows 2pw..2pw+2) for the seven pooled rows that lie inside its 16 rows.
                 const uint32_t smX = base + p.off_pool;
-                const int et = threadIdx.x - 64;                       // 0 .. 128*HALVES-1
+                const int et = threadIdx.x - 64;                       // 0 .. 128*SPLIT-1
                 const int r = row >> 3, j = row & 7;
                 const int half = (warp - 2) >> 2;
-                const int cper = p.BN / HALVES;                        // layers this thread converts
+                const int cper = p.BN / SPLIT;                         // layers this thread converts
                 const int cb = (8 * tc.tw + 2 + j) & 15;
                 const uint32_t xpix = (uint32_t)p.BN * 2u + 16u;          // pixel pitch: 16 bytes of padding keep the 8
                                                                             // pixels a quarter-warp writes in different banks
@@ -739,7 +740,8 @@ struct Plan {
     CUtensorMap a, b, o;
     TcParams p;
     int grid;
-    int halves;      // kernel variant: 1 = two light CTAs per SM, 2 = one CTA per SM
+    int halves;      // 1 = two light CTAs per SM, 2 = one CTA per SM
+    int split;       // epilogue warps / 4 of the kernel variant: 1, 2 or 4
     size_t smem;
 };
 
@@ -820,6 +822,7 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     TcParams& p = plan->p;
     std::memset(&p, 0, sizeof(p));
     plan->halves = halves;
+    plan->split = halves;
     t_smem_limit = halves == 1 ? SMEM_LIMIT_2CTA : SMEM_LIMIT;
     p.Cout = d.Cout;
     p.c_off = d.out_c_offset;
@@ -896,6 +899,9 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
             !choose_layout(p, a_tile, false, 2, &plan->smem))
             return SQN_ERR_UNSUPPORTED;
     }
+    // (sixteen epilogue warps, SPLIT = 4, were measured slower than eight on every SqueezeNet shape: the
+    //  epilogue is limited by conversion and shared-memory throughput, not by latency; the variant is kept
+    //  for shapes where that may differ and is not selected automatically)
     p.use_ptab = 0;
     if (p.patch && p.taps * p.chunks * (p.BKc / 16) <= PARAM_TAB) {
         // operand offsets of every MMA of a tile, in issue order (tap-major, then chunk, then k-step)
@@ -1012,6 +1018,8 @@ int launch_plan(const Plan& plan, cudaStream_t stream)
     std::call_once(once, [] {
         attr_rc = cudaFuncSetAttribute(conv_tc_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
         if (attr_rc == cudaSuccess)
+            attr_rc = cudaFuncSetAttribute(conv_tc_kernel<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
+        if (attr_rc == cudaSuccess)
             attr_rc = cudaFuncSetAttribute(conv_tc_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
         if (attr_rc == cudaSuccess)
             attr_rc = cudaFuncSetAttribute(conv_tc_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -1020,8 +1028,10 @@ int launch_plan(const Plan& plan, cudaStream_t stream)
     if (attr_rc != cudaSuccess) return SQN_ERR_CUDA;
     if (plan.p.pool)
         conv_tc_kernel<2, true><<<plan.grid, threads_for(2), plan.smem, stream>>>(plan.a, plan.b, plan.o, plan.p);
-    else if (plan.halves == 1)
+    else if (plan.split == 1)
         conv_tc_kernel<1, false><<<plan.grid, threads_for(1), plan.smem, stream>>>(plan.a, plan.b, plan.o, plan.p);
+    else if (plan.split == 4)
+        conv_tc_kernel<4, false><<<plan.grid, threads_for(4), plan.smem, stream>>>(plan.a, plan.b, plan.o, plan.p);
     else
         conv_tc_kernel<2, false><<<plan.grid, threads_for(2), plan.smem, stream>>>(plan.a, plan.b, plan.o, plan.p);
     note_launch();
