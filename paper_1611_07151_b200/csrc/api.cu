@@ -336,7 +336,7 @@ extern "C" int squeezenet_layer_output(const sqn_net* net, const char* name, voi
     if (!net || !name || !workspace || !ptr || batch <= 0 || batch > net->max_batch) return SQN_ERR_BADARG;
     const int i = find_slot(net, name);
     if (i < 0) return SQN_ERR_BADARG;
-    if (net->dtype == SQN_BF16 && (std::strcmp(name, "conv1") == 0 || std::strcmp(name, "fire4") == 0))
+    if (net->dtype == SQN_BF16 && batch >= 16 && (std::strcmp(name, "conv1") == 0 || std::strcmp(name, "fire4") == 0))
         return SQN_ERR_UNSUPPORTED;   // computed inside the kernels that write pool1 / pool4, never stored
     std::vector<size_t> offs;
     layout(net, batch, &offs, nullptr);
@@ -395,7 +395,10 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
     int rc;
     ConvDesc d;
     // conv1 7x7/2 + ReLU, then max-pool
-    if (dt == SQN_BF16) {
+    // The fused conv+pool kernels hand a whole strip of 16 output rows to one CTA: worth it once there are
+    // enough strips to fill the GPU (8 per image for conv1, 4 for fire4), i.e. from a batch of 16 on.
+    const bool fuse_pools = dt == SQN_BF16 && batch >= 16;
+    if (fuse_pools) {
         // stem and its max-pool in one kernel: the 96x111x111 map never goes to memory
         rc = make_conv_desc(in_nhwc, net->w[0], net->b[0], buf("pool1"), 3, 96, IMG, IMG, 7, 2, 0, batch, 1, 0, 0, &d);
         if (rc != SQN_OK) return rc;
@@ -407,7 +410,13 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
     } else {
         rc = make_conv_desc(in_nhwc, net->w[0], net->b[0], buf("conv1"), 3, 96, IMG, IMG, 7, 2, 0, batch, 1, 0, 0, &d);
         if (rc != SQN_OK) return rc;
-        if ((rc = launch_conv_f32(d, st)) != SQN_OK) return rc;
+        if (dt == SQN_BF16) {
+            if ((rc = launch_stem_pack_bf16(d, ws + stem_off, total - stem_off, st)) != SQN_OK) return rc;
+            mark("conv1_pack");
+            if ((rc = launch_stem_conv_bf16(d, ws + stem_off, total - stem_off, st)) != SQN_OK) return rc;
+        } else {
+            if ((rc = launch_conv_f32(d, st)) != SQN_OK) return rc;
+        }
         mark("conv1");
         if ((rc = launch_maxpool3x3s2(buf("conv1"), buf("pool1"), 96, 111, 111, batch, dt, st)) != SQN_OK) return rc;
         mark("pool1");
@@ -434,7 +443,7 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
         // bf16: where a max-pool follows and the expands' kernels fit in shared memory, both expands pool
         // in their epilogues and write their halves of the pooled map; the unpooled map is never stored
         bool fused_pool = false;
-        if (f.pool_after && dt == SQN_BF16) {
+        if (f.pool_after && fuse_pools) {
             const std::string pn = std::string("pool") + (f.name + 4);
             ConvDesc p1 = d1, p3 = d3;
             p1.out = p3.out = buf(pn);

@@ -100,23 +100,21 @@ __global__ void maxpool_bf16_s(const __nv_bfloat16* __restrict__ in, __nv_bfloat
     out[idx] = __float2bfloat16(m);
 }
 
-// Global average + softmax.  One block of 1024 threads per image.  Thread t sums layers
-// (2p, 2p+1), p = t % 512 (+512, ...), over one half of the pixels (t / 512): consecutive threads read
-// consecutive 4- or 8-byte words of a pixel, four pixels are in flight per thread.  The halves are
-// combined in shared memory, where the logits stay for the softmax.
+// Global average: block (x = group of 128 layers, y = image), 256 threads = 64 layer pairs x 4 pixel
+// quarters.  Consecutive threads read consecutive 4- or 8-byte words of a pixel; the quarters are combined
+// in shared memory.  Small batches still get C/128 blocks per image.
 template <bool BF16>
-__global__ void __launch_bounds__(1024) avgpool_softmax_kernel(const void* __restrict__ in_, float* __restrict__ logits,
-                                                                float* __restrict__ probs, int C, int HW)
+__global__ void __launch_bounds__(256) global_avgpool_kernel(const void* __restrict__ in_, float* __restrict__ logits,
+                                                             int C, int HW)
 {
-    extern __shared__ float z[];          // [2][C] partial sums, then z[0..C) = logits / exponentials
-    __shared__ float red[32];
-    const int n = blockIdx.x;
+    __shared__ float part[4][128];
+    const int n = blockIdx.y;
     const int tid = threadIdx.x;
-    const int half = tid >> 9, lane_p = tid & 511;
-    const int p_lo = half ? HW / 2 : 0, p_hi = half ? HW : HW / 2;
-    const float inv = 1.0f / (float)HW;
-    for (int c = 2 * lane_p; c < C; c += 1024) {
-        float s0 = 0.f, s1 = 0.f, t0 = 0.f, t1 = 0.f, u0 = 0.f, u1 = 0.f, v0 = 0.f, v1 = 0.f;
+    const int quarter = tid >> 6;
+    const int c = blockIdx.x * 128 + 2 * (tid & 63);
+    const int p_lo = quarter * HW / 4, p_hi = (quarter + 1) * HW / 4;
+    float s0 = 0.f, s1 = 0.f, t0 = 0.f, t1 = 0.f, u0 = 0.f, u1 = 0.f, v0 = 0.f, v1 = 0.f;
+    if (c < C) {
         const bool pair = (c + 1 < C) && (C % 2 == 0);
         auto ld = [&](int p, float& a, float& b) {
             if (BF16) {
@@ -142,30 +140,33 @@ __global__ void __launch_bounds__(1024) avgpool_softmax_kernel(const void* __res
         int p = p_lo;
         for (; p + 4 <= p_hi; p += 4) { ld(p, s0, s1); ld(p + 1, t0, t1); ld(p + 2, u0, u1); ld(p + 3, v0, v1); }
         for (; p < p_hi; ++p) ld(p, s0, s1);
-        z[half * C + c] = (s0 + t0) + (u0 + v0);
-        if (c + 1 < C) z[half * C + c + 1] = (s1 + t1) + (u1 + v1);
     }
+    part[quarter][2 * (tid & 63)] = (s0 + t0) + (u0 + v0);
+    part[quarter][2 * (tid & 63) + 1] = (s1 + t1) + (u1 + v1);
     __syncthreads();
-    for (int c = tid; c < C; c += 1024) {
-        const float s = (z[c] + z[C + c]) * inv;
-        z[c] = s;
-        logits[(size_t)n * C + c] = s;
+    if (tid < 128) {
+        const int cc = blockIdx.x * 128 + tid;
+        if (cc < C)
+            logits[(size_t)n * C + cc] = ((part[0][tid] + part[1][tid]) + (part[2][tid] + part[3][tid])) / (float)HW;
     }
-    __syncthreads();
-    if (probs == nullptr) return;
+}
 
-    const int lane = tid & 31, warp = tid >> 5;
+// Softmax over the C logits of one image per block.
+__global__ void __launch_bounds__(256) softmax_kernel(const float* __restrict__ logits, float* __restrict__ probs, int C)
+{
+    extern __shared__ float z[];
+    __shared__ float red[8];
+    const int n = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     float m = -INFINITY;
-    for (int c = tid; c < C; c += 1024) m = fmaxf(m, z[c]);
+    for (int c = tid; c < C; c += 256) { z[c] = logits[(size_t)n * C + c]; m = fmaxf(m, z[c]); }
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
     if (lane == 0) red[warp] = m;
     __syncthreads();
     m = red[0];
-    for (int i = 1; i < 32; ++i) m = fmaxf(m, red[i]);
+    for (int i = 1; i < 8; ++i) m = fmaxf(m, red[i]);
     __syncthreads();
-
     float s = 0.f;
-    for (int c = tid; c < C; c += 1024) {
+    for (int c = tid; c < C; c += 256) {
         const float e = expf(z[c] - m);
         z[c] = e;
         s += e;
@@ -174,9 +175,9 @@ __global__ void __launch_bounds__(1024) avgpool_softmax_kernel(const void* __res
     if (lane == 0) red[warp] = s;
     __syncthreads();
     s = 0.f;
-    for (int i = 0; i < 32; ++i) s += red[i];
+    for (int i = 0; i < 8; ++i) s += red[i];
     const float r = 1.0f / s;
-    for (int c = tid; c < C; c += 1024) probs[(size_t)n * C + c] = z[c] * r;
+    for (int c = tid; c < C; c += 256) probs[(size_t)n * C + c] = z[c] * r;
 }
 
 }  // namespace
@@ -213,17 +214,15 @@ int launch_maxpool3x3s2(const void* in, void* out, int C, int H, int W, int N, i
 int launch_avgpool_softmax(const void* in, float* logits, float* probs, int C, int H, int W, int N, int dtype,
                            cudaStream_t stream)
 {
-    const size_t smem = 2 * (size_t)C * sizeof(float);
-    if (smem > 48 * 1024) {   // up to 64 KiB for C = 8192: above the default dynamic shared-memory limit
-        if (cudaFuncSetAttribute(avgpool_softmax_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024) != cudaSuccess ||
-            cudaFuncSetAttribute(avgpool_softmax_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024) != cudaSuccess)
-            return SQN_ERR_CUDA;
-    }
-    if (dtype == SQN_F32)
-        avgpool_softmax_kernel<false><<<N, 1024, smem, stream>>>(in, logits, probs, C, H * W);
-    else
-        avgpool_softmax_kernel<true><<<N, 1024, smem, stream>>>(in, logits, probs, C, H * W);
+    const dim3 grid((unsigned)((C + 127) / 128), (unsigned)N);
+    if (dtype == SQN_F32) global_avgpool_kernel<false><<<grid, 256, 0, stream>>>(in, logits, C, H * W);
+    else global_avgpool_kernel<true><<<grid, 256, 0, stream>>>(in, logits, C, H * W);
     note_launch();
+    if (cudaGetLastError() != cudaSuccess) return SQN_ERR_CUDA;
+    if (probs) {
+        softmax_kernel<<<N, 256, (size_t)C * sizeof(float), stream>>>(logits, probs, C);
+        note_launch();
+    }
     return cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
 }
 

@@ -184,3 +184,15 @@ def test_full_forward_bf16_top1():
     flips = logits.argmax(1) != z.argmax(1)
     assert agree >= 0.99 or (gap[flips] <= 2 * err[flips]).all(), (agree, gap[flips], err[flips])
     np.testing.assert_allclose(probs.astype(np.float64).sum(1), 1.0, rtol=0, atol=1e-5)
+
+
+def test_full_forward_bf16_small_batch_keeps_every_map():
+    """Below a batch of 16 the pools are separate kernels and every intermediate map can be read back."""
+    x, params = synth.squeezenet_case(7, 2)
+    trace = {}
+    z, _ = ref.squeezenet(x, params, trace=trace)
+    logits, probs, layers = run_net(x, params, BF16, 2)
+    assert "conv1" in layers and "fire4" in layers and len(layers) == len(trace) - 2      # all but logits, probs
+    assert max(G.rel_err(got, trace[name]) for name, got in layers.items()) <= 5e-2
+    assert G.rel_err(logits, z) <= TOL
+    np.testing.assert_allclose(probs.astype(np.float64).sum(1), 1.0, rtol=0, atol=1e-5)
