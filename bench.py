@@ -26,6 +26,7 @@ from paper_1611_07151_b200 import dist as D
 from paper_1611_07151_b200 import synth
 
 IMG = 227
+NCU_TRAFFIC_BYTES = {("conv1+pool1", "bf16", 256): 204.7e6}
 METRIC = "squeezenet_v1.0_forward_images_per_s"
 UNIT = "images/s"
 
@@ -166,7 +167,7 @@ def run_reference(args):
     sample = "%d of the %d images of the batch per step, full network, all host threads" % (n_img, args.batch)
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64 accumulate, f32 storage",
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
             "data": "synthetic",
             "config": {"workload": workload_name(args), "batch_per_gpu": args.batch, "sample": sample},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
@@ -397,7 +398,9 @@ def main():
     else:
         roof = {"bound": top["bound"], "achieved": top["tflops"], "peak": pipe_tf, "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = None
+    # dram__bytes_read.sum + dram__bytes_write.sum per launch from the single-pass ncu capture summarised in
+    # profiles/conv_tc_kernel_dram_bytes.md; None for any launch or configuration that capture does not cover
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get((top["name"], args.dtype, batch))
     roof["kernel"] = ("conv_tc_kernel" if dtype == B.SQN_BF16 else "conv_f32_kernel") + "[%s]" % top["name"]
     roof["peak_source"] = "of " + peaks["source"]
     roof["launch_ms"] = top["ms"]
