@@ -1,6 +1,7 @@
 // C-ABI entry points: argument validation, dispatch, the fire layer and the SqueezeNet v1.0
 // forward composition, host-side layout helpers.  No device memory is allocated here.
 #include <atomic>
+#include <cstdlib>
 #include <cmath>
 #include <cstring>
 #include <mutex>
@@ -13,6 +14,14 @@ namespace sqn {
 
 static std::atomic<unsigned long long> g_launches{0};
 void note_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+bool chained_launch_enabled()
+{
+    static const bool on = [] {
+        const char* v = std::getenv("SQN_CHAINED_LAUNCH");
+        return !(v && v[0] == '0');
+    }();
+    return on;
+}
 
 __device__ int g_device_status;   // written by kernels whose bounded waits run out
 

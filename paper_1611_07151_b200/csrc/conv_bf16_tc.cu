@@ -240,6 +240,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int nchunks = p.BN / p.CW;
     const int my_tiles = tiles_of_cta(p);
 
+    // The launch is chained to the kernel before it in the stream: this block may be running while
+    // that grid drains.  Up to chain_wait() below it touches only its own shared memory, TMEM and the
+    // kernel parameters.
+    chain_release();
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(smem_u32(&sh->full[s]), 1);
@@ -264,8 +268,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tmem_alloc(smem_u32(&sh->tmem_base), p.tmem_cols);
         tmem_relinquish();
     }
-    // bias of every output layer, once per CTA
-    for (int c = threadIdx.x; c < p.n_tiles * p.BN; c += NUM_THREADS) bias_s[c] = c < p.Cout ? __ldg(p.bias + c) : 0.f;
     if (p.patch) {
         // operand addresses of every MMA of a tile, in issue order (tap-major, then chunk, then k-step)
         const int ksteps = p.BKc / 16;
@@ -277,6 +279,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             sh->mma_tab[e] = make_uint2((a_off >> 4) + 2u * k, ((smB + (uint32_t)it * p.b_tile) >> 4) + 2u * k);
         }
     }
+    chain_wait();       // the earlier grid has finished: global memory may be read and written from here on
+    // bias of every output layer, once per CTA
+    for (int c = threadIdx.x; c < p.n_tiles * p.BN; c += NUM_THREADS) bias_s[c] = c < p.Cout ? __ldg(p.bias + c) : 0.f;
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -653,6 +658,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 __global__ void stem_pack_input(const __nv_bfloat16* __restrict__ in, uint2* __restrict__ out, int N, int H, int W,
                                 int Hp, int Wp)
 {
+    chain_release();
+    chain_wait();
     const int Wq = (Wp + 3) / 4;
     const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
     const long long total = (long long)N * Hp * Wq;
@@ -674,6 +681,8 @@ __global__ void stem_pack_input(const __nv_bfloat16* __restrict__ in, uint2* __r
 // Kernels [Cout][7][7][3] bf16 -> [Cout][7][8][4] bf16 (zero for the eighth column and fourth layer).
 __global__ void stem_pack_weights(const unsigned short* __restrict__ w, unsigned short* __restrict__ out, int Cout)
 {
+    chain_release();
+    chain_wait();       // also keeps the grids chained after this one behind the input repack
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= Cout * 224) return;
     const int c = idx & 3;
@@ -1026,14 +1035,17 @@ int launch_plan(const Plan& plan, cudaStream_t stream)
                                            (int)SMEM_LIMIT_2CTA);
     });
     if (attr_rc != cudaSuccess) return SQN_ERR_CUDA;
+    const dim3 grid((unsigned)plan.grid);
+    cudaError_t rc;
     if (plan.p.pool)
-        conv_tc_kernel<2, true><<<plan.grid, threads_for(2), plan.smem, stream>>>(plan.a, plan.b, plan.o, plan.p);
+        rc = launch_chained(conv_tc_kernel<2, true>, grid, dim3(threads_for(2)), plan.smem, stream, plan.a, plan.b, plan.o, plan.p);
     else if (plan.split == 1)
-        conv_tc_kernel<1, false><<<plan.grid, threads_for(1), plan.smem, stream>>>(plan.a, plan.b, plan.o, plan.p);
+        rc = launch_chained(conv_tc_kernel<1, false>, grid, dim3(threads_for(1)), plan.smem, stream, plan.a, plan.b, plan.o, plan.p);
     else if (plan.split == 4)
-        conv_tc_kernel<4, false><<<plan.grid, threads_for(4), plan.smem, stream>>>(plan.a, plan.b, plan.o, plan.p);
+        rc = launch_chained(conv_tc_kernel<4, false>, grid, dim3(threads_for(4)), plan.smem, stream, plan.a, plan.b, plan.o, plan.p);
     else
-        conv_tc_kernel<2, false><<<plan.grid, threads_for(2), plan.smem, stream>>>(plan.a, plan.b, plan.o, plan.p);
+        rc = launch_chained(conv_tc_kernel<2, false>, grid, dim3(threads_for(2)), plan.smem, stream, plan.a, plan.b, plan.o, plan.p);
+    if (rc != cudaSuccess) return SQN_ERR_CUDA;
     note_launch();
     return cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
 }
@@ -1146,12 +1158,13 @@ int launch_stem_pack_bf16(const ConvDesc& d, void* workspace, size_t workspace_b
     uint2* pin = reinterpret_cast<uint2*>(ws);
     unsigned short* pw = reinterpret_cast<unsigned short*>(ws + align_up((size_t)d.N * Hp * Wp * 8, 1024));
     const long long total = (long long)d.N * Hp * ((Wp + 3) / 4);
-    stem_pack_input<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(d.in), pin,
-                                                                        d.N, d.H, d.W, Hp, Wp);
-    stem_pack_weights<<<(d.Cout * 224 + 255) / 256, 256, 0, stream>>>(static_cast<const unsigned short*>(d.w), pw,
-                                                                       d.Cout);
+    cudaError_t e = launch_chained(stem_pack_input, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, stream,
+                                   static_cast<const __nv_bfloat16*>(d.in), pin, d.N, d.H, d.W, Hp, Wp);
+    if (e == cudaSuccess)
+        e = launch_chained(stem_pack_weights, dim3((unsigned)((d.Cout * 224 + 255) / 256)), dim3(256), 0, stream,
+                           static_cast<const unsigned short*>(d.w), pw, d.Cout);
     note_launch(2);
-    return cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
+    return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
 }
 
 // The stem convolution itself, on the repacked tensors left in the workspace by the call above.

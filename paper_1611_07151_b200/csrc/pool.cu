@@ -18,6 +18,8 @@ __device__ __forceinline__ float4 max4(float4 a, float4 b)
 __global__ void maxpool_f32_v4(const float* __restrict__ in, float* __restrict__ out, int C4, int H, int W, int OH,
                                int OW, long long total)
 {
+    chain_release();
+    chain_wait();
     const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
     if (idx >= total) return;
     const int c4 = (int)(idx % C4);
@@ -38,6 +40,8 @@ __global__ void maxpool_f32_v4(const float* __restrict__ in, float* __restrict__
 __global__ void maxpool_f32_s(const float* __restrict__ in, float* __restrict__ out, int C, int H, int W, int OH,
                               int OW, long long total)
 {
+    chain_release();
+    chain_wait();
     const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
     if (idx >= total) return;
     const int c = (int)(idx % C);
@@ -64,6 +68,8 @@ __device__ __forceinline__ uint32_t bmax2(uint32_t a, uint32_t b)
 __global__ void maxpool_bf16_v8(const uint4* __restrict__ in, uint4* __restrict__ out, int C8, int H, int W, int OH,
                                 int OW, long long total)
 {
+    chain_release();
+    chain_wait();
     const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
     if (idx >= total) return;
     const int c8 = (int)(idx % C8);
@@ -86,6 +92,8 @@ __global__ void maxpool_bf16_v8(const uint4* __restrict__ in, uint4* __restrict_
 __global__ void maxpool_bf16_s(const __nv_bfloat16* __restrict__ in, __nv_bfloat16* __restrict__ out, int C, int H,
                                int W, int OH, int OW, long long total)
 {
+    chain_release();
+    chain_wait();
     const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
     if (idx >= total) return;
     const int c = (int)(idx % C);
@@ -107,6 +115,8 @@ template <bool BF16>
 __global__ void __launch_bounds__(256) global_avgpool_kernel(const void* __restrict__ in_, float* __restrict__ logits,
                                                              int C, int HW)
 {
+    chain_release();
+    chain_wait();
     __shared__ float part[4][128];
     const int n = blockIdx.y;
     const int tid = threadIdx.x;
@@ -154,6 +164,8 @@ __global__ void __launch_bounds__(256) global_avgpool_kernel(const void* __restr
 // Softmax over the C logits of one image per block.
 __global__ void __launch_bounds__(256) softmax_kernel(const float* __restrict__ logits, float* __restrict__ probs, int C)
 {
+    chain_release();
+    chain_wait();
     extern __shared__ float z[];
     __shared__ float red[8];
     const int n = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -189,22 +201,23 @@ int launch_maxpool3x3s2(const void* in, void* out, int C, int H, int W, int N, i
     if (dtype == SQN_F32) {
         if (C % 4 == 0) {
             const long long total = (long long)N * OH * OW * (C / 4);
-            maxpool_f32_v4<<<(unsigned)((total + threads - 1) / threads), threads, 0, stream>>>(
-                static_cast<const float*>(in), static_cast<float*>(out), C / 4, H, W, OH, OW, total);
+            launch_chained(maxpool_f32_v4, dim3((unsigned)((total + threads - 1) / threads)), dim3(threads), 0, stream,
+                           static_cast<const float*>(in), static_cast<float*>(out), C / 4, H, W, OH, OW, total);
         } else {
             const long long total = (long long)N * OH * OW * C;
-            maxpool_f32_s<<<(unsigned)((total + threads - 1) / threads), threads, 0, stream>>>(
-                static_cast<const float*>(in), static_cast<float*>(out), C, H, W, OH, OW, total);
+            launch_chained(maxpool_f32_s, dim3((unsigned)((total + threads - 1) / threads)), dim3(threads), 0, stream,
+                           static_cast<const float*>(in), static_cast<float*>(out), C, H, W, OH, OW, total);
         }
     } else {
         if (C % 8 == 0) {
             const long long total = (long long)N * OH * OW * (C / 8);
-            maxpool_bf16_v8<<<(unsigned)((total + threads - 1) / threads), threads, 0, stream>>>(
-                static_cast<const uint4*>(in), static_cast<uint4*>(out), C / 8, H, W, OH, OW, total);
+            launch_chained(maxpool_bf16_v8, dim3((unsigned)((total + threads - 1) / threads)), dim3(threads), 0, stream,
+                           static_cast<const uint4*>(in), static_cast<uint4*>(out), C / 8, H, W, OH, OW, total);
         } else {
             const long long total = (long long)N * OH * OW * C;
-            maxpool_bf16_s<<<(unsigned)((total + threads - 1) / threads), threads, 0, stream>>>(
-                static_cast<const __nv_bfloat16*>(in), static_cast<__nv_bfloat16*>(out), C, H, W, OH, OW, total);
+            launch_chained(maxpool_bf16_s, dim3((unsigned)((total + threads - 1) / threads)), dim3(threads), 0, stream,
+                           static_cast<const __nv_bfloat16*>(in), static_cast<__nv_bfloat16*>(out), C, H, W, OH, OW,
+                           total);
         }
     }
     note_launch();
@@ -215,12 +228,13 @@ int launch_avgpool_softmax(const void* in, float* logits, float* probs, int C, i
                            cudaStream_t stream)
 {
     const dim3 grid((unsigned)((C + 127) / 128), (unsigned)N);
-    if (dtype == SQN_F32) global_avgpool_kernel<false><<<grid, 256, 0, stream>>>(in, logits, C, H * W);
-    else global_avgpool_kernel<true><<<grid, 256, 0, stream>>>(in, logits, C, H * W);
+    if (dtype == SQN_F32) launch_chained(global_avgpool_kernel<false>, grid, dim3(256), 0, stream, in, logits, C, H * W);
+    else launch_chained(global_avgpool_kernel<true>, grid, dim3(256), 0, stream, in, logits, C, H * W);
     note_launch();
     if (cudaGetLastError() != cudaSuccess) return SQN_ERR_CUDA;
     if (probs) {
-        softmax_kernel<<<N, 256, (size_t)C * sizeof(float), stream>>>(logits, probs, C);
+        launch_chained(softmax_kernel, dim3((unsigned)N), dim3(256), (size_t)C * sizeof(float), stream,
+                       static_cast<const float*>(logits), probs, C);
         note_launch();
     }
     return cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;

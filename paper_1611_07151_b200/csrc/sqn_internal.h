@@ -45,6 +45,36 @@ int launch_maxpool3x3s2(const void* in, void* out, int C, int H, int W, int N, i
 int launch_avgpool_softmax(const void* in, float* logits, float* probs, int C, int H, int W, int N, int dtype,
                            cudaStream_t stream);
 
+// Chained launches.  A kernel launched through launch_chained() may be scheduled while the kernel before it
+// in the stream is still running (programmatic stream serialisation): its blocks take the SMs the earlier
+// grid frees and do their on-chip set-up there.  Every such kernel calls chain_wait() before its first
+// access to global memory; that returns once the earlier grid has finished and its writes are visible, so
+// the data dependences of a plain launch are kept.  chain_release() lets the grid after this one start its
+// own set-up early.  SQN_CHAINED_LAUNCH=0 in the environment turns the attribute off (plain launches).
+bool chained_launch_enabled();
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                  Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = chained_launch_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+#ifdef __CUDACC__
+__device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace sqn
