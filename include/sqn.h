@@ -75,7 +75,7 @@ int conv_forward(const void* in, const void* weights, const void* bias, void* ou
  *   workspace_bytes  device scratch, needed only when conv_workspace_bytes reports > 0
  *   fuse_maxpool   the 3x3 / stride 2 max-pool that follows the layer (paper Section III-E) is applied inside the
  *                  kernel and only the pooled map is written: out is [batch][(outH-3)/2+1][(outW-3)/2+1][out_c_total].
- *                  SQN_BF16 only, K >= 2 (or the stem shape), numOutputLayers a multiple of 32 up to 256, kernels
+ *                  SQN_BF16 only, stride 1 (or the stem shape), numOutputLayers a multiple of 32 up to 256, kernels
  *                  small enough to stay in shared memory; otherwise SQN_ERR_UNSUPPORTED.
  */
 typedef struct {

@@ -12,12 +12,14 @@
 // straight into the layer slice [c_off, c_off+Cout) of the destination tensor; the TMA unit
 // clips the parts of edge tiles that fall outside the map.
 //
-// One persistent CTA per SM, 6 warps:
+// Persistent CTAs (one per SM, or two light ones), warp roles:
 //   warp 0 (one thread)  TMA producer: ring of `stages` {A box, B box} slots, full/empty mbarriers
-//   warp 1 (one thread)  MMA issuer: tcgen05.mma 128 x BN x 16, commits free the slots;
-//                        two accumulators in TMEM so tile i+1 is multiplied while tile i drains
-//   warps 2..5           epilogue: tcgen05.ld (one output pixel per thread), +bias, ReLU, ->bf16,
-//                        swizzled staging tile in shared memory, TMA store
+//   warp 1 (one lane)    MMA issuer: tcgen05.mma 128 x BN x 16, commits free the slots; the last MMA of a
+//                        tile adds the bias (ones x bias rows); two accumulators in TMEM so tile i+1 is
+//                        multiplied while tile i drains
+//   4*SPLIT warps        epilogue: tcgen05.ld (one output pixel per thread), ReLU, ->bf16,
+//                        swizzled staging tile in shared memory
+//   last warp            TMA stores of the staged chunks
 // Every mbarrier wait is bounded: when it runs out the CTA records SQN_ERR_TIMEOUT in the
 // device status word, drains its outstanding copies, frees its TMEM and returns.
 #include <cuda.h>
@@ -25,6 +27,7 @@
 
 #include <cstring>
 #include <map>
+#include <cstddef>
 #include <mutex>
 #include <string>
 
@@ -46,6 +49,7 @@ constexpr int MAX_STG = 4;             // staging ring slots
 constexpr int MAX_TAB = 448;           // MMAs per tile in patch mode
 constexpr int PARAM_TAB = 160;         // ... of which this many can be tabulated in the kernel parameters
 constexpr size_t CTL_BYTES = 4096;
+constexpr size_t CTL_BYTES_NO_TAB = 1024;   // control block without the shared-memory MMA table
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // about two seconds
 constexpr size_t SMEM_LIMIT = 227 * 1024;
 constexpr size_t SMEM_LIMIT_2CTA = 113 * 1024;     // two CTAs share an SM's 228 KB (1 KB reserved each)
@@ -76,7 +80,7 @@ struct TcParams {
     unsigned tmem_cols;
     unsigned a_bytes, b_bytes;       // bytes one item's A box / B box delivers
     unsigned a_tile, b_tile;         // shared-memory bytes reserved per A / B tile
-    unsigned off_b, off_stg, off_bias, off_ctl;   // byte offsets from the 1024-aligned base
+    unsigned off_b, off_stg, off_bias, off_ones, off_ctl;   // byte offsets from the 1024-aligned base
     // fused 3x3/stride-2 max-pool (patch mode only): a CTA walks the tiles of a strip of output rows from
     // left to right, keeps the last columns in shared memory and emits pooled pixels directly
     int pool;                        // 1: write max-pooled output instead of the convolution's own
@@ -230,7 +234,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t smA = base;
     const uint32_t smB = base + p.off_b;
     const uint32_t smStg = base + p.off_stg;
-    float* bias_s = reinterpret_cast<float*>(base_ptr + p.off_bias);
     Shared* sh = reinterpret_cast<Shared*>(base_ptr + p.off_ctl);
 
     const int warp = threadIdx.x >> 5;
@@ -268,7 +271,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tmem_alloc(smem_u32(&sh->tmem_base), p.tmem_cols);
         tmem_relinquish();
     }
-    if (p.patch) {
+    if (p.patch && !p.use_ptab) {
         // operand addresses of every MMA of a tile, in issue order (tap-major, then chunk, then k-step)
         const int ksteps = p.BKc / 16;
         for (int e = threadIdx.x; e < items * ksteps; e += NUM_THREADS) {
@@ -280,8 +283,28 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
     }
     chain_wait();       // the earlier grid has finished: global memory may be read and written from here on
-    // bias of every output layer, once per CTA
-    for (int c = threadIdx.x; c < p.n_tiles * p.BN; c += NUM_THREADS) bias_s[c] = c < p.Cout ? __ldg(p.bias + c) : 0.f;
+    // The bias is added by the tensor core: the last MMA of every tile multiplies a tile of ones
+    // (128 rows, K = 16: ones in the first two places) by the bias rows (one per output layer:
+    // {hi, lo, 0, ...} with hi + lo = bias to 16 bits below its leading bit).  Both tiles have
+    // 32-byte rows in the 32-byte swizzle: 16-byte unit u of row r sits at unit u ^ ((r >> 2) & 1).
+    {
+        uint4* ones = reinterpret_cast<uint4*>(base_ptr + p.off_ones);
+        for (int r = threadIdx.x; r < TILE_M; r += NUM_THREADS) {
+            const int u = (r >> 2) & 1;
+            ones[2 * r + u] = make_uint4(0x3f803f80u, 0u, 0u, 0u);
+            ones[2 * r + (u ^ 1)] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        uint4* rows = reinterpret_cast<uint4*>(base_ptr + p.off_bias);
+        for (int c = threadIdx.x; c < p.n_tiles * p.BN; c += NUM_THREADS) {
+            const float b = c < p.Cout ? __ldg(p.bias + c) : 0.f;
+            const __nv_bfloat16 hi = __float2bfloat16_rn(b);
+            const __nv_bfloat16 lo = __float2bfloat16_rn(b - __bfloat162float(hi));
+            const int u = (c >> 2) & 1;
+            rows[2 * c + u] = make_uint4((uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16), 0u, 0u, 0u);
+            rows[2 * c + (u ^ 1)] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        fence_proxy_async_smem();       // the MMA reads them through the async proxy
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -366,11 +389,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const uint32_t a_tile16 = p.a_tile >> 4, b_tile16 = p.b_tile >> 4;
         const uint32_t smA16 = smA >> 4, smB16 = smB >> 4;
         const int nmma = items * ksteps;
+        // bias MMA: ones tile x bias rows of the tile's output layers (32 bytes = 2 address units per row)
+        const uint64_t bias_da = make_kmajor_desc(base + p.off_ones, 32u, 256u);
+        const uint64_t bias_db0 = make_kmajor_desc(base + p.off_bias, 32u, 256u);
         bool ok = true;
         if (p.b_resident) ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->b_full), 0u, abort_flag, p.status));
         int s = 0, as = 0;
         uint32_t ph = 0, aph = 0;
-        for (int it = 0; it < my_tiles && ok; ++it) {
+        TileCoord tc;
+        tile_first(p, blockIdx.x, tc);
+        for (int it = 0; it < my_tiles && ok; ++it, tile_next(p, tc)) {
+            const uint64_t bias_db = bias_db0 + (uint64_t)(2 * tc.nt * p.BN);
             ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_empty[as]), aph ^ 1u, abort_flag, p.status));
             if (!ok) break;
             tc_fence_after();
@@ -404,6 +433,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         }
                     }
                     mma_commit(smem_u32(&sh->empty[s]));            // patch slot free once these MMAs have read it
+                    mma_bf16_ss(d_tmem, bias_da, bias_db, idesc, 1u);
                     mma_commit(smem_u32(&sh->tmem_full[as]));       // accumulator complete
                 }
                 __syncwarp();
@@ -427,7 +457,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             mma_bf16_ss(d_tmem, da + 6, db + 6, idesc, 1u);
                         }
                         mma_commit(smem_u32(&sh->empty[s]));        // slot free once these MMAs have read it
-                        if (i == items - 1) mma_commit(smem_u32(&sh->tmem_full[as]));   // accumulator complete
+                        if (i == items - 1) {
+                            mma_bf16_ss(d_tmem, bias_da, bias_db, idesc, 1u);
+                            mma_commit(smem_u32(&sh->tmem_full[as]));           // accumulator complete
+                        }
                     }
                     __syncwarp();
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
@@ -439,7 +472,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     } else if (warp < 2 + EPI_WARPS) {
         // -------------------------------------------------------------------- epilogue
         // 4*SPLIT warps: warp w reads TMEM lane quadrant w % 4 (one output pixel per thread) and, of
-        // every chunk of CW layers, the piece(s) given by (w - 2) / 4.  TMEM -> registers, + bias, ReLU, -> bf16,
+        // every chunk of CW layers, the piece(s) given by (w - 2) / 4.  TMEM -> registers (bias already added by the last MMA), ReLU, -> bf16,
         // into a slot of the staging ring (TMA-swizzled rows); the store warp sends the slot to
         // global memory while the next chunk is converted.
         const int q = warp & 3;
@@ -490,17 +523,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     uint32_t v[16];
                     tmem_ld_x16(taddr + (uint32_t)(half * cper + c16), v);
                     tmem_ld_wait();
-                    const float4* bch = reinterpret_cast<const float4*>(bias_s + half * cper + c16);
-                    const float4 b0 = bch[0], b1 = bch[1], b2 = bch[2], b3 = bch[3];
                     float f[16];
-                    f[0] = __uint_as_float(v[0]) + b0.x;   f[1] = __uint_as_float(v[1]) + b0.y;
-                    f[2] = __uint_as_float(v[2]) + b0.z;   f[3] = __uint_as_float(v[3]) + b0.w;
-                    f[4] = __uint_as_float(v[4]) + b1.x;   f[5] = __uint_as_float(v[5]) + b1.y;
-                    f[6] = __uint_as_float(v[6]) + b1.z;   f[7] = __uint_as_float(v[7]) + b1.w;
-                    f[8] = __uint_as_float(v[8]) + b2.x;   f[9] = __uint_as_float(v[9]) + b2.y;
-                    f[10] = __uint_as_float(v[10]) + b2.z; f[11] = __uint_as_float(v[11]) + b2.w;
-                    f[12] = __uint_as_float(v[12]) + b3.x; f[13] = __uint_as_float(v[13]) + b3.y;
-                    f[14] = __uint_as_float(v[14]) + b3.z; f[15] = __uint_as_float(v[15]) + b3.w;
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) f[e] = __uint_as_float(v[e]);
                     uint32_t o[8];
 #pragma unroll
                     for (int e = 0; e < 8; ++e)
@@ -565,26 +590,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                 for (int h = 0; h < NH; ++h) {
                     const int col_h = (half0 + h) * hc;
-                    const float4* bch = reinterpret_cast<const float4*>(bias_s + n0 + c0 + col_h);
                     const uint32_t u_h = (uint32_t)(col_h >> 3);       // first 16-byte unit of this half-chunk
-                    // all bias loads first, then the arithmetic, then the stores: three independent batches
-                    float4 bv[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        if (4 * j < hc) bv[j] = bch[j];
                     uint32_t o[16];
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        if (4 * j < hc) {
-                            float f0 = __uint_as_float(v[h][4 * j + 0]) + bv[j].x, f1 = __uint_as_float(v[h][4 * j + 1]) + bv[j].y;
-                            float f2 = __uint_as_float(v[h][4 * j + 2]) + bv[j].z, f3 = __uint_as_float(v[h][4 * j + 3]) + bv[j].w;
-                            if (p.relu) {
-                                o[2 * j] = pack_relu_bf16x2(f0, f1);
-                                o[2 * j + 1] = pack_relu_bf16x2(f2, f3);
-                            } else {
-                                o[2 * j] = pack_bf16x2(f0, f1);
-                                o[2 * j + 1] = pack_bf16x2(f2, f3);
-                            }
+                    for (int j = 0; j < 16; ++j) {
+                        if (2 * j < hc) {
+                            const float f0 = __uint_as_float(v[h][2 * j]), f1 = __uint_as_float(v[h][2 * j + 1]);
+                            o[j] = p.relu ? pack_relu_bf16x2(f0, f1) : pack_bf16x2(f0, f1);
                         }
                     }
 #pragma unroll
@@ -772,14 +784,17 @@ int num_sms()
 // of A stages that fit (0 if the candidate does not fit at all).
 thread_local size_t t_smem_limit = SMEM_LIMIT;   // budget the layout search below works against
 
-int fit_stages(TcParams& p, size_t a_tile, bool want_resident, int cw, int nstg, size_t* smem_bytes)
+int fit_stages(TcParams& p, size_t a_tile, bool want_resident, int cw, int nstg, bool smem_tab, size_t* smem_bytes)
 {
     const size_t SMEM_LIMIT = t_smem_limit;
     const int items = p.taps * p.chunks;
     const size_t slot = (size_t)TILE_M * cw * 2;
-    const size_t bias_bytes = ((size_t)p.n_tiles * p.BN * sizeof(float) + 1023) / 1024 * 1024;
-    const size_t ctl_bytes = CTL_BYTES;
-    static_assert(sizeof(Shared) <= CTL_BYTES, "control block");
+    // bias rows (32 bytes per output layer) followed by the tile of ones (128 rows of 32 bytes)
+    const size_t bias_rows = ((size_t)p.n_tiles * p.BN * 32 + 1023) / 1024 * 1024;
+    const size_t bias_bytes = bias_rows + (size_t)TILE_M * 32;
+    // the MMA operand table at the end of the control block is only needed when it does not fit the parameters
+    const size_t ctl_bytes = smem_tab ? CTL_BYTES : CTL_BYTES_NO_TAB;
+    static_assert(sizeof(Shared) <= CTL_BYTES && offsetof(Shared, mma_tab) <= CTL_BYTES_NO_TAB, "control block");
     if (SMEM_LIMIT < 1024 + bias_bytes + ctl_bytes) return 0;
     const size_t avail = SMEM_LIMIT - 1024 /*alignment slack*/ - bias_bytes - ctl_bytes;
     const size_t stg_bytes = p.pool ? ((size_t)16 * 16 * (p.BN * 2 + 16) + 1023) / 1024 * 1024   // column ring when pooling
@@ -807,18 +822,19 @@ int fit_stages(TcParams& p, size_t a_tile, bool want_resident, int cw, int nstg,
     p.off_stg = p.off_b + (unsigned)b_region;
     p.off_pool = p.off_stg;
     p.off_bias = p.off_stg + (unsigned)stg_bytes;
+    p.off_ones = p.off_bias + (unsigned)bias_rows;
     p.off_ctl = p.off_bias + (unsigned)bias_bytes;
     *smem_bytes = 1024 + (size_t)p.off_ctl + ctl_bytes;
     return stages;
 }
 
 // Tries the staging candidates in order of preference; true when one gives at least min_stages.
-bool choose_layout(TcParams& p, size_t a_tile, bool want_resident, int min_stages, size_t* smem_bytes)
+bool choose_layout(TcParams& p, size_t a_tile, bool want_resident, int min_stages, bool smem_tab, size_t* smem_bytes)
 {
     static const int cand[][2] = {{64, 4}, {64, 3}, {32, 4}, {64, 2}, {32, 3}, {32, 2}, {16, 4}, {16, 2}};
     for (const auto& c : cand) {
         if (p.BN % c[0] != 0) continue;
-        if (fit_stages(p, a_tile, want_resident, c[0], c[1], smem_bytes) >= min_stages) return true;
+        if (fit_stages(p, a_tile, want_resident, c[0], c[1], smem_tab, smem_bytes) >= min_stages) return true;
     }
     return false;
 }
@@ -889,7 +905,8 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
         if (max_rows < patch_w * patch_h) max_rows = patch_w * patch_h;
         p.patch_tile = ((unsigned)max_rows * row_bytes + 1023u) / 1024u * 1024u;
         if (patch_h <= 256 && p.sbo_bytes < (1u << 18) && p.taps * p.chunks * (p.BKc / 16) <= MAX_TAB &&
-            choose_layout(p, (size_t)p.chunks * p.patch_tile, true, 2, &plan->smem)) {
+            choose_layout(p, (size_t)p.chunks * p.patch_tile, true, 2, p.taps * p.chunks * (p.BKc / 16) > PARAM_TAB,
+                          &plan->smem)) {
             patch_ok = true;
             p.patch = 1;
             p.BW = 8; p.BH = bh; p.BI = 1;
@@ -904,8 +921,8 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
         else choose_box(OW, OH, NI, &p.BW, &p.BH, &p.BI);
         p.a_bytes = (unsigned)(p.BW * p.BH * p.BI) * row_bytes;
         const size_t a_tile = (size_t)TILE_M * row_bytes;
-        if (!choose_layout(p, a_tile, true, 3, &plan->smem) && !choose_layout(p, a_tile, false, 3, &plan->smem) &&
-            !choose_layout(p, a_tile, false, 2, &plan->smem))
+        if (!choose_layout(p, a_tile, true, 3, false, &plan->smem) && !choose_layout(p, a_tile, false, 3, false, &plan->smem) &&
+            !choose_layout(p, a_tile, false, 2, false, &plan->smem))
             return SQN_ERR_UNSUPPORTED;
     }
     // (sixteen epilogue warps, SPLIT = 4, were measured slower than eight on every SqueezeNet shape: the
