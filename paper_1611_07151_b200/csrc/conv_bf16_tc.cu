@@ -1026,13 +1026,13 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
 // Two light CTAs per SM when the layer's tiles, kernels and accumulators fit twice; else one CTA per SM.
 int build_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_ptr, int Hp, int Wp, Plan* plan)
 {
-    // Measured on B200 over the SqueezeNet shapes: the light variant wins where one MMA thread per SM is the
-    // limit (many small MMAs per tile, short epilogue): patch-mode layers up to 64 output layers and 1x1
-    // layers up to 32 output layers with at least three MMAs per tile.  Elsewhere the deeper rings win.
+    // Measured on B200 over the SqueezeNet shapes: two light CTAs per SM (two independent producer / MMA /
+    // epilogue chains) win for patch-mode layers up to 64 output layers and for 1x1 layers whose light layout
+    // still has three A stages; with fewer stages (large kernels resident) or wider tiles the deep rings of
+    // the single CTA win.
     if (build_plan_cfg(d, stem, a_ptr, w_ptr, Hp, Wp, 1, plan) == SQN_OK) {
         const TcParams& p = plan->p;
-        const int nmma = p.taps * p.chunks * (p.BKc / 16);
-        if ((p.patch && p.BN <= 64) || (!p.patch && p.BN <= 32 && nmma >= 3)) return SQN_OK;
+        if ((p.patch && p.BN <= 64) || (!p.patch && p.stages >= 3)) return SQN_OK;
     }
     return build_plan_cfg(d, stem, a_ptr, w_ptr, Hp, Wp, 2, plan);
 }
