@@ -488,13 +488,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         bool ok = true;
         int as = 0, sb = 0;
         uint32_t aph = 0, sph = 0;
-        // fused max-pool: the (pooled pixel, 16-byte vector) items of this thread are the same for every
-        // tile, so they are worked out once (28 pooled pixels x BN/8 vectors over the epilogue threads)
-        int pool_item[4] = {-1, -1, -1, -1};
+        // fused max-pool: a thread's item is the same for every tile: one pooled row, a pair of adjacent
+        // pooled columns (their windows share a column: 15 loads for two outputs) and one 16-byte vector of
+        // layers; 7 rows x 2 pairs x BN/8 vectors <= 224 items over the epilogue threads
+        int pool_vec = -1, pool_pr = 0, pool_pair = 0;
         if (POOL) {
-            const int vecs = p.BN >> 3, nwork = 28 * vecs;
-            for (int k = 0, wk = threadIdx.x - 64; k < 4 && wk < nwork; ++k, wk += EPI_WARPS * 32)
-                pool_item[k] = ((wk / vecs) << 16) | (wk % vecs);
+            const int vecs = p.BN >> 3, wk = threadIdx.x - 64;
+            if (wk < 14 * vecs) {
+                pool_vec = wk % vecs;
+                pool_pair = (wk / vecs) & 1;
+                pool_pr = (wk / vecs) >> 1;
+            }
         }
         TileCoord tc;
         tile_first(p, blockIdx.x, tc);
@@ -542,27 +546,26 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (++as == 2) { as = 0; aph ^= 1u; }
                 asm volatile("bar.sync 1, %0;" ::"r"(EPI_WARPS * 32) : "memory");      // tile is in the ring
                 const int ph0 = tc.th * 7, pw0 = tc.tw * 4 - 1, img = tc.ti;
+                const int ph = ph0 + pool_pr, pwa = pw0 + 2 * pool_pair;     // pooled columns pwa and pwa + 1
+                if (pool_vec >= 0 && ph < p.PH_out && pwa + 1 >= 0 && pwa < p.PW_out) {
+                    uint4 ma = make_uint4(0u, 0u, 0u, 0u), mb = ma;
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {                            // this thread's (pooled pixel, vector) items
-                    if (pool_item[k] < 0) continue;
-                    const int vec = pool_item[k] & 0xffff;
-                    const int px = pool_item[k] >> 16;
-                    const int pi = px & 3, pr = px >> 2;
-                    const int pw = pw0 + pi, ph = ph0 + pr;
-                    if (pw < 0 || pw >= p.PW_out || ph >= p.PH_out) continue;
-                    uint4 m = make_uint4(0u, 0u, 0u, 0u);
+                    for (int dy = 0; dy < 3; ++dy) {
+                        uint4 w[5];
 #pragma unroll
-                    for (int dy = 0; dy < 3; ++dy)
-#pragma unroll
-                        for (int dx = 0; dx < 3; ++dx) {
-                            const int xr = 2 * pr + dy, xc = (8 * tc.tw + 2 * pi + dx) & 15;
-                            uint4 w;
-                            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(w.x), "=r"(w.y), "=r"(w.z), "=r"(w.w)
-                                         : "r"(smX + (uint32_t)(xr * 16 + xc) * xpix + (uint32_t)(vec * 16)) : "memory");
-                            m = (dy == 0 && dx == 0) ? w : bmax8(m, w);
+                        for (int dx = 0; dx < 5; ++dx) {
+                            const int xr = 2 * pool_pr + dy, xc = (8 * tc.tw + 4 * pool_pair + dx) & 15;
+                            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                         : "=r"(w[dx].x), "=r"(w[dx].y), "=r"(w[dx].z), "=r"(w[dx].w)
+                                         : "r"(smX + (uint32_t)(xr * 16 + xc) * xpix + (uint32_t)(pool_vec * 16)) : "memory");
                         }
-                    __nv_bfloat16* dst = p.pool_out + (((size_t)img * p.PH_out + ph) * p.PW_out + pw) * p.pool_ctot + p.c_off + vec * 8;
-                    *reinterpret_cast<uint4*>(dst) = m;
+                        const uint4 ra = bmax8(bmax8(w[0], w[1]), w[2]), rb = bmax8(bmax8(w[2], w[3]), w[4]);
+                        ma = dy == 0 ? ra : bmax8(ma, ra);
+                        mb = dy == 0 ? rb : bmax8(mb, rb);
+                    }
+                    __nv_bfloat16* dst = p.pool_out + (((size_t)img * p.PH_out + ph) * p.PW_out + pwa) * p.pool_ctot + p.c_off + pool_vec * 8;
+                    if (pwa >= 0) *reinterpret_cast<uint4*>(dst) = ma;
+                    if (pwa + 1 < p.PW_out) *reinterpret_cast<uint4*>(dst + p.pool_ctot) = mb;
                 }
                 asm volatile("bar.sync 1, %0;" ::"r"(EPI_WARPS * 32) : "memory");      // ring columns may be overwritten
                 continue;
