@@ -44,6 +44,10 @@ constexpr int TILE_M = 128;            // MMA M: TMEM lanes
 // (large tiles, kernels resident in up to 227 KB); SPLIT = 1: two lighter CTAs per SM, i.e. two MMA issuers,
 // two producers and two store threads per SM, for the layers whose tiles are small.
 __host__ __device__ constexpr int threads_for(int split) { return 96 + 128 * split; }
+// With the max-pool fused the store warp is replaced by POOL_WARPS warps that pool the tiles the epilogue warps wrote.
+constexpr int POOL_WARPS = 8;
+__host__ __device__ constexpr int threads_of(int split, bool pool) { return pool ? 64 + 128 * split + 32 * POOL_WARPS : threads_for(split); }
+constexpr int RING_COLS = 24;          // column ring of the fused max-pool: three tiles of eight columns
 constexpr int MAX_STAGES = 8;
 constexpr int MAX_STG = 4;             // staging ring slots
 constexpr int MAX_TAB = 448;           // MMAs per tile in patch mode
@@ -87,7 +91,7 @@ struct TcParams {
     int h_step;                      // output rows between consecutive tile rows (BH, or 14 when pooling)
     int PW_out, PH_out;              // pooled extents
     int pool_ctot;                   // layers per pixel of the pooled tensor
-    unsigned off_pool;               // shared-memory offset of the column ring [16 rows][16 cols][BN]
+    unsigned off_pool;               // shared-memory offset of the column ring [16 rows][24 cols][BN]
     __nv_bfloat16* pool_out;
     const float* bias;
     int* status;
@@ -105,6 +109,8 @@ struct Shared {                       // control block placed after the tiles
     unsigned long long tmem_empty[2];
     unsigned long long stg_full[MAX_STG];
     unsigned long long stg_free[MAX_STG];
+    unsigned long long ring_full[2];      // fused max-pool: tile written to the column ring / pooled and released
+    unsigned long long ring_free[2];
     unsigned tmem_base;
     volatile int abort_flag;
     uint2 mma_tab[MAX_TAB + 1];           // patch mode: per MMA, {A offset from the stage base, B address} in 16-byte units
@@ -192,22 +198,6 @@ __device__ __forceinline__ int tiles_of_cta(const TcParams& p)
     return p.pool ? mine * p.tiles_w : mine;
 }
 
-// AND of a predicate over the 4*SPLIT epilogue warps (named barrier 2); used where those warps meet at
-// barriers afterwards, so that all of them take the same way out when a bounded wait has run out.
-__device__ __forceinline__ bool epilogue_vote(bool ok, int nthreads)
-{
-    uint32_t all;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.u32 q, %1, 0;\n\t"
-        "bar.red.and.pred p, 2, %2, q;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(all)
-        : "r"((uint32_t)ok), "r"(nthreads)
-        : "memory");
-    return all != 0;
-}
-
 __device__ __forceinline__ uint4 bmax8(uint4 a, uint4 b)
 {
     uint4 r;
@@ -220,11 +210,11 @@ __device__ __forceinline__ uint4 bmax8(uint4 a, uint4 b)
 }
 
 template <int SPLIT, bool POOL>
-__global__ void __launch_bounds__(threads_for(SPLIT), SPLIT == 1 ? 2 : 1)
+__global__ void __launch_bounds__(threads_of(SPLIT, POOL), SPLIT == 1 ? 2 : 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmO, const TcParams p)
 {
-    constexpr int NUM_THREADS = threads_for(SPLIT);
+    constexpr int NUM_THREADS = threads_of(SPLIT, POOL);
     constexpr int EPI_WARPS = 4 * SPLIT;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -260,6 +250,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int b = 0; b < p.nstg; ++b) {
             mbar_init(smem_u32(&sh->stg_full[b]), EPI_WARPS);
             mbar_init(smem_u32(&sh->stg_free[b]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&sh->ring_full[b]), EPI_WARPS);
+            mbar_init(smem_u32(&sh->ring_free[b]), POOL_WARPS);
         }
         sh->abort_flag = 0;
         fence_mbar_init();
@@ -488,41 +482,34 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         bool ok = true;
         int as = 0, sb = 0;
         uint32_t aph = 0, sph = 0;
-        // fused max-pool: a thread's item is the same for every tile: one pooled row, a pair of adjacent
-        // pooled columns (their windows share a column: 15 loads for two outputs) and one 16-byte vector of
-        // layers; 7 rows x 2 pairs x BN/8 vectors <= 224 items over the epilogue threads
-        int pool_vec = -1, pool_pr = 0, pool_pair = 0;
-        if (POOL) {
-            const int vecs = p.BN >> 3, wk = threadIdx.x - 64;
-            if (wk < 14 * vecs) {
-                pool_vec = wk % vecs;
-                pool_pair = (wk / vecs) & 1;
-                pool_pr = (wk / vecs) >> 1;
-            }
-        }
+        int ring0 = 0;                                 // fused max-pool: first ring column of the current tile
         TileCoord tc;
         tile_first(p, blockIdx.x, tc);
         for (int it = 0; it < my_tiles && ok; ++it, tile_next(p, tc)) {
             const int n0 = tc.nt * p.BN;
             ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_full[as]), aph, abort_flag, p.status));
-            if (POOL) ok = epilogue_vote(ok, EPI_WARPS * 32);        // the pooled path meets at barriers below
             if (!ok) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * p.bn_pad);
             if (POOL) {
-                // ---- fused max-pool.  Column ring X[16 rows][16 columns][BN] (bf16): output column x of the
-                // strip lives at ring column (x + 2) & 15, so the two columns a window may need from the
-                // previous tile are still there.  Tile k adds columns 8k..8k+7 and emits the pooled columns
-                // 4k-1..4k+2 (windows 2pw..2pw+2) for the seven pooled rows that lie inside its 16 rows.
+                // ---- fused max-pool, first half: the tile goes into the column ring X[16 rows][24 columns][BN]
+                // (bf16).  The k-th tile of this CTA owns ring columns 8k+2 .. 8k+9 (mod 24); the pool warps
+                // read 8k .. 8k+9, i.e. also the last two columns of the tile before, and emit the pooled
+                // columns 4*tw-1 .. 4*tw+2 of the seven pooled rows inside the tile's 16 rows.  The last
+                // readers of columns 8k+2 .. 8k+9 are the windows of tile k-2 (its columns 8k+8 and 8k+9 mod 24),
+                // so tile k is written while tile k-1 is being pooled.
                 const uint32_t smX = base + p.off_pool;
-                const int et = threadIdx.x - 64;                       // 0 .. 128*SPLIT-1
+                const int rb = it & 1;
+                ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->ring_free[rb]), (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag, p.status));
+                if (!ok) break;
                 const int r = row >> 3, j = row & 7;
                 const int half = (warp - 2) >> 2;
                 const int cper = p.BN / SPLIT;                         // layers this thread converts
-                const int cb = (8 * tc.tw + 2 + j) & 15;
+                int cb = ring0 + 2 + j;
+                if (cb >= RING_COLS) cb -= RING_COLS;
                 const uint32_t xpix = (uint32_t)p.BN * 2u + 16u;          // pixel pitch: 16 bytes of padding keep the 8
                                                                             // pixels a quarter-warp writes in different banks
-                const uint32_t xrow = smX + (uint32_t)(r * 16 + cb) * xpix + (uint32_t)(half * cper * 2);
+                const uint32_t xrow = smX + (uint32_t)(r * RING_COLS + cb) * xpix + (uint32_t)(half * cper * 2);
                 for (int c16 = 0; c16 < cper; c16 += 16) {
                     uint32_t v[16];
                     tmem_ld_x16(taddr + (uint32_t)(half * cper + c16), v);
@@ -539,35 +526,16 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(xrow + (uint32_t)(c16 * 2 + 16)), "r"(o[4]),
                                  "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
                 }
-                // accumulator drained: hand it back to the MMA issuer
+                // accumulator drained: hand it back to the MMA issuer; tile is in the ring: hand it to the pool warps
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[as]));
-                if (++as == 2) { as = 0; aph ^= 1u; }
-                asm volatile("bar.sync 1, %0;" ::"r"(EPI_WARPS * 32) : "memory");      // tile is in the ring
-                const int ph0 = tc.th * 7, pw0 = tc.tw * 4 - 1, img = tc.ti;
-                const int ph = ph0 + pool_pr, pwa = pw0 + 2 * pool_pair;     // pooled columns pwa and pwa + 1
-                if (pool_vec >= 0 && ph < p.PH_out && pwa + 1 >= 0 && pwa < p.PW_out) {
-                    uint4 ma = make_uint4(0u, 0u, 0u, 0u), mb = ma;
-#pragma unroll
-                    for (int dy = 0; dy < 3; ++dy) {
-                        uint4 w[5];
-#pragma unroll
-                        for (int dx = 0; dx < 5; ++dx) {
-                            const int xr = 2 * pool_pr + dy, xc = (8 * tc.tw + 4 * pool_pair + dx) & 15;
-                            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
-                                         : "=r"(w[dx].x), "=r"(w[dx].y), "=r"(w[dx].z), "=r"(w[dx].w)
-                                         : "r"(smX + (uint32_t)(xr * 16 + xc) * xpix + (uint32_t)(pool_vec * 16)) : "memory");
-                        }
-                        const uint4 ra = bmax8(bmax8(w[0], w[1]), w[2]), rb = bmax8(bmax8(w[2], w[3]), w[4]);
-                        ma = dy == 0 ? ra : bmax8(ma, ra);
-                        mb = dy == 0 ? rb : bmax8(mb, rb);
-                    }
-                    __nv_bfloat16* dst = p.pool_out + (((size_t)img * p.PH_out + ph) * p.PW_out + pwa) * p.pool_ctot + p.c_off + pool_vec * 8;
-                    if (pwa >= 0) *reinterpret_cast<uint4*>(dst) = ma;
-                    if (pwa + 1 < p.PW_out) *reinterpret_cast<uint4*>(dst + p.pool_ctot) = mb;
+                if (lane == 0) {
+                    mbar_arrive(smem_u32(&sh->tmem_empty[as]));
+                    mbar_arrive(smem_u32(&sh->ring_full[rb]));
                 }
-                asm volatile("bar.sync 1, %0;" ::"r"(EPI_WARPS * 32) : "memory");      // ring columns may be overwritten
+                if (++as == 2) { as = 0; aph ^= 1u; }
+                ring0 += 8;
+                if (ring0 == RING_COLS) ring0 = 0;
                 continue;
             }
             for (int chunk = 0; chunk < nchunks; ++chunk) {
@@ -623,6 +591,51 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[as]));
             if (++as == 2) { as = 0; aph ^= 1u; }
         }
+    } else if (POOL) {
+        // ---- fused max-pool, second half: POOL_WARPS warps.  A thread's item is the same for every tile: one
+        // pooled row, a pair of adjacent pooled columns (their windows share a column: 15 loads for two
+        // outputs) and one 16-byte vector of layers; 7 rows x 2 pairs x BN/8 vectors <= 224 items.
+        const uint32_t smX = base + p.off_pool;
+        const uint32_t xpix = (uint32_t)p.BN * 2u + 16u;
+        const int vecs = p.BN >> 3, wk = (int)threadIdx.x - (64 + 32 * EPI_WARPS);
+        const bool has_item = wk < 14 * vecs;
+        const int pool_vec = wk % vecs, pool_pair = (wk / vecs) & 1, pool_pr = (wk / vecs) >> 1;
+        bool ok = true;
+        int ring0 = 0;
+        TileCoord tc;
+        tile_first(p, blockIdx.x, tc);
+        for (int it = 0; it < my_tiles && ok; ++it, tile_next(p, tc)) {
+            const int rb = it & 1;
+            ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->ring_full[rb]), ((uint32_t)it >> 1) & 1u, abort_flag, p.status));
+            if (!ok) break;
+            const int ph = tc.th * 7 + pool_pr, pwa = tc.tw * 4 - 1 + 2 * pool_pair;     // pooled columns pwa and pwa + 1
+            if (has_item && ph < p.PH_out && pwa + 1 >= 0 && pwa < p.PW_out) {
+                uint4 ma = make_uint4(0u, 0u, 0u, 0u), mb = ma;
+#pragma unroll
+                for (int dy = 0; dy < 3; ++dy) {
+                    uint4 w[5];
+#pragma unroll
+                    for (int dx = 0; dx < 5; ++dx) {
+                        const int xr = 2 * pool_pr + dy;
+                        int xc = ring0 + 4 * pool_pair + dx;
+                        if (xc >= RING_COLS) xc -= RING_COLS;
+                        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                     : "=r"(w[dx].x), "=r"(w[dx].y), "=r"(w[dx].z), "=r"(w[dx].w)
+                                     : "r"(smX + (uint32_t)(xr * RING_COLS + xc) * xpix + (uint32_t)(pool_vec * 16)) : "memory");
+                    }
+                    const uint4 ra = bmax8(bmax8(w[0], w[1]), w[2]), rb2 = bmax8(bmax8(w[2], w[3]), w[4]);
+                    ma = dy == 0 ? ra : bmax8(ma, ra);
+                    mb = dy == 0 ? rb2 : bmax8(mb, rb2);
+                }
+                __nv_bfloat16* dst = p.pool_out + (((size_t)tc.ti * p.PH_out + ph) * p.PW_out + pwa) * p.pool_ctot + p.c_off + pool_vec * 8;
+                if (pwa >= 0) *reinterpret_cast<uint4*>(dst) = ma;
+                if (pwa + 1 < p.PW_out) *reinterpret_cast<uint4*>(dst + p.pool_ctot) = mb;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->ring_free[rb]));     // (the ring was read with plain loads: in order)
+            ring0 += 8;
+            if (ring0 == RING_COLS) ring0 = 0;
+        }
     } else {
         // ----------------------------------------------------------------- store issuer
         if (lane == 0) {
@@ -632,7 +645,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             uint32_t sph = 0;
             TileCoord tc;
             tile_first(p, blockIdx.x, tc);
-            for (int it = 0; it < (p.pool ? 0 : my_tiles) && ok; ++it, tile_next(p, tc)) {
+            for (int it = 0; it < my_tiles && ok; ++it, tile_next(p, tc)) {
                 const int w0 = tc.tw * p.BW, h0 = tc.th * p.h_step, i0 = tc.ti * p.BI, n0 = tc.nt * p.BN;
                 for (int chunk = 0; chunk < nchunks; ++chunk) {
                     const int c0 = chunk * p.CW;
@@ -800,7 +813,7 @@ int fit_stages(TcParams& p, size_t a_tile, bool want_resident, int cw, int nstg,
     static_assert(sizeof(Shared) <= CTL_BYTES && offsetof(Shared, mma_tab) <= CTL_BYTES_NO_TAB, "control block");
     if (SMEM_LIMIT < 1024 + bias_bytes + ctl_bytes) return 0;
     const size_t avail = SMEM_LIMIT - 1024 /*alignment slack*/ - bias_bytes - ctl_bytes;
-    const size_t stg_bytes = p.pool ? ((size_t)16 * 16 * (p.BN * 2 + 16) + 1023) / 1024 * 1024   // column ring when pooling
+    const size_t stg_bytes = p.pool ? ((size_t)16 * RING_COLS * (p.BN * 2 + 16) + 1023) / 1024 * 1024   // column ring when pooling
                                     : (size_t)nstg * slot;
     const size_t b_all = (size_t)items * p.b_tile;
     int stages;
@@ -1058,7 +1071,7 @@ int launch_plan(const Plan& plan, cudaStream_t stream)
     const dim3 grid((unsigned)plan.grid);
     cudaError_t rc;
     if (plan.p.pool)
-        rc = launch_chained(conv_tc_kernel<2, true>, grid, dim3(threads_for(2)), plan.smem, stream, plan.a, plan.b, plan.o, plan.p);
+        rc = launch_chained(conv_tc_kernel<2, true>, grid, dim3(threads_of(2, true)), plan.smem, stream, plan.a, plan.b, plan.o, plan.p);
     else if (plan.split == 1)
         rc = launch_chained(conv_tc_kernel<1, false>, grid, dim3(threads_for(1)), plan.smem, stream, plan.a, plan.b, plan.o, plan.p);
     else if (plan.split == 4)
