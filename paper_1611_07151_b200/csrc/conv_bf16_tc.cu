@@ -70,7 +70,9 @@ struct TcParams {
     int k_per_tap;                   // reduction elements per tap in the kernel matrix
     int patch;                       // 1: one input patch per tile serves every tap (see below)
     int taps_h;                      // kernel rows
-    int tap_h_rows, tap_w_rows;      // patch rows to skip per kernel row / kernel column
+    unsigned tap_h_bytes, tap_w_bytes;   // patch bytes to skip per kernel row / kernel column
+    int a_lines;                     // 1 (stem): the patch is whole input lines, not swizzled; MMA row j of a line
+                                     // starts 16 bytes (two pixels of four layers) after row j-1, so rows overlap
     int h_mul;                       // input rows per output row (2 for the stride-2 stem)
     unsigned sbo_bytes;              // patch bytes between consecutive groups of 8 output pixels
     unsigned patch_tile;             // shared-memory bytes reserved per reduction chunk of a patch
@@ -272,7 +274,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int k = e % ksteps, it = e / ksteps;
             const int ch = it % p.chunks, tap = it / p.chunks;
             const int kw = tap % p.taps_w, kh = tap / p.taps_w;
-            const uint32_t a_off = (uint32_t)ch * p.patch_tile + (uint32_t)(kh * p.tap_h_rows + kw * p.tap_w_rows) * row_bytes;
+            const uint32_t a_off = (uint32_t)ch * p.patch_tile + (uint32_t)kh * p.tap_h_bytes + (uint32_t)kw * p.tap_w_bytes;
             sh->mma_tab[e] = make_uint2((a_off >> 4) + 2u * k, ((smB + (uint32_t)it * p.b_tile) >> 4) + 2u * k);
         }
     }
@@ -331,9 +333,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if (!wait_bar(smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
                     const uint32_t full = smem_u32(&sh->full[s]);
                     mbar_arrive_expect_tx(full, p.a_bytes);
-                    for (int ch = 0; ch < p.chunks; ++ch)
-                        tma_load_5d(smA + (uint32_t)s * p.a_tile + (uint32_t)ch * p.patch_tile, &tmA, full, ch * p.BKc,
-                                    w0 - p.pad, h0 * p.h_mul - p.pad, i0, 0);
+                    if (p.a_lines)     // stem: 22 pixels of (2*BH+5) input lines, starting at pixel 2*w0 of line 2*h0
+                        tma_load_5d(smA + (uint32_t)s * p.a_tile, &tmA, full, 8 * w0, 2 * h0, i0, 0, 0);
+                    else
+                        for (int ch = 0; ch < p.chunks; ++ch)
+                            tma_load_5d(smA + (uint32_t)s * p.a_tile + (uint32_t)ch * p.patch_tile, &tmA, full, ch * p.BKc,
+                                        w0 - p.pad, h0 * p.h_mul - p.pad, i0, 0);
                     ++issued;
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
                     continue;
@@ -378,7 +383,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // single diverged thread reading a shared-memory table needs about 100).
         const uint32_t idesc = make_idesc_bf16(TILE_M, (uint32_t)p.BN);
         const int ksteps = p.BKc / 16;
-        const uint32_t hiA = (uint32_t)(make_kmajor_desc(0, row_bytes, p.patch ? p.sbo_bytes : 8u * row_bytes) >> 32);
+        const uint32_t hiA = p.a_lines ? (uint32_t)(make_kmajor_desc_plain(0, 16u, p.sbo_bytes) >> 32)
+                                       : (uint32_t)(make_kmajor_desc(0, row_bytes, p.patch ? p.sbo_bytes : 8u * row_bytes) >> 32);
         const uint32_t hiB = (uint32_t)(make_kmajor_desc(0, row_bytes, 8u * row_bytes) >> 32);
         const uint32_t a_tile16 = p.a_tile >> 4, b_tile16 = p.b_tile >> 4;
         const uint32_t smA16 = smA >> 4, smB16 = smB >> 4;
@@ -742,7 +748,8 @@ EncodeTiledFn encode_fn()
 CUtensorMapSwizzle swizzle_for_bytes(unsigned row_bytes)
 {
     return row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
-         : row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
+         : row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+         : row_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE;
 }
 
 bool encode(CUtensorMap* m, int rank, const void* ptr, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
@@ -908,25 +915,33 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     if (!flat && p.n_tiles == 1) {
         const int th = (OH + 15) / 16;
         const int bh = p.pool ? 16 : (OH + th - 1) / th;     // pooling: 16 rows give 7 pooled rows, strips 14 rows apart
-        int max_rows;
+        unsigned patch_bytes;              // bytes one patch box delivers per reduction chunk
         if (stem) {
+            // Input lines 2*h0 .. 2*h0 + 2*BH+4, 22 pixels (176 bytes) of each, stored as they are.  Output pixel
+            // (g, j) of the tile and kernel row kh read the 64 bytes at line 2g + kh, byte 16j: in the MMA's
+            // unswizzled K-major layout that is a row pitch of 16 bytes inside a group of eight rows (the
+            // 16-byte columns of the core matrices are then 16 bytes apart as well) and two lines between groups.
+            const unsigned line_bytes = (2u * 7u + 8u) * 8u;
             patch_w = 8; patch_h = 2 * bh + 5;
-            p.tap_h_rows = 8; p.tap_w_rows = 0; p.sbo_bytes = 16u * row_bytes; p.h_mul = 2;
-            max_rows = 15 * 16 + 8 + 6 * 8;
+            p.a_lines = 1;
+            p.tap_h_bytes = line_bytes; p.tap_w_bytes = 0; p.sbo_bytes = 2u * line_bytes; p.h_mul = 2;
+            patch_bytes = (unsigned)patch_h * line_bytes;
+            p.patch_tile = ((2u * 15u + 7u) * line_bytes + 1023u) / 1024u * 1024u;     // the MMA always reads 16 groups
         } else {
             patch_w = 8 + d.K - 1; patch_h = bh + d.K - 1;
-            p.tap_h_rows = patch_w; p.tap_w_rows = 1; p.sbo_bytes = (unsigned)patch_w * row_bytes;
-            max_rows = 15 * patch_w + 8 + (d.K - 1) * patch_w + (d.K - 1);
+            p.tap_h_bytes = (unsigned)patch_w * row_bytes; p.tap_w_bytes = row_bytes; p.sbo_bytes = (unsigned)patch_w * row_bytes;
+            int max_rows = 15 * patch_w + 8 + (d.K - 1) * patch_w + (d.K - 1);
+            if (max_rows < patch_w * patch_h) max_rows = patch_w * patch_h;
+            patch_bytes = (unsigned)(patch_w * patch_h) * row_bytes;
+            p.patch_tile = ((unsigned)max_rows * row_bytes + 1023u) / 1024u * 1024u;
         }
-        if (max_rows < patch_w * patch_h) max_rows = patch_w * patch_h;
-        p.patch_tile = ((unsigned)max_rows * row_bytes + 1023u) / 1024u * 1024u;
         if (patch_h <= 256 && p.sbo_bytes < (1u << 18) && p.taps * p.chunks * (p.BKc / 16) <= MAX_TAB &&
             choose_layout(p, (size_t)p.chunks * p.patch_tile, true, 2, p.taps * p.chunks * (p.BKc / 16) > PARAM_TAB,
                           &plan->smem)) {
             patch_ok = true;
             p.patch = 1;
             p.BW = 8; p.BH = bh; p.BI = 1;
-            p.a_bytes = (unsigned)p.chunks * (unsigned)(patch_w * patch_h) * row_bytes;
+            p.a_bytes = (unsigned)p.chunks * patch_bytes;
         }
     }
     if (!patch_ok) {
@@ -955,8 +970,7 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
                 for (int ch = 0; ch < p.chunks; ++ch)
                     for (int k = 0; k < ksteps; ++k, ++e) {
                         const unsigned it = (unsigned)((kh * p.taps_w + kw) * p.chunks + ch);
-                        const unsigned a_off = (unsigned)ch * p.patch_tile +
-                                               (unsigned)(kh * p.tap_h_rows + kw * p.tap_w_rows) * row_bytes;
+                        const unsigned a_off = (unsigned)ch * p.patch_tile + (unsigned)kh * p.tap_h_bytes + (unsigned)kw * p.tap_w_bytes;
                         p.ptab[e].x = (a_off >> 4) + 2u * k;
                         p.ptab[e].y = ((it * p.b_tile) >> 4) + 2u * k;
                     }
@@ -997,13 +1011,14 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
 
     // ---- tensor maps
     if (stem) {
-        // [32 window elements][OW windows, 16 B apart][input rows][image]: window ow of row y starts at
-        // pixel 2*ow, so consecutive windows overlap; the patch box is 8 windows x (2*BH+5) rows
+        // [4 layers x Wp pixels of a line][input lines][image]; the patch box is 22 pixels x (2*BH+5) lines,
+        // unswizzled, so a line lands in shared memory as it is in global memory
         const cuuint64_t row_pitch = (cuuint64_t)Wp * 8;
-        cuuint64_t dims[5] = {32, (cuuint64_t)d.OW, (cuuint64_t)Hp, (cuuint64_t)d.N, 1};
-        cuuint64_t str[4] = {16, row_pitch, (cuuint64_t)Hp * row_pitch, (cuuint64_t)Hp * row_pitch * d.N};
-        cuuint32_t box[5] = {32, (cuuint32_t)patch_w, (cuuint32_t)patch_h, 1, 1};
-        if (!encode(&plan->a, 5, a_ptr, dims, str, box, row_bytes)) return SQN_ERR_CUDA;
+        cuuint64_t dims[5] = {(cuuint64_t)Wp * 4, (cuuint64_t)Hp, (cuuint64_t)d.N, 1, 1};
+        cuuint64_t str[4] = {row_pitch, (cuuint64_t)Hp * row_pitch, (cuuint64_t)Hp * row_pitch * d.N,
+                             (cuuint64_t)Hp * row_pitch * d.N};
+        cuuint32_t box[5] = {(2 * 7 + 8) * 4, (cuuint32_t)patch_h, 1, 1, 1};
+        if (!encode(&plan->a, 5, a_ptr, dims, str, box, 0)) return SQN_ERR_CUDA;
     } else if (flat) {
         cuuint64_t dims[5] = {(cuuint64_t)d.Cin, (cuuint64_t)OW, 1, 1, 1};
         const cuuint64_t s1 = (cuuint64_t)d.Cin * 2;

@@ -163,6 +163,19 @@ __device__ __forceinline__ uint64_t make_kmajor_desc(uint32_t smem_addr, uint32_
     return d;
 }
 
+// The same for an unswizzled K-major operand: a core matrix is 8 rows x 16 bytes with the rows 16 bytes
+// apart; `lbo_bytes` from one 16-byte column of core matrices to the next along K (bits 16..29),
+// `sbo_bytes` from one group of 8 rows to the next (bits 32..45); swizzle field 0.
+__device__ __forceinline__ uint64_t make_kmajor_desc_plain(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3ffffu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
+    d |= (uint64_t)1 << 46;
+    return d;
+}
+
 // Instruction descriptor for kind::f16: bf16 x bf16 -> fp32, both operands K-major, M x N tile.
 __host__ __device__ constexpr uint32_t make_idesc_bf16(uint32_t M, uint32_t N)
 {
