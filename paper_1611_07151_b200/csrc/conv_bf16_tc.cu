@@ -687,29 +687,60 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
 // ---------------------------------------------------------------------------- stem repack
 // Input [N][H][W][3] bf16 -> [N][Hp][Wp][4] bf16, zero in the fourth layer and in the padding
-// column/row, so that every pixel is 8 bytes and two pixels are one 16-byte TMA stride.
-// Each thread converts four consecutive pixels of a row (Wp is a multiple of 4 or handled by the tail test).
-__global__ void stem_pack_input(const __nv_bfloat16* __restrict__ in, uint2* __restrict__ out, int N, int H, int W,
-                                int Hp, int Wp)
+// column/row, so that every pixel is 8 bytes and two pixels are one 16-byte unit.
+// A block repacks four rows: each row (6*W bytes, only 2-byte aligned) is brought into shared memory with
+// 16-byte loads from the enclosing aligned range, then every thread writes four pixels (32 bytes).
+// Loads never leave [in, in + in_elems): the units that straddle an end of the tensor are read by halfwords.
+__global__ void __launch_bounds__(256) stem_pack_input(const __nv_bfloat16* __restrict__ in, uint4* __restrict__ out, int N,
+                                                       int H, int W, int Hp, int Wp, long long in_elems, int pitch)
 {
     chain_release();
     chain_wait();
-    const int Wq = (Wp + 3) / 4;
-    const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
-    const long long total = (long long)N * Hp * Wq;
-    if (idx >= total) return;
-    const int x0 = (int)(idx % Wq) * 4;
-    const int y = (int)((idx / Wq) % Hp);
-    const long long n = idx / ((long long)Wq * Hp);
-    const unsigned short* src = reinterpret_cast<const unsigned short*>(in) + ((n * H + y) * W + x0) * 3;
-    unsigned short e[12];
+    extern __shared__ __align__(16) unsigned short rows_s[];
+    const int r = threadIdx.x >> 6, i = threadIdx.x & 63;
+    const long long rowid = blockIdx.x * 4ll + r;                 // over N * Hp
+    const bool live = rowid < (long long)N * Hp;
+    const int y = live ? (int)(rowid % Hp) : 0;
+    const long long n = live ? rowid / Hp : 0;
+    unsigned short* rs = rows_s + (size_t)r * pitch;
+    int shift = 0;                                                // halfwords between the aligned start and the row
+    if (live && y < H) {
+        const unsigned long long lo = reinterpret_cast<unsigned long long>(in), hi = lo + 2ull * (unsigned long long)in_elems;
+        const unsigned long long b0 = lo + 6ull * (unsigned long long)((n * H + y) * W);
+        const unsigned long long a0 = b0 & ~15ull;
+        shift = (int)((b0 - a0) >> 1);
+        const int units = (2 * shift + 6 * W + 15) / 16;
+        for (int u = i; u < units; u += 64) {
+            const unsigned long long a = a0 + 16ull * u;
+            uint4 v;
+            if (a >= lo && a + 16 <= hi) {
+                v = __ldg(reinterpret_cast<const uint4*>(a));
+            } else {
+                unsigned short h[8];
 #pragma unroll
-    for (int j = 0; j < 12; ++j) e[j] = (y < H && x0 + j / 3 < W) ? __ldg(src + j) : (unsigned short)0;
-    uint2* dst = out + (n * Hp + y) * Wp + x0;
+                for (int k = 0; k < 8; ++k) {
+                    const unsigned long long ah = a + 2ull * k;
+                    h[k] = (ah >= lo && ah + 2 <= hi) ? __ldg(reinterpret_cast<const unsigned short*>(ah)) : (unsigned short)0;
+                }
+                v = make_uint4((unsigned)h[0] | ((unsigned)h[1] << 16), (unsigned)h[2] | ((unsigned)h[3] << 16),
+                               (unsigned)h[4] | ((unsigned)h[5] << 16), (unsigned)h[6] | ((unsigned)h[7] << 16));
+            }
+            reinterpret_cast<uint4*>(rs)[u] = v;
+        }
+    }
+    __syncthreads();
+    if (!live) return;
+    for (int x0 = 4 * i; x0 < Wp; x0 += 256) {
+        unsigned short e[12];
 #pragma unroll
-    for (int q = 0; q < 4; ++q)
-        if (x0 + q < Wp)
-            dst[q] = make_uint2((unsigned)e[3 * q] | ((unsigned)e[3 * q + 1] << 16), (unsigned)e[3 * q + 2]);
+        for (int j = 0; j < 12; ++j) e[j] = (y < H && x0 + j / 3 < W) ? rs[shift + 3 * x0 + j] : (unsigned short)0;
+        uint4* dst = out + ((n * Hp + y) * Wp + x0) / 2;           // two pixels per 16 bytes (Wp is even)
+        dst[0] = make_uint4((unsigned)e[0] | ((unsigned)e[1] << 16), (unsigned)e[2],
+                            (unsigned)e[3] | ((unsigned)e[4] << 16), (unsigned)e[5]);
+        if (x0 + 2 < Wp)
+            dst[1] = make_uint4((unsigned)e[6] | ((unsigned)e[7] << 16), (unsigned)e[8],
+                                (unsigned)e[9] | ((unsigned)e[10] << 16), (unsigned)e[11]);
+    }
 }
 
 // Kernels [Cout][7][7][3] bf16 -> [Cout][7][8][4] bf16 (zero for the eighth column and fourth layer).
@@ -1203,11 +1234,13 @@ int launch_stem_pack_bf16(const ConvDesc& d, void* workspace, size_t workspace_b
     if (rc != SQN_OK) return rc;
     const int Hp = (d.H + 1) / 2 * 2, Wp = (d.W + 2) / 2 * 2;
     unsigned char* ws = static_cast<unsigned char*>(workspace);
-    uint2* pin = reinterpret_cast<uint2*>(ws);
+    uint4* pin = reinterpret_cast<uint4*>(ws);
     unsigned short* pw = reinterpret_cast<unsigned short*>(ws + align_up((size_t)d.N * Hp * Wp * 8, 1024));
-    const long long total = (long long)d.N * Hp * ((Wp + 3) / 4);
-    cudaError_t e = launch_chained(stem_pack_input, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, stream,
-                                   static_cast<const __nv_bfloat16*>(d.in), pin, d.N, d.H, d.W, Hp, Wp);
+    const long long rows = (long long)d.N * Hp;
+    const int pitch = (3 * d.W + 23) / 8 * 8;                  // halfwords per staged row: the row, its lead-in, a full last unit
+    cudaError_t e = launch_chained(stem_pack_input, dim3((unsigned)((rows + 3) / 4)), dim3(256), (size_t)4 * pitch * 2, stream,
+                                   static_cast<const __nv_bfloat16*>(d.in), pin, d.N, d.H, d.W, Hp, Wp,
+                                   (long long)d.N * d.H * d.W * 3, pitch);
     if (e == cudaSuccess)
         e = launch_chained(stem_pack_weights, dim3((unsigned)((d.Cout * 224 + 255) / 256)), dim3(256), 0, stream,
                            static_cast<const unsigned short*>(d.w), pw, d.Cout);

@@ -161,6 +161,53 @@ __global__ void __launch_bounds__(256) global_avgpool_kernel(const void* __restr
     }
 }
 
+// Global average of a bf16 map with C % 8 == 0: block (x = group of 128 layers, y = image), 256 threads =
+// 16 groups of 8 layers (one 16-byte load per pixel) x 16 pixel slices, four loads in flight per thread.
+__global__ void __launch_bounds__(256) global_avgpool_bf16_v8(const uint4* __restrict__ in, float* __restrict__ logits,
+                                                              int C, int HW)
+{
+    chain_release();
+    chain_wait();
+    __shared__ float part[16][129];
+    const int n = blockIdx.y, tid = threadIdx.x;
+    const int g = tid & 15, slice = tid >> 4;
+    const int c0 = blockIdx.x * 128 + 8 * g;
+    float acc[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) acc[k] = 0.f;
+    if (c0 < C) {
+        const int C8 = C >> 3;
+        const uint4* src = in + (size_t)n * HW * C8 + (c0 >> 3);
+        auto add = [&](const uint4& v) {
+            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                acc[2 * k] += __low2float(h[k]);
+                acc[2 * k + 1] += __high2float(h[k]);
+            }
+        };
+        int p = slice;
+        for (; p + 48 < HW; p += 64) {
+            const uint4 v0 = __ldg(src + (size_t)p * C8), v1 = __ldg(src + (size_t)(p + 16) * C8);
+            const uint4 v2 = __ldg(src + (size_t)(p + 32) * C8), v3 = __ldg(src + (size_t)(p + 48) * C8);
+            add(v0); add(v1); add(v2); add(v3);
+        }
+        for (; p < HW; p += 16) add(__ldg(src + (size_t)p * C8));
+    }
+#pragma unroll
+    for (int k = 0; k < 8; ++k) part[slice][8 * g + k] = acc[k];
+    __syncthreads();
+    if (tid < 128) {
+        const int c = blockIdx.x * 128 + tid;
+        if (c < C) {
+            float s = 0.f;
+#pragma unroll
+            for (int q = 0; q < 16; ++q) s += part[q][tid];
+            logits[(size_t)n * C + c] = s / (float)HW;
+        }
+    }
+}
+
 // Softmax over the C logits of one image per block.
 __global__ void __launch_bounds__(256) softmax_kernel(const float* __restrict__ logits, float* __restrict__ probs, int C)
 {
@@ -229,6 +276,8 @@ int launch_avgpool_softmax(const void* in, float* logits, float* probs, int C, i
 {
     const dim3 grid((unsigned)((C + 127) / 128), (unsigned)N);
     if (dtype == SQN_F32) launch_chained(global_avgpool_kernel<false>, grid, dim3(256), 0, stream, in, logits, C, H * W);
+    else if (C % 8 == 0 && aligned16(in))
+        launch_chained(global_avgpool_bf16_v8, grid, dim3(256), 0, stream, static_cast<const uint4*>(in), logits, C, H * W);
     else launch_chained(global_avgpool_kernel<true>, grid, dim3(256), 0, stream, in, logits, C, H * W);
     note_launch();
     if (cudaGetLastError() != cudaSuccess) return SQN_ERR_CUDA;
