@@ -40,7 +40,7 @@ namespace {
 using namespace ptx;
 
 constexpr int TILE_M = 128;            // MMA M: TMEM lanes
-// Threads per CTA: producer warp, MMA warp, 4*SPLIT epilogue warps, store warp.  SPLIT = 2 or 4: one CTA per SM
+// Threads per CTA: producer warp, MMA warp, 4*SPLIT epilogue warps, store warp.  SPLIT = 2: one CTA per SM
 // (large tiles, kernels resident in up to 227 KB); SPLIT = 1: two lighter CTAs per SM, i.e. two MMA issuers,
 // two producers and two store threads per SM, for the layers whose tiles are small.
 __host__ __device__ constexpr int threads_for(int split) { return 96 + 128 * split; }
@@ -211,7 +211,9 @@ __device__ __forceinline__ uint4 bmax8(uint4 a, uint4 b)
     return r;
 }
 
-template <int SPLIT, bool POOL>
+// HC: output layers per epilogue piece (8, 16 or 32; a store chunk CW is two pieces), fixed at compile time so
+// that the conversion loop is straight-line code.
+template <int SPLIT, bool POOL, int HC>
 __global__ void __launch_bounds__(threads_of(SPLIT, POOL), SPLIT == 1 ? 2 : 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmO, const TcParams p)
@@ -484,7 +486,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const uint32_t slot_bytes = (uint32_t)TILE_M * cw_bytes;
         const uint32_t sw = cw_bytes == 128 ? (uint32_t)(row & 7)
                           : cw_bytes == 64 ? (uint32_t)((row >> 1) & 3) : (uint32_t)((row >> 2) & 1);
-        const int hc = p.CW / PIECES;                  // layers per piece: 8, 16 or 32
+        constexpr int hc = HC;                         // layers per piece: 8, 16 or 32 (CW / PIECES)
         bool ok = true;
         int as = 0, sb = 0;
         uint32_t aph = 0, sph = 0;
@@ -816,7 +818,7 @@ struct Plan {
     TcParams p;
     int grid;
     int halves;      // 1 = two light CTAs per SM, 2 = one CTA per SM
-    int split;       // epilogue warps / 4 of the kernel variant: 1, 2 or 4
+    int split;       // epilogue warps / 4 of the kernel variant: 1 or 2
     size_t smem;
 };
 
@@ -987,9 +989,6 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
             !choose_layout(p, a_tile, false, 2, false, &plan->smem))
             return SQN_ERR_UNSUPPORTED;
     }
-    // (sixteen epilogue warps, SPLIT = 4, were measured slower than eight on every SqueezeNet shape: the
-    //  epilogue is limited by conversion and shared-memory throughput, not by latency; the variant is kept
-    //  for shapes where that may differ and is not selected automatically)
     p.use_ptab = 0;
     if (p.patch && p.taps * p.chunks * (p.BKc / 16) <= PARAM_TAB) {
         // operand offsets of every MMA of a tile, in issue order (tap-major, then chunk, then k-step)
@@ -1094,36 +1093,33 @@ int build_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_pt
     // the single CTA win.
     if (build_plan_cfg(d, stem, a_ptr, w_ptr, Hp, Wp, 1, plan) == SQN_OK) {
         const TcParams& p = plan->p;
-        if ((p.patch && p.BN <= 64) || (!p.patch && p.stages >= 3)) return SQN_OK;
+        if ((p.patch && p.BN <= 64) || (!p.patch && p.taps == 1 && p.stages >= 3)) return SQN_OK;
     }
     return build_plan_cfg(d, stem, a_ptr, w_ptr, Hp, Wp, 2, plan);
 }
 
+template <int SPLIT, bool POOL, int HC>
+cudaError_t launch_variant(const Plan& plan, cudaStream_t stream)
+{
+    static const cudaError_t attr_rc =
+        cudaFuncSetAttribute(conv_tc_kernel<SPLIT, POOL, HC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(SPLIT == 1 ? SMEM_LIMIT_2CTA : SMEM_LIMIT));
+    if (attr_rc != cudaSuccess) return attr_rc;
+    return launch_chained(conv_tc_kernel<SPLIT, POOL, HC>, dim3((unsigned)plan.grid), dim3(threads_of(SPLIT, POOL)), plan.smem,
+                          stream, plan.a, plan.b, plan.o, plan.p);
+}
+
 int launch_plan(const Plan& plan, cudaStream_t stream)
 {
-    static std::once_flag once;
-    static cudaError_t attr_rc = cudaSuccess;
-    std::call_once(once, [] {
-        attr_rc = cudaFuncSetAttribute(conv_tc_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
-        if (attr_rc == cudaSuccess)
-            attr_rc = cudaFuncSetAttribute(conv_tc_kernel<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
-        if (attr_rc == cudaSuccess)
-            attr_rc = cudaFuncSetAttribute(conv_tc_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
-        if (attr_rc == cudaSuccess)
-            attr_rc = cudaFuncSetAttribute(conv_tc_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           (int)SMEM_LIMIT_2CTA);
-    });
-    if (attr_rc != cudaSuccess) return SQN_ERR_CUDA;
-    const dim3 grid((unsigned)plan.grid);
     cudaError_t rc;
-    if (plan.p.pool)
-        rc = launch_chained(conv_tc_kernel<2, true>, grid, dim3(threads_of(2, true)), plan.smem, stream, plan.a, plan.b, plan.o, plan.p);
+    const int hc = plan.p.CW / 2;
+    if (plan.p.pool) rc = launch_variant<2, true, 32>(plan, stream);
     else if (plan.split == 1)
-        rc = launch_chained(conv_tc_kernel<1, false>, grid, dim3(threads_for(1)), plan.smem, stream, plan.a, plan.b, plan.o, plan.p);
-    else if (plan.split == 4)
-        rc = launch_chained(conv_tc_kernel<4, false>, grid, dim3(threads_for(4)), plan.smem, stream, plan.a, plan.b, plan.o, plan.p);
+        rc = hc == 32 ? launch_variant<1, false, 32>(plan, stream)
+           : hc == 16 ? launch_variant<1, false, 16>(plan, stream) : launch_variant<1, false, 8>(plan, stream);
     else
-        rc = launch_chained(conv_tc_kernel<2, false>, grid, dim3(threads_for(2)), plan.smem, stream, plan.a, plan.b, plan.o, plan.p);
+        rc = hc == 32 ? launch_variant<2, false, 32>(plan, stream)
+           : hc == 16 ? launch_variant<2, false, 16>(plan, stream) : launch_variant<2, false, 8>(plan, stream);
     if (rc != cudaSuccess) return SQN_ERR_CUDA;
     note_launch();
     return cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
