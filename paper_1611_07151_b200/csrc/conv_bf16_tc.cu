@@ -63,6 +63,7 @@ struct TcParams {
     int BW, BH, BI;                  // box extents, BW*BH*BI <= 128
     int n_tiles, BN;                 // output-layer tiles and their width (multiple of 16, <= 256)
     int total_tiles;
+    int reverse;                     // 1: tiles are taken from the last to the first (see build_plan_cfg)
     int g_nt, g_tw, g_th, g_ti;      // gridDim.x written in the mixed radix (n_tiles, tiles_w, tiles_h, tiles_i)
     int Cout;
     int taps, taps_w, pad;           // kernel taps, taps per kernel row, zero padding
@@ -165,6 +166,7 @@ __device__ __forceinline__ void tile_first(const TcParams& p, int t, TileCoord& 
         c.ti = t / p.tiles_h;
         return;
     }
+    if (p.reverse) t = p.total_tiles - 1 - t;
     c.nt = t % p.n_tiles;
     const int mt = t / p.n_tiles;
     c.tw = mt % p.tiles_w;
@@ -181,6 +183,16 @@ __device__ __forceinline__ void tile_next(const TcParams& p, TileCoord& c)
         c.th += p.g_th;
         if (c.th >= p.tiles_h) { c.th -= p.tiles_h; carry = 1; }
         c.ti += p.g_ti + carry;
+        return;
+    }
+    if (p.reverse) {              // the same step downwards, with borrows
+        c.nt -= p.g_nt;
+        if (c.nt < 0) { c.nt += p.n_tiles; carry = 1; }
+        c.tw -= p.g_tw + carry; carry = 0;
+        if (c.tw < 0) { c.tw += p.tiles_w; carry = 1; }
+        c.th -= p.g_th + carry; carry = 0;
+        if (c.th < 0) { c.th += p.tiles_h; carry = 1; }
+        c.ti -= p.g_ti + carry;
         return;
     }
     c.nt += p.g_nt;
@@ -1024,6 +1036,9 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     const long long total = (long long)p.tiles_w * p.tiles_h * p.tiles_i * p.n_tiles;
     if (total > 0x7fffffffLL) return SQN_ERR_UNSUPPORTED;
     p.total_tiles = (int)total;
+    // A 1x1 layer over a map larger than a third of the L2 walks its tiles backwards: the layer before it wrote the
+    // map front to back, so its last part is still in the L2 and is read from there before it is evicted.
+    p.reverse = (!p.patch && p.taps == 1 && !p.pool && (size_t)d.N * d.H * d.W * d.Cin * 2 > ((size_t)40 << 20)) ? 1 : 0;
     const long long ctas = (long long)num_sms() * (halves == 1 ? 2 : 1);
     const long long units = p.pool ? (long long)p.tiles_h * p.tiles_i : total;
     plan->grid = (int)(units < ctas ? units : ctas);
