@@ -712,7 +712,8 @@ __global__ void __launch_bounds__(256) stem_pack_input(const __nv_bfloat16* __re
     chain_wait();
     extern __shared__ __align__(16) unsigned short rows_s[];
     const int r = threadIdx.x >> 6, i = threadIdx.x & 63;
-    const long long rowid = blockIdx.x * 4ll + r;                 // over N * Hp
+    const long long rowid = ((long long)gridDim.x - 1 - blockIdx.x) * 4ll + r;   // over N * Hp, last rows first: the stem kernel that
+                                                                                 // follows starts with the first rows, then still in the L2
     const bool live = rowid < (long long)N * Hp;
     const int y = live ? (int)(rowid % Hp) : 0;
     const long long n = live ? rowid / Hp : 0;

@@ -70,8 +70,9 @@ __global__ void maxpool_bf16_v8(const uint4* __restrict__ in, uint4* __restrict_
 {
     chain_release();
     chain_wait();
-    const long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
-    if (idx >= total) return;
+    // last output first: the end of the input map is what the layer before left in the L2
+    const long long idx = total - 1 - (blockIdx.x * (long long)blockDim.x + threadIdx.x);
+    if (idx < 0) return;
     const int c8 = (int)(idx % C8);
     long long r = idx / C8;
     const int ow = (int)(r % OW); r /= OW;
@@ -169,7 +170,7 @@ __global__ void __launch_bounds__(256) global_avgpool_bf16_v8(const uint4* __res
     chain_release();
     chain_wait();
     __shared__ float part[16][129];
-    const int n = blockIdx.y, tid = threadIdx.x;
+    const int n = gridDim.y - 1 - blockIdx.y, tid = threadIdx.x;      // last image first (still in the L2)
     const int g = tid & 15, slice = tid >> 4;
     const int c0 = blockIdx.x * 128 + 8 * g;
     float acc[8];
