@@ -26,7 +26,7 @@ from paper_1611_07151_b200 import dist as D
 from paper_1611_07151_b200 import synth
 
 IMG = 227
-NCU_TRAFFIC_BYTES = {("conv1+pool1", "bf16", 256): 204.7e6}
+NCU_TRAFFIC_BYTES = {("conv1+pool1", "bf16", 256): 204.5e6}
 METRIC = "squeezenet_v1.0_forward_images_per_s"
 UNIT = "images/s"
 
