@@ -79,6 +79,23 @@ def test_stem_7x7_stride2(hw, batch, cout):
     assert G.rel_err(got, exp) <= TOL
 
 
+def test_large_1x1_map_tiles_taken_last_to_first():
+    """A 1x1 layer whose input map exceeds 40 MB walks its tiles backwards (to meet what the layer before it left
+    in the L2); same values as the oracle, ragged last tile included, and the bias of every layer is applied."""
+    N, C, M, H, W = 9, 128, 16, 151, 157          # 54.6 MB of bf16 input, 213363 pixels = 1666 tiles + 115 pixels
+    rng = np.random.default_rng(77)
+    x = synth.draw_input(rng, (N, C, H, W))
+    w, b = synth.draw_conv_params(rng, C, M, 1)
+    b = b + np.float32(0.5) * rng.standard_normal(M).astype(np.float32)
+    exp = ref.conv2d(x, w, b, S=1, pad=0, relu=True)
+    got = G.gpu_conv(x, w, b, 1, 0, True, BF16)
+    assert got.shape == exp.shape
+    assert G.rel_err(got, exp) <= TOL
+    # per image, so that a tile written to the wrong place cannot hide behind a large global maximum
+    for n in range(N):
+        assert G.rel_err(got[n], exp[n]) <= TOL
+
+
 # (N, Cin, Cout, H, W, K, S, pad): convolution with the following 3x3/2 max-pool fused into its epilogue
 POOLED = [
     (2, 3, 96, 227, 227, 7, 2, 0),     # conv1 + pool1 of the network
@@ -196,3 +213,24 @@ def test_full_forward_bf16_small_batch_keeps_every_map():
     assert max(G.rel_err(got, trace[name]) for name, got in layers.items()) <= 5e-2
     assert G.rel_err(logits, z) <= TOL
     np.testing.assert_allclose(probs.astype(np.float64).sum(1), 1.0, rtol=0, atol=1e-5)
+
+
+def test_plain_launches_give_the_same_values():
+    """SQN_CHAINED_LAUNCH=0 (read once per process) launches every kernel without programmatic stream
+    serialisation; a child process runs the batch-2 network that way and must reproduce this process's logits."""
+    import os, subprocess, sys, tempfile
+    x, params = synth.squeezenet_case(11, 2)
+    here = run_net(x, params, BF16, 2)[0]
+    code = (
+        "import sys, numpy as np; sys.path.insert(0, %r); sys.path.insert(0, %r)\n"
+        "from paper_1611_07151_b200 import binding as B, synth\n"
+        "from test_gpu_f32 import run_net\n"
+        "x, params = synth.squeezenet_case(11, 2)\n"
+        "np.save(sys.argv[1], run_net(x, params, B.SQN_BF16, 2)[0])\n"
+    ) % (os.path.dirname(os.path.dirname(os.path.abspath(__file__))), os.path.dirname(os.path.abspath(__file__)))
+    with tempfile.TemporaryDirectory() as tmp:
+        out = os.path.join(tmp, "logits.npy")
+        env = dict(os.environ, SQN_CHAINED_LAUNCH="0")
+        subprocess.run([sys.executable, "-c", code, out], check=True, env=env, timeout=300)
+        there = np.load(out)
+    np.testing.assert_array_equal(here, there)
