@@ -202,12 +202,17 @@ int squeezenet_destroy(sqn_net* net);
 
 /*
  * The same forward with HOST input and output buffers (the call a user with data in host
- * memory makes).  Enqueues on `stream`: copy of in_host [batch][227][227][3] (net dtype) to the
- * device, the forward, copies of logits (and probs, unless NULL) [batch][1000] fp32 back to
- * the host.  The copies are asynchronous when the host buffers are pinned.  workspace is
- * DEVICE memory of squeezenet_host_workspace_bytes(net, batch) bytes (the forward's scratch
- * plus staging for the input and the two outputs).  The host buffers must stay valid until
- * the stream has passed the call.
+ * memory makes): copy of in_host [batch][227][227][3] (net dtype) to the device, the forward,
+ * copies of logits (and probs, unless NULL) [batch][1000] fp32 back to the host.  The copies
+ * are asynchronous when the host buffers are pinned.  workspace is DEVICE memory of
+ * squeezenet_host_workspace_bytes(net, batch) bytes (the forward's scratch, two staging
+ * buffers for the input and staging for the two outputs).
+ * Ordering: the forward and the copies back are enqueued on `stream`.  The input copy runs on
+ * a stream the net owns (made on the first call on a device) and alternates between the two
+ * staging buffers, so the copy of one call overlaps the forward of the call before it; it is
+ * NOT ordered after work queued earlier on `stream`: in_host must hold the images when the
+ * call is made.  All host buffers must stay valid, and in_host unchanged, until `stream` has
+ * passed the call.  Calls on one net must come from one thread at a time.
  */
 int squeezenet_host_workspace_bytes(const sqn_net* net, int batch, size_t* bytes);
 int squeezenet_forward_host(sqn_net* net, const void* in_host, void* logits_host, void* probs_host,

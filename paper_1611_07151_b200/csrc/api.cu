@@ -259,6 +259,13 @@ struct sqn_net {
     long long prof_forwards = 0;
     std::vector<std::string> prof_names;
     std::vector<std::vector<cudaEvent_t>> prof_events;
+    // squeezenet_forward_host: the input copy of call k runs on a stream of its own into one of two staging
+    // buffers, so that it overlaps the forward of call k-1
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t in_ready[2] = {nullptr, nullptr};   // copy into staging buffer b has finished
+    cudaEvent_t in_free[2] = {nullptr, nullptr};    // the forward that read staging buffer b has finished
+    int copy_device = -1;
+    unsigned long long host_calls = 0;
 };
 
 namespace {
@@ -304,7 +311,21 @@ int find_slot(const sqn_net* net, const char* name)
 
 }  // namespace
 
-namespace { void free_profile(sqn_net* net); }
+namespace {
+void free_profile(sqn_net* net);
+void free_copy_pipeline(sqn_net* net)
+{
+    for (int b = 0; b < 2; ++b) {
+        if (net->in_ready[b]) cudaEventDestroy(net->in_ready[b]);
+        if (net->in_free[b]) cudaEventDestroy(net->in_free[b]);
+        net->in_ready[b] = net->in_free[b] = nullptr;
+    }
+    if (net->copy_stream) cudaStreamDestroy(net->copy_stream);
+    net->copy_stream = nullptr;
+    net->copy_device = -1;
+    net->host_calls = 0;
+}
+}
 
 extern "C" int squeezenet_create(sqn_net** net, const void* const* weights26, const void* const* bias26, int dtype,
                                  int max_batch)
@@ -327,7 +348,10 @@ extern "C" int squeezenet_create(sqn_net** net, const void* const* weights26, co
 
 extern "C" int squeezenet_destroy(sqn_net* net)
 {
-    if (net) free_profile(net);
+    if (net) {
+        free_profile(net);
+        free_copy_pipeline(net);
+    }
     delete net;
     return SQN_OK;
 }
@@ -499,9 +523,29 @@ extern "C" int squeezenet_host_workspace_bytes(const sqn_net* net, int batch, si
     if (!net || !bytes || batch <= 0 || batch > net->max_batch) return SQN_ERR_BADARG;
     const size_t in_bytes = align_up((size_t)batch * IMG * IMG * 3 * esize(net->dtype), 1024);
     const size_t out_bytes = align_up((size_t)batch * 1000 * sizeof(float), 1024);
-    *bytes = layout(net, batch, nullptr, nullptr) + in_bytes + 2 * out_bytes;
+    *bytes = layout(net, batch, nullptr, nullptr) + 2 * in_bytes + 2 * out_bytes;
     return SQN_OK;
 }
+
+namespace {
+// Stream and events of the input-copy pipeline, made on the first host-buffer forward on a device.
+int ensure_copy_pipeline(sqn_net* net)
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return SQN_ERR_CUDA;
+    if (net->copy_stream && net->copy_device == dev) return SQN_OK;
+    free_copy_pipeline(net);
+    if (cudaStreamCreateWithFlags(&net->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return SQN_ERR_CUDA;
+    for (int b = 0; b < 2; ++b)
+        if (cudaEventCreateWithFlags(&net->in_ready[b], cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&net->in_free[b], cudaEventDisableTiming) != cudaSuccess) {
+            free_copy_pipeline(net);
+            return SQN_ERR_CUDA;
+        }
+    net->copy_device = dev;
+    return SQN_OK;
+}
+}  // namespace
 
 extern "C" int squeezenet_forward_host(sqn_net* net, const void* in_host, void* logits_host, void* probs_host,
                                        void* workspace, int batch, void* stream)
@@ -510,15 +554,25 @@ extern "C" int squeezenet_forward_host(sqn_net* net, const void* in_host, void* 
     if (!workspace) return SQN_ERR_WORKSPACE;
     if (!aligned16(workspace)) return SQN_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int rc = ensure_copy_pipeline(net);
+    if (rc != SQN_OK) return rc;
     const size_t fwd_bytes = layout(net, batch, nullptr, nullptr);
     const size_t in_bytes = (size_t)batch * IMG * IMG * 3 * esize(net->dtype);
     const size_t out_bytes = (size_t)batch * 1000 * sizeof(float);
     char* ws = static_cast<char*>(workspace);
-    char* d_in = ws + fwd_bytes;
-    char* d_logits = d_in + align_up(in_bytes, 1024);
+    const int b = (int)(net->host_calls & 1ull);
+    char* d_in = ws + fwd_bytes + (size_t)b * align_up(in_bytes, 1024);
+    char* d_logits = ws + fwd_bytes + 2 * align_up(in_bytes, 1024);
     char* d_probs = d_logits + align_up(out_bytes, 1024);
-    if (cudaMemcpyAsync(d_in, in_host, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return SQN_ERR_CUDA;
-    const int rc = squeezenet_forward(net, d_in, d_logits, probs_host ? d_probs : nullptr, workspace, batch, stream);
+    // Input copy on the copy stream: it waits only for the forward of two calls ago (the last reader of this
+    // staging buffer), not for the work queued on `stream`, and so runs beside the forward of the call before.
+    if (net->host_calls >= 2 && cudaStreamWaitEvent(net->copy_stream, net->in_free[b], 0) != cudaSuccess) return SQN_ERR_CUDA;
+    if (cudaMemcpyAsync(d_in, in_host, in_bytes, cudaMemcpyHostToDevice, net->copy_stream) != cudaSuccess) return SQN_ERR_CUDA;
+    if (cudaEventRecord(net->in_ready[b], net->copy_stream) != cudaSuccess) return SQN_ERR_CUDA;
+    if (cudaStreamWaitEvent(st, net->in_ready[b], 0) != cudaSuccess) return SQN_ERR_CUDA;
+    net->host_calls++;
+    rc = squeezenet_forward(net, d_in, d_logits, probs_host ? d_probs : nullptr, workspace, batch, stream);
+    if (cudaEventRecord(net->in_free[b], st) != cudaSuccess) return SQN_ERR_CUDA;
     if (rc != SQN_OK) return rc;
     if (cudaMemcpyAsync(logits_host, d_logits, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return SQN_ERR_CUDA;
     if (probs_host && cudaMemcpyAsync(probs_host, d_probs, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)

@@ -81,6 +81,9 @@ struct TcParams {
     int relu;
     int stages;                      // A (or A+B) ring slots
     int b_resident;                  // 1: all kernel tiles are loaded once and stay in shared memory
+    int b_early;                     // 1: kernels and bias are not written by the kernel this launch is chained to, so
+                                     // they are fetched before the wait for that kernel (0 for the stem: its kernels
+                                     // are repacked by the launch before it)
     int CW;                          // layers per TMA store (16/32/64)
     int nstg;                        // staging ring slots (2 or 4)
     int bn_pad;                      // TMEM column stride between the two accumulators
@@ -223,6 +226,32 @@ __device__ __forceinline__ uint4 bmax8(uint4 a, uint4 b)
     return r;
 }
 
+// Every kernel tile of the layer, once, into the resident region (one mbarrier counts all of them).
+__device__ __forceinline__ void load_resident_kernels(const TcParams& p, const CUtensorMap& tmB, uint32_t smB, uint32_t bar, int items)
+{
+    mbar_arrive_expect_tx(bar, (uint32_t)items * p.b_bytes);
+    int tap = 0, ch = 0;
+    for (int i = 0; i < items; ++i) {
+        tma_load_2d(smB + (uint32_t)i * p.b_tile, &tmB, bar, tap * p.k_per_tap + ch * p.BKc, 0);
+        if (++ch == p.chunks) { ch = 0; ++tap; }
+    }
+}
+
+// Bias rows of the bias MMA: one 32-byte row {hi, lo, 0, ...} per output layer, hi + lo = the fp32 bias.
+template <int NUM_THREADS>
+__device__ __forceinline__ void fill_bias_rows(const TcParams& p, unsigned char* base_ptr)
+{
+    uint4* rows = reinterpret_cast<uint4*>(base_ptr + p.off_bias);
+    for (int c = threadIdx.x; c < p.n_tiles * p.BN; c += NUM_THREADS) {
+        const float b = c < p.Cout ? __ldg(p.bias + c) : 0.f;
+        const __nv_bfloat16 hi = __float2bfloat16_rn(b);
+        const __nv_bfloat16 lo = __float2bfloat16_rn(b - __bfloat162float(hi));
+        const int u = (c >> 2) & 1;
+        rows[2 * c + u] = make_uint4((uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16), 0u, 0u, 0u);
+        rows[2 * c + (u ^ 1)] = make_uint4(0u, 0u, 0u, 0u);
+    }
+}
+
 // HC: output layers per epilogue piece (8, 16 or 32; a store chunk CW is two pieces), fixed at compile time so
 // that the conversion loop is straight-line code.
 template <int SPLIT, bool POOL, int HC>
@@ -250,8 +279,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int my_tiles = tiles_of_cta(p);
 
     // The launch is chained to the kernel before it in the stream: this block may be running while
-    // that grid drains.  Up to chain_wait() below it touches only its own shared memory, TMEM and the
-    // kernel parameters.
+    // that grid drains.  Up to chain_wait() below it touches only its own shared memory, TMEM, the
+    // kernel parameters and, when b_early is set, the layer's kernels and bias (which that grid does not
+    // write): a CTA that starts in the tail of the layer before has its kernels resident by the time
+    // the first input tile may be read.
     chain_release();
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -276,6 +307,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         prefetch_tensormap(&tmA);
         prefetch_tensormap(&tmB);
         prefetch_tensormap(&tmO);
+        if (p.b_resident && p.b_early) load_resident_kernels(p, tmB, smB, smem_u32(&sh->b_full), items);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(&sh->tmem_base), p.tmem_cols);
@@ -292,7 +324,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             sh->mma_tab[e] = make_uint2((a_off >> 4) + 2u * k, ((smB + (uint32_t)it * p.b_tile) >> 4) + 2u * k);
         }
     }
-    chain_wait();       // the earlier grid has finished: global memory may be read and written from here on
     // The bias is added by the tensor core: the last MMA of every tile multiplies a tile of ones
     // (128 rows, K = 16: ones in the first two places) by the bias rows (one per output layer:
     // {hi, lo, 0, ...} with hi + lo = bias to 16 bits below its leading bit).  Both tiles have
@@ -304,17 +335,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             ones[2 * r + u] = make_uint4(0x3f803f80u, 0u, 0u, 0u);
             ones[2 * r + (u ^ 1)] = make_uint4(0u, 0u, 0u, 0u);
         }
-        uint4* rows = reinterpret_cast<uint4*>(base_ptr + p.off_bias);
-        for (int c = threadIdx.x; c < p.n_tiles * p.BN; c += NUM_THREADS) {
-            const float b = c < p.Cout ? __ldg(p.bias + c) : 0.f;
-            const __nv_bfloat16 hi = __float2bfloat16_rn(b);
-            const __nv_bfloat16 lo = __float2bfloat16_rn(b - __bfloat162float(hi));
-            const int u = (c >> 2) & 1;
-            rows[2 * c + u] = make_uint4((uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16), 0u, 0u, 0u);
-            rows[2 * c + (u ^ 1)] = make_uint4(0u, 0u, 0u, 0u);
-        }
-        fence_proxy_async_smem();       // the MMA reads them through the async proxy
     }
+    if (p.b_early) fill_bias_rows<NUM_THREADS>(p, base_ptr);
+    chain_wait();       // the earlier grid has finished: global memory may be read and written from here on
+    if (!p.b_early) fill_bias_rows<NUM_THREADS>(p, base_ptr);
+    fence_proxy_async_smem();           // the MMA reads the ones and the bias rows through the async proxy
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -325,16 +350,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
             bool ok = true;
-            if (p.b_resident) {
-                // every kernel tile, once: they stay in shared memory for all tiles of this CTA
-                const uint32_t bf = smem_u32(&sh->b_full);
-                mbar_arrive_expect_tx(bf, (uint32_t)items * p.b_bytes);
-                int tap = 0, ch = 0;
-                for (int i = 0; i < items; ++i) {
-                    tma_load_2d(smB + (uint32_t)i * p.b_tile, &tmB, bf, tap * p.k_per_tap + ch * p.BKc, 0);
-                    if (++ch == p.chunks) { ch = 0; ++tap; }
-                }
-            }
+            // every kernel tile, once: they stay in shared memory for all tiles of this CTA
+            if (p.b_resident && !p.b_early) load_resident_kernels(p, tmB, smB, smem_u32(&sh->b_full), items);
             const uint32_t tx = p.b_resident ? p.a_bytes : p.a_bytes + p.b_bytes;
             int s = 0, issued = 0;
             uint32_t ph = 0;
@@ -924,6 +941,7 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     p.bias = d.bias;
     p.status = device_status_word();
     p.h_mul = 1;
+    p.b_early = stem ? 0 : 1;
     p.pool = d.pool ? 1 : 0;
     if (p.pool && (d.OH < 3 || d.OW < 3 || d.Cout % 32 != 0 || d.Cout > 256)) return SQN_ERR_UNSUPPORTED;
     if (stem) {

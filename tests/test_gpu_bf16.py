@@ -234,3 +234,36 @@ def test_plain_launches_give_the_same_values():
         subprocess.run([sys.executable, "-c", code, out], check=True, env=env, timeout=300)
         there = np.load(out)
     np.testing.assert_array_equal(here, there)
+
+
+def test_host_buffer_forward_matches_device_forward_over_calls_in_a_row():
+    """squeezenet_forward_host copies its input on a stream of its own into alternating staging buffers.  Five
+    calls in a row without a synchronisation between them, over three different pinned inputs, must each give
+    exactly the logits of the device-resident forward of the same images (and those match the oracle)."""
+    import torch
+    batch = 4
+    names = [n for n, *_ in synth.SQUEEZENET_CONVS]
+    x, params = synth.squeezenet_case(21, 3 * batch)
+    ws = [G.dev_w(params[n][0], BF16) for n in names]
+    bs = [G.dev_b(params[n][1]) for n in names]
+    net = B.squeezenet_create(ws, bs, BF16, batch)
+    work = torch.empty(B.squeezenet_host_workspace_bytes(net, batch), dtype=torch.uint8, device="cuda")
+    parts = [x[i * batch:(i + 1) * batch] for i in range(3)]
+    pinned = [torch.from_numpy(B.sqn_pack_nchw_to_nhwc(p, BF16).view(np.int16)).pin_memory() for p in parts]
+    want = []
+    for p in parts:
+        logits = torch.empty((batch, 1000), device="cuda")
+        B.squeezenet_forward(net, G.dev_act(p, BF16), logits, None, work, batch)
+        want.append(logits.cpu().numpy())
+    assert B.sqn_check() == B.SQN_OK
+    order = [0, 1, 2, 1, 0]
+    outs = [torch.zeros((2, batch, 1000), dtype=torch.float32).pin_memory() for _ in order]
+    for o, k in zip(outs, order):
+        B.squeezenet_forward_host(net, pinned[k], o[0], o[1], work, batch)
+    assert B.sqn_check() == B.SQN_OK
+    for o, k in zip(outs, order):
+        np.testing.assert_array_equal(o[0].numpy(), want[k])
+        np.testing.assert_allclose(o[1].numpy().astype(np.float64).sum(1), 1.0, rtol=0, atol=1e-5)
+    z, _ = ref.squeezenet(parts[2], params)
+    assert G.rel_err(want[2], z) <= TOL
+    B.squeezenet_destroy(net)
