@@ -99,6 +99,9 @@ struct TcParams {
     int pool_ctot;                   // layers per pixel of the pooled tensor
     unsigned off_pool;               // shared-memory offset of the column ring [16 rows][24 cols][BN]
     __nv_bfloat16* pool_out;
+    const void* w_ptr;               // conv_pool_kernel: the layer's kernels [Cout][ktot] in global memory
+    int ktot;                        // ... their reduction length (taps * layers per tap)
+    int dbuf;                        // ... accumulators in TMEM (2, or 1 when the kernels leave room for one only)
     const float* bias;
     int* status;
     // patch mode, at most PARAM_TAB MMAs per tile: per MMA {A offset from the stage base, B offset from the
@@ -154,6 +157,22 @@ __device__ __forceinline__ uint32_t pack_relu_bf16x2(float lo, float hi)
     uint32_t d;
     asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
     return d;
+}
+
+// maximum of three values in one instruction
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+// fp32 -> bf16 (round to nearest even), with max(., 0) folded into the conversion when relu is set
+__device__ __forceinline__ unsigned short to_bf16_bits(float v, int relu)
+{
+    unsigned short h;
+    if (relu) asm("cvt.rn.relu.bf16.f32 %0, %1;" : "=h"(h) : "f"(v));
+    else asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(h) : "f"(v));
+    return h;
 }
 
 // Position of a tile in (output-layer tile, column tile, row tile, image tile) digits.  A CTA
@@ -716,6 +735,241 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
 }
 
+// ------------------------------------------------------------------- convolution + 3x3/2 max-pool
+// The same implicit GEMM with the roles of the operands exchanged: D[layer][pixel] = sum_k W[layer][k] * X[pixel][k].
+// The kernels of the layer sit in TMEM for the whole CTA (A operand: lane = output layer, one 32-bit column = two
+// consecutive bf16 along the reduction), the pixels of a tile are the B operand, read from the shared-memory patch
+// through the same shifted descriptors as in conv_tc_kernel, and the accumulator has the output layers on the TMEM
+// lanes and the 128 pixels of the tile (8 columns x 16 rows, pixel = 8 * row + column) on its columns.  An epilogue
+// thread therefore owns one output layer and sees all pixels of the tile: the 3x3/2 max-pool is taken in its
+// registers, nothing of it goes through shared memory, and the tensor core reads only the pixel operand from shared
+// memory (half of what an M = 128 tile with both operands there costs for these narrow layers).
+// A CTA walks a strip of 16 output rows (strips 14 rows apart: 7 pooled rows) from left to right; tile k emits the
+// pooled columns 4k-1 .. 4k+2, the vertical maxima of its last two columns are carried to tile k+1 in registers.
+// Warps: 0 TMA producer, 1 MMA issuer, 2..17 epilogue (lane quadrant = warp % 4; the four groups of four warps
+// take two pooled rows of the strip each, the last group one).  The bias is added by one more MMA (bias columns {hi, lo} x tile of ones).
+constexpr int POOLT_THREADS = 64 + 512;
+constexpr int POOLT_N = 128;             // pixels per tile = accumulator columns
+
+__global__ void __launch_bounds__(POOLT_THREADS, 1)
+conv_pool_kernel(const __grid_constant__ CUtensorMap tmA, const TcParams p)
+{
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    unsigned char* base_ptr = smem_raw + (base - raw);
+    const uint32_t smA = base;
+    Shared* sh = reinterpret_cast<Shared*>(base_ptr + p.off_ctl);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t row_bytes = (uint32_t)p.BKc * 2u;
+    const int nmma = p.taps * p.chunks * (p.BKc / 16);
+    const int my_tiles = tiles_of_cta(p);
+    const uint32_t wcols = (uint32_t)p.ktot >> 1;                 // TMEM columns of the kernels
+
+    chain_release();
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) {
+            mbar_init(smem_u32(&sh->full[s]), 1);
+            mbar_init(smem_u32(&sh->empty[s]), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(smem_u32(&sh->tmem_full[a]), 1);
+            mbar_init(smem_u32(&sh->tmem_empty[a]), 16);
+        }
+        sh->abort_flag = 0;
+        fence_mbar_init();
+        prefetch_tensormap(&tmA);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&sh->tmem_base), p.tmem_cols);
+        tmem_relinquish();
+    }
+    {
+        // tile of ones for the bias MMA: 128 rows of 32 bytes in the 32-byte swizzle, ones in the first two places
+        uint4* ones = reinterpret_cast<uint4*>(base_ptr + p.off_ones);
+        for (int r = threadIdx.x; r < TILE_M; r += POOLT_THREADS) {
+            const int u = (r >> 2) & 1;
+            ones[2 * r + u] = make_uint4(0x3f803f80u, 0u, 0u, 0u);
+            ones[2 * r + (u ^ 1)] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        fence_proxy_async_smem();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = sh->tmem_base;
+    const uint32_t tmem_w = tmem_base + (uint32_t)(p.dbuf * POOLT_N);       // kernels, then 8 bias columns
+    volatile int* abort_flag = &sh->abort_flag;
+    if (!p.b_early) chain_wait();           // (stem: the kernels were repacked by the launch before this one)
+    if (warp >= 2 && warp < 6) {
+        // kernels and bias into TMEM: thread = output layer, row of ktot bf16 = ktot/2 columns
+        const int q = warp & 3, m = q * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(q * 32) << 16;
+        const uint4* wrow = reinterpret_cast<const uint4*>(static_cast<const unsigned char*>(p.w_ptr) + (size_t)m * p.ktot * 2);
+        for (uint32_t c = 0; c < wcols; c += 8) {
+            uint32_t v[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+            if (m < p.Cout) {
+                const uint4 a = __ldg(wrow + (c >> 2)), b = __ldg(wrow + (c >> 2) + 1);
+                v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+            }
+            tmem_st_x8(tmem_w + lane_base + c, v);
+        }
+        {
+            uint32_t v[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+            if (m < p.Cout) {
+                const float b = __ldg(p.bias + m);
+                const __nv_bfloat16 hi = __float2bfloat16_rn(b);
+                const __nv_bfloat16 lo = __float2bfloat16_rn(b - __bfloat162float(hi));
+                v[0] = (uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16);
+            }
+            tmem_st_x8(tmem_w + lane_base + wcols, v);
+        }
+        tmem_st_wait();
+    }
+    chain_wait();       // the earlier grid has finished: its output may be read from here on
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer: one patch per tile
+        if (lane == 0) {
+            bool ok = true;
+            int s = 0, issued = 0;
+            uint32_t ph = 0;
+            TileCoord tc;
+            tile_first(p, blockIdx.x, tc);
+            for (int it = 0; it < my_tiles; ++it, tile_next(p, tc)) {
+                const int w0 = tc.tw * p.BW, h0 = tc.th * p.h_step, i0 = tc.ti;
+                if (!wait_bar(smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                const uint32_t full = smem_u32(&sh->full[s]);
+                mbar_arrive_expect_tx(full, p.a_bytes);
+                if (p.a_lines)
+                    tma_load_5d(smA + (uint32_t)s * p.a_tile, &tmA, full, 8 * w0, 2 * h0, i0, 0, 0);
+                else
+                    for (int ch = 0; ch < p.chunks; ++ch)
+                        tma_load_5d(smA + (uint32_t)s * p.a_tile + (uint32_t)ch * p.patch_tile, &tmA, full, ch * p.BKc,
+                                    w0 - p.pad, h0 - p.pad, i0, 0);
+                ++issued;
+                if (++s == p.stages) { s = 0; ph ^= 1u; }
+            }
+            if (!ok) {
+                int pending = issued < p.stages ? issued : p.stages;
+                while (pending-- > 0) {
+                    if (s == 0) { s = p.stages; ph ^= 1u; }
+                    --s;
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(smem_u32(&sh->full[s]), ph)) {
+                        if (clock64() - t0 > WAIT_LIMIT_CYCLES / 8) break;
+                        __nanosleep(100);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        const uint32_t idesc = make_idesc_bf16(TILE_M, POOLT_N);
+        const uint32_t hiX = p.a_lines ? (uint32_t)(make_kmajor_desc_plain(0, 16u, p.sbo_bytes) >> 32)
+                                       : (uint32_t)(make_kmajor_desc(0, row_bytes, p.sbo_bytes) >> 32);
+        const uint32_t a_tile16 = p.a_tile >> 4, smA16 = smA >> 4;
+        const uint64_t ones_desc = make_kmajor_desc(base + p.off_ones, 32u, 256u);
+        bool ok = true;
+        int s = 0, as = 0;
+        uint32_t ph = 0, aph = 0;
+        for (int it = 0; it < my_tiles && ok; ++it) {
+            ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_empty[as]), aph ^ 1u, abort_flag, p.status));
+            if (!ok) break;
+            ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->full[s]), ph, abort_flag, p.status));
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(as * POOLT_N);
+            const uint32_t x_base = smA16 + (uint32_t)s * a_tile16;
+            if (elect_one()) {
+                uint32_t acc = 0u;
+#pragma unroll 2
+                for (int e = 0; e < nmma; ++e) {
+                    mma_bf16_ts(d_tmem, tmem_w + 8u * (uint32_t)e,
+                                ((uint64_t)hiX << 32) | (uint64_t)((x_base + p.ptab[e].x) | 0x10000u), idesc, acc);
+                    acc = 1u;
+                }
+                mma_commit(smem_u32(&sh->empty[s]));                // patch slot free once these MMAs have read it
+                mma_bf16_ts(d_tmem, tmem_w + wcols, ones_desc, idesc, 1u);
+                mma_commit(smem_u32(&sh->tmem_full[as]));           // accumulator complete
+            }
+            __syncwarp();
+            if (++s == p.stages) { s = 0; ph ^= 1u; }
+            if (++as == p.dbuf) { as = 0; aph ^= 1u; }
+        }
+    } else {
+        // -------------------------------------------------------------------- epilogue: pool in registers
+        // group g = (warp - 2) / 4 takes the pooled rows 2g and 2g+1 of the strip (group 3: row 6 only), i.e. the
+        // rows 4g .. 4g+4 of the tile = accumulator columns 32g .. 32g+39
+        const int q = warp & 3, grp = (warp - 2) >> 2;
+        const int m = q * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(q * 32) << 16;
+        const bool live = m < p.Cout, warp_live = q * 32 < p.Cout;
+        const int row_stride = p.PW_out * p.pool_ctot;             // elements between pooled rows
+        float carry[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+        bool ok = true;
+        int as = 0;
+        uint32_t aph = 0;
+        TileCoord tc;
+        tile_first(p, blockIdx.x, tc);
+        for (int it = 0; it < my_tiles && ok; ++it, tile_next(p, tc)) {
+            ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_full[as]), aph, abort_flag, p.status));
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + lane_base + (uint32_t)(as * POOLT_N) + (uint32_t)(grp * 32);
+            uint32_t v[48];
+            tmem_ld_x16(taddr, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
+            tmem_ld_x16(taddr + 16u, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
+            if (grp < 3) tmem_ld_x16(taddr + 32u, *reinterpret_cast<uint32_t(*)[16]>(&v[32]));
+            tmem_ld_wait();
+            // accumulator in registers: hand it back to the MMA issuer
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[as]));
+            if (++as == p.dbuf) { as = 0; aph ^= 1u; }
+
+            if (!warp_live) continue;                                   // lanes past the last output layer
+            const int pw0 = tc.tw * 4 - 1, ph0 = tc.th * 7 + grp * 2;
+            unsigned short* dst0 = reinterpret_cast<unsigned short*>(p.pool_out) +
+                                   (((size_t)tc.ti * p.PH_out + ph0) * p.PW_out + pw0) * p.pool_ctot + p.c_off + m;
+            const bool first = pw0 >= 0 && pw0 < p.PW_out, last3 = pw0 + 3 < p.PW_out, last2 = pw0 + 2 < p.PW_out, last1 = pw0 + 1 < p.PW_out;
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                if (grp == 3 && r == 1) break;                          // the last group has one pooled row
+                float c[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j)                             // vertical maximum of rows 2r, 2r+1, 2r+2, column j
+                    c[j] = max3(__uint_as_float(v[16 * r + j]), __uint_as_float(v[16 * r + 8 + j]),
+                                __uint_as_float(v[16 * r + 16 + j]));
+                const float o0 = max3(carry[r][0], carry[r][1], c[0]), o1 = max3(c[0], c[1], c[2]),
+                            o2 = max3(c[2], c[3], c[4]), o3 = max3(c[4], c[5], c[6]);
+                carry[r][0] = c[6];
+                carry[r][1] = c[7];
+                if (live && ph0 + r < p.PH_out) {
+                    unsigned short* dst = dst0 + r * row_stride;
+                    if (first) dst[0] = to_bf16_bits(o0, p.relu);
+                    if (last1) dst[p.pool_ctot] = to_bf16_bits(o1, p.relu);
+                    if (last2) dst[2 * p.pool_ctot] = to_bf16_bits(o2, p.relu);
+                    if (last3) dst[3 * p.pool_ctot] = to_bf16_bits(o3, p.relu);
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, p.tmem_cols);
+    }
+}
+
 // ---------------------------------------------------------------------------- stem repack
 // Input [N][H][W][3] bf16 -> [N][Hp][Wp][4] bf16, zero in the fourth layer and in the padding
 // column/row, so that every pixel is 8 bytes and two pixels are one 16-byte unit.
@@ -925,6 +1179,23 @@ bool choose_layout(TcParams& p, size_t a_tile, bool want_resident, int min_stage
     return false;
 }
 
+// Shared memory of conv_pool_kernel: the patch ring, the tile of ones, the control block.
+bool pool_layout(TcParams& p, size_t a_tile, size_t* smem_bytes)
+{
+    const size_t fixed = 1024 /*alignment slack*/ + (size_t)TILE_M * 32 + CTL_BYTES_NO_TAB;
+    if (t_smem_limit < fixed + 2 * a_tile) return false;
+    size_t stages = (t_smem_limit - fixed) / a_tile;
+    if (stages > MAX_STAGES) stages = MAX_STAGES;
+    p.stages = (int)stages;
+    p.a_tile = (unsigned)a_tile;
+    p.b_resident = 0;
+    p.off_b = p.off_stg = p.off_pool = p.off_bias = (unsigned)(stages * a_tile);
+    p.off_ones = p.off_bias;
+    p.off_ctl = p.off_ones + (unsigned)TILE_M * 32;
+    *smem_bytes = 1024 + (size_t)p.off_ctl + CTL_BYTES_NO_TAB;
+    return true;
+}
+
 // Builds tensor maps and kernel parameters.  For the stem, a_ptr / w_ptr are the repacked
 // tensors ([N][Hp][Wp][4] and [Cout][7][8][4]).
 int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_ptr, int Hp, int Wp, int halves,
@@ -943,7 +1214,7 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     p.h_mul = 1;
     p.b_early = stem ? 0 : 1;
     p.pool = d.pool ? 1 : 0;
-    if (p.pool && (d.OH < 3 || d.OW < 3 || d.Cout % 32 != 0 || d.Cout > 256)) return SQN_ERR_UNSUPPORTED;
+    if (p.pool && (d.OH < 3 || d.OW < 3 || d.Cout % 32 != 0 || d.Cout > TILE_M)) return SQN_ERR_UNSUPPORTED;
     if (stem) {
         p.taps = 7; p.taps_h = 7; p.taps_w = 1; p.pad = 0; p.BKc = 32; p.chunks = 1; p.k_per_tap = 32;
     } else {
@@ -963,6 +1234,15 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     if (halves == 1 && (cols > 256 || d.pool)) return SQN_ERR_UNSUPPORTED;   // two CTAs share the SM's 512 TMEM columns
     p.b_tile = ((unsigned)p.BN * row_bytes + 1023u) / 1024u * 1024u;
     p.b_bytes = (unsigned)p.BN * row_bytes;
+    if (p.pool) {
+        // conv_pool_kernel: accumulators of 128 columns, then the kernels (two bf16 per column) and 8 bias columns
+        p.w_ptr = w_ptr;
+        p.ktot = p.taps * p.k_per_tap;
+        p.tmem_cols = 512;
+        const int wcols = p.ktot / 2 + 8;
+        p.dbuf = 2 * POOLT_N + wcols <= 512 ? 2 : 1;
+        if (p.dbuf * POOLT_N + wcols > 512) return SQN_ERR_UNSUPPORTED;
+    }
 
     // output-pixel tiling; a 1x1 layer is tiled over the flattened pixel index
     const bool flat = !stem && d.K == 1 && d.pad == 0 && !d.pool;      // (a pooled 1x1 layer needs the 8x16 spatial tiles)
@@ -999,9 +1279,10 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
             patch_bytes = (unsigned)(patch_w * patch_h) * row_bytes;
             p.patch_tile = ((unsigned)max_rows * row_bytes + 1023u) / 1024u * 1024u;
         }
-        if (patch_h <= 256 && p.sbo_bytes < (1u << 18) && p.taps * p.chunks * (p.BKc / 16) <= MAX_TAB &&
-            choose_layout(p, (size_t)p.chunks * p.patch_tile, true, 2, p.taps * p.chunks * (p.BKc / 16) > PARAM_TAB,
-                          &plan->smem)) {
+        const int nmma = p.taps * p.chunks * (p.BKc / 16);
+        if (patch_h <= 256 && p.sbo_bytes < (1u << 18) && nmma <= (p.pool ? PARAM_TAB : MAX_TAB) &&
+            (p.pool ? pool_layout(p, (size_t)p.chunks * p.patch_tile, &plan->smem)
+                    : choose_layout(p, (size_t)p.chunks * p.patch_tile, true, 2, nmma > PARAM_TAB, &plan->smem))) {
             patch_ok = true;
             p.patch = 1;
             p.BW = 8; p.BH = bh; p.BI = 1;
@@ -1097,6 +1378,7 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
                              (cuuint32_t)(p.patch ? patch_h : p.BH), (cuuint32_t)p.BI, 1};
         if (!encode(&plan->a, 5, a_ptr, dims, str, box, row_bytes)) return SQN_ERR_CUDA;
     }
+    if (p.pool) return SQN_OK;      // conv_pool_kernel reads the kernels and writes the pooled map with plain accesses
     {
         const cuuint64_t kdim = (cuuint64_t)p.taps * p.k_per_tap;
         cuuint64_t dims[2] = {kdim, (cuuint64_t)d.Cout};
@@ -1108,11 +1390,9 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
         // extent of the layer dimension stops at the end of this layer's slice so that a
         // partial last tile is clipped instead of spilling into the neighbouring slice
         const cuuint64_t s1 = (cuuint64_t)d.out_c_total * 2;
-        // (when the max-pool is fused the kernel stores pooled pixels itself; the map then only has to be valid)
-        const cuuint64_t ow = p.pool ? (cuuint64_t)p.PW_out : (cuuint64_t)OW, oh = p.pool ? (cuuint64_t)p.PH_out : (cuuint64_t)OH;
-        cuuint64_t dims[4] = {(cuuint64_t)(d.out_c_offset + d.Cout), ow, oh, (cuuint64_t)NI};
-        cuuint64_t str[3] = {s1, s1 * ow, s1 * ow * oh};
-        cuuint32_t box[4] = {(cuuint32_t)p.CW, (cuuint32_t)(p.pool ? 1 : p.BW), (cuuint32_t)(p.pool ? 1 : p.BH), (cuuint32_t)p.BI};
+        cuuint64_t dims[4] = {(cuuint64_t)(d.out_c_offset + d.Cout), (cuuint64_t)OW, (cuuint64_t)OH, (cuuint64_t)NI};
+        cuuint64_t str[3] = {s1, s1 * OW, s1 * OW * OH};
+        cuuint32_t box[4] = {(cuuint32_t)p.CW, (cuuint32_t)p.BW, (cuuint32_t)p.BH, (cuuint32_t)p.BI};
         if (!encode(&plan->o, 4, d.out, dims, str, box, (unsigned)p.CW * 2u)) return SQN_ERR_CUDA;
     }
     return SQN_OK;
@@ -1147,7 +1427,12 @@ int launch_plan(const Plan& plan, cudaStream_t stream)
 {
     cudaError_t rc;
     const int hc = plan.p.CW / 2;
-    if (plan.p.pool) rc = launch_variant<2, true, 32>(plan, stream);
+    if (plan.p.pool) {
+        static const cudaError_t attr_rc =
+            cudaFuncSetAttribute(conv_pool_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
+        rc = attr_rc != cudaSuccess ? attr_rc
+           : launch_chained(conv_pool_kernel, dim3((unsigned)plan.grid), dim3(POOLT_THREADS), plan.smem, stream, plan.a, plan.p);
+    }
     else if (plan.split == 1)
         rc = hc == 32 ? launch_variant<1, false, 32>(plan, stream)
            : hc == 16 ? launch_variant<1, false, 16>(plan, stream) : launch_variant<1, false, 8>(plan, stream);
