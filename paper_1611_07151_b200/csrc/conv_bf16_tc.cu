@@ -99,9 +99,6 @@ struct TcParams {
     int pool_ctot;                   // layers per pixel of the pooled tensor
     unsigned off_pool;               // shared-memory offset of the column ring [16 rows][24 cols][BN]
     __nv_bfloat16* pool_out;
-    const void* w_ptr;               // conv_pool_kernel: the layer's kernels [Cout][ktot] in global memory
-    int ktot;                        // ... their reduction length (taps * layers per tap)
-    int dbuf;                        // ... accumulators in TMEM (2, or 1 when the kernels leave room for one only)
     const float* bias;
     int* status;
     // patch mode, at most PARAM_TAB MMAs per tile: per MMA {A offset from the stage base, B offset from the
@@ -737,36 +734,41 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
 // ------------------------------------------------------------------- convolution + 3x3/2 max-pool
 // The same implicit GEMM with the roles of the operands exchanged: D[layer][pixel] = sum_k W[layer][k] * X[pixel][k].
-// The kernels of the layer sit in TMEM for the whole CTA (A operand: lane = output layer, one 32-bit column = two
-// consecutive bf16 along the reduction), the pixels of a tile are the B operand, read from the shared-memory patch
-// through the same shifted descriptors as in conv_tc_kernel, and the accumulator has the output layers on the TMEM
-// lanes and the 128 pixels of the tile (8 columns x 16 rows, pixel = 8 * row + column) on its columns.  An epilogue
-// thread therefore owns one output layer and sees all pixels of the tile: the 3x3/2 max-pool is taken in its
-// registers, nothing of it goes through shared memory, and the tensor core reads only the pixel operand from shared
-// memory (half of what an M = 128 tile with both operands there costs for these narrow layers).
-// A CTA walks a strip of 16 output rows (strips 14 rows apart: 7 pooled rows) from left to right; tile k emits the
+// The kernels of the layer are the A operand (M = 128 rows = output layers, resident in shared memory), the 256
+// pixels of a tile (8 columns x 32 rows, pixel = 8 * row + column) are the B operand, read from the shared-memory
+// patch through the same shifted descriptors as in conv_tc_kernel, and the accumulator has the output layers on the
+// TMEM lanes and the pixels on its 256 columns.  An epilogue thread therefore owns one output layer and sees all
+// pixels of the tile: the 3x3/2 max-pool is taken in its registers and nothing of it goes through shared memory.
+// One MMA covers 256 pixels, so a tile needs half as many instructions (and per-tile hand-overs) per pixel as the
+// 128-pixel tiles of conv_tc_kernel, which is what bounds these layers with few output layers.
+// A CTA walks a strip of 32 output rows (strips 30 rows apart: 15 pooled rows) from left to right; tile k emits the
 // pooled columns 4k-1 .. 4k+2, the vertical maxima of its last two columns are carried to tile k+1 in registers.
 // Warps: 0 TMA producer, 1 MMA issuer, 2..17 epilogue (lane quadrant = warp % 4; the four groups of four warps
-// take two pooled rows of the strip each, the last group one).  The bias is added by one more MMA (bias columns {hi, lo} x tile of ones).
+// take four pooled rows of the strip each, the last group three).  The bias is added by one more MMA (bias rows
+// {hi, lo} x tile of ones).  Lanes past the last output layer compute on whatever follows the kernels in shared
+// memory and are never read.
 constexpr int POOLT_THREADS = 64 + 512;
-constexpr int POOLT_N = 128;             // pixels per tile = accumulator columns
+constexpr int POOLT_N = 256;             // pixels per tile = accumulator columns
+constexpr int POOLT_ROWS = 32;           // output rows per tile
+constexpr int POOLT_PROWS = 15;          // pooled rows per strip
 
 __global__ void __launch_bounds__(POOLT_THREADS, 1)
-conv_pool_kernel(const __grid_constant__ CUtensorMap tmA, const TcParams p)
+conv_pool_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p)
 {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_raw + (base - raw);
-    const uint32_t smA = base;
+    const uint32_t smA = base + p.off_stg;          // pixel patches (ring of p.stages slots)
+    const uint32_t smB = base + p.off_b;            // the layer's kernels
     Shared* sh = reinterpret_cast<Shared*>(base_ptr + p.off_ctl);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const uint32_t row_bytes = (uint32_t)p.BKc * 2u;
-    const int nmma = p.taps * p.chunks * (p.BKc / 16);
+    const int items = p.taps * p.chunks;
+    const int nmma = items * (p.BKc / 16);
     const int my_tiles = tiles_of_cta(p);
-    const uint32_t wcols = (uint32_t)p.ktot >> 1;                 // TMEM columns of the kernels
 
     chain_release();
     if (threadIdx.x == 0) {
@@ -774,6 +776,7 @@ conv_pool_kernel(const __grid_constant__ CUtensorMap tmA, const TcParams p)
             mbar_init(smem_u32(&sh->full[s]), 1);
             mbar_init(smem_u32(&sh->empty[s]), 1);
         }
+        mbar_init(smem_u32(&sh->b_full), 1);
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&sh->tmem_full[a]), 1);
             mbar_init(smem_u32(&sh->tmem_empty[a]), 16);
@@ -781,61 +784,36 @@ conv_pool_kernel(const __grid_constant__ CUtensorMap tmA, const TcParams p)
         sh->abort_flag = 0;
         fence_mbar_init();
         prefetch_tensormap(&tmA);
+        prefetch_tensormap(&tmB);
+        if (p.b_early) load_resident_kernels(p, tmB, smB, smem_u32(&sh->b_full), items);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(&sh->tmem_base), p.tmem_cols);
         tmem_relinquish();
     }
     {
-        // tile of ones for the bias MMA: 128 rows of 32 bytes in the 32-byte swizzle, ones in the first two places
+        // tile of ones for the bias MMA: 256 rows of 32 bytes in the 32-byte swizzle, ones in the first two places
         uint4* ones = reinterpret_cast<uint4*>(base_ptr + p.off_ones);
-        for (int r = threadIdx.x; r < TILE_M; r += POOLT_THREADS) {
+        for (int r = threadIdx.x; r < POOLT_N; r += POOLT_THREADS) {
             const int u = (r >> 2) & 1;
             ones[2 * r + u] = make_uint4(0x3f803f80u, 0u, 0u, 0u);
             ones[2 * r + (u ^ 1)] = make_uint4(0u, 0u, 0u, 0u);
         }
-        fence_proxy_async_smem();
     }
+    if (p.b_early) fill_bias_rows<POOLT_THREADS>(p, base_ptr);
+    chain_wait();       // the earlier grid has finished: its output may be read from here on
+    if (!p.b_early) fill_bias_rows<POOLT_THREADS>(p, base_ptr);
+    fence_proxy_async_smem();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = sh->tmem_base;
-    const uint32_t tmem_w = tmem_base + (uint32_t)(p.dbuf * POOLT_N);       // kernels, then 8 bias columns
     volatile int* abort_flag = &sh->abort_flag;
-    if (!p.b_early) chain_wait();           // (stem: the kernels were repacked by the launch before this one)
-    if (warp >= 2 && warp < 6) {
-        // kernels and bias into TMEM: thread = output layer, row of ktot bf16 = ktot/2 columns
-        const int q = warp & 3, m = q * 32 + lane;
-        const uint32_t lane_base = (uint32_t)(q * 32) << 16;
-        const uint4* wrow = reinterpret_cast<const uint4*>(static_cast<const unsigned char*>(p.w_ptr) + (size_t)m * p.ktot * 2);
-        for (uint32_t c = 0; c < wcols; c += 8) {
-            uint32_t v[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
-            if (m < p.Cout) {
-                const uint4 a = __ldg(wrow + (c >> 2)), b = __ldg(wrow + (c >> 2) + 1);
-                v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
-            }
-            tmem_st_x8(tmem_w + lane_base + c, v);
-        }
-        {
-            uint32_t v[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
-            if (m < p.Cout) {
-                const float b = __ldg(p.bias + m);
-                const __nv_bfloat16 hi = __float2bfloat16_rn(b);
-                const __nv_bfloat16 lo = __float2bfloat16_rn(b - __bfloat162float(hi));
-                v[0] = (uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16);
-            }
-            tmem_st_x8(tmem_w + lane_base + wcols, v);
-        }
-        tmem_st_wait();
-    }
-    chain_wait();       // the earlier grid has finished: its output may be read from here on
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer: one patch per tile
         if (lane == 0) {
+            if (!p.b_early) load_resident_kernels(p, tmB, smB, smem_u32(&sh->b_full), items);
             bool ok = true;
             int s = 0, issued = 0;
             uint32_t ph = 0;
@@ -873,9 +851,11 @@ conv_pool_kernel(const __grid_constant__ CUtensorMap tmA, const TcParams p)
         const uint32_t idesc = make_idesc_bf16(TILE_M, POOLT_N);
         const uint32_t hiX = p.a_lines ? (uint32_t)(make_kmajor_desc_plain(0, 16u, p.sbo_bytes) >> 32)
                                        : (uint32_t)(make_kmajor_desc(0, row_bytes, p.sbo_bytes) >> 32);
-        const uint32_t a_tile16 = p.a_tile >> 4, smA16 = smA >> 4;
+        const uint32_t hiW = (uint32_t)(make_kmajor_desc(0, row_bytes, 8u * row_bytes) >> 32);
+        const uint32_t a_tile16 = p.a_tile >> 4, smA16 = smA >> 4, smB16 = smB >> 4;
+        const uint64_t bias_desc = make_kmajor_desc(base + p.off_bias, 32u, 256u);
         const uint64_t ones_desc = make_kmajor_desc(base + p.off_ones, 32u, 256u);
-        bool ok = true;
+        bool ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->b_full), 0u, abort_flag, p.status));
         int s = 0, as = 0;
         uint32_t ph = 0, aph = 0;
         for (int it = 0; it < my_tiles && ok; ++it) {
@@ -890,28 +870,29 @@ conv_pool_kernel(const __grid_constant__ CUtensorMap tmA, const TcParams p)
                 uint32_t acc = 0u;
 #pragma unroll 2
                 for (int e = 0; e < nmma; ++e) {
-                    mma_bf16_ts(d_tmem, tmem_w + 8u * (uint32_t)e,
-                                ((uint64_t)hiX << 32) | (uint64_t)((x_base + p.ptab[e].x) | 0x10000u), idesc, acc);
+                    const uint2 o = p.ptab[e];
+                    mma_bf16_ss(d_tmem, ((uint64_t)hiW << 32) | (uint64_t)((smB16 + o.y) | 0x10000u),
+                                ((uint64_t)hiX << 32) | (uint64_t)((x_base + o.x) | 0x10000u), idesc, acc);
                     acc = 1u;
                 }
                 mma_commit(smem_u32(&sh->empty[s]));                // patch slot free once these MMAs have read it
-                mma_bf16_ts(d_tmem, tmem_w + wcols, ones_desc, idesc, 1u);
+                mma_bf16_ss(d_tmem, bias_desc, ones_desc, idesc, 1u);
                 mma_commit(smem_u32(&sh->tmem_full[as]));           // accumulator complete
             }
             __syncwarp();
             if (++s == p.stages) { s = 0; ph ^= 1u; }
-            if (++as == p.dbuf) { as = 0; aph ^= 1u; }
+            if (++as == 2) { as = 0; aph ^= 1u; }
         }
     } else {
         // -------------------------------------------------------------------- epilogue: pool in registers
-        // group g = (warp - 2) / 4 takes the pooled rows 2g and 2g+1 of the strip (group 3: row 6 only), i.e. the
-        // rows 4g .. 4g+4 of the tile = accumulator columns 32g .. 32g+39
+        // group g = (warp - 2) / 4 takes the pooled rows 4g .. 4g+3 of the strip (group 3: three rows), i.e. the
+        // rows 8g .. 8g+8 of the tile = accumulator columns 64g .. 64g+71
         const int q = warp & 3, grp = (warp - 2) >> 2;
         const int m = q * 32 + lane;
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
         const bool live = m < p.Cout, warp_live = q * 32 < p.Cout;
         const int row_stride = p.PW_out * p.pool_ctot;             // elements between pooled rows
-        float carry[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+        float carry[4][2] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
         bool ok = true;
         int as = 0;
         uint32_t aph = 0;
@@ -921,41 +902,50 @@ conv_pool_kernel(const __grid_constant__ CUtensorMap tmA, const TcParams p)
             ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_full[as]), aph, abort_flag, p.status));
             if (!ok) break;
             tc_fence_after();
-            const uint32_t taddr = tmem_base + lane_base + (uint32_t)(as * POOLT_N) + (uint32_t)(grp * 32);
-            uint32_t v[48];
-            tmem_ld_x16(taddr, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
-            tmem_ld_x16(taddr + 16u, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
-            if (grp < 3) tmem_ld_x16(taddr + 32u, *reinterpret_cast<uint32_t(*)[16]>(&v[32]));
-            tmem_ld_wait();
-            // accumulator in registers: hand it back to the MMA issuer
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[as]));
-            if (++as == p.dbuf) { as = 0; aph ^= 1u; }
-
-            if (!warp_live) continue;                                   // lanes past the last output layer
-            const int pw0 = tc.tw * 4 - 1, ph0 = tc.th * 7 + grp * 2;
+            const uint32_t taddr = tmem_base + lane_base + (uint32_t)(as * POOLT_N) + (uint32_t)(grp * 64);
+            const int pw0 = tc.tw * 4 - 1, ph0 = tc.th * POOLT_PROWS + grp * 4;
             unsigned short* dst0 = reinterpret_cast<unsigned short*>(p.pool_out) +
                                    (((size_t)tc.ti * p.PH_out + ph0) * p.PW_out + pw0) * p.pool_ctot + p.c_off + m;
-            const bool first = pw0 >= 0 && pw0 < p.PW_out, last3 = pw0 + 3 < p.PW_out, last2 = pw0 + 2 < p.PW_out, last1 = pw0 + 1 < p.PW_out;
+            const bool first = pw0 >= 0 && pw0 < p.PW_out, last3 = pw0 + 3 < p.PW_out, last2 = pw0 + 2 < p.PW_out,
+                       last1 = pw0 + 1 < p.PW_out;
+            // two rounds of five tile rows (40 accumulator columns) = two pooled rows each
 #pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                if (grp == 3 && r == 1) break;                          // the last group has one pooled row
-                float c[8];
+            for (int rr = 0; rr < 2; ++rr) {
+                uint32_t v[40];
+                if (warp_live) {
+                    tmem_ld_x16(taddr + 32u * rr, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
+                    tmem_ld_x16(taddr + 32u * rr + 16u, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
+                    if (grp < 3 || rr == 0) tmem_ld_x8(taddr + 32u * rr + 32u, *reinterpret_cast<uint32_t(*)[8]>(&v[32]));
+                    tmem_ld_wait();
+                }
+                if (rr == 1) {
+                    // accumulator in registers: hand it back to the MMA issuer
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[as]));
+                    if (++as == 2) { as = 0; aph ^= 1u; }
+                }
+                if (!warp_live) continue;                               // lanes past the last output layer
 #pragma unroll
-                for (int j = 0; j < 8; ++j)                             // vertical maximum of rows 2r, 2r+1, 2r+2, column j
-                    c[j] = max3(__uint_as_float(v[16 * r + j]), __uint_as_float(v[16 * r + 8 + j]),
-                                __uint_as_float(v[16 * r + 16 + j]));
-                const float o0 = max3(carry[r][0], carry[r][1], c[0]), o1 = max3(c[0], c[1], c[2]),
-                            o2 = max3(c[2], c[3], c[4]), o3 = max3(c[4], c[5], c[6]);
-                carry[r][0] = c[6];
-                carry[r][1] = c[7];
-                if (live && ph0 + r < p.PH_out) {
-                    unsigned short* dst = dst0 + r * row_stride;
-                    if (first) dst[0] = to_bf16_bits(o0, p.relu);
-                    if (last1) dst[p.pool_ctot] = to_bf16_bits(o1, p.relu);
-                    if (last2) dst[2 * p.pool_ctot] = to_bf16_bits(o2, p.relu);
-                    if (last3) dst[3 * p.pool_ctot] = to_bf16_bits(o3, p.relu);
+                for (int r2 = 0; r2 < 2; ++r2) {
+                    const int r = 2 * rr + r2;
+                    if (grp == 3 && r == 3) break;                      // the last group has three pooled rows
+                    float c[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)                         // vertical maximum of rows 2r, 2r+1, 2r+2, column j
+                        c[j] = max3(__uint_as_float(v[16 * r2 + j]), __uint_as_float(v[16 * r2 + 8 + j]),
+                                    __uint_as_float(v[16 * r2 + 16 + j]));
+                    const float o0 = max3(carry[r][0], carry[r][1], c[0]), o1 = max3(c[0], c[1], c[2]),
+                                o2 = max3(c[2], c[3], c[4]), o3 = max3(c[4], c[5], c[6]);
+                    carry[r][0] = c[6];
+                    carry[r][1] = c[7];
+                    if (live && ph0 + r < p.PH_out) {
+                        unsigned short* dst = dst0 + r * row_stride;
+                        if (first) dst[0] = to_bf16_bits(o0, p.relu);
+                        if (last1) dst[p.pool_ctot] = to_bf16_bits(o1, p.relu);
+                        if (last2) dst[2 * p.pool_ctot] = to_bf16_bits(o2, p.relu);
+                        if (last3) dst[3 * p.pool_ctot] = to_bf16_bits(o3, p.relu);
+                    }
                 }
             }
         }
@@ -1179,19 +1169,27 @@ bool choose_layout(TcParams& p, size_t a_tile, bool want_resident, int min_stage
     return false;
 }
 
-// Shared memory of conv_pool_kernel: the patch ring, the tile of ones, the control block.
+// Shared memory of conv_pool_kernel: the layer's kernels (tiles of Cout rows; an MMA reads 128 rows from a tile's
+// start, the rows past Cout come from the tiles and patches behind it), the patch ring, bias rows, the tile of ones,
+// the control block.
 bool pool_layout(TcParams& p, size_t a_tile, size_t* smem_bytes)
 {
-    const size_t fixed = 1024 /*alignment slack*/ + (size_t)TILE_M * 32 + CTL_BYTES_NO_TAB;
+    const size_t items = (size_t)p.taps * p.chunks;
+    const size_t w_bytes = items * p.b_tile;
+    const size_t fixed = 1024 /*alignment slack*/ + w_bytes + (size_t)TILE_M * 32 + (size_t)POOLT_N * 32 + CTL_BYTES_NO_TAB;
     if (t_smem_limit < fixed + 2 * a_tile) return false;
     size_t stages = (t_smem_limit - fixed) / a_tile;
     if (stages > MAX_STAGES) stages = MAX_STAGES;
+    // the 128-row read of the last kernel tile must stay inside the patch ring
+    if ((size_t)TILE_M * p.BKc * 2 > p.b_tile + stages * a_tile) return false;
     p.stages = (int)stages;
     p.a_tile = (unsigned)a_tile;
-    p.b_resident = 0;
-    p.off_b = p.off_stg = p.off_pool = p.off_bias = (unsigned)(stages * a_tile);
-    p.off_ones = p.off_bias;
-    p.off_ctl = p.off_ones + (unsigned)TILE_M * 32;
+    p.b_resident = 1;
+    p.off_b = 0;
+    p.off_stg = p.off_pool = (unsigned)w_bytes;
+    p.off_bias = p.off_stg + (unsigned)(stages * a_tile);
+    p.off_ones = p.off_bias + (unsigned)TILE_M * 32;
+    p.off_ctl = p.off_ones + (unsigned)POOLT_N * 32;
     *smem_bytes = 1024 + (size_t)p.off_ctl + CTL_BYTES_NO_TAB;
     return true;
 }
@@ -1235,13 +1233,10 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     p.b_tile = ((unsigned)p.BN * row_bytes + 1023u) / 1024u * 1024u;
     p.b_bytes = (unsigned)p.BN * row_bytes;
     if (p.pool) {
-        // conv_pool_kernel: accumulators of 128 columns, then the kernels (two bf16 per column) and 8 bias columns
-        p.w_ptr = w_ptr;
-        p.ktot = p.taps * p.k_per_tap;
-        p.tmem_cols = 512;
-        const int wcols = p.ktot / 2 + 8;
-        p.dbuf = 2 * POOLT_N + wcols <= 512 ? 2 : 1;
-        if (p.dbuf * POOLT_N + wcols > 512) return SQN_ERR_UNSUPPORTED;
+        // conv_pool_kernel: the kernels are the M = 128 operand; their tiles hold Cout rows and the rows past them
+        // belong to whatever follows in shared memory
+        p.tmem_cols = 2 * POOLT_N;
+        p.b_tile = (unsigned)p.BN * row_bytes;
     }
 
     // output-pixel tiling; a 1x1 layer is tiled over the flattened pixel index
@@ -1258,7 +1253,8 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     bool patch_ok = false;
     if (!flat && p.n_tiles == 1) {
         const int th = (OH + 15) / 16;
-        const int bh = p.pool ? 16 : (OH + th - 1) / th;     // pooling: 16 rows give 7 pooled rows, strips 14 rows apart
+        const int bh = p.pool ? POOLT_ROWS : (OH + th - 1) / th;   // pooling: 32 rows give 15 pooled rows, strips 30 rows apart
+        const unsigned last_group = p.pool ? POOLT_ROWS - 1 : 15;  // the MMA reads 16 (pooling: 32) groups of 8 pixels
         unsigned patch_bytes;              // bytes one patch box delivers per reduction chunk
         if (stem) {
             // Input lines 2*h0 .. 2*h0 + 2*BH+4, 22 pixels (176 bytes) of each, stored as they are.  Output pixel
@@ -1270,11 +1266,11 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
             p.a_lines = 1;
             p.tap_h_bytes = line_bytes; p.tap_w_bytes = 0; p.sbo_bytes = 2u * line_bytes; p.h_mul = 2;
             patch_bytes = (unsigned)patch_h * line_bytes;
-            p.patch_tile = ((2u * 15u + 7u) * line_bytes + 1023u) / 1024u * 1024u;     // the MMA always reads 16 groups
+            p.patch_tile = ((2u * last_group + 7u) * line_bytes + 1023u) / 1024u * 1024u;
         } else {
             patch_w = 8 + d.K - 1; patch_h = bh + d.K - 1;
             p.tap_h_bytes = (unsigned)patch_w * row_bytes; p.tap_w_bytes = row_bytes; p.sbo_bytes = (unsigned)patch_w * row_bytes;
-            int max_rows = 15 * patch_w + 8 + (d.K - 1) * patch_w + (d.K - 1);
+            int max_rows = (int)last_group * patch_w + 8 + (d.K - 1) * patch_w + (d.K - 1);
             if (max_rows < patch_w * patch_h) max_rows = patch_w * patch_h;
             patch_bytes = (unsigned)(patch_w * patch_h) * row_bytes;
             p.patch_tile = ((unsigned)max_rows * row_bytes + 1023u) / 1024u * 1024u;
@@ -1325,8 +1321,8 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     if (p.pool) {
         p.PW_out = (d.OW - 3) / 2 + 1;
         p.PH_out = (d.OH - 3) / 2 + 1;
-        p.h_step = 14;
-        p.tiles_h = (p.PH_out + 6) / 7;                       // seven pooled rows per strip
+        p.h_step = 2 * POOLT_PROWS;
+        p.tiles_h = (p.PH_out + POOLT_PROWS - 1) / POOLT_PROWS;
         const int tw_pool = (p.PW_out + 1 + 3) / 4;            // tile k emits pooled columns 4k-1 .. 4k+2
         if (tw_pool > p.tiles_w) p.tiles_w = tw_pool;
         p.pool_out = static_cast<__nv_bfloat16*>(d.out);
@@ -1378,7 +1374,6 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
                              (cuuint32_t)(p.patch ? patch_h : p.BH), (cuuint32_t)p.BI, 1};
         if (!encode(&plan->a, 5, a_ptr, dims, str, box, row_bytes)) return SQN_ERR_CUDA;
     }
-    if (p.pool) return SQN_OK;      // conv_pool_kernel reads the kernels and writes the pooled map with plain accesses
     {
         const cuuint64_t kdim = (cuuint64_t)p.taps * p.k_per_tap;
         cuuint64_t dims[2] = {kdim, (cuuint64_t)d.Cout};
@@ -1386,7 +1381,7 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
         cuuint32_t box[2] = {(cuuint32_t)p.BKc, (cuuint32_t)p.BN};
         if (!encode(&plan->b, 2, w_ptr, dims, str, box, row_bytes)) return SQN_ERR_CUDA;
     }
-    {
+    if (!p.pool) {                  // (conv_pool_kernel writes the pooled map with plain stores)
         // extent of the layer dimension stops at the end of this layer's slice so that a
         // partial last tile is clipped instead of spilling into the neighbouring slice
         const cuuint64_t s1 = (cuuint64_t)d.out_c_total * 2;
@@ -1431,7 +1426,7 @@ int launch_plan(const Plan& plan, cudaStream_t stream)
         static const cudaError_t attr_rc =
             cudaFuncSetAttribute(conv_pool_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
         rc = attr_rc != cudaSuccess ? attr_rc
-           : launch_chained(conv_pool_kernel, dim3((unsigned)plan.grid), dim3(POOLT_THREADS), plan.smem, stream, plan.a, plan.p);
+           : launch_chained(conv_pool_kernel, dim3((unsigned)plan.grid), dim3(POOLT_THREADS), plan.smem, stream, plan.a, plan.b, plan.p);
     }
     else if (plan.split == 1)
         rc = hc == 32 ? launch_variant<1, false, 32>(plan, stream)
