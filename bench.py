@@ -26,7 +26,7 @@ from paper_1611_07151_b200 import dist as D
 from paper_1611_07151_b200 import synth
 
 IMG = 227
-NCU_TRAFFIC_BYTES = {("conv1+pool1", "bf16", 256): 204.5e6}
+NCU_TRAFFIC_BYTES = {}      # (launch, dtype, batch) -> bytes; emptied whenever that kernel changes, refilled from a new capture
 METRIC = "squeezenet_v1.0_forward_images_per_s"
 UNIT = "images/s"
 
@@ -411,7 +411,8 @@ def main():
     # dram__bytes_read.sum + dram__bytes_write.sum per launch from the single-pass ncu capture summarised in
     # profiles/conv_tc_kernel_dram_bytes.md; None for any launch or configuration that capture does not cover
     roof["traffic"] = NCU_TRAFFIC_BYTES.get((top["name"], args.dtype, batch))
-    roof["kernel"] = ("conv_tc_kernel" if dtype == B.SQN_BF16 else "conv_f32_kernel") + "[%s]" % top["name"]
+    kname = "conv_f32_kernel" if dtype != B.SQN_BF16 else ("conv_pool_kernel" if "+pool" in top["name"] else "conv_tc_kernel")
+    roof["kernel"] = kname + "[%s]" % top["name"]
     roof["peak_source"] = "of " + peaks["source"]
     roof["launch_ms"] = top["ms"]
     roof["share_of_step"] = top["share"]
