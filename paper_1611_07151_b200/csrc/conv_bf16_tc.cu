@@ -44,10 +44,6 @@ constexpr int TILE_M = 128;            // MMA M: TMEM lanes
 // (large tiles, kernels resident in up to 227 KB); SPLIT = 1: two lighter CTAs per SM, i.e. two MMA issuers,
 // two producers and two store threads per SM, for the layers whose tiles are small.
 __host__ __device__ constexpr int threads_for(int split) { return 96 + 128 * split; }
-// With the max-pool fused the store warp is replaced by POOL_WARPS warps that pool the tiles the epilogue warps wrote.
-constexpr int POOL_WARPS = 8;
-__host__ __device__ constexpr int threads_of(int split, bool pool) { return pool ? 64 + 128 * split + 32 * POOL_WARPS : threads_for(split); }
-constexpr int RING_COLS = 24;          // column ring of the fused max-pool: three tiles of eight columns
 constexpr int MAX_STAGES = 8;
 constexpr int MAX_STG = 4;             // staging ring slots
 constexpr int MAX_TAB = 448;           // MMAs per tile in patch mode
@@ -91,13 +87,12 @@ struct TcParams {
     unsigned a_bytes, b_bytes;       // bytes one item's A box / B box delivers
     unsigned a_tile, b_tile;         // shared-memory bytes reserved per A / B tile
     unsigned off_b, off_stg, off_bias, off_ones, off_ctl;   // byte offsets from the 1024-aligned base
-    // fused 3x3/stride-2 max-pool (patch mode only): a CTA walks the tiles of a strip of output rows from
-    // left to right, keeps the last columns in shared memory and emits pooled pixels directly
+    // fused 3x3/stride-2 max-pool (conv_pool_kernel): a CTA walks the tiles of a strip of output rows from
+    // left to right and emits pooled pixels directly
     int pool;                        // 1: write max-pooled output instead of the convolution's own
-    int h_step;                      // output rows between consecutive tile rows (BH, or 14 when pooling)
+    int h_step;                      // output rows between consecutive tile rows (BH, or 30 when pooling)
     int PW_out, PH_out;              // pooled extents
     int pool_ctot;                   // layers per pixel of the pooled tensor
-    unsigned off_pool;               // shared-memory offset of the column ring [16 rows][24 cols][BN]
     __nv_bfloat16* pool_out;
     const float* bias;
     int* status;
@@ -115,8 +110,6 @@ struct Shared {                       // control block placed after the tiles
     unsigned long long tmem_empty[2];
     unsigned long long stg_full[MAX_STG];
     unsigned long long stg_free[MAX_STG];
-    unsigned long long ring_full[2];      // fused max-pool: tile written to the column ring / pooled and released
-    unsigned long long ring_free[2];
     unsigned tmem_base;
     volatile int abort_flag;
     uint2 mma_tab[MAX_TAB + 1];           // patch mode: per MMA, {A offset from the stage base, B address} in 16-byte units
@@ -231,17 +224,6 @@ __device__ __forceinline__ int tiles_of_cta(const TcParams& p)
     return p.pool ? mine * p.tiles_w : mine;
 }
 
-__device__ __forceinline__ uint4 bmax8(uint4 a, uint4 b)
-{
-    uint4 r;
-    __nv_bfloat162 x, y, m;
-    x = *reinterpret_cast<__nv_bfloat162*>(&a.x); y = *reinterpret_cast<__nv_bfloat162*>(&b.x); m = __hmax2(x, y); r.x = *reinterpret_cast<uint32_t*>(&m);
-    x = *reinterpret_cast<__nv_bfloat162*>(&a.y); y = *reinterpret_cast<__nv_bfloat162*>(&b.y); m = __hmax2(x, y); r.y = *reinterpret_cast<uint32_t*>(&m);
-    x = *reinterpret_cast<__nv_bfloat162*>(&a.z); y = *reinterpret_cast<__nv_bfloat162*>(&b.z); m = __hmax2(x, y); r.z = *reinterpret_cast<uint32_t*>(&m);
-    x = *reinterpret_cast<__nv_bfloat162*>(&a.w); y = *reinterpret_cast<__nv_bfloat162*>(&b.w); m = __hmax2(x, y); r.w = *reinterpret_cast<uint32_t*>(&m);
-    return r;
-}
-
 // Every kernel tile of the layer, once, into the resident region (one mbarrier counts all of them).
 __device__ __forceinline__ void load_resident_kernels(const TcParams& p, const CUtensorMap& tmB, uint32_t smB, uint32_t bar, int items)
 {
@@ -270,12 +252,12 @@ __device__ __forceinline__ void fill_bias_rows(const TcParams& p, unsigned char*
 
 // HC: output layers per epilogue piece (8, 16 or 32; a store chunk CW is two pieces), fixed at compile time so
 // that the conversion loop is straight-line code.
-template <int SPLIT, bool POOL, int HC>
-__global__ void __launch_bounds__(threads_of(SPLIT, POOL), SPLIT == 1 ? 2 : 1)
+template <int SPLIT, int HC>
+__global__ void __launch_bounds__(threads_for(SPLIT), SPLIT == 1 ? 2 : 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmO, const TcParams p)
 {
-    constexpr int NUM_THREADS = threads_of(SPLIT, POOL);
+    constexpr int NUM_THREADS = threads_for(SPLIT);
     constexpr int EPI_WARPS = 4 * SPLIT;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -313,10 +295,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int b = 0; b < p.nstg; ++b) {
             mbar_init(smem_u32(&sh->stg_full[b]), EPI_WARPS);
             mbar_init(smem_u32(&sh->stg_free[b]), 1);
-        }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(smem_u32(&sh->ring_full[b]), EPI_WARPS);
-            mbar_init(smem_u32(&sh->ring_free[b]), POOL_WARPS);
         }
         sh->abort_flag = 0;
         fence_mbar_init();
@@ -535,7 +513,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         bool ok = true;
         int as = 0, sb = 0;
         uint32_t aph = 0, sph = 0;
-        int ring0 = 0;                                 // fused max-pool: first ring column of the current tile
         TileCoord tc;
         tile_first(p, blockIdx.x, tc);
         for (int it = 0; it < my_tiles && ok; ++it, tile_next(p, tc)) {
@@ -544,53 +521,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (!ok) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(as * p.bn_pad);
-            if (POOL) {
-                // ---- fused max-pool, first half: the tile goes into the column ring X[16 rows][24 columns][BN]
-                // (bf16).  The k-th tile of this CTA owns ring columns 8k+2 .. 8k+9 (mod 24); the pool warps
-                // read 8k .. 8k+9, i.e. also the last two columns of the tile before, and emit the pooled
-                // columns 4*tw-1 .. 4*tw+2 of the seven pooled rows inside the tile's 16 rows.  The last
-                // readers of columns 8k+2 .. 8k+9 are the windows of tile k-2 (its columns 8k+8 and 8k+9 mod 24),
-                // so tile k is written while tile k-1 is being pooled.
-                const uint32_t smX = base + p.off_pool;
-                const int rb = it & 1;
-                ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->ring_free[rb]), (((uint32_t)it >> 1) & 1u) ^ 1u, abort_flag, p.status));
-                if (!ok) break;
-                const int r = row >> 3, j = row & 7;
-                const int half = (warp - 2) >> 2;
-                const int cper = p.BN / SPLIT;                         // layers this thread converts
-                int cb = ring0 + 2 + j;
-                if (cb >= RING_COLS) cb -= RING_COLS;
-                const uint32_t xpix = (uint32_t)p.BN * 2u + 16u;          // pixel pitch: 16 bytes of padding keep the 8
-                                                                            // pixels a quarter-warp writes in different banks
-                const uint32_t xrow = smX + (uint32_t)(r * RING_COLS + cb) * xpix + (uint32_t)(half * cper * 2);
-                for (int c16 = 0; c16 < cper; c16 += 16) {
-                    uint32_t v[16];
-                    tmem_ld_x16(taddr + (uint32_t)(half * cper + c16), v);
-                    tmem_ld_wait();
-                    float f[16];
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) f[e] = __uint_as_float(v[e]);
-                    uint32_t o[8];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e)
-                        o[e] = p.relu ? pack_relu_bf16x2(f[2 * e], f[2 * e + 1]) : pack_bf16x2(f[2 * e], f[2 * e + 1]);
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(xrow + (uint32_t)(c16 * 2)), "r"(o[0]),
-                                 "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(xrow + (uint32_t)(c16 * 2 + 16)), "r"(o[4]),
-                                 "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
-                }
-                // accumulator drained: hand it back to the MMA issuer; tile is in the ring: hand it to the pool warps
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(smem_u32(&sh->tmem_empty[as]));
-                    mbar_arrive(smem_u32(&sh->ring_full[rb]));
-                }
-                if (++as == 2) { as = 0; aph ^= 1u; }
-                ring0 += 8;
-                if (ring0 == RING_COLS) ring0 = 0;
-                continue;
-            }
             for (int chunk = 0; chunk < nchunks; ++chunk) {
                 const int c0 = chunk * p.CW;
                 if (n0 + c0 >= p.Cout) break;
@@ -643,51 +573,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[as]));
             if (++as == 2) { as = 0; aph ^= 1u; }
-        }
-    } else if (POOL) {
-        // ---- fused max-pool, second half: POOL_WARPS warps.  A thread's item is the same for every tile: one
-        // pooled row, a pair of adjacent pooled columns (their windows share a column: 15 loads for two
-        // outputs) and one 16-byte vector of layers; 7 rows x 2 pairs x BN/8 vectors <= 224 items.
-        const uint32_t smX = base + p.off_pool;
-        const uint32_t xpix = (uint32_t)p.BN * 2u + 16u;
-        const int vecs = p.BN >> 3, wk = (int)threadIdx.x - (64 + 32 * EPI_WARPS);
-        const bool has_item = wk < 14 * vecs;
-        const int pool_vec = wk % vecs, pool_pair = (wk / vecs) & 1, pool_pr = (wk / vecs) >> 1;
-        bool ok = true;
-        int ring0 = 0;
-        TileCoord tc;
-        tile_first(p, blockIdx.x, tc);
-        for (int it = 0; it < my_tiles && ok; ++it, tile_next(p, tc)) {
-            const int rb = it & 1;
-            ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->ring_full[rb]), ((uint32_t)it >> 1) & 1u, abort_flag, p.status));
-            if (!ok) break;
-            const int ph = tc.th * 7 + pool_pr, pwa = tc.tw * 4 - 1 + 2 * pool_pair;     // pooled columns pwa and pwa + 1
-            if (has_item && ph < p.PH_out && pwa + 1 >= 0 && pwa < p.PW_out) {
-                uint4 ma = make_uint4(0u, 0u, 0u, 0u), mb = ma;
-#pragma unroll
-                for (int dy = 0; dy < 3; ++dy) {
-                    uint4 w[5];
-#pragma unroll
-                    for (int dx = 0; dx < 5; ++dx) {
-                        const int xr = 2 * pool_pr + dy;
-                        int xc = ring0 + 4 * pool_pair + dx;
-                        if (xc >= RING_COLS) xc -= RING_COLS;
-                        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
-                                     : "=r"(w[dx].x), "=r"(w[dx].y), "=r"(w[dx].z), "=r"(w[dx].w)
-                                     : "r"(smX + (uint32_t)(xr * RING_COLS + xc) * xpix + (uint32_t)(pool_vec * 16)) : "memory");
-                    }
-                    const uint4 ra = bmax8(bmax8(w[0], w[1]), w[2]), rb2 = bmax8(bmax8(w[2], w[3]), w[4]);
-                    ma = dy == 0 ? ra : bmax8(ma, ra);
-                    mb = dy == 0 ? rb2 : bmax8(mb, rb2);
-                }
-                __nv_bfloat16* dst = p.pool_out + (((size_t)tc.ti * p.PH_out + ph) * p.PW_out + pwa) * p.pool_ctot + p.c_off + pool_vec * 8;
-                if (pwa >= 0) *reinterpret_cast<uint4*>(dst) = ma;
-                if (pwa + 1 < p.PW_out) *reinterpret_cast<uint4*>(dst + p.pool_ctot) = mb;
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sh->ring_free[rb]));     // (the ring was read with plain loads: in order)
-            ring0 += 8;
-            if (ring0 == RING_COLS) ring0 = 0;
         }
     } else {
         // ----------------------------------------------------------------- store issuer
@@ -1127,8 +1012,7 @@ int fit_stages(TcParams& p, size_t a_tile, bool want_resident, int cw, int nstg,
     static_assert(sizeof(Shared) <= CTL_BYTES && offsetof(Shared, mma_tab) <= CTL_BYTES_NO_TAB, "control block");
     if (SMEM_LIMIT < 1024 + bias_bytes + ctl_bytes) return 0;
     const size_t avail = SMEM_LIMIT - 1024 /*alignment slack*/ - bias_bytes - ctl_bytes;
-    const size_t stg_bytes = p.pool ? ((size_t)16 * RING_COLS * (p.BN * 2 + 16) + 1023) / 1024 * 1024   // column ring when pooling
-                                    : (size_t)nstg * slot;
+    const size_t stg_bytes = (size_t)nstg * slot;
     const size_t b_all = (size_t)items * p.b_tile;
     int stages;
     size_t b_region;
@@ -1150,7 +1034,6 @@ int fit_stages(TcParams& p, size_t a_tile, bool want_resident, int cw, int nstg,
     p.a_tile = (unsigned)a_tile;
     p.off_b = (unsigned)((size_t)stages * a_tile);
     p.off_stg = p.off_b + (unsigned)b_region;
-    p.off_pool = p.off_stg;
     p.off_bias = p.off_stg + (unsigned)stg_bytes;
     p.off_ones = p.off_bias + (unsigned)bias_rows;
     p.off_ctl = p.off_bias + (unsigned)bias_bytes;
@@ -1186,7 +1069,7 @@ bool pool_layout(TcParams& p, size_t a_tile, size_t* smem_bytes)
     p.a_tile = (unsigned)a_tile;
     p.b_resident = 1;
     p.off_b = 0;
-    p.off_stg = p.off_pool = (unsigned)w_bytes;
+    p.off_stg = (unsigned)w_bytes;
     p.off_bias = p.off_stg + (unsigned)(stages * a_tile);
     p.off_ones = p.off_bias + (unsigned)TILE_M * 32;
     p.off_ctl = p.off_ones + (unsigned)POOLT_N * 32;
@@ -1407,14 +1290,14 @@ int build_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_pt
     return build_plan_cfg(d, stem, a_ptr, w_ptr, Hp, Wp, 2, plan);
 }
 
-template <int SPLIT, bool POOL, int HC>
+template <int SPLIT, int HC>
 cudaError_t launch_variant(const Plan& plan, cudaStream_t stream)
 {
     static const cudaError_t attr_rc =
-        cudaFuncSetAttribute(conv_tc_kernel<SPLIT, POOL, HC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaFuncSetAttribute(conv_tc_kernel<SPLIT, HC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)(SPLIT == 1 ? SMEM_LIMIT_2CTA : SMEM_LIMIT));
     if (attr_rc != cudaSuccess) return attr_rc;
-    return launch_chained(conv_tc_kernel<SPLIT, POOL, HC>, dim3((unsigned)plan.grid), dim3(threads_of(SPLIT, POOL)), plan.smem,
+    return launch_chained(conv_tc_kernel<SPLIT, HC>, dim3((unsigned)plan.grid), dim3(threads_for(SPLIT)), plan.smem,
                           stream, plan.a, plan.b, plan.o, plan.p);
 }
 
@@ -1429,11 +1312,11 @@ int launch_plan(const Plan& plan, cudaStream_t stream)
            : launch_chained(conv_pool_kernel, dim3((unsigned)plan.grid), dim3(POOLT_THREADS), plan.smem, stream, plan.a, plan.b, plan.p);
     }
     else if (plan.split == 1)
-        rc = hc == 32 ? launch_variant<1, false, 32>(plan, stream)
-           : hc == 16 ? launch_variant<1, false, 16>(plan, stream) : launch_variant<1, false, 8>(plan, stream);
+        rc = hc == 32 ? launch_variant<1, 32>(plan, stream)
+           : hc == 16 ? launch_variant<1, 16>(plan, stream) : launch_variant<1, 8>(plan, stream);
     else
-        rc = hc == 32 ? launch_variant<2, false, 32>(plan, stream)
-           : hc == 16 ? launch_variant<2, false, 16>(plan, stream) : launch_variant<2, false, 8>(plan, stream);
+        rc = hc == 32 ? launch_variant<2, 32>(plan, stream)
+           : hc == 16 ? launch_variant<2, 16>(plan, stream) : launch_variant<2, 8>(plan, stream);
     if (rc != cudaSuccess) return SQN_ERR_CUDA;
     note_launch();
     return cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
