@@ -848,59 +848,85 @@ conv_pool_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 // ---------------------------------------------------------------------------- stem repack
 // Input [N][H][W][3] bf16 -> [N][Hp][Wp][4] bf16, zero in the fourth layer and in the padding
 // column/row, so that every pixel is 8 bytes and two pixels are one 16-byte unit.
-// A block repacks four rows: each row (6*W bytes, only 2-byte aligned) is brought into shared memory with
-// 16-byte loads from the enclosing aligned range, then every thread writes four pixels (32 bytes).
+// A block repacks PACK_ROWS rows: each row (6*W bytes, only 2-byte aligned) is brought into shared memory with
+// 16-byte loads from the enclosing aligned range -- all loads of a thread are issued before the first is used, so a
+// block has its whole input in flight at once -- then every thread writes four pixels (32 bytes) at a time.
 // Loads never leave [in, in + in_elems): the units that straddle an end of the tensor are read by halfwords.
+constexpr int PACK_ROWS = 16;
 __global__ void __launch_bounds__(256) stem_pack_input(const __nv_bfloat16* __restrict__ in, uint4* __restrict__ out, int N,
                                                        int H, int W, int Hp, int Wp, long long in_elems, int pitch)
 {
     chain_release();
     chain_wait();
     extern __shared__ __align__(16) unsigned short rows_s[];
-    const int r = threadIdx.x >> 6, i = threadIdx.x & 63;
-    const long long rowid = ((long long)gridDim.x - 1 - blockIdx.x) * 4ll + r;   // over N * Hp, last rows first: the stem kernel that
-                                                                                 // follows starts with the first rows, then still in the L2
-    const bool live = rowid < (long long)N * Hp;
-    const int y = live ? (int)(rowid % Hp) : 0;
-    const long long n = live ? rowid / Hp : 0;
-    unsigned short* rs = rows_s + (size_t)r * pitch;
-    int shift = 0;                                                // halfwords between the aligned start and the row
-    if (live && y < H) {
-        const unsigned long long lo = reinterpret_cast<unsigned long long>(in), hi = lo + 2ull * (unsigned long long)in_elems;
-        const unsigned long long b0 = lo + 6ull * (unsigned long long)((n * H + y) * W);
-        const unsigned long long a0 = b0 & ~15ull;
-        shift = (int)((b0 - a0) >> 1);
-        const int units = (2 * shift + 6 * W + 15) / 16;
-        for (int u = i; u < units; u += 64) {
-            const unsigned long long a = a0 + 16ull * u;
-            uint4 v;
-            if (a >= lo && a + 16 <= hi) {
-                v = __ldg(reinterpret_cast<const uint4*>(a));
-            } else {
-                unsigned short h[8];
+    constexpr int RPT = PACK_ROWS / 4;                             // rows per thread group (64 threads share a row)
+    const int r0 = threadIdx.x >> 6, i = threadIdx.x & 63;
+    // over N * Hp, last rows first: the stem kernel that follows starts with the first rows, then still in the L2
+    const long long row_base = ((long long)gridDim.x - 1 - blockIdx.x) * PACK_ROWS;
+    const long long total_rows = (long long)N * Hp;
+    const unsigned long long lo = reinterpret_cast<unsigned long long>(in), hi = lo + 2ull * (unsigned long long)in_elems;
+    int shift[RPT];                                                // halfwords between the aligned start and the row
+    const int row_units = pitch / 8;                               // 16-byte units staged per row
+    for (int u0 = 0; u0 < row_units; u0 += 128) {                  // (one round for rows up to 2 KB)
+        uint4 v[RPT][2];
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const unsigned long long ah = a + 2ull * k;
-                    h[k] = (ah >= lo && ah + 2 <= hi) ? __ldg(reinterpret_cast<const unsigned short*>(ah)) : (unsigned short)0;
+        for (int k = 0; k < RPT; ++k) {
+            const long long rowid = row_base + r0 + 4 * k;
+            const int y = rowid < total_rows ? (int)(rowid % Hp) : H;
+            const long long n = rowid < total_rows ? rowid / Hp : 0;
+            shift[k] = 0;
+            v[k][0] = v[k][1] = make_uint4(0u, 0u, 0u, 0u);
+            if (y < H) {
+                const unsigned long long b0 = lo + 6ull * (unsigned long long)((n * H + y) * W);
+                const unsigned long long a0 = b0 & ~15ull;
+                shift[k] = (int)((b0 - a0) >> 1);
+                const int units = (2 * shift[k] + 6 * W + 15) / 16;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int u = u0 + i + 64 * h;
+                    if (u >= units) continue;
+                    const unsigned long long a = a0 + 16ull * u;
+                    if (a >= lo && a + 16 <= hi) {
+                        v[k][h] = __ldg(reinterpret_cast<const uint4*>(a));
+                    } else {
+                        unsigned short e[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const unsigned long long ah = a + 2ull * j;
+                            e[j] = (ah >= lo && ah + 2 <= hi) ? __ldg(reinterpret_cast<const unsigned short*>(ah)) : (unsigned short)0;
+                        }
+                        v[k][h] = make_uint4((unsigned)e[0] | ((unsigned)e[1] << 16), (unsigned)e[2] | ((unsigned)e[3] << 16),
+                                             (unsigned)e[4] | ((unsigned)e[5] << 16), (unsigned)e[6] | ((unsigned)e[7] << 16));
+                    }
                 }
-                v = make_uint4((unsigned)h[0] | ((unsigned)h[1] << 16), (unsigned)h[2] | ((unsigned)h[3] << 16),
-                               (unsigned)h[4] | ((unsigned)h[5] << 16), (unsigned)h[6] | ((unsigned)h[7] << 16));
             }
-            reinterpret_cast<uint4*>(rs)[u] = v;
+        }
+#pragma unroll
+        for (int k = 0; k < RPT; ++k) {
+            uint4* rs = reinterpret_cast<uint4*>(rows_s + (size_t)(r0 + 4 * k) * pitch);
+            if (u0 + i < row_units) rs[u0 + i] = v[k][0];
+            if (u0 + i + 64 < row_units) rs[u0 + i + 64] = v[k][1];
         }
     }
     __syncthreads();
-    if (!live) return;
-    for (int x0 = 4 * i; x0 < Wp; x0 += 256) {
-        unsigned short e[12];
 #pragma unroll
-        for (int j = 0; j < 12; ++j) e[j] = (y < H && x0 + j / 3 < W) ? rs[shift + 3 * x0 + j] : (unsigned short)0;
-        uint4* dst = out + ((n * Hp + y) * Wp + x0) / 2;           // two pixels per 16 bytes (Wp is even)
-        dst[0] = make_uint4((unsigned)e[0] | ((unsigned)e[1] << 16), (unsigned)e[2],
-                            (unsigned)e[3] | ((unsigned)e[4] << 16), (unsigned)e[5]);
-        if (x0 + 2 < Wp)
-            dst[1] = make_uint4((unsigned)e[6] | ((unsigned)e[7] << 16), (unsigned)e[8],
-                                (unsigned)e[9] | ((unsigned)e[10] << 16), (unsigned)e[11]);
+    for (int k = 0; k < RPT; ++k) {
+        const long long rowid = row_base + r0 + 4 * k;
+        if (rowid >= total_rows) continue;
+        const int y = (int)(rowid % Hp);
+        const long long n = rowid / Hp;
+        const unsigned short* rs = rows_s + (size_t)(r0 + 4 * k) * pitch;
+        for (int x0 = 4 * i; x0 < Wp; x0 += 256) {
+            unsigned short e[12];
+#pragma unroll
+            for (int j = 0; j < 12; ++j) e[j] = (y < H && x0 + j / 3 < W) ? rs[shift[k] + 3 * x0 + j] : (unsigned short)0;
+            uint4* dst = out + ((n * Hp + y) * Wp + x0) / 2;           // two pixels per 16 bytes (Wp is even)
+            dst[0] = make_uint4((unsigned)e[0] | ((unsigned)e[1] << 16), (unsigned)e[2],
+                                (unsigned)e[3] | ((unsigned)e[4] << 16), (unsigned)e[5]);
+            if (x0 + 2 < Wp)
+                dst[1] = make_uint4((unsigned)e[6] | ((unsigned)e[7] << 16), (unsigned)e[8],
+                                    (unsigned)e[9] | ((unsigned)e[10] << 16), (unsigned)e[11]);
+        }
     }
 }
 
@@ -1431,7 +1457,8 @@ int launch_stem_pack_bf16(const ConvDesc& d, void* workspace, size_t workspace_b
     unsigned short* pw = reinterpret_cast<unsigned short*>(ws + align_up((size_t)d.N * Hp * Wp * 8, 1024));
     const long long rows = (long long)d.N * Hp;
     const int pitch = (3 * d.W + 23) / 8 * 8;                  // halfwords per staged row: the row, its lead-in, a full last unit
-    cudaError_t e = launch_chained(stem_pack_input, dim3((unsigned)((rows + 3) / 4)), dim3(256), (size_t)4 * pitch * 2, stream,
+    cudaError_t e = launch_chained(stem_pack_input, dim3((unsigned)((rows + PACK_ROWS - 1) / PACK_ROWS)), dim3(256),
+                                   (size_t)PACK_ROWS * pitch * 2, stream,
                                    static_cast<const __nv_bfloat16*>(d.in), pin, d.N, d.H, d.W, Hp, Wp,
                                    (long long)d.N * d.H * d.W * 3, pitch);
     if (e == cudaSuccess)
