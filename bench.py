@@ -71,6 +71,14 @@ def launch_work(batch, es):
     for nm, k in (("fire4_e1", 1), ("fire4_e3", 3)):
         work[nm + "+pool"] = {"flops": work[nm]["flops"],
                               "bytes": float(es * batch * (55 * 55 * 32 + 27 * 27 * 128) + es * 128 * 32 * k * k + 4 * 128)}
+    # both expands of a fire layer in one launch: squeeze map in once, both halves of the output
+    for i in range(2, 10):
+        f = "fire%d" % i
+        for a, b, n in ((f + "_e1", f + "_e3", f + "_e1+e3"), (f + "_e1+pool", f + "_e3+pool", f + "_e1+e3+pool")):
+            if a in work and b in work:
+                sq = es * batch * [c for nm, c, *_ in synth.SQUEEZENET_CONVS if nm == f + "_e1"][0] * \
+                    [hw for nm, *_, hw in synth.SQUEEZENET_CONVS if nm == f + "_e1"][0] ** 2
+                work[n] = {"flops": work[a]["flops"] + work[b]["flops"], "bytes": work[a]["bytes"] + work[b]["bytes"] - sq}
     return work
 
 
@@ -412,6 +420,8 @@ def main():
     # profiles/conv_tc_kernel_dram_bytes.md; None for any launch or configuration that capture does not cover
     roof["traffic"] = NCU_TRAFFIC_BYTES.get((top["name"], args.dtype, batch))
     kname = "conv_f32_kernel" if dtype != B.SQN_BF16 else ("conv_pool_kernel" if "+pool" in top["name"] else "conv_tc_kernel")
+    if "_e1+e3" in top["name"]:
+        kname += "2"
     roof["kernel"] = kname + "[%s]" % top["name"]
     roof["peak_source"] = "of " + peaks["source"]
     roof["launch_ms"] = top["ms"]

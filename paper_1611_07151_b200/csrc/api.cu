@@ -23,6 +23,16 @@ bool chained_launch_enabled()
     return on;
 }
 
+// The two expands of a fire layer go out as one launch (bf16) unless SQN_PAIR_LAUNCH=0.
+bool pair_launch_enabled()
+{
+    static const bool on = [] {
+        const char* v = std::getenv("SQN_PAIR_LAUNCH");
+        return !(v && v[0] == '0');
+    }();
+    return on;
+}
+
 __device__ int g_device_status;   // written by kernels whose bounded waits run out
 
 int* device_status_word()
@@ -95,6 +105,23 @@ int run_conv(const ConvDesc& d, int dtype, void* ws, size_t ws_bytes, cudaStream
     return launch_conv_bf16(d, stream);
 }
 
+// The two expands of a fire layer (same input, disjoint layer slices of one output): one launch where the bf16
+// kernels have a common variant, else two.  *paired tells which.
+int run_expands(const ConvDesc& d1, const ConvDesc& d3, int dtype, cudaStream_t stream, bool* paired)
+{
+    if (paired) *paired = false;
+    if (dtype == SQN_BF16 && pair_launch_enabled() && conv_bf16_supported(d1) == SQN_OK && conv_bf16_supported(d3) == SQN_OK) {
+        const int rc = launch_conv_bf16_pair(d1, d3, stream);
+        if (rc == SQN_OK) {
+            if (paired) *paired = true;
+            return SQN_OK;
+        }
+        if (rc != SQN_ERR_UNSUPPORTED) return rc;
+    }
+    const int rc = run_conv(d1, dtype, nullptr, 0, stream);
+    return rc != SQN_OK ? rc : run_conv(d3, dtype, nullptr, 0, stream);
+}
+
 }  // namespace
 }  // namespace sqn
 
@@ -159,8 +186,7 @@ extern "C" int fire_forward(const void* in, const void* w_sq, const void* b_sq, 
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if ((rc = run_conv(dsq, dtype, nullptr, 0, st)) != SQN_OK) return rc;
-    if ((rc = run_conv(d1, dtype, nullptr, 0, st)) != SQN_OK) return rc;
-    return run_conv(d3, dtype, nullptr, 0, st);
+    return run_expands(d1, d3, dtype, st, nullptr);
 }
 
 // ------------------------------------------------- fire layer without any allocation
@@ -482,19 +508,29 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
             p1.out = p3.out = buf(pn);
             p1.pool = p3.pool = 1;
             if (conv_bf16_pool_fits(p1) && conv_bf16_pool_fits(p3)) {
-                if ((rc = run_conv(p1, dt, nullptr, 0, st)) != SQN_OK) return rc;
-                mark((nm + "_e1+pool").c_str());
-                if ((rc = run_conv(p3, dt, nullptr, 0, st)) != SQN_OK) return rc;
-                mark((nm + "_e3+pool").c_str());
+                if (pair_launch_enabled()) {
+                    if ((rc = run_expands(p1, p3, dt, st, nullptr)) != SQN_OK) return rc;
+                    mark((nm + "_e1+e3+pool").c_str());
+                } else {
+                    if ((rc = run_conv(p1, dt, nullptr, 0, st)) != SQN_OK) return rc;
+                    mark((nm + "_e1+pool").c_str());
+                    if ((rc = run_conv(p3, dt, nullptr, 0, st)) != SQN_OK) return rc;
+                    mark((nm + "_e3+pool").c_str());
+                }
                 cur = buf(pn);
                 fused_pool = true;
             }
         }
         if (!fused_pool) {
-            if ((rc = run_conv(d1, dt, nullptr, 0, st)) != SQN_OK) return rc;
-            mark((nm + "_e1").c_str());
-            if ((rc = run_conv(d3, dt, nullptr, 0, st)) != SQN_OK) return rc;
-            mark((nm + "_e3").c_str());
+            if (dt == SQN_BF16 && pair_launch_enabled()) {
+                if ((rc = run_expands(d1, d3, dt, st, nullptr)) != SQN_OK) return rc;
+                mark((nm + "_e1+e3").c_str());
+            } else {
+                if ((rc = run_conv(d1, dt, nullptr, 0, st)) != SQN_OK) return rc;
+                mark((nm + "_e1").c_str());
+                if ((rc = run_conv(d3, dt, nullptr, 0, st)) != SQN_OK) return rc;
+                mark((nm + "_e3").c_str());
+            }
             cur = out;
             if (f.pool_after) {
                 const std::string pn = std::string("pool") + (f.name + 4);

@@ -60,7 +60,8 @@ struct TcParams {
     int n_tiles, BN;                 // output-layer tiles and their width (multiple of 16, <= 256)
     int total_tiles;
     int reverse;                     // 1: tiles are taken from the last to the first (see build_plan_cfg)
-    int g_nt, g_tw, g_th, g_ti;      // gridDim.x written in the mixed radix (n_tiles, tiles_w, tiles_h, tiles_i)
+    int grid;                        // CTAs working on this layer (the launch may hold a second layer's CTAs as well)
+    int g_nt, g_tw, g_th, g_ti;      // `grid` written in the mixed radix (n_tiles, tiles_w, tiles_h, tiles_i)
     int Cout;
     int taps, taps_w, pad;           // kernel taps, taps per kernel row, zero padding
     int chunks, BKc;                 // reduction chunks per tap, elements per chunk (16/32/64)
@@ -166,7 +167,7 @@ __device__ __forceinline__ unsigned short to_bf16_bits(float v, int relu)
 }
 
 // Position of a tile in (output-layer tile, column tile, row tile, image tile) digits.  A CTA
-// walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...; the step is added digit by digit, so the
+// walks tiles bid, bid + grid, ...; the step is added digit by digit, so the
 // loops below contain no integer division.
 struct TileCoord { int nt, tw, th, ti; };
 
@@ -215,12 +216,13 @@ __device__ __forceinline__ void tile_next(const TcParams& p, TileCoord& c)
     if (c.th >= p.tiles_h) { c.th -= p.tiles_h; carry = 1; }
     c.ti += p.g_ti + carry;
 }
-// Number of tiles this CTA processes (it takes tiles, or strips of tiles_w tiles, blockIdx.x + k*gridDim.x).
-__device__ __forceinline__ int tiles_of_cta(const TcParams& p)
+// Number of tiles CTA `bid` of the layer's `grid` CTAs processes (it takes tiles, or strips of tiles_w tiles,
+// bid + k*grid).
+__device__ __forceinline__ int tiles_of_cta(const TcParams& p, int bid)
 {
     const int units = p.pool ? p.tiles_h * p.tiles_i : p.total_tiles;
-    if ((int)blockIdx.x >= units) return 0;
-    const int mine = (units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    if (bid >= units) return 0;
+    const int mine = (units - bid + p.grid - 1) / p.grid;
     return p.pool ? mine * p.tiles_w : mine;
 }
 
@@ -253,9 +255,8 @@ __device__ __forceinline__ void fill_bias_rows(const TcParams& p, unsigned char*
 // HC: output layers per epilogue piece (8, 16 or 32; a store chunk CW is two pieces), fixed at compile time so
 // that the conversion loop is straight-line code.
 template <int SPLIT, int HC>
-__global__ void __launch_bounds__(threads_for(SPLIT), SPLIT == 1 ? 2 : 1)
-conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               const __grid_constant__ CUtensorMap tmO, const TcParams p)
+__device__ __forceinline__ void conv_tc_body(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmO,
+                                             const TcParams& p, const int bid)
 {
     constexpr int NUM_THREADS = threads_for(SPLIT);
     constexpr int EPI_WARPS = 4 * SPLIT;
@@ -274,7 +275,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t row_bytes = (uint32_t)p.BKc * 2u;
     const int items = p.taps * p.chunks;
     const int nchunks = p.BN / p.CW;
-    const int my_tiles = tiles_of_cta(p);
+    const int my_tiles = tiles_of_cta(p, bid);
 
     // The launch is chained to the kernel before it in the stream: this block may be running while
     // that grid drains.  Up to chain_wait() below it touches only its own shared memory, TMEM, the
@@ -350,7 +351,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             int s = 0, issued = 0;
             uint32_t ph = 0;
             TileCoord tc;
-            tile_first(p, blockIdx.x, tc);
+            tile_first(p, bid, tc);
             for (int it = 0; it < my_tiles && ok; ++it, tile_next(p, tc)) {
                 const int w0 = tc.tw * p.BW, h0 = tc.th * p.h_step, i0 = tc.ti * p.BI, n0 = tc.nt * p.BN;
                 if (p.patch) {
@@ -422,7 +423,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         int s = 0, as = 0;
         uint32_t ph = 0, aph = 0;
         TileCoord tc;
-        tile_first(p, blockIdx.x, tc);
+        tile_first(p, bid, tc);
         for (int it = 0; it < my_tiles && ok; ++it, tile_next(p, tc)) {
             const uint64_t bias_db = bias_db0 + (uint64_t)(2 * tc.nt * p.BN);
             ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_empty[as]), aph ^ 1u, abort_flag, p.status));
@@ -514,7 +515,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         int as = 0, sb = 0;
         uint32_t aph = 0, sph = 0;
         TileCoord tc;
-        tile_first(p, blockIdx.x, tc);
+        tile_first(p, bid, tc);
         for (int it = 0; it < my_tiles && ok; ++it, tile_next(p, tc)) {
             const int n0 = tc.nt * p.BN;
             ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_full[as]), aph, abort_flag, p.status));
@@ -582,7 +583,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             int sb = 0, pend = 0, fb = 0;       // next slot, stores whose slot is not yet released, next slot to release
             uint32_t sph = 0;
             TileCoord tc;
-            tile_first(p, blockIdx.x, tc);
+            tile_first(p, bid, tc);
             for (int it = 0; it < my_tiles && ok; ++it, tile_next(p, tc)) {
                 const int w0 = tc.tw * p.BW, h0 = tc.th * p.h_step, i0 = tc.ti * p.BI, n0 = tc.nt * p.BN;
                 for (int chunk = 0; chunk < nchunks; ++chunk) {
@@ -617,6 +618,28 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
 }
 
+// One layer per launch, or two independent layers that read the same input (the two expands of a fire layer):
+// the first p0.grid CTAs work on the first, the others on the second, so the second fills the tail of the first
+// and the pair costs one launch.
+template <int SPLIT, int HC>
+__global__ void __launch_bounds__(threads_for(SPLIT), SPLIT == 1 ? 2 : 1)
+conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmO, const __grid_constant__ TcParams p)
+{
+    conv_tc_body<SPLIT, HC>(tmA, tmB, tmO, p, (int)blockIdx.x);
+}
+
+template <int SPLIT, int HC>
+__global__ void __launch_bounds__(threads_for(SPLIT), SPLIT == 1 ? 2 : 1)
+conv_tc_kernel2(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
+                const __grid_constant__ CUtensorMap tmO0, const __grid_constant__ TcParams p0,
+                const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
+                const __grid_constant__ CUtensorMap tmO1, const __grid_constant__ TcParams p1)
+{
+    if ((int)blockIdx.x < p0.grid) conv_tc_body<SPLIT, HC>(tmA0, tmB0, tmO0, p0, (int)blockIdx.x);
+    else conv_tc_body<SPLIT, HC>(tmA1, tmB1, tmO1, p1, (int)blockIdx.x - p0.grid);
+}
+
 // ------------------------------------------------------------------- convolution + 3x3/2 max-pool
 // The same implicit GEMM with the roles of the operands exchanged: D[layer][pixel] = sum_k W[layer][k] * X[pixel][k].
 // The kernels of the layer are the A operand (M = 128 rows = output layers, resident in shared memory), the 256
@@ -637,8 +660,7 @@ constexpr int POOLT_N = 256;             // pixels per tile = accumulator column
 constexpr int POOLT_ROWS = 32;           // output rows per tile
 constexpr int POOLT_PROWS = 15;          // pooled rows per strip
 
-__global__ void __launch_bounds__(POOLT_THREADS, 1)
-conv_pool_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcParams p)
+__device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUtensorMap& tmB, const TcParams& p, const int bid)
 {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -653,7 +675,7 @@ conv_pool_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t row_bytes = (uint32_t)p.BKc * 2u;
     const int items = p.taps * p.chunks;
     const int nmma = items * (p.BKc / 16);
-    const int my_tiles = tiles_of_cta(p);
+    const int my_tiles = tiles_of_cta(p, bid);
 
     chain_release();
     if (threadIdx.x == 0) {
@@ -703,7 +725,7 @@ conv_pool_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             int s = 0, issued = 0;
             uint32_t ph = 0;
             TileCoord tc;
-            tile_first(p, blockIdx.x, tc);
+            tile_first(p, bid, tc);
             for (int it = 0; it < my_tiles; ++it, tile_next(p, tc)) {
                 const int w0 = tc.tw * p.BW, h0 = tc.th * p.h_step, i0 = tc.ti;
                 if (!wait_bar(smem_u32(&sh->empty[s]), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
@@ -782,7 +804,7 @@ conv_pool_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         int as = 0;
         uint32_t aph = 0;
         TileCoord tc;
-        tile_first(p, blockIdx.x, tc);
+        tile_first(p, bid, tc);
         for (int it = 0; it < my_tiles && ok; ++it, tile_next(p, tc)) {
             ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_full[as]), aph, abort_flag, p.status));
             if (!ok) break;
@@ -843,6 +865,23 @@ conv_pool_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         tc_fence_after();
         tmem_dealloc(tmem_base, p.tmem_cols);
     }
+}
+
+__global__ void __launch_bounds__(POOLT_THREADS, 1)
+conv_pool_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                 const __grid_constant__ TcParams p)
+{
+    conv_pool_body(tmA, tmB, p, (int)blockIdx.x);
+}
+
+// Two pooled layers over the same input in one launch (see conv_tc_kernel2).
+__global__ void __launch_bounds__(POOLT_THREADS, 1)
+conv_pool_kernel2(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
+                  const __grid_constant__ TcParams p0, const __grid_constant__ CUtensorMap tmA1,
+                  const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ TcParams p1)
+{
+    if ((int)blockIdx.x < p0.grid) conv_pool_body(tmA0, tmB0, p0, (int)blockIdx.x);
+    else conv_pool_body(tmA1, tmB1, p1, (int)blockIdx.x - p0.grid);
 }
 
 // ---------------------------------------------------------------------------- stem repack
@@ -1024,6 +1063,7 @@ int num_sms()
 // Shared-memory layout for one candidate (store chunk width, staging slots); returns the number
 // of A stages that fit (0 if the candidate does not fit at all).
 thread_local size_t t_smem_limit = SMEM_LIMIT;   // budget the layout search below works against
+thread_local int t_force_cw = 0;                 // != 0: only layouts with this store chunk width (see launch_conv_bf16_pair)
 
 int fit_stages(TcParams& p, size_t a_tile, bool want_resident, int cw, int nstg, bool smem_tab, size_t* smem_bytes)
 {
@@ -1072,7 +1112,7 @@ bool choose_layout(TcParams& p, size_t a_tile, bool want_resident, int min_stage
 {
     static const int cand[][2] = {{64, 4}, {64, 3}, {32, 4}, {64, 2}, {32, 3}, {32, 2}, {16, 4}, {16, 2}};
     for (const auto& c : cand) {
-        if (p.BN % c[0] != 0) continue;
+        if (p.BN % c[0] != 0 || (t_force_cw != 0 && c[0] != t_force_cw)) continue;
         if (fit_stages(p, a_tile, want_resident, c[0], c[1], smem_tab, smem_bytes) >= min_stages) return true;
     }
     return false;
@@ -1247,6 +1287,7 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     const long long ctas = (long long)num_sms() * (halves == 1 ? 2 : 1);
     const long long units = p.pool ? (long long)p.tiles_h * p.tiles_i : total;
     plan->grid = (int)(units < ctas ? units : ctas);
+    p.grid = plan->grid;
     if (p.pool) {
         p.g_nt = 0; p.g_tw = 0;
         p.g_th = plan->grid % p.tiles_h;
@@ -1348,6 +1389,44 @@ int launch_plan(const Plan& plan, cudaStream_t stream)
     return cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
 }
 
+template <int SPLIT, int HC>
+cudaError_t launch_variant2(const Plan& a, const Plan& b, cudaStream_t stream)
+{
+    static const cudaError_t attr_rc =
+        cudaFuncSetAttribute(conv_tc_kernel2<SPLIT, HC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(SPLIT == 1 ? SMEM_LIMIT_2CTA : SMEM_LIMIT));
+    if (attr_rc != cudaSuccess) return attr_rc;
+    return launch_chained(conv_tc_kernel2<SPLIT, HC>, dim3((unsigned)(a.grid + b.grid)), dim3(threads_for(SPLIT)),
+                          a.smem > b.smem ? a.smem : b.smem, stream, a.a, a.b, a.o, a.p, b.a, b.b, b.o, b.p);
+}
+
+// Two plans of the same kernel variant in one launch: the first a.grid CTAs run `a`, the others `b`.
+int launch_plan2(const Plan& a, const Plan& b, cudaStream_t stream)
+{
+    cudaError_t rc;
+    const size_t smem = a.smem > b.smem ? a.smem : b.smem;
+    if (a.p.pool != b.p.pool) return SQN_ERR_UNSUPPORTED;
+    if (a.p.pool) {
+        static const cudaError_t attr_rc =
+            cudaFuncSetAttribute(conv_pool_kernel2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
+        rc = attr_rc != cudaSuccess ? attr_rc
+           : launch_chained(conv_pool_kernel2, dim3((unsigned)(a.grid + b.grid)), dim3(POOLT_THREADS), smem, stream, a.a, a.b,
+                            a.p, b.a, b.b, b.p);
+    } else {
+        const int hc = a.p.CW / 2;
+        if (a.split != b.split || a.p.CW != b.p.CW) return SQN_ERR_UNSUPPORTED;
+        if (a.split == 1)
+            rc = hc == 32 ? launch_variant2<1, 32>(a, b, stream)
+               : hc == 16 ? launch_variant2<1, 16>(a, b, stream) : launch_variant2<1, 8>(a, b, stream);
+        else
+            rc = hc == 32 ? launch_variant2<2, 32>(a, b, stream)
+               : hc == 16 ? launch_variant2<2, 16>(a, b, stream) : launch_variant2<2, 8>(a, b, stream);
+    }
+    if (rc != cudaSuccess) return SQN_ERR_CUDA;
+    note_launch();
+    return cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
+}
+
 // Plans are cached by the full request: encoding three tensor maps costs microseconds that a
 // batch-1 forward would notice.
 struct PlanKey {
@@ -1358,14 +1437,16 @@ struct PlanKey {
 std::mutex g_plan_mu;
 std::map<std::string, Plan> g_plans;
 
+// force_halves / force_cw != 0: the plan of that kernel variant (CTAs per SM, store chunk width) instead of the
+// layer's own best one, so that it can share a launch with another layer's plan.
 int cached_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_ptr, int Hp, int Wp, const void* ws,
-                Plan* out)
+                Plan* out, int force_halves = 0, int force_cw = 0)
 {
     PlanKey k;
     std::memset(&k, 0, sizeof(k));
     k.in = d.in; k.w = d.w; k.bias = d.bias; k.out = d.out; k.ws = ws;
     const int v[14] = {d.N, d.Cin, d.H, d.W, d.Cout, d.K, d.S, d.pad, d.out_c_offset, d.out_c_total, d.relu | (d.pool << 1),
-                       stem ? 1 : 0, Hp, Wp};
+                       (stem ? 1 : 0) | (force_halves << 4) | (force_cw << 8), Hp, Wp};
     std::memcpy(k.v, v, sizeof(v));
     int dev = 0;
     cudaGetDevice(&dev);
@@ -1377,7 +1458,14 @@ int cached_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_p
         if (it != g_plans.end()) { *out = it->second; return SQN_OK; }
     }
     Plan plan;
-    const int rc = build_plan(d, stem, a_ptr, w_ptr, Hp, Wp, &plan);
+    int rc;
+    if (force_halves != 0) {
+        t_force_cw = force_cw;
+        rc = build_plan_cfg(d, stem, a_ptr, w_ptr, Hp, Wp, force_halves, &plan);
+        t_force_cw = 0;
+    } else {
+        rc = build_plan(d, stem, a_ptr, w_ptr, Hp, Wp, &plan);
+    }
     if (rc != SQN_OK) return rc;
     {
         std::lock_guard<std::mutex> lock(g_plan_mu);
@@ -1409,6 +1497,25 @@ int launch_conv_bf16(const ConvDesc& d, cudaStream_t stream)
     const int rc = cached_plan(d, false, d.in, d.w, 0, 0, nullptr, &plan);
     if (rc != SQN_OK) return rc;
     return launch_plan(plan, stream);
+}
+
+// Two layers that do not depend on one another (the two expands of a fire layer: same input, disjoint layer slices
+// of one output tensor) in ONE launch.  `big` keeps its own best kernel variant and takes the first CTAs, `small` is
+// planned for the same variant.  SQN_ERR_UNSUPPORTED when no common variant exists: the caller launches them one
+// after the other.
+int launch_conv_bf16_pair(const ConvDesc& small, const ConvDesc& big, cudaStream_t stream)
+{
+    if (small.pool != big.pool) return SQN_ERR_UNSUPPORTED;
+    Plan pb, ps;
+    int rc = cached_plan(big, false, big.in, big.w, 0, 0, nullptr, &pb);
+    if (rc != SQN_OK) return rc;
+    rc = cached_plan(small, false, small.in, small.w, 0, 0, nullptr, &ps);
+    if (rc != SQN_OK) return rc;
+    if (!big.pool && (ps.split != pb.split || ps.p.CW != pb.p.CW)) {
+        rc = cached_plan(small, false, small.in, small.w, 0, 0, nullptr, &ps, pb.halves, pb.p.CW);
+        if (rc != SQN_OK) return SQN_ERR_UNSUPPORTED;
+    }
+    return launch_plan2(pb, ps, stream);
 }
 
 // Host-only feasibility test of the fused max-pool for a layer (shared-memory budget, shape rules).

@@ -217,7 +217,8 @@ def test_full_forward_bf16_small_batch_keeps_every_map():
 
 def test_plain_launches_give_the_same_values():
     """SQN_CHAINED_LAUNCH=0 (read once per process) launches every kernel without programmatic stream
-    serialisation; a child process runs the batch-2 network that way and must reproduce this process's logits."""
+    serialisation and SQN_PAIR_LAUNCH=0 launches the two expands of a fire layer one after the other instead of
+    as one grid; a child process runs the batch-2 network that way and must reproduce this process's logits."""
     import os, subprocess, sys, tempfile
     x, params = synth.squeezenet_case(11, 2)
     here = run_net(x, params, BF16, 2)[0]
@@ -230,7 +231,7 @@ def test_plain_launches_give_the_same_values():
     ) % (os.path.dirname(os.path.dirname(os.path.abspath(__file__))), os.path.dirname(os.path.abspath(__file__)))
     with tempfile.TemporaryDirectory() as tmp:
         out = os.path.join(tmp, "logits.npy")
-        env = dict(os.environ, SQN_CHAINED_LAUNCH="0")
+        env = dict(os.environ, SQN_CHAINED_LAUNCH="0", SQN_PAIR_LAUNCH="0")
         subprocess.run([sys.executable, "-c", code, out], check=True, env=env, timeout=300)
         there = np.load(out)
     np.testing.assert_array_equal(here, there)
