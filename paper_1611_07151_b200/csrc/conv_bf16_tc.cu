@@ -892,16 +892,29 @@ conv_pool_kernel2(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
 // block has its whole input in flight at once -- then every thread writes four pixels (32 bytes) at a time.
 // Loads never leave [in, in + in_elems): the units that straddle an end of the tensor are read by halfwords.
 constexpr int PACK_ROWS = 16;
-__global__ void __launch_bounds__(256) stem_pack_input(const __nv_bfloat16* __restrict__ in, uint4* __restrict__ out, int N,
-                                                       int H, int W, int Hp, int Wp, long long in_elems, int pitch)
+// The blocks past the first `row_blocks` repack the layer's kernels [Cout][7][7][3] -> [Cout][7][8][4] (zero for
+// the eighth column and fourth layer), so that the stem needs one repack launch.
+__global__ void __launch_bounds__(256) stem_pack(const __nv_bfloat16* __restrict__ in, uint4* __restrict__ out, int N, int H, int W,
+                                                 int Hp, int Wp, long long in_elems, int pitch, int row_blocks,
+                                                 const unsigned short* __restrict__ w, unsigned short* __restrict__ w_out, int Cout)
 {
     chain_release();
     chain_wait();
+    if ((int)blockIdx.x >= row_blocks) {
+        const int idx = ((int)blockIdx.x - row_blocks) * 256 + (int)threadIdx.x;
+        if (idx >= Cout * 224) return;
+        const int c = idx & 3;
+        const int px = (idx >> 2) & 7;
+        const int kh = (idx >> 5) % 7;
+        const int m = idx / 224;
+        w_out[idx] = (px < 7 && c < 3) ? w[((m * 7 + kh) * 7 + px) * 3 + c] : (unsigned short)0;
+        return;
+    }
     extern __shared__ __align__(16) unsigned short rows_s[];
     constexpr int RPT = PACK_ROWS / 4;                             // rows per thread group (64 threads share a row)
     const int r0 = threadIdx.x >> 6, i = threadIdx.x & 63;
     // over N * Hp, last rows first: the stem kernel that follows starts with the first rows, then still in the L2
-    const long long row_base = ((long long)gridDim.x - 1 - blockIdx.x) * PACK_ROWS;
+    const long long row_base = ((long long)row_blocks - 1 - blockIdx.x) * PACK_ROWS;
     const long long total_rows = (long long)N * Hp;
     const unsigned long long lo = reinterpret_cast<unsigned long long>(in), hi = lo + 2ull * (unsigned long long)in_elems;
     int shift[RPT];                                                // halfwords between the aligned start and the row
@@ -967,20 +980,6 @@ __global__ void __launch_bounds__(256) stem_pack_input(const __nv_bfloat16* __re
                                     (unsigned)e[9] | ((unsigned)e[10] << 16), (unsigned)e[11]);
         }
     }
-}
-
-// Kernels [Cout][7][7][3] bf16 -> [Cout][7][8][4] bf16 (zero for the eighth column and fourth layer).
-__global__ void stem_pack_weights(const unsigned short* __restrict__ w, unsigned short* __restrict__ out, int Cout)
-{
-    chain_release();
-    chain_wait();       // also keeps the grids chained after this one behind the input repack
-    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= Cout * 224) return;
-    const int c = idx & 3;
-    const int px = (idx >> 2) & 7;
-    const int kh = (idx >> 5) % 7;
-    const int m = idx / 224;
-    out[idx] = (px < 7 && c < 3) ? w[((m * 7 + kh) * 7 + px) * 3 + c] : (unsigned short)0;
 }
 
 // ------------------------------------------------------------------------------ host side
@@ -1553,7 +1552,7 @@ int stem_check(const ConvDesc& d, void* workspace, size_t workspace_bytes)
 }
 }  // namespace
 
-// Repack of the stem's input and kernels into the workspace (two small launches).
+// Repack of the stem's input and kernels into the workspace (one launch).
 int launch_stem_pack_bf16(const ConvDesc& d, void* workspace, size_t workspace_bytes, cudaStream_t stream)
 {
     const int rc = stem_check(d, workspace, workspace_bytes);
@@ -1564,14 +1563,12 @@ int launch_stem_pack_bf16(const ConvDesc& d, void* workspace, size_t workspace_b
     unsigned short* pw = reinterpret_cast<unsigned short*>(ws + align_up((size_t)d.N * Hp * Wp * 8, 1024));
     const long long rows = (long long)d.N * Hp;
     const int pitch = (3 * d.W + 23) / 8 * 8;                  // halfwords per staged row: the row, its lead-in, a full last unit
-    cudaError_t e = launch_chained(stem_pack_input, dim3((unsigned)((rows + PACK_ROWS - 1) / PACK_ROWS)), dim3(256),
-                                   (size_t)PACK_ROWS * pitch * 2, stream,
-                                   static_cast<const __nv_bfloat16*>(d.in), pin, d.N, d.H, d.W, Hp, Wp,
-                                   (long long)d.N * d.H * d.W * 3, pitch);
-    if (e == cudaSuccess)
-        e = launch_chained(stem_pack_weights, dim3((unsigned)((d.Cout * 224 + 255) / 256)), dim3(256), 0, stream,
-                           static_cast<const unsigned short*>(d.w), pw, d.Cout);
-    note_launch(2);
+    const int row_blocks = (int)((rows + PACK_ROWS - 1) / PACK_ROWS), w_blocks = (d.Cout * 224 + 255) / 256;
+    const cudaError_t e = launch_chained(stem_pack, dim3((unsigned)(row_blocks + w_blocks)), dim3(256),
+                                         (size_t)PACK_ROWS * pitch * 2, stream, static_cast<const __nv_bfloat16*>(d.in), pin,
+                                         d.N, d.H, d.W, Hp, Wp, (long long)d.N * d.H * d.W * 3, pitch, row_blocks,
+                                         static_cast<const unsigned short*>(d.w), pw, d.Cout);
+    note_launch(1);
     return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
 }
 
