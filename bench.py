@@ -417,7 +417,7 @@ def main():
         roof = {"bound": top["bound"], "achieved": top["tflops"], "peak": pipe_tf, "unit": "TFLOP/s"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     # dram__bytes_read.sum + dram__bytes_write.sum per launch from the single-pass ncu capture summarised in
-    # profiles/conv_tc_kernel_dram_bytes.md; None for any launch or configuration that capture does not cover
+    # profiles/conv_kernels_dram_bytes.md; None for any launch or configuration that capture does not cover
     roof["traffic"] = NCU_TRAFFIC_BYTES.get((top["name"], args.dtype, batch))
     kname = "conv_f32_kernel" if dtype != B.SQN_BF16 else ("conv_pool_kernel" if "+pool" in top["name"] else "conv_tc_kernel")
     if "_e1+e3" in top["name"]:
