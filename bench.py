@@ -26,7 +26,9 @@ from paper_1611_07151_b200 import dist as D
 from paper_1611_07151_b200 import synth
 
 IMG = 227
-NCU_TRAFFIC_BYTES = {}      # (launch, dtype, batch) -> bytes; emptied whenever that kernel changes, refilled from a new capture
+# (launch, dtype, batch) -> dram__bytes_read.sum + dram__bytes_write.sum of one launch (profiles/conv_kernels_dram_bytes.md);
+# emptied whenever that kernel changes, refilled from a new capture
+NCU_TRAFFIC_BYTES = {("conv1+pool1", "bf16", 256): 205.3e6}
 METRIC = "squeezenet_v1.0_forward_images_per_s"
 UNIT = "images/s"
 
@@ -454,6 +456,12 @@ def main():
     batch1 = None
     if rank == 0 and world == 1 and not args.no_batch1:
         batch1 = run_batch1(B, ws, bs, x_pinned, dtype, dev)
+        if dtype == B.SQN_BF16:
+            # the exact path at batch 1 (fp32 storage and FFMA arithmetic): the same kernels packed as fp32
+            ws32 = [B.to_device(B.sqn_pack_weights_oihw_to_ohwi(params[n][0], B.SQN_F32), B.SQN_F32) for n in names]
+            x32 = x_pinned[:1].float().pin_memory()
+            batch1["f32"] = run_batch1(B, ws32, bs, x32, B.SQN_F32, dev)
+            del ws32
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -25,6 +25,8 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <cstddef>
@@ -1490,9 +1492,20 @@ int conv_bf16_supported(const ConvDesc& d)
     return SQN_OK;
 }
 
+// Tuning aid: SQN_TC_VARIANT="<CTAs per SM: 1|2>,<store chunk width: 16|32|64>" in the environment (read at every
+// call, so a sweep can change it between calls) makes single-layer launches use that kernel variant instead of the
+// layer's own choice; SQN_ERR_UNSUPPORTED where the variant does not fit.  `bench.py --variants` sweeps it per
+// layer, the analogue of the paper's thread-granularity study (Section III-D, Tables 1 and 3).
 int launch_conv_bf16(const ConvDesc& d, cudaStream_t stream)
 {
     Plan plan;
+    int ctas = 0, cw = 0;
+    const char* v = d.pool ? nullptr : std::getenv("SQN_TC_VARIANT");
+    if (v && std::sscanf(v, "%d,%d", &ctas, &cw) == 2 && (ctas == 1 || ctas == 2) && (cw == 16 || cw == 32 || cw == 64)) {
+        const int rc = cached_plan(d, false, d.in, d.w, 0, 0, nullptr, &plan, ctas == 1 ? 2 : 1, cw);
+        if (rc != SQN_OK) return SQN_ERR_UNSUPPORTED;
+        return launch_plan(plan, stream);
+    }
     const int rc = cached_plan(d, false, d.in, d.w, 0, 0, nullptr, &plan);
     if (rc != SQN_OK) return rc;
     return launch_plan(plan, stream);
