@@ -290,6 +290,67 @@ def run_sweep(B):
                       "note": "bf16 stem time includes its repack launches; one launch, L2 flushed, median of 10"}))
 
 
+def run_variants(B, batch):
+    """The B200 analogue of the paper's thread-granularity study (Section III-D, Tables 1 and 3): every distinct conv
+    shape (bf16, one batch) under every kernel variant that fits -- CTAs per SM (1 heavy or 2 light) x store chunk width
+    (16/32/64 output layers) -- against the variant the library picks itself; optimal, pessimal and chosen per layer."""
+    import torch
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(4)
+    seen, rows = set(), []
+    for name, cin, cout, k, s, pad, hw in synth.SQUEEZENET_CONVS:
+        key = (cin, cout, k, s, pad, hw)
+        if key in seen or (k == 7):          # (the stem has one kernel variant)
+            continue
+        seen.add(key)
+        oh = (hw + 2 * pad - k) // s + 1
+        x = torch.rand((batch, hw, hw, cin), device=dev, generator=gen).to(torch.bfloat16)
+        w = (torch.randn((cout, k, k, cin), device=dev, generator=gen) * (2.0 / (cin * k * k)) ** 0.5).to(torch.bfloat16)
+        b = torch.randn((cout,), device=dev, generator=gen) * 0.01
+        out = torch.empty((batch, oh, oh, cout), device=dev, dtype=torch.bfloat16)
+
+        def timed():
+            def call():
+                B.conv_forward_ex(x, w, b, out, cin, cout, hw, hw, k, s, pad, batch, dtype=B.SQN_BF16)
+            try:
+                for _ in range(3):
+                    call()
+            except B.SqnError as e:
+                assert e.status == B.SQN_ERR_UNSUPPORTED
+                return None
+            ts = []
+            for _ in range(10):
+                flush.zero_()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                call()
+                e1.record()
+                torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1))
+            return float(np.median(ts)) * 1e3
+
+        os.environ.pop("SQN_TC_VARIANT", None)
+        row = {"layer": name, "batch": batch, "chosen_us": timed(), "variants": {}}
+        for ctas in (1, 2):
+            for cw in (16, 32, 64):
+                os.environ["SQN_TC_VARIANT"] = "%d,%d" % (ctas, cw)
+                t = timed()
+                if t is not None:
+                    row["variants"]["%dx%d" % (ctas, cw)] = t
+        os.environ.pop("SQN_TC_VARIANT", None)
+        best = min(row["variants"].items(), key=lambda kv: kv[1])
+        worst = max(row["variants"].items(), key=lambda kv: kv[1])
+        row.update({"optimal": best[0], "optimal_us": best[1], "pessimal": worst[0], "pessimal_us": worst[1]})
+        rows.append(row)
+        del x, w, out
+    assert B.sqn_check() == B.SQN_OK
+    print(json.dumps({"variants": rows, "note": "variant = <CTAs per SM>x<store chunk width>; one launch, L2 flushed, "
+                      "median of 10, microseconds; a missing variant does not fit the layer"}))
+
+
 def workload_name(args):
     return "squeezenet_v1.0_forward_b%d_%s" % (args.batch, args.dtype)
 
@@ -307,6 +368,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-batch1", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="per-layer sweep of every conv shape instead of the network")
+    ap.add_argument("--variants", action="store_true", help="per-layer sweep of the bf16 kernel variants at --batch")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -320,6 +382,9 @@ def main():
 
     if args.sweep:
         run_sweep(B)
+        return
+    if args.variants:
+        run_variants(B, args.batch)
         return
 
     rank, local_rank, world = D.env_world()
