@@ -332,13 +332,40 @@ int launch_conv_f32(const ConvDesc& d, cudaStream_t stream)
         const long long waste = (long long)((d.Cout + bn - 1) / bn) * bn - d.Cout;
         if (best_waste < 0 || waste < best_waste) { best_waste = waste; best = bn; }
     }
-    switch (best) {
-        case 128: return launch_cfg<128, 128, 4, 2>(p, vec, stream);
-        case 96: return launch_cfg<128, 96, 2, 3>(p, vec, stream);
-        case 64: return launch_cfg<128, 64, 4, 1>(p, vec, stream);
-        case 48: return launch_cfg<128, 48, 1, 3>(p, vec, stream);
-        case 32: return launch_cfg<256, 32, 4, 1>(p, vec, stream);
-        default: return launch_cfg<256, 16, 2, 1>(p, vec, stream);
+    // Small layers (a batch of one image): that tile would give the GPU a handful of CTAs.  When it leaves SMs
+    // idle, the tile with the least estimated time is taken instead: rounds of CTAs per SM x tile area / relative
+    // FFMA efficiency of the thread tile (8 x TN: fewer output layers per thread mean more shared-memory loads per
+    // FFMA).  The sum over the reduction index runs in the same order for every tile shape, so the values do not
+    // depend on this choice.
+    int sms = 148;
+    {
+        int dev = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (sms <= 0) sms = 148;
+    }
+    auto ctas_of = [&](int tm, int tn) { return ((M + tm - 1) / tm) * (long long)((d.Cout + tn - 1) / tn); };
+    int bm = best <= 32 ? 256 : 128, bn = best;
+    if (ctas_of(bm, bn) < sms) {
+        static const struct { int bm, bn; double eff; } shapes[9] = {
+            {128, 128, 1.0}, {128, 96, 0.95}, {128, 64, 0.85}, {64, 128, 0.85}, {128, 48, 0.75},
+            {256, 32, 0.85}, {64, 64, 0.6},   {256, 16, 0.6},  {64, 32, 0.4}};
+        double best_t = -1.0;
+        for (const auto& sh : shapes) {
+            const long long c = ctas_of(sh.bm, sh.bn);
+            const double t = (double)((c + sms - 1) / sms) * sh.bm * sh.bn / sh.eff;
+            if (best_t < 0 || t < best_t) { best_t = t; bm = sh.bm; bn = sh.bn; }
+        }
+    }
+    switch (bm * 1000 + bn) {
+        case 128128: return launch_cfg<128, 128, 4, 2>(p, vec, stream);
+        case 128096: return launch_cfg<128, 96, 2, 3>(p, vec, stream);
+        case 128064: return launch_cfg<128, 64, 4, 1>(p, vec, stream);
+        case 128048: return launch_cfg<128, 48, 1, 3>(p, vec, stream);
+        case 256032: return launch_cfg<256, 32, 4, 1>(p, vec, stream);
+        case 256016: return launch_cfg<256, 16, 2, 1>(p, vec, stream);
+        case 64128: return launch_cfg<64, 128, 4, 1>(p, vec, stream);
+        case 64064: return launch_cfg<64, 64, 2, 1>(p, vec, stream);
+        default: return launch_cfg<64, 32, 1, 1>(p, vec, stream);
     }
 }
 
