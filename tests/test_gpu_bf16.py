@@ -268,3 +268,32 @@ def test_host_buffer_forward_matches_device_forward_over_calls_in_a_row():
     z, _ = ref.squeezenet(parts[2], params)
     assert G.rel_err(want[2], z) <= TOL
     B.squeezenet_destroy(net)
+
+
+def test_forced_kernel_variants_give_the_same_values():
+    """SQN_TC_VARIANT (read at every call) makes a single-layer launch use a given kernel variant -- CTAs per SM x
+    store chunk width -- instead of the layer's own choice.  Every variant that fits a 3x3 layer and a 1x1 layer must
+    give exactly the values of the default plan; one that cannot fit is refused, not replaced."""
+    import os
+    ran = 0
+    try:
+        for (N, C, M, H, K, pad) in [(2, 32, 128, 27, 3, 1), (3, 64, 64, 13, 1, 0)]:
+            rng = np.random.default_rng(C + M + K)
+            x = synth.draw_input(rng, (N, C, H, H))
+            w, b = synth.draw_conv_params(rng, C, M, K)
+            os.environ.pop("SQN_TC_VARIANT", None)
+            want = G.gpu_conv(x, w, b, 1, pad, True, BF16)
+            assert G.rel_err(want, ref.conv2d(x, w, b, S=1, pad=pad, relu=True)) <= TOL
+            for ctas in (1, 2):
+                for cw in (16, 32, 64):
+                    os.environ["SQN_TC_VARIANT"] = "%d,%d" % (ctas, cw)
+                    try:
+                        got = G.gpu_conv(x, w, b, 1, pad, True, BF16)
+                    except B.SqnError as e:
+                        assert e.status == B.SQN_ERR_UNSUPPORTED
+                        continue
+                    np.testing.assert_array_equal(got, want)
+                    ran += 1
+    finally:
+        os.environ.pop("SQN_TC_VARIANT", None)
+    assert ran >= 6
