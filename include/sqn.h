@@ -227,7 +227,9 @@ int squeezenet_forward_host(sqn_net* net, const void* in_host, void* logits_host
  *   time of launch group i summed over *forwards recorded forwards; *launches = number of
  *   groups per forward.  ms_sum may be NULL to query the counts only.
  * squeezenet_profile_name(net, i): name of group i ("conv1_pack", "conv1", "pool1",
- *   "fire2_sq", "fire2_e1", "fire2_e3", ..., "conv10", "head"); "" if out of range.
+ *   "fire2_sq", "fire2_e1", "fire2_e3", ..., "conv10", "head"; launches that cover several
+ *   steps carry all of them: "conv1+pool1", "fire2_e1+e3", "fire4_e1+e3+pool"); "" if out
+ *   of range.
  */
 int squeezenet_profile(sqn_net* net, int slots);
 int squeezenet_profile_read(sqn_net* net, float* ms_sum, int capacity, int* launches, int* forwards);
