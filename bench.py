@@ -69,10 +69,11 @@ def launch_work(batch, es):
     # stem with its max-pool fused: the 96x111x111 map is never stored, only the pooled 96x55x55 one
     work["conv1+pool1"] = {"flops": work["conv1"]["flops"],
                            "bytes": float(es * batch * (IMG * IMG * 3 + 55 * 55 * 96) + es * 96 * 147 + 4 * 96)}
-    # fire4's expands with pool4 fused: squeeze map in, pooled half (128 x 27 x 27) out
-    for nm, k in (("fire4_e1", 1), ("fire4_e3", 3)):
-        work[nm + "+pool"] = {"flops": work[nm]["flops"],
-                              "bytes": float(es * batch * (55 * 55 * 32 + 27 * 27 * 128) + es * 128 * 32 * k * k + 4 * 128)}
+    # fire4's / fire8's expands with the following pool fused: squeeze map in, pooled half of the output out
+    for fire, hw, ph, sq, e in ((4, 55, 27, 32, 128), (8, 27, 13, 64, 256)):
+        for nm, k in (("fire%d_e1" % fire, 1), ("fire%d_e3" % fire, 3)):
+            work[nm + "+pool"] = {"flops": work[nm]["flops"],
+                                  "bytes": float(es * batch * (hw * hw * sq + ph * ph * e) + es * e * sq * k * k + 4 * e)}
     # both expands of a fire layer in one launch: squeeze map in once, both halves of the output
     for i in range(2, 10):
         f = "fire%d" % i

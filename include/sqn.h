@@ -187,8 +187,8 @@ int avgpool_softmax_forward(const void* in, void* logits_f32, void* probs_f32, i
  *   gives the device address, layer count and extent of a named intermediate
  *   ("conv1", "pool1", "fire2_sq", "fire2", ..., "pool8", "fire9", "conv10");
  *   the data is in the net's dtype, NHWC, valid until the next forward.  From a batch of 16 on a bf16 net
- *   computes conv1+pool1 and fire4+pool4 in fused kernels and never stores the maps of conv1 and fire4:
- *   asking for "conv1" or "fire4" then returns SQN_ERR_UNSUPPORTED.
+ *   computes conv1+pool1, fire4+pool4 and fire8+pool8 in fused kernels and never stores the maps of conv1, fire4
+ *   and fire8: asking for one of those then returns SQN_ERR_UNSUPPORTED.
  */
 typedef struct sqn_net sqn_net;
 int squeezenet_create(sqn_net** net, const void* const* weights26, const void* const* bias26, int dtype,

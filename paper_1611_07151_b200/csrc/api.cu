@@ -395,7 +395,8 @@ extern "C" int squeezenet_layer_output(const sqn_net* net, const char* name, voi
     if (!net || !name || !workspace || !ptr || batch <= 0 || batch > net->max_batch) return SQN_ERR_BADARG;
     const int i = find_slot(net, name);
     if (i < 0) return SQN_ERR_BADARG;
-    if (net->dtype == SQN_BF16 && batch >= 16 && (std::strcmp(name, "conv1") == 0 || std::strcmp(name, "fire4") == 0))
+    if (net->dtype == SQN_BF16 && batch >= 16 &&
+        (std::strcmp(name, "conv1") == 0 || std::strcmp(name, "fire4") == 0 || std::strcmp(name, "fire8") == 0))
         return SQN_ERR_UNSUPPORTED;   // computed inside the kernels that write pool1 / pool4, never stored
     std::vector<size_t> offs;
     layout(net, batch, &offs, nullptr);
@@ -507,14 +508,32 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
             ConvDesc p1 = d1, p3 = d3;
             p1.out = p3.out = buf(pn);
             p1.pool = p3.pool = 1;
-            if (conv_bf16_pool_fits(p1) && conv_bf16_pool_fits(p3)) {
+            // the pooled kernels take up to 128 output layers: wider expands (fire8: 256) go out in slices of 128
+            const int parts = f.e > 128 && f.e % 128 == 0 ? f.e / 128 : 1;
+            ConvDesc q1[4], q3[4];
+            bool fits = parts <= 4;
+            for (int h = 0; h < parts && fits; ++h) {
+                q1[h] = p1; q3[h] = p3;
+                q1[h].Cout = q3[h].Cout = f.e / parts;
+                q1[h].w = static_cast<const char*>(p1.w) + (size_t)h * (f.e / parts) * f.s * esize(dt);
+                q3[h].w = static_cast<const char*>(p3.w) + (size_t)h * (f.e / parts) * 9 * f.s * esize(dt);
+                q1[h].bias = p1.bias + h * (f.e / parts);
+                q3[h].bias = p3.bias + h * (f.e / parts);
+                q1[h].out_c_offset = p1.out_c_offset + h * (f.e / parts);
+                q3[h].out_c_offset = p3.out_c_offset + h * (f.e / parts);
+                fits = conv_bf16_pool_fits(q1[h]) && conv_bf16_pool_fits(q3[h]);
+            }
+            if (fits) {
                 if (pair_launch_enabled()) {
-                    if ((rc = run_expands(p1, p3, dt, st, nullptr)) != SQN_OK) return rc;
+                    for (int h = 0; h < parts; ++h)
+                        if ((rc = run_expands(q1[h], q3[h], dt, st, nullptr)) != SQN_OK) return rc;
                     mark((nm + "_e1+e3+pool").c_str());
                 } else {
-                    if ((rc = run_conv(p1, dt, nullptr, 0, st)) != SQN_OK) return rc;
+                    for (int h = 0; h < parts; ++h)
+                        if ((rc = run_conv(q1[h], dt, nullptr, 0, st)) != SQN_OK) return rc;
                     mark((nm + "_e1+pool").c_str());
-                    if ((rc = run_conv(p3, dt, nullptr, 0, st)) != SQN_OK) return rc;
+                    for (int h = 0; h < parts; ++h)
+                        if ((rc = run_conv(q3[h], dt, nullptr, 0, st)) != SQN_OK) return rc;
                     mark((nm + "_e3+pool").c_str());
                 }
                 cur = buf(pn);

@@ -97,6 +97,7 @@ struct TcParams {
     int PW_out, PH_out;              // pooled extents
     int pool_ctot;                   // layers per pixel of the pooled tensor
     __nv_bfloat16* pool_out;
+    int npix;                        // conv_pool_kernel: pixels per tile, 256 or 128
     const float* bias;
     int* status;
     // patch mode, at most PARAM_TAB MMAs per tile: per MMA {A offset from the stage base, B offset from the
@@ -658,12 +659,20 @@ conv_tc_kernel2(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
 // {hi, lo} x tile of ones).  Lanes past the last output layer compute on whatever follows the kernels in shared
 // memory and are never read.
 constexpr int POOLT_THREADS = 64 + 512;
-constexpr int POOLT_N = 256;             // pixels per tile = accumulator columns
-constexpr int POOLT_ROWS = 32;           // output rows per tile
-constexpr int POOLT_PROWS = 15;          // pooled rows per strip
+__host__ __device__ constexpr int poolt_rows(int npix) { return npix / 8; }                 // output rows per tile
+__host__ __device__ constexpr int poolt_prows(int npix) { return (npix / 8 - 2) / 2; }      // pooled rows per strip
+
+// NPIX = 256 (8 x 32 pixels per tile, 15 pooled rows per strip) where the layer's kernels leave room for the larger
+// patches, else 128 (8 x 16 pixels, 7 pooled rows).
+template <int NPIX>
 
 __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUtensorMap& tmB, const TcParams& p, const int bid)
 {
+    constexpr int PROWS = poolt_prows(NPIX);          // 15 or 7
+    constexpr int PR = (PROWS + 3) / 4;               // pooled rows per epilogue group: 4 or 2
+    constexpr int ROUNDS = PR == 4 ? 2 : 1;           // TMEM read rounds per tile
+    constexpr int RPR = PR / ROUNDS;                  // pooled rows per round: 2
+    constexpr int RCOLS = 16 * RPR + 8;               // accumulator columns per round: 40
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -703,7 +712,7 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
     {
         // tile of ones for the bias MMA: 256 rows of 32 bytes in the 32-byte swizzle, ones in the first two places
         uint4* ones = reinterpret_cast<uint4*>(base_ptr + p.off_ones);
-        for (int r = threadIdx.x; r < POOLT_N; r += POOLT_THREADS) {
+        for (int r = threadIdx.x; r < NPIX; r += POOLT_THREADS) {
             const int u = (r >> 2) & 1;
             ones[2 * r + u] = make_uint4(0x3f803f80u, 0u, 0u, 0u);
             ones[2 * r + (u ^ 1)] = make_uint4(0u, 0u, 0u, 0u);
@@ -757,7 +766,7 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        const uint32_t idesc = make_idesc_bf16(TILE_M, POOLT_N);
+        const uint32_t idesc = make_idesc_bf16(TILE_M, NPIX);
         const uint32_t hiX = p.a_lines ? (uint32_t)(make_kmajor_desc_plain(0, 16u, p.sbo_bytes) >> 32)
                                        : (uint32_t)(make_kmajor_desc(0, row_bytes, p.sbo_bytes) >> 32);
         const uint32_t hiW = (uint32_t)(make_kmajor_desc(0, row_bytes, 8u * row_bytes) >> 32);
@@ -773,7 +782,7 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
             ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->full[s]), ph, abort_flag, p.status));
             if (!ok) break;
             tc_fence_after();
-            const uint32_t d_tmem = tmem_base + (uint32_t)(as * POOLT_N);
+            const uint32_t d_tmem = tmem_base + (uint32_t)(as * NPIX);
             const uint32_t x_base = smA16 + (uint32_t)s * a_tile16;
             if (elect_one()) {
                 uint32_t acc = 0u;
@@ -794,14 +803,16 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
         }
     } else {
         // -------------------------------------------------------------------- epilogue: pool in registers
-        // group g = (warp - 2) / 4 takes the pooled rows 4g .. 4g+3 of the strip (group 3: three rows), i.e. the
-        // rows 8g .. 8g+8 of the tile = accumulator columns 64g .. 64g+71
+        // group g = (warp - 2) / 4 takes the pooled rows PR*g .. PR*g + PR-1 of the strip (group 3: one fewer), i.e.
+        // the rows 2*PR*g .. 2*PR*g + 2*PR of the tile = accumulator columns 16*PR*g .. 16*PR*g + 16*PR + 7
         const int q = warp & 3, grp = (warp - 2) >> 2;
         const int m = q * 32 + lane;
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
         const bool live = m < p.Cout, warp_live = q * 32 < p.Cout;
         const int row_stride = p.PW_out * p.pool_ctot;             // elements between pooled rows
-        float carry[4][2] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
+        float carry[PR][2];
+#pragma unroll
+        for (int r = 0; r < PR; ++r) carry[r][0] = carry[r][1] = 0.f;
         bool ok = true;
         int as = 0;
         uint32_t aph = 0;
@@ -811,23 +822,25 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
             ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_full[as]), aph, abort_flag, p.status));
             if (!ok) break;
             tc_fence_after();
-            const uint32_t taddr = tmem_base + lane_base + (uint32_t)(as * POOLT_N) + (uint32_t)(grp * 64);
-            const int pw0 = tc.tw * 4 - 1, ph0 = tc.th * POOLT_PROWS + grp * 4;
+            const uint32_t taddr = tmem_base + lane_base + (uint32_t)(as * NPIX) + (uint32_t)(grp * 16 * PR);
+            const int pw0 = tc.tw * 4 - 1, ph0 = tc.th * PROWS + grp * PR;
             unsigned short* dst0 = reinterpret_cast<unsigned short*>(p.pool_out) +
                                    (((size_t)tc.ti * p.PH_out + ph0) * p.PW_out + pw0) * p.pool_ctot + p.c_off + m;
             const bool first = pw0 >= 0 && pw0 < p.PW_out, last3 = pw0 + 3 < p.PW_out, last2 = pw0 + 2 < p.PW_out,
                        last1 = pw0 + 1 < p.PW_out;
-            // two rounds of five tile rows (40 accumulator columns) = two pooled rows each
+            // ROUNDS rounds of 2*RPR + 1 tile rows (RCOLS accumulator columns) = RPR pooled rows each
 #pragma unroll
-            for (int rr = 0; rr < 2; ++rr) {
-                uint32_t v[40];
+            for (int rr = 0; rr < ROUNDS; ++rr) {
+                uint32_t v[RCOLS];
                 if (warp_live) {
-                    tmem_ld_x16(taddr + 32u * rr, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
-                    tmem_ld_x16(taddr + 32u * rr + 16u, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
-                    if (grp < 3 || rr == 0) tmem_ld_x8(taddr + 32u * rr + 32u, *reinterpret_cast<uint32_t(*)[8]>(&v[32]));
+                    const uint32_t ta = taddr + (uint32_t)(16 * RPR * rr);
+                    tmem_ld_x16(ta, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
+                    tmem_ld_x16(ta + 16u, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
+                    if (grp < 3 || rr < ROUNDS - 1) tmem_ld_x8(ta + 32u, *reinterpret_cast<uint32_t(*)[8]>(&v[32]));   // (past the
+                                                                             // accumulator for the last group's last round)
                     tmem_ld_wait();
                 }
-                if (rr == 1) {
+                if (rr == ROUNDS - 1) {
                     // accumulator in registers: hand it back to the MMA issuer
                     tc_fence_before();
                     __syncwarp();
@@ -836,9 +849,9 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
                 }
                 if (!warp_live) continue;                               // lanes past the last output layer
 #pragma unroll
-                for (int r2 = 0; r2 < 2; ++r2) {
-                    const int r = 2 * rr + r2;
-                    if (grp == 3 && r == 3) break;                      // the last group has three pooled rows
+                for (int r2 = 0; r2 < RPR; ++r2) {
+                    const int r = RPR * rr + r2;
+                    if (grp == 3 && r == PR - 1) break;                 // the last group has one pooled row fewer
                     float c[8];
 #pragma unroll
                     for (int j = 0; j < 8; ++j)                         // vertical maximum of rows 2r, 2r+1, 2r+2, column j
@@ -873,7 +886,8 @@ __global__ void __launch_bounds__(POOLT_THREADS, 1)
 conv_pool_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ TcParams p)
 {
-    conv_pool_body(tmA, tmB, p, (int)blockIdx.x);
+    if (p.npix == 256) conv_pool_body<256>(tmA, tmB, p, (int)blockIdx.x);
+    else conv_pool_body<128>(tmA, tmB, p, (int)blockIdx.x);
 }
 
 // Two pooled layers over the same input in one launch (see conv_tc_kernel2).
@@ -882,8 +896,13 @@ conv_pool_kernel2(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
                   const __grid_constant__ TcParams p0, const __grid_constant__ CUtensorMap tmA1,
                   const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ TcParams p1)
 {
-    if ((int)blockIdx.x < p0.grid) conv_pool_body(tmA0, tmB0, p0, (int)blockIdx.x);
-    else conv_pool_body(tmA1, tmB1, p1, (int)blockIdx.x - p0.grid);
+    if (p0.npix == 256) {           // (both layers have the same tile size)
+        if ((int)blockIdx.x < p0.grid) conv_pool_body<256>(tmA0, tmB0, p0, (int)blockIdx.x);
+        else conv_pool_body<256>(tmA1, tmB1, p1, (int)blockIdx.x - p0.grid);
+    } else {
+        if ((int)blockIdx.x < p0.grid) conv_pool_body<128>(tmA0, tmB0, p0, (int)blockIdx.x);
+        else conv_pool_body<128>(tmA1, tmB1, p1, (int)blockIdx.x - p0.grid);
+    }
 }
 
 // ---------------------------------------------------------------------------- stem repack
@@ -1064,6 +1083,7 @@ int num_sms()
 // Shared-memory layout for one candidate (store chunk width, staging slots); returns the number
 // of A stages that fit (0 if the candidate does not fit at all).
 thread_local size_t t_smem_limit = SMEM_LIMIT;   // budget the layout search below works against
+thread_local int t_pool_npix = 256;              // conv_pool_kernel: pixels per tile the plan is built for (256 or 128)
 thread_local int t_force_cw = 0;                 // != 0: only layouts with this store chunk width (see launch_conv_bf16_pair)
 
 int fit_stages(TcParams& p, size_t a_tile, bool want_resident, int cw, int nstg, bool smem_tab, size_t* smem_bytes)
@@ -1126,7 +1146,7 @@ bool pool_layout(TcParams& p, size_t a_tile, size_t* smem_bytes)
 {
     const size_t items = (size_t)p.taps * p.chunks;
     const size_t w_bytes = items * p.b_tile;
-    const size_t fixed = 1024 /*alignment slack*/ + w_bytes + (size_t)TILE_M * 32 + (size_t)POOLT_N * 32 + CTL_BYTES_NO_TAB;
+    const size_t fixed = 1024 /*alignment slack*/ + w_bytes + (size_t)TILE_M * 32 + (size_t)p.npix * 32 + CTL_BYTES_NO_TAB;
     if (t_smem_limit < fixed + 2 * a_tile) return false;
     size_t stages = (t_smem_limit - fixed) / a_tile;
     if (stages > MAX_STAGES) stages = MAX_STAGES;
@@ -1139,7 +1159,7 @@ bool pool_layout(TcParams& p, size_t a_tile, size_t* smem_bytes)
     p.off_stg = (unsigned)w_bytes;
     p.off_bias = p.off_stg + (unsigned)(stages * a_tile);
     p.off_ones = p.off_bias + (unsigned)TILE_M * 32;
-    p.off_ctl = p.off_ones + (unsigned)POOLT_N * 32;
+    p.off_ctl = p.off_ones + (unsigned)p.npix * 32;
     *smem_bytes = 1024 + (size_t)p.off_ctl + CTL_BYTES_NO_TAB;
     return true;
 }
@@ -1185,7 +1205,8 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     if (p.pool) {
         // conv_pool_kernel: the kernels are the M = 128 operand; their tiles hold Cout rows and the rows past them
         // belong to whatever follows in shared memory
-        p.tmem_cols = 2 * POOLT_N;
+        p.npix = t_pool_npix;
+        p.tmem_cols = 2 * (unsigned)p.npix;
         p.b_tile = (unsigned)p.BN * row_bytes;
     }
 
@@ -1203,8 +1224,8 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     bool patch_ok = false;
     if (!flat && p.n_tiles == 1) {
         const int th = (OH + 15) / 16;
-        const int bh = p.pool ? POOLT_ROWS : (OH + th - 1) / th;   // pooling: 32 rows give 15 pooled rows, strips 30 rows apart
-        const unsigned last_group = p.pool ? POOLT_ROWS - 1 : 15;  // the MMA reads 16 (pooling: 32) groups of 8 pixels
+        const int bh = p.pool ? poolt_rows(p.npix) : (OH + th - 1) / th;   // pooling: 32 (16) rows give 15 (7) pooled rows
+        const unsigned last_group = p.pool ? poolt_rows(p.npix) - 1 : 15;  // the MMA reads 16 (pooling: 32 or 16) groups of 8 pixels
         unsigned patch_bytes;              // bytes one patch box delivers per reduction chunk
         if (stem) {
             // Input lines 2*h0 .. 2*h0 + 2*BH+4, 22 pixels (176 bytes) of each, stored as they are.  Output pixel
@@ -1271,8 +1292,8 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     if (p.pool) {
         p.PW_out = (d.OW - 3) / 2 + 1;
         p.PH_out = (d.OH - 3) / 2 + 1;
-        p.h_step = 2 * POOLT_PROWS;
-        p.tiles_h = (p.PH_out + POOLT_PROWS - 1) / POOLT_PROWS;
+        p.h_step = 2 * poolt_prows(p.npix);
+        p.tiles_h = (p.PH_out + poolt_prows(p.npix) - 1) / poolt_prows(p.npix);
         const int tw_pool = (p.PW_out + 1 + 3) / 4;            // tile k emits pooled columns 4k-1 .. 4k+2
         if (tw_pool > p.tiles_w) p.tiles_w = tw_pool;
         p.pool_out = static_cast<__nv_bfloat16*>(d.out);
@@ -1355,6 +1376,16 @@ int build_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_pt
         const TcParams& p = plan->p;
         if ((p.patch && p.BN <= 64) || (!p.patch && p.taps == 1 && p.stages >= 3)) return SQN_OK;
     }
+    if (d.pool) {       // the larger tiles where the layer's kernels leave room for their patches
+        t_pool_npix = 256;
+        int rc = build_plan_cfg(d, stem, a_ptr, w_ptr, Hp, Wp, 2, plan);
+        if (rc != SQN_OK) {
+            t_pool_npix = 128;
+            rc = build_plan_cfg(d, stem, a_ptr, w_ptr, Hp, Wp, 2, plan);
+            t_pool_npix = 256;
+        }
+        return rc;
+    }
     return build_plan_cfg(d, stem, a_ptr, w_ptr, Hp, Wp, 2, plan);
 }
 
@@ -1408,6 +1439,7 @@ int launch_plan2(const Plan& a, const Plan& b, cudaStream_t stream)
     const size_t smem = a.smem > b.smem ? a.smem : b.smem;
     if (a.p.pool != b.p.pool) return SQN_ERR_UNSUPPORTED;
     if (a.p.pool) {
+        if (a.p.npix != b.p.npix) return SQN_ERR_UNSUPPORTED;
         static const cudaError_t attr_rc =
             cudaFuncSetAttribute(conv_pool_kernel2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
         rc = attr_rc != cudaSuccess ? attr_rc
@@ -1447,7 +1479,7 @@ int cached_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_p
     std::memset(&k, 0, sizeof(k));
     k.in = d.in; k.w = d.w; k.bias = d.bias; k.out = d.out; k.ws = ws;
     const int v[14] = {d.N, d.Cin, d.H, d.W, d.Cout, d.K, d.S, d.pad, d.out_c_offset, d.out_c_total, d.relu | (d.pool << 1),
-                       (stem ? 1 : 0) | (force_halves << 4) | (force_cw << 8), Hp, Wp};
+                       (stem ? 1 : 0) | (force_halves << 4) | ((force_cw & 0xffff) << 8), Hp, Wp};
     std::memcpy(k.v, v, sizeof(v));
     int dev = 0;
     cudaGetDevice(&dev);
@@ -1461,9 +1493,11 @@ int cached_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_p
     Plan plan;
     int rc;
     if (force_halves != 0) {
-        t_force_cw = force_cw;
+        t_force_cw = force_cw < 0 ? 0 : force_cw;
+        t_pool_npix = force_cw == -128 ? 128 : 256;       // (pooled layers: the tile size instead of a chunk width)
         rc = build_plan_cfg(d, stem, a_ptr, w_ptr, Hp, Wp, force_halves, &plan);
         t_force_cw = 0;
+        t_pool_npix = 256;
     } else {
         rc = build_plan(d, stem, a_ptr, w_ptr, Hp, Wp, &plan);
     }
@@ -1523,6 +1557,11 @@ int launch_conv_bf16_pair(const ConvDesc& small, const ConvDesc& big, cudaStream
     if (rc != SQN_OK) return rc;
     rc = cached_plan(small, false, small.in, small.w, 0, 0, nullptr, &ps);
     if (rc != SQN_OK) return rc;
+    if (big.pool && ps.p.npix != pb.p.npix) {          // both with the smaller tiles
+        if (cached_plan(big, false, big.in, big.w, 0, 0, nullptr, &pb, 2, -128) != SQN_OK ||
+            cached_plan(small, false, small.in, small.w, 0, 0, nullptr, &ps, 2, -128) != SQN_OK)
+            return SQN_ERR_UNSUPPORTED;
+    }
     if (!big.pool && (ps.split != pb.split || ps.p.CW != pb.p.CW)) {
         rc = cached_plan(small, false, small.in, small.w, 0, 0, nullptr, &ps, pb.halves, pb.p.CW);
         if (rc != SQN_OK) return SQN_ERR_UNSUPPORTED;
