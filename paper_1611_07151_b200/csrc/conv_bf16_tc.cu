@@ -22,6 +22,11 @@
 //   last warp            TMA stores of the staged chunks
 // Every mbarrier wait is bounded: when it runs out the CTA records SQN_ERR_TIMEOUT in the
 // device status word, drains its outstanding copies, frees its TMEM and returns.
+//
+// Kernels in this file: conv_tc_kernel (one layer), conv_tc_kernel2 (two independent layers, e.g. the two
+// expands of a fire layer, in one grid), conv_pool_kernel / conv_pool_kernel2 (convolution with the following
+// 3x3/2 max-pool: output layers on the TMEM lanes, pool taken in registers), stem_pack (repack of the stem's
+// 3-layer input and kernels).  The kernel bodies are __device__ functions of (tensor maps, parameters, CTA index).
 #include <cuda.h>
 #include <cuda_bf16.h>
 
