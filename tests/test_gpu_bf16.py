@@ -105,6 +105,8 @@ POOLED = [
     (2, 64, 32, 9, 12, 3, 1, 0),
     (2, 32, 128, 55, 55, 1, 1, 0),     # 1x1 layer (fire4 expand-1x1 followed by pool4)
     (3, 16, 64, 7, 9, 1, 1, 0),
+    (2, 64, 128, 27, 27, 3, 1, 1),     # 144 KB of kernels: the 128-pixel tiles (a 128-layer slice of fire8 expand-3x3 + pool8)
+    (1, 64, 128, 30, 19, 1, 1, 0),     # a 1x1 layer of the same width on a non-square map
 ]
 
 
