@@ -85,6 +85,8 @@ struct TcParams {
     int relu;
     int stages;                      // A (or A+B) ring slots
     int b_resident;                  // 1: all kernel tiles are loaded once and stay in shared memory
+    int bias_in_k;                   // 1 (stem): the bias sits in two unused places of the repacked kernels and meets a
+                                     // constant 1 in the fourth layer of the repacked image: no bias MMA
     int b_early;                     // 1: kernels and bias are not written by the kernel this launch is chained to, so
                                      // they are fetched before the wait for that kernel (0 for the stem: its kernels
                                      // are repacked by the launch before it)
@@ -467,7 +469,7 @@ __device__ __forceinline__ void conv_tc_body(const CUtensorMap& tmA, const CUten
                         }
                     }
                     mma_commit(smem_u32(&sh->empty[s]));            // patch slot free once these MMAs have read it
-                    mma_bf16_ss(d_tmem, bias_da, bias_db, idesc, 1u);
+                    if (!p.bias_in_k) mma_bf16_ss(d_tmem, bias_da, bias_db, idesc, 1u);
                     mma_commit(smem_u32(&sh->tmem_full[as]));       // accumulator complete
                 }
                 __syncwarp();
@@ -799,7 +801,7 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
                     acc = 1u;
                 }
                 mma_commit(smem_u32(&sh->empty[s]));                // patch slot free once these MMAs have read it
-                mma_bf16_ss(d_tmem, bias_desc, ones_desc, idesc, 1u);
+                if (!p.bias_in_k) mma_bf16_ss(d_tmem, bias_desc, ones_desc, idesc, 1u);
                 mma_commit(smem_u32(&sh->tmem_full[as]));           // accumulator complete
             }
             __syncwarp();
@@ -911,7 +913,7 @@ conv_pool_kernel2(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
 }
 
 // ---------------------------------------------------------------------------- stem repack
-// Input [N][H][W][3] bf16 -> [N][Hp][Wp][4] bf16, zero in the fourth layer and in the padding
+// Input [N][H][W][3] bf16 -> [N][Hp][Wp][4] bf16, 1.0 in the fourth layer of the image's pixels, zero in the padding
 // column/row, so that every pixel is 8 bytes and two pixels are one 16-byte unit.
 // A block repacks PACK_ROWS rows: each row (6*W bytes, only 2-byte aligned) is brought into shared memory with
 // 16-byte loads from the enclosing aligned range -- all loads of a thread are issued before the first is used, so a
@@ -919,10 +921,12 @@ conv_pool_kernel2(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
 // Loads never leave [in, in + in_elems): the units that straddle an end of the tensor are read by halfwords.
 constexpr int PACK_ROWS = 16;
 // The blocks past the first `row_blocks` repack the layer's kernels [Cout][7][7][3] -> [Cout][7][8][4] (zero for
-// the eighth column and fourth layer), so that the stem needs one repack launch.
+// the eighth column and fourth layer, except that the fourth layer of the first two pixels of the first kernel row
+// holds the bias as hi + lo: with the constant 1 of the repacked image the convolution itself adds the bias), so that the stem needs one repack launch.
 __global__ void __launch_bounds__(256) stem_pack(const __nv_bfloat16* __restrict__ in, uint4* __restrict__ out, int N, int H, int W,
                                                  int Hp, int Wp, long long in_elems, int pitch, int row_blocks,
-                                                 const unsigned short* __restrict__ w, unsigned short* __restrict__ w_out, int Cout)
+                                                 const unsigned short* __restrict__ w, unsigned short* __restrict__ w_out, int Cout,
+                                                 const float* __restrict__ bias)
 {
     chain_release();
     chain_wait();
@@ -933,7 +937,13 @@ __global__ void __launch_bounds__(256) stem_pack(const __nv_bfloat16* __restrict
         const int px = (idx >> 2) & 7;
         const int kh = (idx >> 5) % 7;
         const int m = idx / 224;
-        w_out[idx] = (px < 7 && c < 3) ? w[((m * 7 + kh) * 7 + px) * 3 + c] : (unsigned short)0;
+        unsigned short v = (px < 7 && c < 3) ? w[((m * 7 + kh) * 7 + px) * 3 + c] : (unsigned short)0;
+        if (c == 3 && kh == 0 && px < 2) {          // fourth layer of the first two pixels of the first kernel row: bias hi, lo
+            const float b = __ldg(bias + m);
+            const __nv_bfloat16 hi = __float2bfloat16_rn(b);
+            v = px == 0 ? __bfloat16_as_ushort(hi) : __bfloat16_as_ushort(__float2bfloat16_rn(b - __bfloat162float(hi)));
+        }
+        w_out[idx] = v;
         return;
     }
     extern __shared__ __align__(16) unsigned short rows_s[];
@@ -999,11 +1009,15 @@ __global__ void __launch_bounds__(256) stem_pack(const __nv_bfloat16* __restrict
 #pragma unroll
             for (int j = 0; j < 12; ++j) e[j] = (y < H && x0 + j / 3 < W) ? rs[shift[k] + 3 * x0 + j] : (unsigned short)0;
             uint4* dst = out + ((n * Hp + y) * Wp + x0) / 2;           // two pixels per 16 bytes (Wp is even)
-            dst[0] = make_uint4((unsigned)e[0] | ((unsigned)e[1] << 16), (unsigned)e[2],
-                                (unsigned)e[3] | ((unsigned)e[4] << 16), (unsigned)e[5]);
+            // fourth layer of a pixel of the image: 1.0 (it meets the bias in the repacked kernels), else 0
+            unsigned one[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) one[q] = (y < H && x0 + q < W) ? 0x3f800000u : 0u;
+            dst[0] = make_uint4((unsigned)e[0] | ((unsigned)e[1] << 16), (unsigned)e[2] | one[0],
+                                (unsigned)e[3] | ((unsigned)e[4] << 16), (unsigned)e[5] | one[1]);
             if (x0 + 2 < Wp)
-                dst[1] = make_uint4((unsigned)e[6] | ((unsigned)e[7] << 16), (unsigned)e[8],
-                                    (unsigned)e[9] | ((unsigned)e[10] << 16), (unsigned)e[11]);
+                dst[1] = make_uint4((unsigned)e[6] | ((unsigned)e[7] << 16), (unsigned)e[8] | one[2],
+                                    (unsigned)e[9] | ((unsigned)e[10] << 16), (unsigned)e[11] | one[3]);
         }
     }
 }
@@ -1186,6 +1200,7 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     p.status = device_status_word();
     p.h_mul = 1;
     p.b_early = stem ? 0 : 1;
+    p.bias_in_k = stem ? 1 : 0;
     p.pool = d.pool ? 1 : 0;
     if (p.pool && (d.OH < 3 || d.OW < 3 || d.Cout % 32 != 0 || d.Cout > TILE_M)) return SQN_ERR_UNSUPPORTED;
     if (stem) {
@@ -1624,7 +1639,7 @@ int launch_stem_pack_bf16(const ConvDesc& d, void* workspace, size_t workspace_b
     const cudaError_t e = launch_chained(stem_pack, dim3((unsigned)(row_blocks + w_blocks)), dim3(256),
                                          (size_t)PACK_ROWS * pitch * 2, stream, static_cast<const __nv_bfloat16*>(d.in), pin,
                                          d.N, d.H, d.W, Hp, Wp, (long long)d.N * d.H * d.W * 3, pitch, row_blocks,
-                                         static_cast<const unsigned short*>(d.w), pw, d.Cout);
+                                         static_cast<const unsigned short*>(d.w), pw, d.Cout, d.bias);
     note_launch(1);
     return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
 }
