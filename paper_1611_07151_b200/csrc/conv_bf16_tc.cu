@@ -704,7 +704,7 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
         mbar_init(smem_u32(&sh->b_full), 1);
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&sh->tmem_full[a]), 1);
-            mbar_init(smem_u32(&sh->tmem_empty[a]), 16);
+            mbar_init(smem_u32(&sh->tmem_empty[a]), 4 * ((p.Cout + 31) / 32));     // the epilogue warps that have output layers
         }
         sh->abort_flag = 0;
         fence_mbar_init();
@@ -825,7 +825,8 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
         uint32_t aph = 0;
         TileCoord tc;
         tile_first(p, bid, tc);
-        for (int it = 0; it < my_tiles && ok; ++it, tile_next(p, tc)) {
+        // (warps whose lanes lie past the last output layer have nothing to do and are not counted by tmem_empty)
+        for (int it = 0; it < my_tiles && ok && warp_live; ++it, tile_next(p, tc)) {
             ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_full[as]), aph, abort_flag, p.status));
             if (!ok) break;
             tc_fence_after();
