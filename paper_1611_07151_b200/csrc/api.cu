@@ -525,7 +525,14 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
             }
             if (fits) {
                 if (pair_launch_enabled()) {
-                    for (int h = 0; h < parts; ++h)
+                    bool done = false;
+                    if (parts == 2) {           // both slices of both expands as one grid, the 3x3 slices first
+                        const ConvDesc four[4] = {q3[0], q3[1], q1[0], q1[1]};
+                        rc = launch_conv_bf16_pool4(four, st);
+                        if (rc != SQN_OK && rc != SQN_ERR_UNSUPPORTED) return rc;
+                        done = rc == SQN_OK;
+                    }
+                    for (int h = 0; h < parts && !done; ++h)
                         if ((rc = run_expands(q1[h], q3[h], dt, st, nullptr)) != SQN_OK) return rc;
                     mark((nm + "_e1+e3+pool").c_str());
                 } else {

@@ -24,7 +24,7 @@
 // device status word, drains its outstanding copies, frees its TMEM and returns.
 //
 // Kernels in this file: conv_tc_kernel (one layer), conv_tc_kernel2 (two independent layers, e.g. the two
-// expands of a fire layer, in one grid), conv_pool_kernel / conv_pool_kernel2 (convolution with the following
+// expands of a fire layer, in one grid), conv_pool_kernel / conv_pool_kernel2 / conv_pool_kernel4 (convolution with the following
 // 3x3/2 max-pool: output layers on the TMEM lanes, pool taken in registers), stem_pack (repack of the stem's
 // 3-layer input and kernels).  The kernel bodies are __device__ functions of (tensor maps, parameters, CTA index).
 #include <cuda.h>
@@ -913,6 +913,24 @@ conv_pool_kernel2(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
     }
 }
 
+// Four pooled layers over the same input in one launch (the two 128-layer slices of both expands of fire8).
+__global__ void __launch_bounds__(POOLT_THREADS, 1)
+conv_pool_kernel4(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
+                  const __grid_constant__ TcParams p0, const __grid_constant__ CUtensorMap tmA1,
+                  const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ TcParams p1,
+                  const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB2,
+                  const __grid_constant__ TcParams p2, const __grid_constant__ CUtensorMap tmA3,
+                  const __grid_constant__ CUtensorMap tmB3, const __grid_constant__ TcParams p3)
+{
+    int b = (int)blockIdx.x;                       // (all four layers have 128-pixel tiles)
+    if (b < p0.grid) { conv_pool_body<128>(tmA0, tmB0, p0, b); return; }
+    b -= p0.grid;
+    if (b < p1.grid) { conv_pool_body<128>(tmA1, tmB1, p1, b); return; }
+    b -= p1.grid;
+    if (b < p2.grid) { conv_pool_body<128>(tmA2, tmB2, p2, b); return; }
+    conv_pool_body<128>(tmA3, tmB3, p3, b - p2.grid);
+}
+
 // ---------------------------------------------------------------------------- stem repack
 // Input [N][H][W][3] bf16 -> [N][Hp][Wp][4] bf16, 1.0 in the fourth layer of the image's pixels, zero in the padding
 // column/row, so that every pixel is 8 bytes and two pixels are one 16-byte unit.
@@ -1588,6 +1606,29 @@ int launch_conv_bf16_pair(const ConvDesc& small, const ConvDesc& big, cudaStream
         if (rc != SQN_OK) return SQN_ERR_UNSUPPORTED;
     }
     return launch_plan2(pb, ps, stream);
+}
+
+// Four pooled layers that read the same input (two slices of each expand of a fire layer) in ONE launch, in the order
+// given (the heavy ones first); all with the 128-pixel tiles.  SQN_ERR_UNSUPPORTED if one of them cannot be planned so.
+int launch_conv_bf16_pool4(const ConvDesc* d, cudaStream_t stream)
+{
+    Plan pl[4];
+    size_t smem = 0;
+    int grid = 0;
+    for (int i = 0; i < 4; ++i) {
+        if (!d[i].pool || cached_plan(d[i], false, d[i].in, d[i].w, 0, 0, nullptr, &pl[i], 2, -128) != SQN_OK || pl[i].p.npix != 128)
+            return SQN_ERR_UNSUPPORTED;
+        if (pl[i].smem > smem) smem = pl[i].smem;
+        grid += pl[i].grid;
+    }
+    static const cudaError_t attr_rc =
+        cudaFuncSetAttribute(conv_pool_kernel4, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
+    if (attr_rc != cudaSuccess) return SQN_ERR_CUDA;
+    const cudaError_t rc = launch_chained(conv_pool_kernel4, dim3((unsigned)grid), dim3(POOLT_THREADS), smem, stream, pl[0].a, pl[0].b,
+                                          pl[0].p, pl[1].a, pl[1].b, pl[1].p, pl[2].a, pl[2].b, pl[2].p, pl[3].a, pl[3].b, pl[3].p);
+    if (rc != cudaSuccess) return SQN_ERR_CUDA;
+    note_launch();
+    return cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
 }
 
 // Host-only feasibility test of the fused max-pool for a layer (shared-memory budget, shape rules).

@@ -36,6 +36,7 @@ int launch_conv_bf16(const ConvDesc& d, cudaStream_t stream);
 // Two independent layers in one launch (first `big`'s CTAs, then `small`'s); SQN_ERR_UNSUPPORTED if they share no
 // kernel variant.
 int launch_conv_bf16_pair(const ConvDesc& small, const ConvDesc& big, cudaStream_t stream);
+int launch_conv_bf16_pool4(const ConvDesc* four, cudaStream_t stream);   // four pooled layers over one input, one launch
 bool conv_bf16_pool_fits(const ConvDesc& d);   // true when the layer can run with its max-pool fused (d.pool = 1)
 int launch_conv_bf16_uncached(const ConvDesc& d, cudaStream_t stream);   // no plan cache, no allocation
 // Stem (7x7/2 on 3 layers): needs scratch for the repacked input and kernels.
