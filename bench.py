@@ -28,7 +28,7 @@ from paper_1611_07151_b200 import synth
 IMG = 227
 # (launch, dtype, batch) -> dram__bytes_read.sum + dram__bytes_write.sum of one launch (profiles/conv_kernels_dram_bytes.md);
 # emptied whenever that kernel changes, refilled from a new capture
-NCU_TRAFFIC_BYTES = {("conv1+pool1", "bf16", 256): 206.9e6}
+NCU_TRAFFIC_BYTES = {("conv1+pool1", "bf16", 256): 205.2e6}
 METRIC = "squeezenet_v1.0_forward_images_per_s"
 UNIT = "images/s"
 
