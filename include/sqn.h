@@ -75,7 +75,7 @@ int conv_forward(const void* in, const void* weights, const void* bias, void* ou
  *   workspace_bytes  device scratch, needed only when conv_workspace_bytes reports > 0
  *   fuse_maxpool   the 3x3 / stride 2 max-pool that follows the layer (paper Section III-E) is applied inside the
  *                  kernel and only the pooled map is written: out is [batch][(outH-3)/2+1][(outW-3)/2+1][out_c_total].
- *                  SQN_BF16 only, stride 1 (or the stem shape), numOutputLayers a multiple of 32 up to 256, kernels
+ *                  SQN_BF16 only, stride 1 (or the stem shape), numOutputLayers a multiple of 32 up to 128, kernels
  *                  small enough to stay in shared memory; otherwise SQN_ERR_UNSUPPORTED.
  */
 typedef struct {
@@ -162,7 +162,8 @@ int maxpool3x3s2_forward(const void* in, void* out, int C, int H, int W, int bat
  *   logits[n][c] = mean over H*W of in[n][.][.][c]        (fp32)
  *   probs[n][c]  = exp(logits[n][c] - max_c) / sum_c exp(logits[n][c] - max_c)
  * in has dtype `dtype`; logits and probs are fp32 [batch][C]; probs may be NULL.
- * C <= 8192.
+ * C <= 8192 and batch <= 65535 (else SQN_ERR_UNSUPPORTED); in 16-byte aligned, logits and probs
+ * 4-byte aligned (else SQN_ERR_ALIGN).
  */
 int avgpool_softmax_forward(const void* in, void* logits_f32, void* probs_f32, int C, int H, int W, int batch,
                             int dtype, void* stream);
@@ -179,6 +180,9 @@ int avgpool_softmax_forward(const void* in, void* logits_f32, void* probs_f32, i
  *   network order (conv1; fireN squeeze, expand1x1, expand3x3 for N=2..9; conv10),
  *   kernels OHWI in `dtype`, bias fp32.  The net stores the pointers (the caller
  *   keeps the memory alive) and host-side launch plans; it holds no device memory.
+ *   The kernels and bias must be complete before squeezenet_forward is called: the
+ *   forward's launches may fetch them while earlier work on `stream` is still running
+ *   (conv_forward_ex and fire_forward make no such assumption).
  * squeezenet_workspace_bytes: device scratch one forward of `batch` images needs.
  * squeezenet_forward: in_nhwc [batch][227][227][3] in the net's dtype;
  *   logits_f32, probs_f32 fp32 [batch][1000] (probs may be NULL);

@@ -87,6 +87,7 @@ int make_conv_desc(const void* in, const void* w, const void* bias, void* out, i
     d->OH = out_extent(H, K, S, pad); d->OW = out_extent(W, K, S, pad);
     d->out_c_offset = c_off; d->out_c_total = c_total; d->relu = relu ? 1 : 0;
     d->pool = 0;
+    d->params_static = 0;
     return SQN_OK;
 }
 
@@ -219,8 +220,12 @@ extern "C" int fire_forward_static(const void* in, const void* w_sq, const void*
     if (dtype != SQN_F32 && dtype != SQN_BF16) return SQN_ERR_BADARG;
     if (e1 <= 0 || e3 <= 0 || s <= 0 || H <= 0 || W <= 0 || batch <= 0) return SQN_ERR_BADARG;
     // the squeeze map must fit the built-in scratch
-    const unsigned long long need = (unsigned long long)batch * H * W * s * esize(dtype);
-    if (need > kStaticFireScratchBytes) return SQN_ERR_WORKSPACE;
+    // (checked factor by factor: the product of four ints can wrap a 64-bit word)
+    unsigned long long need = esize(dtype);
+    for (const int f : {batch, H, W, s}) {
+        need *= (unsigned long long)f;
+        if (need > kStaticFireScratchBytes) return SQN_ERR_WORKSPACE;
+    }
     void* scratch = fire_static_scratch_ptr();
     if (!scratch) return SQN_ERR_CUDA;
     ConvDesc dsq, d1, d3;
@@ -256,7 +261,10 @@ extern "C" int avgpool_softmax_forward(const void* in, void* logits_f32, void* p
 {
     if (!in || !logits_f32 || C <= 0 || H <= 0 || W <= 0 || batch <= 0) return SQN_ERR_BADARG;
     if (dtype != SQN_F32 && dtype != SQN_BF16) return SQN_ERR_BADARG;
-    if (C > 8192) return SQN_ERR_UNSUPPORTED;
+    if (C > 8192 || batch > 65535) return SQN_ERR_UNSUPPORTED;       // (the image index is the grid's y dimension)
+    // the kernels read the map with 16-byte (bf16) or 8-byte (fp32) loads and the logits as floats
+    if (!aligned16(in) || (reinterpret_cast<uintptr_t>(logits_f32) & 3u) || (reinterpret_cast<uintptr_t>(probs_f32) & 3u))
+        return SQN_ERR_ALIGN;
     return launch_avgpool_softmax(in, static_cast<float*>(logits_f32), static_cast<float*>(probs_f32), C, H, W, batch,
                                   dtype, static_cast<cudaStream_t>(stream));
 }
@@ -497,6 +505,8 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
         rc = make_conv_desc(sq, net->w[3 + 3 * i], net->b[3 + 3 * i], out, f.s, f.e, f.hw, f.hw, 3, 1, 1, batch, 1, f.e,
                             2 * f.e, &d3);
         if (rc != SQN_OK) return rc;
+        // the net's kernels and bias are not written by anything this forward enqueues
+        dsq.params_static = d1.params_static = d3.params_static = 1;
         const std::string nm(f.name);
         if ((rc = run_conv(dsq, dt, nullptr, 0, st)) != SQN_OK) return rc;
         mark((nm + "_sq").c_str());
@@ -570,6 +580,7 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
     // conv10 1x1 + ReLU, global average, softmax
     rc = make_conv_desc(cur, net->w[25], net->b[25], buf("conv10"), 512, 1000, 13, 13, 1, 1, 0, batch, 1, 0, 0, &d);
     if (rc != SQN_OK) return rc;
+    d.params_static = 1;
     if ((rc = run_conv(d, dt, nullptr, 0, st)) != SQN_OK) return rc;
     mark("conv10");
     rc = launch_avgpool_softmax(buf("conv10"), static_cast<float*>(logits_f32), static_cast<float*>(probs_f32), 1000,

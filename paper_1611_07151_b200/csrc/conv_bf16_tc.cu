@@ -291,8 +291,8 @@ __device__ __forceinline__ void conv_tc_body(const CUtensorMap& tmA, const CUten
     // that grid drains.  Up to chain_wait() below it touches only its own shared memory, TMEM, the
     // kernel parameters and, when b_early is set, the layer's kernels and bias (which that grid does not
     // write): a CTA that starts in the tail of the layer before has its kernels resident by the time
-    // the first input tile may be read.
-    chain_release();
+    // the first input tile may be read.  The grid after this one is let go by warp 1 once this CTA
+    // holds its TMEM (see below).
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(smem_u32(&sh->full[s]), 1);
@@ -317,6 +317,10 @@ __device__ __forceinline__ void conv_tc_body(const CUtensorMap& tmA, const CUten
     if (warp == 1) {
         tmem_alloc(smem_u32(&sh->tmem_base), p.tmem_cols);
         tmem_relinquish();
+        // Only now may the next grid in the stream be scheduled: every CTA of a grid that has let its
+        // dependents go already holds its TMEM, so a CTA waiting in tcgen05.alloc can only be waiting for
+        // columns of grids that do not wait for it.
+        chain_release();
     }
     if (p.patch && !p.use_ptab) {
         // operand addresses of every MMA of a tile, in issue order (tap-major, then chunk, then k-step)
@@ -695,7 +699,6 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
     const int nmma = items * (p.BKc / 16);
     const int my_tiles = tiles_of_cta(p, bid);
 
-    chain_release();
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(smem_u32(&sh->full[s]), 1);
@@ -715,6 +718,10 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
     if (warp == 1) {
         tmem_alloc(smem_u32(&sh->tmem_base), p.tmem_cols);
         tmem_relinquish();
+        // Only now may the next grid in the stream be scheduled: every CTA of a grid that has let its
+        // dependents go already holds its TMEM, so a CTA waiting in tcgen05.alloc can only be waiting for
+        // columns of grids that do not wait for it.
+        chain_release();
     }
     {
         // tile of ones for the bias MMA: 256 rows of 32 bytes in the 32-byte swizzle, ones in the first two places
@@ -1218,7 +1225,7 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     p.bias = d.bias;
     p.status = device_status_word();
     p.h_mul = 1;
-    p.b_early = stem ? 0 : 1;
+    p.b_early = (!stem && d.params_static) ? 1 : 0;
     p.bias_in_k = stem ? 1 : 0;
     p.pool = d.pool ? 1 : 0;
     if (p.pool && (d.OH < 3 || d.OW < 3 || d.Cout % 32 != 0 || d.Cout > TILE_M)) return SQN_ERR_UNSUPPORTED;
@@ -1517,7 +1524,7 @@ int cached_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_p
     PlanKey k;
     std::memset(&k, 0, sizeof(k));
     k.in = d.in; k.w = d.w; k.bias = d.bias; k.out = d.out; k.ws = ws;
-    const int v[14] = {d.N, d.Cin, d.H, d.W, d.Cout, d.K, d.S, d.pad, d.out_c_offset, d.out_c_total, d.relu | (d.pool << 1),
+    const int v[14] = {d.N, d.Cin, d.H, d.W, d.Cout, d.K, d.S, d.pad, d.out_c_offset, d.out_c_total, d.relu | (d.pool << 1) | (d.params_static << 2),
                        (stem ? 1 : 0) | (force_halves << 4) | ((force_cw & 0xffff) << 8), Hp, Wp};
     std::memcpy(k.v, v, sizeof(v));
     int dev = 0;

@@ -18,6 +18,8 @@ struct ConvDesc {
     int N, Cin, H, W, Cout, K, S, pad, OH, OW;
     int out_c_offset, out_c_total, relu;
     int pool;             // 1: out receives the 3x3/stride-2 max-pool of the layer's output (bf16 path only)
+    int params_static;    // 1: kernels and bias are not written by earlier work on the stream (a net's own parameters), so
+                          //    a chained launch may fetch them before the kernel ahead of it has finished
 };
 
 // Launch counter (host side): every kernel launch goes through note_launch().

@@ -51,6 +51,13 @@ def test_bad_arguments_are_rejected_before_any_launch():
     assert l.conv_forward_ex(p, p, p, p, 3, 4, 8, 8, 3, 1, 1, 1, opts) == B.SQN_ERR_BADARG   # slice overruns
     assert l.maxpool3x3s2_forward(p, p, 8, 2, 8, 1, 0, None) == B.SQN_ERR_BADARG
     assert l.avgpool_softmax_forward(p, p, p, 10000, 2, 2, 1, 0, None) == B.SQN_ERR_UNSUPPORTED
+    assert l.avgpool_softmax_forward(p, p, p, 1000, 13, 13, 70000, 1, None) == B.SQN_ERR_UNSUPPORTED   # batch > 65535
+    assert l.avgpool_softmax_forward(p + 4, p, p, 1000, 13, 13, 1, 0, None) == B.SQN_ERR_ALIGN    # fp32 map, 4-byte aligned
+    assert l.avgpool_softmax_forward(p + 2, p, p, 1000, 13, 13, 1, 1, None) == B.SQN_ERR_ALIGN    # bf16 map, 2-byte aligned
+    assert l.avgpool_softmax_forward(p, p + 2, p, 1000, 13, 13, 1, 0, None) == B.SQN_ERR_ALIGN    # logits
+    assert l.avgpool_softmax_forward(p, p, p + 1, 1000, 13, 13, 1, 0, None) == B.SQN_ERR_ALIGN    # probs
+    # fire_forward_static: a squeeze map whose byte count wraps 64 bits is refused like any other that is too large
+    assert l.fire_forward_static(p, p, p, p, p, p, p, p, 16, 65536, 16, 16, 65536, 65536, 65536, 0, None) == B.SQN_ERR_WORKSPACE
     assert l.fire_forward(p, p, p, p, p, p, p, None, p, 8, 4, 8, 8, 5, 5, 1, 0, None) == B.SQN_ERR_BADARG
     assert B.sqn_launch_count() == n0
 

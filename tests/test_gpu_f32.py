@@ -129,7 +129,13 @@ def test_config1_fire4():
     assert G.rel_err(got[:, 128:], exp[:, 128:]) <= TOL
 
 
-def run_net(x, params, dtype, batch):
+LAYER_NAMES = ["conv1", "pool1"] + ["fire%d%s" % (i, s) for i in range(2, 10) for s in ("_sq", "")] + \
+    ["pool4", "pool8", "conv10"]
+
+
+def run_net_device(x, params, dtype, batch):
+    """One forward through squeezenet_forward.  Returns (logits, probs, {layer name: device view [batch][H][W][C]});
+    the views alias the forward's workspace (kept alive by them)."""
     import torch
     names = [n for n, *_ in synth.SQUEEZENET_CONVS]
     ws = [G.dev_w(params[n][0], dtype) for n in names]
@@ -141,9 +147,8 @@ def run_net(x, params, dtype, batch):
     probs = torch.empty((batch, 1000), device="cuda")
     B.squeezenet_forward(net, G.dev_act(x, dtype), logits, probs, work, batch)
     assert B.sqn_check() == B.SQN_OK
-    layers = {}
-    for name in ["conv1", "pool1"] + ["fire%d%s" % (i, s) for i in range(2, 10) for s in ("_sq", "")] + \
-            ["pool4", "pool8", "conv10"]:
+    views = {}
+    for name in LAYER_NAMES:
         try:
             ptr, C, H, W = B.squeezenet_layer_output(net, name, work, batch)
         except B.SqnError as e:          # a layer the net fused away (bf16: conv1 lives inside conv1+pool1)
@@ -152,10 +157,14 @@ def run_net(x, params, dtype, batch):
         off = ptr - work.data_ptr()
         es = 4 if dtype == F32 else 2
         raw = work[off:off + batch * C * H * W * es]
-        t = raw.view(torch.float32 if dtype == F32 else torch.bfloat16).view(batch, H, W, C)
-        layers[name] = G.host_act(t, dtype)
+        views[name] = raw.view(torch.float32 if dtype == F32 else torch.bfloat16).view(batch, H, W, C)
     B.squeezenet_destroy(net)
-    return logits.cpu().numpy(), probs.cpu().numpy(), layers
+    return logits.cpu().numpy(), probs.cpu().numpy(), views
+
+
+def run_net(x, params, dtype, batch):
+    logits, probs, views = run_net_device(x, params, dtype, batch)
+    return logits, probs, {name: G.host_act(t, dtype) for name, t in views.items()}
 
 
 def test_config2_full_forward_batch1():

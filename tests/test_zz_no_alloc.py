@@ -9,6 +9,7 @@ already run every other test."""
 import numpy as np
 import pytest
 
+from oracle import ref
 from paper_1611_07151_b200 import binding as B
 from paper_1611_07151_b200 import synth
 import gpu_util as G
@@ -31,6 +32,9 @@ def _run_both(seed, batch, cin, s, e, hw, dtype):
     a, b = G.host_act(ref_out, dtype), G.host_act(new_out, dtype)
     assert not np.isnan(b).any()
     assert G.rel_err(b, a) <= G.TOL[dtype]
+    exp = ref.fire(x, *sq, *e1, *e3)                        # and against the oracle, each expand on its own scale
+    assert G.rel_err(b[:, :e], exp[:, :e]) <= G.TOL[dtype]
+    assert G.rel_err(b[:, e:], exp[:, e:]) <= G.TOL[dtype]
     return b
 
 
@@ -49,3 +53,27 @@ def test_request_beyond_the_built_in_buffer_is_refused():
         B.fire_forward_static(p, p, p, p, p, p, p, p, 128, 32, 128, 128, 55, 55, 64, B.SQN_F32)   # 24.8 MB squeeze map
     assert e.value.status == B.SQN_ERR_WORKSPACE
     assert B.sqn_launch_count() == n0
+
+
+def test_calls_leave_the_free_device_memory_unchanged():
+    """The point of the entry point: after a first call on the device (which looks up the built-in buffer's address)
+    further calls, in either dtype, take no device memory."""
+    import torch
+    cases = []
+    for dtype in (B.SQN_F32, B.SQN_BF16):
+        x, sq, e1, e3 = synth.fire_case(5, 2, 64, 16, 64, 64, 13)
+        dev = [G.dev_act(x, dtype), G.dev_w(sq[0], dtype), G.dev_b(sq[1]), G.dev_w(e1[0], dtype), G.dev_b(e1[1]),
+               G.dev_w(e3[0], dtype), G.dev_b(e3[1])]
+        cases.append((dev, B.empty_device((2, 13, 13, 128), dtype), dtype))
+    for dev, out, dtype in cases:                          # first calls: address look-up, kernel images loaded
+        B.fire_forward_static(*dev, out, 64, 16, 64, 64, 13, 13, 2, dtype)
+    assert B.sqn_check() == B.SQN_OK
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for _ in range(3):
+        for dev, out, dtype in cases:
+            B.fire_forward_static(*dev, out, 64, 16, 64, 64, 13, 13, 2, dtype)
+    assert B.sqn_check() == B.SQN_OK
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
