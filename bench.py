@@ -26,9 +26,24 @@ from paper_1611_07151_b200 import dist as D
 from paper_1611_07151_b200 import synth
 
 IMG = 227
-# (launch, dtype, batch) -> dram__bytes_read.sum + dram__bytes_write.sum of one launch (profiles/conv_kernels_dram_bytes.md);
-# emptied whenever that kernel changes, refilled from a new capture
-NCU_TRAFFIC_BYTES = {("conv1+pool1", "bf16", 256): 205.2e6}
+TRAFFIC_TABLE = os.path.join(ROOT, "profiles", "dram_bytes_per_launch.txt")
+
+
+def ncu_traffic_bytes(launch, dtype, batch):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the committed table of single-pass ncu
+    captures (lines: launch dtype batch bytes); None when the table has no line for this launch and configuration."""
+    try:
+        with open(TRAFFIC_TABLE) as f:
+            for line in f:
+                parts = line.split()
+                if len(parts) >= 4 and not line.startswith("#") and parts[0] == launch and parts[1] == dtype \
+                        and int(parts[2]) == batch:
+                    return float(parts[3])
+    except OSError:
+        pass
+    return None
+
+
 METRIC = "squeezenet_v1.0_forward_images_per_s"
 UNIT = "images/s"
 
@@ -89,7 +104,7 @@ def launch_work(batch, es):
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs (read only)."""
 
-    def __init__(self, index, period=0.02):
+    def __init__(self, index, period=0.002):
         super().__init__(daemon=True)
         self.index, self.period = index, period
         self.samples, self.reasons, self.max_mhz = [], set(), None
@@ -186,16 +201,18 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
-def run_batch1(B, ws, bs, x_pinned, dtype, dev, iters=300):
-    """The paper's own regime: one image at a time.  Launch-latency bound (all tensors sit in L2); timed
-    as back-to-back launches and as replays of a CUDA graph captured around the same call."""
+def run_batch1(B, ws, bs, x1, dtype, dev, prepacked=False, iters=300):
+    """The paper's own regime: one image at a time.  Launch-latency bound; timed hot (back-to-back launches, and
+    replays of a CUDA graph captured around the same call: every tensor stays in the L2) and cold (the L2 is
+    overwritten before every forward, one forward per event pair, median and mean)."""
     import torch
     net1 = B.squeezenet_create(ws, bs, dtype, 1)
+    if prepacked:
+        B.squeezenet_set_stem_prepacked(net1, True)
     work = torch.empty(B.squeezenet_workspace_bytes(net1, 1), dtype=torch.uint8, device=dev)
-    x1 = x_pinned[:1].to(dev)
     logits = torch.empty((1, 1000), dtype=torch.float32, device=dev)
     probs = torch.empty((1, 1000), dtype=torch.float32, device=dev)
-    out = {"note": "batch 1, inputs and activations resident in L2 (hot)"}
+    out = {"note": "batch 1; hot = inputs and activations resident in L2, cold = L2 overwritten before each forward"}
     for _ in range(5):
         B.squeezenet_forward(net1, x1, logits, probs, work, 1)
     torch.cuda.synchronize()
@@ -207,6 +224,18 @@ def run_batch1(B, ws, bs, x_pinned, dtype, dev, iters=300):
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / iters
     out["eager"] = {"images_per_s": 1e3 / ms, "latency_us": ms * 1e3}
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    cold = []
+    for _ in range(40):
+        flush.zero_()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        B.squeezenet_forward(net1, x1, logits, probs, work, 1)
+        b.record()
+        torch.cuda.synchronize()
+        cold.append(a.elapsed_time(b) * 1e3)
+    out["cold"] = {"latency_us_median": float(np.median(cold)), "latency_us_mean": float(np.mean(cold)), "forwards": len(cold)}
+    del flush
     try:
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
@@ -232,6 +261,48 @@ def run_batch1(B, ws, bs, x_pinned, dtype, dev, iters=300):
     assert B.sqn_check() == B.SQN_OK
     B.squeezenet_destroy(net1)
     return out
+
+
+def layer_table(B, net, step, steps, batch, es, dtype_tag, peaks, sm_count, sm_mhz, stream):
+    """Per-launch times of `steps` forwards (CUDA events recorded by the library on the launching stream) -> one
+    record per launch with its algorithmic work, its bound and the achieved fraction of it.  bf16 fractions are
+    against the burst tensor peak (`frac`; a launch lasts tens of microseconds) with the sustained figure beside
+    it; HBM fractions against the measured copy bandwidth with the nominal 8 TB/s beside it."""
+    import torch
+    B.squeezenet_profile(net, steps)
+    pe0, pe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    pe0.record(stream)
+    for i in range(steps):
+        step(i)
+    pe1.record(stream)
+    torch.cuda.synchronize()
+    ms_step = pe0.elapsed_time(pe1) / steps
+    lnames, lms, nfwd = B.squeezenet_profile_read(net)
+    B.squeezenet_profile(net, 0)
+    bf16 = dtype_tag == "bf16"
+    pipe = peaks["bf16_tflops"] if bf16 else fp32_ffma_peak_tflops(sm_count, sm_mhz)
+    pipe_sus = peaks["bf16_tflops_sustained"] if bf16 else pipe
+    work = launch_work(batch, es)
+    layers = []
+    total_ms = sum(lms) / max(nfwd, 1)
+    for n, ms_sum in zip(lnames, lms):
+        ms = ms_sum / max(nfwd, 1)
+        w = work.get(n, {"flops": 0.0, "bytes": 0.0})
+        t_hbm = w["bytes"] / (peaks["hbm_gbs"] * 1e9)
+        t_pipe = w["flops"] / (pipe * 1e12)
+        bound = "hbm" if t_hbm >= t_pipe else ("tensor" if bf16 else "alu")
+        rec = {"name": n, "ms": ms, "share": ms / total_ms if total_ms else 0.0, "bound": bound,
+               "gbs": w["bytes"] / (ms * 1e-3) / 1e9 if ms > 0 else 0.0,
+               "tflops": w["flops"] / (ms * 1e-3) / 1e12 if ms > 0 else 0.0,
+               "frac": max(t_hbm, t_pipe) / (ms * 1e-3) if ms > 0 else 0.0,
+               "bytes": w["bytes"], "flops": w["flops"]}
+        if bound == "hbm":
+            rec["frac_nominal_8tbs"] = rec["gbs"] / 8000.0
+        elif bf16:
+            rec["frac_sustained"] = rec["tflops"] / pipe_sus
+        rec["meets_60pct"] = bool(rec["frac"] >= 0.6)
+        layers.append(rec)
+    return layers, ms_step, pipe, pipe_sus
 
 
 def run_sweep(B):
@@ -397,22 +468,38 @@ def main():
     dtype = B.SQN_BF16 if args.dtype == "bf16" else B.SQN_F32
     es = 2 if dtype == B.SQN_BF16 else 4
     batch = args.batch
+    bf16 = dtype == B.SQN_BF16
 
     # ---- synthetic workload: U[0,1) images, He-normal kernels, N(0,.01) bias (seed 3 + rank)
     x, params = synth.squeezenet_case(3 + rank, batch)
     names = [n for n, *_ in synth.SQUEEZENET_CONVS]
     ws = [B.to_device(B.sqn_pack_weights_oihw_to_ohwi(params[n][0], dtype), dtype) for n in names]
     bs = [B.to_device(np.ascontiguousarray(params[n][1], dtype=np.float32)) for n in names]
-    x_host = B.sqn_pack_nchw_to_nhwc(x, dtype)
-    del x
-    host_t = torch.from_numpy(x_host)
-    if dtype == B.SQN_BF16:
-        host_t = host_t.view(torch.int16).view(torch.bfloat16)
-    x_pinned = host_t.pin_memory()
-    inputs = [x_pinned.to(dev), torch.flip(x_pinned, dims=[0]).contiguous().to(dev)]   # rotated between steps
 
-    net = B.squeezenet_create(ws, bs, dtype, batch)
-    work_bytes = B.squeezenet_host_workspace_bytes(net, batch)
+    def pinned(a):
+        t = torch.from_numpy(a)
+        if bf16:
+            t = t.view(torch.int16).view(torch.bfloat16)
+        return t.pin_memory()
+
+    x_pinned = pinned(B.sqn_pack_nchw_to_nhwc(x, dtype))              # [batch][227][227][3]: what a user's loader holds
+    # Device-resident run: the bf16 stem reads operands reordered offline (input [batch][228][228][4], conv1's
+    # kernels [96][7][8][4] with the bias folded in), so the forward launches no repack pass.
+    if bf16:
+        ws_dev = list(ws)
+        ws_dev[0] = B.to_device(B.sqn_pack_stem_weights(*params["conv1"]), dtype)
+        x_dev_host = pinned(B.sqn_pack_stem_input(x))
+    else:
+        ws_dev, x_dev_host = ws, x_pinned
+    x32_one = np.ascontiguousarray(x[:1])
+    del x
+    inputs = [x_dev_host.to(dev), torch.flip(x_dev_host, dims=[0]).contiguous().to(dev)]   # rotated between steps
+
+    net = B.squeezenet_create(ws_dev, bs, dtype, batch)
+    if bf16:
+        B.squeezenet_set_stem_prepacked(net, True)
+    net_host = B.squeezenet_create(ws, bs, dtype, batch)            # host-buffer path: 3-layer images as they are
+    work_bytes = B.squeezenet_host_workspace_bytes(net_host, batch)
     workspace = torch.empty(work_bytes, dtype=torch.uint8, device=dev)
     logits = torch.empty((batch, 1000), dtype=torch.float32, device=dev)
     probs = torch.empty((batch, 1000), dtype=torch.float32, device=dev)
@@ -438,63 +525,51 @@ def main():
     ev1.record(stream)
     torch.cuda.synchronize()
     D.barrier()
-    clocks = sampler.stop()
     gpu_launches = B.sqn_launch_count() - launches0
     ms_local = ev0.elapsed_time(ev1)
     status = B.sqn_check()
     assert status == B.SQN_OK, B.sqn_status_string(status)
     value, ms_total = D.job_throughput(batch * args.steps, ms_local, dev)
 
+    # ---- the same steps once more with an event after every step: median beside the mean
+    n_med = min(args.steps, 200)
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(n_med + 1)]
+    evs[0].record(stream)
+    for i in range(n_med):
+        step(i)
+        evs[i + 1].record(stream)
+    torch.cuda.synchronize()
+    per_step = [evs[i].elapsed_time(evs[i + 1]) for i in range(n_med)]
+
     # ---- per-launch times -> per-layer roofline.  One CUDA event per launch keeps a chained launch from starting
     # in the tail of the one before it (12 % on the whole forward at batch 256), so the events are recorded in a
-    # second pass over the same steps, directly after the timed region, and the timed region itself runs without.
-    prof_steps = min(args.steps, 256)
-    B.squeezenet_profile(net, prof_steps)
-    pe0, pe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    pe0.record(stream)
-    for i in range(prof_steps):
-        step(i)
-    pe1.record(stream)
-    torch.cuda.synchronize()
-    ms_step_with_events = pe0.elapsed_time(pe1) / prof_steps
-    lnames, lms, nfwd = B.squeezenet_profile_read(net)
-    B.squeezenet_profile(net, 0)
+    # further pass over the same steps and the timed region itself runs without.  The clock sampler runs across it.
     peaks = measured_peaks()
     props = torch.cuda.get_device_properties(local_rank)
-    sm_mhz = clocks["sm_mhz"] or clocks["sm_max_mhz"] or 1965
-    pipe_tf = peaks["bf16_tflops_sustained"] if dtype == B.SQN_BF16 else fp32_ffma_peak_tflops(
-        props.multi_processor_count, sm_mhz)
-    work = launch_work(batch, es)
-    layers = []
-    total_ms = sum(lms) / max(nfwd, 1)
-    for n, ms_sum in zip(lnames, lms):
-        ms = ms_sum / max(nfwd, 1)
-        w = work.get(n, {"flops": 0.0, "bytes": 0.0})
-        t_hbm = w["bytes"] / (peaks["hbm_gbs"] * 1e9)
-        t_pipe = w["flops"] / (pipe_tf * 1e12)
-        bound = "hbm" if t_hbm >= t_pipe else ("tensor" if dtype == B.SQN_BF16 else "alu")
-        layers.append({"name": n, "ms": ms, "share": ms / total_ms if total_ms else 0.0, "bound": bound,
-                       "gbs": w["bytes"] / (ms * 1e-3) / 1e9 if ms > 0 else 0.0,
-                       "tflops": w["flops"] / (ms * 1e-3) / 1e12 if ms > 0 else 0.0,
-                       "frac": max(t_hbm, t_pipe) / (ms * 1e-3) if ms > 0 else 0.0,
-                       "bytes": w["bytes"], "flops": w["flops"]})
+    prof_steps = min(args.steps, 256)
+    layers, ms_step_with_events, pipe_tf, pipe_sus = layer_table(
+        B, net, step, prof_steps, batch, es, args.dtype, peaks, props.multi_processor_count, 1965.0, stream)
+    clocks = sampler.stop()
     top = max(layers, key=lambda l: l["ms"])
     if top["bound"] == "hbm":
-        roof = {"bound": "hbm", "achieved": top["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+        roof = {"bound": "hbm", "achieved": top["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac_nominal_8tbs": top["gbs"] / 8000.0}
     else:
         roof = {"bound": top["bound"], "achieved": top["tflops"], "peak": pipe_tf, "unit": "TFLOP/s"}
+        if bf16:
+            roof["peak_kind"] = ("burst (a launch lasts %.0f us at full clocks); sustained peak %.1f beside it"
+                                 % (top["ms"] * 1e3, pipe_sus))
+            roof["frac_sustained"] = top["tflops"] / pipe_sus
     roof["frac"] = roof["achieved"] / roof["peak"]
-    # dram__bytes_read.sum + dram__bytes_write.sum per launch from the single-pass ncu capture summarised in
-    # profiles/conv_kernels_dram_bytes.md; None for any launch or configuration that capture does not cover
-    roof["traffic"] = NCU_TRAFFIC_BYTES.get((top["name"], args.dtype, batch))
-    kname = "conv_f32_kernel" if dtype != B.SQN_BF16 else ("conv_pool_kernel" if "+pool" in top["name"] else "conv_tc_kernel")
+    roof["traffic"] = ncu_traffic_bytes(top["name"], args.dtype, batch)
+    kname = "conv_f32_kernel" if not bf16 else ("conv_pool_kernel" if "+pool" in top["name"] else "conv_tc_kernel")
     if "_e1+e3" in top["name"]:
         kname += "2"
     roof["kernel"] = kname + "[%s]" % top["name"]
     roof["peak_source"] = "of " + peaks["source"]
     roof["launch_ms"] = top["ms"]
     roof["share_of_step"] = top["share"]
-    roof["timing"] = ("CUDA events around every launch, %d steps run directly after the timed region; with the events "
+    roof["timing"] = ("CUDA events around every launch, %d steps run after the timed region; with the events "
                       "a step takes %.4f ms (launches no longer overlap the tail of the one before)"
                       % (prof_steps, ms_step_with_events))
     sum_bound_ms = sum(l["frac"] * l["ms"] for l in layers)
@@ -504,13 +579,13 @@ def main():
     e2e_steps = args.e2e_steps or min(args.steps, 50)
     out_host = torch.empty((2, batch, 1000), dtype=torch.float32).pin_memory()
     for i in range(3):
-        B.squeezenet_forward_host(net, x_pinned, out_host[0], out_host[1], workspace, batch)
+        B.squeezenet_forward_host(net_host, x_pinned, out_host[0], out_host[1], workspace, batch)
     torch.cuda.synchronize()
     D.barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for i in range(e2e_steps):
-        B.squeezenet_forward_host(net, x_pinned, out_host[0], out_host[1], workspace, batch)
+        B.squeezenet_forward_host(net_host, x_pinned, out_host[0], out_host[1], workspace, batch)
     e1.record(stream)
     torch.cuda.synchronize()
     D.barrier()
@@ -518,43 +593,86 @@ def main():
     h2d = batch * IMG * IMG * 3 * es
     d2h = 2 * batch * 1000 * 4
     assert abs(float(out_host[1].sum()) - batch) < 1e-2 * batch     # probabilities came back
+    # the host-buffer forward and the device-resident one classify the batch alike
+    step(0)
+    torch.cuda.synchronize()
+    same_top1 = float((out_host[0].argmax(1) == logits.cpu().argmax(1)).float().mean())
 
     batch1 = None
+    f32_record = None
     if rank == 0 and world == 1 and not args.no_batch1:
-        batch1 = run_batch1(B, ws, bs, x_pinned, dtype, dev)
-        if dtype == B.SQN_BF16:
-            # the exact path at batch 1 (fp32 storage and FFMA arithmetic): the same kernels packed as fp32
+        batch1 = run_batch1(B, ws_dev, bs, inputs[0][:1].contiguous(), dtype, dev, prepacked=bf16)
+        if bf16:
+            # the exact path (fp32 storage and FFMA arithmetic): the same kernels packed as fp32
             ws32 = [B.to_device(B.sqn_pack_weights_oihw_to_ohwi(params[n][0], B.SQN_F32), B.SQN_F32) for n in names]
-            x32 = x_pinned[:1].float().pin_memory()
+            x32 = B.to_device(B.sqn_pack_nchw_to_nhwc(x32_one, B.SQN_F32), B.SQN_F32)
             batch1["f32"] = run_batch1(B, ws32, bs, x32, B.SQN_F32, dev)
-            del ws32
+            # ... and at the bench's batch: images/s and the per-launch fractions of the FP32 pipe peak
+            fb = min(batch, 256)
+            net32 = B.squeezenet_create(ws32, bs, B.SQN_F32, fb)
+            work32 = torch.empty(B.squeezenet_workspace_bytes(net32, fb), dtype=torch.uint8, device=dev)
+            xin32 = inputs[0][:fb, :IMG, :IMG, :3].float().contiguous()
+
+            def step32(i):
+                B.squeezenet_forward(net32, xin32, logits[:fb], probs[:fb], work32, fb)
+            for i in range(3):
+                step32(i)
+            torch.cuda.synchronize()
+            n32 = 10
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for i in range(n32):
+                step32(i)
+            b.record(stream)
+            torch.cuda.synchronize()
+            ms32 = a.elapsed_time(b) / n32
+            l32, _, pipe32, _ = layer_table(B, net32, step32, n32, fb, 4, "f32", peaks, props.multi_processor_count,
+                                            clocks["sm_mhz"] or 1965.0, stream)
+            f32_record = {"images_per_s": fb / (ms32 * 1e-3), "ms_per_step": ms32, "batch": fb, "steps": n32,
+                          "ffma_peak_tflops": pipe32,
+                          "layers": [{"name": l["name"], "ms": round(l["ms"], 6), "bound": l["bound"],
+                                      "frac": round(l["frac"], 4), "meets_60pct": l["meets_60pct"]} for l in l32]}
+            assert B.sqn_check() == B.SQN_OK
+            B.squeezenet_destroy(net32)
+            del ws32, work32, xin32
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import ref
         v1, cores = oracle_images_per_s(1, 3)
         n = int(min(64, max(2, 15.0 * v1)))
         v, cores = oracle_images_per_s(n, 3)
+        ref.set_threads(1)
+        v_single, _ = oracle_images_per_s(1, 3)
+        ref.set_threads(cores)
         cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": "%d of the %d images of one batch, full network, double accumulation" % (n, batch)}
+               "sample": "%d of the %d images of one batch, full network, double accumulation" % (n, batch),
+               "single_thread_images_per_s": v_single}
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+                "warmup": args.warmup, "ms_per_step": ms_total / args.steps,
+                "ms_per_step_median": float(np.median(per_step)), "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": args.dtype, "data": "synthetic",
                 "config": {"workload": workload_name(args), "batch_per_gpu": batch, "global_batch": batch * world,
                            "image": "227x227x3", "parallelism": "replicas, batch sharded by image, no collective",
+                           "input_layout": ("device-resident run: stem operands reordered offline ([228][228][4] images, "
+                                            "[96][7][8][4] kernels); e2e: [227][227][3] images, repacked on the device")
+                           if bf16 else "[227][227][3]",
                            "l2": "per-step activations (%.1f GB) exceed the 126 MB L2; two input batches alternate"
                                  % (B.squeezenet_workspace_bytes(net, batch) / 1e9)},
                 "clocks": clocks,
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                        "steps": e2e_steps},
+                        "steps": e2e_steps, "top1_same_as_device_resident": same_top1},
                 "gpu_launches": int(gpu_launches),
                 "roofline": roof,
                 "cpu_baseline": cpu,
                 "batch1": batch1,
+                "f32": f32_record,
                 "layers": [{k: (round(v, 6) if isinstance(v, float) else v) for k, v in l.items()} for l in layers]}
         print(json.dumps(line), flush=True)
     B.squeezenet_destroy(net)
+    B.squeezenet_destroy(net_host)
 
 
 if __name__ == "__main__":

@@ -205,6 +205,25 @@ int squeezenet_layer_output(const sqn_net* net, const char* name, void* workspac
 int squeezenet_destroy(sqn_net* net);
 
 /*
+ * Stem operands reordered offline (the paper, Section III-C, reorders the model file once so that no
+ * layer repacks data at run time; here the same is done for the one layer whose operands the tensor
+ * cores cannot read as they are: conv1, 7x7 / stride 2 on 3 input layers, bf16).
+ * squeezenet_set_stem_prepacked(net, 1) (bf16 nets only, else SQN_ERR_UNSUPPORTED) declares that
+ *   - squeezenet_forward's input is [batch][Hp][Wp][4] bf16 as written by sqn_pack_stem_input
+ *     (Hp, Wp from sqn_stem_packed_extent(227, 227): 228 x 228; the fourth layer of every image pixel
+ *     holds 1.0, padding rows and columns are zero), and
+ *   - the net's first kernel pointer (weights26[0]) is [96][7][8][4] bf16 as written by
+ *     sqn_pack_stem_weights, which folds conv1's bias into two unused places; bias26[0] is then not read.
+ * The forward then launches no repack kernel.  squeezenet_forward_host copies such an input as it is.
+ * The three helpers take HOST pointers: src [N][3][H][W] fp32 (the oracle's order), kernels [O][3][7][7]
+ * fp32, bias [O] fp32; dst must hold N*Hp*Wp*4, respectively O*224, 16-bit words.
+ */
+int squeezenet_set_stem_prepacked(sqn_net* net, int on);
+int sqn_stem_packed_extent(int H, int W, int* Hp, int* Wp);
+int sqn_pack_stem_input(const float* src, void* dst, int N, int H, int W);
+int sqn_pack_stem_weights(const float* src, const float* bias, void* dst, int O);
+
+/*
  * The same forward with HOST input and output buffers (the call a user with data in host
  * memory makes): copy of in_host [batch][227][227][3] (net dtype) to the device, the forward,
  * copies of logits (and probs, unless NULL) [batch][1000] fp32 back to the host.  The copies

@@ -48,6 +48,10 @@ SIGNATURES = {
     "squeezenet_layer_output": (_c_int, [_c_vp, ctypes.c_char_p, _c_vp, _c_int, ctypes.POINTER(_c_vp),
                                          ctypes.POINTER(_c_int), ctypes.POINTER(_c_int), ctypes.POINTER(_c_int)]),
     "squeezenet_destroy": (_c_int, [_c_vp]),
+    "squeezenet_set_stem_prepacked": (_c_int, [_c_vp, _c_int]),
+    "sqn_stem_packed_extent": (_c_int, [_c_int, _c_int, ctypes.POINTER(_c_int), ctypes.POINTER(_c_int)]),
+    "sqn_pack_stem_input": (_c_int, [_c_vp, _c_vp, _c_int, _c_int, _c_int]),
+    "sqn_pack_stem_weights": (_c_int, [_c_vp, _c_vp, _c_vp, _c_int]),
     "squeezenet_host_workspace_bytes": (_c_int, [_c_vp, _c_int, ctypes.POINTER(_c_sz)]),
     "squeezenet_forward_host": (_c_int, [_c_vp] * 5 + [_c_int, _c_vp]),
     "squeezenet_profile": (_c_int, [_c_vp, _c_int]),
@@ -191,6 +195,38 @@ def squeezenet_layer_output(net, name, workspace, batch):
 
 def squeezenet_destroy(net):
     _check(lib().squeezenet_destroy(net), "squeezenet_destroy")
+
+
+def squeezenet_set_stem_prepacked(net, on=True):
+    _check(lib().squeezenet_set_stem_prepacked(net, 1 if on else 0), "squeezenet_set_stem_prepacked")
+
+
+def sqn_stem_packed_extent(H, W):
+    hp, wp = _c_int(0), _c_int(0)
+    _check(lib().sqn_stem_packed_extent(H, W, ctypes.byref(hp), ctypes.byref(wp)), "sqn_stem_packed_extent")
+    return hp.value, wp.value
+
+
+def sqn_pack_stem_input(src):
+    """[N][3][H][W] float32 -> [N][Hp][Wp][4] bf16 words (the layout the bf16 stem kernel reads)."""
+    src = np.ascontiguousarray(src, dtype=np.float32)
+    N, C, H, W = src.shape
+    assert C == 3
+    hp, wp = sqn_stem_packed_extent(H, W)
+    dst = np.empty((N, hp, wp, 4), dtype=np.uint16)
+    _check(lib().sqn_pack_stem_input(src.ctypes.data, dst.ctypes.data, N, H, W), "sqn_pack_stem_input")
+    return dst
+
+
+def sqn_pack_stem_weights(src, bias):
+    """[O][3][7][7] float32 kernels and [O] bias -> [O][7][8][4] bf16 words with the bias folded in."""
+    src = np.ascontiguousarray(src, dtype=np.float32)
+    bias = np.ascontiguousarray(bias, dtype=np.float32)
+    O = src.shape[0]
+    assert src.shape == (O, 3, 7, 7) and bias.shape == (O,)
+    dst = np.empty((O, 7, 8, 4), dtype=np.uint16)
+    _check(lib().sqn_pack_stem_weights(src.ctypes.data, bias.ctypes.data, dst.ctypes.data, O), "sqn_pack_stem_weights")
+    return dst
 
 
 def squeezenet_host_workspace_bytes(net, batch):

@@ -88,6 +88,7 @@ int make_conv_desc(const void* in, const void* w, const void* bias, void* out, i
     d->out_c_offset = c_off; d->out_c_total = c_total; d->relu = relu ? 1 : 0;
     d->pool = 0;
     d->params_static = 0;
+    d->stem_prepacked = 0;
     return SQN_OK;
 }
 
@@ -300,6 +301,7 @@ struct sqn_net {
     cudaEvent_t in_free[2] = {nullptr, nullptr};    // the forward that read staging buffer b has finished
     int copy_device = -1;
     unsigned long long host_calls = 0;
+    int stem_prepacked = 0;     // squeezenet_set_stem_prepacked
 };
 
 namespace {
@@ -334,6 +336,13 @@ size_t layout(const sqn_net* net, int batch, std::vector<size_t>* offs, size_t* 
     if (stem_off) *stem_off = cur;
     if (net->dtype == SQN_BF16) cur = align_up(cur + stem_bf16_workspace_bytes(batch, IMG, IMG, 96), 1024);
     return cur;
+}
+
+// Bytes of one input batch in the layout the net reads.
+size_t input_bytes(const sqn_net* net, int batch)
+{
+    if (net->stem_prepacked) return (size_t)batch * stem_packed_rows(IMG) * stem_packed_cols(IMG) * 4 * 2;
+    return (size_t)batch * IMG * IMG * 3 * esize(net->dtype);
 }
 
 int find_slot(const sqn_net* net, const char* name)
@@ -387,6 +396,14 @@ extern "C" int squeezenet_destroy(sqn_net* net)
         free_copy_pipeline(net);
     }
     delete net;
+    return SQN_OK;
+}
+
+extern "C" int squeezenet_set_stem_prepacked(sqn_net* net, int on)
+{
+    if (!net) return SQN_ERR_BADARG;
+    if (net->dtype != SQN_BF16) return on ? SQN_ERR_UNSUPPORTED : SQN_OK;
+    net->stem_prepacked = on ? 1 : 0;
     return SQN_OK;
 }
 
@@ -466,22 +483,30 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
     // The fused conv+pool kernels hand a whole strip of 16 output rows to one CTA: worth it once there are
     // enough strips to fill the GPU (8 per image for conv1, 4 for fire4), i.e. from a batch of 16 on.
     const bool fuse_pools = dt == SQN_BF16 && batch >= 16;
+    // bf16 stem: on operands packed offline (squeezenet_set_stem_prepacked), else after a repack pass
+    auto stem_bf16 = [&](ConvDesc& sd) -> int {
+        sd.params_static = 1;
+        if (net->stem_prepacked) {
+            sd.stem_prepacked = 1;
+            return launch_stem_conv_bf16_prepacked(sd, st);
+        }
+        const int prc = launch_stem_pack_bf16(sd, ws + stem_off, total - stem_off, st);
+        if (prc != SQN_OK) return prc;
+        mark("conv1_pack");
+        return launch_stem_conv_bf16(sd, ws + stem_off, total - stem_off, st);
+    };
     if (fuse_pools) {
         // stem and its max-pool in one kernel: the 96x111x111 map never goes to memory
         rc = make_conv_desc(in_nhwc, net->w[0], net->b[0], buf("pool1"), 3, 96, IMG, IMG, 7, 2, 0, batch, 1, 0, 0, &d);
         if (rc != SQN_OK) return rc;
         d.pool = 1;
-        if ((rc = launch_stem_pack_bf16(d, ws + stem_off, total - stem_off, st)) != SQN_OK) return rc;
-        mark("conv1_pack");
-        if ((rc = launch_stem_conv_bf16(d, ws + stem_off, total - stem_off, st)) != SQN_OK) return rc;
+        if ((rc = stem_bf16(d)) != SQN_OK) return rc;
         mark("conv1+pool1");
     } else {
         rc = make_conv_desc(in_nhwc, net->w[0], net->b[0], buf("conv1"), 3, 96, IMG, IMG, 7, 2, 0, batch, 1, 0, 0, &d);
         if (rc != SQN_OK) return rc;
         if (dt == SQN_BF16) {
-            if ((rc = launch_stem_pack_bf16(d, ws + stem_off, total - stem_off, st)) != SQN_OK) return rc;
-            mark("conv1_pack");
-            if ((rc = launch_stem_conv_bf16(d, ws + stem_off, total - stem_off, st)) != SQN_OK) return rc;
+            if ((rc = stem_bf16(d)) != SQN_OK) return rc;
         } else {
             if ((rc = launch_conv_f32(d, st)) != SQN_OK) return rc;
         }
@@ -594,7 +619,7 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
 extern "C" int squeezenet_host_workspace_bytes(const sqn_net* net, int batch, size_t* bytes)
 {
     if (!net || !bytes || batch <= 0 || batch > net->max_batch) return SQN_ERR_BADARG;
-    const size_t in_bytes = align_up((size_t)batch * IMG * IMG * 3 * esize(net->dtype), 1024);
+    const size_t in_bytes = align_up(input_bytes(net, batch), 1024);
     const size_t out_bytes = align_up((size_t)batch * 1000 * sizeof(float), 1024);
     *bytes = layout(net, batch, nullptr, nullptr) + 2 * in_bytes + 2 * out_bytes;
     return SQN_OK;
@@ -630,7 +655,7 @@ extern "C" int squeezenet_forward_host(sqn_net* net, const void* in_host, void* 
     int rc = ensure_copy_pipeline(net);
     if (rc != SQN_OK) return rc;
     const size_t fwd_bytes = layout(net, batch, nullptr, nullptr);
-    const size_t in_bytes = (size_t)batch * IMG * IMG * 3 * esize(net->dtype);
+    const size_t in_bytes = input_bytes(net, batch);
     const size_t out_bytes = (size_t)batch * 1000 * sizeof(float);
     char* ws = static_cast<char*>(workspace);
     const int b = (int)(net->host_calls & 1ull);
@@ -736,6 +761,52 @@ extern "C" int sqn_unpack_nhwc_to_nchw(const void* src, float* dst, int N, int C
                     const float v = dtype == SQN_F32 ? static_cast<const float*>(src)[si]
                                                      : bf16_to_f32(static_cast<const uint16_t*>(src)[si]);
                     dst[(((size_t)n * C + c) * H + h) * W + w] = v;
+                }
+    return SQN_OK;
+}
+
+// Stem operands in the layouts the bf16 stem kernel reads (what stem_pack produces on the device).
+extern "C" int sqn_stem_packed_extent(int H, int W, int* Hp, int* Wp)
+{
+    if (H <= 0 || W <= 0 || !Hp || !Wp) return SQN_ERR_BADARG;
+    *Hp = stem_packed_rows(H);
+    *Wp = stem_packed_cols(W);
+    return SQN_OK;
+}
+
+extern "C" int sqn_pack_stem_input(const float* src, void* dst, int N, int H, int W)
+{
+    if (!src || !dst || N <= 0 || H <= 0 || W <= 0) return SQN_ERR_BADARG;
+    const int Hp = stem_packed_rows(H), Wp = stem_packed_cols(W);
+    uint16_t* o = static_cast<uint16_t*>(dst);
+    const uint16_t one = f32_to_bf16_rne(1.0f);
+    for (int n = 0; n < N; ++n)
+        for (int y = 0; y < Hp; ++y)
+            for (int x = 0; x < Wp; ++x) {
+                uint16_t* px = o + (((size_t)n * Hp + y) * Wp + x) * 4;
+                const bool inside = y < H && x < W;
+                for (int c = 0; c < 3; ++c)
+                    px[c] = inside ? f32_to_bf16_rne(src[(((size_t)n * 3 + c) * H + y) * W + x]) : (uint16_t)0;
+                px[3] = inside ? one : (uint16_t)0;        // meets the bias folded into the kernels
+            }
+    return SQN_OK;
+}
+
+extern "C" int sqn_pack_stem_weights(const float* src, const float* bias, void* dst, int O)
+{
+    if (!src || !bias || !dst || O <= 0) return SQN_ERR_BADARG;
+    uint16_t* o = static_cast<uint16_t*>(dst);
+    for (int m = 0; m < O; ++m)
+        for (int kh = 0; kh < 7; ++kh)
+            for (int px = 0; px < 8; ++px)
+                for (int c = 0; c < 4; ++c) {
+                    uint16_t v = 0;
+                    if (px < 7 && c < 3) v = f32_to_bf16_rne(src[(((size_t)m * 3 + c) * 7 + kh) * 7 + px]);
+                    if (c == 3 && kh == 0 && px < 2) {          // the bias as hi + lo, against the input's constant 1
+                        const uint16_t hi = f32_to_bf16_rne(bias[m]);
+                        v = px == 0 ? hi : f32_to_bf16_rne(bias[m] - bf16_to_f32(hi));
+                    }
+                    o[(((size_t)m * 7 + kh) * 8 + px) * 4 + c] = v;
                 }
     return SQN_OK;
 }

@@ -1225,7 +1225,7 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     p.bias = d.bias;
     p.status = device_status_word();
     p.h_mul = 1;
-    p.b_early = (!stem && d.params_static) ? 1 : 0;
+    p.b_early = (d.params_static && (!stem || d.stem_prepacked)) ? 1 : 0;   // (the stem's kernels are otherwise repacked by the launch before it)
     p.bias_in_k = stem ? 1 : 0;
     p.pool = d.pool ? 1 : 0;
     if (p.pool && (d.OH < 3 || d.OW < 3 || d.Cout % 32 != 0 || d.Cout > TILE_M)) return SQN_ERR_UNSUPPORTED;
@@ -1524,7 +1524,7 @@ int cached_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_p
     PlanKey k;
     std::memset(&k, 0, sizeof(k));
     k.in = d.in; k.w = d.w; k.bias = d.bias; k.out = d.out; k.ws = ws;
-    const int v[14] = {d.N, d.Cin, d.H, d.W, d.Cout, d.K, d.S, d.pad, d.out_c_offset, d.out_c_total, d.relu | (d.pool << 1) | (d.params_static << 2),
+    const int v[14] = {d.N, d.Cin, d.H, d.W, d.Cout, d.K, d.S, d.pad, d.out_c_offset, d.out_c_total, d.relu | (d.pool << 1) | (d.params_static << 2) | (d.stem_prepacked << 3),
                        (stem ? 1 : 0) | (force_halves << 4) | ((force_cw & 0xffff) << 8), Hp, Wp};
     std::memcpy(k.v, v, sizeof(v));
     int dev = 0;
@@ -1698,10 +1698,21 @@ int launch_stem_conv_bf16(const ConvDesc& d, void* workspace, size_t workspace_b
 {
     int rc = stem_check(d, workspace, workspace_bytes);
     if (rc != SQN_OK) return rc;
-    const int Hp = (d.H + 1) / 2 * 2, Wp = (d.W + 2) / 2 * 2;
+    const int Hp = stem_packed_rows(d.H), Wp = stem_packed_cols(d.W);
     unsigned char* ws = static_cast<unsigned char*>(workspace);
     Plan plan;
     rc = cached_plan(d, true, ws, ws + align_up((size_t)d.N * Hp * Wp * 8, 1024), Hp, Wp, workspace, &plan);
+    if (rc != SQN_OK) return rc;
+    return launch_plan(plan, stream);
+}
+
+int launch_stem_conv_bf16_prepacked(const ConvDesc& d, cudaStream_t stream)
+{
+    if (!d.stem_prepacked) return SQN_ERR_BADARG;
+    if (d.Cout % 16 != 0 || d.Cout > 256) return SQN_ERR_UNSUPPORTED;
+    if (d.out_c_offset % 8 != 0 || d.out_c_total % 8 != 0) return SQN_ERR_ALIGN;
+    Plan plan;
+    const int rc = cached_plan(d, true, d.in, d.w, stem_packed_rows(d.H), stem_packed_cols(d.W), nullptr, &plan);
     if (rc != SQN_OK) return rc;
     return launch_plan(plan, stream);
 }

@@ -20,6 +20,7 @@ struct ConvDesc {
     int pool;             // 1: out receives the 3x3/stride-2 max-pool of the layer's output (bf16 path only)
     int params_static;    // 1: kernels and bias are not written by earlier work on the stream (a net's own parameters), so
                           //    a chained launch may fetch them before the kernel ahead of it has finished
+    int stem_prepacked;   // 1 (stem only): in and w already have the stem kernel's own layouts, see sqn_pack_stem_input
 };
 
 // Launch counter (host side): every kernel launch goes through note_launch().
@@ -45,6 +46,10 @@ int launch_conv_bf16_uncached(const ConvDesc& d, cudaStream_t stream);   // no p
 size_t stem_bf16_workspace_bytes(int N, int H, int W, int Cout);
 int launch_stem_pack_bf16(const ConvDesc& d, void* workspace, size_t workspace_bytes, cudaStream_t stream);
 int launch_stem_conv_bf16(const ConvDesc& d, void* workspace, size_t workspace_bytes, cudaStream_t stream);
+// The stem on operands the caller packed offline (d.in = [N][Hp][Wp][4], d.w = [Cout][7][8][4] with the bias folded in).
+int launch_stem_conv_bf16_prepacked(const ConvDesc& d, cudaStream_t stream);
+inline int stem_packed_rows(int H) { return (H + 1) / 2 * 2; }
+inline int stem_packed_cols(int W) { return (W + 2) / 2 * 2; }
 
 // Pooling / head.
 int launch_maxpool3x3s2(const void* in, void* out, int C, int H, int W, int N, int dtype, cudaStream_t stream);

@@ -112,3 +112,31 @@ def test_squeezenet_handle_and_workspace_without_gpu():
     with pytest.raises(B.SqnError):
         B.squeezenet_layer_output(h, "fire99", 0x100000, 1)
     B.squeezenet_destroy(h)
+
+
+def test_stem_pack_helpers_give_the_layout_the_stem_kernel_reads():
+    """[N][3][H][W] -> [N][Hp][Wp][4] with 1.0 in the fourth layer of image pixels and zero padding; kernels
+    [O][3][7][7] -> [O][7][8][4] with bias hi + lo in the fourth layer of the first two pixels of the first row."""
+    rng = np.random.default_rng(5)
+    x = rng.random((2, 3, 9, 11), dtype=np.float32)
+    assert B.sqn_stem_packed_extent(9, 11) == (10, 12) and B.sqn_stem_packed_extent(227, 227) == (228, 228)
+    got = B.sqn_pack_stem_input(x)
+    bf = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    exp = np.zeros((2, 10, 12, 4), dtype=np.uint16)
+    exp[:, :9, :11, :3] = bf(x.transpose(0, 2, 3, 1))
+    exp[:, :9, :11, 3] = 0x3f80
+    np.testing.assert_array_equal(got, exp)
+    w = rng.standard_normal((5, 3, 7, 7)).astype(np.float32)
+    b = rng.standard_normal(5).astype(np.float32)
+    gw = B.sqn_pack_stem_weights(w, b)
+    ew = np.zeros((5, 7, 8, 4), dtype=np.uint16)
+    ew[:, :, :7, :3] = bf(w.transpose(0, 2, 3, 1))
+    hi = torch.from_numpy(b).to(torch.bfloat16)
+    lo = (torch.from_numpy(b) - hi.float()).to(torch.bfloat16)
+    ew[:, 0, 0, 3] = hi.view(torch.int16).numpy().view(np.uint16)
+    ew[:, 0, 1, 3] = lo.view(torch.int16).numpy().view(np.uint16)
+    np.testing.assert_array_equal(gw, ew)
+    h = B.squeezenet_create([0x1000] * 26, [0x1000] * 26, B.SQN_F32, 1)
+    with pytest.raises(B.SqnError):
+        B.squeezenet_set_stem_prepacked(h, True)          # bf16 nets only
+    B.squeezenet_destroy(h)

@@ -388,3 +388,39 @@ def test_forced_kernel_variants_give_the_same_values():
     finally:
         os.environ.pop("SQN_TC_VARIANT", None)
     assert ran >= 6
+
+
+@pytest.mark.parametrize("batch", [2, 20])
+def test_stem_operands_packed_offline_give_the_same_logits(batch):
+    """squeezenet_set_stem_prepacked: the forward reads [228][228][4] images and [96][7][8][4] kernels written by the
+    host helpers and launches no repack kernel; the logits are exactly those of the forward that repacks on the
+    device (batch 2: separate pools; batch 20: fused pools), also through the host-buffer entry point."""
+    import torch
+    names = [n for n, *_ in synth.SQUEEZENET_CONVS]
+    x, params = synth.squeezenet_case(40 + batch, batch)
+    want = run_net(x, params, BF16, batch)[0]
+    ws = [G.dev_w(params[n][0], BF16) for n in names]
+    ws[0] = B.to_device(B.sqn_pack_stem_weights(*params["conv1"]), BF16)
+    bs = [G.dev_b(params[n][1]) for n in names]
+    net = B.squeezenet_create(ws, bs, BF16, batch)
+    B.squeezenet_set_stem_prepacked(net, True)
+    work = torch.empty(B.squeezenet_host_workspace_bytes(net, batch), dtype=torch.uint8, device="cuda")
+    packed = B.sqn_pack_stem_input(x)
+    logits = torch.empty((batch, 1000), device="cuda")
+    n0 = B.sqn_launch_count()
+    B.squeezenet_forward(net, B.to_device(packed, BF16), logits, None, work, batch)
+    assert B.sqn_check() == B.SQN_OK
+    launches = B.sqn_launch_count() - n0
+    np.testing.assert_array_equal(logits.cpu().numpy(), want)
+    out = torch.zeros((batch, 1000), dtype=torch.float32).pin_memory()
+    B.squeezenet_forward_host(net, torch.from_numpy(packed.view(np.int16)).pin_memory(), out, None, work, batch)
+    assert B.sqn_check() == B.SQN_OK
+    np.testing.assert_array_equal(out.numpy(), want)
+    B.squeezenet_destroy(net)
+    # one launch fewer than the forward that repacks
+    net2 = B.squeezenet_create([G.dev_w(params[n][0], BF16) for n in names], bs, BF16, batch)
+    n0 = B.sqn_launch_count()
+    B.squeezenet_forward(net2, G.dev_act(x, BF16), logits, None, work, batch)
+    assert B.sqn_check() == B.SQN_OK
+    assert B.sqn_launch_count() - n0 == launches + 1
+    B.squeezenet_destroy(net2)
