@@ -187,6 +187,10 @@ extern "C" int fire_forward(const void* in, const void* w_sq, const void* b_sq, 
         if ((rc = conv_bf16_supported(d3)) != SQN_OK) return rc;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (dtype == SQN_BF16 && fused_fire_enabled()) {
+        rc = launch_fire_fused_bf16(dsq, d1, d3, st);       // one kernel, squeeze_scratch stays untouched
+        if (rc != SQN_ERR_UNSUPPORTED) return rc;
+    }
     if ((rc = run_conv(dsq, dtype, nullptr, 0, st)) != SQN_OK) return rc;
     return run_expands(d1, d3, dtype, st, nullptr);
 }
@@ -302,6 +306,7 @@ struct sqn_net {
     int copy_device = -1;
     unsigned long long host_calls = 0;
     int stem_prepacked = 0;     // squeezenet_set_stem_prepacked
+    unsigned fused_fire_mask = 0;   // bit i: the last forward ran fire layer i as one kernel (its squeeze map was not stored)
 };
 
 namespace {
@@ -423,6 +428,9 @@ extern "C" int squeezenet_layer_output(const sqn_net* net, const char* name, voi
     if (net->dtype == SQN_BF16 && batch >= 16 &&
         (std::strcmp(name, "conv1") == 0 || std::strcmp(name, "fire4") == 0 || std::strcmp(name, "fire8") == 0))
         return SQN_ERR_UNSUPPORTED;   // computed inside the kernels that write pool1 / pool4, never stored
+    for (int f = 0; f < 8; ++f)
+        if ((net->fused_fire_mask >> f & 1u) && std::string(kFire[f].name) + "_sq" == name)
+            return SQN_ERR_UNSUPPORTED;   // kept in shared memory by the fused fire kernel of the last forward
     std::vector<size_t> offs;
     layout(net, batch, &offs, nullptr);
     *ptr = static_cast<char*>(workspace) + offs[i];
@@ -516,6 +524,7 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
     }
 
     const void* cur = buf("pool1");
+    net->fused_fire_mask = 0;
     for (int i = 0; i < 8; ++i) {
         const FireSpec& f = kFire[i];
         void* sq = buf(std::string(f.name) + "_sq");
@@ -533,6 +542,24 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
         // the net's kernels and bias are not written by anything this forward enqueues
         dsq.params_static = d1.params_static = d3.params_static = 1;
         const std::string nm(f.name);
+        // bf16: squeeze and both expands as one kernel where it applies (no pool behind the layer)
+        if (dt == SQN_BF16 && fused_fire_enabled() && !(f.pool_after && fuse_pools)) {
+            rc = launch_fire_fused_bf16(dsq, d1, d3, st);
+            if (rc == SQN_OK) {
+                net->fused_fire_mask |= 1u << i;
+                mark((nm + "_fused").c_str());
+                cur = out;
+                if (f.pool_after) {
+                    const std::string pn = std::string("pool") + (f.name + 4);
+                    void* po = buf(pn);
+                    if ((rc = launch_maxpool3x3s2(cur, po, 2 * f.e, f.hw, f.hw, batch, dt, st)) != SQN_OK) return rc;
+                    mark(pn.c_str());
+                    cur = po;
+                }
+                continue;
+            }
+            if (rc != SQN_ERR_UNSUPPORTED) return rc;
+        }
         if ((rc = run_conv(dsq, dt, nullptr, 0, st)) != SQN_OK) return rc;
         mark((nm + "_sq").c_str());
         // bf16: where a max-pool follows and the expands' kernels fit in shared memory, both expands pool

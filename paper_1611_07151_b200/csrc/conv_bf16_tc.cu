@@ -40,6 +40,8 @@
 
 #include "ptx_sm100.cuh"
 #include "sqn_internal.h"
+#include "tc_common.cuh"
+#include "tc_host.h"
 
 namespace sqn {
 namespace {
@@ -57,7 +59,6 @@ constexpr int MAX_TAB = 448;           // MMAs per tile in patch mode
 constexpr int PARAM_TAB = 160;         // ... of which this many can be tabulated in the kernel parameters
 constexpr size_t CTL_BYTES = 4096;
 constexpr size_t CTL_BYTES_NO_TAB = 1024;   // control block without the shared-memory MMA table
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // about two seconds
 constexpr size_t SMEM_LIMIT = 227 * 1024;
 constexpr size_t SMEM_LIMIT_2CTA = 113 * 1024;     // two CTAs share an SM's 228 KB (1 KB reserved each)
 
@@ -125,56 +126,6 @@ struct Shared {                       // control block placed after the tiles
     volatile int abort_flag;
     uint2 mma_tab[MAX_TAB + 1];           // patch mode: per MMA, {A offset from the stage base, B address} in 16-byte units
 };
-
-// Bounded mbarrier wait.  Polls back to back at first (hand-offs between the roles take a few
-// hundred cycles), backs off with nanosleep on long waits, and gives up after WAIT_LIMIT_CYCLES:
-// the CTA then records SQN_ERR_TIMEOUT and every role leaves its loop.
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (uint32_t i = 1;; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 255u) == 0u) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
-                *abort_flag = 1;
-                if (status) atomicExch(status, (int)SQN_ERR_TIMEOUT);
-                return false;
-            }
-        }
-        if (i > 4096u) __nanosleep(128);
-    }
-}
-
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
-{
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&v);
-}
-// max(.,0) and round-to-nearest-even conversion of two values in one instruction
-__device__ __forceinline__ uint32_t pack_relu_bf16x2(float lo, float hi)
-{
-    uint32_t d;
-    asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
-    return d;
-}
-
-// maximum of three values in one instruction
-__device__ __forceinline__ float max3(float a, float b, float c)
-{
-    float r;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
-    return r;
-}
-// fp32 -> bf16 (round to nearest even), with max(., 0) folded into the conversion when relu is set
-__device__ __forceinline__ unsigned short to_bf16_bits(float v, int relu)
-{
-    unsigned short h;
-    if (relu) asm("cvt.rn.relu.bf16.f32 %0, %1;" : "=h"(h) : "f"(v));
-    else asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(h) : "f"(v));
-    return h;
-}
 
 // Position of a tile in (output-layer tile, column tile, row tile, image tile) digits.  A CTA
 // walks tiles bid, bid + grid, ...; the step is added digit by digit, so the
@@ -1560,6 +1511,13 @@ int cached_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_p
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 }  // namespace
+
+bool tmap_encode_bf16(CUtensorMap* m, int rank, const void* ptr, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
+                      const cuuint32_t* box, unsigned inner_bytes)
+{
+    return encode(m, rank, ptr, dims, strides_bytes, box, inner_bytes);
+}
+int sm_count() { return num_sms(); }
 
 int conv_bf16_supported(const ConvDesc& d)
 {

@@ -1,0 +1,706 @@
+// Fire layer (paper Section II: one squeeze layer feeding two expand layers) as ONE kernel, bf16 on the tensor cores:
+// the squeeze map never leaves the SM.  Section III-C of the paper has every layer write its output in the order
+// the next layer reads, so that nothing is repacked between layers; here the squeeze layer writes its output
+// straight into the shared-memory operand of the two expand layers, so that nothing is stored between them at all.
+//
+// Work item = a band of R output rows of one image.  For a band the CTA
+//   1. squeezes the band's input rows and one halo row above and below (1x1 convolution: rows of the flat pixel
+//      index are the M = 128 operand, read by TMA as they lie in memory; the squeeze kernels stay in shared
+//      memory), and its epilogue warps write the result -- bias added, ReLU, rounded to bf16 -- as a flat array of
+//      pixels with a pitch of P = W + 2 pixels per image row: "the patch".  The two extra columns and the rows
+//      outside the image are the zero padding of the 3x3 expand and stay zero;
+//   2. runs both expands on the patch.  Output tile t = RT image rows = RT*P <= 128 consecutive patch pixels (the two
+//      padding pixels of every row compute garbage that is never stored).  Kernel tap (kh, kw) of the 3x3 expand is
+//      one MMA whose A descriptor starts (kh*P + kw) pixels further into the patch; the 1x1 expand is the centre
+//      tap, so its kernels are appended to the centre tap's and one MMA of N = e3 + e1 serves both.  The accumulator
+//      holds e3 + e1 <= 256 columns; the epilogue converts it chunk by chunk into a staging tile of RT rows x W
+//      pixels (the padding pixels dropped) that one TMA store sends to the layer slices of the output tensor.
+// The jobs of a CTA -- squeeze tiles, then expand tiles, item after item -- alternate between two TMEM accumulators
+// and are drained in issue order, so the epilogue of one job overlaps the MMAs of the next, and the squeeze epilogue
+// of the next band cannot overwrite the patch before the expand MMAs of this band have read it.
+// Warps: 0 TMA producer (input tiles; all kernels once), 1 MMA issuer, 2..9 epilogue, 10 TMA stores.
+// Every mbarrier wait is bounded (see wait_bar).
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <algorithm>
+#include <cstdlib>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <string>
+
+#include "ptx_sm100.cuh"
+#include "sqn_internal.h"
+#include "tc_common.cuh"
+#include "tc_host.h"
+
+namespace sqn {
+namespace {
+
+using namespace ptx;
+
+constexpr int FF_EPI_WARPS = 8;
+constexpr int FF_THREADS = 32 * (2 + FF_EPI_WARPS + 1);
+constexpr int FF_MAX_STAGES = 8;
+constexpr int FF_MAX_STG = 4;
+constexpr int FF_MAX_EMMA = 40;            // MMAs of one expand tile: 9 taps x at most 4 k-steps, + spare
+constexpr size_t FF_SMEM_LIMIT = 227 * 1024;
+constexpr int FF_CW = 64;                  // output layers per store chunk
+
+struct FireParams {
+    int H, W, P, N;                  // map extent, patch pitch (W + 2), images
+    int Cin, s, e1, e3;
+    int RT, R, NB;                   // image rows per expand tile, rows per band, bands per image
+    int items, grid;
+    int chunks_in, BKc_in, ksteps_in;   // squeeze reduction: chunks, elements per chunk, MMAs per chunk
+    int ksteps_s;                    // MMAs per expand tap (s / 16)
+    int n_emma;                      // MMAs of an expand tile (without the bias MMA)
+    int nchunks;                     // store chunks per expand tile ((e3 + e1) / FF_CW)
+    int stages, nstg;
+    int slot_cols;                   // TMEM columns per accumulator
+    unsigned tmem_cols;
+    int c_tot;                       // layers per pixel of the output tensor
+    int b_early;                     // kernels and bias may be fetched before the wait for the grid ahead
+    unsigned rb_in, rb_s;            // bytes per row of the input / squeeze-kernel tiles and of the patch / expand-kernel tiles
+    unsigned x_bytes;                // bytes one input box delivers
+    unsigned w_bytes;                // bytes of all kernel tiles together
+    unsigned off_wsq, wsq_tile;      // squeeze kernels: chunks_in tiles of s rows
+    unsigned off_we;                 // expand kernels: centre tap, 1x1, then the other eight taps
+    unsigned off_tap[9], off_w1;     // ... offsets of the tiles from off_we
+    unsigned off_patch, patch_bytes;
+    unsigned off_x, x_tile;
+    unsigned off_stg, stg_slot;
+    unsigned off_bias_s, off_bias_e, off_ones, off_ctl;
+    const float *bias_sq, *bias_e1, *bias_e3;
+    int* status;
+    uint2 etab[FF_MAX_EMMA];         // per expand MMA: {A offset from the tile's first patch pixel, B offset from off_we}, 16-byte units
+};
+
+struct FireShared {
+    unsigned long long full[FF_MAX_STAGES];
+    unsigned long long empty[FF_MAX_STAGES];
+    unsigned long long w_full;
+    unsigned long long tmem_full[2];
+    unsigned long long tmem_empty[2];
+    unsigned long long patch_ready;
+    unsigned long long stg_full[FF_MAX_STG];
+    unsigned long long stg_free[FF_MAX_STG];
+    unsigned tmem_base;
+    volatile int abort_flag;
+};
+
+// A band of an image: rows [y0, y0 + rows) are produced, input rows [ylo, yhi) are squeezed.
+struct Band { int n, y0, rows, ylo, npx, n_s, n_e; };
+
+__device__ __forceinline__ Band band_of(const FireParams& p, int item)
+{
+    Band b;
+    b.n = item / p.NB;
+    const int k = item - b.n * p.NB;
+    b.y0 = k * p.R;
+    b.rows = p.H - b.y0 < p.R ? p.H - b.y0 : p.R;
+    b.ylo = b.y0 > 0 ? b.y0 - 1 : 0;
+    const int yhi = b.y0 + b.rows + 1 < p.H ? b.y0 + b.rows + 1 : p.H;
+    b.npx = (yhi - b.ylo) * p.W;
+    b.n_s = (b.npx + 127) >> 7;
+    b.n_e = (b.rows + p.RT - 1) / p.RT;
+    return b;
+}
+
+// 16-byte unit `u` of row `r` of a tile with `rb`-byte rows written by TMA with the swizzle of that width (tile base
+// aligned to 1024 bytes): the unit index is XORed with address bits 7.. of the row.
+__device__ __forceinline__ uint32_t swz(uint32_t r, uint32_t rb)
+{
+    return rb == 128 ? (r & 7u) : rb == 64 ? ((r >> 1) & 3u) : ((r >> 2) & 1u);
+}
+
+// Bias rows of the bias MMA: one 32-byte row {hi, lo, 0, ...} per output layer, hi + lo = the fp32 bias.
+__device__ __forceinline__ void bias_row(uint4* rows, int c, float b)
+{
+    const __nv_bfloat16 hi = __float2bfloat16_rn(b);
+    const __nv_bfloat16 lo = __float2bfloat16_rn(b - __bfloat162float(hi));
+    const int u = (c >> 2) & 1;
+    rows[2 * c + u] = make_uint4((uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16), 0u, 0u, 0u);
+    rows[2 * c + (u ^ 1)] = make_uint4(0u, 0u, 0u, 0u);
+}
+
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+__global__ void __launch_bounds__(FF_THREADS, 1)
+fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmWsq,
+                  const __grid_constant__ CUtensorMap tmW3, const __grid_constant__ CUtensorMap tmW1,
+                  const __grid_constant__ CUtensorMap tmO, const __grid_constant__ FireParams p)
+{
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    unsigned char* base_ptr = smem_raw + (base - raw);
+    FireShared* sh = reinterpret_cast<FireShared*>(base_ptr + p.off_ctl);
+    const uint32_t smWsq = base + p.off_wsq, smWe = base + p.off_we, smPatch = base + p.off_patch;
+    const uint32_t smX = base + p.off_x, smStg = base + p.off_stg;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int bid = (int)blockIdx.x;
+
+    auto load_kernels = [&]() {          // every kernel tile of the layer, once (one mbarrier counts them all)
+        const uint32_t bar = smem_u32(&sh->w_full);
+        mbar_arrive_expect_tx(bar, p.w_bytes);
+        for (int ch = 0; ch < p.chunks_in; ++ch)
+            tma_load_2d(smWsq + (uint32_t)ch * p.wsq_tile, &tmWsq, bar, ch * p.BKc_in, 0);
+        for (int tap = 0; tap < 9; ++tap) tma_load_2d(smWe + p.off_tap[tap], &tmW3, bar, tap * p.s, 0);
+        tma_load_2d(smWe + p.off_w1, &tmW1, bar, 0, 0);
+    };
+    auto fill_bias = [&]() {
+        uint4* rs = reinterpret_cast<uint4*>(base_ptr + p.off_bias_s);
+        for (int c = threadIdx.x; c < p.s; c += FF_THREADS) bias_row(rs, c, __ldg(p.bias_sq + c));
+        uint4* re = reinterpret_cast<uint4*>(base_ptr + p.off_bias_e);
+        for (int c = threadIdx.x; c < p.e3 + p.e1; c += FF_THREADS)
+            bias_row(re, c, c < p.e3 ? __ldg(p.bias_e3 + c) : __ldg(p.bias_e1 + c - p.e3));
+    };
+
+    // Up to chain_wait() this block touches only its own shared memory, TMEM, the kernel parameters and, when
+    // b_early is set, the layer's kernels and bias (see conv_tc_body).
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) {
+            mbar_init(smem_u32(&sh->full[s]), 1);
+            mbar_init(smem_u32(&sh->empty[s]), 1);
+        }
+        mbar_init(smem_u32(&sh->w_full), 1);
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(smem_u32(&sh->tmem_full[a]), 1);
+            mbar_init(smem_u32(&sh->tmem_empty[a]), FF_EPI_WARPS);
+        }
+        mbar_init(smem_u32(&sh->patch_ready), FF_EPI_WARPS);
+        for (int b = 0; b < p.nstg; ++b) {
+            mbar_init(smem_u32(&sh->stg_full[b]), FF_EPI_WARPS);
+            mbar_init(smem_u32(&sh->stg_free[b]), 1);
+        }
+        sh->abort_flag = 0;
+        fence_mbar_init();
+        prefetch_tensormap(&tmX);
+        prefetch_tensormap(&tmWsq);
+        prefetch_tensormap(&tmW3);
+        prefetch_tensormap(&tmW1);
+        prefetch_tensormap(&tmO);
+        if (p.b_early) load_kernels();
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&sh->tmem_base), p.tmem_cols);
+        tmem_relinquish();
+        chain_release();            // (only once this CTA holds its TMEM: see conv_tc_body)
+    }
+    // the patch starts as zeros: its two padding columns and the rows outside the image are never written
+    for (uint32_t i = threadIdx.x; i < p.patch_bytes / 16u; i += FF_THREADS) st_shared_v4(smPatch + 16u * i, 0u, 0u, 0u, 0u);
+    {
+        // tile of ones for the bias MMAs: 128 rows of 32 bytes in the 32-byte swizzle, ones in the first two places
+        uint4* ones = reinterpret_cast<uint4*>(base_ptr + p.off_ones);
+        for (int r = threadIdx.x; r < 128; r += FF_THREADS) {
+            const int u = (r >> 2) & 1;
+            ones[2 * r + u] = make_uint4(0x3f803f80u, 0u, 0u, 0u);
+            ones[2 * r + (u ^ 1)] = make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
+    if (p.b_early) fill_bias();
+    chain_wait();       // the grid ahead has finished: global memory may be read and written from here on
+    if (!p.b_early) fill_bias();
+    fence_proxy_async_smem();           // the MMAs read patch, ones and bias rows through the async proxy
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = sh->tmem_base;
+    volatile int* abort_flag = &sh->abort_flag;
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer: input tiles of the squeeze
+        if (lane == 0) {
+            if (!p.b_early) load_kernels();
+            bool ok = true;
+            int st = 0, issued = 0;
+            uint32_t ph = 0;
+            for (int item = bid; item < p.items && ok; item += p.grid) {
+                const Band b = band_of(p, item);
+                const int px0 = (b.n * p.H + b.ylo) * p.W;
+                for (int t = 0; t < b.n_s && ok; ++t)
+                    for (int ch = 0; ch < p.chunks_in; ++ch) {
+                        if (!wait_bar(smem_u32(&sh->empty[st]), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                        const uint32_t full = smem_u32(&sh->full[st]);
+                        mbar_arrive_expect_tx(full, p.x_bytes);
+                        tma_load_2d(smX + (uint32_t)st * p.x_tile, &tmX, full, ch * p.BKc_in, px0 + 128 * t);
+                        ++issued;
+                        if (++st == p.stages) { st = 0; ph ^= 1u; }
+                    }
+            }
+            if (!ok) {      // give the copies already issued a bounded chance to land before the CTA exits
+                int pending = issued < p.stages ? issued : p.stages;
+                while (pending-- > 0) {
+                    if (st == 0) { st = p.stages; ph ^= 1u; }
+                    --st;
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(smem_u32(&sh->full[st]), ph)) {
+                        if (clock64() - t0 > WAIT_LIMIT_CYCLES / 8) break;
+                        __nanosleep(100);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        // The whole warp walks the loops converged; one elected lane issues the MMAs and their commits.
+        const uint32_t idesc_s = make_idesc_bf16(128, (uint32_t)p.s);
+        const uint32_t idesc_c = make_idesc_bf16(128, (uint32_t)(p.e3 + p.e1));
+        const uint32_t idesc_3 = make_idesc_bf16(128, (uint32_t)p.e3);
+        const uint32_t hi_in = (uint32_t)(make_kmajor_desc(0, p.rb_in, 8u * p.rb_in) >> 32);
+        const uint32_t hi_s = (uint32_t)(make_kmajor_desc(0, p.rb_s, 8u * p.rb_s) >> 32);
+        const uint64_t ones_desc = make_kmajor_desc(base + p.off_ones, 32u, 256u);
+        const uint64_t bias_s_desc = make_kmajor_desc(base + p.off_bias_s, 32u, 256u);
+        const uint64_t bias_e_desc = make_kmajor_desc(base + p.off_bias_e, 32u, 256u);
+        const uint32_t smX16 = smX >> 4, x_tile16 = p.x_tile >> 4, smWsq16 = smWsq >> 4, wsq_tile16 = p.wsq_tile >> 4;
+        const uint32_t smWe16 = smWe >> 4, patch16 = smPatch >> 4;
+        const uint32_t tile_step16 = ((uint32_t)(p.RT * p.P) * p.rb_s) >> 4;      // patch units between expand tiles
+        bool ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->w_full), 0u, abort_flag, p.status));
+        int st = 0, as = 0;
+        uint32_t ph = 0, aph = 0, pph = 0;
+        for (int item = bid; item < p.items && ok; item += p.grid) {
+            const Band b = band_of(p, item);
+            // squeeze tiles
+            for (int t = 0; t < b.n_s && ok; ++t) {
+                ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_empty[as]), aph ^ 1u, abort_flag, p.status));
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(as * p.slot_cols);
+                for (int ch = 0; ch < p.chunks_in; ++ch) {
+                    ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->full[st]), ph, abort_flag, p.status));
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (elect_one()) {
+                        const uint64_t da = ((uint64_t)hi_in << 32) | (uint64_t)((smX16 + (uint32_t)st * x_tile16) | 0x10000u);
+                        const uint64_t db = ((uint64_t)hi_in << 32) | (uint64_t)((smWsq16 + (uint32_t)ch * wsq_tile16) | 0x10000u);
+                        for (int k = 0; k < p.ksteps_in; ++k)
+                            mma_bf16_ss(d_tmem, da + 2u * k, db + 2u * k, idesc_s, (ch | k) ? 1u : 0u);
+                        mma_commit(smem_u32(&sh->empty[st]));           // input slot free once these MMAs have read it
+                        if (ch == p.chunks_in - 1) {
+                            mma_bf16_ss(d_tmem, ones_desc, bias_s_desc, idesc_s, 1u);
+                            mma_commit(smem_u32(&sh->tmem_full[as]));
+                        }
+                    }
+                    __syncwarp();
+                    if (++st == p.stages) { st = 0; ph ^= 1u; }
+                }
+                if (!ok) break;
+                if (++as == 2) { as = 0; aph ^= 1u; }
+            }
+            if (!ok) break;
+            // the patch of this band is complete once every epilogue warp has passed its last squeeze tile
+            ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->patch_ready), pph, abort_flag, p.status));
+            if (!ok) break;
+            pph ^= 1u;
+            tc_fence_after();
+            // expand tiles
+            for (int t = 0; t < b.n_e; ++t) {
+                ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_empty[as]), aph ^ 1u, abort_flag, p.status));
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(as * p.slot_cols);
+                const uint32_t a_base = patch16 + (uint32_t)t * tile_step16;
+                if (elect_one()) {
+                    uint32_t acc = 0u;
+#pragma unroll 2
+                    for (int e = 0; e < p.n_emma; ++e) {
+                        const uint2 o = p.etab[e];
+                        // the centre tap comes first and carries the 1x1 expand's kernels: N = e3 + e1
+                        mma_bf16_ss(d_tmem, ((uint64_t)hi_s << 32) | (uint64_t)((a_base + o.x) | 0x10000u),
+                                    ((uint64_t)hi_s << 32) | (uint64_t)((smWe16 + o.y) | 0x10000u),
+                                    e < p.ksteps_s ? idesc_c : idesc_3, acc);
+                        acc = 1u;
+                    }
+                    mma_bf16_ss(d_tmem, ones_desc, bias_e_desc, idesc_c, 1u);
+                    mma_commit(smem_u32(&sh->tmem_full[as]));
+                }
+                __syncwarp();
+                if (++as == 2) { as = 0; aph ^= 1u; }
+            }
+        }
+    } else if (warp < 2 + FF_EPI_WARPS) {
+        // -------------------------------------------------------------------- epilogue
+        // warp w reads TMEM lane quadrant w % 4 (one M row per thread); the two warps of a quadrant split the columns.
+        const int q = warp & 3, hf = (warp - 2) >> 2;
+        const int row = q * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(q * 32) << 16;
+        const int eidx = (warp - 2) * 32 + lane;                 // index among the 256 epilogue threads
+        // expand tiles: M row -> (image row r of the tile, patch column c); the staging tile drops the padding columns
+        const int r_e = row / p.P, c_e = row - r_e * p.P;
+        const bool e_valid = c_e < p.W && r_e < p.RT;
+        const uint32_t stg_row = (uint32_t)(r_e * p.W + c_e);
+        const uint32_t stg_off = stg_row * (uint32_t)(FF_CW * 2);
+        const uint32_t sw_e = stg_row & 7u;
+        const int hs = p.s >> 1;                                 // squeeze columns per thread: 8, 16 or 32
+        const uint32_t units_s = (uint32_t)hs >> 3;             // ... = this many 16-byte units of a patch row
+        bool ok = true;
+        int as = 0, sb = 0;
+        uint32_t aph = 0, sph = 0;
+        for (int item = bid; item < p.items && ok; item += p.grid) {
+            const Band b = band_of(p, item);
+            for (int t = 0; t < b.n_s; ++t) {
+                ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_full[as]), aph, abort_flag, p.status));
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t ta = tmem_base + lane_base + (uint32_t)(as * p.slot_cols + hf * hs);
+                uint32_t v[32];
+                if (hs == 32) {
+                    tmem_ld_x16(ta, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
+                    tmem_ld_x16(ta + 16u, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
+                } else if (hs == 16) {
+                    tmem_ld_x16(ta, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
+                } else {
+                    tmem_ld_x8(ta, *reinterpret_cast<uint32_t(*)[8]>(&v[0]));
+                }
+                tmem_ld_wait();
+                // accumulator in registers: hand it back to the MMA issuer
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[as]));
+                if (++as == 2) { as = 0; aph ^= 1u; }
+                const int g = t * 128 + row;                      // pixel of the band's input rows
+                if (g < b.npx) {
+                    const int yy = g / p.W, xx = g - yy * p.W;
+                    const uint32_t pr = (uint32_t)((yy + b.ylo - b.y0 + 1) * p.P + xx + 1);
+                    const uint32_t rbase = smPatch + pr * p.rb_s;
+                    const uint32_t sw = swz(pr, p.rb_s);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        if ((uint32_t)u < units_s) {
+                            uint32_t o[4];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                o[j] = pack_relu_bf16x2(__uint_as_float(v[8 * u + 2 * j]), __uint_as_float(v[8 * u + 2 * j + 1]));
+                            st_shared_v4(rbase + ((((uint32_t)hf * units_s + (uint32_t)u) ^ sw) << 4), o[0], o[1], o[2], o[3]);
+                        }
+                    }
+                }
+            }
+            if (!ok) break;
+            // patch rows that lie outside the image (above the first band, below the last) hold what an earlier band left
+            {
+                const uint32_t row_units = ((uint32_t)p.P * p.rb_s) >> 4;
+                if (b.y0 == 0)
+                    for (uint32_t i = (uint32_t)eidx; i < row_units; i += 32u * FF_EPI_WARPS) st_shared_v4(smPatch + 16u * i, 0u, 0u, 0u, 0u);
+                if (b.y0 + b.rows == p.H) {
+                    const uint32_t a0 = smPatch + (uint32_t)((b.rows + 1) * p.P) * p.rb_s;
+                    for (uint32_t i = (uint32_t)eidx; i < row_units; i += 32u * FF_EPI_WARPS) st_shared_v4(a0 + 16u * i, 0u, 0u, 0u, 0u);
+                }
+            }
+            fence_proxy_async_smem();             // patch visible to the tensor core
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->patch_ready));
+            for (int t = 0; t < b.n_e; ++t) {
+                ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_full[as]), aph, abort_flag, p.status));
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t ta0 = tmem_base + lane_base + (uint32_t)(as * p.slot_cols + hf * 32);
+                for (int chunk = 0; chunk < p.nchunks; ++chunk) {
+                    uint32_t v[32];
+                    const uint32_t ta = ta0 + (uint32_t)(chunk * FF_CW);
+                    tmem_ld_x16(ta, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
+                    tmem_ld_x16(ta + 16u, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
+                    ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->stg_free[sb]), sph ^ 1u, abort_flag, p.status));
+                    tmem_ld_wait();
+                    if (!ok) break;
+                    if (e_valid) {
+                        const uint32_t rbase = smStg + (uint32_t)sb * p.stg_slot + stg_off;
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            uint32_t o[4];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                o[j] = pack_relu_bf16x2(__uint_as_float(v[8 * u + 2 * j]), __uint_as_float(v[8 * u + 2 * j + 1]));
+                            st_shared_v4(rbase + ((((uint32_t)hf * 4u + (uint32_t)u) ^ sw_e) << 4), o[0], o[1], o[2], o[3]);
+                        }
+                    }
+                    fence_proxy_async_smem();             // staging rows visible to the TMA unit
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&sh->stg_full[sb]));
+                    if (++sb == p.nstg) { sb = 0; sph ^= 1u; }
+                }
+                if (!ok) break;
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[as]));
+                if (++as == 2) { as = 0; aph ^= 1u; }
+            }
+        }
+    } else {
+        // ----------------------------------------------------------------- store issuer
+        if (lane == 0) {
+            bool ok = true;
+            int sb = 0, pend = 0, fb = 0;       // next slot, stores whose slot is not yet released, next slot to release
+            uint32_t sph = 0;
+            for (int item = bid; item < p.items && ok; item += p.grid) {
+                const Band b = band_of(p, item);
+                for (int t = 0; t < b.n_e && ok; ++t)
+                    for (int chunk = 0; chunk < p.nchunks; ++chunk) {
+                        if (!wait_bar(smem_u32(&sh->stg_full[sb]), sph, abort_flag, p.status)) { ok = false; break; }
+                        // accumulator columns [0, e3) are the 3x3 expand (output layers e1 ..), the rest the 1x1 expand
+                        const int col = chunk * FF_CW;
+                        const int cc = col < p.e3 ? p.e1 + col : col - p.e3;
+                        tma_store_4d(&tmO, smStg + (uint32_t)sb * p.stg_slot, cc, 0, b.y0 + t * p.RT, b.n);
+                        tma_store_commit();
+                        if (++sb == p.nstg) { sb = 0; sph ^= 1u; }
+                        if (++pend == p.nstg) {
+                            if (p.nstg == 4) asm volatile("cp.async.bulk.wait_group.read 3;" ::: "memory");
+                            else if (p.nstg == 3) asm volatile("cp.async.bulk.wait_group.read 2;" ::: "memory");
+                            else asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                            mbar_arrive(smem_u32(&sh->stg_free[fb]));
+                            if (++fb == p.nstg) fb = 0;
+                            --pend;
+                        }
+                    }
+            }
+            tma_store_wait_all();
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, p.tmem_cols);
+    }
+}
+
+// ------------------------------------------------------------------------------ host side
+struct FirePlan {
+    CUtensorMap x, wsq, w3, w1, o;
+    FireParams p;
+    size_t smem;
+};
+
+inline size_t up1k(size_t v) { return (v + 1023) / 1024 * 1024; }
+
+// Rows per band: SQN_FIRE_BAND in the environment (tuning aid, read at every call), else 14 rows for maps of 40 rows
+// and more (equal bands for 55 rows), 16 rows from 20 rows on (a smaller patch leaves room for a deeper input ring),
+// else the whole image.
+int band_rows(int H, int RT)
+{
+    int R = H >= 40 ? 14 : H >= 20 ? 16 : H;
+    if (const char* v = std::getenv("SQN_FIRE_BAND")) {
+        const int r = std::atoi(v);
+        if (r > 0) R = r;
+    }
+    if (R > H) R = H;
+    R = (R + RT - 1) / RT * RT;          // a band is a whole number of expand tiles
+    return R;
+}
+
+int build_fire_plan(const ConvDesc& dsq, const ConvDesc& d1, const ConvDesc& d3, FirePlan* plan)
+{
+    FireParams& p = plan->p;
+    std::memset(&p, 0, sizeof(p));
+    const int H = dsq.H, W = dsq.W, N = dsq.N, Cin = dsq.Cin, s = dsq.Cout, e1 = d1.Cout, e3 = d3.Cout;
+    if (s != 16 && s != 32 && s != 64) return SQN_ERR_UNSUPPORTED;            // one swizzled row per patch pixel
+    if (e1 % FF_CW != 0 || e3 % FF_CW != 0 || e1 + e3 > 256) return SQN_ERR_UNSUPPORTED;
+    if (Cin % 32 != 0) return SQN_ERR_UNSUPPORTED;
+    if (W + 2 > 128 || H < 1) return SQN_ERR_UNSUPPORTED;
+    if (d1.out != d3.out || d1.out_c_total != d3.out_c_total || d1.out_c_offset != 0 || d3.out_c_offset != e1 ||
+        d1.out_c_total % 8 != 0)
+        return SQN_ERR_UNSUPPORTED;
+    if ((long long)N * H * W > 0x7fffffffLL / 2) return SQN_ERR_UNSUPPORTED;
+    p.H = H; p.W = W; p.P = W + 2; p.N = N; p.Cin = Cin; p.s = s; p.e1 = e1; p.e3 = e3;
+    p.RT = 128 / p.P;
+    p.R = band_rows(H, p.RT);
+    p.NB = (H + p.R - 1) / p.R;
+    p.items = N * p.NB;
+    p.BKc_in = Cin % 64 == 0 ? 64 : 32;
+    p.chunks_in = Cin / p.BKc_in;
+    p.ksteps_in = p.BKc_in / 16;
+    p.ksteps_s = s / 16;
+    p.n_emma = 9 * p.ksteps_s;
+    p.nchunks = (e1 + e3) / FF_CW;
+    p.slot_cols = e1 + e3;                 // (>= s)
+    p.tmem_cols = 2u * (unsigned)p.slot_cols <= 256u ? 256u : 512u;
+    p.c_tot = d1.out_c_total;
+    p.b_early = (dsq.params_static && d1.params_static && d3.params_static) ? 1 : 0;
+    p.rb_in = (unsigned)p.BKc_in * 2u;
+    p.rb_s = (unsigned)s * 2u;
+    p.x_bytes = 128u * p.rb_in;
+    p.bias_sq = dsq.bias; p.bias_e1 = d1.bias; p.bias_e3 = d3.bias;
+    p.status = device_status_word();
+
+    // ---- shared-memory layout
+    size_t cur = 0;
+    p.off_wsq = 0;
+    p.wsq_tile = (unsigned)up1k((size_t)s * p.rb_in);
+    cur += (size_t)p.chunks_in * p.wsq_tile;
+    p.off_we = (unsigned)cur;
+    {
+        // centre tap, then the 1x1 expand's kernels directly behind it (one B operand of e3 + e1 rows), then the others
+        const unsigned t3 = (unsigned)e3 * p.rb_s, t1 = (unsigned)e1 * p.rb_s;
+        if (t3 % 1024u != 0) return SQN_ERR_UNSUPPORTED;          // the appended tile must continue the swizzle pattern
+        unsigned o = 0;
+        p.off_tap[4] = o; o += t3;
+        p.off_w1 = o; o += (unsigned)up1k(t1);
+        for (int tap = 0; tap < 9; ++tap)
+            if (tap != 4) { p.off_tap[tap] = o; o += t3; }
+        cur += o;
+        p.w_bytes = (unsigned)((size_t)p.chunks_in * s * p.rb_in + 9u * t3 + t1);
+        if (p.w_bytes >= (1u << 20)) return SQN_ERR_UNSUPPORTED;  // one mbarrier transaction count
+    }
+    p.off_patch = (unsigned)cur;
+    {
+        const int t_max = p.R / p.RT;
+        size_t rows = (size_t)(p.R + 2) * p.P;
+        const size_t reach = (size_t)(t_max - 1) * p.RT * p.P + 2 * p.P + 2 + 128;     // last row an expand MMA reads
+        if (reach > rows) rows = reach;
+        p.patch_bytes = (unsigned)up1k(rows * p.rb_s);
+        cur += p.patch_bytes;
+    }
+    p.off_bias_s = (unsigned)cur; cur += up1k((size_t)s * 32);
+    p.off_bias_e = (unsigned)cur; cur += up1k((size_t)(e1 + e3) * 32);
+    p.off_ones = (unsigned)cur; cur += 128 * 32;
+    p.off_ctl = (unsigned)cur; cur += 1024;
+    static_assert(sizeof(FireShared) <= 1024, "control block");
+    p.stg_slot = (unsigned)up1k((size_t)p.RT * W * FF_CW * 2);
+    p.x_tile = (unsigned)up1k(p.x_bytes);
+    const size_t fixed = 1024 /*alignment slack*/ + cur;
+    if (fixed + 2 * p.stg_slot + 2 * p.x_tile > FF_SMEM_LIMIT) return SQN_ERR_UNSUPPORTED;
+    // input ring first (it feeds the HBM-bound part), then staging slots
+    size_t left = FF_SMEM_LIMIT - fixed;
+    p.nstg = 2;
+    left -= 2 * p.stg_slot;
+    int stages = (int)(left / p.x_tile);
+    // with room to spare, two more staging slots are worth more than input slots beyond what covers the memory latency
+    const int want = 2 * p.chunks_in > 4 ? 2 * p.chunks_in : 4;
+    if (stages >= want + (int)(2 * p.stg_slot / p.x_tile) + 1) {
+        p.nstg = 4;
+        left -= 2 * p.stg_slot;
+        stages = (int)(left / p.x_tile);
+    }
+    if (stages > FF_MAX_STAGES) stages = FF_MAX_STAGES;
+    if (stages < 2) return SQN_ERR_UNSUPPORTED;
+    p.stages = stages;
+    p.off_x = (unsigned)cur; cur += (size_t)stages * p.x_tile;
+    p.off_stg = (unsigned)cur; cur += (size_t)p.nstg * p.stg_slot;
+    plan->smem = 1024 + cur;
+    if (plan->smem > FF_SMEM_LIMIT) return SQN_ERR_UNSUPPORTED;
+
+    // ---- MMAs of an expand tile: centre tap first (it overwrites all e3 + e1 columns), then the other taps
+    {
+        int e = 0;
+        static const int order[9] = {4, 0, 1, 2, 3, 5, 6, 7, 8};
+        for (int i = 0; i < 9; ++i) {
+            const int tap = order[i], kh = tap / 3, kw = tap % 3;
+            for (int k = 0; k < p.ksteps_s; ++k, ++e) {
+                p.etab[e].x = (((unsigned)(kh * p.P + kw) * p.rb_s) >> 4) + 2u * k;
+                p.etab[e].y = (p.off_tap[tap] >> 4) + 2u * k;
+            }
+        }
+    }
+    // CTA b takes items b, b + grid, ...: with a grid that shares no factor with the bands per image every CTA
+    // meets all bands of an image in turn (they differ in height: the last one is shorter)
+    int g = sm_count();
+    if (p.items <= g) g = p.items;
+    else
+        while (g > 1 && std::__gcd(g, p.NB) != 1) --g;
+    p.grid = g;
+
+    // ---- tensor maps
+    {
+        // input as a flat list of pixels: [Cin][N*H*W], boxes of 128 pixels
+        const cuuint64_t npx = (cuuint64_t)N * H * W;
+        cuuint64_t dims[2] = {(cuuint64_t)Cin, npx};
+        cuuint64_t str[1] = {(cuuint64_t)Cin * 2};
+        cuuint32_t box[2] = {(cuuint32_t)p.BKc_in, 128};
+        if (!tmap_encode_bf16(&plan->x, 2, dsq.in, dims, str, box, p.rb_in)) return SQN_ERR_CUDA;
+    }
+    {
+        cuuint64_t dims[2] = {(cuuint64_t)Cin, (cuuint64_t)s};
+        cuuint64_t str[1] = {(cuuint64_t)Cin * 2};
+        cuuint32_t box[2] = {(cuuint32_t)p.BKc_in, (cuuint32_t)s};
+        if (!tmap_encode_bf16(&plan->wsq, 2, dsq.w, dims, str, box, p.rb_in)) return SQN_ERR_CUDA;
+    }
+    {
+        cuuint64_t dims[2] = {(cuuint64_t)9 * s, (cuuint64_t)e3};
+        cuuint64_t str[1] = {(cuuint64_t)9 * s * 2};
+        cuuint32_t box[2] = {(cuuint32_t)s, (cuuint32_t)e3};
+        if (!tmap_encode_bf16(&plan->w3, 2, d3.w, dims, str, box, p.rb_s)) return SQN_ERR_CUDA;
+    }
+    {
+        cuuint64_t dims[2] = {(cuuint64_t)s, (cuuint64_t)e1};
+        cuuint64_t str[1] = {(cuuint64_t)s * 2};
+        cuuint32_t box[2] = {(cuuint32_t)s, (cuuint32_t)e1};
+        if (!tmap_encode_bf16(&plan->w1, 2, d1.w, dims, str, box, p.rb_s)) return SQN_ERR_CUDA;
+    }
+    {
+        const cuuint64_t s1 = (cuuint64_t)p.c_tot * 2;
+        cuuint64_t dims[4] = {(cuuint64_t)(e1 + e3), (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
+        cuuint64_t str[3] = {s1, s1 * W, s1 * W * H};
+        cuuint32_t box[4] = {(cuuint32_t)FF_CW, (cuuint32_t)W, (cuuint32_t)p.RT, 1};
+        if (!tmap_encode_bf16(&plan->o, 4, d1.out, dims, str, box, FF_CW * 2)) return SQN_ERR_CUDA;
+    }
+    return SQN_OK;
+}
+
+struct FireKey {
+    const void *in, *wsq, *w1, *w3, *bsq, *b1, *b3, *out;
+    int v[12];
+};
+
+std::mutex g_fire_mu;
+std::map<std::string, FirePlan> g_fire_plans;
+
+}  // namespace
+
+bool fused_fire_enabled()
+{
+    const char* v = std::getenv("SQN_FUSED_FIRE");        // read at every call: tests switch it
+    return !(v && v[0] == '0');
+}
+
+// The whole fire layer in one launch; SQN_ERR_UNSUPPORTED where the kernel does not apply (the caller then launches
+// the squeeze and the expands separately).
+int launch_fire_fused_bf16(const ConvDesc& dsq, const ConvDesc& d1, const ConvDesc& d3, cudaStream_t stream)
+{
+    if (dsq.K != 1 || d1.K != 1 || d3.K != 3 || d3.pad != 1 || dsq.S != 1 || d1.S != 1 || d3.S != 1 || !dsq.relu || !d1.relu ||
+        !d3.relu || dsq.pool || d1.pool || d3.pool || d1.in != dsq.out || d3.in != dsq.out || d1.Cin != dsq.Cout ||
+        d3.Cin != dsq.Cout || d1.H != dsq.H || d1.W != dsq.W || d1.N != dsq.N)
+        return SQN_ERR_UNSUPPORTED;
+    FireKey k;
+    std::memset(&k, 0, sizeof(k));
+    k.in = dsq.in; k.wsq = dsq.w; k.w1 = d1.w; k.w3 = d3.w; k.bsq = dsq.bias; k.b1 = d1.bias; k.b3 = d3.bias; k.out = d1.out;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const int band = band_rows(dsq.H, 128 / (dsq.W + 2) > 0 ? 128 / (dsq.W + 2) : 1);
+    const int v[12] = {dsq.N, dsq.Cin, dsq.H, dsq.W, dsq.Cout, d1.Cout, d3.Cout, d1.out_c_total,
+                       dsq.params_static | (d1.params_static << 1) | (d3.params_static << 2), dev, band, 0};
+    std::memcpy(k.v, v, sizeof(v));
+    const std::string key(reinterpret_cast<const char*>(&k), sizeof(k));
+    FirePlan plan;
+    bool have = false;
+    {
+        std::lock_guard<std::mutex> lock(g_fire_mu);
+        auto it = g_fire_plans.find(key);
+        if (it != g_fire_plans.end()) { plan = it->second; have = true; }
+    }
+    if (!have) {
+        const int rc = build_fire_plan(dsq, d1, d3, &plan);
+        if (rc != SQN_OK) return rc;
+        std::lock_guard<std::mutex> lock(g_fire_mu);
+        if (g_fire_plans.size() > 1024) g_fire_plans.clear();
+        g_fire_plans[key] = plan;
+    }
+    static const cudaError_t attr_rc =
+        cudaFuncSetAttribute(fire_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FF_SMEM_LIMIT);
+    if (attr_rc != cudaSuccess) return SQN_ERR_CUDA;
+    const cudaError_t rc = launch_chained(fire_fused_kernel, dim3((unsigned)plan.p.grid), dim3(FF_THREADS), plan.smem, stream,
+                                          plan.x, plan.wsq, plan.w3, plan.w1, plan.o, plan.p);
+    if (rc != cudaSuccess) return SQN_ERR_CUDA;
+    note_launch();
+    return cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
+}
+
+}  // namespace sqn

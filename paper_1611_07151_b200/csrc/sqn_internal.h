@@ -51,6 +51,11 @@ int launch_stem_conv_bf16_prepacked(const ConvDesc& d, cudaStream_t stream);
 inline int stem_packed_rows(int H) { return (H + 1) / 2 * 2; }
 inline int stem_packed_cols(int W) { return (W + 2) / 2 * 2; }
 
+// The whole fire layer (squeeze, both expands) in one launch, the squeeze map kept in shared memory; SQN_ERR_UNSUPPORTED
+// where that kernel does not apply.  SQN_FUSED_FIRE=0 in the environment turns it off.
+bool fused_fire_enabled();
+int launch_fire_fused_bf16(const ConvDesc& dsq, const ConvDesc& d1, const ConvDesc& d3, cudaStream_t stream);
+
 // Pooling / head.
 int launch_maxpool3x3s2(const void* in, void* out, int C, int H, int W, int N, int dtype, cudaStream_t stream);
 int launch_avgpool_softmax(const void* in, float* logits, float* probs, int C, int H, int W, int N, int dtype,

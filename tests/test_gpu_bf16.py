@@ -204,7 +204,7 @@ def test_config3_headline_batch256_all_images_against_the_oracle():
     x, params = synth.squeezenet_case(3, batch)
     logits, probs, views = run_net_device(x, params, BF16, batch)
     assert "conv1" not in views and "fire4" not in views and "fire8" not in views       # fused with their pools
-    assert {"pool1", "pool4", "pool8", "conv10", "fire2_sq", "fire9"} <= set(views)
+    assert {"pool1", "pool4", "pool8", "conv10", "fire2", "fire6_sq", "fire9"} <= set(views)
     worst_d = {n: 0.0 for n in views}
     worst_r = {n: 0.0 for n in views}
     zs = []
@@ -295,15 +295,27 @@ def test_full_forward_bf16_batch32():
 
 
 def test_full_forward_bf16_small_batch_keeps_every_map():
-    """Below a batch of 16 the pools are separate kernels and every intermediate map can be read back."""
+    """Below a batch of 16 the pools are separate kernels; with SQN_FUSED_FIRE=0 (read at every call) the fire layers
+    are separate launches too and every intermediate map can be read back.  By default the squeeze maps of the fire
+    layers that run as one kernel are not stored, and the logits agree with the separate launches to rounding."""
+    import os
     x, params = synth.squeezenet_case(7, 2)
     trace = {}
     z, _ = ref.squeezenet(x, params, trace=trace)
-    logits, probs, layers = run_net(x, params, BF16, 2)
+    os.environ["SQN_FUSED_FIRE"] = "0"
+    try:
+        logits, probs, layers = run_net(x, params, BF16, 2)
+    finally:
+        os.environ.pop("SQN_FUSED_FIRE", None)
     assert "conv1" in layers and "fire4" in layers and len(layers) == len(trace) - 2      # all but logits, probs
     assert max(G.rel_err(got, trace[name]) for name, got in layers.items()) <= 5e-2
     assert G.rel_err(logits, z) <= TOL
     np.testing.assert_allclose(probs.astype(np.float64).sum(1), 1.0, rtol=0, atol=1e-5)
+    logits_f, _probs, layers_f = run_net(x, params, BF16, 2)
+    assert "fire2_sq" not in layers_f and "fire5_sq" not in layers_f and "fire2" in layers_f and "fire6_sq" in layers_f
+    assert max(G.rel_err(got, trace[name]) for name, got in layers_f.items()) <= 5e-2
+    assert G.rel_err(logits_f, z) <= TOL
+    assert G.rel_err(logits_f, logits) <= 1e-2
 
 
 def test_plain_launches_give_the_same_values():

@@ -1,0 +1,133 @@
+"""The fire layer as one kernel (squeeze map kept in shared memory), bf16, against the fp32 oracle through
+fire_forward.  Bar: max|delta| / max|ref| <= 2e-2 for each expand on its own scale."""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import ref
+from paper_1611_07151_b200 import binding as B
+from paper_1611_07151_b200 import synth
+import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+BF16 = B.SQN_BF16
+TOL = G.TOL[BF16]
+
+
+def _fire_case(seed, batch, cin, s, e1, e3, H, W):
+    rng = np.random.default_rng(seed)
+    x = synth.draw_input(rng, (batch, cin, H, W), "absnormal")
+    sq = synth.draw_conv_params(rng, cin, s, 1)
+    x1 = synth.draw_conv_params(rng, s, e1, 1)
+    x3 = synth.draw_conv_params(rng, s, e3, 3)
+    # biases large enough to matter, some squeeze layers mostly negative (ReLU clips them)
+    sq = (sq[0], sq[1] + np.float32(0.3) * rng.standard_normal(s).astype(np.float32))
+    x1 = (x1[0], x1[1] + np.float32(0.3) * rng.standard_normal(e1).astype(np.float32))
+    x3 = (x3[0], x3[1] + np.float32(0.3) * rng.standard_normal(e3).astype(np.float32))
+    return x, sq, x1, x3
+
+
+def _run(x, sq, x1, x3, fused=True, band=None):
+    N, cin, H, W = x.shape
+    s, e1, e3 = sq[0].shape[0], x1[0].shape[0], x3[0].shape[0]
+    scratch = B.empty_device((N, H, W, s), BF16)
+    scratch.fill_(float("nan"))
+    out = B.empty_device((N, H, W, e1 + e3), BF16)
+    out.fill_(float("nan"))
+    old = {k: os.environ.get(k) for k in ("SQN_FUSED_FIRE", "SQN_FIRE_BAND")}
+    try:
+        os.environ["SQN_FUSED_FIRE"] = "1" if fused else "0"
+        if band is not None:
+            os.environ["SQN_FIRE_BAND"] = str(band)
+        else:
+            os.environ.pop("SQN_FIRE_BAND", None)
+        n0 = B.sqn_launch_count()
+        B.fire_forward(G.dev_act(x, BF16), G.dev_w(sq[0], BF16), G.dev_b(sq[1]), G.dev_w(x1[0], BF16), G.dev_b(x1[1]),
+                       G.dev_w(x3[0], BF16), G.dev_b(x3[1]), scratch, out, cin, s, e1, e3, H, W, N, BF16)
+        assert B.sqn_check() == B.SQN_OK
+        launches = B.sqn_launch_count() - n0
+    finally:
+        for k, v in old.items():
+            if v is None:
+                os.environ.pop(k, None)
+            else:
+                os.environ[k] = v
+    return G.host_act(out, BF16), launches, scratch
+
+
+def _check(got, exp, e1):
+    assert got.shape == exp.shape
+    assert not np.isnan(got).any()
+    assert G.rel_err(got[:, :e1], exp[:, :e1]) <= TOL
+    assert G.rel_err(got[:, e1:], exp[:, e1:]) <= TOL
+    for n in range(got.shape[0]):          # per image: a band written to the wrong place must not hide
+        assert G.rel_err(got[n], exp[n]) <= TOL, n
+
+
+# (batch, Cin, s, e1, e3, H, W)
+SHAPES = [
+    (2, 96, 16, 64, 64, 55, 55),        # fire2: four bands per image, three 32-layer reduction chunks
+    (3, 128, 16, 64, 64, 55, 55),       # fire3
+    (2, 128, 32, 128, 128, 55, 55),     # fire4 (without its pool): both accumulators fill the TMEM
+    (3, 256, 32, 128, 128, 27, 27),     # fire5: two bands of 16 and 11 rows
+    (5, 256, 64, 64, 64, 13, 13),       # 128-byte patch rows, whole image per band, four reduction chunks
+    (2, 64, 16, 64, 64, 9, 20),         # small non-square map
+    (1, 32, 32, 64, 192, 31, 17),       # e1 != e3, odd extents
+    (3, 64, 16, 64, 64, 3, 3),          # smaller than one tile
+    (1, 32, 16, 64, 64, 1, 126),        # one row, widest supported map
+]
+
+
+@pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_fused_fire_matches_the_oracle(shape):
+    N, cin, s, e1, e3, H, W = shape
+    x, sq, x1, x3 = _fire_case(sum(shape), N, cin, s, e1, e3, H, W)
+    exp = ref.fire(x, *sq, *x1, *x3)
+    got, launches, scratch = _run(x, sq, x1, x3)
+    assert launches == 1                                   # one kernel for the whole layer
+    assert bool(scratch.isnan().all())                     # the squeeze map was not stored
+    _check(got, exp, e1)
+    # the three-launch path on the same operands agrees to output rounding (the accumulation order differs)
+    sep, launches, _ = _run(x, sq, x1, x3, fused=False)
+    assert launches >= 2
+    assert G.rel_err(got, sep) <= 1e-2
+
+
+@pytest.mark.parametrize("band", [2, 6, 28, 56])
+def test_fused_fire_band_heights(band):
+    """Any band height gives the same layer: bands of one tile, of many, and the whole image (where it fits)."""
+    N, cin, s, e, H = 2, 96, 16, 64, 55
+    x, sq, x1, x3 = _fire_case(100 + band, N, cin, s, e, e, H, H)
+    exp = ref.fire(x, *sq, *x1, *x3)
+    got, launches, _ = _run(x, sq, x1, x3, band=band)
+    assert launches == 1
+    _check(got, exp, e)
+
+
+def test_fused_fire_many_items_per_cta():
+    """More bands than CTAs: every CTA walks several bands (top, middle and bottom ones of different images), the
+    patch is reused and its border rows are cleared in between."""
+    N, cin, s, e, H = 160, 96, 16, 64, 55                    # 640 bands on at most 148 CTAs
+    x, sq, x1, x3 = _fire_case(7, N, cin, s, e, e, H, H)
+    exp = ref.fire(x, *sq, *x1, *x3)
+    got, launches, _ = _run(x, sq, x1, x3)
+    assert launches == 1
+    _check(got, exp, e)
+    N, cin, s, e, H = 200, 256, 32, 128, 27                  # fire5 shape: 400 bands of 16 and 11 rows
+    x, sq, x1, x3 = _fire_case(8, N, cin, s, e, e, H, H)
+    exp = ref.fire(x, *sq, *x1, *x3)
+    got, launches, _ = _run(x, sq, x1, x3)
+    assert launches == 1
+    _check(got, exp, e)
+
+
+def test_shapes_outside_the_fused_kernel_take_the_separate_launches():
+    """s = 48 (fire6/7) and e1 + e3 > 256 (fire8/9) are not covered by the one-kernel path: fire_forward must still
+    give the layer, with more than one launch."""
+    for (N, cin, s, e, H) in [(2, 256, 48, 192, 27), (2, 512, 64, 256, 13)]:
+        x, sq, x1, x3 = _fire_case(N + s, N, cin, s, e, e, H, H)
+        exp = ref.fire(x, *sq, *x1, *x3)
+        got, launches, scratch = _run(x, sq, x1, x3)
+        assert launches >= 2 and not bool(scratch.isnan().any())
+        _check(got, exp, e)
