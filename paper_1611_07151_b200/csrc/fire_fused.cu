@@ -6,19 +6,23 @@
 // Work item = a band of R output rows of one image.  For a band the CTA
 //   1. squeezes the band's input rows and one halo row above and below (1x1 convolution: rows of the flat pixel
 //      index are the M = 128 operand, read by TMA as they lie in memory; the squeeze kernels stay in shared
-//      memory), and its epilogue warps write the result -- bias added, ReLU, rounded to bf16 -- as a flat array of
+//      memory), and the squeeze epilogue writes the result -- bias added, ReLU, rounded to bf16 -- as a flat array of
 //      pixels with a pitch of P = W + 2 pixels per image row: "the patch".  The two extra columns and the rows
 //      outside the image are the zero padding of the 3x3 expand and stay zero;
 //   2. runs both expands on the patch.  Output tile t = RT image rows = RT*P <= 128 consecutive patch pixels (the two
 //      padding pixels of every row compute garbage that is never stored).  Kernel tap (kh, kw) of the 3x3 expand is
 //      one MMA whose A descriptor starts (kh*P + kw) pixels further into the patch; the 1x1 expand is the centre
-//      tap, so its kernels are appended to the centre tap's and one MMA of N = e3 + e1 serves both.  The accumulator
-//      holds e3 + e1 <= 256 columns; the epilogue converts it chunk by chunk into a staging tile of RT rows x W
-//      pixels (the padding pixels dropped) that one TMA store sends to the layer slices of the output tensor.
-// The jobs of a CTA -- squeeze tiles, then expand tiles, item after item -- alternate between two TMEM accumulators
-// and are drained in issue order, so the epilogue of one job overlaps the MMAs of the next, and the squeeze epilogue
-// of the next band cannot overwrite the patch before the expand MMAs of this band have read it.
-// Warps: 0 TMA producer (input tiles; all kernels once), 1 MMA issuer, 2..9 epilogue, 10 TMA stores.
+//      tap.  Where both expands fit one accumulator twice over, the 1x1 kernels are appended to the centre tap's and
+//      one MMA of N = e3 + e1 serves both (one job per tile); else the 3x3 and the 1x1 expand of a tile are two jobs.
+//      The expand epilogue converts an accumulator chunk by chunk into staging tiles of RT rows x W pixels (the
+//      padding pixels dropped) that TMA stores send to the layer slices of the output tensor.
+// The two steps are two pipelines that run side by side, each with its own MMA issuer, TMEM accumulators and
+// epilogue warps -- issuing an MMA costs tens of clocks whatever its size, and with the small N of these layers one
+// issuing thread would be the limit:
+//   squeeze:  TMA producer -> input ring -> squeeze issuer -> 2 accumulators -> 4 epilogue warps -> patch
+//   expand:   patch -> expand issuer -> 2 or 3 accumulators -> 8 epilogue warps -> staging ring -> store warp
+// With two patches (where shared memory allows) the squeeze pipeline works on the CTA's next band while the expand
+// pipeline works on this one; patch_ready / patch_free barriers hand a patch back and forth.
 // Every mbarrier wait is bounded (see wait_bar).
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -40,11 +44,13 @@ namespace {
 
 using namespace ptx;
 
-constexpr int FF_EPI_WARPS = 8;
-constexpr int FF_THREADS = 32 * (2 + FF_EPI_WARPS + 1);
+constexpr int FF_SEPI_WARPS = 4;           // squeeze epilogue warps (one per TMEM lane quadrant)
+constexpr int FF_EEPI_WARPS = 8;           // expand epilogue warps (two per quadrant)
+constexpr int FF_THREADS = 32 * (4 + FF_SEPI_WARPS + FF_EEPI_WARPS);     // + producer, two issuers, store warp
 constexpr int FF_MAX_STAGES = 8;
 constexpr int FF_MAX_STG = 4;
-constexpr int FF_MAX_EMMA = 40;            // MMAs of one expand tile: 9 taps x at most 4 k-steps, + spare
+constexpr int FF_MAX_EMMA = 48;            // MMAs of one expand tile: 10 taps x at most 4 k-steps, + spare
+constexpr int FF_MAX_ESLOTS = 3;
 constexpr size_t FF_SMEM_LIMIT = 227 * 1024;
 constexpr int FF_CW = 64;                  // output layers per store chunk
 
@@ -55,10 +61,16 @@ struct FireParams {
     int items, grid;
     int chunks_in, BKc_in, ksteps_in;   // squeeze reduction: chunks, elements per chunk, MMAs per chunk
     int ksteps_s;                    // MMAs per expand tap (s / 16)
-    int n_emma;                      // MMAs of an expand tile (without the bias MMA)
-    int nchunks;                     // store chunks per expand tile ((e3 + e1) / FF_CW)
     int stages, nstg;
-    int slot_cols;                   // TMEM columns per accumulator
+    int two_patches;
+    // expand jobs of a tile: one (both expands in one accumulator) or two (3x3, then 1x1)
+    int njobs;
+    int job_e0[2], job_en[2];        // the job's MMAs: entries [e0, en) of etab
+    int job_chunk0[2], job_nchunks[2];   // its store chunks (chunk c = accumulator-order columns [64c, 64c + 64))
+    unsigned job_bias16[2];          // its bias rows, in 16-byte units from off_bias_e
+    unsigned job_idesc[2];           // instruction descriptor of its bias MMA (all of its columns)
+    int s_slot_cols;                 // TMEM: two squeeze accumulators of s_slot_cols columns, then eslots expand
+    int eslots, eslot_cols;          //       accumulators of eslot_cols columns
     unsigned tmem_cols;
     int c_tot;                       // layers per pixel of the output tensor
     int b_early;                     // kernels and bias may be fetched before the wait for the grid ahead
@@ -68,22 +80,23 @@ struct FireParams {
     unsigned off_wsq, wsq_tile;      // squeeze kernels: chunks_in tiles of s rows
     unsigned off_we;                 // expand kernels: centre tap, 1x1, then the other eight taps
     unsigned off_tap[9], off_w1;     // ... offsets of the tiles from off_we
-    unsigned off_patch, patch_bytes;
+    unsigned off_patch, patch_bytes; // one or two patches of patch_bytes each
     unsigned off_x, x_tile;
     unsigned off_stg, stg_slot;
     unsigned off_bias_s, off_bias_e, off_ones, off_ctl;
     const float *bias_sq, *bias_e1, *bias_e3;
     int* status;
     uint2 etab[FF_MAX_EMMA];         // per expand MMA: {A offset from the tile's first patch pixel, B offset from off_we}, 16-byte units
+    unsigned eidesc[FF_MAX_EMMA];    // ... and its instruction descriptor (N differs between the MMAs of a job)
 };
 
 struct FireShared {
     unsigned long long full[FF_MAX_STAGES];
     unsigned long long empty[FF_MAX_STAGES];
     unsigned long long w_full;
-    unsigned long long tmem_full[2];
-    unsigned long long tmem_empty[2];
-    unsigned long long patch_ready;
+    unsigned long long s_full[2], s_empty[2];
+    unsigned long long e_full[FF_MAX_ESLOTS], e_empty[FF_MAX_ESLOTS];
+    unsigned long long patch_ready[2], patch_free[2];
     unsigned long long stg_full[FF_MAX_STG];
     unsigned long long stg_free[FF_MAX_STG];
     unsigned tmem_base;
@@ -130,6 +143,18 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
+// 16 accumulator columns -> ReLU, bf16 -> two 16-byte units at unit index u0, u0 + 1 of a swizzled row
+__device__ __forceinline__ void store16(const uint32_t* v, uint32_t rbase, uint32_t u0, uint32_t sw)
+{
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+        uint32_t o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) o[j] = pack_relu_bf16x2(__uint_as_float(v[8 * u + 2 * j]), __uint_as_float(v[8 * u + 2 * j + 1]));
+        st_shared_v4(rbase + (((u0 + (uint32_t)u) ^ sw) << 4), o[0], o[1], o[2], o[3]);
+    }
+}
+
 __global__ void __launch_bounds__(FF_THREADS, 1)
 fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmWsq,
                   const __grid_constant__ CUtensorMap tmW3, const __grid_constant__ CUtensorMap tmW1,
@@ -146,6 +171,7 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int bid = (int)blockIdx.x;
+    const int nbuf = p.two_patches ? 2 : 1;
 
     auto load_kernels = [&]() {          // every kernel tile of the layer, once (one mbarrier counts them all)
         const uint32_t bar = smem_u32(&sh->w_full);
@@ -172,12 +198,17 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         }
         mbar_init(smem_u32(&sh->w_full), 1);
         for (int a = 0; a < 2; ++a) {
-            mbar_init(smem_u32(&sh->tmem_full[a]), 1);
-            mbar_init(smem_u32(&sh->tmem_empty[a]), FF_EPI_WARPS);
+            mbar_init(smem_u32(&sh->s_full[a]), 1);
+            mbar_init(smem_u32(&sh->s_empty[a]), FF_SEPI_WARPS);
+            mbar_init(smem_u32(&sh->patch_ready[a]), FF_SEPI_WARPS);
+            mbar_init(smem_u32(&sh->patch_free[a]), 1);
         }
-        mbar_init(smem_u32(&sh->patch_ready), FF_EPI_WARPS);
+        for (int a = 0; a < FF_MAX_ESLOTS; ++a) {
+            mbar_init(smem_u32(&sh->e_full[a]), 1);
+            mbar_init(smem_u32(&sh->e_empty[a]), FF_EEPI_WARPS);
+        }
         for (int b = 0; b < p.nstg; ++b) {
-            mbar_init(smem_u32(&sh->stg_full[b]), FF_EPI_WARPS);
+            mbar_init(smem_u32(&sh->stg_full[b]), FF_EEPI_WARPS);
             mbar_init(smem_u32(&sh->stg_free[b]), 1);
         }
         sh->abort_flag = 0;
@@ -194,8 +225,9 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         tmem_relinquish();
         chain_release();            // (only once this CTA holds its TMEM: see conv_tc_body)
     }
-    // the patch starts as zeros: its two padding columns and the rows outside the image are never written
-    for (uint32_t i = threadIdx.x; i < p.patch_bytes / 16u; i += FF_THREADS) st_shared_v4(smPatch + 16u * i, 0u, 0u, 0u, 0u);
+    // the patches start as zeros: their two padding columns and the rows outside the image are never written
+    for (uint32_t i = threadIdx.x; i < (uint32_t)nbuf * p.patch_bytes / 16u; i += FF_THREADS)
+        st_shared_v4(smPatch + 16u * i, 0u, 0u, 0u, 0u);
     {
         // tile of ones for the bias MMAs: 128 rows of 32 bytes in the 32-byte swizzle, ones in the first two places
         uint4* ones = reinterpret_cast<uint4*>(base_ptr + p.off_ones);
@@ -214,6 +246,7 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     tc_fence_after();
     const uint32_t tmem_base = sh->tmem_base;
     volatile int* abort_flag = &sh->abort_flag;
+    const uint32_t tmem_e = tmem_base + (uint32_t)(2 * p.s_slot_cols);      // first expand accumulator
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer: input tiles of the squeeze
@@ -249,30 +282,23 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
+        // ------------------------------------------------------------------ squeeze issuer
         // The whole warp walks the loops converged; one elected lane issues the MMAs and their commits.
         const uint32_t idesc_s = make_idesc_bf16(128, (uint32_t)p.s);
-        const uint32_t idesc_c = make_idesc_bf16(128, (uint32_t)(p.e3 + p.e1));
-        const uint32_t idesc_3 = make_idesc_bf16(128, (uint32_t)p.e3);
         const uint32_t hi_in = (uint32_t)(make_kmajor_desc(0, p.rb_in, 8u * p.rb_in) >> 32);
-        const uint32_t hi_s = (uint32_t)(make_kmajor_desc(0, p.rb_s, 8u * p.rb_s) >> 32);
         const uint64_t ones_desc = make_kmajor_desc(base + p.off_ones, 32u, 256u);
         const uint64_t bias_s_desc = make_kmajor_desc(base + p.off_bias_s, 32u, 256u);
-        const uint64_t bias_e_desc = make_kmajor_desc(base + p.off_bias_e, 32u, 256u);
         const uint32_t smX16 = smX >> 4, x_tile16 = p.x_tile >> 4, smWsq16 = smWsq >> 4, wsq_tile16 = p.wsq_tile >> 4;
-        const uint32_t smWe16 = smWe >> 4, patch16 = smPatch >> 4;
-        const uint32_t tile_step16 = ((uint32_t)(p.RT * p.P) * p.rb_s) >> 4;      // patch units between expand tiles
         bool ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->w_full), 0u, abort_flag, p.status));
         int st = 0, as = 0;
-        uint32_t ph = 0, aph = 0, pph = 0;
+        uint32_t ph = 0, aph = 0;
         for (int item = bid; item < p.items && ok; item += p.grid) {
             const Band b = band_of(p, item);
-            // squeeze tiles
             for (int t = 0; t < b.n_s && ok; ++t) {
-                ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_empty[as]), aph ^ 1u, abort_flag, p.status));
+                ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->s_empty[as]), aph ^ 1u, abort_flag, p.status));
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(as * p.slot_cols);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(as * p.s_slot_cols);
                 for (int ch = 0; ch < p.chunks_in; ++ch) {
                     ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->full[st]), ph, abort_flag, p.status));
                     if (!ok) break;
@@ -280,12 +306,16 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
                     if (elect_one()) {
                         const uint64_t da = ((uint64_t)hi_in << 32) | (uint64_t)((smX16 + (uint32_t)st * x_tile16) | 0x10000u);
                         const uint64_t db = ((uint64_t)hi_in << 32) | (uint64_t)((smWsq16 + (uint32_t)ch * wsq_tile16) | 0x10000u);
-                        for (int k = 0; k < p.ksteps_in; ++k)
-                            mma_bf16_ss(d_tmem, da + 2u * k, db + 2u * k, idesc_s, (ch | k) ? 1u : 0u);
+                        mma_bf16_ss(d_tmem, da, db, idesc_s, ch ? 1u : 0u);
+                        mma_bf16_ss(d_tmem, da + 2u, db + 2u, idesc_s, 1u);
+                        if (p.ksteps_in == 4) {
+                            mma_bf16_ss(d_tmem, da + 4u, db + 4u, idesc_s, 1u);
+                            mma_bf16_ss(d_tmem, da + 6u, db + 6u, idesc_s, 1u);
+                        }
                         mma_commit(smem_u32(&sh->empty[st]));           // input slot free once these MMAs have read it
                         if (ch == p.chunks_in - 1) {
                             mma_bf16_ss(d_tmem, ones_desc, bias_s_desc, idesc_s, 1u);
-                            mma_commit(smem_u32(&sh->tmem_full[as]));
+                            mma_commit(smem_u32(&sh->s_full[as]));
                         }
                     }
                     __syncwarp();
@@ -294,157 +324,65 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
                 if (!ok) break;
                 if (++as == 2) { as = 0; aph ^= 1u; }
             }
-            if (!ok) break;
-            // the patch of this band is complete once every epilogue warp has passed its last squeeze tile
-            ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->patch_ready), pph, abort_flag, p.status));
-            if (!ok) break;
-            pph ^= 1u;
-            tc_fence_after();
-            // expand tiles
-            for (int t = 0; t < b.n_e; ++t) {
-                ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_empty[as]), aph ^ 1u, abort_flag, p.status));
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(as * p.slot_cols);
-                const uint32_t a_base = patch16 + (uint32_t)t * tile_step16;
-                if (elect_one()) {
-                    uint32_t acc = 0u;
-#pragma unroll 2
-                    for (int e = 0; e < p.n_emma; ++e) {
-                        const uint2 o = p.etab[e];
-                        // the centre tap comes first and carries the 1x1 expand's kernels: N = e3 + e1
-                        mma_bf16_ss(d_tmem, ((uint64_t)hi_s << 32) | (uint64_t)((a_base + o.x) | 0x10000u),
-                                    ((uint64_t)hi_s << 32) | (uint64_t)((smWe16 + o.y) | 0x10000u),
-                                    e < p.ksteps_s ? idesc_c : idesc_3, acc);
-                        acc = 1u;
-                    }
-                    mma_bf16_ss(d_tmem, ones_desc, bias_e_desc, idesc_c, 1u);
-                    mma_commit(smem_u32(&sh->tmem_full[as]));
-                }
-                __syncwarp();
-                if (++as == 2) { as = 0; aph ^= 1u; }
-            }
         }
-    } else if (warp < 2 + FF_EPI_WARPS) {
-        // -------------------------------------------------------------------- epilogue
-        // warp w reads TMEM lane quadrant w % 4 (one M row per thread); the two warps of a quadrant split the columns.
-        const int q = warp & 3, hf = (warp - 2) >> 2;
-        const int row = q * 32 + lane;
-        const uint32_t lane_base = (uint32_t)(q * 32) << 16;
-        const int eidx = (warp - 2) * 32 + lane;                 // index among the 256 epilogue threads
-        // expand tiles: M row -> (image row r of the tile, patch column c); the staging tile drops the padding columns
-        const int r_e = row / p.P, c_e = row - r_e * p.P;
-        const bool e_valid = c_e < p.W && r_e < p.RT;
-        const uint32_t stg_row = (uint32_t)(r_e * p.W + c_e);
-        const uint32_t stg_off = stg_row * (uint32_t)(FF_CW * 2);
-        const uint32_t sw_e = stg_row & 7u;
-        const int hs = p.s >> 1;                                 // squeeze columns per thread: 8, 16 or 32
-        const uint32_t units_s = (uint32_t)hs >> 3;             // ... = this many 16-byte units of a patch row
-        bool ok = true;
-        int as = 0, sb = 0;
-        uint32_t aph = 0, sph = 0;
-        for (int item = bid; item < p.items && ok; item += p.grid) {
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ expand issuer
+        const uint32_t hi_s = (uint32_t)(make_kmajor_desc(0, p.rb_s, 8u * p.rb_s) >> 32);
+        const uint64_t ones_desc = make_kmajor_desc(base + p.off_ones, 32u, 256u);
+        const uint64_t bias_e_desc = make_kmajor_desc(base + p.off_bias_e, 32u, 256u);
+        const uint32_t smWe16 = smWe >> 4, patch16 = smPatch >> 4;
+        const uint32_t tile_step16 = ((uint32_t)(p.RT * p.P) * p.rb_s) >> 4;      // patch units between expand tiles
+        bool ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->w_full), 0u, abort_flag, p.status));
+        int es = 0;
+        uint32_t eph = 0;
+        int j = 0;                              // band count of this CTA
+        for (int item = bid; item < p.items && ok; item += p.grid, ++j) {
             const Band b = band_of(p, item);
-            for (int t = 0; t < b.n_s; ++t) {
-                ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_full[as]), aph, abort_flag, p.status));
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t ta = tmem_base + lane_base + (uint32_t)(as * p.slot_cols + hf * hs);
-                uint32_t v[32];
-                if (hs == 32) {
-                    tmem_ld_x16(ta, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
-                    tmem_ld_x16(ta + 16u, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
-                } else if (hs == 16) {
-                    tmem_ld_x16(ta, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
-                } else {
-                    tmem_ld_x8(ta, *reinterpret_cast<uint32_t(*)[8]>(&v[0]));
-                }
-                tmem_ld_wait();
-                // accumulator in registers: hand it back to the MMA issuer
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[as]));
-                if (++as == 2) { as = 0; aph ^= 1u; }
-                const int g = t * 128 + row;                      // pixel of the band's input rows
-                if (g < b.npx) {
-                    const int yy = g / p.W, xx = g - yy * p.W;
-                    const uint32_t pr = (uint32_t)((yy + b.ylo - b.y0 + 1) * p.P + xx + 1);
-                    const uint32_t rbase = smPatch + pr * p.rb_s;
-                    const uint32_t sw = swz(pr, p.rb_s);
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        if ((uint32_t)u < units_s) {
-                            uint32_t o[4];
-#pragma unroll
-                            for (int j = 0; j < 4; ++j)
-                                o[j] = pack_relu_bf16x2(__uint_as_float(v[8 * u + 2 * j]), __uint_as_float(v[8 * u + 2 * j + 1]));
-                            st_shared_v4(rbase + ((((uint32_t)hf * units_s + (uint32_t)u) ^ sw) << 4), o[0], o[1], o[2], o[3]);
-                        }
-                    }
-                }
-            }
+            const int buf = j % nbuf;
+            // the band's patch is complete once every squeeze epilogue warp has passed the band's last squeeze tile
+            ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->patch_ready[buf]), (uint32_t)(j / nbuf) & 1u, abort_flag, p.status));
             if (!ok) break;
-            // patch rows that lie outside the image (above the first band, below the last) hold what an earlier band left
-            {
-                const uint32_t row_units = ((uint32_t)p.P * p.rb_s) >> 4;
-                if (b.y0 == 0)
-                    for (uint32_t i = (uint32_t)eidx; i < row_units; i += 32u * FF_EPI_WARPS) st_shared_v4(smPatch + 16u * i, 0u, 0u, 0u, 0u);
-                if (b.y0 + b.rows == p.H) {
-                    const uint32_t a0 = smPatch + (uint32_t)((b.rows + 1) * p.P) * p.rb_s;
-                    for (uint32_t i = (uint32_t)eidx; i < row_units; i += 32u * FF_EPI_WARPS) st_shared_v4(a0 + 16u * i, 0u, 0u, 0u, 0u);
-                }
-            }
-            fence_proxy_async_smem();             // patch visible to the tensor core
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sh->patch_ready));
-            for (int t = 0; t < b.n_e; ++t) {
-                ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_full[as]), aph, abort_flag, p.status));
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t ta0 = tmem_base + lane_base + (uint32_t)(as * p.slot_cols + hf * 32);
-                for (int chunk = 0; chunk < p.nchunks; ++chunk) {
-                    uint32_t v[32];
-                    const uint32_t ta = ta0 + (uint32_t)(chunk * FF_CW);
-                    tmem_ld_x16(ta, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
-                    tmem_ld_x16(ta + 16u, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
-                    ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->stg_free[sb]), sph ^ 1u, abort_flag, p.status));
-                    tmem_ld_wait();
+            tc_fence_after();
+            for (int t = 0; t < b.n_e && ok; ++t) {
+                const uint32_t a_base = patch16 + (uint32_t)buf * (p.patch_bytes >> 4) + (uint32_t)t * tile_step16;
+                for (int job = 0; job < p.njobs; ++job) {
+                    ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->e_empty[es]), eph ^ 1u, abort_flag, p.status));
                     if (!ok) break;
-                    if (e_valid) {
-                        const uint32_t rbase = smStg + (uint32_t)sb * p.stg_slot + stg_off;
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            uint32_t o[4];
-#pragma unroll
-                            for (int j = 0; j < 4; ++j)
-                                o[j] = pack_relu_bf16x2(__uint_as_float(v[8 * u + 2 * j]), __uint_as_float(v[8 * u + 2 * j + 1]));
-                            st_shared_v4(rbase + ((((uint32_t)hf * 4u + (uint32_t)u) ^ sw_e) << 4), o[0], o[1], o[2], o[3]);
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_e + (uint32_t)(es * p.eslot_cols);
+                    if (elect_one()) {
+                        uint32_t acc = 0u;
+                        const int en = p.job_en[job];
+#pragma unroll 2
+                        for (int e = p.job_e0[job]; e < en; ++e) {
+                            const uint2 o = p.etab[e];
+                            mma_bf16_ss(d_tmem, ((uint64_t)hi_s << 32) | (uint64_t)((a_base + o.x) | 0x10000u),
+                                        ((uint64_t)hi_s << 32) | (uint64_t)((smWe16 + o.y) | 0x10000u), p.eidesc[e], acc);
+                            acc = 1u;
                         }
+                        mma_bf16_ss(d_tmem, ones_desc, bias_e_desc + (uint64_t)p.job_bias16[job], p.job_idesc[job], 1u);
+                        mma_commit(smem_u32(&sh->e_full[es]));
+                        // after the band's last job: the patch may be overwritten once these MMAs have read it
+                        if (t == b.n_e - 1 && job == p.njobs - 1) mma_commit(smem_u32(&sh->patch_free[buf]));
                     }
-                    fence_proxy_async_smem();             // staging rows visible to the TMA unit
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&sh->stg_full[sb]));
-                    if (++sb == p.nstg) { sb = 0; sph ^= 1u; }
+                    if (++es == p.eslots) { es = 0; eph ^= 1u; }
                 }
-                if (!ok) break;
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[as]));
-                if (++as == 2) { as = 0; aph ^= 1u; }
             }
         }
-    } else {
+    } else if (warp == 3) {
         // ----------------------------------------------------------------- store issuer
         if (lane == 0) {
             bool ok = true;
             int sb = 0, pend = 0, fb = 0;       // next slot, stores whose slot is not yet released, next slot to release
             uint32_t sph = 0;
+            const int nchunks = p.job_chunk0[p.njobs - 1] + p.job_nchunks[p.njobs - 1];
             for (int item = bid; item < p.items && ok; item += p.grid) {
                 const Band b = band_of(p, item);
                 for (int t = 0; t < b.n_e && ok; ++t)
-                    for (int chunk = 0; chunk < p.nchunks; ++chunk) {
+                    for (int chunk = 0; chunk < nchunks; ++chunk) {
                         if (!wait_bar(smem_u32(&sh->stg_full[sb]), sph, abort_flag, p.status)) { ok = false; break; }
-                        // accumulator columns [0, e3) are the 3x3 expand (output layers e1 ..), the rest the 1x1 expand
+                        // accumulator-order columns [0, e3) are the 3x3 expand (output layers e1 ..), the rest the 1x1 expand
                         const int col = chunk * FF_CW;
                         const int cc = col < p.e3 ? p.e1 + col : col - p.e3;
                         tma_store_4d(&tmO, smStg + (uint32_t)sb * p.stg_slot, cc, 0, b.y0 + t * p.RT, b.n);
@@ -461,6 +399,120 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
                     }
             }
             tma_store_wait_all();
+        }
+    } else if (warp < 4 + FF_SEPI_WARPS) {
+        // -------------------------------------------------------------------- squeeze epilogue
+        // warp w reads TMEM lane quadrant w % 4: one input pixel per thread, all s layers of it
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(q * 32) << 16;
+        const int sidx = (warp - 4) * 32 + lane;                 // index among the squeeze epilogue threads
+        bool ok = true;
+        int as = 0, j = 0;
+        uint32_t aph = 0;
+        for (int item = bid; item < p.items && ok; item += p.grid, ++j) {
+            const Band b = band_of(p, item);
+            const int buf = j % nbuf;
+            const uint32_t patch = smPatch + (uint32_t)buf * p.patch_bytes;
+            for (int t = 0; t < b.n_s; ++t) {
+                ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->s_full[as]), aph, abort_flag, p.status));
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t ta = tmem_base + lane_base + (uint32_t)(as * p.s_slot_cols);
+                uint32_t v[64];
+                tmem_ld_x16(ta, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
+                if (p.s >= 32) tmem_ld_x16(ta + 16u, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
+                if (p.s == 64) {
+                    tmem_ld_x16(ta + 32u, *reinterpret_cast<uint32_t(*)[16]>(&v[32]));
+                    tmem_ld_x16(ta + 48u, *reinterpret_cast<uint32_t(*)[16]>(&v[48]));
+                }
+                tmem_ld_wait();
+                // accumulator in registers: hand it back to the issuer
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sh->s_empty[as]));
+                if (++as == 2) { as = 0; aph ^= 1u; }
+                if (t == 0 && j >= nbuf) {
+                    // the expand MMAs of the band that used this patch before must have read it
+                    ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->patch_free[buf]), (uint32_t)(j / nbuf - 1) & 1u, abort_flag, p.status));
+                    if (!ok) break;
+                }
+                const int g = t * 128 + row;                      // pixel of the band's input rows
+                if (g < b.npx) {
+                    const int yy = g / p.W, xx = g - yy * p.W;
+                    const uint32_t pr = (uint32_t)((yy + b.ylo - b.y0 + 1) * p.P + xx + 1);
+                    const uint32_t rbase = patch + pr * p.rb_s;
+                    const uint32_t sw = swz(pr, p.rb_s);
+                    store16(&v[0], rbase, 0u, sw);
+                    if (p.s >= 32) store16(&v[16], rbase, 2u, sw);
+                    if (p.s == 64) {
+                        store16(&v[32], rbase, 4u, sw);
+                        store16(&v[48], rbase, 6u, sw);
+                    }
+                }
+            }
+            if (!ok) break;
+            {
+                // patch rows that lie outside the image (above its first band, below its last) hold what an earlier band left
+                const uint32_t row_units = ((uint32_t)p.P * p.rb_s) >> 4;
+                if (b.y0 == 0)
+                    for (uint32_t i = (uint32_t)sidx; i < row_units; i += 32u * FF_SEPI_WARPS) st_shared_v4(patch + 16u * i, 0u, 0u, 0u, 0u);
+                if (b.y0 + b.rows == p.H) {
+                    const uint32_t a0 = patch + (uint32_t)((b.rows + 1) * p.P) * p.rb_s;
+                    for (uint32_t i = (uint32_t)sidx; i < row_units; i += 32u * FF_SEPI_WARPS) st_shared_v4(a0 + 16u * i, 0u, 0u, 0u, 0u);
+                }
+            }
+            fence_proxy_async_smem();             // patch visible to the tensor core
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->patch_ready[buf]));
+        }
+    } else {
+        // -------------------------------------------------------------------- expand epilogue
+        // warp w reads TMEM lane quadrant w % 4 (one M row per thread); the two warps of a quadrant split a chunk's columns
+        const int q = warp & 3, hf = (warp - 4 - FF_SEPI_WARPS) >> 2;
+        const int row = q * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(q * 32) << 16;
+        // M row -> (image row r of the tile, patch column c); the staging tile drops the padding columns
+        const int r_e = row / p.P, c_e = row - r_e * p.P;
+        const bool e_valid = c_e < p.W && r_e < p.RT;
+        const uint32_t stg_row = (uint32_t)(r_e * p.W + c_e);
+        const uint32_t stg_off = stg_row * (uint32_t)(FF_CW * 2);
+        const uint32_t sw_e = stg_row & 7u;
+        bool ok = true;
+        int es = 0, sb = 0;
+        uint32_t eph = 0, sph = 0;
+        for (int item = bid; item < p.items && ok; item += p.grid) {
+            const Band b = band_of(p, item);
+            for (int t = 0; t < b.n_e && ok; ++t)
+                for (int job = 0; job < p.njobs; ++job) {
+                    ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->e_full[es]), eph, abort_flag, p.status));
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t ta0 = tmem_e + lane_base + (uint32_t)(es * p.eslot_cols + hf * 32);
+                    for (int chunk = 0; chunk < p.job_nchunks[job]; ++chunk) {
+                        uint32_t v[32];
+                        const uint32_t ta = ta0 + (uint32_t)(chunk * FF_CW);
+                        tmem_ld_x16(ta, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
+                        tmem_ld_x16(ta + 16u, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
+                        ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->stg_free[sb]), sph ^ 1u, abort_flag, p.status));
+                        tmem_ld_wait();
+                        if (!ok) break;
+                        if (e_valid) {
+                            const uint32_t rbase = smStg + (uint32_t)sb * p.stg_slot + stg_off;
+                            store16(&v[0], rbase, (uint32_t)hf * 4u, sw_e);
+                            store16(&v[16], rbase, (uint32_t)hf * 4u + 2u, sw_e);
+                        }
+                        fence_proxy_async_smem();             // staging rows visible to the TMA unit
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&sh->stg_full[sb]));
+                        if (++sb == p.nstg) { sb = 0; sph ^= 1u; }
+                    }
+                    if (!ok) break;
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&sh->e_empty[es]));
+                    if (++es == p.eslots) { es = 0; eph ^= 1u; }
+                }
         }
     }
 
@@ -482,19 +534,100 @@ struct FirePlan {
 
 inline size_t up1k(size_t v) { return (v + 1023) / 1024 * 1024; }
 
-// Rows per band: SQN_FIRE_BAND in the environment (tuning aid, read at every call), else 14 rows for maps of 40 rows
-// and more (equal bands for 55 rows), 16 rows from 20 rows on (a smaller patch leaves room for a deeper input ring),
-// else the whole image.
-int band_rows(int H, int RT)
+// Shared-memory layout for one choice of band height R, number of patches (2: squeeze of the next band overlaps the
+// expands of this one; 1: they take turns) and input chunk width.  Returns the input ring's depth (0: does not fit).
+int fire_layout(FireParams& p, int R, int patches, int BKc_in, size_t* smem_bytes)
 {
-    int R = H >= 40 ? 14 : H >= 20 ? 16 : H;
+    const int s = p.s, e1 = p.e1, e3 = p.e3, W = p.W, H = p.H;
+    p.R = R;
+    p.NB = (H + R - 1) / R;
+    p.items = p.N * p.NB;
+    p.two_patches = patches == 2 ? 1 : 0;
+    p.BKc_in = BKc_in;
+    p.chunks_in = p.Cin / BKc_in;
+    p.ksteps_in = BKc_in / 16;
+    p.rb_in = (unsigned)BKc_in * 2u;
+    p.x_bytes = 128u * p.rb_in;
+    size_t cur = 0;
+    p.off_wsq = 0;
+    p.wsq_tile = (unsigned)up1k((size_t)s * p.rb_in);
+    cur += (size_t)p.chunks_in * p.wsq_tile;
+    p.off_we = (unsigned)cur;
+    {
+        // centre tap, then the 1x1 expand's kernels directly behind it (one B operand of e3 + e1 rows), then the others
+        const unsigned t3 = (unsigned)e3 * p.rb_s, t1 = (unsigned)e1 * p.rb_s;
+        if (t3 % 1024u != 0) return 0;          // the appended tile must continue the swizzle pattern
+        unsigned o = 0;
+        p.off_tap[4] = o; o += t3;
+        p.off_w1 = o; o += (unsigned)up1k(t1);
+        for (int tap = 0; tap < 9; ++tap)
+            if (tap != 4) { p.off_tap[tap] = o; o += t3; }
+        cur += o;
+        p.w_bytes = (unsigned)((size_t)p.chunks_in * s * p.rb_in + 9u * t3 + t1);
+        if (p.w_bytes >= (1u << 20)) return 0;  // one mbarrier transaction count
+    }
+    p.off_patch = (unsigned)cur;
+    {
+        const int t_max = R / p.RT;
+        size_t rows = (size_t)(R + 2) * p.P;
+        const size_t reach = (size_t)(t_max - 1) * p.RT * p.P + 2 * p.P + 2 + 128;     // last row an expand MMA reads
+        if (reach > rows) rows = reach;
+        p.patch_bytes = (unsigned)up1k(rows * p.rb_s);
+        cur += (size_t)patches * p.patch_bytes;
+    }
+    p.off_bias_s = (unsigned)cur; cur += up1k((size_t)s * 32);
+    p.off_bias_e = (unsigned)cur; cur += up1k((size_t)(e1 + e3) * 32);
+    p.off_ones = (unsigned)cur; cur += 128 * 32;
+    p.off_ctl = (unsigned)cur; cur += 1024;
+    static_assert(sizeof(FireShared) <= 1024, "control block");
+    p.stg_slot = (unsigned)up1k((size_t)p.RT * W * FF_CW * 2);
+    p.x_tile = (unsigned)up1k(p.x_bytes);
+    const size_t fixed = 1024 /*alignment slack*/ + cur;
+    if (fixed + 2 * p.stg_slot + 2 * p.x_tile > FF_SMEM_LIMIT) return 0;
+    // input ring first (it feeds the memory-bound part), then staging slots
+    size_t left = FF_SMEM_LIMIT - fixed;
+    p.nstg = 2;
+    left -= 2 * p.stg_slot;
+    int stages = (int)(left / p.x_tile);
+    // with room to spare, two more staging slots are worth more than input slots beyond what covers the memory latency
+    const int want = 2 * p.chunks_in > 4 ? 2 * p.chunks_in : 4;
+    if (stages >= want + (int)(2 * p.stg_slot / p.x_tile) + 1) {
+        p.nstg = 4;
+        left -= 2 * p.stg_slot;
+        stages = (int)(left / p.x_tile);
+    }
+    if (stages > FF_MAX_STAGES) stages = FF_MAX_STAGES;
+    if (stages < 2) return 0;
+    p.stages = stages;
+    p.off_x = (unsigned)cur; cur += (size_t)stages * p.x_tile;
+    p.off_stg = (unsigned)cur; cur += (size_t)p.nstg * p.stg_slot;
+    *smem_bytes = 1024 + cur;
+    return *smem_bytes <= FF_SMEM_LIMIT ? stages : 0;
+}
+
+// Band heights to try, best first: SQN_FIRE_BAND in the environment (tuning aid, read at every call) names one;
+// else 14 rows for maps of 40 rows and more (four equal bands for 55 rows), 12 for 20 rows and more, else the whole
+// image.  A band is a whole number of expand tiles.
+int band_candidates(int H, int RT, int* out)
+{
+    int n = 0;
+    auto add = [&](int R) {
+        if (R > H) R = H;
+        R = (R + RT - 1) / RT * RT;
+        for (int i = 0; i < n; ++i)
+            if (out[i] == R) return;
+        out[n++] = R;
+    };
     if (const char* v = std::getenv("SQN_FIRE_BAND")) {
         const int r = std::atoi(v);
-        if (r > 0) R = r;
+        if (r > 0) { add(r); return n; }
     }
-    if (R > H) R = H;
-    R = (R + RT - 1) / RT * RT;          // a band is a whole number of expand tiles
-    return R;
+    if (H >= 40) { add(14); add(8); }
+    else if (H >= 20) { add(12); add(16); add(8); }
+    else add(H);
+    add(2 * RT);
+    add(RT);
+    return n;
 }
 
 int build_fire_plan(const ConvDesc& dsq, const ConvDesc& d1, const ConvDesc& d3, FirePlan* plan)
@@ -512,92 +645,80 @@ int build_fire_plan(const ConvDesc& dsq, const ConvDesc& d1, const ConvDesc& d3,
     if ((long long)N * H * W > 0x7fffffffLL / 2) return SQN_ERR_UNSUPPORTED;
     p.H = H; p.W = W; p.P = W + 2; p.N = N; p.Cin = Cin; p.s = s; p.e1 = e1; p.e3 = e3;
     p.RT = 128 / p.P;
-    p.R = band_rows(H, p.RT);
-    p.NB = (H + p.R - 1) / p.R;
-    p.items = N * p.NB;
-    p.BKc_in = Cin % 64 == 0 ? 64 : 32;
-    p.chunks_in = Cin / p.BKc_in;
-    p.ksteps_in = p.BKc_in / 16;
     p.ksteps_s = s / 16;
-    p.n_emma = 9 * p.ksteps_s;
-    p.nchunks = (e1 + e3) / FF_CW;
-    p.slot_cols = e1 + e3;                 // (>= s)
-    p.tmem_cols = 2u * (unsigned)p.slot_cols <= 256u ? 256u : 512u;
+    p.rb_s = (unsigned)s * 2u;
+    // TMEM: two squeeze accumulators, then the expand accumulators.  Both expands in one accumulator (the 1x1
+    // kernels ride on the centre tap) where two such accumulators fit, else two jobs per tile over three (or two)
+    // accumulators of max(e1, e3) columns.
+    p.s_slot_cols = s < 32 ? 32 : s;
+    p.tmem_cols = 512;
+    const bool combined = 2 * p.s_slot_cols + 2 * (e1 + e3) <= 512 && ((unsigned)e3 * p.rb_s) % 1024u == 0;
+    if (combined) {
+        p.njobs = 1;
+        p.eslots = 2;
+        p.eslot_cols = e1 + e3;
+    } else {
+        p.njobs = 2;
+        p.eslot_cols = e1 > e3 ? e1 : e3;
+        p.eslots = 2 * p.s_slot_cols + 3 * p.eslot_cols <= 512 ? 3 : 2;
+        if (2 * p.s_slot_cols + p.eslots * p.eslot_cols > 512) return SQN_ERR_UNSUPPORTED;
+    }
     p.c_tot = d1.out_c_total;
     p.b_early = (dsq.params_static && d1.params_static && d3.params_static) ? 1 : 0;
-    p.rb_in = (unsigned)p.BKc_in * 2u;
-    p.rb_s = (unsigned)s * 2u;
-    p.x_bytes = 128u * p.rb_in;
     p.bias_sq = dsq.bias; p.bias_e1 = d1.bias; p.bias_e3 = d3.bias;
     p.status = device_status_word();
 
-    // ---- shared-memory layout
-    size_t cur = 0;
-    p.off_wsq = 0;
-    p.wsq_tile = (unsigned)up1k((size_t)s * p.rb_in);
-    cur += (size_t)p.chunks_in * p.wsq_tile;
-    p.off_we = (unsigned)cur;
+    // ---- shared-memory layout: two patches with an input ring of 32 KB or more and three slots or more, else one
+    // patch under the same condition, else whatever fits
     {
-        // centre tap, then the 1x1 expand's kernels directly behind it (one B operand of e3 + e1 rows), then the others
-        const unsigned t3 = (unsigned)e3 * p.rb_s, t1 = (unsigned)e1 * p.rb_s;
-        if (t3 % 1024u != 0) return SQN_ERR_UNSUPPORTED;          // the appended tile must continue the swizzle pattern
-        unsigned o = 0;
-        p.off_tap[4] = o; o += t3;
-        p.off_w1 = o; o += (unsigned)up1k(t1);
-        for (int tap = 0; tap < 9; ++tap)
-            if (tap != 4) { p.off_tap[tap] = o; o += t3; }
-        cur += o;
-        p.w_bytes = (unsigned)((size_t)p.chunks_in * s * p.rb_in + 9u * t3 + t1);
-        if (p.w_bytes >= (1u << 20)) return SQN_ERR_UNSUPPORTED;  // one mbarrier transaction count
+        int cand[8];
+        const int nc = band_candidates(H, p.RT, cand);
+        bool found = false;
+        for (int pass = 0; pass < 3 && !found; ++pass)
+            for (int i = 0; i < nc && !found; ++i)
+                for (int patches = (pass == 1 ? 1 : 2); patches >= (pass == 0 ? 2 : 1) && !found; --patches)
+                    for (int bk = 64; bk >= 32 && !found; bk -= 32) {
+                        if (Cin % bk != 0) continue;
+                        const int st = fire_layout(p, cand[i], patches, bk, &plan->smem);
+                        if (st == 0) continue;
+                        if (pass == 2 || (st >= 3 && (size_t)st * p.x_tile >= 32 * 1024)) found = true;
+                    }
+        if (!found) return SQN_ERR_UNSUPPORTED;
     }
-    p.off_patch = (unsigned)cur;
-    {
-        const int t_max = p.R / p.RT;
-        size_t rows = (size_t)(p.R + 2) * p.P;
-        const size_t reach = (size_t)(t_max - 1) * p.RT * p.P + 2 * p.P + 2 + 128;     // last row an expand MMA reads
-        if (reach > rows) rows = reach;
-        p.patch_bytes = (unsigned)up1k(rows * p.rb_s);
-        cur += p.patch_bytes;
-    }
-    p.off_bias_s = (unsigned)cur; cur += up1k((size_t)s * 32);
-    p.off_bias_e = (unsigned)cur; cur += up1k((size_t)(e1 + e3) * 32);
-    p.off_ones = (unsigned)cur; cur += 128 * 32;
-    p.off_ctl = (unsigned)cur; cur += 1024;
-    static_assert(sizeof(FireShared) <= 1024, "control block");
-    p.stg_slot = (unsigned)up1k((size_t)p.RT * W * FF_CW * 2);
-    p.x_tile = (unsigned)up1k(p.x_bytes);
-    const size_t fixed = 1024 /*alignment slack*/ + cur;
-    if (fixed + 2 * p.stg_slot + 2 * p.x_tile > FF_SMEM_LIMIT) return SQN_ERR_UNSUPPORTED;
-    // input ring first (it feeds the HBM-bound part), then staging slots
-    size_t left = FF_SMEM_LIMIT - fixed;
-    p.nstg = 2;
-    left -= 2 * p.stg_slot;
-    int stages = (int)(left / p.x_tile);
-    // with room to spare, two more staging slots are worth more than input slots beyond what covers the memory latency
-    const int want = 2 * p.chunks_in > 4 ? 2 * p.chunks_in : 4;
-    if (stages >= want + (int)(2 * p.stg_slot / p.x_tile) + 1) {
-        p.nstg = 4;
-        left -= 2 * p.stg_slot;
-        stages = (int)(left / p.x_tile);
-    }
-    if (stages > FF_MAX_STAGES) stages = FF_MAX_STAGES;
-    if (stages < 2) return SQN_ERR_UNSUPPORTED;
-    p.stages = stages;
-    p.off_x = (unsigned)cur; cur += (size_t)stages * p.x_tile;
-    p.off_stg = (unsigned)cur; cur += (size_t)p.nstg * p.stg_slot;
-    plan->smem = 1024 + cur;
-    if (plan->smem > FF_SMEM_LIMIT) return SQN_ERR_UNSUPPORTED;
 
-    // ---- MMAs of an expand tile: centre tap first (it overwrites all e3 + e1 columns), then the other taps
+    // ---- MMAs of an expand tile
     {
         int e = 0;
-        static const int order[9] = {4, 0, 1, 2, 3, 5, 6, 7, 8};
-        for (int i = 0; i < 9; ++i) {
-            const int tap = order[i], kh = tap / 3, kw = tap % 3;
+        auto tap_mmas = [&](int tap, unsigned b_off, int ncols) {
+            const int kh = tap / 3, kw = tap % 3;
             for (int k = 0; k < p.ksteps_s; ++k, ++e) {
                 p.etab[e].x = (((unsigned)(kh * p.P + kw) * p.rb_s) >> 4) + 2u * k;
-                p.etab[e].y = (p.off_tap[tap] >> 4) + 2u * k;
+                p.etab[e].y = (b_off >> 4) + 2u * k;
+                p.eidesc[e] = make_idesc_bf16(128, (unsigned)ncols);
             }
+        };
+        if (combined) {
+            // centre tap first: its B operand is the centre tap's kernels followed by the 1x1 kernels, and as the first
+            // MMA of the tile it overwrites all e3 + e1 columns; the other taps add to the first e3
+            p.job_e0[0] = 0;
+            tap_mmas(4, p.off_tap[4], e3 + e1);
+            for (int tap = 0; tap < 9; ++tap)
+                if (tap != 4) tap_mmas(tap, p.off_tap[tap], e3);
+            p.job_en[0] = e;
+            p.job_chunk0[0] = 0; p.job_nchunks[0] = (e1 + e3) / FF_CW;
+            p.job_bias16[0] = 0; p.job_idesc[0] = make_idesc_bf16(128, (unsigned)(e3 + e1));
+        } else {
+            p.job_e0[0] = 0;
+            for (int tap = 0; tap < 9; ++tap) tap_mmas(tap, p.off_tap[tap], e3);
+            p.job_en[0] = e;
+            p.job_chunk0[0] = 0; p.job_nchunks[0] = e3 / FF_CW;
+            p.job_bias16[0] = 0; p.job_idesc[0] = make_idesc_bf16(128, (unsigned)e3);
+            p.job_e0[1] = e;
+            tap_mmas(4, p.off_w1, e1);                  // the 1x1 expand reads the centre pixel
+            p.job_en[1] = e;
+            p.job_chunk0[1] = e3 / FF_CW; p.job_nchunks[1] = e1 / FF_CW;
+            p.job_bias16[1] = (unsigned)e3 * 2u;        // bias rows are 32 bytes each, the 3x3 expand's come first
+            p.job_idesc[1] = make_idesc_bf16(128, (unsigned)e1);
         }
     }
     // CTA b takes items b, b + grid, ...: with a grid that shares no factor with the bands per image every CTA
@@ -674,7 +795,8 @@ int launch_fire_fused_bf16(const ConvDesc& dsq, const ConvDesc& d1, const ConvDe
     k.in = dsq.in; k.wsq = dsq.w; k.w1 = d1.w; k.w3 = d3.w; k.bsq = dsq.bias; k.b1 = d1.bias; k.b3 = d3.bias; k.out = d1.out;
     int dev = 0;
     cudaGetDevice(&dev);
-    const int band = band_rows(dsq.H, 128 / (dsq.W + 2) > 0 ? 128 / (dsq.W + 2) : 1);
+    const char* bv = std::getenv("SQN_FIRE_BAND");
+    const int band = bv ? std::atoi(bv) : 0;
     const int v[12] = {dsq.N, dsq.Cin, dsq.H, dsq.W, dsq.Cout, d1.Cout, d3.Cout, d1.out_c_total,
                        dsq.params_static | (d1.params_static << 1) | (d3.params_static << 2), dev, band, 0};
     std::memcpy(k.v, v, sizeof(v));
