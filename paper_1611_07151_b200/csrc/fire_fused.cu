@@ -46,8 +46,11 @@ using namespace ptx;
 
 constexpr int FF_SEPI_WARPS = 4;           // squeeze epilogue warps (one per TMEM lane quadrant)
 constexpr int FF_EEPI_WARPS = 8;           // expand epilogue warps (two per quadrant)
-constexpr int FF_THREADS = 32 * (4 + FF_SEPI_WARPS + FF_EEPI_WARPS);     // + producer, two issuers, store warp
-constexpr int FF_MAX_STAGES = 8;
+constexpr int FF_ISSUERS = 2;              // MMA issuer warps per pipeline: they take the pipeline's jobs in turn
+constexpr int FF_W_SMMA = 1, FF_W_EMMA = FF_W_SMMA + FF_ISSUERS, FF_W_STORE = FF_W_EMMA + FF_ISSUERS;      // first warp of each role
+constexpr int FF_W_SEPI = FF_W_STORE + 1, FF_W_EEPI = FF_W_SEPI + FF_SEPI_WARPS;
+constexpr int FF_THREADS = 32 * (FF_W_EEPI + FF_EEPI_WARPS);
+constexpr int FF_MAX_STAGES = 16;
 constexpr int FF_MAX_STG = 4;
 constexpr int FF_MAX_EMMA = 48;            // MMAs of one expand tile: 10 taps x at most 4 k-steps, + spare
 constexpr int FF_MAX_ESLOTS = 3;
@@ -62,6 +65,7 @@ struct FireParams {
     int chunks_in, BKc_in, ksteps_in;   // squeeze reduction: chunks, elements per chunk, MMAs per chunk
     int ksteps_s;                    // MMAs per expand tap (s / 16)
     int stages, nstg;
+    int s_issuers;                   // squeeze issuer warps at work: 2 where the input ring holds two tiles' chunks, else 1
     int two_patches;
     // expand jobs of a tile: one (both expands in one accumulator) or two (3x3, then 1x1)
     int njobs;
@@ -201,7 +205,7 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             mbar_init(smem_u32(&sh->s_full[a]), 1);
             mbar_init(smem_u32(&sh->s_empty[a]), FF_SEPI_WARPS);
             mbar_init(smem_u32(&sh->patch_ready[a]), FF_SEPI_WARPS);
-            mbar_init(smem_u32(&sh->patch_free[a]), 1);
+            mbar_init(smem_u32(&sh->patch_free[a]), FF_ISSUERS);
         }
         for (int a = 0; a < FF_MAX_ESLOTS; ++a) {
             mbar_init(smem_u32(&sh->e_full[a]), 1);
@@ -220,7 +224,7 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         prefetch_tensormap(&tmO);
         if (p.b_early) load_kernels();
     }
-    if (warp == 1) {
+    if (warp == FF_W_SMMA) {
         tmem_alloc(smem_u32(&sh->tmem_base), p.tmem_cols);
         tmem_relinquish();
         chain_release();            // (only once this CTA holds its TMEM: see conv_tc_body)
@@ -281,20 +285,29 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
                 }
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ squeeze issuer
-        // The whole warp walks the loops converged; one elected lane issues the MMAs and their commits.
+    } else if (warp < FF_W_EMMA) {
+        // ------------------------------------------------------------------ squeeze issuers
+        // Issuing an MMA and the hand-shakes around it cost the issuing thread far more clocks than these small MMAs
+        // cost the tensor core, so two warps take the squeeze tiles in turn (issuer w fills accumulator w).  Each
+        // warp walks the loops converged; one elected lane issues the MMAs and their commits.
+        const int w = warp - FF_W_SMMA;
         const uint32_t idesc_s = make_idesc_bf16(128, (uint32_t)p.s);
         const uint32_t hi_in = (uint32_t)(make_kmajor_desc(0, p.rb_in, 8u * p.rb_in) >> 32);
         const uint64_t ones_desc = make_kmajor_desc(base + p.off_ones, 32u, 256u);
         const uint64_t bias_s_desc = make_kmajor_desc(base + p.off_bias_s, 32u, 256u);
         const uint32_t smX16 = smX >> 4, x_tile16 = p.x_tile >> 4, smWsq16 = smWsq >> 4, wsq_tile16 = p.wsq_tile >> 4;
         bool ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->w_full), 0u, abort_flag, p.status));
-        int st = 0, as = 0;
+        int st = 0, as = 0;                     // tile k goes to accumulator k & 1 and, with two issuers, to issuer k & 1
         uint32_t ph = 0, aph = 0;
         for (int item = bid; item < p.items && ok; item += p.grid) {
             const Band b = band_of(p, item);
             for (int t = 0; t < b.n_s && ok; ++t) {
+                if ((p.s_issuers == 2 ? as : 0) != w) {         // the other issuer's tile: step over its input slots
+                    st += p.chunks_in;
+                    while (st >= p.stages) { st -= p.stages; ph ^= 1u; }
+                    if (++as == 2) { as = 0; aph ^= 1u; }
+                    continue;
+                }
                 ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->s_empty[as]), aph ^ 1u, abort_flag, p.status));
                 if (!ok) break;
                 tc_fence_after();
@@ -325,52 +338,58 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
                 if (++as == 2) { as = 0; aph ^= 1u; }
             }
         }
-    } else if (warp == 2) {
-        // ------------------------------------------------------------------ expand issuer
+    } else if (warp < FF_W_STORE) {
+        // ------------------------------------------------------------------ expand issuers (the jobs in turn)
+        const int w = warp - FF_W_EMMA;
         const uint32_t hi_s = (uint32_t)(make_kmajor_desc(0, p.rb_s, 8u * p.rb_s) >> 32);
         const uint64_t ones_desc = make_kmajor_desc(base + p.off_ones, 32u, 256u);
         const uint64_t bias_e_desc = make_kmajor_desc(base + p.off_bias_e, 32u, 256u);
         const uint32_t smWe16 = smWe >> 4, patch16 = smPatch >> 4;
         const uint32_t tile_step16 = ((uint32_t)(p.RT * p.P) * p.rb_s) >> 4;      // patch units between expand tiles
         bool ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->w_full), 0u, abort_flag, p.status));
-        int es = 0;
+        int es = 0, turn = 0;
         uint32_t eph = 0;
-        int j = 0;                              // band count of this CTA
-        for (int item = bid; item < p.items && ok; item += p.grid, ++j) {
+        int buf = 0;
+        uint32_t rph = 0;                       // parity of patch_ready[buf] for the band at hand
+        for (int item = bid; item < p.items && ok; item += p.grid) {
             const Band b = band_of(p, item);
-            const int buf = j % nbuf;
             // the band's patch is complete once every squeeze epilogue warp has passed the band's last squeeze tile
-            ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->patch_ready[buf]), (uint32_t)(j / nbuf) & 1u, abort_flag, p.status));
+            ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->patch_ready[buf]), rph, abort_flag, p.status));
             if (!ok) break;
             tc_fence_after();
             for (int t = 0; t < b.n_e && ok; ++t) {
                 const uint32_t a_base = patch16 + (uint32_t)buf * (p.patch_bytes >> 4) + (uint32_t)t * tile_step16;
-                for (int job = 0; job < p.njobs; ++job) {
-                    ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->e_empty[es]), eph ^ 1u, abort_flag, p.status));
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t d_tmem = tmem_e + (uint32_t)(es * p.eslot_cols);
-                    if (elect_one()) {
-                        uint32_t acc = 0u;
-                        const int en = p.job_en[job];
+                for (int job = 0; job < p.njobs; ++job, turn ^= 1) {
+                    if (turn == w) {
+                        ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->e_empty[es]), eph ^ 1u, abort_flag, p.status));
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t d_tmem = tmem_e + (uint32_t)(es * p.eslot_cols);
+                        if (elect_one()) {
+                            uint32_t acc = 0u;
+                            const int en = p.job_en[job];
 #pragma unroll 2
-                        for (int e = p.job_e0[job]; e < en; ++e) {
-                            const uint2 o = p.etab[e];
-                            mma_bf16_ss(d_tmem, ((uint64_t)hi_s << 32) | (uint64_t)((a_base + o.x) | 0x10000u),
-                                        ((uint64_t)hi_s << 32) | (uint64_t)((smWe16 + o.y) | 0x10000u), p.eidesc[e], acc);
-                            acc = 1u;
+                            for (int e = p.job_e0[job]; e < en; ++e) {
+                                const uint2 o = p.etab[e];
+                                mma_bf16_ss(d_tmem, ((uint64_t)hi_s << 32) | (uint64_t)((a_base + o.x) | 0x10000u),
+                                            ((uint64_t)hi_s << 32) | (uint64_t)((smWe16 + o.y) | 0x10000u), p.eidesc[e], acc);
+                                acc = 1u;
+                            }
+                            mma_bf16_ss(d_tmem, ones_desc, bias_e_desc + (uint64_t)p.job_bias16[job], p.job_idesc[job], 1u);
+                            mma_commit(smem_u32(&sh->e_full[es]));
                         }
-                        mma_bf16_ss(d_tmem, ones_desc, bias_e_desc + (uint64_t)p.job_bias16[job], p.job_idesc[job], 1u);
-                        mma_commit(smem_u32(&sh->e_full[es]));
-                        // after the band's last job: the patch may be overwritten once these MMAs have read it
-                        if (t == b.n_e - 1 && job == p.njobs - 1) mma_commit(smem_u32(&sh->patch_free[buf]));
+                        __syncwarp();
                     }
-                    __syncwarp();
                     if (++es == p.eslots) { es = 0; eph ^= 1u; }
                 }
             }
+            if (!ok) break;
+            // the patch may be overwritten once the MMAs of both issuers have read it
+            if (elect_one()) mma_commit(smem_u32(&sh->patch_free[buf]));
+            __syncwarp();
+            if (++buf == nbuf) { buf = 0; rph ^= 1u; }
         }
-    } else if (warp == 3) {
+    } else if (warp == FF_W_STORE) {
         // ----------------------------------------------------------------- store issuer
         if (lane == 0) {
             bool ok = true;
@@ -400,19 +419,18 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             }
             tma_store_wait_all();
         }
-    } else if (warp < 4 + FF_SEPI_WARPS) {
+    } else if (warp < FF_W_EEPI) {
         // -------------------------------------------------------------------- squeeze epilogue
         // warp w reads TMEM lane quadrant w % 4: one input pixel per thread, all s layers of it
         const int q = warp & 3;
         const int row = q * 32 + lane;
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
-        const int sidx = (warp - 4) * 32 + lane;                 // index among the squeeze epilogue threads
+        const int sidx = (warp - FF_W_SEPI) * 32 + lane;                 // index among the squeeze epilogue threads
         bool ok = true;
-        int as = 0, j = 0;
-        uint32_t aph = 0;
+        int as = 0, j = 0, buf = 0;
+        uint32_t aph = 0, fph = 0;              // fph: parity of patch_free[buf] for the patch's previous band
         for (int item = bid; item < p.items && ok; item += p.grid, ++j) {
             const Band b = band_of(p, item);
-            const int buf = j % nbuf;
             const uint32_t patch = smPatch + (uint32_t)buf * p.patch_bytes;
             for (int t = 0; t < b.n_s; ++t) {
                 ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->s_full[as]), aph, abort_flag, p.status));
@@ -434,7 +452,7 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
                 if (++as == 2) { as = 0; aph ^= 1u; }
                 if (t == 0 && j >= nbuf) {
                     // the expand MMAs of the band that used this patch before must have read it
-                    ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->patch_free[buf]), (uint32_t)(j / nbuf - 1) & 1u, abort_flag, p.status));
+                    ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->patch_free[buf]), fph, abort_flag, p.status));
                     if (!ok) break;
                 }
                 const int g = t * 128 + row;                      // pixel of the band's input rows
@@ -465,11 +483,12 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             fence_proxy_async_smem();             // patch visible to the tensor core
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh->patch_ready[buf]));
+            if (++buf == nbuf) { buf = 0; if (j >= nbuf) fph ^= 1u; }
         }
     } else {
         // -------------------------------------------------------------------- expand epilogue
         // warp w reads TMEM lane quadrant w % 4 (one M row per thread); the two warps of a quadrant split a chunk's columns
-        const int q = warp & 3, hf = (warp - 4 - FF_SEPI_WARPS) >> 2;
+        const int q = warp & 3, hf = (warp - FF_W_EEPI) >> 2;
         const int row = q * 32 + lane;
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
         // M row -> (image row r of the tile, patch column c); the staging tile drops the padding columns
@@ -518,7 +537,7 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == FF_W_SMMA) {
         __syncwarp();
         tc_fence_after();
         tmem_dealloc(tmem_base, p.tmem_cols);
@@ -589,9 +608,9 @@ int fire_layout(FireParams& p, int R, int patches, int BKc_in, size_t* smem_byte
     p.nstg = 2;
     left -= 2 * p.stg_slot;
     int stages = (int)(left / p.x_tile);
-    // with room to spare, two more staging slots are worth more than input slots beyond what covers the memory latency
-    const int want = 2 * p.chunks_in > 4 ? 2 * p.chunks_in : 4;
-    if (stages >= want + (int)(2 * p.stg_slot / p.x_tile) + 1) {
+    // The ring must hold what is in flight between this SM and memory (about 100 KB at full bandwidth); only beyond
+    // that are two more staging slots worth their shared memory.
+    if (left >= 2 * p.stg_slot + (size_t)128 * 1024) {
         p.nstg = 4;
         left -= 2 * p.stg_slot;
         stages = (int)(left / p.x_tile);
@@ -599,6 +618,9 @@ int fire_layout(FireParams& p, int R, int patches, int BKc_in, size_t* smem_byte
     if (stages > FF_MAX_STAGES) stages = FF_MAX_STAGES;
     if (stages < 2) return 0;
     p.stages = stages;
+    // Two issuers wait on the ring's barriers out of step; a wait must never be two phases ahead of its barrier
+    // (its parity would match a phase long past), which holds when the ring is at least two tiles deep.
+    p.s_issuers = stages >= 2 * p.chunks_in ? 2 : 1;
     p.off_x = (unsigned)cur; cur += (size_t)stages * p.x_tile;
     p.off_stg = (unsigned)cur; cur += (size_t)p.nstg * p.stg_slot;
     *smem_bytes = 1024 + cur;
@@ -606,7 +628,7 @@ int fire_layout(FireParams& p, int R, int patches, int BKc_in, size_t* smem_byte
 }
 
 // Band heights to try, best first: SQN_FIRE_BAND in the environment (tuning aid, read at every call) names one;
-// else 14 rows for maps of 40 rows and more (four equal bands for 55 rows), 12 for 20 rows and more, else the whole
+// else 14 rows for maps of 40 rows and more (four equal bands for 55 rows), 8 for 20 rows and more, else the whole
 // image.  A band is a whole number of expand tiles.
 int band_candidates(int H, int RT, int* out)
 {
@@ -623,7 +645,7 @@ int band_candidates(int H, int RT, int* out)
         if (r > 0) { add(r); return n; }
     }
     if (H >= 40) { add(14); add(8); }
-    else if (H >= 20) { add(12); add(16); add(8); }
+    else if (H >= 20) { add(8); add(12); add(16); }
     else add(H);
     add(2 * RT);
     add(RT);
