@@ -112,6 +112,14 @@ int run_conv(const ConvDesc& d, int dtype, void* ws, size_t ws_bytes, cudaStream
 int run_expands(const ConvDesc& d1, const ConvDesc& d3, int dtype, cudaStream_t stream, bool* paired)
 {
     if (paired) *paired = false;
+    if (dtype == SQN_BF16 && fused_fire_enabled() && !d1.pool && !d3.pool) {
+        const int rc = launch_fire_expands_bf16(d1, d3, stream);     // flat-patch kernel, kernels resident per CTA
+        if (rc == SQN_OK) {
+            if (paired) *paired = true;
+            return SQN_OK;
+        }
+        if (rc != SQN_ERR_UNSUPPORTED) return rc;
+    }
     if (dtype == SQN_BF16 && pair_launch_enabled() && conv_bf16_supported(d1) == SQN_OK && conv_bf16_supported(d3) == SQN_OK) {
         const int rc = launch_conv_bf16_pair(d1, d3, stream);
         if (rc == SQN_OK) {

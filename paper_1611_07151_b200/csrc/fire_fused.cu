@@ -45,7 +45,7 @@ namespace {
 using namespace ptx;
 
 constexpr int FF_SEPI_WARPS = 4;           // squeeze epilogue warps (one per TMEM lane quadrant)
-constexpr int FF_EEPI_WARPS = 8;           // expand epilogue warps (two per quadrant)
+constexpr int FF_EEPI_WARPS = 8;           // expand epilogue warps: two groups of four (one warp per quadrant)
 constexpr int FF_ISSUERS = 2;              // MMA issuer warps per pipeline: they take the pipeline's jobs in turn
 constexpr int FF_W_SMMA = 1, FF_W_EMMA = FF_W_SMMA + FF_ISSUERS, FF_W_STORE = FF_W_EMMA + FF_ISSUERS;      // first warp of each role
 constexpr int FF_W_SEPI = FF_W_STORE + 1, FF_W_EEPI = FF_W_SEPI + FF_SEPI_WARPS;
@@ -55,7 +55,6 @@ constexpr int FF_MAX_STG = 4;
 constexpr int FF_MAX_EMMA = 48;            // MMAs of one expand tile: 10 taps x at most 4 k-steps, + spare
 constexpr int FF_MAX_ESLOTS = 3;
 constexpr size_t FF_SMEM_LIMIT = 227 * 1024;
-constexpr int FF_CW = 64;                  // output layers per store chunk
 
 struct FireParams {
     int H, W, P, N;                  // map extent, patch pitch (W + 2), images
@@ -63,14 +62,17 @@ struct FireParams {
     int RT, R, NB;                   // image rows per expand tile, rows per band, bands per image
     int items, grid;
     int chunks_in, BKc_in, ksteps_in;   // squeeze reduction: chunks, elements per chunk, MMAs per chunk
-    int ksteps_s;                    // MMAs per expand tap (s / 16)
+    int src_tma;                     // 1: no squeeze pipeline -- the patch is loaded by TMA from a stored squeeze map
+    int chunks_s, BKs, ksteps_s;     // expand reduction per tap: chunks_s chunks of BKs layers (s = chunks_s * BKs), BKs / 16 MMAs each
+    int CS, e3p, e1p;                // the output layers are split over CS CTAs ("parts") of e3p + e1p layers each
+    int CW;                          // output layers per store chunk (32 or 64)
     int stages, nstg;
     int s_issuers;                   // squeeze issuer warps at work: 2 where the input ring holds two tiles' chunks, else 1
     int two_patches;
     // expand jobs of a tile: one (both expands in one accumulator) or two (3x3, then 1x1)
     int njobs;
     int job_e0[2], job_en[2];        // the job's MMAs: entries [e0, en) of etab
-    int job_chunk0[2], job_nchunks[2];   // its store chunks (chunk c = accumulator-order columns [64c, 64c + 64))
+    int job_chunk0[2], job_nchunks[2];   // its store chunks (chunk c = accumulator-order columns [CW*c, CW*c + CW) of the part)
     unsigned job_bias16[2];          // its bias rows, in 16-byte units from off_bias_e
     unsigned job_idesc[2];           // instruction descriptor of its bias MMA (all of its columns)
     int s_slot_cols;                 // TMEM: two squeeze accumulators of s_slot_cols columns, then eslots expand
@@ -78,13 +80,15 @@ struct FireParams {
     unsigned tmem_cols;
     int c_tot;                       // layers per pixel of the output tensor
     int b_early;                     // kernels and bias may be fetched before the wait for the grid ahead
-    unsigned rb_in, rb_s;            // bytes per row of the input / squeeze-kernel tiles and of the patch / expand-kernel tiles
+    unsigned rb_in, rb_s;            // bytes per row of the input / squeeze-kernel tiles and of the patch / expand-kernel tiles (2 * BKs)
     unsigned x_bytes;                // bytes one input box delivers
     unsigned w_bytes;                // bytes of all kernel tiles together
     unsigned off_wsq, wsq_tile;      // squeeze kernels: chunks_in tiles of s rows
     unsigned off_we;                 // expand kernels: centre tap, 1x1, then the other eight taps
-    unsigned off_tap[9], off_w1;     // ... offsets of the tiles from off_we
-    unsigned off_patch, patch_bytes; // one or two patches of patch_bytes each
+    unsigned off_w3[9][3], off_w1c[3];   // ... offsets from off_we of the tiles of (tap, chunk) and of the 1x1 kernels' chunks
+    unsigned off_patch, patch_bytes; // one or two patches of patch_bytes each,
+    unsigned patch_chunk;            // ... each made of chunks_s arrays of patch_chunk bytes (rows of BKs layers)
+    unsigned patch_box_bytes;        // bytes one patch box delivers (src_tma)
     unsigned off_x, x_tile;
     unsigned off_stg, stg_slot;
     unsigned off_bias_s, off_bias_e, off_ones, off_ctl;
@@ -174,23 +178,30 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int bid = (int)blockIdx.x;
+    // CTA -> (part of the output layers, first band); it walks the bands bid, bid + gstep, ...
+    const int part = (int)blockIdx.x % p.CS;
+    const int bid = (int)blockIdx.x / p.CS, gstep = p.grid / p.CS;
     const int nbuf = p.two_patches ? 2 : 1;
 
-    auto load_kernels = [&]() {          // every kernel tile of the layer, once (one mbarrier counts them all)
+    auto load_kernels = [&]() {          // every kernel tile of the layer (this CTA's part of it), once; one mbarrier counts them all
         const uint32_t bar = smem_u32(&sh->w_full);
         mbar_arrive_expect_tx(bar, p.w_bytes);
-        for (int ch = 0; ch < p.chunks_in; ++ch)
-            tma_load_2d(smWsq + (uint32_t)ch * p.wsq_tile, &tmWsq, bar, ch * p.BKc_in, 0);
-        for (int tap = 0; tap < 9; ++tap) tma_load_2d(smWe + p.off_tap[tap], &tmW3, bar, tap * p.s, 0);
-        tma_load_2d(smWe + p.off_w1, &tmW1, bar, 0, 0);
+        if (!p.src_tma)
+            for (int ch = 0; ch < p.chunks_in; ++ch)
+                tma_load_2d(smWsq + (uint32_t)ch * p.wsq_tile, &tmWsq, bar, ch * p.BKc_in, 0);
+        for (int tap = 0; tap < 9; ++tap)
+            for (int ch = 0; ch < p.chunks_s; ++ch)
+                tma_load_2d(smWe + p.off_w3[tap][ch], &tmW3, bar, tap * p.s + ch * p.BKs, part * p.e3p);
+        for (int ch = 0; ch < p.chunks_s; ++ch) tma_load_2d(smWe + p.off_w1c[ch], &tmW1, bar, ch * p.BKs, part * p.e1p);
     };
     auto fill_bias = [&]() {
-        uint4* rs = reinterpret_cast<uint4*>(base_ptr + p.off_bias_s);
-        for (int c = threadIdx.x; c < p.s; c += FF_THREADS) bias_row(rs, c, __ldg(p.bias_sq + c));
+        if (!p.src_tma) {
+            uint4* rs = reinterpret_cast<uint4*>(base_ptr + p.off_bias_s);
+            for (int c = threadIdx.x; c < p.s; c += FF_THREADS) bias_row(rs, c, __ldg(p.bias_sq + c));
+        }
         uint4* re = reinterpret_cast<uint4*>(base_ptr + p.off_bias_e);
-        for (int c = threadIdx.x; c < p.e3 + p.e1; c += FF_THREADS)
-            bias_row(re, c, c < p.e3 ? __ldg(p.bias_e3 + c) : __ldg(p.bias_e1 + c - p.e3));
+        for (int c = threadIdx.x; c < p.e3p + p.e1p; c += FF_THREADS)
+            bias_row(re, c, c < p.e3p ? __ldg(p.bias_e3 + part * p.e3p + c) : __ldg(p.bias_e1 + part * p.e1p + c - p.e3p));
     };
 
     // Up to chain_wait() this block touches only its own shared memory, TMEM, the kernel parameters and, when
@@ -204,7 +215,7 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&sh->s_full[a]), 1);
             mbar_init(smem_u32(&sh->s_empty[a]), FF_SEPI_WARPS);
-            mbar_init(smem_u32(&sh->patch_ready[a]), FF_SEPI_WARPS);
+            mbar_init(smem_u32(&sh->patch_ready[a]), p.src_tma ? 1 : FF_SEPI_WARPS);
             mbar_init(smem_u32(&sh->patch_free[a]), FF_ISSUERS);
         }
         for (int a = 0; a < FF_MAX_ESLOTS; ++a) {
@@ -212,7 +223,7 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             mbar_init(smem_u32(&sh->e_empty[a]), FF_EEPI_WARPS);
         }
         for (int b = 0; b < p.nstg; ++b) {
-            mbar_init(smem_u32(&sh->stg_full[b]), FF_EEPI_WARPS);
+            mbar_init(smem_u32(&sh->stg_full[b]), FF_EEPI_WARPS / 2);      // one group of the expand epilogue
             mbar_init(smem_u32(&sh->stg_free[b]), 1);
         }
         sh->abort_flag = 0;
@@ -250,16 +261,44 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     tc_fence_after();
     const uint32_t tmem_base = sh->tmem_base;
     volatile int* abort_flag = &sh->abort_flag;
-    const uint32_t tmem_e = tmem_base + (uint32_t)(2 * p.s_slot_cols);      // first expand accumulator
+    const uint32_t tmem_e = tmem_base + (uint32_t)(2 * p.s_slot_cols);      // first expand accumulator (s_slot_cols = 0 without a squeeze pipeline)
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer: input tiles of the squeeze
-        if (lane == 0) {
+        if (lane == 0 && p.src_tma) {
+            // the patch of a band straight from the stored squeeze map: one box per chunk of layers, one pixel to the left
+            // of and one row above the band; what lies outside the map is filled with zeros, which is the padding
+            if (!p.b_early) load_kernels();
+            bool ok = true;
+            int buf = 0, j = 0, loaded = 0;
+            uint32_t fph = 0;
+            for (int item = bid; item < p.items && ok; item += gstep, ++j) {
+                const Band b = band_of(p, item);
+                if (j >= nbuf && !wait_bar(smem_u32(&sh->patch_free[buf]), fph, abort_flag, p.status)) { ok = false; break; }
+                const uint32_t bar = smem_u32(&sh->patch_ready[buf]);
+                mbar_arrive_expect_tx(bar, (uint32_t)p.chunks_s * p.patch_box_bytes);
+                for (int ch = 0; ch < p.chunks_s; ++ch)
+                    tma_load_5d(smPatch + (uint32_t)buf * p.patch_bytes + (uint32_t)ch * p.patch_chunk, &tmX, bar, ch * p.BKs, -1,
+                                b.y0 - 1, b.n, 0);
+                ++loaded;
+                if (++buf == nbuf) { buf = 0; if (j >= nbuf) fph ^= 1u; }
+            }
+            if (!ok) {      // give the boxes already issued a bounded chance to land before the CTA exits
+                for (int k = 0; k < nbuf && k < loaded; ++k) {
+                    const int jj = loaded - 1 - k;
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(smem_u32(&sh->patch_ready[jj % nbuf]), (uint32_t)(jj / nbuf) & 1u)) {
+                        if (clock64() - t0 > WAIT_LIMIT_CYCLES / 8) break;
+                        __nanosleep(100);
+                    }
+                }
+            }
+        } else if (lane == 0) {
             if (!p.b_early) load_kernels();
             bool ok = true;
             int st = 0, issued = 0;
             uint32_t ph = 0;
-            for (int item = bid; item < p.items && ok; item += p.grid) {
+            for (int item = bid; item < p.items && ok; item += gstep) {
                 const Band b = band_of(p, item);
                 const int px0 = (b.n * p.H + b.ylo) * p.W;
                 for (int t = 0; t < b.n_s && ok; ++t)
@@ -296,10 +335,10 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         const uint64_t ones_desc = make_kmajor_desc(base + p.off_ones, 32u, 256u);
         const uint64_t bias_s_desc = make_kmajor_desc(base + p.off_bias_s, 32u, 256u);
         const uint32_t smX16 = smX >> 4, x_tile16 = p.x_tile >> 4, smWsq16 = smWsq >> 4, wsq_tile16 = p.wsq_tile >> 4;
-        bool ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->w_full), 0u, abort_flag, p.status));
+        bool ok = !p.src_tma && __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->w_full), 0u, abort_flag, p.status));
         int st = 0, as = 0;                     // tile k goes to accumulator k & 1 and, with two issuers, to issuer k & 1
         uint32_t ph = 0, aph = 0;
-        for (int item = bid; item < p.items && ok; item += p.grid) {
+        for (int item = bid; item < p.items && ok; item += gstep) {
             const Band b = band_of(p, item);
             for (int t = 0; t < b.n_s && ok; ++t) {
                 if ((p.s_issuers == 2 ? as : 0) != w) {         // the other issuer's tile: step over its input slots
@@ -351,7 +390,7 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         uint32_t eph = 0;
         int buf = 0;
         uint32_t rph = 0;                       // parity of patch_ready[buf] for the band at hand
-        for (int item = bid; item < p.items && ok; item += p.grid) {
+        for (int item = bid; item < p.items && ok; item += gstep) {
             const Band b = band_of(p, item);
             // the band's patch is complete once every squeeze epilogue warp has passed the band's last squeeze tile
             ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->patch_ready[buf]), rph, abort_flag, p.status));
@@ -396,14 +435,14 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             int sb = 0, pend = 0, fb = 0;       // next slot, stores whose slot is not yet released, next slot to release
             uint32_t sph = 0;
             const int nchunks = p.job_chunk0[p.njobs - 1] + p.job_nchunks[p.njobs - 1];
-            for (int item = bid; item < p.items && ok; item += p.grid) {
+            for (int item = bid; item < p.items && ok; item += gstep) {
                 const Band b = band_of(p, item);
                 for (int t = 0; t < b.n_e && ok; ++t)
                     for (int chunk = 0; chunk < nchunks; ++chunk) {
                         if (!wait_bar(smem_u32(&sh->stg_full[sb]), sph, abort_flag, p.status)) { ok = false; break; }
-                        // accumulator-order columns [0, e3) are the 3x3 expand (output layers e1 ..), the rest the 1x1 expand
-                        const int col = chunk * FF_CW;
-                        const int cc = col < p.e3 ? p.e1 + col : col - p.e3;
+                        // accumulator-order columns [0, e3p) are the part's 3x3 layers (output layers e1 + ..), the rest its 1x1 layers
+                        const int col = chunk * p.CW;
+                        const int cc = col < p.e3p ? p.e1 + part * p.e3p + col : part * p.e1p + col - p.e3p;
                         tma_store_4d(&tmO, smStg + (uint32_t)sb * p.stg_slot, cc, 0, b.y0 + t * p.RT, b.n);
                         tma_store_commit();
                         if (++sb == p.nstg) { sb = 0; sph ^= 1u; }
@@ -426,10 +465,10 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         const int row = q * 32 + lane;
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
         const int sidx = (warp - FF_W_SEPI) * 32 + lane;                 // index among the squeeze epilogue threads
-        bool ok = true;
+        bool ok = !p.src_tma;
         int as = 0, j = 0, buf = 0;
         uint32_t aph = 0, fph = 0;              // fph: parity of patch_free[buf] for the patch's previous band
-        for (int item = bid; item < p.items && ok; item += p.grid, ++j) {
+        for (int item = bid; item < p.items && ok; item += gstep, ++j) {
             const Band b = band_of(p, item);
             const uint32_t patch = smPatch + (uint32_t)buf * p.patch_bytes;
             for (int t = 0; t < b.n_s; ++t) {
@@ -487,46 +526,59 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         }
     } else {
         // -------------------------------------------------------------------- expand epilogue
-        // warp w reads TMEM lane quadrant w % 4 (one M row per thread); the two warps of a quadrant split a chunk's columns
-        const int q = warp & 3, hf = (warp - FF_W_EEPI) >> 2;
+        // Two groups of four warps (one warp per TMEM lane quadrant, one M row per thread) take the store chunks in
+        // turn, so that two chunks are converted at a time: a chunk is a chain of latencies (TMEM load, wait for the
+        // staging slot, conversion, proxy fence, hand-over) far longer than its instructions.
+        const int q = warp & 3, grp = (warp - FF_W_EEPI) >> 2;
         const int row = q * 32 + lane;
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
         // M row -> (image row r of the tile, patch column c); the staging tile drops the padding columns
         const int r_e = row / p.P, c_e = row - r_e * p.P;
         const bool e_valid = c_e < p.W && r_e < p.RT;
         const uint32_t stg_row = (uint32_t)(r_e * p.W + c_e);
-        const uint32_t stg_off = stg_row * (uint32_t)(FF_CW * 2);
-        const uint32_t sw_e = stg_row & 7u;
+        const uint32_t stg_off = stg_row * (uint32_t)(p.CW * 2);
+        const uint32_t sw_e = swz(stg_row, (uint32_t)(p.CW * 2));
         bool ok = true;
-        int es = 0, sb = 0;
+        int es = 0, sb = 0, turn = 0;           // turn: the group whose chunk the next one is
         uint32_t eph = 0, sph = 0;
-        for (int item = bid; item < p.items && ok; item += p.grid) {
+        for (int item = bid; item < p.items && ok; item += gstep) {
             const Band b = band_of(p, item);
             for (int t = 0; t < b.n_e && ok; ++t)
                 for (int job = 0; job < p.njobs; ++job) {
                     ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->e_full[es]), eph, abort_flag, p.status));
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t ta0 = tmem_e + lane_base + (uint32_t)(es * p.eslot_cols + hf * 32);
-                    for (int chunk = 0; chunk < p.job_nchunks[job]; ++chunk) {
-                        uint32_t v[32];
-                        const uint32_t ta = ta0 + (uint32_t)(chunk * FF_CW);
-                        tmem_ld_x16(ta, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
-                        tmem_ld_x16(ta + 16u, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
-                        ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->stg_free[sb]), sph ^ 1u, abort_flag, p.status));
-                        tmem_ld_wait();
-                        if (!ok) break;
-                        if (e_valid) {
-                            const uint32_t rbase = smStg + (uint32_t)sb * p.stg_slot + stg_off;
-                            store16(&v[0], rbase, (uint32_t)hf * 4u, sw_e);
-                            store16(&v[16], rbase, (uint32_t)hf * 4u + 2u, sw_e);
+                    const uint32_t ta0 = tmem_e + lane_base + (uint32_t)(es * p.eslot_cols);
+                    for (int chunk = 0; chunk < p.job_nchunks[job]; ++chunk, turn ^= 1) {
+                        if (turn == grp) {
+                            uint32_t v[64];
+                            const uint32_t ta = ta0 + (uint32_t)(chunk * p.CW);
+                            tmem_ld_x16(ta, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
+                            tmem_ld_x16(ta + 16u, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
+                            if (p.CW == 64) {
+                                tmem_ld_x16(ta + 32u, *reinterpret_cast<uint32_t(*)[16]>(&v[32]));
+                                tmem_ld_x16(ta + 48u, *reinterpret_cast<uint32_t(*)[16]>(&v[48]));
+                            }
+                            ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->stg_free[sb]), sph ^ 1u, abort_flag, p.status));
+                            tmem_ld_wait();
+                            if (!ok) break;
+                            if (e_valid) {
+                                const uint32_t rbase = smStg + (uint32_t)sb * p.stg_slot + stg_off;
+                                store16(&v[0], rbase, 0u, sw_e);
+                                store16(&v[16], rbase, 2u, sw_e);
+                                if (p.CW == 64) {
+                                    store16(&v[32], rbase, 4u, sw_e);
+                                    store16(&v[48], rbase, 6u, sw_e);
+                                }
+                            }
+                            fence_proxy_async_smem();             // staging rows visible to the TMA unit
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(smem_u32(&sh->stg_full[sb]));
                         }
-                        fence_proxy_async_smem();             // staging rows visible to the TMA unit
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(smem_u32(&sh->stg_full[sb]));
                         if (++sb == p.nstg) { sb = 0; sph ^= 1u; }
                     }
                     if (!ok) break;
+                    // this group's part of the accumulator is in its staging tiles: hand it back to the issuers
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&sh->e_empty[es]));
@@ -553,36 +605,45 @@ struct FirePlan {
 
 inline size_t up1k(size_t v) { return (v + 1023) / 1024 * 1024; }
 
-// Shared-memory layout for one choice of band height R, number of patches (2: squeeze of the next band overlaps the
-// expands of this one; 1: they take turns) and input chunk width.  Returns the input ring's depth (0: does not fit).
+// Shared-memory layout for one choice of band height R, number of patches (2: the next band's patch is made while the
+// expands run on this one; 1: they take turns) and, with a squeeze pipeline, input chunk width.  Fills the offsets;
+// returns 0 if it does not fit, else 1 + the depth of the input ring (1 when there is no squeeze pipeline).
 int fire_layout(FireParams& p, int R, int patches, int BKc_in, size_t* smem_bytes)
 {
-    const int s = p.s, e1 = p.e1, e3 = p.e3, W = p.W, H = p.H;
+    const int s = p.s, W = p.W, H = p.H;
     p.R = R;
     p.NB = (H + R - 1) / R;
     p.items = p.N * p.NB;
     p.two_patches = patches == 2 ? 1 : 0;
-    p.BKc_in = BKc_in;
-    p.chunks_in = p.Cin / BKc_in;
-    p.ksteps_in = BKc_in / 16;
-    p.rb_in = (unsigned)BKc_in * 2u;
-    p.x_bytes = 128u * p.rb_in;
     size_t cur = 0;
+    p.w_bytes = 0;
     p.off_wsq = 0;
-    p.wsq_tile = (unsigned)up1k((size_t)s * p.rb_in);
-    cur += (size_t)p.chunks_in * p.wsq_tile;
+    if (!p.src_tma) {
+        p.BKc_in = BKc_in;
+        p.chunks_in = p.Cin / BKc_in;
+        p.ksteps_in = BKc_in / 16;
+        p.rb_in = (unsigned)BKc_in * 2u;
+        p.x_bytes = 128u * p.rb_in;
+        p.wsq_tile = (unsigned)up1k((size_t)s * p.rb_in);
+        cur += (size_t)p.chunks_in * p.wsq_tile;
+        p.w_bytes += (unsigned)((size_t)p.chunks_in * s * p.rb_in);
+    }
     p.off_we = (unsigned)cur;
     {
-        // centre tap, then the 1x1 expand's kernels directly behind it (one B operand of e3 + e1 rows), then the others
-        const unsigned t3 = (unsigned)e3 * p.rb_s, t1 = (unsigned)e1 * p.rb_s;
-        if (t3 % 1024u != 0) return 0;          // the appended tile must continue the swizzle pattern
+        // per chunk of layers: the centre tap's kernels, then the 1x1 expand's directly behind them (one B operand of
+        // e3p + e1p rows); then the other eight taps
+        const unsigned t3 = (unsigned)p.e3p * p.rb_s, t1 = (unsigned)p.e1p * p.rb_s;
         unsigned o = 0;
-        p.off_tap[4] = o; o += t3;
-        p.off_w1 = o; o += (unsigned)up1k(t1);
+        for (int ch = 0; ch < p.chunks_s; ++ch) {
+            p.off_w3[4][ch] = o; o += t3;
+            p.off_w1c[ch] = o; o += t1;
+            o = (unsigned)up1k(o);
+        }
         for (int tap = 0; tap < 9; ++tap)
-            if (tap != 4) { p.off_tap[tap] = o; o += t3; }
+            if (tap != 4)
+                for (int ch = 0; ch < p.chunks_s; ++ch) { p.off_w3[tap][ch] = o; o += (unsigned)up1k(t3); }
         cur += o;
-        p.w_bytes = (unsigned)((size_t)p.chunks_in * s * p.rb_in + 9u * t3 + t1);
+        p.w_bytes += (unsigned)p.chunks_s * (9u * t3 + t1);
         if (p.w_bytes >= (1u << 20)) return 0;  // one mbarrier transaction count
     }
     p.off_patch = (unsigned)cur;
@@ -591,17 +652,30 @@ int fire_layout(FireParams& p, int R, int patches, int BKc_in, size_t* smem_byte
         size_t rows = (size_t)(R + 2) * p.P;
         const size_t reach = (size_t)(t_max - 1) * p.RT * p.P + 2 * p.P + 2 + 128;     // last row an expand MMA reads
         if (reach > rows) rows = reach;
-        p.patch_bytes = (unsigned)up1k(rows * p.rb_s);
+        p.patch_chunk = (unsigned)up1k(rows * p.rb_s);
+        p.patch_bytes = (unsigned)p.chunks_s * p.patch_chunk;
+        p.patch_box_bytes = (unsigned)((size_t)(R + 2) * p.P * p.rb_s);
         cur += (size_t)patches * p.patch_bytes;
     }
     p.off_bias_s = (unsigned)cur; cur += up1k((size_t)s * 32);
-    p.off_bias_e = (unsigned)cur; cur += up1k((size_t)(e1 + e3) * 32);
+    p.off_bias_e = (unsigned)cur; cur += up1k((size_t)(p.e1p + p.e3p) * 32);
     p.off_ones = (unsigned)cur; cur += 128 * 32;
     p.off_ctl = (unsigned)cur; cur += 1024;
     static_assert(sizeof(FireShared) <= 1024, "control block");
-    p.stg_slot = (unsigned)up1k((size_t)p.RT * W * FF_CW * 2);
-    p.x_tile = (unsigned)up1k(p.x_bytes);
+    p.stg_slot = (unsigned)up1k((size_t)p.RT * W * p.CW * 2);
     const size_t fixed = 1024 /*alignment slack*/ + cur;
+    if (p.src_tma) {
+        if (fixed + 2 * p.stg_slot > FF_SMEM_LIMIT) return 0;
+        p.nstg = fixed + 4 * p.stg_slot <= FF_SMEM_LIMIT ? 4 : 2;
+        p.stages = 1;                       // (no input ring; its barriers are still initialised)
+        p.s_issuers = 1;
+        p.off_x = (unsigned)cur;
+        p.x_tile = 0;
+        p.off_stg = (unsigned)cur; cur += (size_t)p.nstg * p.stg_slot;
+        *smem_bytes = 1024 + cur;
+        return 1;
+    }
+    p.x_tile = (unsigned)up1k(p.x_bytes);
     if (fixed + 2 * p.stg_slot + 2 * p.x_tile > FF_SMEM_LIMIT) return 0;
     // input ring first (it feeds the memory-bound part), then staging slots
     size_t left = FF_SMEM_LIMIT - fixed;
@@ -624,7 +698,7 @@ int fire_layout(FireParams& p, int R, int patches, int BKc_in, size_t* smem_byte
     p.off_x = (unsigned)cur; cur += (size_t)stages * p.x_tile;
     p.off_stg = (unsigned)cur; cur += (size_t)p.nstg * p.stg_slot;
     *smem_bytes = 1024 + cur;
-    return *smem_bytes <= FF_SMEM_LIMIT ? stages : 0;
+    return *smem_bytes <= FF_SMEM_LIMIT ? 1 + stages : 0;
 }
 
 // Band heights to try, best first: SQN_FIRE_BAND in the environment (tuning aid, read at every call) names one;
@@ -652,14 +726,16 @@ int band_candidates(int H, int RT, int* out)
     return n;
 }
 
-int build_fire_plan(const ConvDesc& dsq, const ConvDesc& d1, const ConvDesc& d3, FirePlan* plan)
+// Plan for a fire layer: with dsq the whole layer (squeeze pipeline in the kernel), without it the two expands on a
+// stored squeeze map (the patch comes by TMA).
+int build_fire_plan(const ConvDesc* dsq, const ConvDesc& d1, const ConvDesc& d3, FirePlan* plan)
 {
     FireParams& p = plan->p;
     std::memset(&p, 0, sizeof(p));
-    const int H = dsq.H, W = dsq.W, N = dsq.N, Cin = dsq.Cin, s = dsq.Cout, e1 = d1.Cout, e3 = d3.Cout;
-    if (s != 16 && s != 32 && s != 64) return SQN_ERR_UNSUPPORTED;            // one swizzled row per patch pixel
-    if (e1 % FF_CW != 0 || e3 % FF_CW != 0 || e1 + e3 > 256) return SQN_ERR_UNSUPPORTED;
-    if (Cin % 32 != 0) return SQN_ERR_UNSUPPORTED;
+    const int H = d1.H, W = d1.W, N = d1.N, s = d1.Cin, e1 = d1.Cout, e3 = d3.Cout;
+    const int Cin = dsq ? dsq->Cin : 0;
+    p.src_tma = dsq ? 0 : 1;
+    if (s % 16 != 0 || e1 % 32 != 0 || e3 % 32 != 0) return SQN_ERR_UNSUPPORTED;
     if (W + 2 > 128 || H < 1) return SQN_ERR_UNSUPPORTED;
     if (d1.out != d3.out || d1.out_c_total != d3.out_c_total || d1.out_c_offset != 0 || d3.out_c_offset != e1 ||
         d1.out_c_total % 8 != 0)
@@ -667,123 +743,156 @@ int build_fire_plan(const ConvDesc& dsq, const ConvDesc& d1, const ConvDesc& d3,
     if ((long long)N * H * W > 0x7fffffffLL / 2) return SQN_ERR_UNSUPPORTED;
     p.H = H; p.W = W; p.P = W + 2; p.N = N; p.Cin = Cin; p.s = s; p.e1 = e1; p.e3 = e3;
     p.RT = 128 / p.P;
-    p.ksteps_s = s / 16;
-    p.rb_s = (unsigned)s * 2u;
-    // TMEM: two squeeze accumulators, then the expand accumulators.  Both expands in one accumulator (the 1x1
-    // kernels ride on the centre tap) where two such accumulators fit, else two jobs per tile over three (or two)
-    // accumulators of max(e1, e3) columns.
-    p.s_slot_cols = s < 32 ? 32 : s;
-    p.tmem_cols = 512;
-    const bool combined = 2 * p.s_slot_cols + 2 * (e1 + e3) <= 512 && ((unsigned)e3 * p.rb_s) % 1024u == 0;
-    if (combined) {
-        p.njobs = 1;
-        p.eslots = 2;
-        p.eslot_cols = e1 + e3;
-    } else {
-        p.njobs = 2;
-        p.eslot_cols = e1 > e3 ? e1 : e3;
-        p.eslots = 2 * p.s_slot_cols + 3 * p.eslot_cols <= 512 ? 3 : 2;
-        if (2 * p.s_slot_cols + p.eslots * p.eslot_cols > 512) return SQN_ERR_UNSUPPORTED;
+    p.BKs = s % 64 == 0 ? 64 : s % 32 == 0 ? 32 : 16;
+    p.chunks_s = s / p.BKs;
+    p.ksteps_s = p.BKs / 16;
+    p.rb_s = (unsigned)p.BKs * 2u;
+    if (p.chunks_s > 3) return SQN_ERR_UNSUPPORTED;
+    if (dsq) {
+        // the squeeze epilogue writes one swizzled row per patch pixel
+        if (p.chunks_s != 1 || Cin % 32 != 0) return SQN_ERR_UNSUPPORTED;
     }
+    p.tmem_cols = 512;
     p.c_tot = d1.out_c_total;
-    p.b_early = (dsq.params_static && d1.params_static && d3.params_static) ? 1 : 0;
-    p.bias_sq = dsq.bias; p.bias_e1 = d1.bias; p.bias_e3 = d3.bias;
+    p.b_early = ((!dsq || dsq->params_static) && d1.params_static && d3.params_static) ? 1 : 0;
+    p.bias_sq = dsq ? dsq->bias : nullptr; p.bias_e1 = d1.bias; p.bias_e3 = d3.bias;
     p.status = device_status_word();
+    p.s_slot_cols = dsq ? (s < 32 ? 32 : s) : 0;
 
-    // ---- shared-memory layout: two patches with an input ring of 32 KB or more and three slots or more, else one
-    // patch under the same condition, else whatever fits
-    {
+    // ---- over how many CTAs the output layers are split (the kernels of a part must fit in shared memory beside the
+    // patches), accumulators, shared-memory layout
+    bool found = false;
+    bool combined = false;
+    // (first the splits whose parts are whole 64-layer store chunks: half as many chunk hand-overs in the epilogue)
+    for (int round = 0; round < 2 && !found; ++round)
+    for (int cs = 1; cs <= (dsq ? 1 : 4) && !found; ++cs) {
+        if (e1 % (32 * cs) != 0 || e3 % (32 * cs) != 0) continue;
+        p.CS = cs; p.e3p = e3 / cs; p.e1p = e1 / cs;
+        p.CW = (p.e3p % 64 == 0 && p.e1p % 64 == 0) ? 64 : 32;
+        if ((p.CW == 64) != (round == 0)) continue;
+        if (9 * p.chunks_s * p.ksteps_s + p.chunks_s * p.ksteps_s > FF_MAX_EMMA) continue;
+        // TMEM: two squeeze accumulators (if any), then the expand accumulators.  Both expands in one accumulator (the
+        // 1x1 kernels ride on the centre tap) where two such accumulators fit, else two jobs per tile over three
+        // (or two) accumulators of max(e1p, e3p) columns.
+        combined = p.e3p + p.e1p <= 256 && 2 * p.s_slot_cols + 2 * (p.e1p + p.e3p) <= 512 && ((unsigned)p.e3p * p.rb_s) % 256u == 0;
+        if (combined) {
+            p.njobs = 1; p.eslots = 2; p.eslot_cols = p.e1p + p.e3p;
+        } else {
+            p.njobs = 2;
+            p.eslot_cols = p.e1p > p.e3p ? p.e1p : p.e3p;
+            if (p.eslot_cols > 256) continue;
+            p.eslots = 2 * p.s_slot_cols + 3 * p.eslot_cols <= 512 ? 3 : 2;
+            if (2 * p.s_slot_cols + p.eslots * p.eslot_cols > 512) continue;
+        }
+        // two patches with (if there is one) an input ring of 32 KB or more and three slots or more, else one patch
+        // under the same condition, else whatever fits
         int cand[8];
         const int nc = band_candidates(H, p.RT, cand);
-        bool found = false;
         for (int pass = 0; pass < 3 && !found; ++pass)
             for (int i = 0; i < nc && !found; ++i)
                 for (int patches = (pass == 1 ? 1 : 2); patches >= (pass == 0 ? 2 : 1) && !found; --patches)
                     for (int bk = 64; bk >= 32 && !found; bk -= 32) {
-                        if (Cin % bk != 0) continue;
-                        const int st = fire_layout(p, cand[i], patches, bk, &plan->smem);
-                        if (st == 0) continue;
-                        if (pass == 2 || (st >= 3 && (size_t)st * p.x_tile >= 32 * 1024)) found = true;
+                        if (dsq && Cin % bk != 0) continue;
+                        if (!dsq && bk != 64) continue;
+                        const int fit = fire_layout(p, cand[i], patches, bk, &plan->smem);
+                        if (fit == 0) continue;
+                        const int st = fit - 1;
+                        if (pass == 2 || !dsq || (st >= 3 && (size_t)st * p.x_tile >= 32 * 1024)) found = true;
                     }
-        if (!found) return SQN_ERR_UNSUPPORTED;
     }
+    if (!found) return SQN_ERR_UNSUPPORTED;
 
     // ---- MMAs of an expand tile
     {
         int e = 0;
-        auto tap_mmas = [&](int tap, unsigned b_off, int ncols) {
+        auto tap_mmas = [&](int tap, const unsigned* b_off, int ncols) {        // b_off: the tile of each chunk
             const int kh = tap / 3, kw = tap % 3;
-            for (int k = 0; k < p.ksteps_s; ++k, ++e) {
-                p.etab[e].x = (((unsigned)(kh * p.P + kw) * p.rb_s) >> 4) + 2u * k;
-                p.etab[e].y = (b_off >> 4) + 2u * k;
-                p.eidesc[e] = make_idesc_bf16(128, (unsigned)ncols);
-            }
+            for (int ch = 0; ch < p.chunks_s; ++ch)
+                for (int k = 0; k < p.ksteps_s; ++k, ++e) {
+                    p.etab[e].x = (((unsigned)ch * p.patch_chunk + (unsigned)(kh * p.P + kw) * p.rb_s) >> 4) + 2u * k;
+                    p.etab[e].y = (b_off[ch] >> 4) + 2u * k;
+                    p.eidesc[e] = make_idesc_bf16(128, (unsigned)ncols);
+                }
         };
         if (combined) {
-            // centre tap first: its B operand is the centre tap's kernels followed by the 1x1 kernels, and as the first
-            // MMA of the tile it overwrites all e3 + e1 columns; the other taps add to the first e3
+            // centre tap first: its B operand is the centre tap's kernels followed by the 1x1 kernels, and the tile's
+            // first MMA overwrites all e3p + e1p columns (with several chunks the later centre-tap MMAs add to all of
+            // them as well); the other taps add to the first e3p
             p.job_e0[0] = 0;
-            tap_mmas(4, p.off_tap[4], e3 + e1);
+            tap_mmas(4, p.off_w3[4], p.e3p + p.e1p);
             for (int tap = 0; tap < 9; ++tap)
-                if (tap != 4) tap_mmas(tap, p.off_tap[tap], e3);
+                if (tap != 4) tap_mmas(tap, p.off_w3[tap], p.e3p);
             p.job_en[0] = e;
-            p.job_chunk0[0] = 0; p.job_nchunks[0] = (e1 + e3) / FF_CW;
-            p.job_bias16[0] = 0; p.job_idesc[0] = make_idesc_bf16(128, (unsigned)(e3 + e1));
+            p.job_chunk0[0] = 0; p.job_nchunks[0] = (p.e1p + p.e3p) / p.CW;
+            p.job_bias16[0] = 0; p.job_idesc[0] = make_idesc_bf16(128, (unsigned)(p.e3p + p.e1p));
         } else {
             p.job_e0[0] = 0;
-            for (int tap = 0; tap < 9; ++tap) tap_mmas(tap, p.off_tap[tap], e3);
+            for (int tap = 0; tap < 9; ++tap) tap_mmas(tap, p.off_w3[tap], p.e3p);
             p.job_en[0] = e;
-            p.job_chunk0[0] = 0; p.job_nchunks[0] = e3 / FF_CW;
-            p.job_bias16[0] = 0; p.job_idesc[0] = make_idesc_bf16(128, (unsigned)e3);
+            p.job_chunk0[0] = 0; p.job_nchunks[0] = p.e3p / p.CW;
+            p.job_bias16[0] = 0; p.job_idesc[0] = make_idesc_bf16(128, (unsigned)p.e3p);
             p.job_e0[1] = e;
-            tap_mmas(4, p.off_w1, e1);                  // the 1x1 expand reads the centre pixel
+            tap_mmas(4, p.off_w1c, p.e1p);              // the 1x1 expand reads the centre pixel
             p.job_en[1] = e;
-            p.job_chunk0[1] = e3 / FF_CW; p.job_nchunks[1] = e1 / FF_CW;
-            p.job_bias16[1] = (unsigned)e3 * 2u;        // bias rows are 32 bytes each, the 3x3 expand's come first
-            p.job_idesc[1] = make_idesc_bf16(128, (unsigned)e1);
+            p.job_chunk0[1] = p.e3p / p.CW; p.job_nchunks[1] = p.e1p / p.CW;
+            p.job_bias16[1] = (unsigned)p.e3p * 2u;     // bias rows are 32 bytes each, the 3x3 expand's come first
+            p.job_idesc[1] = make_idesc_bf16(128, (unsigned)p.e1p);
         }
     }
-    // CTA b takes items b, b + grid, ...: with a grid that shares no factor with the bands per image every CTA
-    // meets all bands of an image in turn (they differ in height: the last one is shorter)
-    int g = sm_count();
+    // CS consecutive CTAs work on the same bands, one part of the output layers each; such a group takes bands g,
+    // g + groups, ...: with a group count that shares no factor with the bands per image every group meets all bands
+    // of an image in turn (they differ in height: the last one is shorter)
+    int g = sm_count() / p.CS;
+    if (g < 1) return SQN_ERR_UNSUPPORTED;
     if (p.items <= g) g = p.items;
     else
         while (g > 1 && std::__gcd(g, p.NB) != 1) --g;
-    p.grid = g;
+    p.grid = g * p.CS;
 
     // ---- tensor maps
-    {
-        // input as a flat list of pixels: [Cin][N*H*W], boxes of 128 pixels
-        const cuuint64_t npx = (cuuint64_t)N * H * W;
-        cuuint64_t dims[2] = {(cuuint64_t)Cin, npx};
-        cuuint64_t str[1] = {(cuuint64_t)Cin * 2};
-        cuuint32_t box[2] = {(cuuint32_t)p.BKc_in, 128};
-        if (!tmap_encode_bf16(&plan->x, 2, dsq.in, dims, str, box, p.rb_in)) return SQN_ERR_CUDA;
-    }
-    {
-        cuuint64_t dims[2] = {(cuuint64_t)Cin, (cuuint64_t)s};
-        cuuint64_t str[1] = {(cuuint64_t)Cin * 2};
-        cuuint32_t box[2] = {(cuuint32_t)p.BKc_in, (cuuint32_t)s};
-        if (!tmap_encode_bf16(&plan->wsq, 2, dsq.w, dims, str, box, p.rb_in)) return SQN_ERR_CUDA;
+    if (dsq) {
+        {
+            // input as a flat list of pixels: [Cin][N*H*W], boxes of 128 pixels
+            const cuuint64_t npx = (cuuint64_t)N * H * W;
+            cuuint64_t dims[2] = {(cuuint64_t)Cin, npx};
+            cuuint64_t str[1] = {(cuuint64_t)Cin * 2};
+            cuuint32_t box[2] = {(cuuint32_t)p.BKc_in, 128};
+            if (!tmap_encode_bf16(&plan->x, 2, dsq->in, dims, str, box, p.rb_in)) return SQN_ERR_CUDA;
+        }
+        {
+            cuuint64_t dims[2] = {(cuuint64_t)Cin, (cuuint64_t)s};
+            cuuint64_t str[1] = {(cuuint64_t)Cin * 2};
+            cuuint32_t box[2] = {(cuuint32_t)p.BKc_in, (cuuint32_t)s};
+            if (!tmap_encode_bf16(&plan->wsq, 2, dsq->w, dims, str, box, p.rb_in)) return SQN_ERR_CUDA;
+        }
+    } else {
+        // the squeeze map [s][W][H][N]: a patch box is P pixels x (R + 2) rows of one chunk of layers
+        if (p.R + 2 > 256) return SQN_ERR_UNSUPPORTED;
+        const cuuint64_t s1 = (cuuint64_t)s * 2;
+        cuuint64_t dims[5] = {(cuuint64_t)s, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N, 1};
+        cuuint64_t str[4] = {s1, s1 * W, s1 * W * H, s1 * W * H * N};
+        cuuint32_t box[5] = {(cuuint32_t)p.BKs, (cuuint32_t)p.P, (cuuint32_t)(p.R + 2), 1, 1};
+        if (!tmap_encode_bf16(&plan->x, 5, d1.in, dims, str, box, p.rb_s)) return SQN_ERR_CUDA;
+        plan->wsq = plan->x;            // (not read)
     }
     {
         cuuint64_t dims[2] = {(cuuint64_t)9 * s, (cuuint64_t)e3};
         cuuint64_t str[1] = {(cuuint64_t)9 * s * 2};
-        cuuint32_t box[2] = {(cuuint32_t)s, (cuuint32_t)e3};
+        cuuint32_t box[2] = {(cuuint32_t)p.BKs, (cuuint32_t)p.e3p};
         if (!tmap_encode_bf16(&plan->w3, 2, d3.w, dims, str, box, p.rb_s)) return SQN_ERR_CUDA;
     }
     {
         cuuint64_t dims[2] = {(cuuint64_t)s, (cuuint64_t)e1};
         cuuint64_t str[1] = {(cuuint64_t)s * 2};
-        cuuint32_t box[2] = {(cuuint32_t)s, (cuuint32_t)e1};
+        cuuint32_t box[2] = {(cuuint32_t)p.BKs, (cuuint32_t)p.e1p};
         if (!tmap_encode_bf16(&plan->w1, 2, d1.w, dims, str, box, p.rb_s)) return SQN_ERR_CUDA;
     }
     {
         const cuuint64_t s1 = (cuuint64_t)p.c_tot * 2;
         cuuint64_t dims[4] = {(cuuint64_t)(e1 + e3), (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
         cuuint64_t str[3] = {s1, s1 * W, s1 * W * H};
-        cuuint32_t box[4] = {(cuuint32_t)FF_CW, (cuuint32_t)W, (cuuint32_t)p.RT, 1};
-        if (!tmap_encode_bf16(&plan->o, 4, d1.out, dims, str, box, FF_CW * 2)) return SQN_ERR_CUDA;
+        cuuint32_t box[4] = {(cuuint32_t)p.CW, (cuuint32_t)W, (cuuint32_t)p.RT, 1};
+        if (!tmap_encode_bf16(&plan->o, 4, d1.out, dims, str, box, (unsigned)p.CW * 2u)) return SQN_ERR_CUDA;
     }
     return SQN_OK;
 }
@@ -796,31 +905,24 @@ struct FireKey {
 std::mutex g_fire_mu;
 std::map<std::string, FirePlan> g_fire_plans;
 
-}  // namespace
-
-bool fused_fire_enabled()
+int launch_fire(const ConvDesc* dsq, const ConvDesc& d1, const ConvDesc& d3, cudaStream_t stream)
 {
-    const char* v = std::getenv("SQN_FUSED_FIRE");        // read at every call: tests switch it
-    return !(v && v[0] == '0');
-}
-
-// The whole fire layer in one launch; SQN_ERR_UNSUPPORTED where the kernel does not apply (the caller then launches
-// the squeeze and the expands separately).
-int launch_fire_fused_bf16(const ConvDesc& dsq, const ConvDesc& d1, const ConvDesc& d3, cudaStream_t stream)
-{
-    if (dsq.K != 1 || d1.K != 1 || d3.K != 3 || d3.pad != 1 || dsq.S != 1 || d1.S != 1 || d3.S != 1 || !dsq.relu || !d1.relu ||
-        !d3.relu || dsq.pool || d1.pool || d3.pool || d1.in != dsq.out || d3.in != dsq.out || d1.Cin != dsq.Cout ||
-        d3.Cin != dsq.Cout || d1.H != dsq.H || d1.W != dsq.W || d1.N != dsq.N)
+    if (d1.K != 1 || d3.K != 3 || d3.pad != 1 || d1.S != 1 || d3.S != 1 || !d1.relu || !d3.relu || d1.pool || d3.pool ||
+        d1.in != d3.in || d1.Cin != d3.Cin || d1.H != d3.H || d1.W != d3.W || d1.N != d3.N)
+        return SQN_ERR_UNSUPPORTED;
+    if (dsq && (dsq->K != 1 || dsq->S != 1 || !dsq->relu || dsq->pool || d1.in != dsq->out || d1.Cin != dsq->Cout ||
+                d1.H != dsq->H || d1.W != dsq->W || d1.N != dsq->N))
         return SQN_ERR_UNSUPPORTED;
     FireKey k;
     std::memset(&k, 0, sizeof(k));
-    k.in = dsq.in; k.wsq = dsq.w; k.w1 = d1.w; k.w3 = d3.w; k.bsq = dsq.bias; k.b1 = d1.bias; k.b3 = d3.bias; k.out = d1.out;
+    k.in = dsq ? dsq->in : d1.in; k.wsq = dsq ? dsq->w : nullptr; k.w1 = d1.w; k.w3 = d3.w; k.bsq = dsq ? dsq->bias : nullptr;
+    k.b1 = d1.bias; k.b3 = d3.bias; k.out = d1.out;
     int dev = 0;
     cudaGetDevice(&dev);
     const char* bv = std::getenv("SQN_FIRE_BAND");
     const int band = bv ? std::atoi(bv) : 0;
-    const int v[12] = {dsq.N, dsq.Cin, dsq.H, dsq.W, dsq.Cout, d1.Cout, d3.Cout, d1.out_c_total,
-                       dsq.params_static | (d1.params_static << 1) | (d3.params_static << 2), dev, band, 0};
+    const int v[12] = {d1.N, dsq ? dsq->Cin : -1, d1.H, d1.W, d1.Cin, d1.Cout, d3.Cout, d1.out_c_total,
+                       (dsq ? dsq->params_static : 0) | (d1.params_static << 1) | (d3.params_static << 2), dev, band, 0};
     std::memcpy(k.v, v, sizeof(v));
     const std::string key(reinterpret_cast<const char*>(&k), sizeof(k));
     FirePlan plan;
@@ -845,6 +947,28 @@ int launch_fire_fused_bf16(const ConvDesc& dsq, const ConvDesc& d1, const ConvDe
     if (rc != cudaSuccess) return SQN_ERR_CUDA;
     note_launch();
     return cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
+}
+
+}  // namespace
+
+bool fused_fire_enabled()
+{
+    const char* v = std::getenv("SQN_FUSED_FIRE");        // read at every call: tests switch it
+    return !(v && v[0] == '0');
+}
+
+// The whole fire layer in one launch; SQN_ERR_UNSUPPORTED where the kernel does not apply (the caller then launches
+// the squeeze and the expands separately).
+int launch_fire_fused_bf16(const ConvDesc& dsq, const ConvDesc& d1, const ConvDesc& d3, cudaStream_t stream)
+{
+    return launch_fire(&dsq, d1, d3, stream);
+}
+
+// Both expands of a fire layer on a stored squeeze map in one launch of the same kernel (its expand pipeline alone, the
+// patch loaded by TMA, the output layers split over up to four CTAs so that each CTA's kernels stay in shared memory).
+int launch_fire_expands_bf16(const ConvDesc& d1, const ConvDesc& d3, cudaStream_t stream)
+{
+    return launch_fire(nullptr, d1, d3, stream);
 }
 
 }  // namespace sqn

@@ -55,6 +55,8 @@ inline int stem_packed_cols(int W) { return (W + 2) / 2 * 2; }
 // where that kernel does not apply.  SQN_FUSED_FIRE=0 in the environment turns it off.
 bool fused_fire_enabled();
 int launch_fire_fused_bf16(const ConvDesc& dsq, const ConvDesc& d1, const ConvDesc& d3, cudaStream_t stream);
+// Both expands on a stored squeeze map with the same kernel's expand pipeline (SQN_ERR_UNSUPPORTED where it does not apply).
+int launch_fire_expands_bf16(const ConvDesc& d1, const ConvDesc& d3, cudaStream_t stream);
 
 // Pooling / head.
 int launch_maxpool3x3s2(const void* in, void* out, int C, int H, int W, int N, int dtype, cudaStream_t stream);

@@ -320,11 +320,11 @@ def test_full_forward_bf16_small_batch_keeps_every_map():
 
 def test_plain_launches_give_the_same_values():
     """SQN_CHAINED_LAUNCH=0 (read once per process) launches every kernel without programmatic stream
-    serialisation and SQN_PAIR_LAUNCH=0 launches the two expands of a fire layer one after the other instead of
-    as one grid; a child process runs the batch-2 network that way and must reproduce this process's logits."""
+    serialisation; a child process runs the batch-2 network that way and must reproduce this process's logits bit
+    for bit.  With SQN_FUSED_FIRE=0 (tap-by-tap expand kernels) SQN_PAIR_LAUNCH=0 also launches the two expands of a
+    fire layer one after the other instead of as one grid: same logits again."""
     import os, subprocess, sys, tempfile
     x, params = synth.squeezenet_case(11, 2)
-    here = run_net(x, params, BF16, 2)[0]
     code = (
         "import sys, numpy as np; sys.path.insert(0, %r); sys.path.insert(0, %r)\n"
         "from paper_1611_07151_b200 import binding as B, synth\n"
@@ -332,12 +332,19 @@ def test_plain_launches_give_the_same_values():
         "x, params = synth.squeezenet_case(11, 2)\n"
         "np.save(sys.argv[1], run_net(x, params, B.SQN_BF16, 2)[0])\n"
     ) % (os.path.dirname(os.path.dirname(os.path.abspath(__file__))), os.path.dirname(os.path.abspath(__file__)))
-    with tempfile.TemporaryDirectory() as tmp:
-        out = os.path.join(tmp, "logits.npy")
-        env = dict(os.environ, SQN_CHAINED_LAUNCH="0", SQN_PAIR_LAUNCH="0")
-        subprocess.run([sys.executable, "-c", code, out], check=True, env=env, timeout=300)
-        there = np.load(out)
-    np.testing.assert_array_equal(here, there)
+    for fused, child_env in (("1", {"SQN_CHAINED_LAUNCH": "0"}),
+                             ("0", {"SQN_CHAINED_LAUNCH": "0", "SQN_PAIR_LAUNCH": "0", "SQN_FUSED_FIRE": "0"})):
+        os.environ["SQN_FUSED_FIRE"] = fused
+        try:
+            here = run_net(x, params, BF16, 2)[0]
+        finally:
+            os.environ.pop("SQN_FUSED_FIRE", None)
+        with tempfile.TemporaryDirectory() as tmp:
+            out = os.path.join(tmp, "logits.npy")
+            env = dict(os.environ, **child_env)
+            subprocess.run([sys.executable, "-c", code, out], check=True, env=env, timeout=300)
+            there = np.load(out)
+        np.testing.assert_array_equal(here, there)
 
 
 def test_host_buffer_forward_matches_device_forward_over_calls_in_a_row():

@@ -76,6 +76,7 @@ SHAPES = [
     (1, 32, 32, 64, 192, 31, 17),       # e1 != e3, odd extents
     (3, 64, 16, 64, 64, 3, 3),          # smaller than one tile
     (1, 32, 16, 64, 64, 1, 126),        # one row, widest supported map
+    (2, 32, 16, 32, 32, 10, 9),         # 32-layer store chunks
 ]
 
 
@@ -122,12 +123,43 @@ def test_fused_fire_many_items_per_cta():
     _check(got, exp, e)
 
 
-def test_shapes_outside_the_fused_kernel_take_the_separate_launches():
-    """s = 48 (fire6/7) and e1 + e3 > 256 (fire8/9) are not covered by the one-kernel path: fire_forward must still
-    give the layer, with more than one launch."""
-    for (N, cin, s, e, H) in [(2, 256, 48, 192, 27), (2, 512, 64, 256, 13)]:
-        x, sq, x1, x3 = _fire_case(N + s, N, cin, s, e, e, H, H)
-        exp = ref.fire(x, *sq, *x1, *x3)
-        got, launches, scratch = _run(x, sq, x1, x3)
-        assert launches >= 2 and not bool(scratch.isnan().any())
-        _check(got, exp, e)
+# (batch, Cin, s, e1, e3, H, W): layers whose kernels do not fit one CTA beside a squeeze pipeline
+SPLIT_SHAPES = [
+    (2, 256, 48, 192, 192, 27, 27),     # fire6: three 16-layer chunks per tap, output layers split over two CTAs
+    (2, 384, 48, 192, 192, 27, 27),     # fire7
+    (3, 512, 64, 256, 256, 13, 13),     # fire9: output layers split over four CTAs
+    (2, 384, 64, 256, 256, 27, 27),     # fire8 (without its pool)
+    (1, 64, 96, 64, 128, 21, 30),       # three 32-layer chunks, e1 != e3, non-square
+]
+
+
+@pytest.mark.parametrize("shape", SPLIT_SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_expands_on_a_stored_squeeze_map(shape):
+    """Where the one-kernel path does not apply (s = 48, or kernels too large for one CTA), fire_forward runs the squeeze
+    as its own launch and both expands as one launch of the flat-patch kernel (patch loaded by TMA, output layers
+    split over up to four CTAs)."""
+    N, cin, s, e1, e3, H, W = shape
+    x, sq, x1, x3 = _fire_case(sum(shape), N, cin, s, e1, e3, H, W)
+    exp = ref.fire(x, *sq, *x1, *x3)
+    got, launches, scratch = _run(x, sq, x1, x3)
+    assert launches == 2 and not bool(scratch.isnan().any())
+    _check(got, exp, e1)
+    # the tap-by-tap kernels on the same operands agree to output rounding
+    sep, launches, _ = _run(x, sq, x1, x3, fused=False)
+    assert launches >= 2
+    assert G.rel_err(got, sep) <= 1e-2
+
+
+def test_expands_many_bands_per_cta():
+    N, cin, s, e, H = 100, 256, 48, 192, 27                  # 400 bands on 73 groups of two CTAs
+    x, sq, x1, x3 = _fire_case(9, N, cin, s, e, e, H, H)
+    exp = ref.fire(x, *sq, *x1, *x3)
+    got, launches, _ = _run(x, sq, x1, x3)
+    assert launches == 2
+    _check(got, exp, e)
+    N, cin, s, e, H = 150, 512, 64, 256, 13                  # 150 images on 37 groups of four CTAs
+    x, sq, x1, x3 = _fire_case(10, N, cin, s, e, e, H, H)
+    exp = ref.fire(x, *sq, *x1, *x3)
+    got, launches, _ = _run(x, sq, x1, x3)
+    assert launches == 2
+    _check(got, exp, e)
