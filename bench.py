@@ -79,6 +79,17 @@ def launch_work(batch, es):
         o = (h - 3) // 2 + 1
         work[name] = {"flops": 0.0, "bytes": float(es * batch * c * (h * h + o * o))}
     work["head"] = {"flops": 0.0, "bytes": float(batch * (es * 1000 * 169 + 8 * 1000))}
+    # conv10, ReLU and the global average in one kernel: 512x13x13 in, 1000 means out; the softmax on its own
+    work["conv10+avgpool"] = {"flops": work["conv10"]["flops"],
+                              "bytes": float(batch * (es * 512 * 169 + 4 * 1000) + es * 1000 * 512 + 4 * 1000)}
+    work["softmax"] = {"flops": 0.0, "bytes": float(batch * 8 * 1000)}
+    # a whole fire layer in one kernel: input map in, both expands' output out, all kernels once
+    for i in range(2, 10):
+        f = "fire%d" % i
+        cin, s_, hw = [(c, co, h) for nm, c, co, k, st, pd, h in synth.SQUEEZENET_CONVS if nm == f + "_sq"][0]
+        e_ = [co for nm, c, co, *_ in synth.SQUEEZENET_CONVS if nm == f + "_e1"][0]
+        work[f + "_fused"] = {"flops": work[f + "_sq"]["flops"] + work[f + "_e1"]["flops"] + work[f + "_e3"]["flops"],
+                              "bytes": float(es * batch * hw * hw * (cin + 2 * e_) + es * (s_ * cin + 10 * e_ * s_) + 4 * (s_ + 2 * e_))}
     # repack of the stem's input (3 -> 4 layers, padded rows): an extra pass, counted at its real traffic
     work["conv1_pack"] = {"flops": 0.0, "bytes": float(batch * (IMG * IMG * 3 * 2 + 228 * 228 * 8))}
     # stem with its max-pool fused: the 96x111x111 map is never stored, only the pooled 96x55x55 one

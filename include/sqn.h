@@ -73,6 +73,11 @@ int conv_forward(const void* in, const void* weights, const void* bias, void* ou
  *   stream         cudaStream_t
  *   workspace,
  *   workspace_bytes  device scratch, needed only when conv_workspace_bytes reports > 0
+ *   fuse_global_avgpool   the global average pooling that follows the layer (paper Section III-E) is taken inside the
+ *                  kernel and the layer's own map is never stored: out is fp32 [batch][numOutputLayers], the mean over
+ *                  all outH x outW pixels of max(0, .) of the layer (or of the layer itself when relu is zero).
+ *                  SQN_BF16 only, K = 1, S = 1, pad = 0, numInputLayers a multiple of 64, at most 256 pixels per
+ *                  image, out_c_total = 0, not together with fuse_maxpool; otherwise SQN_ERR_UNSUPPORTED / SQN_ERR_BADARG.
  *   fuse_maxpool   the 3x3 / stride 2 max-pool that follows the layer (paper Section III-E) is applied inside the
  *                  kernel and only the pooled map is written: out is [batch][(outH-3)/2+1][(outW-3)/2+1][out_c_total].
  *                  SQN_BF16 only, stride 1 (or the stem shape), numOutputLayers a multiple of 32 up to 128, kernels
@@ -87,6 +92,7 @@ typedef struct {
     void* workspace;
     size_t workspace_bytes;
     int fuse_maxpool;   /* non-zero: out receives maxpool3x3/stride2 of the layer's output, extent ((outH-3)/2+1) */
+    int fuse_global_avgpool;   /* non-zero: out receives the per-layer mean of the layer's output, fp32 [batch][numOutputLayers] */
 } sqn_conv_opts;
 
 /*
@@ -192,7 +198,12 @@ int avgpool_softmax_forward(const void* in, void* logits_f32, void* probs_f32, i
  *   ("conv1", "pool1", "fire2_sq", "fire2", ..., "pool8", "fire9", "conv10");
  *   the data is in the net's dtype, NHWC, valid until the next forward.  From a batch of 16 on a bf16 net
  *   computes conv1+pool1, fire4+pool4 and fire8+pool8 in fused kernels and never stores the maps of conv1, fire4
- *   and fire8: asking for one of those then returns SQN_ERR_UNSUPPORTED.
+ *   and fire8: asking for one of those then returns SQN_ERR_UNSUPPORTED.  A bf16 net also runs the fire layers whose
+ *   kernels fit in shared memory (fire2, fire3, fire5; fire4 too below a batch of 16) as one kernel each, without
+ *   storing their squeeze maps, and takes conv10, its ReLU and the global average in one kernel without storing
+ *   conv10's map: "fireN_sq" of those layers and "conv10" then return SQN_ERR_UNSUPPORTED as well.  With
+ *   SQN_FUSED_FIRE=0 and SQN_FUSED_HEAD=0 in the environment (read at every call) these layers run as separate
+ *   launches and their maps can be read.
  */
 typedef struct sqn_net sqn_net;
 int squeezenet_create(sqn_net** net, const void* const* weights26, const void* const* bias26, int dtype,

@@ -30,7 +30,8 @@ _c_sz = ctypes.c_size_t
 
 class sqn_conv_opts(ctypes.Structure):
     _fields_ = [("dtype", _c_int), ("relu", _c_int), ("out_c_offset", _c_int), ("out_c_total", _c_int),
-                ("stream", _c_vp), ("workspace", _c_vp), ("workspace_bytes", _c_sz), ("fuse_maxpool", _c_int)]
+                ("stream", _c_vp), ("workspace", _c_vp), ("workspace_bytes", _c_sz), ("fuse_maxpool", _c_int),
+                ("fuse_global_avgpool", _c_int)]
 
 
 # name -> (restype, argtypes); the same list is checked against include/sqn.h by the tests
@@ -123,10 +124,10 @@ def conv_forward(inp, weights, bias, out, numInputLayers, numOutputLayers, H, W,
 
 def conv_forward_ex(inp, weights, bias, out, numInputLayers, numOutputLayers, H, W, K, S, pad, batch, dtype=SQN_F32,
                     relu=True, out_c_offset=0, out_c_total=0, stream=None, workspace=None, workspace_bytes=0,
-                    fuse_maxpool=False):
+                    fuse_maxpool=False, fuse_global_avgpool=False):
     opts = sqn_conv_opts(dtype, 1 if relu else 0, out_c_offset, out_c_total,
                          current_stream() if stream is None else stream, _p(workspace), workspace_bytes,
-                         1 if fuse_maxpool else 0)
+                         1 if fuse_maxpool else 0, 1 if fuse_global_avgpool else 0)
     _check(lib().conv_forward_ex(_p(inp), _p(weights), _p(bias), _p(out), numInputLayers, numOutputLayers, H, W, K, S,
                                  pad, batch, ctypes.byref(opts)), "conv_forward_ex")
 

@@ -150,6 +150,11 @@ extern "C" int conv_forward_ex(const void* in, const void* weights, const void* 
     const int rc = make_conv_desc(in, weights, bias, out, numInputLayers, numOutputLayers, H, W, K, S, pad, batch,
                                   o.relu, o.out_c_offset, o.out_c_total, &d);
     if (rc != SQN_OK) return rc;
+    if (o.fuse_global_avgpool) {
+        if (o.fuse_maxpool || o.out_c_total != 0) return SQN_ERR_BADARG;
+        if (o.dtype != SQN_BF16) return SQN_ERR_UNSUPPORTED;
+        return launch_conv_avgpool_bf16(d, static_cast<float*>(out), static_cast<cudaStream_t>(o.stream));
+    }
     if (o.fuse_maxpool) {
         if (d.OH < 3 || d.OW < 3) return SQN_ERR_BADARG;
         d.pool = 1;
@@ -314,6 +319,7 @@ struct sqn_net {
     int copy_device = -1;
     unsigned long long host_calls = 0;
     int stem_prepacked = 0;     // squeezenet_set_stem_prepacked
+    int fused_head = 0;             // the last forward took conv10 and the average in one kernel (conv10's map was not stored)
     unsigned fused_fire_mask = 0;   // bit i: the last forward ran fire layer i as one kernel (its squeeze map was not stored)
 };
 
@@ -436,6 +442,7 @@ extern "C" int squeezenet_layer_output(const sqn_net* net, const char* name, voi
     if (net->dtype == SQN_BF16 && batch >= 16 &&
         (std::strcmp(name, "conv1") == 0 || std::strcmp(name, "fire4") == 0 || std::strcmp(name, "fire8") == 0))
         return SQN_ERR_UNSUPPORTED;   // computed inside the kernels that write pool1 / pool4, never stored
+    if (net->fused_head && std::strcmp(name, "conv10") == 0) return SQN_ERR_UNSUPPORTED;     // averaged inside the kernel
     for (int f = 0; f < 8; ++f)
         if ((net->fused_fire_mask >> f & 1u) && std::string(kFire[f].name) + "_sq" == name)
             return SQN_ERR_UNSUPPORTED;   // kept in shared memory by the fused fire kernel of the last forward
@@ -641,6 +648,23 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
     rc = make_conv_desc(cur, net->w[25], net->b[25], buf("conv10"), 512, 1000, 13, 13, 1, 1, 0, batch, 1, 0, 0, &d);
     if (rc != SQN_OK) return rc;
     d.params_static = 1;
+    net->fused_head = 0;
+    if (dt == SQN_BF16 && fused_head_enabled()) {
+        // conv10, ReLU and the global average in one kernel: the 1000 x 13 x 13 map is never stored
+        rc = launch_conv_avgpool_bf16(d, static_cast<float*>(logits_f32), st);
+        if (rc == SQN_OK) {
+            net->fused_head = 1;
+            mark("conv10+avgpool");
+            if (probs_f32) {
+                if ((rc = launch_softmax(static_cast<const float*>(logits_f32), static_cast<float*>(probs_f32), 1000, batch, st)) != SQN_OK)
+                    return rc;
+                mark("softmax");
+            }
+            if (prof) net->prof_forwards++;
+            return SQN_OK;
+        }
+        if (rc != SQN_ERR_UNSUPPORTED) return rc;
+    }
     if ((rc = run_conv(d, dt, nullptr, 0, st)) != SQN_OK) return rc;
     mark("conv10");
     rc = launch_avgpool_softmax(buf("conv10"), static_cast<float*>(logits_f32), static_cast<float*>(probs_f32), 1000,

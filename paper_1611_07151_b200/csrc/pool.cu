@@ -282,11 +282,14 @@ int launch_avgpool_softmax(const void* in, float* logits, float* probs, int C, i
     else launch_chained(global_avgpool_kernel<true>, grid, dim3(256), 0, stream, in, logits, C, H * W);
     note_launch();
     if (cudaGetLastError() != cudaSuccess) return SQN_ERR_CUDA;
-    if (probs) {
-        launch_chained(softmax_kernel, dim3((unsigned)N), dim3(256), (size_t)C * sizeof(float), stream,
-                       static_cast<const float*>(logits), probs, C);
-        note_launch();
-    }
+    if (probs) return launch_softmax(logits, probs, C, N, stream);
+    return SQN_OK;
+}
+
+int launch_softmax(const float* logits, float* probs, int C, int N, cudaStream_t stream)
+{
+    launch_chained(softmax_kernel, dim3((unsigned)N), dim3(256), (size_t)C * sizeof(float), stream, logits, probs, C);
+    note_launch();
     return cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
 }
 

@@ -58,10 +58,16 @@ int launch_fire_fused_bf16(const ConvDesc& dsq, const ConvDesc& d1, const ConvDe
 // Both expands on a stored squeeze map with the same kernel's expand pipeline (SQN_ERR_UNSUPPORTED where it does not apply).
 int launch_fire_expands_bf16(const ConvDesc& d1, const ConvDesc& d3, cudaStream_t stream);
 
+// 1x1 convolution + ReLU + global average in one launch (the map is not stored): logits[n][m], fp32.
+// SQN_FUSED_HEAD=0 in the environment turns its use by squeezenet_forward off.
+bool fused_head_enabled();
+int launch_conv_avgpool_bf16(const ConvDesc& d, float* logits, cudaStream_t stream);
+
 // Pooling / head.
 int launch_maxpool3x3s2(const void* in, void* out, int C, int H, int W, int N, int dtype, cudaStream_t stream);
 int launch_avgpool_softmax(const void* in, float* logits, float* probs, int C, int H, int W, int N, int dtype,
                            cudaStream_t stream);
+int launch_softmax(const float* logits, float* probs, int C, int N, cudaStream_t stream);
 
 // Chained launches.  A kernel launched through launch_chained() may be scheduled while the kernel before it
 // in the stream is still running (programmatic stream serialisation): its blocks take the SMs the earlier

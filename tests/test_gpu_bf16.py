@@ -204,7 +204,8 @@ def test_config3_headline_batch256_all_images_against_the_oracle():
     x, params = synth.squeezenet_case(3, batch)
     logits, probs, views = run_net_device(x, params, BF16, batch)
     assert "conv1" not in views and "fire4" not in views and "fire8" not in views       # fused with their pools
-    assert {"pool1", "pool4", "pool8", "conv10", "fire2", "fire6_sq", "fire9"} <= set(views)
+    assert {"pool1", "pool4", "pool8", "fire2", "fire6_sq", "fire9"} <= set(views)
+    assert "conv10" not in views and "fire2_sq" not in views         # averaged / kept in shared memory inside fused kernels
     worst_d = {n: 0.0 for n in views}
     worst_r = {n: 0.0 for n in views}
     zs = []
@@ -296,23 +297,26 @@ def test_full_forward_bf16_batch32():
 
 def test_full_forward_bf16_small_batch_keeps_every_map():
     """Below a batch of 16 the pools are separate kernels; with SQN_FUSED_FIRE=0 (read at every call) the fire layers
-    are separate launches too and every intermediate map can be read back.  By default the squeeze maps of the fire
+    and the head are separate launches too (SQN_FUSED_HEAD=0) and every intermediate map can be read back.  By default the squeeze maps of the fire
     layers that run as one kernel are not stored, and the logits agree with the separate launches to rounding."""
     import os
     x, params = synth.squeezenet_case(7, 2)
     trace = {}
     z, _ = ref.squeezenet(x, params, trace=trace)
     os.environ["SQN_FUSED_FIRE"] = "0"
+    os.environ["SQN_FUSED_HEAD"] = "0"
     try:
         logits, probs, layers = run_net(x, params, BF16, 2)
     finally:
         os.environ.pop("SQN_FUSED_FIRE", None)
+        os.environ.pop("SQN_FUSED_HEAD", None)
     assert "conv1" in layers and "fire4" in layers and len(layers) == len(trace) - 2      # all but logits, probs
     assert max(G.rel_err(got, trace[name]) for name, got in layers.items()) <= 5e-2
     assert G.rel_err(logits, z) <= TOL
     np.testing.assert_allclose(probs.astype(np.float64).sum(1), 1.0, rtol=0, atol=1e-5)
     logits_f, _probs, layers_f = run_net(x, params, BF16, 2)
     assert "fire2_sq" not in layers_f and "fire5_sq" not in layers_f and "fire2" in layers_f and "fire6_sq" in layers_f
+    assert "conv10" not in layers_f
     assert max(G.rel_err(got, trace[name]) for name, got in layers_f.items()) <= 5e-2
     assert G.rel_err(logits_f, z) <= TOL
     assert G.rel_err(logits_f, logits) <= 1e-2
@@ -443,3 +447,48 @@ def test_stem_operands_packed_offline_give_the_same_logits(batch):
     assert B.sqn_check() == B.SQN_OK
     assert B.sqn_launch_count() - n0 == launches + 1
     B.squeezenet_destroy(net2)
+
+
+# (N, Cin, Cout, H, W)
+HEAD_SHAPES = [
+    (3, 512, 1000, 13, 13),        # conv10: eight layer tiles, the last one ragged; 169 pixels in an MMA of 176
+    (40, 512, 1000, 13, 13),       # several images per CTA (18 groups of eight CTAs): both accumulators reused
+    (2, 64, 128, 4, 5),            # one tile, one reduction chunk, 20 pixels
+    (5, 128, 200, 16, 16),         # 256 pixels: the widest MMA
+    (4, 64, 40, 1, 1),             # a single pixel per image
+]
+
+
+@pytest.mark.parametrize("shape", HEAD_SHAPES, ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("relu", [True, False])
+def test_conv_with_fused_global_average(shape, relu):
+    """fuse_global_avgpool: 1x1 convolution, ReLU and the global average in one kernel; only the fp32 means are
+    written.  Against the oracle's convolution followed by its global average."""
+    import torch
+    N, C, M, H, W = shape
+    rng = np.random.default_rng(sum(shape))
+    x = synth.draw_input(rng, (N, C, H, W)) - (0.0 if relu else 0.5)
+    w, b = synth.draw_conv_params(rng, C, M, 1)
+    b = b + np.float32(0.1) * rng.standard_normal(M).astype(np.float32)
+    exp = ref.global_avgpool(ref.conv2d(x, w, b, S=1, pad=0, relu=relu))
+    out = torch.full((N, M), float("nan"), device="cuda")
+    B.conv_forward_ex(G.dev_act(x, BF16), G.dev_w(w, BF16), G.dev_b(b), out, C, M, H, W, 1, 1, 0, N, dtype=BF16, relu=relu,
+                      fuse_global_avgpool=True)
+    assert B.sqn_check() == B.SQN_OK
+    got = out.cpu().numpy()
+    assert not np.isnan(got).any()
+    assert G.rel_err(got, exp) <= TOL
+    # tighter: the oracle on the same bf16-rounded operands (the kernel rounds nothing else)
+    exp_r = ref.global_avgpool(ref.conv2d(bf16_round(x), bf16_round(w), b, S=1, pad=0, relu=relu))
+    assert G.rel_err(got, exp_r) <= 1e-4
+
+
+def test_fused_global_average_is_refused_where_it_cannot_run():
+    import torch
+    p = torch.empty(64, device="cuda")
+    for (dtype, cin, k, hw, pool) in [(B.SQN_F32, 64, 1, 13, False), (BF16, 48, 1, 13, False), (BF16, 64, 3, 13, False),
+                                      (BF16, 64, 1, 17, False), (BF16, 64, 1, 13, True)]:
+        with pytest.raises(B.SqnError) as e:
+            B.conv_forward_ex(p, p, p, p, cin, 32, hw, hw, k, 1, k // 2, 1, dtype=dtype, fuse_global_avgpool=True,
+                              fuse_maxpool=pool)
+        assert e.value.status in (B.SQN_ERR_UNSUPPORTED, B.SQN_ERR_BADARG)
