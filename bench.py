@@ -434,6 +434,90 @@ def run_variants(B, batch):
                       "median of 10, microseconds; a missing variant does not fit the layer"}))
 
 
+def run_kernel_case(B, name, batch, steps):
+    """One layer (or fire layer, or the fused head) of the network on its own, bf16, seed-4 recipe drawn on the device:
+    `steps` back-to-back launches over rotating buffer sets larger than the L2 (mean), then single launches with the L2
+    overwritten in between (median).  The small cases of the ncu captures under profiles/ are runs of this mode."""
+    import torch
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(4)
+    bf = torch.bfloat16
+    convs = {n: (cin, cout, k, s, pad, hw) for n, cin, cout, k, s, pad, hw in synth.SQUEEZENET_CONVS}
+
+    def conv_params(cin, cout, k):
+        w = (torch.randn((cout, k, k, cin), device=dev, generator=gen) * (2.0 / (cin * k * k)) ** 0.5).to(bf)
+        return w, torch.randn((cout,), device=dev, generator=gen) * 0.01
+
+    sets = []
+    if name.startswith("fire") and "_" not in name:
+        cin, s_, _k, _s, _p, hw = convs[name + "_sq"]
+        e = convs[name + "_e1"][1]
+        wsq, bsq = conv_params(cin, s_, 1)
+        w1, b1 = conv_params(s_, e, 1)
+        w3, b3 = conv_params(s_, e, 3)
+        per_set = batch * hw * hw * (cin + s_ + 2 * e) * 2
+        nsets = max(2, int(200e6 // per_set) + 1)
+        for _ in range(nsets):
+            sets.append((torch.rand((batch, hw, hw, cin), device=dev, generator=gen).to(bf),
+                         torch.empty((batch, hw, hw, s_), device=dev, dtype=bf), torch.empty((batch, hw, hw, 2 * e), device=dev, dtype=bf)))
+
+        def call(i):
+            x, sc, out = sets[i % nsets]
+            B.fire_forward(x, wsq, bsq, w1, b1, w3, b3, sc, out, cin, s_, e, e, hw, hw, batch, B.SQN_BF16)
+        flops = 2.0 * batch * hw * hw * (cin * s_ + 10 * s_ * e)
+        byts = 2.0 * batch * hw * hw * (cin + 2 * e)
+    else:
+        base = name.split("+")[0]
+        cin, cout, k, s_, pad, hw = convs[base]
+        pool, avg = name.endswith("+pool") or name.endswith("+pool1"), name.endswith("+avgpool")
+        oh = (hw + 2 * pad - k) // s_ + 1
+        w, b = conv_params(cin, cout, k)
+        nb = B.conv_workspace_bytes(cin, cout, hw, hw, k, s_, pad, batch, B.SQN_BF16)
+        po = (oh - 3) // 2 + 1
+        out_shape = (batch, cout) if avg else ((batch, po, po, cout) if pool else (batch, oh, oh, cout))
+        per_set = batch * hw * hw * cin * 2 + int(np.prod(out_shape)) * 2
+        nsets = max(2, int(200e6 // per_set) + 1)
+        for _ in range(nsets):
+            sets.append((torch.rand((batch, hw, hw, cin), device=dev, generator=gen).to(bf),
+                         torch.empty(out_shape, device=dev, dtype=torch.float32 if avg else bf),
+                         torch.empty(max(nb, 16), dtype=torch.uint8, device=dev)))
+
+        def call(i):
+            x, out, wsb = sets[i % nsets]
+            B.conv_forward_ex(x, w, b, out, cin, cout, hw, hw, k, s_, pad, batch, dtype=B.SQN_BF16, workspace=wsb,
+                              workspace_bytes=nb, fuse_maxpool=pool, fuse_global_avgpool=avg)
+        flops = 2.0 * batch * oh * oh * cout * cin * k * k
+        byts = 2.0 * batch * hw * hw * cin + (4.0 if avg else 2.0) * float(np.prod(out_shape))
+    for i in range(5):
+        call(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        call(i)
+    e1.record()
+    torch.cuda.synchronize()
+    mean_us = e0.elapsed_time(e1) / steps * 1e3
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    singles = []
+    for i in range(min(steps, 20)):
+        flush.zero_()
+        a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        call(i)
+        c.record()
+        torch.cuda.synchronize()
+        singles.append(a.elapsed_time(c) * 1e3)
+    assert B.sqn_check() == B.SQN_OK
+    peaks = measured_peaks()
+    print(json.dumps({"kernel_case": name, "batch": batch, "steps": steps, "us_mean_back_to_back": mean_us,
+                      "us_median_single_cold": float(np.median(singles)), "tflops": flops / mean_us / 1e6,
+                      "gbs": byts / mean_us / 1e3, "frac_tensor_burst": flops / mean_us / 1e6 / peaks["bf16_tflops"],
+                      "frac_hbm": byts / mean_us / 1e3 / peaks["hbm_gbs"], "buffer_sets": nsets}))
+
+
 def workload_name(args):
     return "squeezenet_v1.0_forward_b%d_%s" % (args.batch, args.dtype)
 
@@ -452,6 +536,8 @@ def main():
     ap.add_argument("--no-batch1", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="per-layer sweep of every conv shape instead of the network")
     ap.add_argument("--variants", action="store_true", help="per-layer sweep of the bf16 kernel variants at --batch")
+    ap.add_argument("--kernel", default=None, help="one layer on its own (bf16): a conv name (conv1, fire6_e3, ...), "
+                    "NAME+pool, conv10+avgpool, or a fire layer (fire2 ... fire9)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -468,6 +554,9 @@ def main():
         return
     if args.variants:
         run_variants(B, args.batch)
+        return
+    if args.kernel:
+        run_kernel_case(B, args.kernel, args.batch, args.steps)
         return
 
     rank, local_rank, world = D.env_world()

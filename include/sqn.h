@@ -285,6 +285,16 @@ int sqn_unpack_nhwc_to_nchw(const void* src, float* dst, int N, int C, int H, in
  */
 int sqn_check(void* stream);
 
+/*
+ * Self-test of the failure path every kernel of the library shares.  All device-side waits are bounded: when one
+ * runs out the CTA records SQN_ERR_TIMEOUT, lets its outstanding copies land, frees its tensor memory and returns,
+ * so the context stays usable and the next sqn_check reports the error.  This call launches one small CTA that
+ * waits, for at most limit_cycles SM clocks (1e3 .. 2e9), on a barrier nothing arrives on.  After it, sqn_check
+ * returns SQN_ERR_TIMEOUT once, then SQN_OK, and every other entry point works as before.  (Diagnostic: the paper
+ * has no counterpart.)
+ */
+int sqn_selftest_wait_timeout(long long limit_cycles, void* stream);
+
 /* Static, human-readable name of a status code. */
 const char* sqn_status_string(int status);
 

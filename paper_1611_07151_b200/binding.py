@@ -63,6 +63,7 @@ SIGNATURES = {
     "sqn_pack_nchw_to_nhwc": (_c_int, [_c_vp, _c_vp] + [_c_int] * 5),
     "sqn_unpack_nhwc_to_nchw": (_c_int, [_c_vp, _c_vp] + [_c_int] * 5),
     "sqn_check": (_c_int, [_c_vp]),
+    "sqn_selftest_wait_timeout": (_c_int, [ctypes.c_longlong, _c_vp]),
     "sqn_status_string": (ctypes.c_char_p, [_c_int]),
     "sqn_launch_count": (ctypes.c_ulonglong, []),
 }
@@ -258,6 +259,11 @@ def squeezenet_profile_read(net):
 
 def sqn_check(stream=None):
     return lib().sqn_check(current_stream() if stream is None else stream)
+
+
+def sqn_selftest_wait_timeout(limit_cycles, stream=None):
+    _check(lib().sqn_selftest_wait_timeout(limit_cycles, current_stream() if stream is None else stream),
+           "sqn_selftest_wait_timeout")
 
 
 def sqn_status_string(status):

@@ -602,8 +602,14 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
             }
             if (fits) {
                 if (pair_launch_enabled()) {
+                    // the 1x1 expand riding on the 3x3 expand's patches (per slice of 128 layers), all in one launch
                     bool done = false;
-                    if (parts == 2) {           // both slices of both expands as one grid, the 3x3 slices first
+                    if (parts <= 2) {
+                        rc = launch_conv_bf16_pool_riders(q3, q1, parts, st);
+                        if (rc != SQN_OK && rc != SQN_ERR_UNSUPPORTED) return rc;
+                        done = rc == SQN_OK;
+                    }
+                    if (!done && parts == 2) {  // both slices of both expands as one grid, the 3x3 slices first
                         const ConvDesc four[4] = {q3[0], q3[1], q1[0], q1[1]};
                         rc = launch_conv_bf16_pool4(four, st);
                         if (rc != SQN_OK && rc != SQN_ERR_UNSUPPORTED) return rc;
@@ -883,6 +889,12 @@ extern "C" int sqn_check(void* stream)
         if (cudaMemcpy(word, &zero, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) return SQN_ERR_CUDA;
     }
     return v;
+}
+
+extern "C" int sqn_selftest_wait_timeout(long long limit_cycles, void* stream)
+{
+    if (limit_cycles < 1000 || limit_cycles > 2000000000LL) return SQN_ERR_BADARG;
+    return launch_wait_timeout_selftest(limit_cycles, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" const char* sqn_status_string(int status)

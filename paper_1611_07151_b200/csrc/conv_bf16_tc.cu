@@ -106,6 +106,16 @@ struct TcParams {
     int pool_ctot;                   // layers per pixel of the pooled tensor
     __nv_bfloat16* pool_out;
     int npix;                        // conv_pool_kernel: pixels per tile, 256 or 128
+    // conv_pool_kernel: a second layer, 1x1 on the same input with as many output layers, that rides on this layer's
+    // patches: after a tile's own MMAs the rider's go into the other accumulator from the same patch, and the epilogue
+    // pools both (the 1x1 expand of a fire layer beside the 3x3 expand)
+    int rider;
+    int r_nmma;                      // the rider's MMAs per tile
+    unsigned r_off_b, r_off_bias;    // its kernels (chunks tiles of Cout rows) and bias rows in shared memory
+    unsigned r_b_bytes;              // bytes of its kernels
+    int r_c_off;                     // its first output layer in the pooled tensor
+    const float* r_bias;
+    uint2 r_ptab[8];                 // per MMA {patch offset, kernel offset from r_off_b}, 16-byte units
     const float* bias;
     int* status;
     // patch mode, at most PARAM_TAB MMAs per tile: per MMA {A offset from the stage base, B offset from the
@@ -627,8 +637,8 @@ __host__ __device__ constexpr int poolt_prows(int npix) { return (npix / 8 - 2) 
 // NPIX = 256 (8 x 32 pixels per tile, 15 pooled rows per strip) where the layer's kernels leave room for the larger
 // patches, else 128 (8 x 16 pixels, 7 pooled rows).
 template <int NPIX>
-
-__device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUtensorMap& tmB, const TcParams& p, const int bid)
+__device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB2,
+                                               const TcParams& p, const int bid)
 {
     constexpr int PROWS = poolt_prows(NPIX);          // 15 or 7
     constexpr int PR = (PROWS + 3) / 4;               // pooled rows per epilogue group: 4 or 2
@@ -649,6 +659,32 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
     const int items = p.taps * p.chunks;
     const int nmma = items * (p.BKc / 16);
     const int my_tiles = tiles_of_cta(p, bid);
+    // every kernel tile of the layer (and of its rider), once: one mbarrier counts them all
+    auto load_kernels = [&]() {
+        const uint32_t bar = smem_u32(&sh->b_full);
+        mbar_arrive_expect_tx(bar, (uint32_t)items * p.b_bytes + (p.rider ? p.r_b_bytes : 0u));
+        int tap = 0, ch = 0;
+        for (int i = 0; i < items; ++i) {
+            tma_load_2d(smB + (uint32_t)i * p.b_tile, &tmB, bar, tap * p.k_per_tap + ch * p.BKc, 0);
+            if (++ch == p.chunks) { ch = 0; ++tap; }
+        }
+        if (p.rider)
+            for (int c = 0; c < p.chunks; ++c) tma_load_2d(base + p.r_off_b + (uint32_t)c * p.b_tile, &tmB2, bar, c * p.BKc, 0);
+    };
+    auto fill_bias = [&]() {
+        fill_bias_rows<POOLT_THREADS>(p, base_ptr);
+        if (p.rider) {
+            uint4* rows = reinterpret_cast<uint4*>(base_ptr + p.r_off_bias);
+            for (int c = threadIdx.x; c < TILE_M; c += POOLT_THREADS) {
+                const float b = c < p.Cout ? __ldg(p.r_bias + c) : 0.f;
+                const __nv_bfloat16 hi = __float2bfloat16_rn(b);
+                const __nv_bfloat16 lo = __float2bfloat16_rn(b - __bfloat162float(hi));
+                const int u = (c >> 2) & 1;
+                rows[2 * c + u] = make_uint4((uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16), 0u, 0u, 0u);
+                rows[2 * c + (u ^ 1)] = make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
+    };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -664,7 +700,7 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
         fence_mbar_init();
         prefetch_tensormap(&tmA);
         prefetch_tensormap(&tmB);
-        if (p.b_early) load_resident_kernels(p, tmB, smB, smem_u32(&sh->b_full), items);
+        if (p.b_early) load_kernels();
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(&sh->tmem_base), p.tmem_cols);
@@ -683,9 +719,9 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
             ones[2 * r + (u ^ 1)] = make_uint4(0u, 0u, 0u, 0u);
         }
     }
-    if (p.b_early) fill_bias_rows<POOLT_THREADS>(p, base_ptr);
+    if (p.b_early) fill_bias();
     chain_wait();       // the earlier grid has finished: its output may be read from here on
-    if (!p.b_early) fill_bias_rows<POOLT_THREADS>(p, base_ptr);
+    if (!p.b_early) fill_bias();
     fence_proxy_async_smem();
     tc_fence_before();
     __syncthreads();
@@ -696,7 +732,7 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer: one patch per tile
         if (lane == 0) {
-            if (!p.b_early) load_resident_kernels(p, tmB, smB, smem_u32(&sh->b_full), items);
+            if (!p.b_early) load_kernels();
             bool ok = true;
             int s = 0, issued = 0;
             uint32_t ph = 0;
@@ -758,13 +794,35 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
                                 ((uint64_t)hiX << 32) | (uint64_t)((x_base + o.x) | 0x10000u), idesc, acc);
                     acc = 1u;
                 }
-                mma_commit(smem_u32(&sh->empty[s]));                // patch slot free once these MMAs have read it
+                if (!p.rider) mma_commit(smem_u32(&sh->empty[s]));  // patch slot free once these MMAs have read it
                 if (!p.bias_in_k) mma_bf16_ss(d_tmem, bias_desc, ones_desc, idesc, 1u);
                 mma_commit(smem_u32(&sh->tmem_full[as]));           // accumulator complete
             }
             __syncwarp();
-            if (++s == p.stages) { s = 0; ph ^= 1u; }
             if (++as == 2) { as = 0; aph ^= 1u; }
+            if (p.rider) {
+                // the rider's tile from the same patch, into the other accumulator
+                ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_empty[as]), aph ^ 1u, abort_flag, p.status));
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d2 = tmem_base + (uint32_t)(as * NPIX);
+                if (elect_one()) {
+                    const uint32_t smR16 = (base + p.r_off_b) >> 4;
+                    uint32_t acc = 0u;
+                    for (int e = 0; e < p.r_nmma; ++e) {
+                        const uint2 o = p.r_ptab[e];
+                        mma_bf16_ss(d2, ((uint64_t)hiW << 32) | (uint64_t)((smR16 + o.y) | 0x10000u),
+                                    ((uint64_t)hiX << 32) | (uint64_t)((x_base + o.x) | 0x10000u), idesc, acc);
+                        acc = 1u;
+                    }
+                    mma_commit(smem_u32(&sh->empty[s]));            // patch slot free once both layers have read it
+                    mma_bf16_ss(d2, make_kmajor_desc(base + p.r_off_bias, 32u, 256u), ones_desc, idesc, 1u);
+                    mma_commit(smem_u32(&sh->tmem_full[as]));
+                }
+                __syncwarp();
+                if (++as == 2) { as = 0; aph ^= 1u; }
+            }
+            if (++s == p.stages) { s = 0; ph ^= 1u; }
         }
     } else {
         // -------------------------------------------------------------------- epilogue: pool in registers
@@ -775,23 +833,23 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
         const bool live = m < p.Cout, warp_live = q * 32 < p.Cout;
         const int row_stride = p.PW_out * p.pool_ctot;             // elements between pooled rows
-        float carry[PR][2];
+        float carry[PR][2], carry2[PR][2];              // (carry2: the rider's)
 #pragma unroll
-        for (int r = 0; r < PR; ++r) carry[r][0] = carry[r][1] = 0.f;
+        for (int r = 0; r < PR; ++r) carry[r][0] = carry[r][1] = carry2[r][0] = carry2[r][1] = 0.f;
         bool ok = true;
         int as = 0;
         uint32_t aph = 0;
         TileCoord tc;
         tile_first(p, bid, tc);
-        // (warps whose lanes lie past the last output layer have nothing to do and are not counted by tmem_empty)
-        for (int it = 0; it < my_tiles && ok && warp_live; ++it, tile_next(p, tc)) {
+        // one accumulator -> pooled pixels of one layer; `cr` carries the vertical maxima of the tile's last two columns
+        auto pool_tile = [&](float (&cr)[PR][2], const int c_off) {
             ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_full[as]), aph, abort_flag, p.status));
-            if (!ok) break;
+            if (!ok) return;
             tc_fence_after();
             const uint32_t taddr = tmem_base + lane_base + (uint32_t)(as * NPIX) + (uint32_t)(grp * 16 * PR);
             const int pw0 = tc.tw * 4 - 1, ph0 = tc.th * PROWS + grp * PR;
             unsigned short* dst0 = reinterpret_cast<unsigned short*>(p.pool_out) +
-                                   (((size_t)tc.ti * p.PH_out + ph0) * p.PW_out + pw0) * p.pool_ctot + p.c_off + m;
+                                   (((size_t)tc.ti * p.PH_out + ph0) * p.PW_out + pw0) * p.pool_ctot + c_off + m;
             const bool first = pw0 >= 0 && pw0 < p.PW_out, last3 = pw0 + 3 < p.PW_out, last2 = pw0 + 2 < p.PW_out,
                        last1 = pw0 + 1 < p.PW_out;
             // ROUNDS rounds of 2*RPR + 1 tile rows (RCOLS accumulator columns) = RPR pooled rows each
@@ -823,10 +881,10 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
                     for (int j = 0; j < 8; ++j)                         // vertical maximum of rows 2r, 2r+1, 2r+2, column j
                         c[j] = max3(__uint_as_float(v[16 * r2 + j]), __uint_as_float(v[16 * r2 + 8 + j]),
                                     __uint_as_float(v[16 * r2 + 16 + j]));
-                    const float o0 = max3(carry[r][0], carry[r][1], c[0]), o1 = max3(c[0], c[1], c[2]),
+                    const float o0 = max3(cr[r][0], cr[r][1], c[0]), o1 = max3(c[0], c[1], c[2]),
                                 o2 = max3(c[2], c[3], c[4]), o3 = max3(c[4], c[5], c[6]);
-                    carry[r][0] = c[6];
-                    carry[r][1] = c[7];
+                    cr[r][0] = c[6];
+                    cr[r][1] = c[7];
                     if (live && ph0 + r < p.PH_out) {
                         unsigned short* dst = dst0 + r * row_stride;
                         if (first) dst[0] = to_bf16_bits(o0, p.relu);
@@ -836,6 +894,11 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
                     }
                 }
             }
+        };
+        // (warps whose lanes lie past the last output layer have nothing to do and are not counted by tmem_empty)
+        for (int it = 0; it < my_tiles && ok && warp_live; ++it, tile_next(p, tc)) {
+            pool_tile(carry, p.c_off);
+            if (p.rider && ok) pool_tile(carry2, p.r_c_off);
         }
     }
 
@@ -850,24 +913,25 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
 
 __global__ void __launch_bounds__(POOLT_THREADS, 1)
 conv_pool_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                 const __grid_constant__ TcParams p)
+                 const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ TcParams p)
 {
-    if (p.npix == 256) conv_pool_body<256>(tmA, tmB, p, (int)blockIdx.x);
-    else conv_pool_body<128>(tmA, tmB, p, (int)blockIdx.x);
+    if (p.npix == 256) conv_pool_body<256>(tmA, tmB, tmB2, p, (int)blockIdx.x);
+    else conv_pool_body<128>(tmA, tmB, tmB2, p, (int)blockIdx.x);
 }
 
-// Two pooled layers over the same input in one launch (see conv_tc_kernel2).
+// Two pooled layers (each possibly with its rider) over the same input in one launch (see conv_tc_kernel2).
 __global__ void __launch_bounds__(POOLT_THREADS, 1)
 conv_pool_kernel2(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
-                  const __grid_constant__ TcParams p0, const __grid_constant__ CUtensorMap tmA1,
-                  const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ TcParams p1)
+                  const __grid_constant__ CUtensorMap tmR0, const __grid_constant__ TcParams p0,
+                  const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
+                  const __grid_constant__ CUtensorMap tmR1, const __grid_constant__ TcParams p1)
 {
     if (p0.npix == 256) {           // (both layers have the same tile size)
-        if ((int)blockIdx.x < p0.grid) conv_pool_body<256>(tmA0, tmB0, p0, (int)blockIdx.x);
-        else conv_pool_body<256>(tmA1, tmB1, p1, (int)blockIdx.x - p0.grid);
+        if ((int)blockIdx.x < p0.grid) conv_pool_body<256>(tmA0, tmB0, tmR0, p0, (int)blockIdx.x);
+        else conv_pool_body<256>(tmA1, tmB1, tmR1, p1, (int)blockIdx.x - p0.grid);
     } else {
-        if ((int)blockIdx.x < p0.grid) conv_pool_body<128>(tmA0, tmB0, p0, (int)blockIdx.x);
-        else conv_pool_body<128>(tmA1, tmB1, p1, (int)blockIdx.x - p0.grid);
+        if ((int)blockIdx.x < p0.grid) conv_pool_body<128>(tmA0, tmB0, tmR0, p0, (int)blockIdx.x);
+        else conv_pool_body<128>(tmA1, tmB1, tmR1, p1, (int)blockIdx.x - p0.grid);
     }
 }
 
@@ -881,12 +945,12 @@ conv_pool_kernel4(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
                   const __grid_constant__ CUtensorMap tmB3, const __grid_constant__ TcParams p3)
 {
     int b = (int)blockIdx.x;                       // (all four layers have 128-pixel tiles)
-    if (b < p0.grid) { conv_pool_body<128>(tmA0, tmB0, p0, b); return; }
+    if (b < p0.grid) { conv_pool_body<128>(tmA0, tmB0, tmB0, p0, b); return; }
     b -= p0.grid;
-    if (b < p1.grid) { conv_pool_body<128>(tmA1, tmB1, p1, b); return; }
+    if (b < p1.grid) { conv_pool_body<128>(tmA1, tmB1, tmB1, p1, b); return; }
     b -= p1.grid;
-    if (b < p2.grid) { conv_pool_body<128>(tmA2, tmB2, p2, b); return; }
-    conv_pool_body<128>(tmA3, tmB3, p3, b - p2.grid);
+    if (b < p2.grid) { conv_pool_body<128>(tmA2, tmB2, tmB2, p2, b); return; }
+    conv_pool_body<128>(tmA3, tmB3, tmB3, p3, b - p2.grid);
 }
 
 // ---------------------------------------------------------------------------- stem repack
@@ -1055,6 +1119,7 @@ void choose_box(int W, int H, int N, int* BW, int* BH, int* BI)
 
 struct Plan {
     CUtensorMap a, b, o;
+    CUtensorMap r;   // the rider's kernels (conv_pool_kernel), else a copy of b
     TcParams p;
     int grid;
     int halves;      // 1 = two light CTAs per SM, 2 = one CTA per SM
@@ -1080,6 +1145,7 @@ int num_sms()
 // of A stages that fit (0 if the candidate does not fit at all).
 thread_local size_t t_smem_limit = SMEM_LIMIT;   // budget the layout search below works against
 thread_local int t_pool_npix = 256;              // conv_pool_kernel: pixels per tile the plan is built for (256 or 128)
+thread_local const ConvDesc* t_rider = nullptr;  // conv_pool_kernel: the 1x1 layer that rides on the plan's layer (see TcParams::rider)
 thread_local int t_force_cw = 0;                 // != 0: only layouts with this store chunk width (see launch_conv_bf16_pair)
 
 int fit_stages(TcParams& p, size_t a_tile, bool want_resident, int cw, int nstg, bool smem_tab, size_t* smem_bytes)
@@ -1142,7 +1208,9 @@ bool pool_layout(TcParams& p, size_t a_tile, size_t* smem_bytes)
 {
     const size_t items = (size_t)p.taps * p.chunks;
     const size_t w_bytes = items * p.b_tile;
-    const size_t fixed = 1024 /*alignment slack*/ + w_bytes + (size_t)TILE_M * 32 + (size_t)p.npix * 32 + CTL_BYTES_NO_TAB;
+    // (a rider adds its kernels -- one tile of Cout rows per reduction chunk -- and its bias rows)
+    const size_t r_bytes = p.rider ? (size_t)p.chunks * p.b_tile + (size_t)TILE_M * 32 : 0;
+    const size_t fixed = 1024 /*alignment slack*/ + w_bytes + r_bytes + (size_t)TILE_M * 32 + (size_t)p.npix * 32 + CTL_BYTES_NO_TAB;
     if (t_smem_limit < fixed + 2 * a_tile) return false;
     size_t stages = (t_smem_limit - fixed) / a_tile;
     if (stages > MAX_STAGES) stages = MAX_STAGES;
@@ -1156,6 +1224,12 @@ bool pool_layout(TcParams& p, size_t a_tile, size_t* smem_bytes)
     p.off_bias = p.off_stg + (unsigned)(stages * a_tile);
     p.off_ones = p.off_bias + (unsigned)TILE_M * 32;
     p.off_ctl = p.off_ones + (unsigned)p.npix * 32;
+    if (p.rider) {
+        p.r_off_bias = p.off_ctl;
+        p.r_off_b = p.r_off_bias + (unsigned)TILE_M * 32;
+        p.off_ctl = p.r_off_b + (unsigned)((size_t)p.chunks * p.b_tile);
+        // (the 128-row read of the rider's last kernel tile ends inside the control block or the slack behind it)
+    }
     *smem_bytes = 1024 + (size_t)p.off_ctl + CTL_BYTES_NO_TAB;
     return true;
 }
@@ -1180,6 +1254,14 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     p.bias_in_k = stem ? 1 : 0;
     p.pool = d.pool ? 1 : 0;
     if (p.pool && (d.OH < 3 || d.OW < 3 || d.Cout % 32 != 0 || d.Cout > TILE_M)) return SQN_ERR_UNSUPPORTED;
+    const ConvDesc* rider = p.pool ? t_rider : nullptr;
+    if (rider) {
+        if (stem || d.Cout != TILE_M || rider->Cout != d.Cout || rider->Cin != d.Cin || rider->K != 1 || rider->S != 1 || rider->pad != 0 ||
+            rider->in != d.in || rider->H != d.H || rider->W != d.W || rider->N != d.N || rider->out != d.out ||
+            rider->out_c_total != d.out_c_total || rider->relu != d.relu || !rider->pool || rider->out_c_offset % 8 != 0)
+            return SQN_ERR_UNSUPPORTED;
+        p.rider = 1;
+    }
     if (stem) {
         p.taps = 7; p.taps_h = 7; p.taps_w = 1; p.pad = 0; p.BKc = 32; p.chunks = 1; p.k_per_tap = 32;
     } else {
@@ -1282,6 +1364,22 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
                     }
     }
     if (plan->smem > t_smem_limit) return SQN_ERR_UNSUPPORTED;
+    if (rider) {
+        // the rider's MMAs read the centre of the patch (the layer's own padding shifted away)
+        const int ksteps = p.BKc / 16;
+        p.r_nmma = p.chunks * ksteps;
+        if (!p.patch || p.r_nmma > 8) return SQN_ERR_UNSUPPORTED;
+        int e = 0;
+        for (int ch = 0; ch < p.chunks; ++ch)
+            for (int k = 0; k < ksteps; ++k, ++e) {
+                const unsigned a_off = (unsigned)ch * p.patch_tile + (unsigned)p.pad * p.tap_h_bytes + (unsigned)p.pad * p.tap_w_bytes;
+                p.r_ptab[e].x = (a_off >> 4) + 2u * k;
+                p.r_ptab[e].y = (((unsigned)ch * p.b_tile) >> 4) + 2u * k;
+            }
+        p.r_b_bytes = (unsigned)p.chunks * p.b_bytes;
+        p.r_c_off = rider->out_c_offset;
+        p.r_bias = rider->bias;
+    }
     p.tiles_w = (OW + p.BW - 1) / p.BW;
     p.tiles_h = (OH + p.BH - 1) / p.BH;
     p.tiles_i = (NI + p.BI - 1) / p.BI;
@@ -1350,6 +1448,13 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
         cuuint32_t box[2] = {(cuuint32_t)p.BKc, (cuuint32_t)p.BN};
         if (!encode(&plan->b, 2, w_ptr, dims, str, box, row_bytes)) return SQN_ERR_CUDA;
     }
+    plan->r = plan->b;
+    if (rider) {
+        cuuint64_t dims[2] = {(cuuint64_t)d.Cin, (cuuint64_t)rider->Cout};
+        cuuint64_t str[1] = {(cuuint64_t)d.Cin * 2};
+        cuuint32_t box[2] = {(cuuint32_t)p.BKc, (cuuint32_t)p.BN};
+        if (!encode(&plan->r, 2, rider->w, dims, str, box, row_bytes)) return SQN_ERR_CUDA;
+    }
     if (!p.pool) {                  // (conv_pool_kernel writes the pooled map with plain stores)
         // extent of the layer dimension stops at the end of this layer's slice so that a
         // partial last tile is clipped instead of spilling into the neighbouring slice
@@ -1405,7 +1510,8 @@ int launch_plan(const Plan& plan, cudaStream_t stream)
         static const cudaError_t attr_rc =
             cudaFuncSetAttribute(conv_pool_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
         rc = attr_rc != cudaSuccess ? attr_rc
-           : launch_chained(conv_pool_kernel, dim3((unsigned)plan.grid), dim3(POOLT_THREADS), plan.smem, stream, plan.a, plan.b, plan.p);
+           : launch_chained(conv_pool_kernel, dim3((unsigned)plan.grid), dim3(POOLT_THREADS), plan.smem, stream, plan.a, plan.b, plan.r,
+                            plan.p);
     }
     else if (plan.split == 1)
         rc = hc == 32 ? launch_variant<1, 32>(plan, stream)
@@ -1441,7 +1547,7 @@ int launch_plan2(const Plan& a, const Plan& b, cudaStream_t stream)
             cudaFuncSetAttribute(conv_pool_kernel2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_LIMIT);
         rc = attr_rc != cudaSuccess ? attr_rc
            : launch_chained(conv_pool_kernel2, dim3((unsigned)(a.grid + b.grid)), dim3(POOLT_THREADS), smem, stream, a.a, a.b,
-                            a.p, b.a, b.b, b.p);
+                            a.r, a.p, b.a, b.b, b.r, b.p);
     } else {
         const int hc = a.p.CW / 2;
         if (a.split != b.split || a.p.CW != b.p.CW) return SQN_ERR_UNSUPPORTED;
@@ -1461,7 +1567,9 @@ int launch_plan2(const Plan& a, const Plan& b, cudaStream_t stream)
 // batch-1 forward would notice.
 struct PlanKey {
     const void *in, *w, *bias, *out, *ws;
+    const void *rw, *rbias;     // the rider's kernels and bias (conv_pool_kernel), else null
     int v[14];
+    int r_c_off;
 };
 
 std::mutex g_plan_mu;
@@ -1475,6 +1583,7 @@ int cached_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_p
     PlanKey k;
     std::memset(&k, 0, sizeof(k));
     k.in = d.in; k.w = d.w; k.bias = d.bias; k.out = d.out; k.ws = ws;
+    if (t_rider) { k.rw = t_rider->w; k.rbias = t_rider->bias; k.r_c_off = t_rider->out_c_offset + 1; }
     const int v[14] = {d.N, d.Cin, d.H, d.W, d.Cout, d.K, d.S, d.pad, d.out_c_offset, d.out_c_total, d.relu | (d.pool << 1) | (d.params_static << 2) | (d.stem_prepacked << 3),
                        (stem ? 1 : 0) | (force_halves << 4) | ((force_cw & 0xffff) << 8), Hp, Wp};
     std::memcpy(k.v, v, sizeof(v));
@@ -1594,6 +1703,26 @@ int launch_conv_bf16_pool4(const ConvDesc* d, cudaStream_t stream)
     if (rc != cudaSuccess) return SQN_ERR_CUDA;
     note_launch();
     return cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
+}
+
+// Pooled 3x3 layers each with a pooled 1x1 layer on the same input riding on its patches (both expands of a fire layer
+// followed by a max-pool; n = 1, or 2 for two slices of the output layers): ONE launch, one pass over the input, the
+// 1x1 layer's few MMAs hidden behind the 3x3 layer's.  SQN_ERR_UNSUPPORTED where the kernels of both do not fit.
+int launch_conv_bf16_pool_riders(const ConvDesc* big, const ConvDesc* rider, int n, cudaStream_t stream)
+{
+    if (n < 1 || n > 2) return SQN_ERR_UNSUPPORTED;
+    Plan pl[2];
+    for (int i = 0; i < n; ++i) {
+        if (!big[i].pool || !rider[i].pool) return SQN_ERR_UNSUPPORTED;
+        t_rider = &rider[i];
+        int rc = cached_plan(big[i], false, big[i].in, big[i].w, 0, 0, nullptr, &pl[i]);
+        if (rc == SQN_OK && n == 2 && i == 1 && pl[1].p.npix != pl[0].p.npix)
+            rc = SQN_ERR_UNSUPPORTED;
+        t_rider = nullptr;
+        if (rc != SQN_OK) return rc == SQN_ERR_CUDA ? rc : SQN_ERR_UNSUPPORTED;
+        if (!pl[i].p.rider) return SQN_ERR_UNSUPPORTED;
+    }
+    return n == 1 ? launch_plan(pl[0], stream) : launch_plan2(pl[0], pl[1], stream);
 }
 
 // Host-only feasibility test of the fused max-pool for a layer (shared-memory budget, shape rules).

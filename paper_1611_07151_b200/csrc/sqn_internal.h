@@ -40,6 +40,8 @@ int launch_conv_bf16(const ConvDesc& d, cudaStream_t stream);
 // kernel variant.
 int launch_conv_bf16_pair(const ConvDesc& small, const ConvDesc& big, cudaStream_t stream);
 int launch_conv_bf16_pool4(const ConvDesc* four, cudaStream_t stream);   // four pooled layers over one input, one launch
+// n (1 or 2) pooled 3x3 layers, each with a pooled 1x1 layer on the same input riding on its patches: one launch
+int launch_conv_bf16_pool_riders(const ConvDesc* big, const ConvDesc* rider, int n, cudaStream_t stream);
 bool conv_bf16_pool_fits(const ConvDesc& d);   // true when the layer can run with its max-pool fused (d.pool = 1)
 int launch_conv_bf16_uncached(const ConvDesc& d, cudaStream_t stream);   // no plan cache, no allocation
 // Stem (7x7/2 on 3 layers): needs scratch for the repacked input and kernels.
@@ -62,6 +64,9 @@ int launch_fire_expands_bf16(const ConvDesc& d1, const ConvDesc& d3, cudaStream_
 // SQN_FUSED_HEAD=0 in the environment turns its use by squeezenet_forward off.
 bool fused_head_enabled();
 int launch_conv_avgpool_bf16(const ConvDesc& d, float* logits, cudaStream_t stream);
+
+// A kernel whose bounded wait runs out (see sqn_selftest_wait_timeout).
+int launch_wait_timeout_selftest(long long limit_cycles, cudaStream_t stream);
 
 // Pooling / head.
 int launch_maxpool3x3s2(const void* in, void* out, int C, int H, int W, int N, int dtype, cudaStream_t stream);

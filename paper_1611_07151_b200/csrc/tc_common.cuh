@@ -11,9 +11,9 @@ namespace sqn {
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // about two seconds
 
 // Bounded mbarrier wait.  Polls back to back at first (hand-offs between the roles take a few
-// hundred cycles), backs off with nanosleep on long waits, and gives up after WAIT_LIMIT_CYCLES:
+// hundred cycles), backs off with nanosleep on long waits, and gives up after `limit` cycles:
 // the CTA then records SQN_ERR_TIMEOUT and every role leaves its loop.
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status)
+__device__ __forceinline__ bool wait_bar_limit(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, long long limit)
 {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
@@ -21,7 +21,7 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
         if (ptx::mbar_try_wait(bar, parity)) return true;
         if ((i & 255u) == 0u) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+            if (clock64() - t0 > limit) {
                 *abort_flag = 1;
                 if (status) atomicExch(status, (int)SQN_ERR_TIMEOUT);
                 return false;
@@ -29,6 +29,10 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
         }
         if (i > 4096u) __nanosleep(128);
     }
+}
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status)
+{
+    return wait_bar_limit(bar, parity, abort_flag, status, WAIT_LIMIT_CYCLES);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)

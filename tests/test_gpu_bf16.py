@@ -492,3 +492,19 @@ def test_fused_global_average_is_refused_where_it_cannot_run():
             B.conv_forward_ex(p, p, p, p, cin, 32, hw, hw, k, 1, k // 2, 1, dtype=dtype, fuse_global_avgpool=True,
                               fuse_maxpool=pool)
         assert e.value.status in (B.SQN_ERR_UNSUPPORTED, B.SQN_ERR_BADARG)
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_leaves_the_library_usable():
+    """Failure detection without a fault: a CTA waits (for about a millisecond) on a barrier nothing arrives on.  The
+    wait runs out, sqn_check reports SQN_ERR_TIMEOUT exactly once, and a convolution launched afterwards -- which
+    needs the tensor memory the timed-out CTA had to give back -- still matches the oracle."""
+    assert B.sqn_check() == B.SQN_OK
+    B.sqn_selftest_wait_timeout(2_000_000)
+    assert B.sqn_check() == B.SQN_ERR_TIMEOUT
+    assert B.sqn_check() == B.SQN_OK
+    with pytest.raises(B.SqnError):
+        B.sqn_selftest_wait_timeout(10)                  # limits outside 1e3 .. 2e9 cycles are refused
+    x, w, b = synth.conv_layer_case(5, 2, 32, 128, 27, 3)
+    exp = ref.conv2d(x, w, b, S=1, pad=1, relu=True)
+    got = G.gpu_conv(x, w, b, 1, 1, True, BF16)
+    assert G.rel_err(got, exp) <= TOL
