@@ -703,8 +703,8 @@ int fire_layout(FireParams& p, int R, int patches, int BKc_in, size_t* smem_byte
 
 // Band heights to try, best first: SQN_FIRE_BAND in the environment (tuning aid, read at every call) names one;
 // else 14 rows for maps of 40 rows and more (four equal bands for 55 rows), 8 for 20 rows and more, else the whole
-// image.  A band is a whole number of expand tiles.
-int band_candidates(int H, int RT, int* out)
+// image; with so few images that this leaves SMs idle, one tile.  A band is a whole number of expand tiles.
+int band_candidates(int H, int RT, int N, int* out)
 {
     int n = 0;
     auto add = [&](int R) {
@@ -718,6 +718,9 @@ int band_candidates(int H, int RT, int* out)
         const int r = std::atoi(v);
         if (r > 0) { add(r); return n; }
     }
+    // few images: bands of one tile, so that as many CTAs as possible have work (the layer is latency-bound then)
+    const int pref = H >= 40 ? 14 : H >= 20 ? 8 : H;
+    if ((long long)N * ((H + pref - 1) / pref) < sm_count()) { add(RT); add(2 * RT); }
     if (H >= 40) { add(14); add(8); }
     else if (H >= 20) { add(8); add(12); add(16); }
     else add(H);
@@ -787,7 +790,7 @@ int build_fire_plan(const ConvDesc* dsq, const ConvDesc& d1, const ConvDesc& d3,
         // two patches with (if there is one) an input ring of 32 KB or more and three slots or more, else one patch
         // under the same condition, else whatever fits
         int cand[8];
-        const int nc = band_candidates(H, p.RT, cand);
+        const int nc = band_candidates(H, p.RT, N, cand);
         for (int pass = 0; pass < 3 && !found; ++pass)
             for (int i = 0; i < nc && !found; ++i)
                 for (int patches = (pass == 1 ? 1 : 2); patches >= (pass == 0 ? 2 : 1) && !found; --patches)
