@@ -536,6 +536,7 @@ def main():
     ap.add_argument("--no-batch1", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="per-layer sweep of every conv shape instead of the network")
     ap.add_argument("--variants", action="store_true", help="per-layer sweep of the bf16 kernel variants at --batch")
+    ap.add_argument("--mma-rate", action="store_true", help="clocks per tcgen05.mma as a function of N (diagnostic)")
     ap.add_argument("--kernel", default=None, help="one layer on its own (bf16): a conv name (conv1, fire6_e3, ...), "
                     "NAME+pool, conv10+avgpool, or a fire layer (fire2 ... fire9)")
     args = ap.parse_args()
@@ -557,6 +558,19 @@ def main():
         return
     if args.kernel:
         run_kernel_case(B, args.kernel, args.batch, args.steps)
+        return
+    if args.mma_rate:
+        rows = []
+        for rb in (32, 128):
+            for n in (16, 32, 64, 96, 128, 192, 256):
+                (issue, done), = B.sqn_selftest_mma_rate(n, rb, 1)
+                rows.append({"row_bytes": rb, "N": n, "issuers": 1, "clocks_per_mma_issue": issue, "clocks_per_mma": done})
+        for n in (16, 64, 128, 256):
+            (i0, d0), (i1, d1) = B.sqn_selftest_mma_rate(n, 128, 2)
+            rows.append({"row_bytes": 128, "N": n, "issuers": 2, "clocks_per_mma": [d0, d1]})
+        assert B.sqn_check() == B.SQN_OK
+        print(json.dumps({"mma_rate": rows, "note": "tcgen05.mma 128 x N x 16, bf16 operands in shared memory, issued back to "
+                          "back by one elected thread per issuer warp on every SM; ideal N/2 clocks"}))
         return
 
     rank, local_rank, world = D.env_world()

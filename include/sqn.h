@@ -295,6 +295,15 @@ int sqn_check(void* stream);
  */
 int sqn_selftest_wait_timeout(long long limit_cycles, void* stream);
 
+/*
+ * Measurement behind the kernels' role layout: on every SM `issuers` (1 or 2) warps each issue `iters` tensor-core
+ * MMAs of 128 x n x 16 (bf16 operands in shared memory, rows of row_bytes = 32 / 64 / 128 in the matching swizzle)
+ * back to back.  out is DEVICE memory for 6 64-bit integers per SM (the SM count is returned in *sm_count_out, a host
+ * pointer, may be NULL): per issuer {clocks until the last MMA was issued, clocks until all had completed, 1 if the
+ * bounded wait for them ended in time}.  n a multiple of 16 in 16 .. 256.  (Diagnostic: the paper has no counterpart.)
+ */
+int sqn_selftest_mma_rate(int n, int row_bytes, int issuers, int iters, void* out, int* sm_count_out, void* stream);
+
 /* Static, human-readable name of a status code. */
 const char* sqn_status_string(int status);
 

@@ -64,6 +64,7 @@ SIGNATURES = {
     "sqn_unpack_nhwc_to_nchw": (_c_int, [_c_vp, _c_vp] + [_c_int] * 5),
     "sqn_check": (_c_int, [_c_vp]),
     "sqn_selftest_wait_timeout": (_c_int, [ctypes.c_longlong, _c_vp]),
+    "sqn_selftest_mma_rate": (_c_int, [_c_int, _c_int, _c_int, _c_int, _c_vp, ctypes.POINTER(_c_int), _c_vp]),
     "sqn_status_string": (ctypes.c_char_p, [_c_int]),
     "sqn_launch_count": (ctypes.c_ulonglong, []),
 }
@@ -264,6 +265,19 @@ def sqn_check(stream=None):
 def sqn_selftest_wait_timeout(limit_cycles, stream=None):
     _check(lib().sqn_selftest_wait_timeout(limit_cycles, current_stream() if stream is None else stream),
            "sqn_selftest_wait_timeout")
+
+
+def sqn_selftest_mma_rate(n, row_bytes=128, issuers=1, iters=2000):
+    """Clocks per tcgen05.mma of 128 x n x 16 (mean over the SMs): (issue loop, until complete) per issuer."""
+    import torch
+    out = torch.zeros(6 * 256, dtype=torch.int64, device="cuda")
+    sms = _c_int(0)
+    _check(lib().sqn_selftest_mma_rate(n, row_bytes, issuers, iters, _p(out), ctypes.byref(sms), current_stream()),
+           "sqn_selftest_mma_rate")
+    torch.cuda.synchronize()
+    o = out[:6 * sms.value].view(sms.value, 2, 3).cpu().numpy()
+    assert (o[:, :issuers, 2] == 1).all()
+    return [(float(o[:, w, 0].mean()) / iters, float(o[:, w, 1].mean()) / iters) for w in range(issuers)]
 
 
 def sqn_status_string(status):

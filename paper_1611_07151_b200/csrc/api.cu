@@ -897,6 +897,21 @@ extern "C" int sqn_selftest_wait_timeout(long long limit_cycles, void* stream)
     return launch_wait_timeout_selftest(limit_cycles, static_cast<cudaStream_t>(stream));
 }
 
+extern "C" int sqn_selftest_mma_rate(int n, int row_bytes, int issuers, int iters, void* out, int* sm_count_out, void* stream)
+{
+    if (n < 16 || n > 256 || n % 16 != 0 || (row_bytes != 32 && row_bytes != 64 && row_bytes != 128) || issuers < 1 || issuers > 2 ||
+        iters < 1 || iters > 1000000 || !out)
+        return SQN_ERR_BADARG;
+    if (reinterpret_cast<uintptr_t>(out) & 7u) return SQN_ERR_ALIGN;
+    if (sm_count_out) {
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return SQN_ERR_CUDA;
+        *sm_count_out = sms;
+    }
+    return launch_mma_rate_selftest(n, row_bytes, issuers, iters, static_cast<long long*>(out), static_cast<cudaStream_t>(stream));
+}
+
 extern "C" const char* sqn_status_string(int status)
 {
     switch (status) {

@@ -300,51 +300,7 @@ int build_head_plan(const ConvDesc& d, float* logits, HeadPlan* plan)
     return SQN_OK;
 }
 
-// One CTA with the roles' skeleton of the kernels above -- barriers, a TMEM allocation, a bounded wait -- whose wait
-// is for an mbarrier that nothing ever arrives on: the wait runs out after `limit` cycles, the CTA records
-// SQN_ERR_TIMEOUT in the status word, frees its TMEM and returns like any other.
-__global__ void __launch_bounds__(64, 1) wait_timeout_kernel(long long limit, int* status)
-{
-    __shared__ unsigned long long bar;
-    __shared__ unsigned tmem_base_s;
-    __shared__ volatile int abort_flag;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (threadIdx.x == 0) {
-        mbar_init(smem_u32(&bar), 1);
-        abort_flag = 0;
-        fence_mbar_init();
-    }
-    if (warp == 1) {
-        tmem_alloc(smem_u32(&tmem_base_s), 32);
-        tmem_relinquish();
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    if (warp == 0) {
-        // the whole warp waits, as the MMA issuers do; every lane sees the time-out
-        const bool ok = __all_sync(0xffffffffu, wait_bar_limit(smem_u32(&bar), 0u, &abort_flag, status, limit));
-        if (ok && lane == 0) atomicExch(status, (int)SQN_ERR_CUDA);        // (cannot happen: nothing arrives)
-    }
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 1) {
-        __syncwarp();
-        tc_fence_after();
-        tmem_dealloc(tmem_base_s, 32);
-    }
-}
-
 }  // namespace
-
-int launch_wait_timeout_selftest(long long limit_cycles, cudaStream_t stream)
-{
-    int* status = device_status_word();
-    if (!status) return SQN_ERR_CUDA;
-    wait_timeout_kernel<<<1, 64, 0, stream>>>(limit_cycles, status);
-    note_launch();
-    return cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
-}
 
 bool fused_head_enabled()
 {

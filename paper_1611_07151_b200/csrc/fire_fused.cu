@@ -704,7 +704,16 @@ int fire_layout(FireParams& p, int R, int patches, int BKc_in, size_t* smem_byte
 // Band heights to try, best first: SQN_FIRE_BAND in the environment (tuning aid, read at every call) names one;
 // else 14 rows for maps of 40 rows and more (four equal bands for 55 rows), 8 for 20 rows and more, else the whole
 // image; with so few images that this leaves SMs idle, one tile.  A band is a whole number of expand tiles.
-int band_candidates(int H, int RT, int N, int* out)
+// Winners of the band-height sweep at batch 256 (`bench.py --kernel fireN` under SQN_FIRE_BAND = 4 ... 28), frozen per
+// layer shape: {H, Cin, s, e1 + e3, rows}.  Shapes not listed take the rule below.
+struct BandChoice { int H, Cin, s, e, R; };
+const BandChoice kBandTable[] = {
+    {55, 96, 16, 128, 14},      // fire2: 66.6 us (8 rows: 66.9, 28 rows: 76.2)
+    {55, 128, 16, 128, 4},      // fire3: 71.7 us (14 rows: 77.8, 28 rows: 91.2)
+    {27, 256, 32, 256, 16},     // fire5: 51.5 us (8 rows: 51.9, 12 rows: 59.7)
+};
+
+int band_candidates(int H, int RT, int N, int Cin, int s, int e, int* out)
 {
     int n = 0;
     auto add = [&](int R) {
@@ -721,6 +730,9 @@ int band_candidates(int H, int RT, int N, int* out)
     // few images: bands of one tile, so that as many CTAs as possible have work (the layer is latency-bound then)
     const int pref = H >= 40 ? 14 : H >= 20 ? 8 : H;
     if ((long long)N * ((H + pref - 1) / pref) < sm_count()) { add(RT); add(2 * RT); }
+    else
+        for (const BandChoice& c : kBandTable)
+            if (c.H == H && c.Cin == Cin && c.s == s && c.e == e) add(c.R);
     if (H >= 40) { add(14); add(8); }
     else if (H >= 20) { add(8); add(12); add(16); }
     else add(H);
@@ -790,7 +802,7 @@ int build_fire_plan(const ConvDesc* dsq, const ConvDesc& d1, const ConvDesc& d3,
         // two patches with (if there is one) an input ring of 32 KB or more and three slots or more, else one patch
         // under the same condition, else whatever fits
         int cand[8];
-        const int nc = band_candidates(H, p.RT, N, cand);
+        const int nc = band_candidates(H, p.RT, N, Cin, s, e1 + e3, cand);
         for (int pass = 0; pass < 3 && !found; ++pass)
             for (int i = 0; i < nc && !found; ++i)
                 for (int patches = (pass == 1 ? 1 : 2); patches >= (pass == 0 ? 2 : 1) && !found; --patches)

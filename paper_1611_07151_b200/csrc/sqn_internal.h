@@ -67,6 +67,8 @@ int launch_conv_avgpool_bf16(const ConvDesc& d, float* logits, cudaStream_t stre
 
 // A kernel whose bounded wait runs out (see sqn_selftest_wait_timeout).
 int launch_wait_timeout_selftest(long long limit_cycles, cudaStream_t stream);
+// tcgen05.mma issue rate (see sqn_selftest_mma_rate); out: 6 values per SM.
+int launch_mma_rate_selftest(int n, int row_bytes, int issuers, int iters, long long* out, cudaStream_t stream);
 
 // Pooling / head.
 int launch_maxpool3x3s2(const void* in, void* out, int C, int H, int W, int N, int dtype, cudaStream_t stream);

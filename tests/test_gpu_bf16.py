@@ -508,3 +508,17 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_leaves_the_library_usable(
     exp = ref.conv2d(x, w, b, S=1, pad=1, relu=True)
     got = G.gpu_conv(x, w, b, 1, 1, True, BF16)
     assert G.rel_err(got, exp) <= TOL
+
+
+def test_mma_rate_selftest_reports_the_tensor_pipe_rate():
+    """sqn_selftest_mma_rate: clocks per tcgen05.mma of 128 x N x 16.  A 256-wide MMA cannot beat N/2 = 128 clocks and
+    a narrow one is not faster in proportion (the fact the two-issuer pipelines of the fused fire kernel rest on)."""
+    (issue256, done256), = B.sqn_selftest_mma_rate(256, 128, 1, 500)
+    (issue16, done16), = B.sqn_selftest_mma_rate(16, 128, 1, 500)
+    assert B.sqn_check() == B.SQN_OK
+    assert 120.0 <= done256 <= 400.0
+    assert 16.0 / 2 <= done16 <= done256
+    both = B.sqn_selftest_mma_rate(64, 32, 2, 500)
+    assert len(both) == 2 and all(d > 0 for _i, d in both)
+    with pytest.raises(B.SqnError):
+        B.sqn_selftest_mma_rate(20)
