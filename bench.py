@@ -290,7 +290,7 @@ def layer_table(B, net, step, steps, batch, es, dtype_tag, peaks, sm_count, sm_m
     ms_step = pe0.elapsed_time(pe1) / steps
     lnames, lms, nfwd = B.squeezenet_profile_read(net)
     B.squeezenet_profile(net, 0)
-    bf16 = dtype_tag == "bf16"
+    bf16 = dtype_tag in ("bf16", "f16")          # (the 16-bit tensor-core paths: same MMA rate)
     pipe = peaks["bf16_tflops"] if bf16 else fp32_ffma_peak_tflops(sm_count, sm_mhz)
     pipe_sus = peaks["bf16_tflops_sustained"] if bf16 else pipe
     work = launch_work(batch, es)
@@ -530,7 +530,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=256, help="images per GPU per step")
-    ap.add_argument("--dtype", default="bf16", choices=["bf16", "f32"])
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "f16", "f32"])
     ap.add_argument("--e2e-steps", type=int, default=0, help="steps of the host-buffer loop (0: min(steps, 50))")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-batch1", action="store_true")
@@ -579,10 +579,11 @@ def main():
     D.init("nccl")
     B.lib()                                     # raises if the CUDA library is missing: no other path exists
 
-    dtype = B.SQN_BF16 if args.dtype == "bf16" else B.SQN_F32
-    es = 2 if dtype == B.SQN_BF16 else 4
+    dtype = {"bf16": B.SQN_BF16, "f16": B.SQN_F16, "f32": B.SQN_F32}[args.dtype]
+    es = 4 if dtype == B.SQN_F32 else 2
     batch = args.batch
-    bf16 = dtype == B.SQN_BF16
+    bf16 = dtype == B.SQN_BF16          # (the stem's offline layouts and the fp32 sub-record go with the bf16 headline run)
+    half = dtype != B.SQN_F32           # a 16-bit tensor-core path
 
     # ---- synthetic workload: U[0,1) images, He-normal kernels, N(0,.01) bias (seed 3 + rank)
     x, params = synth.squeezenet_case(3 + rank, batch)
@@ -592,8 +593,8 @@ def main():
 
     def pinned(a):
         t = torch.from_numpy(a)
-        if bf16:
-            t = t.view(torch.int16).view(torch.bfloat16)
+        if half:
+            t = t.view(torch.int16).view(torch.bfloat16 if bf16 else torch.float16)
         return t.pin_memory()
 
     x_pinned = pinned(B.sqn_pack_nchw_to_nhwc(x, dtype))              # [batch][227][227][3]: what a user's loader holds
@@ -670,15 +671,20 @@ def main():
                 "frac_nominal_8tbs": top["gbs"] / 8000.0}
     else:
         roof = {"bound": top["bound"], "achieved": top["tflops"], "peak": pipe_tf, "unit": "TFLOP/s"}
-        if bf16:
+        if half:
             roof["peak_kind"] = ("burst (a launch lasts %.0f us at full clocks); sustained peak %.1f beside it"
                                  % (top["ms"] * 1e3, pipe_sus))
             roof["frac_sustained"] = top["tflops"] / pipe_sus
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = ncu_traffic_bytes(top["name"], args.dtype, batch)
-    kname = "conv_f32_kernel" if not bf16 else ("conv_pool_kernel" if "+pool" in top["name"] else "conv_tc_kernel")
-    if "_e1+e3" in top["name"]:
-        kname += "2"
+    if not half:
+        kname = "conv_f32_kernel"
+    elif "_fused" in top["name"] or ("_e1+e3" in top["name"] and "+pool" not in top["name"]):
+        kname = "fire_fused_kernel"
+    elif "+avgpool" in top["name"]:
+        kname = "conv_head_kernel"
+    else:
+        kname = "conv_pool_kernel" if "+pool" in top["name"] else "conv_tc_kernel"
     roof["kernel"] = kname + "[%s]" % top["name"]
     roof["peak_source"] = "of " + peaks["source"]
     roof["launch_ms"] = top["ms"]

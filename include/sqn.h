@@ -16,6 +16,13 @@
  *    dtype SQN_BF16: activations and kernels bf16, fp32 accumulation on the
  *    tensor cores, bias/ReLU/pooling arithmetic in fp32, outputs rounded to
  *    bf16 (round to nearest even).  Logits and probabilities are always fp32.
+ *    dtype SQN_F16: the same kernels on IEEE half precision (10 mantissa bits
+ *    instead of bf16's 7, a narrower exponent): a third precision point between
+ *    the exact path and bf16 (the paper, Section IV-B, trades precision for speed
+ *    in two steps, "relaxed" and "imprecise", and accepts a step when the
+ *    predictions do not change).  Wherever this header says SQN_BF16 about shapes
+ *    and alignment, SQN_F16 is accepted under the same rules; values above 65504
+ *    overflow to infinity as in any fp16 computation.
  *  - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is
  *    the legacy default stream).  No entry point synchronises except sqn_check.
  *  - Every argument is validated on the host before anything is launched.  On
@@ -43,7 +50,7 @@ typedef enum {
     SQN_ERR_WORKSPACE = -6     /* workspace missing or too small */
 } sqn_status;
 
-typedef enum { SQN_F32 = 0, SQN_BF16 = 1 } sqn_dtype;
+typedef enum { SQN_F32 = 0, SQN_BF16 = 1, SQN_F16 = 2 } sqn_dtype;
 
 /*
  * Convolution layer (paper Section II; Section III Fig. 2 prose; Eq. 1):
@@ -219,7 +226,7 @@ int squeezenet_destroy(sqn_net* net);
  * Stem operands reordered offline (the paper, Section III-C, reorders the model file once so that no
  * layer repacks data at run time; here the same is done for the one layer whose operands the tensor
  * cores cannot read as they are: conv1, 7x7 / stride 2 on 3 input layers, bf16).
- * squeezenet_set_stem_prepacked(net, 1) (bf16 nets only, else SQN_ERR_UNSUPPORTED) declares that
+ * squeezenet_set_stem_prepacked(net, 1) (SQN_BF16 nets only, else SQN_ERR_UNSUPPORTED) declares that
  *   - squeezenet_forward's input is [batch][Hp][Wp][4] bf16 as written by sqn_pack_stem_input
  *     (Hp, Wp from sqn_stem_packed_extent(227, 227): 228 x 228; the fourth layer of every image pixel
  *     holds 1.0, padding rows and columns are zero), and

@@ -12,6 +12,7 @@ import numpy as np
 
 SQN_F32 = 0
 SQN_BF16 = 1
+SQN_F16 = 2
 
 SQN_OK = 0
 SQN_ERR_BADARG = -1
@@ -291,7 +292,7 @@ def sqn_launch_count():
 # ------------------------------------------------- host layout helpers (numpy in/out)
 
 def _np_dtype(dtype):
-    return np.float32 if dtype == SQN_F32 else np.uint16     # bf16 travels as raw 16-bit words
+    return np.float32 if dtype == SQN_F32 else np.uint16     # bf16 / fp16 travel as raw 16-bit words
 
 
 def sqn_pack_weights_oihw_to_ohwi(src, dtype=SQN_F32):
@@ -327,17 +328,19 @@ def to_device(a, dtype=SQN_F32):
     t = torch.from_numpy(np.ascontiguousarray(a))
     if dtype == SQN_BF16:
         t = t.view(torch.int16).view(torch.bfloat16)
+    elif dtype == SQN_F16:
+        t = t.view(torch.int16).view(torch.float16)
     return t.cuda()
 
 
 def to_host(t, dtype=SQN_F32):
     """CUDA tensor -> host array in the form the unpack helper takes."""
     import torch
-    if dtype == SQN_BF16:
+    if dtype in (SQN_BF16, SQN_F16):
         return t.detach().cpu().view(torch.int16).numpy().view(np.uint16)
     return t.detach().cpu().numpy()
 
 
 def empty_device(shape, dtype=SQN_F32):
     import torch
-    return torch.empty(shape, dtype=torch.float32 if dtype == SQN_F32 else torch.bfloat16, device="cuda")
+    return torch.empty(shape, dtype={SQN_F32: torch.float32, SQN_BF16: torch.bfloat16, SQN_F16: torch.float16}[dtype], device="cuda")

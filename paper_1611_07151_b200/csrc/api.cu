@@ -8,6 +8,8 @@
 #include <string>
 #include <vector>
 
+#include <cuda_fp16.h>
+
 #include "sqn_internal.h"
 
 namespace sqn {
@@ -52,7 +54,9 @@ int* device_status_word()
 
 namespace {
 
-inline size_t esize(int dtype) { return dtype == SQN_BF16 ? 2 : 4; }
+inline bool is16(int dtype) { return dtype == SQN_BF16 || dtype == SQN_F16; }      // the tensor-core paths
+inline bool valid_dtype(int dtype) { return dtype == SQN_F32 || is16(dtype); }
+inline size_t esize(int dtype) { return is16(dtype) ? 2 : 4; }
 inline int out_extent(int H, int K, int S, int pad) { return (H + 2 * pad - K) / S + 1; }
 
 inline uint16_t f32_to_bf16_rne(float f)
@@ -69,6 +73,26 @@ inline float bf16_to_f32(uint16_t h)
     float f;
     std::memcpy(&f, &u, 4);
     return f;
+}
+// fp32 <-> the 16-bit storage type `dtype` (bf16 or fp16), round to nearest even
+inline uint16_t f32_to_16(float f, int dtype)
+{
+    if (dtype == SQN_F16) {
+        const __half h = __float2half_rn(f);
+        uint16_t u;
+        std::memcpy(&u, &h, 2);
+        return u;
+    }
+    return f32_to_bf16_rne(f);
+}
+inline float f16bits_to_f32(uint16_t u, int dtype)
+{
+    if (dtype == SQN_F16) {
+        __half h;
+        std::memcpy(&h, &u, 2);
+        return __half2float(h);
+    }
+    return bf16_to_f32(u);
 }
 
 // Validates one convolution request and fills the descriptor.
@@ -89,15 +113,18 @@ int make_conv_desc(const void* in, const void* w, const void* bias, void* out, i
     d->pool = 0;
     d->params_static = 0;
     d->stem_prepacked = 0;
+    d->f16 = 0;
     return SQN_OK;
 }
 
 inline bool is_stem_shape(const ConvDesc& d) { return d.K == 7 && d.S == 2 && d.pad == 0 && d.Cin == 3; }
 
-int run_conv(const ConvDesc& d, int dtype, void* ws, size_t ws_bytes, cudaStream_t stream)
+int run_conv(const ConvDesc& d_in, int dtype, void* ws, size_t ws_bytes, cudaStream_t stream)
 {
-    if (dtype == SQN_F32) return d.pool ? SQN_ERR_UNSUPPORTED : launch_conv_f32(d, stream);
-    if (dtype != SQN_BF16) return SQN_ERR_BADARG;
+    if (dtype == SQN_F32) return d_in.pool ? SQN_ERR_UNSUPPORTED : launch_conv_f32(d_in, stream);
+    if (!is16(dtype)) return SQN_ERR_BADARG;
+    ConvDesc d = d_in;
+    d.f16 = dtype == SQN_F16 ? 1 : 0;
     if (is_stem_shape(d)) {
         const int rc = launch_stem_pack_bf16(d, ws, ws_bytes, stream);
         return rc != SQN_OK ? rc : launch_stem_conv_bf16(d, ws, ws_bytes, stream);
@@ -109,10 +136,12 @@ int run_conv(const ConvDesc& d, int dtype, void* ws, size_t ws_bytes, cudaStream
 
 // The two expands of a fire layer (same input, disjoint layer slices of one output): one launch where the bf16
 // kernels have a common variant, else two.  *paired tells which.
-int run_expands(const ConvDesc& d1, const ConvDesc& d3, int dtype, cudaStream_t stream, bool* paired)
+int run_expands(const ConvDesc& d1_in, const ConvDesc& d3_in, int dtype, cudaStream_t stream, bool* paired)
 {
     if (paired) *paired = false;
-    if (dtype == SQN_BF16 && fused_fire_enabled() && !d1.pool && !d3.pool) {
+    ConvDesc d1 = d1_in, d3 = d3_in;
+    d1.f16 = d3.f16 = dtype == SQN_F16 ? 1 : 0;
+    if (is16(dtype) && fused_fire_enabled() && !d1.pool && !d3.pool) {
         const int rc = launch_fire_expands_bf16(d1, d3, stream);     // flat-patch kernel, kernels resident per CTA
         if (rc == SQN_OK) {
             if (paired) *paired = true;
@@ -120,7 +149,7 @@ int run_expands(const ConvDesc& d1, const ConvDesc& d3, int dtype, cudaStream_t 
         }
         if (rc != SQN_ERR_UNSUPPORTED) return rc;
     }
-    if (dtype == SQN_BF16 && pair_launch_enabled() && conv_bf16_supported(d1) == SQN_OK && conv_bf16_supported(d3) == SQN_OK) {
+    if (is16(dtype) && pair_launch_enabled() && conv_bf16_supported(d1) == SQN_OK && conv_bf16_supported(d3) == SQN_OK) {
         const int rc = launch_conv_bf16_pair(d1, d3, stream);
         if (rc == SQN_OK) {
             if (paired) *paired = true;
@@ -145,14 +174,15 @@ extern "C" int conv_forward_ex(const void* in, const void* weights, const void* 
     sqn_conv_opts o;
     if (opts) o = *opts;
     else { std::memset(&o, 0, sizeof(o)); o.dtype = SQN_F32; o.relu = 1; }
-    if (o.dtype != SQN_F32 && o.dtype != SQN_BF16) return SQN_ERR_BADARG;
+    if (!valid_dtype(o.dtype)) return SQN_ERR_BADARG;
     ConvDesc d;
     const int rc = make_conv_desc(in, weights, bias, out, numInputLayers, numOutputLayers, H, W, K, S, pad, batch,
                                   o.relu, o.out_c_offset, o.out_c_total, &d);
     if (rc != SQN_OK) return rc;
     if (o.fuse_global_avgpool) {
         if (o.fuse_maxpool || o.out_c_total != 0) return SQN_ERR_BADARG;
-        if (o.dtype != SQN_BF16) return SQN_ERR_UNSUPPORTED;
+        if (!is16(o.dtype)) return SQN_ERR_UNSUPPORTED;
+        d.f16 = o.dtype == SQN_F16 ? 1 : 0;
         return launch_conv_avgpool_bf16(d, static_cast<float*>(out), static_cast<cudaStream_t>(o.stream));
     }
     if (o.fuse_maxpool) {
@@ -173,9 +203,9 @@ extern "C" int conv_workspace_bytes(int Cin, int Cout, int H, int W, int K, int 
 {
     if (!bytes || Cin <= 0 || Cout <= 0 || H <= 0 || W <= 0 || K <= 0 || S <= 0 || pad < 0 || batch <= 0)
         return SQN_ERR_BADARG;
-    if (dtype != SQN_F32 && dtype != SQN_BF16) return SQN_ERR_BADARG;
+    if (!valid_dtype(dtype)) return SQN_ERR_BADARG;
     *bytes = 0;
-    if (dtype == SQN_BF16 && K == 7 && S == 2 && pad == 0 && Cin == 3) *bytes = stem_bf16_workspace_bytes(batch, H, W, Cout);
+    if (is16(dtype) && K == 7 && S == 2 && pad == 0 && Cin == 3) *bytes = stem_bf16_workspace_bytes(batch, H, W, Cout);
     return SQN_OK;
 }
 
@@ -184,7 +214,7 @@ extern "C" int fire_forward(const void* in, const void* w_sq, const void* b_sq, 
                             const void* w_e3, const void* b_e3, void* squeeze_scratch, void* out, int Cin, int s,
                             int e1, int e3, int H, int W, int batch, int dtype, void* stream)
 {
-    if (dtype != SQN_F32 && dtype != SQN_BF16) return SQN_ERR_BADARG;
+    if (!valid_dtype(dtype)) return SQN_ERR_BADARG;
     if (!squeeze_scratch) return SQN_ERR_BADARG;
     if (e1 <= 0 || e3 <= 0) return SQN_ERR_BADARG;
     ConvDesc dsq, d1, d3;
@@ -194,13 +224,14 @@ extern "C" int fire_forward(const void* in, const void* w_sq, const void* b_sq, 
     if (rc != SQN_OK) return rc;
     rc = make_conv_desc(squeeze_scratch, w_e3, b_e3, out, s, e3, H, W, 3, 1, 1, batch, 1, e1, e1 + e3, &d3);
     if (rc != SQN_OK) return rc;
-    if (dtype == SQN_BF16) {
+    dsq.f16 = d1.f16 = d3.f16 = dtype == SQN_F16 ? 1 : 0;
+    if (is16(dtype)) {
         if ((rc = conv_bf16_supported(dsq)) != SQN_OK) return rc;
         if ((rc = conv_bf16_supported(d1)) != SQN_OK) return rc;
         if ((rc = conv_bf16_supported(d3)) != SQN_OK) return rc;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (dtype == SQN_BF16 && fused_fire_enabled()) {
+    if (is16(dtype) && fused_fire_enabled()) {
         rc = launch_fire_fused_bf16(dsq, d1, d3, st);       // one kernel, squeeze_scratch stays untouched
         if (rc != SQN_ERR_UNSUPPORTED) return rc;
     }
@@ -235,7 +266,7 @@ extern "C" int fire_forward_static(const void* in, const void* w_sq, const void*
                                    const void* b_e1, const void* w_e3, const void* b_e3, void* out, int Cin, int s,
                                    int e1, int e3, int H, int W, int batch, int dtype, void* stream)
 {
-    if (dtype != SQN_F32 && dtype != SQN_BF16) return SQN_ERR_BADARG;
+    if (!valid_dtype(dtype)) return SQN_ERR_BADARG;
     if (e1 <= 0 || e3 <= 0 || s <= 0 || H <= 0 || W <= 0 || batch <= 0) return SQN_ERR_BADARG;
     // the squeeze map must fit the built-in scratch
     // (checked factor by factor: the product of four ints can wrap a 64-bit word)
@@ -255,7 +286,8 @@ extern "C" int fire_forward_static(const void* in, const void* w_sq, const void*
     if (rc != SQN_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const ConvDesc* seq[3] = {&dsq, &d1, &d3};
-    if (dtype == SQN_BF16)
+    dsq.f16 = d1.f16 = d3.f16 = dtype == SQN_F16 ? 1 : 0;
+    if (is16(dtype))
         for (const ConvDesc* d : seq)
             if ((rc = conv_bf16_supported(*d)) != SQN_OK) return rc;
     for (const ConvDesc* d : seq) {
@@ -269,7 +301,7 @@ extern "C" int fire_forward_static(const void* in, const void* w_sq, const void*
 extern "C" int maxpool3x3s2_forward(const void* in, void* out, int C, int H, int W, int batch, int dtype, void* stream)
 {
     if (!in || !out || C <= 0 || H < 3 || W < 3 || batch <= 0) return SQN_ERR_BADARG;
-    if (dtype != SQN_F32 && dtype != SQN_BF16) return SQN_ERR_BADARG;
+    if (!valid_dtype(dtype)) return SQN_ERR_BADARG;
     if (!aligned16(in) || !aligned16(out)) return SQN_ERR_ALIGN;
     return launch_maxpool3x3s2(in, out, C, H, W, batch, dtype, static_cast<cudaStream_t>(stream));
 }
@@ -278,7 +310,7 @@ extern "C" int avgpool_softmax_forward(const void* in, void* logits_f32, void* p
                                        int batch, int dtype, void* stream)
 {
     if (!in || !logits_f32 || C <= 0 || H <= 0 || W <= 0 || batch <= 0) return SQN_ERR_BADARG;
-    if (dtype != SQN_F32 && dtype != SQN_BF16) return SQN_ERR_BADARG;
+    if (!valid_dtype(dtype)) return SQN_ERR_BADARG;
     if (C > 8192 || batch > 65535) return SQN_ERR_UNSUPPORTED;       // (the image index is the grid's y dimension)
     // the kernels read the map with 16-byte (bf16) or 8-byte (fp32) loads and the logits as floats
     if (!aligned16(in) || (reinterpret_cast<uintptr_t>(logits_f32) & 3u) || (reinterpret_cast<uintptr_t>(probs_f32) & 3u))
@@ -353,7 +385,7 @@ size_t layout(const sqn_net* net, int batch, std::vector<size_t>* offs, size_t* 
         cur = align_up(cur + (size_t)batch * s.C * s.H * s.W * es, 1024);
     }
     if (stem_off) *stem_off = cur;
-    if (net->dtype == SQN_BF16) cur = align_up(cur + stem_bf16_workspace_bytes(batch, IMG, IMG, 96), 1024);
+    if (is16(net->dtype)) cur = align_up(cur + stem_bf16_workspace_bytes(batch, IMG, IMG, 96), 1024);
     return cur;
 }
 
@@ -393,7 +425,7 @@ extern "C" int squeezenet_create(sqn_net** net, const void* const* weights26, co
                                  int max_batch)
 {
     if (!net || !weights26 || !bias26 || max_batch <= 0) return SQN_ERR_BADARG;
-    if (dtype != SQN_F32 && dtype != SQN_BF16) return SQN_ERR_BADARG;
+    if (!valid_dtype(dtype)) return SQN_ERR_BADARG;
     for (int i = 0; i < 26; ++i) {
         if (!weights26[i] || !bias26[i]) return SQN_ERR_BADARG;
         if (!aligned16(weights26[i]) || (reinterpret_cast<uintptr_t>(bias26[i]) & 3u)) return SQN_ERR_ALIGN;
@@ -421,7 +453,7 @@ extern "C" int squeezenet_destroy(sqn_net* net)
 extern "C" int squeezenet_set_stem_prepacked(sqn_net* net, int on)
 {
     if (!net) return SQN_ERR_BADARG;
-    if (net->dtype != SQN_BF16) return on ? SQN_ERR_UNSUPPORTED : SQN_OK;
+    if (net->dtype != SQN_BF16) return on ? SQN_ERR_UNSUPPORTED : SQN_OK;      // (the pack helpers write bf16)
     net->stem_prepacked = on ? 1 : 0;
     return SQN_OK;
 }
@@ -439,7 +471,7 @@ extern "C" int squeezenet_layer_output(const sqn_net* net, const char* name, voi
     if (!net || !name || !workspace || !ptr || batch <= 0 || batch > net->max_batch) return SQN_ERR_BADARG;
     const int i = find_slot(net, name);
     if (i < 0) return SQN_ERR_BADARG;
-    if (net->dtype == SQN_BF16 && batch >= 16 &&
+    if (is16(net->dtype) && batch >= 16 &&
         (std::strcmp(name, "conv1") == 0 || std::strcmp(name, "fire4") == 0 || std::strcmp(name, "fire8") == 0))
         return SQN_ERR_UNSUPPORTED;   // computed inside the kernels that write pool1 / pool4, never stored
     if (net->fused_head && std::strcmp(name, "conv10") == 0) return SQN_ERR_UNSUPPORTED;     // averaged inside the kernel
@@ -505,10 +537,12 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
     // conv1 7x7/2 + ReLU, then max-pool
     // The fused conv+pool kernels hand a whole strip of 16 output rows to one CTA: worth it once there are
     // enough strips to fill the GPU (8 per image for conv1, 4 for fire4), i.e. from a batch of 16 on.
-    const bool fuse_pools = dt == SQN_BF16 && batch >= 16;
+    const bool fuse_pools = is16(dt) && batch >= 16;
+    const int f16 = dt == SQN_F16 ? 1 : 0;
     // bf16 stem: on operands packed offline (squeezenet_set_stem_prepacked), else after a repack pass
     auto stem_bf16 = [&](ConvDesc& sd) -> int {
         sd.params_static = 1;
+        sd.f16 = f16;
         if (net->stem_prepacked) {
             sd.stem_prepacked = 1;
             return launch_stem_conv_bf16_prepacked(sd, st);
@@ -528,7 +562,7 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
     } else {
         rc = make_conv_desc(in_nhwc, net->w[0], net->b[0], buf("conv1"), 3, 96, IMG, IMG, 7, 2, 0, batch, 1, 0, 0, &d);
         if (rc != SQN_OK) return rc;
-        if (dt == SQN_BF16) {
+        if (is16(dt)) {
             if ((rc = stem_bf16(d)) != SQN_OK) return rc;
         } else {
             if ((rc = launch_conv_f32(d, st)) != SQN_OK) return rc;
@@ -556,9 +590,10 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
         if (rc != SQN_OK) return rc;
         // the net's kernels and bias are not written by anything this forward enqueues
         dsq.params_static = d1.params_static = d3.params_static = 1;
+        dsq.f16 = d1.f16 = d3.f16 = f16;
         const std::string nm(f.name);
         // bf16: squeeze and both expands as one kernel where it applies (no pool behind the layer)
-        if (dt == SQN_BF16 && fused_fire_enabled() && !(f.pool_after && fuse_pools)) {
+        if (is16(dt) && fused_fire_enabled() && !(f.pool_after && fuse_pools)) {
             rc = launch_fire_fused_bf16(dsq, d1, d3, st);
             if (rc == SQN_OK) {
                 net->fused_fire_mask |= 1u << i;
@@ -631,7 +666,7 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
             }
         }
         if (!fused_pool) {
-            if (dt == SQN_BF16 && pair_launch_enabled()) {
+            if (is16(dt) && pair_launch_enabled()) {
                 if ((rc = run_expands(d1, d3, dt, st, nullptr)) != SQN_OK) return rc;
                 mark((nm + "_e1+e3").c_str());
             } else {
@@ -654,8 +689,9 @@ extern "C" int squeezenet_forward(sqn_net* net, const void* in_nhwc, void* logit
     rc = make_conv_desc(cur, net->w[25], net->b[25], buf("conv10"), 512, 1000, 13, 13, 1, 1, 0, batch, 1, 0, 0, &d);
     if (rc != SQN_OK) return rc;
     d.params_static = 1;
+    d.f16 = f16;
     net->fused_head = 0;
-    if (dt == SQN_BF16 && fused_head_enabled()) {
+    if (is16(dt) && fused_head_enabled()) {
         // conv10, ReLU and the global average in one kernel: the 1000 x 13 x 13 map is never stored
         rc = launch_conv_avgpool_bf16(d, static_cast<float*>(logits_f32), st);
         if (rc == SQN_OK) {
@@ -785,7 +821,7 @@ extern "C" const char* squeezenet_profile_name(const sqn_net* net, int i)
 extern "C" int sqn_pack_weights_oihw_to_ohwi(const float* src, void* dst, int O, int I, int K, int dtype)
 {
     if (!src || !dst || O <= 0 || I <= 0 || K <= 0) return SQN_ERR_BADARG;
-    if (dtype != SQN_F32 && dtype != SQN_BF16) return SQN_ERR_BADARG;
+    if (!valid_dtype(dtype)) return SQN_ERR_BADARG;
     for (int o = 0; o < O; ++o)
         for (int i = 0; i < I; ++i)
             for (int kh = 0; kh < K; ++kh)
@@ -793,7 +829,7 @@ extern "C" int sqn_pack_weights_oihw_to_ohwi(const float* src, void* dst, int O,
                     const float v = src[(((size_t)o * I + i) * K + kh) * K + kw];
                     const size_t di = (((size_t)o * K + kh) * K + kw) * I + i;
                     if (dtype == SQN_F32) static_cast<float*>(dst)[di] = v;
-                    else static_cast<uint16_t*>(dst)[di] = f32_to_bf16_rne(v);
+                    else static_cast<uint16_t*>(dst)[di] = f32_to_16(v, dtype);
                 }
     return SQN_OK;
 }
@@ -801,7 +837,7 @@ extern "C" int sqn_pack_weights_oihw_to_ohwi(const float* src, void* dst, int O,
 extern "C" int sqn_pack_nchw_to_nhwc(const float* src, void* dst, int N, int C, int H, int W, int dtype)
 {
     if (!src || !dst || N <= 0 || C <= 0 || H <= 0 || W <= 0) return SQN_ERR_BADARG;
-    if (dtype != SQN_F32 && dtype != SQN_BF16) return SQN_ERR_BADARG;
+    if (!valid_dtype(dtype)) return SQN_ERR_BADARG;
     for (int n = 0; n < N; ++n)
         for (int c = 0; c < C; ++c)
             for (int h = 0; h < H; ++h)
@@ -809,7 +845,7 @@ extern "C" int sqn_pack_nchw_to_nhwc(const float* src, void* dst, int N, int C, 
                     const float v = src[(((size_t)n * C + c) * H + h) * W + w];
                     const size_t di = (((size_t)n * H + h) * W + w) * C + c;
                     if (dtype == SQN_F32) static_cast<float*>(dst)[di] = v;
-                    else static_cast<uint16_t*>(dst)[di] = f32_to_bf16_rne(v);
+                    else static_cast<uint16_t*>(dst)[di] = f32_to_16(v, dtype);
                 }
     return SQN_OK;
 }
@@ -817,14 +853,14 @@ extern "C" int sqn_pack_nchw_to_nhwc(const float* src, void* dst, int N, int C, 
 extern "C" int sqn_unpack_nhwc_to_nchw(const void* src, float* dst, int N, int C, int H, int W, int dtype)
 {
     if (!src || !dst || N <= 0 || C <= 0 || H <= 0 || W <= 0) return SQN_ERR_BADARG;
-    if (dtype != SQN_F32 && dtype != SQN_BF16) return SQN_ERR_BADARG;
+    if (!valid_dtype(dtype)) return SQN_ERR_BADARG;
     for (int n = 0; n < N; ++n)
         for (int h = 0; h < H; ++h)
             for (int w = 0; w < W; ++w)
                 for (int c = 0; c < C; ++c) {
                     const size_t si = (((size_t)n * H + h) * W + w) * C + c;
                     const float v = dtype == SQN_F32 ? static_cast<const float*>(src)[si]
-                                                     : bf16_to_f32(static_cast<const uint16_t*>(src)[si]);
+                                                     : f16bits_to_f32(static_cast<const uint16_t*>(src)[si], dtype);
                     dst[(((size_t)n * C + c) * H + h) * W + w] = v;
                 }
     return SQN_OK;

@@ -106,6 +106,7 @@ struct TcParams {
     int pool_ctot;                   // layers per pixel of the pooled tensor
     __nv_bfloat16* pool_out;
     int npix;                        // conv_pool_kernel: pixels per tile, 256 or 128
+    int f16;                         // 1: the 16-bit type is fp16, 0: bf16
     // conv_pool_kernel: a second layer, 1x1 on the same input with as many output layers, that rides on this layer's
     // patches: after a tile's own MMAs the rider's go into the other accumulator from the same patch, and the epilogue
     // pools both (the 1x1 expand of a fire layer beside the 3x3 expand)
@@ -213,19 +214,12 @@ template <int NUM_THREADS>
 __device__ __forceinline__ void fill_bias_rows(const TcParams& p, unsigned char* base_ptr)
 {
     uint4* rows = reinterpret_cast<uint4*>(base_ptr + p.off_bias);
-    for (int c = threadIdx.x; c < p.n_tiles * p.BN; c += NUM_THREADS) {
-        const float b = c < p.Cout ? __ldg(p.bias + c) : 0.f;
-        const __nv_bfloat16 hi = __float2bfloat16_rn(b);
-        const __nv_bfloat16 lo = __float2bfloat16_rn(b - __bfloat162float(hi));
-        const int u = (c >> 2) & 1;
-        rows[2 * c + u] = make_uint4((uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16), 0u, 0u, 0u);
-        rows[2 * c + (u ^ 1)] = make_uint4(0u, 0u, 0u, 0u);
-    }
+    for (int c = threadIdx.x; c < p.n_tiles * p.BN; c += NUM_THREADS) bias_row(rows, c, c < p.Cout ? __ldg(p.bias + c) : 0.f, p.f16);
 }
 
 // HC: output layers per epilogue piece (8, 16 or 32; a store chunk CW is two pieces), fixed at compile time so
 // that the conversion loop is straight-line code.
-template <int SPLIT, int HC>
+template <int SPLIT, int HC, bool F16>
 __device__ __forceinline__ void conv_tc_body(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmO,
                                              const TcParams& p, const int bid)
 {
@@ -302,7 +296,7 @@ __device__ __forceinline__ void conv_tc_body(const CUtensorMap& tmA, const CUten
         uint4* ones = reinterpret_cast<uint4*>(base_ptr + p.off_ones);
         for (int r = threadIdx.x; r < TILE_M; r += NUM_THREADS) {
             const int u = (r >> 2) & 1;
-            ones[2 * r + u] = make_uint4(0x3f803f80u, 0u, 0u, 0u);
+            ones[2 * r + u] = make_uint4(one_x2(p.f16), 0u, 0u, 0u);
             ones[2 * r + (u ^ 1)] = make_uint4(0u, 0u, 0u, 0u);
         }
     }
@@ -382,7 +376,7 @@ __device__ __forceinline__ void conv_tc_body(const CUtensorMap& tmA, const CUten
         // parameters everything the issuing instruction needs is warp-uniform, which is what lets the
         // MMAs go out back to back (about 55 clocks each for N <= 128, the tensor pipe's own rate; a
         // single diverged thread reading a shared-memory table needs about 100).
-        const uint32_t idesc = make_idesc_bf16(TILE_M, (uint32_t)p.BN);
+        const uint32_t idesc = make_idesc_bf16(TILE_M, (uint32_t)p.BN, (uint32_t)p.f16);
         const int ksteps = p.BKc / 16;
         const uint32_t hiA = p.a_lines ? (uint32_t)(make_kmajor_desc_plain(0, 16u, p.sbo_bytes) >> 32)
                                        : (uint32_t)(make_kmajor_desc(0, row_bytes, p.patch ? p.sbo_bytes : 8u * row_bytes) >> 32);
@@ -526,7 +520,7 @@ __device__ __forceinline__ void conv_tc_body(const CUtensorMap& tmA, const CUten
                     for (int j = 0; j < 16; ++j) {
                         if (2 * j < hc) {
                             const float f0 = __uint_as_float(v[h][2 * j]), f1 = __uint_as_float(v[h][2 * j + 1]);
-                            o[j] = p.relu ? pack_relu_bf16x2(f0, f1) : pack_bf16x2(f0, f1);
+                            o[j] = p.relu ? pack_relu_x2(f0, f1, F16) : pack_x2(f0, f1, F16);
                         }
                     }
 #pragma unroll
@@ -601,7 +595,9 @@ __global__ void __launch_bounds__(threads_for(SPLIT), SPLIT == 1 ? 2 : 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmO, const __grid_constant__ TcParams p)
 {
-    conv_tc_body<SPLIT, HC>(tmA, tmB, tmO, p, (int)blockIdx.x);
+    // (the 16-bit type is a compile-time constant of the body: the epilogue's conversion loop is straight-line code)
+    if (p.f16) conv_tc_body<SPLIT, HC, true>(tmA, tmB, tmO, p, (int)blockIdx.x);
+    else conv_tc_body<SPLIT, HC, false>(tmA, tmB, tmO, p, (int)blockIdx.x);
 }
 
 template <int SPLIT, int HC>
@@ -611,8 +607,13 @@ conv_tc_kernel2(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
                 const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1,
                 const __grid_constant__ CUtensorMap tmO1, const __grid_constant__ TcParams p1)
 {
-    if ((int)blockIdx.x < p0.grid) conv_tc_body<SPLIT, HC>(tmA0, tmB0, tmO0, p0, (int)blockIdx.x);
-    else conv_tc_body<SPLIT, HC>(tmA1, tmB1, tmO1, p1, (int)blockIdx.x - p0.grid);
+    if (p0.f16) {
+        if ((int)blockIdx.x < p0.grid) conv_tc_body<SPLIT, HC, true>(tmA0, tmB0, tmO0, p0, (int)blockIdx.x);
+        else conv_tc_body<SPLIT, HC, true>(tmA1, tmB1, tmO1, p1, (int)blockIdx.x - p0.grid);
+    } else {
+        if ((int)blockIdx.x < p0.grid) conv_tc_body<SPLIT, HC, false>(tmA0, tmB0, tmO0, p0, (int)blockIdx.x);
+        else conv_tc_body<SPLIT, HC, false>(tmA1, tmB1, tmO1, p1, (int)blockIdx.x - p0.grid);
+    }
 }
 
 // ------------------------------------------------------------------- convolution + 3x3/2 max-pool
@@ -636,7 +637,7 @@ __host__ __device__ constexpr int poolt_prows(int npix) { return (npix / 8 - 2) 
 
 // NPIX = 256 (8 x 32 pixels per tile, 15 pooled rows per strip) where the layer's kernels leave room for the larger
 // patches, else 128 (8 x 16 pixels, 7 pooled rows).
-template <int NPIX>
+template <int NPIX, bool F16>
 __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB2,
                                                const TcParams& p, const int bid)
 {
@@ -675,14 +676,7 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
         fill_bias_rows<POOLT_THREADS>(p, base_ptr);
         if (p.rider) {
             uint4* rows = reinterpret_cast<uint4*>(base_ptr + p.r_off_bias);
-            for (int c = threadIdx.x; c < TILE_M; c += POOLT_THREADS) {
-                const float b = c < p.Cout ? __ldg(p.r_bias + c) : 0.f;
-                const __nv_bfloat16 hi = __float2bfloat16_rn(b);
-                const __nv_bfloat16 lo = __float2bfloat16_rn(b - __bfloat162float(hi));
-                const int u = (c >> 2) & 1;
-                rows[2 * c + u] = make_uint4((uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16), 0u, 0u, 0u);
-                rows[2 * c + (u ^ 1)] = make_uint4(0u, 0u, 0u, 0u);
-            }
+            for (int c = threadIdx.x; c < TILE_M; c += POOLT_THREADS) bias_row(rows, c, c < p.Cout ? __ldg(p.r_bias + c) : 0.f, p.f16);
         }
     };
 
@@ -715,7 +709,7 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
         uint4* ones = reinterpret_cast<uint4*>(base_ptr + p.off_ones);
         for (int r = threadIdx.x; r < NPIX; r += POOLT_THREADS) {
             const int u = (r >> 2) & 1;
-            ones[2 * r + u] = make_uint4(0x3f803f80u, 0u, 0u, 0u);
+            ones[2 * r + u] = make_uint4(one_x2(p.f16), 0u, 0u, 0u);
             ones[2 * r + (u ^ 1)] = make_uint4(0u, 0u, 0u, 0u);
         }
     }
@@ -767,7 +761,7 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        const uint32_t idesc = make_idesc_bf16(TILE_M, NPIX);
+        const uint32_t idesc = make_idesc_bf16(TILE_M, NPIX, (uint32_t)p.f16);
         const uint32_t hiX = p.a_lines ? (uint32_t)(make_kmajor_desc_plain(0, 16u, p.sbo_bytes) >> 32)
                                        : (uint32_t)(make_kmajor_desc(0, row_bytes, p.sbo_bytes) >> 32);
         const uint32_t hiW = (uint32_t)(make_kmajor_desc(0, row_bytes, 8u * row_bytes) >> 32);
@@ -887,10 +881,10 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
                     cr[r][1] = c[7];
                     if (live && ph0 + r < p.PH_out) {
                         unsigned short* dst = dst0 + r * row_stride;
-                        if (first) dst[0] = to_bf16_bits(o0, p.relu);
-                        if (last1) dst[p.pool_ctot] = to_bf16_bits(o1, p.relu);
-                        if (last2) dst[2 * p.pool_ctot] = to_bf16_bits(o2, p.relu);
-                        if (last3) dst[3 * p.pool_ctot] = to_bf16_bits(o3, p.relu);
+                        if (first) dst[0] = to_16_bits(o0, p.relu, F16);
+                        if (last1) dst[p.pool_ctot] = to_16_bits(o1, p.relu, F16);
+                        if (last2) dst[2 * p.pool_ctot] = to_16_bits(o2, p.relu, F16);
+                        if (last3) dst[3 * p.pool_ctot] = to_16_bits(o3, p.relu, F16);
                     }
                 }
             }
@@ -911,12 +905,21 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
     }
 }
 
+// (tile size and 16-bit type are compile-time constants of the body)
+template <int NPIX>
+__device__ __forceinline__ void pool_body(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB2, const TcParams& p,
+                                          const int bid)
+{
+    if (p.f16) conv_pool_body<NPIX, true>(tmA, tmB, tmB2, p, bid);
+    else conv_pool_body<NPIX, false>(tmA, tmB, tmB2, p, bid);
+}
+
 __global__ void __launch_bounds__(POOLT_THREADS, 1)
 conv_pool_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ TcParams p)
 {
-    if (p.npix == 256) conv_pool_body<256>(tmA, tmB, tmB2, p, (int)blockIdx.x);
-    else conv_pool_body<128>(tmA, tmB, tmB2, p, (int)blockIdx.x);
+    if (p.npix == 256) pool_body<256>(tmA, tmB, tmB2, p, (int)blockIdx.x);
+    else pool_body<128>(tmA, tmB, tmB2, p, (int)blockIdx.x);
 }
 
 // Two pooled layers (each possibly with its rider) over the same input in one launch (see conv_tc_kernel2).
@@ -927,11 +930,11 @@ conv_pool_kernel2(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
                   const __grid_constant__ CUtensorMap tmR1, const __grid_constant__ TcParams p1)
 {
     if (p0.npix == 256) {           // (both layers have the same tile size)
-        if ((int)blockIdx.x < p0.grid) conv_pool_body<256>(tmA0, tmB0, tmR0, p0, (int)blockIdx.x);
-        else conv_pool_body<256>(tmA1, tmB1, tmR1, p1, (int)blockIdx.x - p0.grid);
+        if ((int)blockIdx.x < p0.grid) pool_body<256>(tmA0, tmB0, tmR0, p0, (int)blockIdx.x);
+        else pool_body<256>(tmA1, tmB1, tmR1, p1, (int)blockIdx.x - p0.grid);
     } else {
-        if ((int)blockIdx.x < p0.grid) conv_pool_body<128>(tmA0, tmB0, tmR0, p0, (int)blockIdx.x);
-        else conv_pool_body<128>(tmA1, tmB1, tmR1, p1, (int)blockIdx.x - p0.grid);
+        if ((int)blockIdx.x < p0.grid) pool_body<128>(tmA0, tmB0, tmR0, p0, (int)blockIdx.x);
+        else pool_body<128>(tmA1, tmB1, tmR1, p1, (int)blockIdx.x - p0.grid);
     }
 }
 
@@ -945,12 +948,12 @@ conv_pool_kernel4(const __grid_constant__ CUtensorMap tmA0, const __grid_constan
                   const __grid_constant__ CUtensorMap tmB3, const __grid_constant__ TcParams p3)
 {
     int b = (int)blockIdx.x;                       // (all four layers have 128-pixel tiles)
-    if (b < p0.grid) { conv_pool_body<128>(tmA0, tmB0, tmB0, p0, b); return; }
+    if (b < p0.grid) { pool_body<128>(tmA0, tmB0, tmB0, p0, b); return; }
     b -= p0.grid;
-    if (b < p1.grid) { conv_pool_body<128>(tmA1, tmB1, tmB1, p1, b); return; }
+    if (b < p1.grid) { pool_body<128>(tmA1, tmB1, tmB1, p1, b); return; }
     b -= p1.grid;
-    if (b < p2.grid) { conv_pool_body<128>(tmA2, tmB2, tmB2, p2, b); return; }
-    conv_pool_body<128>(tmA3, tmB3, tmB3, p3, b - p2.grid);
+    if (b < p2.grid) { pool_body<128>(tmA2, tmB2, tmB2, p2, b); return; }
+    pool_body<128>(tmA3, tmB3, tmB3, p3, b - p2.grid);
 }
 
 // ---------------------------------------------------------------------------- stem repack
@@ -967,7 +970,7 @@ constexpr int PACK_ROWS = 16;
 __global__ void __launch_bounds__(256) stem_pack(const __nv_bfloat16* __restrict__ in, uint4* __restrict__ out, int N, int H, int W,
                                                  int Hp, int Wp, long long in_elems, int pitch, int row_blocks,
                                                  const unsigned short* __restrict__ w, unsigned short* __restrict__ w_out, int Cout,
-                                                 const float* __restrict__ bias)
+                                                 const float* __restrict__ bias, int f16)
 {
     chain_release();
     chain_wait();
@@ -980,9 +983,8 @@ __global__ void __launch_bounds__(256) stem_pack(const __nv_bfloat16* __restrict
         const int m = idx / 224;
         unsigned short v = (px < 7 && c < 3) ? w[((m * 7 + kh) * 7 + px) * 3 + c] : (unsigned short)0;
         if (c == 3 && kh == 0 && px < 2) {          // fourth layer of the first two pixels of the first kernel row: bias hi, lo
-            const float b = __ldg(bias + m);
-            const __nv_bfloat16 hi = __float2bfloat16_rn(b);
-            v = px == 0 ? __bfloat16_as_ushort(hi) : __bfloat16_as_ushort(__float2bfloat16_rn(b - __bfloat162float(hi)));
+            const uint32_t hl = bias_hi_lo(__ldg(bias + m), f16);
+            v = px == 0 ? (unsigned short)(hl & 0xffffu) : (unsigned short)(hl >> 16);
         }
         w_out[idx] = v;
         return;
@@ -1053,7 +1055,7 @@ __global__ void __launch_bounds__(256) stem_pack(const __nv_bfloat16* __restrict
             // fourth layer of a pixel of the image: 1.0 (it meets the bias in the repacked kernels), else 0
             unsigned one[4];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) one[q] = (y < H && x0 + q < W) ? 0x3f800000u : 0u;
+            for (int q = 0; q < 4; ++q) one[q] = (y < H && x0 + q < W) ? (one_x2(f16) & 0xffff0000u) : 0u;
             dst[0] = make_uint4((unsigned)e[0] | ((unsigned)e[1] << 16), (unsigned)e[2] | one[0],
                                 (unsigned)e[3] | ((unsigned)e[4] << 16), (unsigned)e[5] | one[1]);
             if (x0 + 2 < Wp)
@@ -1089,13 +1091,15 @@ CUtensorMapSwizzle swizzle_for_bytes(unsigned row_bytes)
          : row_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE;
 }
 
+thread_local int t_f16 = 0;      // element type of the tensor maps being encoded: 0 bf16, 1 fp16
+
 bool encode(CUtensorMap* m, int rank, const void* ptr, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
             const cuuint32_t* box, unsigned inner_bytes)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint32_t ones[5] = {1, 1, 1, 1, 1};
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(ptr), dims, strides_bytes, box,
+    return fn(m, t_f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(ptr), dims, strides_bytes, box,
               ones, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for_bytes(inner_bytes), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -1244,6 +1248,8 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
     plan->halves = halves;
     plan->split = halves;
     t_smem_limit = halves == 1 ? SMEM_LIMIT_2CTA : SMEM_LIMIT;
+    p.f16 = d.f16;
+    t_f16 = d.f16;
     p.Cout = d.Cout;
     p.c_off = d.out_c_offset;
     p.relu = d.relu;
@@ -1584,7 +1590,7 @@ int cached_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_p
     std::memset(&k, 0, sizeof(k));
     k.in = d.in; k.w = d.w; k.bias = d.bias; k.out = d.out; k.ws = ws;
     if (t_rider) { k.rw = t_rider->w; k.rbias = t_rider->bias; k.r_c_off = t_rider->out_c_offset + 1; }
-    const int v[14] = {d.N, d.Cin, d.H, d.W, d.Cout, d.K, d.S, d.pad, d.out_c_offset, d.out_c_total, d.relu | (d.pool << 1) | (d.params_static << 2) | (d.stem_prepacked << 3),
+    const int v[14] = {d.N, d.Cin, d.H, d.W, d.Cout, d.K, d.S, d.pad, d.out_c_offset, d.out_c_total, d.relu | (d.pool << 1) | (d.params_static << 2) | (d.stem_prepacked << 3) | (d.f16 << 4),
                        (stem ? 1 : 0) | (force_halves << 4) | ((force_cw & 0xffff) << 8), Hp, Wp};
     std::memcpy(k.v, v, sizeof(v));
     int dev = 0;
@@ -1621,9 +1627,10 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 }  // namespace
 
-bool tmap_encode_bf16(CUtensorMap* m, int rank, const void* ptr, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
-                      const cuuint32_t* box, unsigned inner_bytes)
+bool tmap_encode_16(CUtensorMap* m, int rank, const void* ptr, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
+                    const cuuint32_t* box, unsigned inner_bytes, int f16)
 {
+    t_f16 = f16;
     return encode(m, rank, ptr, dims, strides_bytes, box, inner_bytes);
 }
 int sm_count() { return num_sms(); }
@@ -1775,7 +1782,7 @@ int launch_stem_pack_bf16(const ConvDesc& d, void* workspace, size_t workspace_b
     const cudaError_t e = launch_chained(stem_pack, dim3((unsigned)(row_blocks + w_blocks)), dim3(256),
                                          (size_t)PACK_ROWS * pitch * 2, stream, static_cast<const __nv_bfloat16*>(d.in), pin,
                                          d.N, d.H, d.W, Hp, Wp, (long long)d.N * d.H * d.W * 3, pitch, row_blocks,
-                                         static_cast<const unsigned short*>(d.w), pw, d.Cout, d.bias);
+                                         static_cast<const unsigned short*>(d.w), pw, d.Cout, d.bias, d.f16);
     note_launch(1);
     return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;
 }

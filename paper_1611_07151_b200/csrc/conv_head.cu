@@ -42,6 +42,7 @@ struct HeadParams {
     int groups;                      // CTAs per layer tile; group g takes images g, g + groups, ...
     int stages;
     int relu;
+    int f16;                         // 1: fp16 operands, 0: bf16
     int b_early;
     unsigned x_tile, x_bytes;        // ring slot size / bytes one pixel box delivers
     unsigned off_x, off_ctl;         // (the kernels start at offset 0: `chunks` tiles of 128 rows x 128 bytes)
@@ -140,7 +141,7 @@ conv_head_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        const uint32_t idesc = make_idesc_bf16(128, (uint32_t)p.NP);
+        const uint32_t idesc = make_idesc_bf16(128, (uint32_t)p.NP, (uint32_t)p.f16);
         const uint32_t hi = (uint32_t)(make_kmajor_desc(0, 128u, 1024u) >> 32);
         const uint32_t smW16 = smW >> 4, smX16 = smX >> 4, x_tile16 = p.x_tile >> 4;
         bool ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->w_full), 0u, abort_flag, p.status));
@@ -260,6 +261,7 @@ int build_head_plan(const ConvDesc& d, float* logits, HeadPlan* plan)
     p.chunks = d.Cin / 64;
     p.n_tiles = (d.Cout + 127) / 128;
     p.relu = d.relu;
+    p.f16 = d.f16;
     p.b_early = d.params_static ? 1 : 0;
     p.bias = d.bias;
     p.logits = logits;
@@ -289,13 +291,13 @@ int build_head_plan(const ConvDesc& d, float* logits, HeadPlan* plan)
         cuuint64_t dims[2] = {(cuuint64_t)d.Cin, (cuuint64_t)d.N * HW};
         cuuint64_t str[1] = {(cuuint64_t)d.Cin * 2};
         cuuint32_t box[2] = {64, (cuuint32_t)p.NP};
-        if (!tmap_encode_bf16(&plan->x, 2, d.in, dims, str, box, 128)) return SQN_ERR_CUDA;
+        if (!tmap_encode_16(&plan->x, 2, d.in, dims, str, box, 128, p.f16)) return SQN_ERR_CUDA;
     }
     {
         cuuint64_t dims[2] = {(cuuint64_t)d.Cin, (cuuint64_t)d.Cout};
         cuuint64_t str[1] = {(cuuint64_t)d.Cin * 2};
         cuuint32_t box[2] = {64, 128};
-        if (!tmap_encode_bf16(&plan->w, 2, d.w, dims, str, box, 128)) return SQN_ERR_CUDA;
+        if (!tmap_encode_16(&plan->w, 2, d.w, dims, str, box, 128, p.f16)) return SQN_ERR_CUDA;
     }
     return SQN_OK;
 }
@@ -317,7 +319,7 @@ int launch_conv_avgpool_bf16(const ConvDesc& d, float* logits, cudaStream_t stre
     k.in = d.in; k.w = d.w; k.bias = d.bias; k.out = logits;
     int dev = 0;
     cudaGetDevice(&dev);
-    const int v[8] = {d.N, d.Cin, d.H, d.W, d.Cout, d.relu | (d.params_static << 1), dev, d.K | (d.S << 8) | (d.pad << 16)};
+    const int v[8] = {d.N, d.Cin, d.H, d.W, d.Cout, d.relu | (d.params_static << 1) | (d.f16 << 2), dev, d.K | (d.S << 8) | (d.pad << 16)};
     std::memcpy(k.v, v, sizeof(v));
     const std::string key(reinterpret_cast<const char*>(&k), sizeof(k));
     HeadPlan plan;

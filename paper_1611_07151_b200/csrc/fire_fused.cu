@@ -66,6 +66,7 @@ struct FireParams {
     int chunks_s, BKs, ksteps_s;     // expand reduction per tap: chunks_s chunks of BKs layers (s = chunks_s * BKs), BKs / 16 MMAs each
     int CS, e3p, e1p;                // the output layers are split over CS CTAs ("parts") of e3p + e1p layers each
     int CW;                          // output layers per store chunk (32 or 64)
+    int f16;                         // 1: the 16-bit type is fp16, 0: bf16
     int stages, nstg;
     int s_issuers;                   // squeeze issuer warps at work: 2 where the input ring holds two tiles' chunks, else 1
     int two_patches;
@@ -136,33 +137,25 @@ __device__ __forceinline__ uint32_t swz(uint32_t r, uint32_t rb)
     return rb == 128 ? (r & 7u) : rb == 64 ? ((r >> 1) & 3u) : ((r >> 2) & 1u);
 }
 
-// Bias rows of the bias MMA: one 32-byte row {hi, lo, 0, ...} per output layer, hi + lo = the fp32 bias.
-__device__ __forceinline__ void bias_row(uint4* rows, int c, float b)
-{
-    const __nv_bfloat16 hi = __float2bfloat16_rn(b);
-    const __nv_bfloat16 lo = __float2bfloat16_rn(b - __bfloat162float(hi));
-    const int u = (c >> 2) & 1;
-    rows[2 * c + u] = make_uint4((uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16), 0u, 0u, 0u);
-    rows[2 * c + (u ^ 1)] = make_uint4(0u, 0u, 0u, 0u);
-}
-
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
 {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
 // 16 accumulator columns -> ReLU, bf16 -> two 16-byte units at unit index u0, u0 + 1 of a swizzled row
+template <bool F16>
 __device__ __forceinline__ void store16(const uint32_t* v, uint32_t rbase, uint32_t u0, uint32_t sw)
 {
 #pragma unroll
     for (int u = 0; u < 2; ++u) {
         uint32_t o[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) o[j] = pack_relu_bf16x2(__uint_as_float(v[8 * u + 2 * j]), __uint_as_float(v[8 * u + 2 * j + 1]));
+        for (int j = 0; j < 4; ++j) o[j] = pack_relu_x2(__uint_as_float(v[8 * u + 2 * j]), __uint_as_float(v[8 * u + 2 * j + 1]), F16);
         st_shared_v4(rbase + (((u0 + (uint32_t)u) ^ sw) << 4), o[0], o[1], o[2], o[3]);
     }
 }
 
+template <bool F16>
 __global__ void __launch_bounds__(FF_THREADS, 1)
 fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmWsq,
                   const __grid_constant__ CUtensorMap tmW3, const __grid_constant__ CUtensorMap tmW1,
@@ -197,11 +190,11 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     auto fill_bias = [&]() {
         if (!p.src_tma) {
             uint4* rs = reinterpret_cast<uint4*>(base_ptr + p.off_bias_s);
-            for (int c = threadIdx.x; c < p.s; c += FF_THREADS) bias_row(rs, c, __ldg(p.bias_sq + c));
+            for (int c = threadIdx.x; c < p.s; c += FF_THREADS) bias_row(rs, c, __ldg(p.bias_sq + c), p.f16);
         }
         uint4* re = reinterpret_cast<uint4*>(base_ptr + p.off_bias_e);
         for (int c = threadIdx.x; c < p.e3p + p.e1p; c += FF_THREADS)
-            bias_row(re, c, c < p.e3p ? __ldg(p.bias_e3 + part * p.e3p + c) : __ldg(p.bias_e1 + part * p.e1p + c - p.e3p));
+            bias_row(re, c, c < p.e3p ? __ldg(p.bias_e3 + part * p.e3p + c) : __ldg(p.bias_e1 + part * p.e1p + c - p.e3p), p.f16);
     };
 
     // Up to chain_wait() this block touches only its own shared memory, TMEM, the kernel parameters and, when
@@ -248,7 +241,7 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         uint4* ones = reinterpret_cast<uint4*>(base_ptr + p.off_ones);
         for (int r = threadIdx.x; r < 128; r += FF_THREADS) {
             const int u = (r >> 2) & 1;
-            ones[2 * r + u] = make_uint4(0x3f803f80u, 0u, 0u, 0u);
+            ones[2 * r + u] = make_uint4(one_x2(p.f16), 0u, 0u, 0u);
             ones[2 * r + (u ^ 1)] = make_uint4(0u, 0u, 0u, 0u);
         }
     }
@@ -330,7 +323,7 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         // cost the tensor core, so two warps take the squeeze tiles in turn (issuer w fills accumulator w).  Each
         // warp walks the loops converged; one elected lane issues the MMAs and their commits.
         const int w = warp - FF_W_SMMA;
-        const uint32_t idesc_s = make_idesc_bf16(128, (uint32_t)p.s);
+        const uint32_t idesc_s = make_idesc_bf16(128, (uint32_t)p.s, (uint32_t)p.f16);
         const uint32_t hi_in = (uint32_t)(make_kmajor_desc(0, p.rb_in, 8u * p.rb_in) >> 32);
         const uint64_t ones_desc = make_kmajor_desc(base + p.off_ones, 32u, 256u);
         const uint64_t bias_s_desc = make_kmajor_desc(base + p.off_bias_s, 32u, 256u);
@@ -500,11 +493,11 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
                     const uint32_t pr = (uint32_t)((yy + b.ylo - b.y0 + 1) * p.P + xx + 1);
                     const uint32_t rbase = patch + pr * p.rb_s;
                     const uint32_t sw = swz(pr, p.rb_s);
-                    store16(&v[0], rbase, 0u, sw);
-                    if (p.s >= 32) store16(&v[16], rbase, 2u, sw);
+                    store16<F16>(&v[0], rbase, 0u, sw);
+                    if (p.s >= 32) store16<F16>(&v[16], rbase, 2u, sw);
                     if (p.s == 64) {
-                        store16(&v[32], rbase, 4u, sw);
-                        store16(&v[48], rbase, 6u, sw);
+                        store16<F16>(&v[32], rbase, 4u, sw);
+                        store16<F16>(&v[48], rbase, 6u, sw);
                     }
                 }
             }
@@ -564,11 +557,11 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
                             if (!ok) break;
                             if (e_valid) {
                                 const uint32_t rbase = smStg + (uint32_t)sb * p.stg_slot + stg_off;
-                                store16(&v[0], rbase, 0u, sw_e);
-                                store16(&v[16], rbase, 2u, sw_e);
+                                store16<F16>(&v[0], rbase, 0u, sw_e);
+                                store16<F16>(&v[16], rbase, 2u, sw_e);
                                 if (p.CW == 64) {
-                                    store16(&v[32], rbase, 4u, sw_e);
-                                    store16(&v[48], rbase, 6u, sw_e);
+                                    store16<F16>(&v[32], rbase, 4u, sw_e);
+                                    store16<F16>(&v[48], rbase, 6u, sw_e);
                                 }
                             }
                             fence_proxy_async_smem();             // staging rows visible to the TMA unit
@@ -756,6 +749,8 @@ int build_fire_plan(const ConvDesc* dsq, const ConvDesc& d1, const ConvDesc& d3,
         d1.out_c_total % 8 != 0)
         return SQN_ERR_UNSUPPORTED;
     if ((long long)N * H * W > 0x7fffffffLL / 2) return SQN_ERR_UNSUPPORTED;
+    if ((dsq && dsq->f16 != d1.f16) || d1.f16 != d3.f16) return SQN_ERR_UNSUPPORTED;
+    p.f16 = d1.f16;
     p.H = H; p.W = W; p.P = W + 2; p.N = N; p.Cin = Cin; p.s = s; p.e1 = e1; p.e3 = e3;
     p.RT = 128 / p.P;
     p.BKs = s % 64 == 0 ? 64 : s % 32 == 0 ? 32 : 16;
@@ -826,7 +821,7 @@ int build_fire_plan(const ConvDesc* dsq, const ConvDesc& d1, const ConvDesc& d3,
                 for (int k = 0; k < p.ksteps_s; ++k, ++e) {
                     p.etab[e].x = (((unsigned)ch * p.patch_chunk + (unsigned)(kh * p.P + kw) * p.rb_s) >> 4) + 2u * k;
                     p.etab[e].y = (b_off[ch] >> 4) + 2u * k;
-                    p.eidesc[e] = make_idesc_bf16(128, (unsigned)ncols);
+                    p.eidesc[e] = make_idesc_bf16(128, (unsigned)ncols, (unsigned)p.f16);
                 }
         };
         if (combined) {
@@ -839,19 +834,19 @@ int build_fire_plan(const ConvDesc* dsq, const ConvDesc& d1, const ConvDesc& d3,
                 if (tap != 4) tap_mmas(tap, p.off_w3[tap], p.e3p);
             p.job_en[0] = e;
             p.job_chunk0[0] = 0; p.job_nchunks[0] = (p.e1p + p.e3p) / p.CW;
-            p.job_bias16[0] = 0; p.job_idesc[0] = make_idesc_bf16(128, (unsigned)(p.e3p + p.e1p));
+            p.job_bias16[0] = 0; p.job_idesc[0] = make_idesc_bf16(128, (unsigned)(p.e3p + p.e1p), (unsigned)p.f16);
         } else {
             p.job_e0[0] = 0;
             for (int tap = 0; tap < 9; ++tap) tap_mmas(tap, p.off_w3[tap], p.e3p);
             p.job_en[0] = e;
             p.job_chunk0[0] = 0; p.job_nchunks[0] = p.e3p / p.CW;
-            p.job_bias16[0] = 0; p.job_idesc[0] = make_idesc_bf16(128, (unsigned)p.e3p);
+            p.job_bias16[0] = 0; p.job_idesc[0] = make_idesc_bf16(128, (unsigned)p.e3p, (unsigned)p.f16);
             p.job_e0[1] = e;
             tap_mmas(4, p.off_w1c, p.e1p);              // the 1x1 expand reads the centre pixel
             p.job_en[1] = e;
             p.job_chunk0[1] = p.e3p / p.CW; p.job_nchunks[1] = p.e1p / p.CW;
             p.job_bias16[1] = (unsigned)p.e3p * 2u;     // bias rows are 32 bytes each, the 3x3 expand's come first
-            p.job_idesc[1] = make_idesc_bf16(128, (unsigned)p.e1p);
+            p.job_idesc[1] = make_idesc_bf16(128, (unsigned)p.e1p, (unsigned)p.f16);
         }
     }
     // CS consecutive CTAs work on the same bands, one part of the output layers each; such a group takes bands g,
@@ -872,13 +867,13 @@ int build_fire_plan(const ConvDesc* dsq, const ConvDesc& d1, const ConvDesc& d3,
             cuuint64_t dims[2] = {(cuuint64_t)Cin, npx};
             cuuint64_t str[1] = {(cuuint64_t)Cin * 2};
             cuuint32_t box[2] = {(cuuint32_t)p.BKc_in, 128};
-            if (!tmap_encode_bf16(&plan->x, 2, dsq->in, dims, str, box, p.rb_in)) return SQN_ERR_CUDA;
+            if (!tmap_encode_16(&plan->x, 2, dsq->in, dims, str, box, p.rb_in, p.f16)) return SQN_ERR_CUDA;
         }
         {
             cuuint64_t dims[2] = {(cuuint64_t)Cin, (cuuint64_t)s};
             cuuint64_t str[1] = {(cuuint64_t)Cin * 2};
             cuuint32_t box[2] = {(cuuint32_t)p.BKc_in, (cuuint32_t)s};
-            if (!tmap_encode_bf16(&plan->wsq, 2, dsq->w, dims, str, box, p.rb_in)) return SQN_ERR_CUDA;
+            if (!tmap_encode_16(&plan->wsq, 2, dsq->w, dims, str, box, p.rb_in, p.f16)) return SQN_ERR_CUDA;
         }
     } else {
         // the squeeze map [s][W][H][N]: a patch box is P pixels x (R + 2) rows of one chunk of layers
@@ -887,27 +882,27 @@ int build_fire_plan(const ConvDesc* dsq, const ConvDesc& d1, const ConvDesc& d3,
         cuuint64_t dims[5] = {(cuuint64_t)s, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N, 1};
         cuuint64_t str[4] = {s1, s1 * W, s1 * W * H, s1 * W * H * N};
         cuuint32_t box[5] = {(cuuint32_t)p.BKs, (cuuint32_t)p.P, (cuuint32_t)(p.R + 2), 1, 1};
-        if (!tmap_encode_bf16(&plan->x, 5, d1.in, dims, str, box, p.rb_s)) return SQN_ERR_CUDA;
+        if (!tmap_encode_16(&plan->x, 5, d1.in, dims, str, box, p.rb_s, p.f16)) return SQN_ERR_CUDA;
         plan->wsq = plan->x;            // (not read)
     }
     {
         cuuint64_t dims[2] = {(cuuint64_t)9 * s, (cuuint64_t)e3};
         cuuint64_t str[1] = {(cuuint64_t)9 * s * 2};
         cuuint32_t box[2] = {(cuuint32_t)p.BKs, (cuuint32_t)p.e3p};
-        if (!tmap_encode_bf16(&plan->w3, 2, d3.w, dims, str, box, p.rb_s)) return SQN_ERR_CUDA;
+        if (!tmap_encode_16(&plan->w3, 2, d3.w, dims, str, box, p.rb_s, p.f16)) return SQN_ERR_CUDA;
     }
     {
         cuuint64_t dims[2] = {(cuuint64_t)s, (cuuint64_t)e1};
         cuuint64_t str[1] = {(cuuint64_t)s * 2};
         cuuint32_t box[2] = {(cuuint32_t)p.BKs, (cuuint32_t)p.e1p};
-        if (!tmap_encode_bf16(&plan->w1, 2, d1.w, dims, str, box, p.rb_s)) return SQN_ERR_CUDA;
+        if (!tmap_encode_16(&plan->w1, 2, d1.w, dims, str, box, p.rb_s, p.f16)) return SQN_ERR_CUDA;
     }
     {
         const cuuint64_t s1 = (cuuint64_t)p.c_tot * 2;
         cuuint64_t dims[4] = {(cuuint64_t)(e1 + e3), (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)N};
         cuuint64_t str[3] = {s1, s1 * W, s1 * W * H};
         cuuint32_t box[4] = {(cuuint32_t)p.CW, (cuuint32_t)W, (cuuint32_t)p.RT, 1};
-        if (!tmap_encode_bf16(&plan->o, 4, d1.out, dims, str, box, (unsigned)p.CW * 2u)) return SQN_ERR_CUDA;
+        if (!tmap_encode_16(&plan->o, 4, d1.out, dims, str, box, (unsigned)p.CW * 2u, p.f16)) return SQN_ERR_CUDA;
     }
     return SQN_OK;
 }
@@ -937,7 +932,7 @@ int launch_fire(const ConvDesc* dsq, const ConvDesc& d1, const ConvDesc& d3, cud
     const char* bv = std::getenv("SQN_FIRE_BAND");
     const int band = bv ? std::atoi(bv) : 0;
     const int v[12] = {d1.N, dsq ? dsq->Cin : -1, d1.H, d1.W, d1.Cin, d1.Cout, d3.Cout, d1.out_c_total,
-                       (dsq ? dsq->params_static : 0) | (d1.params_static << 1) | (d3.params_static << 2), dev, band, 0};
+                       (dsq ? dsq->params_static : 0) | (d1.params_static << 1) | (d3.params_static << 2), dev, band, d1.f16};
     std::memcpy(k.v, v, sizeof(v));
     const std::string key(reinterpret_cast<const char*>(&k), sizeof(k));
     FirePlan plan;
@@ -954,11 +949,14 @@ int launch_fire(const ConvDesc* dsq, const ConvDesc& d1, const ConvDesc& d3, cud
         if (g_fire_plans.size() > 1024) g_fire_plans.clear();
         g_fire_plans[key] = plan;
     }
-    static const cudaError_t attr_rc =
-        cudaFuncSetAttribute(fire_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FF_SMEM_LIMIT);
-    if (attr_rc != cudaSuccess) return SQN_ERR_CUDA;
-    const cudaError_t rc = launch_chained(fire_fused_kernel, dim3((unsigned)plan.p.grid), dim3(FF_THREADS), plan.smem, stream,
-                                          plan.x, plan.wsq, plan.w3, plan.w1, plan.o, plan.p);
+    // (the 16-bit type is a compile-time constant of the kernel: the epilogues' conversion loops are straight-line code)
+    static const cudaError_t attr_rc0 =
+        cudaFuncSetAttribute(fire_fused_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FF_SMEM_LIMIT);
+    static const cudaError_t attr_rc1 =
+        cudaFuncSetAttribute(fire_fused_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FF_SMEM_LIMIT);
+    if (attr_rc0 != cudaSuccess || attr_rc1 != cudaSuccess) return SQN_ERR_CUDA;
+    const cudaError_t rc = launch_chained(plan.p.f16 ? fire_fused_kernel<true> : fire_fused_kernel<false>, dim3((unsigned)plan.p.grid),
+                                          dim3(FF_THREADS), plan.smem, stream, plan.x, plan.wsq, plan.w3, plan.w1, plan.o, plan.p);
     if (rc != cudaSuccess) return SQN_ERR_CUDA;
     note_launch();
     return cudaGetLastError() == cudaSuccess ? SQN_OK : SQN_ERR_CUDA;

@@ -3,6 +3,7 @@
 //   128-bit loads and stores along the layer dimension (memory bound: one read, one write);
 //   global average pooling + softmax: one block per image.
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include "sqn_internal.h"
 
@@ -56,15 +57,25 @@ __global__ void maxpool_f32_s(const float* __restrict__ in, float* __restrict__ 
     out[idx] = m;
 }
 
+// 16-bit element types of the tensor-core paths: scalar type, packed pair
+struct Bf16 { typedef __nv_bfloat16 T; typedef __nv_bfloat162 T2; };
+struct Fp16 { typedef __half T; typedef __half2 T2; };
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ float to_f32(__half v) { return __half2float(v); }
+__device__ __forceinline__ void from_f32(float f, __nv_bfloat16* o) { *o = __float2bfloat16(f); }
+__device__ __forceinline__ void from_f32(float f, __half* o) { *o = __float2half(f); }
+
+template <typename E>
 __device__ __forceinline__ uint32_t bmax2(uint32_t a, uint32_t b)
 {
-    __nv_bfloat162 x = *reinterpret_cast<__nv_bfloat162*>(&a);
-    __nv_bfloat162 y = *reinterpret_cast<__nv_bfloat162*>(&b);
-    __nv_bfloat162 m = __hmax2(x, y);
+    typename E::T2 x = *reinterpret_cast<typename E::T2*>(&a);
+    typename E::T2 y = *reinterpret_cast<typename E::T2*>(&b);
+    typename E::T2 m = __hmax2(x, y);
     return *reinterpret_cast<uint32_t*>(&m);
 }
 
-// bf16, C % 8 == 0: each thread produces 8 layers (16 bytes) of one output pixel.
+// 16-bit types, C % 8 == 0: each thread produces 8 layers (16 bytes) of one output pixel.
+template <typename E>
 __global__ void maxpool_bf16_v8(const uint4* __restrict__ in, uint4* __restrict__ out, int C8, int H, int W, int OH,
                                 int OW, long long total)
 {
@@ -85,12 +96,13 @@ __global__ void maxpool_bf16_v8(const uint4* __restrict__ in, uint4* __restrict_
 #pragma unroll
         for (int j = 0; j < 3; ++j) {
             const uint4 v = __ldg(src + ((long long)i * W + j) * C8);
-            m.x = bmax2(m.x, v.x); m.y = bmax2(m.y, v.y); m.z = bmax2(m.z, v.z); m.w = bmax2(m.w, v.w);
+            m.x = bmax2<E>(m.x, v.x); m.y = bmax2<E>(m.y, v.y); m.z = bmax2<E>(m.z, v.z); m.w = bmax2<E>(m.w, v.w);
         }
     out[idx] = m;
 }
 
-__global__ void maxpool_bf16_s(const __nv_bfloat16* __restrict__ in, __nv_bfloat16* __restrict__ out, int C, int H,
+template <typename E>
+__global__ void maxpool_bf16_s(const typename E::T* __restrict__ in, typename E::T* __restrict__ out, int C, int H,
                                int W, int OH, int OW, long long total)
 {
     chain_release();
@@ -102,17 +114,17 @@ __global__ void maxpool_bf16_s(const __nv_bfloat16* __restrict__ in, __nv_bfloat
     const int ow = (int)(r % OW); r /= OW;
     const int oh = (int)(r % OH);
     const long long n = r / OH;
-    const __nv_bfloat16* src = in + ((n * H + 2 * oh) * W + 2 * ow) * C + c;
-    float m = __bfloat162float(src[0]);
+    const typename E::T* src = in + ((n * H + 2 * oh) * W + 2 * ow) * C + c;
+    float m = to_f32(src[0]);
     for (int i = 0; i < 3; ++i)
-        for (int j = 0; j < 3; ++j) m = fmaxf(m, __bfloat162float(src[((long long)i * W + j) * C]));
-    out[idx] = __float2bfloat16(m);
+        for (int j = 0; j < 3; ++j) m = fmaxf(m, to_f32(src[((long long)i * W + j) * C]));
+    from_f32(m, &out[idx]);
 }
 
 // Global average: block (x = group of 128 layers, y = image), 256 threads = 64 layer pairs x 4 pixel
 // quarters.  Consecutive threads read consecutive 4- or 8-byte words of a pixel; the quarters are combined
 // in shared memory.  Small batches still get C/128 blocks per image.
-template <bool BF16>
+template <int MODE>        // 0: fp32, 1: bf16, 2: fp16
 __global__ void __launch_bounds__(256) global_avgpool_kernel(const void* __restrict__ in_, float* __restrict__ logits,
                                                              int C, int HW)
 {
@@ -128,7 +140,7 @@ __global__ void __launch_bounds__(256) global_avgpool_kernel(const void* __restr
     if (c < C) {
         const bool pair = (c + 1 < C) && (C % 2 == 0);
         auto ld = [&](int p, float& a, float& b) {
-            if (BF16) {
+            if (MODE == 1) {
                 const __nv_bfloat16* src = static_cast<const __nv_bfloat16*>(in_) + ((size_t)n * HW + p) * C + c;
                 if (pair) {
                     const __nv_bfloat162 w = *reinterpret_cast<const __nv_bfloat162*>(src);
@@ -136,6 +148,15 @@ __global__ void __launch_bounds__(256) global_avgpool_kernel(const void* __restr
                 } else {
                     a += __bfloat162float(src[0]);
                     if (c + 1 < C) b += __bfloat162float(src[1]);
+                }
+            } else if (MODE == 2) {
+                const __half* src = static_cast<const __half*>(in_) + ((size_t)n * HW + p) * C + c;
+                if (pair) {
+                    const __half2 w = *reinterpret_cast<const __half2*>(src);
+                    a += __low2float(w); b += __high2float(w);
+                } else {
+                    a += __half2float(src[0]);
+                    if (c + 1 < C) b += __half2float(src[1]);
                 }
             } else {
                 const float* src = static_cast<const float*>(in_) + ((size_t)n * HW + p) * C + c;
@@ -162,8 +183,9 @@ __global__ void __launch_bounds__(256) global_avgpool_kernel(const void* __restr
     }
 }
 
-// Global average of a bf16 map with C % 8 == 0: block (x = group of 128 layers, y = image), 256 threads =
+// Global average of a 16-bit map with C % 8 == 0: block (x = group of 128 layers, y = image), 256 threads =
 // 16 groups of 8 layers (one 16-byte load per pixel) x 16 pixel slices, four loads in flight per thread.
+template <typename E>
 __global__ void __launch_bounds__(256) global_avgpool_bf16_v8(const uint4* __restrict__ in, float* __restrict__ logits,
                                                               int C, int HW)
 {
@@ -180,7 +202,7 @@ __global__ void __launch_bounds__(256) global_avgpool_bf16_v8(const uint4* __res
         const int C8 = C >> 3;
         const uint4* src = in + (size_t)n * HW * C8 + (c0 >> 3);
         auto add = [&](const uint4& v) {
-            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+            const typename E::T2* h = reinterpret_cast<const typename E::T2*>(&v);
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 acc[2 * k] += __low2float(h[k]);
@@ -257,15 +279,21 @@ int launch_maxpool3x3s2(const void* in, void* out, int C, int H, int W, int N, i
                            static_cast<const float*>(in), static_cast<float*>(out), C, H, W, OH, OW, total);
         }
     } else {
+        const bool f16 = dtype == SQN_F16;
         if (C % 8 == 0) {
             const long long total = (long long)N * OH * OW * (C / 8);
-            launch_chained(maxpool_bf16_v8, dim3((unsigned)((total + threads - 1) / threads)), dim3(threads), 0, stream,
-                           static_cast<const uint4*>(in), static_cast<uint4*>(out), C / 8, H, W, OH, OW, total);
+            const dim3 grid((unsigned)((total + threads - 1) / threads));
+            if (f16) launch_chained(maxpool_bf16_v8<Fp16>, grid, dim3(threads), 0, stream, static_cast<const uint4*>(in),
+                                    static_cast<uint4*>(out), C / 8, H, W, OH, OW, total);
+            else launch_chained(maxpool_bf16_v8<Bf16>, grid, dim3(threads), 0, stream, static_cast<const uint4*>(in),
+                                static_cast<uint4*>(out), C / 8, H, W, OH, OW, total);
         } else {
             const long long total = (long long)N * OH * OW * C;
-            launch_chained(maxpool_bf16_s, dim3((unsigned)((total + threads - 1) / threads)), dim3(threads), 0, stream,
-                           static_cast<const __nv_bfloat16*>(in), static_cast<__nv_bfloat16*>(out), C, H, W, OH, OW,
-                           total);
+            const dim3 grid((unsigned)((total + threads - 1) / threads));
+            if (f16) launch_chained(maxpool_bf16_s<Fp16>, grid, dim3(threads), 0, stream, static_cast<const __half*>(in),
+                                    static_cast<__half*>(out), C, H, W, OH, OW, total);
+            else launch_chained(maxpool_bf16_s<Bf16>, grid, dim3(threads), 0, stream, static_cast<const __nv_bfloat16*>(in),
+                                static_cast<__nv_bfloat16*>(out), C, H, W, OH, OW, total);
         }
     }
     note_launch();
@@ -276,10 +304,14 @@ int launch_avgpool_softmax(const void* in, float* logits, float* probs, int C, i
                            cudaStream_t stream)
 {
     const dim3 grid((unsigned)((C + 127) / 128), (unsigned)N);
-    if (dtype == SQN_F32) launch_chained(global_avgpool_kernel<false>, grid, dim3(256), 0, stream, in, logits, C, H * W);
-    else if (C % 8 == 0 && aligned16(in))
-        launch_chained(global_avgpool_bf16_v8, grid, dim3(256), 0, stream, static_cast<const uint4*>(in), logits, C, H * W);
-    else launch_chained(global_avgpool_kernel<true>, grid, dim3(256), 0, stream, in, logits, C, H * W);
+    if (dtype == SQN_F32) launch_chained(global_avgpool_kernel<0>, grid, dim3(256), 0, stream, in, logits, C, H * W);
+    else if (C % 8 == 0 && aligned16(in)) {
+        if (dtype == SQN_F16)
+            launch_chained(global_avgpool_bf16_v8<Fp16>, grid, dim3(256), 0, stream, static_cast<const uint4*>(in), logits, C, H * W);
+        else
+            launch_chained(global_avgpool_bf16_v8<Bf16>, grid, dim3(256), 0, stream, static_cast<const uint4*>(in), logits, C, H * W);
+    } else if (dtype == SQN_F16) launch_chained(global_avgpool_kernel<2>, grid, dim3(256), 0, stream, in, logits, C, H * W);
+    else launch_chained(global_avgpool_kernel<1>, grid, dim3(256), 0, stream, in, logits, C, H * W);
     note_launch();
     if (cudaGetLastError() != cudaSuccess) return SQN_ERR_CUDA;
     if (probs) return launch_softmax(logits, probs, C, N, stream);

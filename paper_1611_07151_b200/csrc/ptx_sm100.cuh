@@ -176,12 +176,13 @@ __device__ __forceinline__ uint64_t make_kmajor_desc_plain(uint32_t smem_addr, u
     return d;
 }
 
-// Instruction descriptor for kind::f16: bf16 x bf16 -> fp32, both operands K-major, M x N tile.
-__host__ __device__ constexpr uint32_t make_idesc_bf16(uint32_t M, uint32_t N)
+// Instruction descriptor for kind::f16: 16-bit operands (bf16, or fp16 when `f16` is set: both operands always of
+// the same type) -> fp32, both operands K-major, M x N tile.
+__host__ __device__ constexpr uint32_t make_idesc_bf16(uint32_t M, uint32_t N, uint32_t f16 = 0)
 {
-    return (1u << 4)      // D format: f32
-         | (1u << 7)      // A format: bf16
-         | (1u << 10)     // B format: bf16
+    return (1u << 4)                    // D format: f32
+         | ((f16 ? 0u : 1u) << 7)       // A format: 0 = f16, 1 = bf16
+         | ((f16 ? 0u : 1u) << 10)      // B format
          | ((N >> 3) << 17)
          | ((M >> 4) << 24);
 }

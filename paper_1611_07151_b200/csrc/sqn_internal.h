@@ -20,6 +20,7 @@ struct ConvDesc {
     int pool;             // 1: out receives the 3x3/stride-2 max-pool of the layer's output (bf16 path only)
     int params_static;    // 1: kernels and bias are not written by earlier work on the stream (a net's own parameters), so
                           //    a chained launch may fetch them before the kernel ahead of it has finished
+    int f16;              // tensor-core paths: 1 = activations and kernels are fp16, 0 = bf16
     int stem_prepacked;   // 1 (stem only): in and w already have the stem kernel's own layouts, see sqn_pack_stem_input
 };
 

@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include "ptx_sm100.cuh"
 #include "sqn_internal.h"
@@ -35,16 +36,21 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     return wait_bar_limit(bar, parity, abort_flag, status, WAIT_LIMIT_CYCLES);
 }
 
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
-{
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&v);
-}
-// max(.,0) and round-to-nearest-even conversion of two values in one instruction
-__device__ __forceinline__ uint32_t pack_relu_bf16x2(float lo, float hi)
+// The 16-bit storage type of the tensor-core paths is bf16, or fp16 where `f16` is set (same size, same layouts).
+// two fp32 values -> packed pair, round to nearest even
+__device__ __forceinline__ uint32_t pack_x2(float lo, float hi, int f16)
 {
     uint32_t d;
-    asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    if (f16) asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    else asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+// max(.,0) and the conversion of two values in one instruction
+__device__ __forceinline__ uint32_t pack_relu_x2(float lo, float hi, int f16)
+{
+    uint32_t d;
+    if (f16) asm("cvt.rn.relu.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    else asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
     return d;
 }
 
@@ -55,14 +61,39 @@ __device__ __forceinline__ float max3(float a, float b, float c)
     asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
     return r;
 }
-// fp32 -> bf16 (round to nearest even), with max(., 0) folded into the conversion when relu is set
-__device__ __forceinline__ unsigned short to_bf16_bits(float v, int relu)
+// fp32 -> 16 bits (round to nearest even), with max(., 0) folded into the conversion when relu is set
+__device__ __forceinline__ unsigned short to_16_bits(float v, int relu, int f16)
 {
     unsigned short h;
-    if (relu) asm("cvt.rn.relu.bf16.f32 %0, %1;" : "=h"(h) : "f"(v));
-    else asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(h) : "f"(v));
+    if (f16) {
+        if (relu) asm("cvt.rn.relu.f16.f32 %0, %1;" : "=h"(h) : "f"(v));
+        else asm("cvt.rn.f16.f32 %0, %1;" : "=h"(h) : "f"(v));
+    } else {
+        if (relu) asm("cvt.rn.relu.bf16.f32 %0, %1;" : "=h"(h) : "f"(v));
+        else asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(h) : "f"(v));
+    }
     return h;
 }
-
+// 1.0 twice
+__device__ __forceinline__ uint32_t one_x2(int f16) { return f16 ? 0x3c003c00u : 0x3f803f80u; }
+// b as {hi, lo} with hi + lo = b to 16 (bf16) or 22 (fp16) bits below its leading bit
+__device__ __forceinline__ uint32_t bias_hi_lo(float b, int f16)
+{
+    if (f16) {
+        const __half hi = __float2half_rn(b);
+        const __half lo = __float2half_rn(b - __half2float(hi));
+        return (uint32_t)__half_as_ushort(hi) | ((uint32_t)__half_as_ushort(lo) << 16);
+    }
+    const __nv_bfloat16 hi = __float2bfloat16_rn(b);
+    const __nv_bfloat16 lo = __float2bfloat16_rn(b - __bfloat162float(hi));
+    return (uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(lo) << 16);
+}
+// Bias row of the bias MMAs: one 32-byte row {hi, lo, 0, ...} per output layer in the 32-byte swizzle.
+__device__ __forceinline__ void bias_row(uint4* rows, int c, float b, int f16)
+{
+    const int u = (c >> 2) & 1;
+    rows[2 * c + u] = make_uint4(bias_hi_lo(b, f16), 0u, 0u, 0u);
+    rows[2 * c + (u ^ 1)] = make_uint4(0u, 0u, 0u, 0u);
+}
 
 }  // namespace sqn

@@ -140,3 +140,15 @@ def test_stem_pack_helpers_give_the_layout_the_stem_kernel_reads():
     with pytest.raises(B.SqnError):
         B.squeezenet_set_stem_prepacked(h, True)          # bf16 nets only
     B.squeezenet_destroy(h)
+
+
+def test_fp16_rounding_is_nearest_even():
+    rng = np.random.default_rng(2)
+    x = np.concatenate([rng.standard_normal(4096).astype(np.float32) * 10,
+                        np.array([0.0, -0.0, 1.0, 1.00048828125, 1.0009765625, 65504.0, 65520.0, 1e-8, 6e-8, np.inf], np.float32)])
+    x = x.reshape(1, -1, 1, 1)
+    got = B.sqn_pack_nchw_to_nhwc(x, B.SQN_F16).ravel()
+    exp = torch.from_numpy(x.ravel()).to(torch.float16).view(torch.int16).numpy().view(np.uint16)
+    np.testing.assert_array_equal(got, exp)
+    back = B.sqn_unpack_nhwc_to_nchw(got.reshape(1, 1, 1, -1), B.SQN_F16).ravel()
+    np.testing.assert_array_equal(back, torch.from_numpy(x.ravel()).to(torch.float16).float().numpy())

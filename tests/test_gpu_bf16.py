@@ -227,6 +227,13 @@ def test_config3_headline_batch256_all_images_against_the_oracle():
           "layer error %.2e; logits %.2e" % (agree, flips, batch, near, max(chained.values()), G.rel_err(logits, z)))
     assert agree >= 0.99, (agree, flips, near)
     np.testing.assert_allclose(probs.astype(np.float64).sum(1), 1.0, rtol=0, atol=1e-5)
+    # the same batch through the fp16 path (third precision point) against the same oracle run
+    del views
+    logits16, probs16, _views16 = run_net_device(x, params, B.SQN_F16, batch)
+    agree16, flips16, near16 = _top1_report(logits16, z)
+    print("config 3 in fp16: top-1 agreement %.4f (%d differ); logits %.2e" % (agree16, flips16, G.rel_err(logits16, z)))
+    assert G.rel_err(logits16, z) <= G.TOL[B.SQN_F16]
+    assert agree16 >= 0.99, (agree16, flips16, near16)
 
 
 # (N, Cin, Cout, H, W, K, S, pad): fused max-pool with more strips than CTAs, so that CTAs take a second strip

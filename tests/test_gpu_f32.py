@@ -157,7 +157,7 @@ def run_net_device(x, params, dtype, batch):
         off = ptr - work.data_ptr()
         es = 4 if dtype == F32 else 2
         raw = work[off:off + batch * C * H * W * es]
-        views[name] = raw.view(torch.float32 if dtype == F32 else torch.bfloat16).view(batch, H, W, C)
+        views[name] = raw.view({F32: torch.float32, B.SQN_BF16: torch.bfloat16, B.SQN_F16: torch.float16}[dtype]).view(batch, H, W, C)
     B.squeezenet_destroy(net)
     return logits.cpu().numpy(), probs.cpu().numpy(), views
 
