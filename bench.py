@@ -316,9 +316,10 @@ def layer_table(B, net, step, steps, batch, es, dtype_tag, peaks, sm_count, sm_m
     return layers, ms_step, pipe, pipe_sus
 
 
-def run_sweep(B):
-    """Every distinct SqueezeNet conv shape at batch 1, 16, 64, 256 in fp32 and bf16 (seed 4 recipe, values
-    drawn on the device): time per launch with CUDA events, L2 flushed before each timed launch."""
+def run_sweep(B, family="squeezenet"):
+    """Every distinct conv shape of a workload (SqueezeNet v1.0, or the bottleneck-network family) at batch 1, 16, 64,
+    256 in fp32 and bf16 (seed 4 recipe, values drawn on the device): median of ten single launches with the L2
+    overwritten before each, and the mean of 20 back-to-back launches over rotating buffers."""
     import torch
     peaks = measured_peaks()
     dev = "cuda:0"
@@ -328,7 +329,7 @@ def run_sweep(B):
     gen = torch.Generator(device=dev)
     gen.manual_seed(4)
     seen, rows = set(), []
-    for name, cin, cout, k, s, pad, hw in synth.SQUEEZENET_CONVS:
+    for name, cin, cout, k, s, pad, hw in (synth.SQUEEZENET_CONVS if family == "squeezenet" else synth.BOTTLENECK_CONVS):
         key = (cin, cout, k, s, pad, hw)
         if key in seen:
             continue
@@ -361,16 +362,31 @@ def run_sweep(B):
                     torch.cuda.synchronize()
                     times.append(e0.elapsed_time(e1))
                 ms = float(np.median(times))
+                # ... and back to back over a second buffer set (mean of 20 launches)
+                x2, out2 = x.clone(), torch.empty_like(out)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for i in range(20):
+                    if i & 1:
+                        B.conv_forward_ex(x2, w, b, out2, cin, cout, hw, hw, k, s, pad, batch, dtype=dtype, workspace=wsb,
+                                          workspace_bytes=nb)
+                    else:
+                        call()
+                e1.record()
+                torch.cuda.synchronize()
+                ms_b2b = e0.elapsed_time(e1) / 20
+                del x2, out2
                 flops = 2.0 * batch * oh * oh * cout * cin * k * k
                 byts = es * batch * (hw * hw * cin + oh * oh * cout) + es * cout * cin * k * k + 4 * cout
                 t_hbm, t_pipe = byts / (peaks["hbm_gbs"] * 1e9), flops / (pipe_tf * 1e12)
-                rows.append({"layer": name, "dtype": tag, "batch": batch, "ms": ms, "tflops": flops / ms / 1e9,
+                rows.append({"layer": name, "dtype": tag, "batch": batch, "ms": ms, "ms_back_to_back": ms_b2b, "tflops": flops / ms / 1e9,
                              "gbs": byts / ms / 1e6, "bound": "hbm" if t_hbm >= t_pipe else ("tensor" if tag == "bf16" else "alu"),
                              "frac": max(t_hbm, t_pipe) / (ms * 1e-3)})
                 del x, w, out
     assert B.sqn_check() == B.SQN_OK
-    print(json.dumps({"sweep": rows, "peaks": peaks,
-                      "note": "bf16 stem time includes its repack launches; one launch, L2 flushed, median of 10"}))
+    print(json.dumps({"sweep": rows, "family": family, "peaks": peaks,
+                      "note": "bf16 stem time includes its repack launches; ms: one launch, L2 flushed, median of 10; "
+                              "ms_back_to_back: mean of 20 launches alternating two buffer sets"}))
 
 
 def run_variants(B, batch):
@@ -395,24 +411,31 @@ def run_variants(B, batch):
         b = torch.randn((cout,), device=dev, generator=gen) * 0.01
         out = torch.empty((batch, oh, oh, cout), device=dev, dtype=torch.bfloat16)
 
+        x2, out2 = x.clone(), torch.empty_like(out)
+
         def timed():
-            def call():
-                B.conv_forward_ex(x, w, b, out, cin, cout, hw, hw, k, s, pad, batch, dtype=B.SQN_BF16)
+            """Mean of 20 back-to-back launches alternating two buffer sets (microseconds); None if the variant does not fit."""
+            def call(i):
+                if i & 1:
+                    B.conv_forward_ex(x2, w, b, out2, cin, cout, hw, hw, k, s, pad, batch, dtype=B.SQN_BF16)
+                else:
+                    B.conv_forward_ex(x, w, b, out, cin, cout, hw, hw, k, s, pad, batch, dtype=B.SQN_BF16)
             try:
-                for _ in range(3):
-                    call()
+                for i in range(4):
+                    call(i)
             except B.SqnError as e:
                 assert e.status == B.SQN_ERR_UNSUPPORTED
                 return None
             ts = []
-            for _ in range(10):
+            for _ in range(3):
                 flush.zero_()
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record()
-                call()
+                for i in range(20):
+                    call(i)
                 e1.record()
                 torch.cuda.synchronize()
-                ts.append(e0.elapsed_time(e1))
+                ts.append(e0.elapsed_time(e1) / 20)
             return float(np.median(ts)) * 1e3
 
         os.environ.pop("SQN_TC_VARIANT", None)
@@ -428,10 +451,10 @@ def run_variants(B, batch):
         worst = max(row["variants"].items(), key=lambda kv: kv[1])
         row.update({"optimal": best[0], "optimal_us": best[1], "pessimal": worst[0], "pessimal_us": worst[1]})
         rows.append(row)
-        del x, w, out
+        del x, w, out, x2, out2
     assert B.sqn_check() == B.SQN_OK
-    print(json.dumps({"variants": rows, "note": "variant = <CTAs per SM>x<store chunk width>; one launch, L2 flushed, "
-                      "median of 10, microseconds; a missing variant does not fit the layer"}))
+    print(json.dumps({"variants": rows, "note": "variant = <CTAs per SM>x<store chunk width>; mean of 20 back-to-back launches "
+                      "alternating two buffer sets, median of 3 such runs, microseconds; a missing variant does not fit the layer"}))
 
 
 def run_kernel_case(B, name, batch, steps):
@@ -535,6 +558,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-batch1", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="per-layer sweep of every conv shape instead of the network")
+    ap.add_argument("--family", default="squeezenet", choices=["squeezenet", "bottleneck"],
+                    help="--sweep: the workload whose conv shapes are swept (bottleneck: the 1x1 / 3x3 shapes of a residual network)")
     ap.add_argument("--variants", action="store_true", help="per-layer sweep of the bf16 kernel variants at --batch")
     ap.add_argument("--mma-rate", action="store_true", help="clocks per tcgen05.mma as a function of N (diagnostic)")
     ap.add_argument("--kernel", default=None, help="one layer on its own (bf16): a conv name (conv1, fire6_e3, ...), "
@@ -551,7 +576,7 @@ def main():
     from paper_1611_07151_b200 import binding as B
 
     if args.sweep:
-        run_sweep(B)
+        run_sweep(B, args.family)
         return
     if args.variants:
         run_variants(B, args.batch)

@@ -47,7 +47,8 @@ typedef enum {
     SQN_ERR_ALIGN = -3,        /* pointer or layer count breaks an alignment rule */
     SQN_ERR_CUDA = -4,         /* a CUDA runtime/driver call failed */
     SQN_ERR_TIMEOUT = -5,      /* a bounded device-side wait ran out (reported by sqn_check) */
-    SQN_ERR_WORKSPACE = -6     /* workspace missing or too small */
+    SQN_ERR_WORKSPACE = -6,    /* workspace missing or too small */
+    SQN_ERR_DEBUG = -7         /* an index check of the debug build (-DSQN_DEBUG) failed; the access was skipped (sqn_check) */
 } sqn_status;
 
 typedef enum { SQN_F32 = 0, SQN_BF16 = 1, SQN_F16 = 2 } sqn_dtype;

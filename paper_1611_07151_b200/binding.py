@@ -21,8 +21,10 @@ SQN_ERR_ALIGN = -3
 SQN_ERR_CUDA = -4
 SQN_ERR_TIMEOUT = -5
 SQN_ERR_WORKSPACE = -6
+SQN_ERR_DEBUG = -7
 
-LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libsqn.so")
+# SQN_LIBRARY in the environment names another build of the same library (the bounds-checked libsqn_debug.so)
+LIB_PATH = os.environ.get("SQN_LIBRARY") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libsqn.so")
 
 _c_int = ctypes.c_int
 _c_vp = ctypes.c_void_p

@@ -11,6 +11,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libsqn.so")
+LIB_DEBUG = os.path.join(PKG, "libsqn_debug.so")      # the same sources with -DSQN_DEBUG: index checks in the kernels
 OBJ_DIR = os.path.join(PKG, "_build")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -26,24 +27,26 @@ def _deps():
         glob.glob(os.path.join(ROOT, "include", "*.h"))
 
 
-def up_to_date():
-    if not os.path.exists(LIB):
+def up_to_date(lib=LIB):
+    if not os.path.exists(lib):
         return False
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     return all(os.path.getmtime(f) <= t for f in _deps())
 
 
-def build(force=False, verbose=False):
-    """Compile every .cu under csrc/ and link them into libsqn.so."""
-    if not force and up_to_date():
-        return LIB
+def build(force=False, verbose=False, debug=False):
+    """Compile every .cu under csrc/ and link them into libsqn.so (debug=True: libsqn_debug.so, with -DSQN_DEBUG)."""
+    lib = LIB_DEBUG if debug else LIB
+    if not force and up_to_date(lib):
+        return lib
     nvcc = os.environ.get("NVCC", "nvcc")
-    os.makedirs(OBJ_DIR, exist_ok=True)
-    extra = ["-Xptxas", "-v"] if verbose else []
+    obj_dir = OBJ_DIR + ("_debug" if debug else "")
+    os.makedirs(obj_dir, exist_ok=True)
+    extra = (["-Xptxas", "-v"] if verbose else []) + (["-DSQN_DEBUG"] if debug else [])
     hdr_t = max(os.path.getmtime(f) for f in _deps() if not f.endswith(".cu"))
     objs, procs = [], []
     for src in _sources():
-        obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
+        obj = os.path.join(obj_dir, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
         if (not force and os.path.exists(obj)
                 and os.path.getmtime(obj) >= max(os.path.getmtime(src), hdr_t)):
@@ -52,11 +55,11 @@ def build(force=False, verbose=False):
     for src, p in procs:
         if p.wait() != 0:
             raise RuntimeError("nvcc failed on " + src)
-    tmp = LIB + ".tmp.%d" % os.getpid()
+    tmp = lib + ".tmp.%d" % os.getpid()
     subprocess.run([nvcc, "-shared", "-o", tmp] + objs + ["-lcudart"], check=True)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, debug="--debug" in sys.argv))

@@ -958,6 +958,7 @@ extern "C" const char* sqn_status_string(int status)
         case SQN_ERR_CUDA: return "CUDA call failed";
         case SQN_ERR_TIMEOUT: return "device-side wait timed out";
         case SQN_ERR_WORKSPACE: return "workspace missing or too small";
+        case SQN_ERR_DEBUG: return "index check of the debug build failed";
         default: return "unknown status";
     }
 }

@@ -559,6 +559,7 @@ __device__ __forceinline__ void conv_tc_body(const CUtensorMap& tmA, const CUten
                     const int c0 = chunk * p.CW;
                     if (n0 + c0 >= p.Cout) break;
                     if (!wait_bar(smem_u32(&sh->stg_full[sb]), sph, abort_flag, p.status)) { ok = false; break; }
+                    if (sqn_dbg_ok(n0 + c0 < p.Cout && w0 < p.tiles_w * p.BW && h0 < p.tiles_h * p.BH && i0 < p.tiles_i * p.BI && sb < p.nstg, p.status))
                     tma_store_4d(&tmO, smStg + (uint32_t)sb * slot_bytes, p.c_off + n0 + c0, w0, h0, i0);
                     tma_store_commit();
                     if (++sb == p.nstg) { sb = 0; sph ^= 1u; }
@@ -879,7 +880,7 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
                                 o2 = max3(c[2], c[3], c[4]), o3 = max3(c[4], c[5], c[6]);
                     cr[r][0] = c[6];
                     cr[r][1] = c[7];
-                    if (live && ph0 + r < p.PH_out) {
+                    if (live && ph0 + r < p.PH_out && sqn_dbg_ok(tc.ti < p.tiles_i && c_off + m < p.pool_ctot, p.status)) {
                         unsigned short* dst = dst0 + r * row_stride;
                         if (first) dst[0] = to_16_bits(o0, p.relu, F16);
                         if (last1) dst[p.pool_ctot] = to_16_bits(o1, p.relu, F16);

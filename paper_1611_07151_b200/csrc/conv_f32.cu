@@ -21,6 +21,7 @@ struct F32Params {
     const float* w;
     const float* bias;
     float* out;
+    int* status;
     int N, Cin, H, W, Cout, K, S, pad, OH, OW;
     int M;      // N*OH*OW
     int Kdim;   // K*K*Cin
@@ -280,6 +281,7 @@ __global__ void __launch_bounds__(NTHREADS, 2) conv_f32_kernel(const F32Params p
                 v[j] = acc[i][q * VN + j] + bv[j];
                 if (p.relu) v[j] = fmaxf(v[j], 0.f);
             }
+            if (!sqn_dbg_ok(m >= 0 && p.out_c_offset + col0 >= 0 && p.out_c_offset + (col0 < p.Cout ? col0 : 0) < p.out_c_total, p.status)) continue;
             float* dst = p.out + (size_t)m * p.out_c_total + p.out_c_offset + col0;
             if (vec_store && col0 + VN <= p.Cout) {
                 if (VN == 4) *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
@@ -312,6 +314,7 @@ int launch_conv_f32(const ConvDesc& d, cudaStream_t stream)
     p.w = static_cast<const float*>(d.w);
     p.bias = d.bias;
     p.out = static_cast<float*>(d.out);
+    p.status = device_status_word();
     p.N = d.N; p.Cin = d.Cin; p.H = d.H; p.W = d.W; p.Cout = d.Cout; p.K = d.K; p.S = d.S; p.pad = d.pad;
     p.OH = d.OH; p.OW = d.OW;
     const long long M = (long long)d.N * d.OH * d.OW;

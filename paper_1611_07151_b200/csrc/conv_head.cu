@@ -220,7 +220,7 @@ conv_head_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[as]));
             if (++as == 2) { as = 0; aph ^= 1u; }
-            if (live) p.logits[(size_t)n * p.Cout + layer] = ((s0 + s1) + (s2 + s3)) * p.inv_hw;
+            if (live && sqn_dbg_ok(n < p.N && layer < p.Cout, p.status)) p.logits[(size_t)n * p.Cout + layer] = ((s0 + s1) + (s2 + s3)) * p.inv_hw;
         }
     }
 

@@ -436,6 +436,7 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
                         // accumulator-order columns [0, e3p) are the part's 3x3 layers (output layers e1 + ..), the rest its 1x1 layers
                         const int col = chunk * p.CW;
                         const int cc = col < p.e3p ? p.e1 + part * p.e3p + col : part * p.e1p + col - p.e3p;
+                        if (sqn_dbg_ok(cc >= 0 && cc + p.CW <= p.e1 + p.e3 && b.y0 + t * p.RT < p.H && b.n < p.N, p.status))
                         tma_store_4d(&tmO, smStg + (uint32_t)sb * p.stg_slot, cc, 0, b.y0 + t * p.RT, b.n);
                         tma_store_commit();
                         if (++sb == p.nstg) { sb = 0; sph ^= 1u; }
@@ -491,6 +492,7 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
                 if (g < b.npx) {
                     const int yy = g / p.W, xx = g - yy * p.W;
                     const uint32_t pr = (uint32_t)((yy + b.ylo - b.y0 + 1) * p.P + xx + 1);
+                    if (!sqn_dbg_ok((pr + 1u) * p.rb_s <= p.patch_chunk, p.status)) continue;      // (the row lies inside the patch)
                     const uint32_t rbase = patch + pr * p.rb_s;
                     const uint32_t sw = swz(pr, p.rb_s);
                     store16<F16>(&v[0], rbase, 0u, sw);
@@ -555,7 +557,7 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
                             ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->stg_free[sb]), sph ^ 1u, abort_flag, p.status));
                             tmem_ld_wait();
                             if (!ok) break;
-                            if (e_valid) {
+                            if (e_valid && sqn_dbg_ok(stg_off + (uint32_t)(p.CW * 2) <= p.stg_slot && sb < p.nstg, p.status)) {
                                 const uint32_t rbase = smStg + (uint32_t)sb * p.stg_slot + stg_off;
                                 store16<F16>(&v[0], rbase, 0u, sw_e);
                                 store16<F16>(&v[16], rbase, 2u, sw_e);

@@ -107,6 +107,20 @@ __device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.l
 __device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 #endif
 
+// Debug build (-DSQN_DEBUG): index checks in the kernels.  A failed check records SQN_ERR_DEBUG in the status word and
+// the guarded access is skipped; nothing traps.  In the normal build the checks compile to nothing.
+#ifdef __CUDACC__
+#ifdef SQN_DEBUG
+__device__ __forceinline__ bool sqn_dbg_ok(bool cond, int* status)
+{
+    if (!cond && status) atomicExch(status, (int)SQN_ERR_DEBUG);
+    return cond;
+}
+#else
+__device__ __forceinline__ bool sqn_dbg_ok(bool, int*) { return true; }
+#endif
+#endif
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace sqn

@@ -26,6 +26,16 @@ for _name, _cin, _s, _e, _hw in [("fire2", 96, 16, 64, 55), ("fire3", 128, 16, 6
 SQUEEZENET_CONVS.append(("conv10", 512, 1000, 1, 1, 0, 13))
 
 
+# A second workload for the single-layer entry points: the distinct 1x1 / 3x3 stride-1 convolution shapes of a
+# bottleneck residual network on a 224x224 image (name, Cin, Cout, K, S, pad, input H=W).
+BOTTLENECK_CONVS = [
+    ("stage2_reduce", 256, 64, 1, 1, 0, 56), ("stage2_3x3", 64, 64, 3, 1, 1, 56), ("stage2_expand", 64, 256, 1, 1, 0, 56),
+    ("stage3_reduce", 512, 128, 1, 1, 0, 28), ("stage3_3x3", 128, 128, 3, 1, 1, 28), ("stage3_expand", 128, 512, 1, 1, 0, 28),
+    ("stage4_reduce", 1024, 256, 1, 1, 0, 14), ("stage4_3x3", 256, 256, 3, 1, 1, 14), ("stage4_expand", 256, 1024, 1, 1, 0, 14),
+    ("stage5_reduce", 2048, 512, 1, 1, 0, 7), ("stage5_3x3", 512, 512, 3, 1, 1, 7), ("stage5_expand", 512, 2048, 1, 1, 0, 7),
+]
+
+
 def draw_input(rng, shape, dist="uniform"):
     if dist == "uniform":
         return rng.random(shape, dtype=np.float32)
