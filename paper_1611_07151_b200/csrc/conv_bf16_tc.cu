@@ -129,8 +129,8 @@ struct Shared {                       // control block placed after the tiles
     unsigned long long full[MAX_STAGES];
     unsigned long long empty[MAX_STAGES];
     unsigned long long b_full;
-    unsigned long long tmem_full[2];
-    unsigned long long tmem_empty[2];
+    unsigned long long tmem_full[4];      // (conv_pool_kernel with a rider: two accumulators per layer)
+    unsigned long long tmem_empty[4];
     unsigned long long stg_full[MAX_STG];
     unsigned long long stg_free[MAX_STG];
     unsigned tmem_base;
@@ -628,25 +628,25 @@ conv_tc_kernel2(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
 // 128-pixel tiles of conv_tc_kernel, which is what bounds these layers with few output layers.
 // A CTA walks a strip of 32 output rows (strips 30 rows apart: 15 pooled rows) from left to right; tile k emits the
 // pooled columns 4k-1 .. 4k+2, the vertical maxima of its last two columns are carried to tile k+1 in registers.
-// Warps: 0 TMA producer, 1 MMA issuer, 2..17 epilogue (lane quadrant = warp % 4; the four groups of four warps
-// take four pooled rows of the strip each, the last group three).  The bias is added by one more MMA (bias rows
+// Warps: 0 TMA producer, 1 MMA issuer, 18 the rider's MMA issuer, 2..17 epilogue (lane quadrant = warp % 4; the four
+// groups of four warps take four (two) pooled rows of the strip each, the last group one fewer).  The bias is added by one more MMA (bias rows
 // {hi, lo} x tile of ones).  Lanes past the last output layer compute on whatever follows the kernels in shared
 // memory and are never read.
-constexpr int POOLT_THREADS = 64 + 512;
+constexpr int POOLT_THREADS = 64 + 512 + 32;
+constexpr int POOLT_RIDER_WARP = 18;           // issues the rider's MMAs (idle without a rider)
 __host__ __device__ constexpr int poolt_rows(int npix) { return npix / 8; }                 // output rows per tile
 __host__ __device__ constexpr int poolt_prows(int npix) { return (npix / 8 - 2) / 2; }      // pooled rows per strip
 
 // NPIX = 256 (8 x 32 pixels per tile, 15 pooled rows per strip) where the layer's kernels leave room for the larger
 // patches, else 128 (8 x 16 pixels, 7 pooled rows).
-template <int NPIX, bool F16>
+// CTOT: the layers per pixel of the pooled tensor as a compile-time constant (0: read from the parameters) -- the
+// four stores of a pooled row then differ by immediate offsets.
+template <int NPIX, bool F16, int CTOT>
 __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB2,
                                                const TcParams& p, const int bid)
 {
     constexpr int PROWS = poolt_prows(NPIX);          // 15 or 7
     constexpr int PR = (PROWS + 3) / 4;               // pooled rows per epilogue group: 4 or 2
-    constexpr int ROUNDS = PR == 4 ? 2 : 1;           // TMEM read rounds per tile
-    constexpr int RPR = PR / ROUNDS;                  // pooled rows per round: 2
-    constexpr int RCOLS = 16 * RPR + 8;               // accumulator columns per round: 40
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -661,6 +661,7 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
     const int items = p.taps * p.chunks;
     const int nmma = items * (p.BKc / 16);
     const int my_tiles = tiles_of_cta(p, bid);
+    const int n_acc = p.rider ? 3 : 2;              // accumulators of the layer itself
     // every kernel tile of the layer (and of its rider), once: one mbarrier counts them all
     auto load_kernels = [&]() {
         const uint32_t bar = smem_u32(&sh->b_full);
@@ -684,10 +685,10 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(smem_u32(&sh->full[s]), 1);
-            mbar_init(smem_u32(&sh->empty[s]), 1);
+            mbar_init(smem_u32(&sh->empty[s]), p.rider ? 2 : 1);      // (a rider's issuer reads the patch too)
         }
         mbar_init(smem_u32(&sh->b_full), 1);
-        for (int a = 0; a < 2; ++a) {
+        for (int a = 0; a < 4; ++a) {
             mbar_init(smem_u32(&sh->tmem_full[a]), 1);
             mbar_init(smem_u32(&sh->tmem_empty[a]), 4 * ((p.Cout + 31) / 32));     // the epilogue warps that have output layers
         }
@@ -770,6 +771,11 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
         const uint64_t bias_desc = make_kmajor_desc(base + p.off_bias, 32u, 256u);
         const uint64_t ones_desc = make_kmajor_desc(base + p.off_ones, 32u, 256u);
         bool ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->b_full), 0u, abort_flag, p.status));
+        // The tiles take the layer's accumulators in turn: two, or with a rider (128-pixel tiles) three, the rider's few
+        // MMAs going to the fourth.  From the commit of a tile's MMAs to the issuer seeing its accumulator free again
+        // (MMA drain, the epilogue's wake-up and TMEM loads, the way back) is about as long as two such tiles' MMAs.
+        // The rider's MMAs are issued by a warp of their own: with 64 clocks per MMA issuing, not the tensor pipe, is
+        // what a single thread is bound by.
         int s = 0, as = 0;
         uint32_t ph = 0, aph = 0;
         for (int it = 0; it < my_tiles && ok; ++it) {
@@ -789,20 +795,38 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
                                 ((uint64_t)hiX << 32) | (uint64_t)((x_base + o.x) | 0x10000u), idesc, acc);
                     acc = 1u;
                 }
-                if (!p.rider) mma_commit(smem_u32(&sh->empty[s]));  // patch slot free once these MMAs have read it
+                mma_commit(smem_u32(&sh->empty[s]));                // patch slot free once these MMAs (and the rider's) have read it
                 if (!p.bias_in_k) mma_bf16_ss(d_tmem, bias_desc, ones_desc, idesc, 1u);
                 mma_commit(smem_u32(&sh->tmem_full[as]));           // accumulator complete
             }
             __syncwarp();
-            if (++as == 2) { as = 0; aph ^= 1u; }
-            if (p.rider) {
-                // the rider's tile from the same patch, into the other accumulator
-                ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_empty[as]), aph ^ 1u, abort_flag, p.status));
+            if (++as == n_acc) { as = 0; aph ^= 1u; }
+            if (++s == p.stages) { s = 0; ph ^= 1u; }
+        }
+    } else if (warp == POOLT_RIDER_WARP) {
+        // ------------------------------------------------------------------ the rider's MMA issuer
+        // the rider's tile from the same patch (its centre tap), into an accumulator of the rider's own
+        if (p.rider) {
+            const uint32_t idesc = make_idesc_bf16(TILE_M, NPIX, (uint32_t)p.f16);
+            const uint32_t hiX = (uint32_t)(make_kmajor_desc(0, row_bytes, p.sbo_bytes) >> 32);
+            const uint32_t hiW = (uint32_t)(make_kmajor_desc(0, row_bytes, 8u * row_bytes) >> 32);
+            const uint32_t a_tile16 = p.a_tile >> 4, smA16 = smA >> 4, smR16 = (base + p.r_off_b) >> 4;
+            const uint64_t bias_desc = make_kmajor_desc(base + p.r_off_bias, 32u, 256u);
+            const uint64_t ones_desc = make_kmajor_desc(base + p.off_ones, 32u, 256u);
+            bool ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->b_full), 0u, abort_flag, p.status));
+            int s = 0;
+            uint32_t ph = 0;
+            for (int it = 0; it < my_tiles && ok; ++it) {
+                const int ar = 3;
+                const uint32_t aph = (uint32_t)it & 1u;
+                ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_empty[ar]), aph ^ 1u, abort_flag, p.status));
+                if (!ok) break;
+                ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->full[s]), ph, abort_flag, p.status));
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t d2 = tmem_base + (uint32_t)(as * NPIX);
+                const uint32_t d2 = tmem_base + (uint32_t)(ar * NPIX);
+                const uint32_t x_base = smA16 + (uint32_t)s * a_tile16;
                 if (elect_one()) {
-                    const uint32_t smR16 = (base + p.r_off_b) >> 4;
                     uint32_t acc = 0u;
                     for (int e = 0; e < p.r_nmma; ++e) {
                         const uint2 o = p.r_ptab[e];
@@ -810,14 +834,13 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
                                     ((uint64_t)hiX << 32) | (uint64_t)((x_base + o.x) | 0x10000u), idesc, acc);
                         acc = 1u;
                     }
-                    mma_commit(smem_u32(&sh->empty[s]));            // patch slot free once both layers have read it
-                    mma_bf16_ss(d2, make_kmajor_desc(base + p.r_off_bias, 32u, 256u), ones_desc, idesc, 1u);
-                    mma_commit(smem_u32(&sh->tmem_full[as]));
+                    mma_commit(smem_u32(&sh->empty[s]));
+                    mma_bf16_ss(d2, bias_desc, ones_desc, idesc, 1u);
+                    mma_commit(smem_u32(&sh->tmem_full[ar]));
                 }
                 __syncwarp();
-                if (++as == 2) { as = 0; aph ^= 1u; }
+                if (++s == p.stages) { s = 0; ph ^= 1u; }
             }
-            if (++s == p.stages) { s = 0; ph ^= 1u; }
         }
     } else {
         // -------------------------------------------------------------------- epilogue: pool in registers
@@ -827,73 +850,88 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
         const int m = q * 32 + lane;
         const uint32_t lane_base = (uint32_t)(q * 32) << 16;
         const bool live = m < p.Cout, warp_live = q * 32 < p.Cout;
-        const int row_stride = p.PW_out * p.pool_ctot;             // elements between pooled rows
+        const bool warp_full = q * 32 + 32 <= p.Cout && p.relu != 0;      // (and the layer has a ReLU: the common case's stores carry no predicates)
+        const int ctot = CTOT ? CTOT : p.pool_ctot;
+        const int row_stride = p.PW_out * ctot;                    // elements between pooled rows
         float carry[PR][2], carry2[PR][2];              // (carry2: the rider's)
 #pragma unroll
         for (int r = 0; r < PR; ++r) carry[r][0] = carry[r][1] = carry2[r][0] = carry2[r][1] = 0.f;
         bool ok = true;
-        int as = 0;
-        uint32_t aph = 0;
+        int eas = 0;
+        uint32_t eaph = 0;
         TileCoord tc;
         tile_first(p, bid, tc);
-        // one accumulator -> pooled pixels of one layer; `cr` carries the vertical maxima of the tile's last two columns
-        auto pool_tile = [&](float (&cr)[PR][2], const int c_off) {
+        // accumulator `as` -> pooled pixels of one layer; `cr` carries the vertical maxima of the tile's last two columns
+        auto pool_tile = [&](float (&cr)[PR][2], const int c_off, const int as, const uint32_t aph) {
             ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_full[as]), aph, abort_flag, p.status));
             if (!ok) return;
             tc_fence_after();
             const uint32_t taddr = tmem_base + lane_base + (uint32_t)(as * NPIX) + (uint32_t)(grp * 16 * PR);
             const int pw0 = tc.tw * 4 - 1, ph0 = tc.th * PROWS + grp * PR;
             unsigned short* dst0 = reinterpret_cast<unsigned short*>(p.pool_out) +
-                                   (((size_t)tc.ti * p.PH_out + ph0) * p.PW_out + pw0) * p.pool_ctot + c_off + m;
+                                   (((size_t)tc.ti * p.PH_out + ph0) * p.PW_out + pw0) * ctot + c_off + m;
             const bool first = pw0 >= 0 && pw0 < p.PW_out, last3 = pw0 + 3 < p.PW_out, last2 = pw0 + 2 < p.PW_out,
                        last1 = pw0 + 1 < p.PW_out;
-            // ROUNDS rounds of 2*RPR + 1 tile rows (RCOLS accumulator columns) = RPR pooled rows each
+            const bool inner = warp_full && pw0 >= 0 && last3;       // all four pooled columns of the tile exist (the same for the whole warp)
+            // One pooled row per step: its three tile rows are the last row of the step before (still in registers) and
+            // two new ones (16 accumulator columns).  The load of step r + 1 is issued before the maxima of step r are
+            // taken, so that only the first load's latency is exposed; three buffers rotate (the step before, this one,
+            // the one in flight).  The last group has one pooled row -- one step -- fewer.
+            const int nsteps = grp == 3 ? PR - 1 : PR;
+            uint32_t row0[8], buf[3][16];
+            tmem_ld_x8(taddr, row0);
+            tmem_ld_x16(taddr + 8u, buf[0]);
+            tmem_ld_wait_x8(row0);
+            tmem_ld_wait_x16(buf[0]);
+            auto release = [&]() {          // accumulator in registers: hand it back to the MMA issuer
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[as]));
+            };
+            if (nsteps == 1) release();
 #pragma unroll
-            for (int rr = 0; rr < ROUNDS; ++rr) {
-                uint32_t v[RCOLS];
-                if (warp_live) {
-                    const uint32_t ta = taddr + (uint32_t)(16 * RPR * rr);
-                    tmem_ld_x16(ta, *reinterpret_cast<uint32_t(*)[16]>(&v[0]));
-                    tmem_ld_x16(ta + 16u, *reinterpret_cast<uint32_t(*)[16]>(&v[16]));
-                    if (grp < 3 || rr < ROUNDS - 1) tmem_ld_x8(ta + 32u, *reinterpret_cast<uint32_t(*)[8]>(&v[32]));   // (past the
-                                                                             // accumulator for the last group's last round)
-                    tmem_ld_wait();
-                }
-                if (rr == ROUNDS - 1) {
-                    // accumulator in registers: hand it back to the MMA issuer
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[as]));
-                    if (++as == 2) { as = 0; aph ^= 1u; }
-                }
-                if (!warp_live) continue;                               // lanes past the last output layer
+            for (int r = 0; r < PR; ++r) {
+                if (r >= nsteps) break;
+                const bool more = r + 1 < nsteps;
+                if (more) tmem_ld_x16(taddr + 8u + (uint32_t)(16 * (r + 1)), buf[(r + 1) % 3]);
+                const uint32_t* top = r == 0 ? &row0[0] : &buf[(r + 2) % 3][8];         // (row 2r: the last row of the step before)
+                const uint32_t(&cur)[16] = buf[r % 3];
+                float c[8];
 #pragma unroll
-                for (int r2 = 0; r2 < RPR; ++r2) {
-                    const int r = RPR * rr + r2;
-                    if (grp == 3 && r == PR - 1) break;                 // the last group has one pooled row fewer
-                    float c[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j)                         // vertical maximum of rows 2r, 2r+1, 2r+2, column j
-                        c[j] = max3(__uint_as_float(v[16 * r2 + j]), __uint_as_float(v[16 * r2 + 8 + j]),
-                                    __uint_as_float(v[16 * r2 + 16 + j]));
-                    const float o0 = max3(cr[r][0], cr[r][1], c[0]), o1 = max3(c[0], c[1], c[2]),
-                                o2 = max3(c[2], c[3], c[4]), o3 = max3(c[4], c[5], c[6]);
-                    cr[r][0] = c[6];
-                    cr[r][1] = c[7];
-                    if (live && ph0 + r < p.PH_out && sqn_dbg_ok(tc.ti < p.tiles_i && c_off + m < p.pool_ctot, p.status)) {
+                for (int j = 0; j < 8; ++j)                             // vertical maximum of rows 2r, 2r+1, 2r+2, column j
+                    c[j] = max3(__uint_as_float(top[j]), __uint_as_float(cur[j]), __uint_as_float(cur[8 + j]));
+                const float o0 = max3(cr[r][0], cr[r][1], c[0]), o1 = max3(c[0], c[1], c[2]),
+                            o2 = max3(c[2], c[3], c[4]), o3 = max3(c[4], c[5], c[6]);
+                cr[r][0] = c[6];
+                cr[r][1] = c[7];
+                if (inner) {
+                    if (ph0 + r < p.PH_out && sqn_dbg_ok(tc.ti < p.tiles_i && c_off + m < ctot, p.status)) {
+                        // (two values per conversion: a single-value conversion costs the pipe as much as the pair)
                         unsigned short* dst = dst0 + r * row_stride;
-                        if (first) dst[0] = to_16_bits(o0, p.relu, F16);
-                        if (last1) dst[p.pool_ctot] = to_16_bits(o1, p.relu, F16);
-                        if (last2) dst[2 * p.pool_ctot] = to_16_bits(o2, p.relu, F16);
-                        if (last3) dst[3 * p.pool_ctot] = to_16_bits(o3, p.relu, F16);
+                        const uint32_t o01 = pack_relu_x2(o0, o1, F16), o23 = pack_relu_x2(o2, o3, F16);
+                        dst[0] = (unsigned short)(o01 & 0xffffu);
+                        dst[ctot] = (unsigned short)(o01 >> 16);
+                        dst[2 * ctot] = (unsigned short)(o23 & 0xffffu);
+                        dst[3 * ctot] = (unsigned short)(o23 >> 16);
                     }
+                } else if (live && ph0 + r < p.PH_out && sqn_dbg_ok(tc.ti < p.tiles_i && c_off + m < ctot, p.status)) {
+                    unsigned short* dst = dst0 + r * row_stride;
+                    if (first) dst[0] = to_16_bits(o0, p.relu, F16);
+                    if (last1) dst[ctot] = to_16_bits(o1, p.relu, F16);
+                    if (last2) dst[2 * ctot] = to_16_bits(o2, p.relu, F16);
+                    if (last3) dst[3 * ctot] = to_16_bits(o3, p.relu, F16);
+                }
+                if (more) {
+                    tmem_ld_wait_x16(buf[(r + 1) % 3]);
+                    if (r + 2 == nsteps) release();                     // that was the accumulator's last load
                 }
             }
         };
         // (warps whose lanes lie past the last output layer have nothing to do and are not counted by tmem_empty)
         for (int it = 0; it < my_tiles && ok && warp_live; ++it, tile_next(p, tc)) {
-            pool_tile(carry, p.c_off);
-            if (p.rider && ok) pool_tile(carry2, p.r_c_off);
+            pool_tile(carry, p.c_off, eas, eaph);
+            if (++eas == n_acc) { eas = 0; eaph ^= 1u; }
+            if (p.rider && ok) pool_tile(carry2, p.r_c_off, 3, (uint32_t)it & 1u);
         }
     }
 
@@ -906,13 +944,16 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
     }
 }
 
-// (tile size and 16-bit type are compile-time constants of the body)
+// (tile size, 16-bit type and -- for the pooled tensors of SqueezeNet -- the layers per pixel are compile-time constants of the body)
 template <int NPIX>
 __device__ __forceinline__ void pool_body(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB2, const TcParams& p,
                                           const int bid)
 {
-    if (p.f16) conv_pool_body<NPIX, true>(tmA, tmB, tmB2, p, bid);
-    else conv_pool_body<NPIX, false>(tmA, tmB, tmB2, p, bid);
+    if (p.f16) conv_pool_body<NPIX, true, 0>(tmA, tmB, tmB2, p, bid);
+    else if (p.pool_ctot == 256) conv_pool_body<NPIX, false, 256>(tmA, tmB, tmB2, p, bid);
+    else if (NPIX == 256 && p.pool_ctot == 96) conv_pool_body<NPIX, false, 96>(tmA, tmB, tmB2, p, bid);
+    else if (NPIX == 128 && p.pool_ctot == 512) conv_pool_body<NPIX, false, 512>(tmA, tmB, tmB2, p, bid);
+    else conv_pool_body<NPIX, false, 0>(tmA, tmB, tmB2, p, bid);
 }
 
 __global__ void __launch_bounds__(POOLT_THREADS, 1)
@@ -1292,7 +1333,8 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
         // conv_pool_kernel: the kernels are the M = 128 operand; their tiles hold Cout rows and the rows past them
         // belong to whatever follows in shared memory
         p.npix = t_pool_npix;
-        p.tmem_cols = 2 * (unsigned)p.npix;
+        if (p.rider && p.npix != 128) return SQN_ERR_UNSUPPORTED;      // (three accumulators for the layer, one for the rider: 4 x 128 columns)
+        p.tmem_cols = (p.rider ? 4u : 2u) * (unsigned)p.npix;
         p.b_tile = (unsigned)p.BN * row_bytes;
     }
 
@@ -1723,7 +1765,7 @@ int launch_conv_bf16_pool_riders(const ConvDesc* big, const ConvDesc* rider, int
     for (int i = 0; i < n; ++i) {
         if (!big[i].pool || !rider[i].pool) return SQN_ERR_UNSUPPORTED;
         t_rider = &rider[i];
-        int rc = cached_plan(big[i], false, big[i].in, big[i].w, 0, 0, nullptr, &pl[i]);
+        int rc = cached_plan(big[i], false, big[i].in, big[i].w, 0, 0, nullptr, &pl[i], 2, -128);      // (the 128-pixel tiles)
         if (rc == SQN_OK && n == 2 && i == 1 && pl[1].p.npix != pl[0].p.npix)
             rc = SQN_ERR_UNSUPPORTED;
         t_rider = nullptr;

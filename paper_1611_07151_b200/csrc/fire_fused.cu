@@ -53,7 +53,7 @@ constexpr int FF_THREADS = 32 * (FF_W_EEPI + FF_EEPI_WARPS);
 constexpr int FF_MAX_STAGES = 16;
 constexpr int FF_MAX_STG = 4;
 constexpr int FF_MAX_EMMA = 48;            // MMAs of one expand tile: 10 taps x at most 4 k-steps, + spare
-constexpr int FF_MAX_ESLOTS = 3;
+constexpr int FF_MAX_ESLOTS = 4;
 constexpr size_t FF_SMEM_LIMIT = 227 * 1024;
 
 struct FireParams {
@@ -788,14 +788,21 @@ int build_fire_plan(const ConvDesc* dsq, const ConvDesc& d1, const ConvDesc& d3,
         // (or two) accumulators of max(e1p, e3p) columns.
         combined = p.e3p + p.e1p <= 256 && 2 * p.s_slot_cols + 2 * (p.e1p + p.e3p) <= 512 && ((unsigned)p.e3p * p.rb_s) % 256u == 0;
         if (combined) {
-            p.njobs = 1; p.eslots = 2; p.eslot_cols = p.e1p + p.e3p;
+            p.njobs = 1; p.eslot_cols = p.e1p + p.e3p;
         } else {
             p.njobs = 2;
             p.eslot_cols = p.e1p > p.e3p ? p.e1p : p.e3p;
             if (p.eslot_cols > 256) continue;
-            p.eslots = 2 * p.s_slot_cols + 3 * p.eslot_cols <= 512 ? 3 : 2;
-            if (2 * p.s_slot_cols + p.eslots * p.eslot_cols > 512) continue;
         }
+        // as many expand accumulators as the 512 columns hold (up to four): an issuer that finds the next one still
+        // with the epilogue stands idle, and a tile's epilogue is a longer chain of latencies than its MMAs
+        p.eslots = (512 - 2 * p.s_slot_cols) / p.eslot_cols;
+        if (p.eslots > FF_MAX_ESLOTS) p.eslots = FF_MAX_ESLOTS;
+        if (const char* v = std::getenv("SQN_FIRE_ESLOTS")) {          // (tuning aid, read when a plan is built)
+            const int n = std::atoi(v);
+            if (n >= 2 && n < p.eslots) p.eslots = n;
+        }
+        if (p.eslots < 2) continue;
         // two patches with (if there is one) an input ring of 32 KB or more and three slots or more, else one patch
         // under the same condition, else whatever fits
         int cand[8];
@@ -932,7 +939,8 @@ int launch_fire(const ConvDesc* dsq, const ConvDesc& d1, const ConvDesc& d3, cud
     int dev = 0;
     cudaGetDevice(&dev);
     const char* bv = std::getenv("SQN_FIRE_BAND");
-    const int band = bv ? std::atoi(bv) : 0;
+    const char* ev = std::getenv("SQN_FIRE_ESLOTS");
+    const int band = (bv ? std::atoi(bv) : 0) + 1000 * (ev ? std::atoi(ev) : 0);
     const int v[12] = {d1.N, dsq ? dsq->Cin : -1, d1.H, d1.W, d1.Cin, d1.Cout, d3.Cout, d1.out_c_total,
                        (dsq ? dsq->params_static : 0) | (d1.params_static << 1) | (d3.params_static << 2), dev, band, d1.f16};
     std::memcpy(k.v, v, sizeof(v));
