@@ -776,8 +776,11 @@ int build_fire_plan(const ConvDesc* dsq, const ConvDesc& d1, const ConvDesc& d3,
     bool found = false;
     bool combined = false;
     // (first the splits whose parts are whole 64-layer store chunks: half as many chunk hand-overs in the epilogue)
+    const char* csv = std::getenv("SQN_FIRE_CS");           // (tuning aid, read when a plan is built: forces the split)
+    const int force_cs = csv && !dsq ? std::atoi(csv) : 0;
     for (int round = 0; round < 2 && !found; ++round)
     for (int cs = 1; cs <= (dsq ? 1 : 4) && !found; ++cs) {
+        if (force_cs > 0 && cs != force_cs) continue;
         if (e1 % (32 * cs) != 0 || e3 % (32 * cs) != 0) continue;
         p.CS = cs; p.e3p = e3 / cs; p.e1p = e1 / cs;
         p.CW = (p.e3p % 64 == 0 && p.e1p % 64 == 0) ? 64 : 32;
@@ -940,7 +943,8 @@ int launch_fire(const ConvDesc* dsq, const ConvDesc& d1, const ConvDesc& d3, cud
     cudaGetDevice(&dev);
     const char* bv = std::getenv("SQN_FIRE_BAND");
     const char* ev = std::getenv("SQN_FIRE_ESLOTS");
-    const int band = (bv ? std::atoi(bv) : 0) + 1000 * (ev ? std::atoi(ev) : 0);
+    const char* cv = std::getenv("SQN_FIRE_CS");
+    const int band = (bv ? std::atoi(bv) : 0) + 1000 * (ev ? std::atoi(ev) : 0) + 100000 * (cv ? std::atoi(cv) : 0);
     const int v[12] = {d1.N, dsq ? dsq->Cin : -1, d1.H, d1.W, d1.Cin, d1.Cout, d3.Cout, d1.out_c_total,
                        (dsq ? dsq->params_static : 0) | (d1.params_static << 1) | (d3.params_static << 2), dev, band, d1.f16};
     std::memcpy(k.v, v, sizeof(v));
