@@ -106,8 +106,6 @@ struct TcParams {
     int pool_ctot;                   // layers per pixel of the pooled tensor
     __nv_bfloat16* pool_out;
     int npix;                        // conv_pool_kernel: pixels per tile, 256 or 128
-    int n_acc;                       // ... accumulators the layer's tiles take in turn (2, 3 or 4)
-    int two_issuers;                 // ... 1: two warps issue the layer's MMAs, even and odd tiles (the ring then has an even number of slots)
     int f16;                         // 1: the 16-bit type is fp16, 0: bf16
     // conv_pool_kernel: a second layer, 1x1 on the same input with as many output layers, that rides on this layer's
     // patches: after a tile's own MMAs the rider's go into the other accumulator from the same patch, and the epilogue
@@ -634,9 +632,8 @@ conv_tc_kernel2(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
 // groups of four warps take four (two) pooled rows of the strip each, the last group one fewer).  The bias is added by one more MMA (bias rows
 // {hi, lo} x tile of ones).  Lanes past the last output layer compute on whatever follows the kernels in shared
 // memory and are never read.
-constexpr int POOLT_THREADS = 64 + 512 + 64;
+constexpr int POOLT_THREADS = 64 + 512 + 32;
 constexpr int POOLT_RIDER_WARP = 18;           // issues the rider's MMAs (idle without a rider)
-constexpr int POOLT_ISSUER2_WARP = 19;         // second issuer of the layer's own MMAs (128-pixel tiles: it takes the odd tiles)
 __host__ __device__ constexpr int poolt_rows(int npix) { return npix / 8; }                 // output rows per tile
 __host__ __device__ constexpr int poolt_prows(int npix) { return (npix / 8 - 2) / 2; }      // pooled rows per strip
 
@@ -664,7 +661,7 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
     const int items = p.taps * p.chunks;
     const int nmma = items * (p.BKc / 16);
     const int my_tiles = tiles_of_cta(p, bid);
-    const int n_acc = p.n_acc;                      // accumulators of the layer itself
+    const int n_acc = p.rider ? 3 : 2;              // accumulators of the layer itself
     // every kernel tile of the layer (and of its rider), once: one mbarrier counts them all
     auto load_kernels = [&]() {
         const uint32_t bar = smem_u32(&sh->b_full);
@@ -764,14 +761,8 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
                 }
             }
         }
-    } else if (warp == 1 || (warp == POOLT_ISSUER2_WARP && p.two_issuers)) {
-        // ------------------------------------------------------------------ MMA issuer(s)
-        // With 128-pixel tiles an MMA lasts 64 clocks and a tile's hand-shakes cost its issuer as much as several MMAs:
-        // one thread cannot keep the tensor pipe busy, so two warps take the tiles in turn (each keeps count of ring
-        // slot and accumulator of all tiles).  A wait on a barrier must not be two phases ahead of it; with an even
-        // number of ring slots an issuer meets only slots whose previous tile was its own, and the accumulators'
-        // barriers are released in tile order by the epilogue.
-        const int step = p.two_issuers ? 2 : 1, first = warp == 1 ? 0 : 1;
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
         const uint32_t idesc = make_idesc_bf16(TILE_M, NPIX, (uint32_t)p.f16);
         const uint32_t hiX = p.a_lines ? (uint32_t)(make_kmajor_desc_plain(0, 16u, p.sbo_bytes) >> 32)
                                        : (uint32_t)(make_kmajor_desc(0, row_bytes, p.sbo_bytes) >> 32);
@@ -785,9 +776,9 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
         // (MMA drain, the epilogue's wake-up and TMEM loads, the way back) is about as long as two such tiles' MMAs.
         // The rider's MMAs are issued by a warp of their own: with 64 clocks per MMA issuing, not the tensor pipe, is
         // what a single thread is bound by.
-        int s = first, as = first;              // (two issuers: at least two ring slots and two accumulators)
+        int s = 0, as = 0;
         uint32_t ph = 0, aph = 0;
-        for (int it = first; it < my_tiles && ok; it += step) {
+        for (int it = 0; it < my_tiles && ok; ++it) {
             ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_empty[as]), aph ^ 1u, abort_flag, p.status));
             if (!ok) break;
             ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->full[s]), ph, abort_flag, p.status));
@@ -809,10 +800,8 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
                 mma_commit(smem_u32(&sh->tmem_full[as]));           // accumulator complete
             }
             __syncwarp();
-            as += step;
-            if (as >= n_acc) { as -= n_acc; aph ^= 1u; }
-            s += step;
-            if (s >= p.stages) { s -= p.stages; ph ^= 1u; }
+            if (++as == n_acc) { as = 0; aph ^= 1u; }
+            if (++s == p.stages) { s = 0; ph ^= 1u; }
         }
     } else if (warp == POOLT_RIDER_WARP) {
         // ------------------------------------------------------------------ the rider's MMA issuer
@@ -853,7 +842,7 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
                 if (++s == p.stages) { s = 0; ph ^= 1u; }
             }
         }
-    } else if (warp < POOLT_RIDER_WARP) {
+    } else {
         // -------------------------------------------------------------------- epilogue: pool in registers
         // group g = (warp - 2) / 4 takes the pooled rows PR*g .. PR*g + PR-1 of the strip (group 3: one fewer), i.e.
         // the rows 2*PR*g .. 2*PR*g + 2*PR of the tile = accumulator columns 16*PR*g .. 16*PR*g + 16*PR + 7
@@ -1271,8 +1260,6 @@ bool pool_layout(TcParams& p, size_t a_tile, size_t* smem_bytes)
     if (t_smem_limit < fixed + 2 * a_tile) return false;
     size_t stages = (t_smem_limit - fixed) / a_tile;
     if (stages > MAX_STAGES) stages = MAX_STAGES;
-    p.two_issuers = p.npix == 128 ? 1 : 0;
-    if (p.two_issuers) stages &= ~(size_t)1;        // (an even number of ring slots: see the issuers)
     // the 128-row read of the last kernel tile must stay inside the patch ring
     if ((size_t)TILE_M * p.BKc * 2 > p.b_tile + stages * a_tile) return false;
     p.stages = (int)stages;
@@ -1347,8 +1334,7 @@ int build_plan_cfg(const ConvDesc& d, bool stem, const void* a_ptr, const void* 
         // belong to whatever follows in shared memory
         p.npix = t_pool_npix;
         if (p.rider && p.npix != 128) return SQN_ERR_UNSUPPORTED;      // (three accumulators for the layer, one for the rider: 4 x 128 columns)
-        p.n_acc = p.npix == 128 ? (p.rider ? 3 : 4) : 2;
-        p.tmem_cols = 512;
+        p.tmem_cols = (p.rider ? 4u : 2u) * (unsigned)p.npix;
         p.b_tile = (unsigned)p.BN * row_bytes;
     }
 
