@@ -457,8 +457,8 @@ def run_variants(B, batch):
                       "alternating two buffer sets, median of 3 such runs, microseconds; a missing variant does not fit the layer"}))
 
 
-def run_kernel_case(B, name, batch, steps):
-    """One layer (or fire layer, or the fused head) of the network on its own, bf16, seed-4 recipe drawn on the device:
+def run_kernel_case(B, name, batch, steps, dtype="bf16"):
+    """One layer (or fire layer, or the fused head) of the network on its own (bf16 / f16 / f32), seed-4 recipe drawn on the device:
     `steps` back-to-back launches over rotating buffer sets larger than the L2 (mean), then single launches with the L2
     overwritten in between (median).  The small cases of the ncu captures under profiles/ are runs of this mode."""
     import torch
@@ -466,7 +466,9 @@ def run_kernel_case(B, name, batch, steps):
     torch.cuda.set_device(0)
     gen = torch.Generator(device=dev)
     gen.manual_seed(4)
-    bf = torch.bfloat16
+    bf = {"bf16": torch.bfloat16, "f16": torch.float16, "f32": torch.float32}[dtype]
+    code = {"bf16": B.SQN_BF16, "f16": B.SQN_F16, "f32": B.SQN_F32}[dtype]
+    es = 4 if dtype == "f32" else 2
     convs = {n: (cin, cout, k, s, pad, hw) for n, cin, cout, k, s, pad, hw in synth.SQUEEZENET_CONVS}
 
     def conv_params(cin, cout, k):
@@ -480,7 +482,7 @@ def run_kernel_case(B, name, batch, steps):
         wsq, bsq = conv_params(cin, s_, 1)
         w1, b1 = conv_params(s_, e, 1)
         w3, b3 = conv_params(s_, e, 3)
-        per_set = batch * hw * hw * (cin + s_ + 2 * e) * 2
+        per_set = batch * hw * hw * (cin + s_ + 2 * e) * es
         nsets = max(2, int(200e6 // per_set) + 1)
         for _ in range(nsets):
             sets.append((torch.rand((batch, hw, hw, cin), device=dev, generator=gen).to(bf),
@@ -488,19 +490,19 @@ def run_kernel_case(B, name, batch, steps):
 
         def call(i):
             x, sc, out = sets[i % nsets]
-            B.fire_forward(x, wsq, bsq, w1, b1, w3, b3, sc, out, cin, s_, e, e, hw, hw, batch, B.SQN_BF16)
+            B.fire_forward(x, wsq, bsq, w1, b1, w3, b3, sc, out, cin, s_, e, e, hw, hw, batch, code)
         flops = 2.0 * batch * hw * hw * (cin * s_ + 10 * s_ * e)
-        byts = 2.0 * batch * hw * hw * (cin + 2 * e)
+        byts = float(es) * batch * hw * hw * (cin + 2 * e)
     else:
         base = name.split("+")[0]
         cin, cout, k, s_, pad, hw = convs[base]
         pool, avg = name.endswith("+pool") or name.endswith("+pool1"), name.endswith("+avgpool")
         oh = (hw + 2 * pad - k) // s_ + 1
         w, b = conv_params(cin, cout, k)
-        nb = B.conv_workspace_bytes(cin, cout, hw, hw, k, s_, pad, batch, B.SQN_BF16)
+        nb = B.conv_workspace_bytes(cin, cout, hw, hw, k, s_, pad, batch, code)
         po = (oh - 3) // 2 + 1
         out_shape = (batch, cout) if avg else ((batch, po, po, cout) if pool else (batch, oh, oh, cout))
-        per_set = batch * hw * hw * cin * 2 + int(np.prod(out_shape)) * 2
+        per_set = batch * hw * hw * cin * es + int(np.prod(out_shape)) * es
         nsets = max(2, int(200e6 // per_set) + 1)
         for _ in range(nsets):
             sets.append((torch.rand((batch, hw, hw, cin), device=dev, generator=gen).to(bf),
@@ -509,10 +511,10 @@ def run_kernel_case(B, name, batch, steps):
 
         def call(i):
             x, out, wsb = sets[i % nsets]
-            B.conv_forward_ex(x, w, b, out, cin, cout, hw, hw, k, s_, pad, batch, dtype=B.SQN_BF16, workspace=wsb,
+            B.conv_forward_ex(x, w, b, out, cin, cout, hw, hw, k, s_, pad, batch, dtype=code, workspace=wsb,
                               workspace_bytes=nb, fuse_maxpool=pool, fuse_global_avgpool=avg)
         flops = 2.0 * batch * oh * oh * cout * cin * k * k
-        byts = 2.0 * batch * hw * hw * cin + (4.0 if avg else 2.0) * float(np.prod(out_shape))
+        byts = float(es) * batch * hw * hw * cin + (4.0 if avg else float(es)) * float(np.prod(out_shape))
     for i in range(5):
         call(i)
     torch.cuda.synchronize()
@@ -535,9 +537,9 @@ def run_kernel_case(B, name, batch, steps):
         singles.append(a.elapsed_time(c) * 1e3)
     assert B.sqn_check() == B.SQN_OK
     peaks = measured_peaks()
-    print(json.dumps({"kernel_case": name, "batch": batch, "steps": steps, "us_mean_back_to_back": mean_us,
+    print(json.dumps({"kernel_case": name, "dtype": dtype, "batch": batch, "steps": steps, "us_mean_back_to_back": mean_us,
                       "us_median_single_cold": float(np.median(singles)), "tflops": flops / mean_us / 1e6,
-                      "gbs": byts / mean_us / 1e3, "frac_tensor_burst": flops / mean_us / 1e6 / peaks["bf16_tflops"],
+                      "gbs": byts / mean_us / 1e3, ("frac_ffma_peak" if dtype == "f32" else "frac_tensor_burst"): flops / mean_us / 1e6 / (fp32_ffma_peak_tflops(torch.cuda.get_device_properties(0).multi_processor_count, 1965) if dtype == "f32" else peaks["bf16_tflops"]),
                       "frac_hbm": byts / mean_us / 1e3 / peaks["hbm_gbs"], "buffer_sets": nsets}))
 
 
@@ -582,7 +584,7 @@ def main():
         run_variants(B, args.batch)
         return
     if args.kernel:
-        run_kernel_case(B, args.kernel, args.batch, args.steps)
+        run_kernel_case(B, args.kernel, args.batch, args.steps, args.dtype)
         return
     if args.mma_rate:
         rows = []

@@ -108,8 +108,8 @@ struct TcParams {
     int npix;                        // conv_pool_kernel: pixels per tile, 256 or 128
     int f16;                         // 1: the 16-bit type is fp16, 0: bf16
     // conv_pool_kernel: a second layer, 1x1 on the same input with as many output layers, that rides on this layer's
-    // patches: after a tile's own MMAs the rider's go into the other accumulator from the same patch, and the epilogue
-    // pools both (the 1x1 expand of a fire layer beside the 3x3 expand)
+    // patches: its MMAs read the centre of the same patch and fill an accumulator of their own, and the epilogue pools
+    // both (the 1x1 expand of a fire layer beside the 3x3 expand)
     int rider;
     int r_nmma;                      // the rider's MMAs per tile
     unsigned r_off_b, r_off_bias;    // its kernels (chunks tiles of Cout rows) and bias rows in shared memory
@@ -629,9 +629,13 @@ conv_tc_kernel2(const __grid_constant__ CUtensorMap tmA0, const __grid_constant_
 // A CTA walks a strip of 32 output rows (strips 30 rows apart: 15 pooled rows) from left to right; tile k emits the
 // pooled columns 4k-1 .. 4k+2, the vertical maxima of its last two columns are carried to tile k+1 in registers.
 // Warps: 0 TMA producer, 1 MMA issuer, 18 the rider's MMA issuer, 2..17 epilogue (lane quadrant = warp % 4; the four
-// groups of four warps take four (two) pooled rows of the strip each, the last group one fewer).  The bias is added by one more MMA (bias rows
-// {hi, lo} x tile of ones).  Lanes past the last output layer compute on whatever follows the kernels in shared
-// memory and are never read.
+// groups of four warps take four (128-pixel tiles: two) pooled rows of the strip each, the last group one fewer).
+// The bias is added by one more MMA (bias rows {hi, lo} x tile of ones).  Lanes past the last output layer compute on
+// whatever follows the kernels in shared memory and are never read.
+// With a rider (a 1x1 layer on the same input) the tiles are 128 pixels: the layer's tiles take three accumulators of
+// 128 columns in turn, the rider's the fourth, and the rider's MMAs come from a warp of their own -- with one thread
+// issuing both, and one accumulator for the layer, the layer's MMAs, its pooling and the rider's MMAs ran one after
+// the other (fire4 + pool4: 84 us; 75 us so).
 constexpr int POOLT_THREADS = 64 + 512 + 32;
 constexpr int POOLT_RIDER_WARP = 18;           // issues the rider's MMAs (idle without a rider)
 __host__ __device__ constexpr int poolt_rows(int npix) { return npix / 8; }                 // output rows per tile
