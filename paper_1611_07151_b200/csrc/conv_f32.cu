@@ -30,9 +30,10 @@ struct F32Params {
 
 __host__ __device__ constexpr int ld_for(int bn) { return bn <= 32 ? 32 : (bn <= 64 ? 64 : 128); }
 
-// Column permutation applied to row k of a transposed tile so that the four k-groups a warp
-// stores at once land in different banks.  Keeps groups of 8 columns intact.
-__device__ __forceinline__ int swz(int k) { return ((k >> 2) & 3) << 3; }
+// Rows of the transposed tiles are padded by PADF floats: the compute loop then reads them at addresses that differ
+// from a per-thread base by compile-time offsets only (no index arithmetic between the FFMAs), and the four k-groups a
+// warp stores at once fall into two banks' worth of conflicts at most (the stores are 1.5 % of the instructions).
+constexpr int PADF = 4;
 
 template <int BM, int BN, int VN, int QN, bool VEC>
 __global__ void __launch_bounds__(NTHREADS, 2) conv_f32_kernel(const F32Params p)
@@ -45,8 +46,8 @@ __global__ void __launch_bounds__(NTHREADS, 2) conv_f32_kernel(const F32Params p
     static_assert(TX * TN == BN && TY * TM == BM, "tile shape");
     constexpr int LDB = ld_for(BN);
 
-    __shared__ __align__(16) float As[2][BK][BM];
-    __shared__ __align__(16) float Bs[2][BK][LDB];
+    __shared__ __align__(16) float As[2][BK][BM + PADF];
+    __shared__ __align__(16) float Bs[2][BK][LDB + PADF];
     __shared__ int tbl_off[VEC ? 1 : TBL_MAX];
     __shared__ int tbl_hw[VEC ? 1 : TBL_MAX];
 
@@ -175,10 +176,9 @@ __global__ void __launch_bounds__(NTHREADS, 2) conv_f32_kernel(const F32Params p
     auto store_tile = [&](int buf) {
         if (VEC) {
             const int k4 = tid & 3;
-            const int s = k4 << 3;   // swz(4*k4 + i) for i < 4
 #pragma unroll
             for (int j = 0; j < A_LOADS; ++j) {
-                const int row = ((tid >> 2) + 64 * j) ^ s;
+                const int row = (tid >> 2) + 64 * j;
                 As[buf][4 * k4 + 0][row] = ra4[j].x;
                 As[buf][4 * k4 + 1][row] = ra4[j].y;
                 As[buf][4 * k4 + 2][row] = ra4[j].z;
@@ -188,7 +188,7 @@ __global__ void __launch_bounds__(NTHREADS, 2) conv_f32_kernel(const F32Params p
             for (int j = 0; j < B_LOADS_V; ++j) {
                 const int n = (tid >> 2) + 64 * j;
                 if (n < BN) {
-                    const int col = n ^ s;
+                    const int col = n;
                     Bs[buf][4 * k4 + 0][col] = rb4[j].x;
                     Bs[buf][4 * k4 + 1][col] = rb4[j].y;
                     Bs[buf][4 * k4 + 2][col] = rb4[j].z;
@@ -202,13 +202,13 @@ __global__ void __launch_bounds__(NTHREADS, 2) conv_f32_kernel(const F32Params p
 #pragma unroll
             for (int j = 0; j < A_LOADS; ++j) {
                 const int kk = kk0 + KSTEP * j;
-                As[buf][kk][row ^ swz(kk)] = ra1[j];
+                As[buf][kk][row] = ra1[j];
             }
             const int kk = tid & 15;
 #pragma unroll
             for (int j = 0; j < B_LOADS_S; ++j) {
                 const int n = (tid >> 4) + 16 * j;
-                Bs[buf][kk][n ^ swz(kk)] = rb1[j];
+                Bs[buf][kk][n] = rb1[j];
             }
         }
     };
@@ -230,16 +230,15 @@ __global__ void __launch_bounds__(NTHREADS, 2) conv_f32_kernel(const F32Params p
 
 #pragma unroll
         for (int kk = 0; kk < BK; ++kk) {
-            const int s = swz(kk);
             float a[TM], b[TN];
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
-                const float4 v = *reinterpret_cast<const float4*>(&As[buf][kk][(q * (BM / 2) + ty * 4) ^ s]);
+                const float4 v = *reinterpret_cast<const float4*>(&As[buf][kk][q * (BM / 2) + ty * 4]);
                 a[4 * q + 0] = v.x; a[4 * q + 1] = v.y; a[4 * q + 2] = v.z; a[4 * q + 3] = v.w;
             }
 #pragma unroll
             for (int q = 0; q < QN; ++q) {
-                const int cb = (q * (BN / QN) + tx * VN) ^ s;
+                const int cb = q * (BN / QN) + tx * VN;
                 if (VN == 4) {
                     const float4 v = *reinterpret_cast<const float4*>(&Bs[buf][kk][cb]);
                     b[q * VN + 0] = v.x; b[q * VN + 1] = v.y; b[q * VN + 2] = v.z; b[q * VN + 3] = v.w;
