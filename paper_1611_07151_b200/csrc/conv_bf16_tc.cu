@@ -106,6 +106,7 @@ struct TcParams {
     int pool_ctot;                   // layers per pixel of the pooled tensor
     __nv_bfloat16* pool_out;
     int npix;                        // conv_pool_kernel: pixels per tile, 256 or 128
+    int two_issuers;                 // ... 1 (no rider): warp 18 issues the odd tiles' MMAs (the ring then has an even number of slots)
     int f16;                         // 1: the 16-bit type is fp16, 0: bf16
     // conv_pool_kernel: a second layer, 1x1 on the same input with as many output layers, that rides on this layer's
     // patches: its MMAs read the centre of the same patch and fill an accumulator of their own, and the epilogue pools
@@ -765,8 +766,15 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
                 }
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
+    } else if (warp == 1 || (warp == POOLT_RIDER_WARP && p.two_issuers)) {
+        // ------------------------------------------------------------------ MMA issuer(s)
+        // Between a tile's last MMA and the next tile's first the issuing thread spends some 500 clocks on barriers,
+        // fences and commits, more than the tensor pipe's queue holds: without a rider the warp that would issue the
+        // rider's MMAs takes the odd tiles, so that one thread's hand-shakes fall into the other's MMAs.  Each issuer
+        // keeps count of ring slot and accumulator of all tiles.  A wait on a barrier must not be two phases ahead of
+        // it: with an even number of ring slots and two accumulators an issuer only meets slots and accumulators whose
+        // previous tile was its own.
+        const int step = p.two_issuers ? 2 : 1, first = warp == 1 ? 0 : 1;
         const uint32_t idesc = make_idesc_bf16(TILE_M, NPIX, (uint32_t)p.f16);
         const uint32_t hiX = p.a_lines ? (uint32_t)(make_kmajor_desc_plain(0, 16u, p.sbo_bytes) >> 32)
                                        : (uint32_t)(make_kmajor_desc(0, row_bytes, p.sbo_bytes) >> 32);
@@ -780,9 +788,9 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
         // (MMA drain, the epilogue's wake-up and TMEM loads, the way back) is about as long as two such tiles' MMAs.
         // The rider's MMAs are issued by a warp of their own: with 64 clocks per MMA issuing, not the tensor pipe, is
         // what a single thread is bound by.
-        int s = 0, as = 0;
+        int s = first, as = first;              // (two issuers: at least two ring slots, two accumulators)
         uint32_t ph = 0, aph = 0;
-        for (int it = 0; it < my_tiles && ok; ++it) {
+        for (int it = first; it < my_tiles && ok; it += step) {
             ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->tmem_empty[as]), aph ^ 1u, abort_flag, p.status));
             if (!ok) break;
             ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->full[s]), ph, abort_flag, p.status));
@@ -804,8 +812,10 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
                 mma_commit(smem_u32(&sh->tmem_full[as]));           // accumulator complete
             }
             __syncwarp();
-            if (++as == n_acc) { as = 0; aph ^= 1u; }
-            if (++s == p.stages) { s = 0; ph ^= 1u; }
+            as += step;
+            if (as >= n_acc) { as -= n_acc; aph ^= 1u; }
+            s += step;
+            if (s >= p.stages) { s -= p.stages; ph ^= 1u; }
         }
     } else if (warp == POOLT_RIDER_WARP) {
         // ------------------------------------------------------------------ the rider's MMA issuer
@@ -846,7 +856,7 @@ __device__ __forceinline__ void conv_pool_body(const CUtensorMap& tmA, const CUt
                 if (++s == p.stages) { s = 0; ph ^= 1u; }
             }
         }
-    } else {
+    } else if (warp < POOLT_RIDER_WARP) {
         // -------------------------------------------------------------------- epilogue: pool in registers
         // group g = (warp - 2) / 4 takes the pooled rows PR*g .. PR*g + PR-1 of the strip (group 3: one fewer), i.e.
         // the rows 2*PR*g .. 2*PR*g + 2*PR of the tile = accumulator columns 16*PR*g .. 16*PR*g + 16*PR + 7
@@ -1264,6 +1274,9 @@ bool pool_layout(TcParams& p, size_t a_tile, size_t* smem_bytes)
     if (t_smem_limit < fixed + 2 * a_tile) return false;
     size_t stages = (t_smem_limit - fixed) / a_tile;
     if (stages > MAX_STAGES) stages = MAX_STAGES;
+    p.two_issuers = p.rider ? 0 : 1;
+    if (const char* v = std::getenv("SQN_POOL_ISSUERS")) p.two_issuers = (!p.rider && std::atoi(v) == 2) ? 1 : 0;      // (tuning aid, read when a plan is built)
+    if (p.two_issuers) stages &= ~(size_t)1;        // (an even number of ring slots: see the issuers)
     // the 128-row read of the last kernel tile must stay inside the patch ring
     if ((size_t)TILE_M * p.BKc * 2 > p.b_tile + stages * a_tile) return false;
     p.stages = (int)stages;
