@@ -69,7 +69,7 @@ struct FireParams {
     int f16;                         // 1: the 16-bit type is fp16, 0: bf16
     int stages, nstg;
     int s_issuers;                   // squeeze issuer warps at work: 2 where the input ring holds two tiles' chunks, else 1
-    int two_patches;
+    int npatch;                      // patches in shared memory: 1, 2, or (flat expands, where they fit) 3
     // expand jobs of a tile: one (both expands in one accumulator) or two (3x3, then 1x1)
     int njobs;
     int job_e0[2], job_en[2];        // the job's MMAs: entries [e0, en) of etab
@@ -105,7 +105,7 @@ struct FireShared {
     unsigned long long w_full;
     unsigned long long s_full[2], s_empty[2];
     unsigned long long e_full[FF_MAX_ESLOTS], e_empty[FF_MAX_ESLOTS];
-    unsigned long long patch_ready[2], patch_free[2];
+    unsigned long long patch_ready[4], patch_free[4];
     unsigned long long stg_full[FF_MAX_STG];
     unsigned long long stg_free[FF_MAX_STG];
     unsigned tmem_base;
@@ -174,7 +174,7 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     // CTA -> (part of the output layers, first band); it walks the bands bid, bid + gstep, ...
     const int part = (int)blockIdx.x % p.CS;
     const int bid = (int)blockIdx.x / p.CS, gstep = p.grid / p.CS;
-    const int nbuf = p.two_patches ? 2 : 1;
+    const int nbuf = p.npatch;
 
     auto load_kernels = [&]() {          // every kernel tile of the layer (this CTA's part of it), once; one mbarrier counts them all
         const uint32_t bar = smem_u32(&sh->w_full);
@@ -208,6 +208,8 @@ fire_fused_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&sh->s_full[a]), 1);
             mbar_init(smem_u32(&sh->s_empty[a]), FF_SEPI_WARPS);
+        }
+        for (int a = 0; a < 4; ++a) {
             mbar_init(smem_u32(&sh->patch_ready[a]), p.src_tma ? 1 : FF_SEPI_WARPS);
             mbar_init(smem_u32(&sh->patch_free[a]), FF_ISSUERS);
         }
@@ -609,7 +611,7 @@ int fire_layout(FireParams& p, int R, int patches, int BKc_in, size_t* smem_byte
     p.R = R;
     p.NB = (H + R - 1) / R;
     p.items = p.N * p.NB;
-    p.two_patches = patches == 2 ? 1 : 0;
+    p.npatch = patches;
     size_t cur = 0;
     p.w_bytes = 0;
     p.off_wsq = 0;
@@ -810,9 +812,13 @@ int build_fire_plan(const ConvDesc* dsq, const ConvDesc& d1, const ConvDesc& d3,
         // under the same condition, else whatever fits
         int cand[8];
         const int nc = band_candidates(H, p.RT, N, Cin, s, e1 + e3, cand);
+        // (flat expands: a third patch first -- the box of band j + 2 can only be requested once band j's MMAs are
+        // done, and with two patches the request's latency shows in the issuers' waits; SQN_FIRE_PATCHES=2 tuning aid)
+        const char* pv = std::getenv("SQN_FIRE_PATCHES");
+        const int max_patches = !dsq ? (pv && std::atoi(pv) >= 2 && std::atoi(pv) <= 4 ? std::atoi(pv) : 3) : 2;
         for (int pass = 0; pass < 3 && !found; ++pass)
             for (int i = 0; i < nc && !found; ++i)
-                for (int patches = (pass == 1 ? 1 : 2); patches >= (pass == 0 ? 2 : 1) && !found; --patches)
+                for (int patches = (pass == 1 ? 1 : max_patches); patches >= (pass == 0 ? 2 : 1) && !found; --patches)
                     for (int bk = 64; bk >= 32 && !found; bk -= 32) {
                         if (dsq && Cin % bk != 0) continue;
                         if (!dsq && bk != 64) continue;
@@ -944,7 +950,8 @@ int launch_fire(const ConvDesc* dsq, const ConvDesc& d1, const ConvDesc& d3, cud
     const char* bv = std::getenv("SQN_FIRE_BAND");
     const char* ev = std::getenv("SQN_FIRE_ESLOTS");
     const char* cv = std::getenv("SQN_FIRE_CS");
-    const int band = (bv ? std::atoi(bv) : 0) + 1000 * (ev ? std::atoi(ev) : 0) + 100000 * (cv ? std::atoi(cv) : 0);
+    const char* pv = std::getenv("SQN_FIRE_PATCHES");
+    const int band = (bv ? std::atoi(bv) : 0) + 1000 * (ev ? std::atoi(ev) : 0) + 100000 * (cv ? std::atoi(cv) : 0) + 1000000 * (pv ? std::atoi(pv) : 0);
     const int v[12] = {d1.N, dsq ? dsq->Cin : -1, d1.H, d1.W, d1.Cin, d1.Cout, d3.Cout, d1.out_c_total,
                        (dsq ? dsq->params_static : 0) | (d1.params_static << 1) | (d3.params_static << 2), dev, band, d1.f16};
     std::memcpy(k.v, v, sizeof(v));
