@@ -1264,6 +1264,8 @@ bool choose_layout(TcParams& p, size_t a_tile, bool want_resident, int min_stage
 // Shared memory of conv_pool_kernel: the layer's kernels (tiles of Cout rows; an MMA reads 128 rows from a tile's
 // start, the rows past Cout come from the tiles and patches behind it), the patch ring, bias rows, the tile of ones,
 // the control block.
+int pool_issuers_env();
+
 bool pool_layout(TcParams& p, size_t a_tile, size_t* smem_bytes)
 {
     const size_t items = (size_t)p.taps * p.chunks;
@@ -1275,7 +1277,7 @@ bool pool_layout(TcParams& p, size_t a_tile, size_t* smem_bytes)
     size_t stages = (t_smem_limit - fixed) / a_tile;
     if (stages > MAX_STAGES) stages = MAX_STAGES;
     p.two_issuers = p.rider ? 0 : 1;
-    if (const char* v = std::getenv("SQN_POOL_ISSUERS")) p.two_issuers = (!p.rider && std::atoi(v) == 2) ? 1 : 0;      // (tuning aid, read when a plan is built)
+    if (pool_issuers_env() == 1) p.two_issuers = 0;
     if (p.two_issuers) stages &= ~(size_t)1;        // (an even number of ring slots: see the issuers)
     // the 128-row read of the last kernel tile must stay inside the patch ring
     if ((size_t)TILE_M * p.BKc * 2 > p.b_tile + stages * a_tile) return false;
@@ -1641,6 +1643,14 @@ struct PlanKey {
 std::mutex g_plan_mu;
 std::map<std::string, Plan> g_plans;
 
+// SQN_POOL_ISSUERS in the environment (tuning aid: 1 or 2 issuer warps for a pooled convolution without a rider), 0 if unset
+int pool_issuers_env()
+{
+    const char* v = std::getenv("SQN_POOL_ISSUERS");
+    const int n = v ? std::atoi(v) : 0;
+    return n == 1 || n == 2 ? n : 0;
+}
+
 // force_halves / force_cw != 0: the plan of that kernel variant (CTAs per SM, store chunk width) instead of the
 // layer's own best one, so that it can share a launch with another layer's plan.
 int cached_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_ptr, int Hp, int Wp, const void* ws,
@@ -1651,7 +1661,7 @@ int cached_plan(const ConvDesc& d, bool stem, const void* a_ptr, const void* w_p
     k.in = d.in; k.w = d.w; k.bias = d.bias; k.out = d.out; k.ws = ws;
     if (t_rider) { k.rw = t_rider->w; k.rbias = t_rider->bias; k.r_c_off = t_rider->out_c_offset + 1; }
     const int v[14] = {d.N, d.Cin, d.H, d.W, d.Cout, d.K, d.S, d.pad, d.out_c_offset, d.out_c_total, d.relu | (d.pool << 1) | (d.params_static << 2) | (d.stem_prepacked << 3) | (d.f16 << 4),
-                       (stem ? 1 : 0) | (force_halves << 4) | ((force_cw & 0xffff) << 8), Hp, Wp};
+                       (stem ? 1 : 0) | (force_halves << 4) | ((force_cw & 0xffff) << 8) | (pool_issuers_env() << 24), Hp, Wp};
     std::memcpy(k.v, v, sizeof(v));
     int dev = 0;
     cudaGetDevice(&dev);

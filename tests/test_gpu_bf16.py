@@ -420,6 +420,28 @@ def test_forced_kernel_variants_give_the_same_values():
     assert ran >= 6
 
 
+def test_one_or_two_issuer_warps_give_the_same_pooled_values():
+    """SQN_POOL_ISSUERS: a pooled convolution without a rider has its MMAs issued by one warp or by two taking the
+    tiles in turn; the pooled map must not depend on it (a stem-shaped and a 3x3 layer, several strips per CTA)."""
+    import os
+    old = os.environ.get("SQN_POOL_ISSUERS")
+    try:
+        for (N, C, M, H, K, S, pad) in [(40, 3, 96, 227, 7, 2, 0), (80, 32, 128, 55, 3, 1, 1)]:
+            rng = np.random.default_rng(N + C + M)
+            x = synth.draw_input(rng, (N, C, H, H))
+            w, b = synth.draw_conv_params(rng, C, M, K)
+            outs = []
+            for n in ("1", "2"):
+                os.environ["SQN_POOL_ISSUERS"] = n
+                outs.append(G.gpu_conv(x, w, b, S, pad, True, BF16, fuse_maxpool=True))
+            np.testing.assert_array_equal(outs[0], outs[1])
+    finally:
+        if old is None:
+            os.environ.pop("SQN_POOL_ISSUERS", None)
+        else:
+            os.environ["SQN_POOL_ISSUERS"] = old
+
+
 @pytest.mark.parametrize("batch", [2, 20])
 def test_stem_operands_packed_offline_give_the_same_logits(batch):
     """squeezenet_set_stem_prepacked: the forward reads [228][228][4] images and [96][7][8][4] kernels written by the

@@ -163,3 +163,42 @@ def test_expands_many_bands_per_cta():
     got, launches, _ = _run(x, sq, x1, x3)
     assert launches == 2
     _check(got, exp, e)
+
+
+def test_tuning_knobs_of_the_flat_expands_give_the_same_values():
+    """SQN_FIRE_PATCHES (patches in shared memory), SQN_FIRE_CS (split of the output layers over CTAs) and
+    SQN_FIRE_ESLOTS (expand accumulators) only change how the flat expand kernel is scheduled: every number of patches
+    and accumulators that fits must give exactly the values of the library's own choice, every split the same values up
+    to the rounding of the output (more bands than CTAs, so that patches are reused)."""
+    x, sq, x1, x3 = _fire_case(61, 70, 384, 48, 192, 192, 27, 27)
+    knobs = ("SQN_FIRE_PATCHES", "SQN_FIRE_CS", "SQN_FIRE_ESLOTS")
+    old = {k: os.environ.get(k) for k in knobs}
+    ran = 0
+    try:
+        for k in knobs:
+            os.environ.pop(k, None)
+        want, launches, _ = _run(x, sq, x1, x3)
+        assert launches == 2
+        for knob, values in (("SQN_FIRE_PATCHES", (2, 3, 4)), ("SQN_FIRE_CS", (2, 3, 4)), ("SQN_FIRE_ESLOTS", (2, 3))):
+            for v in values:
+                os.environ[knob] = str(v)
+                try:
+                    got, launches, _ = _run(x, sq, x1, x3)
+                finally:
+                    os.environ.pop(knob, None)
+                if launches != 2:           # (the setting does not fit: the layer ran on other kernels)
+                    continue
+                if knob == "SQN_FIRE_CS":
+                    # another split adds the taps' products in another order (the 1x1 expand rides on the centre tap
+                    # or is a job of its own): equal up to the rounding of the stored value
+                    assert G.rel_err(got, want) <= 1e-2, (knob, v)
+                else:
+                    np.testing.assert_array_equal(got, want, err_msg="%s=%d" % (knob, v))
+                ran += 1
+    finally:
+        for k, v in old.items():
+            if v is None:
+                os.environ.pop(k, None)
+            else:
+                os.environ[k] = v
+    assert ran >= 5
